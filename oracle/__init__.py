@@ -1,0 +1,228 @@
+"""CPU oracle for the Rollout-ResQ FP4 linear layer -- TEST INFRASTRUCTURE ONLY.
+
+A thin ctypes wrapper over ``resq_oracle.c`` (plain scalar C, fp64).  Only the
+tests, the smoke check and the benchmark's cpu-baseline leg may import this
+package; the CUDA library never does, and shares no code with it.
+
+The C file states which passage of the paper each function follows and which
+choices are readings of this project (the paper fixes the HiF4 field widths but
+not the group sizes, bias, scale rule or packing: those are "parity unpinned").
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Dict, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "resq_oracle.c")
+_LIB = os.path.join(_HERE, "libresq_oracle.so")
+
+S_NONE, S_DENSE, S_2_4, S_ROW50, S_CHAN50, S_BLOCK = 0, 1, 2, 3, 4, 5
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain -O2, OpenMP over rows)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
+                               "-ffp-contract=off", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        i64, dbl, vp, ci = ctypes.c_int64, ctypes.c_double, ctypes.c_void_p, ctypes.c_int
+        for name in ("oracle_hif4_e6m2_value", "oracle_hif4_s1p2_value", "oracle_e2m1_value", "oracle_e8m0_value"):
+            getattr(L, name).restype = dbl
+            getattr(L, name).argtypes = [ci]
+        L.oracle_hif4_encode.argtypes = [vp, i64, i64, vp, vp]
+        L.oracle_hif4_decode.argtypes = [vp, vp, i64, i64, vp]
+        L.oracle_mxfp4_encode.argtypes = [vp, i64, i64, vp, vp]
+        L.oracle_mxfp4_decode.argtypes = [vp, vp, i64, i64, vp]
+        L.oracle_residual.argtypes = [vp, vp, i64, vp]
+        L.oracle_residual.restype = i64
+        L.oracle_mask.argtypes = [vp, i64, i64, ci, vp, vp, vp]
+        L.oracle_apply_mask.argtypes = [vp, vp, i64, i64, vp]
+        L.oracle_apply_mask.restype = None
+        L.oracle_matmul.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
+        L.oracle_matmul.restype = None
+        _lib = L
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f32(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    assert x.ndim == 2
+    return x
+
+
+# ------------------------------------------------------------------ formats
+
+def e6m2_value(s: int) -> float:
+    return float(lib().oracle_hif4_e6m2_value(int(s)))
+
+
+def s1p2_value(code: int) -> float:
+    return float(lib().oracle_hif4_s1p2_value(int(code)))
+
+
+def e2m1_value(code: int) -> float:
+    return float(lib().oracle_e2m1_value(int(code)))
+
+
+def e8m0_value(code: int) -> float:
+    return float(lib().oracle_e8m0_value(int(code)))
+
+
+def hif4_encode(x: np.ndarray):
+    """x float32 [rows,K] -> (codes uint8 [rows,K/2], meta uint32 [rows,K/64])."""
+    x = _f32(x)
+    rows, K = x.shape
+    codes = np.empty((rows, K // 2), dtype=np.uint8)
+    meta = np.empty((rows, K // 64), dtype=np.uint32)
+    rc = lib().oracle_hif4_encode(_p(x), rows, K, _p(codes), _p(meta))
+    if rc:
+        raise ValueError("HiF4 needs K % 64 == 0")
+    return codes, meta
+
+
+def hif4_decode(codes: np.ndarray, meta: np.ndarray) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    meta = np.ascontiguousarray(meta, dtype=np.uint32)
+    rows, K = codes.shape[0], codes.shape[1] * 2
+    out = np.empty((rows, K), dtype=np.float64)
+    rc = lib().oracle_hif4_decode(_p(codes), _p(meta), rows, K, _p(out))
+    if rc:
+        raise ValueError("HiF4 needs K % 64 == 0")
+    return out
+
+
+def mxfp4_encode(x: np.ndarray):
+    """x float32 [rows,K] -> (codes uint8 [rows,K/2], scale uint8 [rows,K/32])."""
+    x = _f32(x)
+    rows, K = x.shape
+    codes = np.empty((rows, K // 2), dtype=np.uint8)
+    scale = np.empty((rows, K // 32), dtype=np.uint8)
+    rc = lib().oracle_mxfp4_encode(_p(x), rows, K, _p(codes), _p(scale))
+    if rc:
+        raise ValueError("MXFP4 needs K % 32 == 0")
+    return codes, scale
+
+
+def mxfp4_decode(codes: np.ndarray, scale: np.ndarray) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    scale = np.ascontiguousarray(scale, dtype=np.uint8)
+    rows, K = codes.shape[0], codes.shape[1] * 2
+    out = np.empty((rows, K), dtype=np.float64)
+    rc = lib().oracle_mxfp4_decode(_p(codes), _p(scale), rows, K, _p(out))
+    if rc:
+        raise ValueError("MXFP4 needs K % 32 == 0")
+    return out
+
+
+def encode(fmt: str, x: np.ndarray):
+    return hif4_encode(x) if fmt == "hif4" else mxfp4_encode(x)
+
+
+def decode(fmt: str, codes: np.ndarray, side: np.ndarray) -> np.ndarray:
+    return hif4_decode(codes, side) if fmt == "hif4" else mxfp4_decode(codes, side)
+
+
+# ------------------------------------------------------------------ residual, masks, product
+
+def residual(x: np.ndarray, deq: np.ndarray) -> np.ndarray:
+    """Eq. (3): x - deq(Q(x)), returned as float32; raises if any difference is not fp32-exact."""
+    x = _f32(x)
+    deq = np.ascontiguousarray(deq, dtype=np.float64)
+    dx = np.empty_like(x)
+    bad = lib().oracle_residual(_p(x), _p(deq), x.size, _p(dx))
+    if bad:
+        raise ArithmeticError(f"{bad} residual elements are not exact in fp32")
+    return dx
+
+
+def mask(v: np.ndarray, pattern: int, want_scores: bool = False):
+    """Selection S on the decoded quantized residual v [M,K] -> (mask_bits uint8 [M,K/8], info dict)."""
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    M, K = v.shape
+    bits = np.empty((M, K // 8), dtype=np.uint8)
+    info = np.zeros(2, dtype=np.float64)
+    scores = None
+    if want_scores and pattern == S_CHAN50:
+        scores = np.zeros(K, dtype=np.float64)
+    if want_scores and pattern == S_BLOCK:
+        scores = np.zeros((M // 32) * (K // 64), dtype=np.float64)
+    rc = lib().oracle_mask(_p(v), M, K, int(pattern), _p(bits), _p(info), _p(scores))
+    if rc == -1:
+        raise ValueError("shape not valid for this pattern")
+    if rc == -2:
+        raise ValueError("unknown pattern")
+    return bits, {"exact": bool(info[0]), "margin": float(info[1]), "scores": scores}
+
+
+def apply_mask(r: np.ndarray, bits: np.ndarray) -> np.ndarray:
+    r = np.ascontiguousarray(r, dtype=np.float64)
+    bits = np.ascontiguousarray(bits, dtype=np.uint8)
+    out = np.empty_like(r)
+    lib().oracle_apply_mask(_p(r), _p(bits), r.shape[0], r.shape[1], _p(out))
+    return out
+
+
+def matmul(a: np.ndarray, r: Optional[np.ndarray], w: np.ndarray, want_abs: bool = True):
+    """Eq. (5) on decoded operands: a@w.T + r@w.T in fp64 -> (y [M,N], abs_sum [M,N] or None)."""
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    if r is not None:
+        r = np.ascontiguousarray(r, dtype=np.float64)
+    M, K = a.shape
+    N = w.shape[0]
+    assert w.shape[1] == K
+    y = np.empty((M, N), dtype=np.float64)
+    ab = np.empty((M, N), dtype=np.float64) if want_abs else None
+    lib().oracle_matmul(_p(a), _p(r), _p(w), M, N, K, _p(y), _p(ab))
+    return y, ab
+
+
+def quantize_residual_mask(x_f32: np.ndarray, pattern: int, fmt: str = "hif4") -> Dict[str, np.ndarray]:
+    """Steps Q(X), Eq. (3), Q(dX), S(.) in the paper's order."""
+    x_f32 = _f32(x_f32)
+    x_codes, x_side = encode(fmt, x_f32)
+    a = decode(fmt, x_codes, x_side)
+    out = {"x_codes": x_codes, "x_side": x_side, "a": a}
+    if pattern == S_NONE:
+        return out
+    dx = residual(x_f32, a)
+    r_codes, r_side = encode(fmt, dx)
+    r = decode(fmt, r_codes, r_side)
+    bits, info = mask(r, pattern)
+    out.update({"dx": dx, "r_codes": r_codes, "r_side": r_side, "r": r, "mask": bits,
+                "mask_info": info, "r_masked": apply_mask(r, bits)})
+    return out
+
+
+def resq_linear(x_f32: np.ndarray, w_f32: np.ndarray, pattern: int, fmt: str = "hif4",
+                want_abs: bool = True) -> Dict[str, np.ndarray]:
+    """The whole path: pack W, quantize X, residual, mask, two-term product."""
+    out = quantize_residual_mask(x_f32, pattern, fmt)
+    w_codes, w_side = encode(fmt, _f32(w_f32))
+    w = decode(fmt, w_codes, w_side)
+    y, ab = matmul(out["a"], out.get("r_masked"), w, want_abs)
+    out.update({"w_codes": w_codes, "w_side": w_side, "w": w, "y": y, "abs_sum": ab})
+    return out

@@ -1,0 +1,425 @@
+/*
+ * CPU oracle for the Rollout-ResQ FP4 linear layer.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the slow, plain statement of what the hot path computes; the CUDA
+ * library is checked against it and shares no code with it.  Only the tests, the
+ * smoke check and the benchmark's cpu-baseline leg may call it.
+ *
+ * What it follows (paper sections / equations):
+ *   - HiF4 format: Section 3, "Block-Scaled Quantization": blocks of 64, a first
+ *     level E6M2 scaler, E1 scalers at levels two and three, S1P2 (= E1M2)
+ *     elements.  The paper fixes no more than that; every further choice
+ *     (sub-group sizes 8 and 4, exponent bias 48, how the scales are derived,
+ *     rounding, tie rules, bit packing) is a reading of this project and is a
+ *     named constant or a short rule below.  PARITY UNPINNED by the paper for:
+ *     HIF4_E6M2_BIAS, HIF4_L2_GROUP, HIF4_L3_GROUP, the "smallest scale that does
+ *     not clip" rule, tie-breaks, the orientation of the 32x64 block and the
+ *     global top-k of the block/channel patterns.
+ *   - MXFP4 format: Section 3: blocks of 32, E8M0 scale, E2M1 elements; scale and
+ *     rounding rule follow the open microscaling convention (floor(log2 amax)
+ *     minus the element format's largest exponent, round-to-nearest-even,
+ *     saturate).
+ *   - Residual: Eq. (3)  dX = X - Q(X).
+ *   - Dense correction: Eq. (4)  Y = Q(X)Q(W)^T + Q(dX)Q(W)^T.
+ *   - Sparse correction: Eq. (5) Y = Q(X)Q(W)^T + S(Q(dX))Q(W)^T with S one of
+ *     S_2:4, S_50% (channel-wise by L2 norm, Section 4.3 item (1); and a per-row
+ *     variant the benchmark configuration asks for), S^{32x64}_50% (item (3)),
+ *     identity (Rollout-ResQ-Dense) or none (Eq. (1)).
+ *
+ * Arithmetic is fp64 and exact wherever the quantities are dyadic rationals
+ * (all encoder decisions are exact comparisons); only the final dot products
+ * round (fp64).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define HIF4_BLOCK 64
+#define HIF4_L2_GROUP 8   /* elements per level-2 scaler  [reading] */
+#define HIF4_L3_GROUP 4   /* elements per level-3 scaler  [reading] */
+#define HIF4_E6M2_BIAS 48 /* S1 = (1 + Mn/4) * 2^(E - 48)  [reading] */
+#define MXFP4_BLOCK 32
+#define MX_E8M0_BIAS 127
+
+enum { S_NONE = 0, S_DENSE = 1, S_2_4 = 2, S_ROW50 = 3, S_CHAN50 = 4, S_BLOCK32x64 = 5 };
+#define BLK_ROWS 32
+#define BLK_COLS 64
+
+/* ---------------------------------------------------------------- tables */
+
+/* E6M2 code s = E<<2 | Mn  ->  (1 + Mn/4) * 2^(E - bias).  All 256 codes are values. */
+double oracle_hif4_e6m2_value(int s) {
+    int E = (s >> 2) & 63, Mn = s & 3;
+    return ldexp(1.0 + Mn / 4.0, E - HIF4_E6M2_BIAS);
+}
+
+/* S1P2 magnitude: sign + 1 integer bit + 2 fraction bits, q in 0..7 -> q/4
+ * (the same eight values as E1M2 with bias 1: 0, .25, .5, .75, 1, 1.25, 1.5, 1.75). */
+double oracle_hif4_s1p2_value(int code) {
+    int q = code & 7;
+    double v = q / 4.0;
+    return (code & 8) ? -v : v;
+}
+
+static const double E2M1_GRID[8] = {0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0};
+
+double oracle_e2m1_value(int code) {
+    double v = E2M1_GRID[code & 7];
+    return (code & 8) ? -v : v;
+}
+
+/* E8M0: 2^(code - 127); code 255 is NaN in the format and never produced here. */
+double oracle_e8m0_value(int code) { return ldexp(1.0, code - MX_E8M0_BIAS); }
+
+/* ---------------------------------------------------------------- HiF4 */
+
+/* Encode one block of 64 values.  code[k] = sign<<3 | q.
+ * meta: bits 7:0 = s (E6M2), bit 8+i = e2[i] (i = 0..7), bit 16+j = e3[j] (j = 0..15). */
+static void hif4_encode_block(const double *x, uint8_t *code, uint32_t *meta_out) {
+    double amax = 0.0;
+    for (int k = 0; k < HIF4_BLOCK; ++k) {
+        double a = fabs(x[k]);
+        if (a > amax) amax = a;
+    }
+    /* level 1: the smallest scale whose largest representable magnitude, 1.75 * 2 * 2 * S1 = 7 S1,
+     * still covers the block maximum (no clipping); 255 if none does; 0 for an all-zero block. */
+    int s = 0;
+    if (amax > 0.0) {
+        s = 255;
+        for (int c = 0; c < 256; ++c) {
+            if (7.0 * oracle_hif4_e6m2_value(c) >= amax) { s = c; break; }
+        }
+    }
+    double S1 = oracle_hif4_e6m2_value(s);
+    uint32_t meta = (uint32_t)s;
+    int e2[HIF4_BLOCK / HIF4_L2_GROUP], e3[HIF4_BLOCK / HIF4_L3_GROUP];
+    /* level 2: raise the group of 8 only if it would clip with e2 = 0 (and e3 = 1). */
+    for (int i = 0; i < HIF4_BLOCK / HIF4_L2_GROUP; ++i) {
+        double gmax = 0.0;
+        for (int k = 0; k < HIF4_L2_GROUP; ++k) {
+            double a = fabs(x[i * HIF4_L2_GROUP + k]);
+            if (a > gmax) gmax = a;
+        }
+        e2[i] = (gmax > 3.5 * S1) ? 1 : 0;
+        meta |= (uint32_t)e2[i] << (8 + i);
+    }
+    /* level 3: raise the group of 4 only if it would clip at its level-2 scale. */
+    for (int j = 0; j < HIF4_BLOCK / HIF4_L3_GROUP; ++j) {
+        int i = (j * HIF4_L3_GROUP) / HIF4_L2_GROUP;
+        double gmax = 0.0;
+        for (int k = 0; k < HIF4_L3_GROUP; ++k) {
+            double a = fabs(x[j * HIF4_L3_GROUP + k]);
+            if (a > gmax) gmax = a;
+        }
+        e3[j] = (gmax > 1.75 * S1 * ldexp(1.0, e2[i])) ? 1 : 0;
+        meta |= (uint32_t)e3[j] << (16 + j);
+    }
+    /* elements: nearest multiple of step in 0..7 steps, ties to the even count. */
+    for (int k = 0; k < HIF4_BLOCK; ++k) {
+        double step = S1 * ldexp(1.0, e2[k / HIF4_L2_GROUP] + e3[k / HIF4_L3_GROUP]) / 4.0;
+        double a = fabs(x[k]);
+        int q = 0;
+        for (int c = 0; c < 7; ++c) {
+            double mid = (2 * c + 1) * step / 2.0; /* exact: small integer times a dyadic */
+            if (a > mid || (a == mid && (c & 1))) q = c + 1;
+        }
+        code[k] = (uint8_t)((signbit(x[k]) ? 8 : 0) | q);
+    }
+    *meta_out = meta;
+}
+
+static void hif4_decode_block(const uint8_t *code, uint32_t meta, double *v) {
+    double S1 = oracle_hif4_e6m2_value((int)(meta & 0xFF));
+    for (int k = 0; k < HIF4_BLOCK; ++k) {
+        int e2 = (meta >> (8 + k / HIF4_L2_GROUP)) & 1;
+        int e3 = (meta >> (16 + k / HIF4_L3_GROUP)) & 1;
+        v[k] = oracle_hif4_s1p2_value(code[k]) * ldexp(1.0, e2 + e3) * S1;
+    }
+}
+
+/* Packed layout: codes[row][k/2], element 2j in bits 3:0 and 2j+1 in bits 7:4;
+ * meta[row][K/64] as uint32.  Returns 0, or -1 if K is not a multiple of 64. */
+int oracle_hif4_encode(const float *x, int64_t rows, int64_t K, uint8_t *codes, uint32_t *meta) {
+    if (K % HIF4_BLOCK) return -1;
+    int64_t G = K / HIF4_BLOCK;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t b = 0; b < G; ++b) {
+            double xb[HIF4_BLOCK];
+            uint8_t cb[HIF4_BLOCK];
+            for (int k = 0; k < HIF4_BLOCK; ++k) xb[k] = (double)x[r * K + b * HIF4_BLOCK + k];
+            hif4_encode_block(xb, cb, &meta[r * G + b]);
+            for (int k = 0; k < HIF4_BLOCK; k += 2)
+                codes[r * (K / 2) + (b * HIF4_BLOCK + k) / 2] = (uint8_t)(cb[k] | (cb[k + 1] << 4));
+        }
+    }
+    return 0;
+}
+
+int oracle_hif4_decode(const uint8_t *codes, const uint32_t *meta, int64_t rows, int64_t K, double *out) {
+    if (K % HIF4_BLOCK) return -1;
+    int64_t G = K / HIF4_BLOCK;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t b = 0; b < G; ++b) {
+            uint8_t cb[HIF4_BLOCK];
+            for (int k = 0; k < HIF4_BLOCK; k += 2) {
+                uint8_t byte = codes[r * (K / 2) + (b * HIF4_BLOCK + k) / 2];
+                cb[k] = byte & 15;
+                cb[k + 1] = byte >> 4;
+            }
+            hif4_decode_block(cb, meta[r * G + b], &out[r * K + b * HIF4_BLOCK]);
+        }
+    }
+    return 0;
+}
+
+/* ---------------------------------------------------------------- MXFP4 */
+
+static void mxfp4_encode_block(const double *x, uint8_t *code, uint8_t *scale_out) {
+    double amax = 0.0;
+    for (int k = 0; k < MXFP4_BLOCK; ++k) {
+        double a = fabs(x[k]);
+        if (a > amax) amax = a;
+    }
+    int e = -MX_E8M0_BIAS; /* all-zero block: scale code 0 */
+    if (amax > 0.0) {
+        int ex;
+        (void)frexp(amax, &ex);  /* amax = f * 2^ex, f in [0.5, 1)  =>  floor(log2 amax) = ex - 1 */
+        e = (ex - 1) - 2;        /* 2 = exponent of the largest E2M1 value, 6 = 1.5 * 2^2 */
+        if (e < -MX_E8M0_BIAS) e = -MX_E8M0_BIAS;
+        if (e > MX_E8M0_BIAS) e = MX_E8M0_BIAS;
+    }
+    *scale_out = (uint8_t)(e + MX_E8M0_BIAS);
+    for (int k = 0; k < MXFP4_BLOCK; ++k) {
+        double t = ldexp(fabs(x[k]), -e); /* exact */
+        int idx = 0;
+        for (int c = 0; c < 7; ++c) {
+            double mid = (E2M1_GRID[c] + E2M1_GRID[c + 1]) / 2.0;
+            if (t > mid || (t == mid && (c & 1))) idx = c + 1; /* tie -> even code; above 6 stays 7 */
+        }
+        code[k] = (uint8_t)((signbit(x[k]) ? 8 : 0) | idx);
+    }
+}
+
+int oracle_mxfp4_encode(const float *x, int64_t rows, int64_t K, uint8_t *codes, uint8_t *scale) {
+    if (K % MXFP4_BLOCK) return -1;
+    int64_t G = K / MXFP4_BLOCK;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t b = 0; b < G; ++b) {
+            double xb[MXFP4_BLOCK];
+            uint8_t cb[MXFP4_BLOCK];
+            for (int k = 0; k < MXFP4_BLOCK; ++k) xb[k] = (double)x[r * K + b * MXFP4_BLOCK + k];
+            mxfp4_encode_block(xb, cb, &scale[r * G + b]);
+            for (int k = 0; k < MXFP4_BLOCK; k += 2)
+                codes[r * (K / 2) + (b * MXFP4_BLOCK + k) / 2] = (uint8_t)(cb[k] | (cb[k + 1] << 4));
+        }
+    }
+    return 0;
+}
+
+int oracle_mxfp4_decode(const uint8_t *codes, const uint8_t *scale, int64_t rows, int64_t K, double *out) {
+    if (K % MXFP4_BLOCK) return -1;
+    int64_t G = K / MXFP4_BLOCK;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t k = 0; k < K; ++k) {
+            uint8_t byte = codes[r * (K / 2) + k / 2];
+            int c = (k & 1) ? (byte >> 4) : (byte & 15);
+            out[r * K + k] = oracle_e2m1_value(c) * oracle_e8m0_value(scale[r * G + k / MXFP4_BLOCK]);
+        }
+    }
+    return 0;
+}
+
+/* ---------------------------------------------------------------- residual, Eq. (3) */
+
+/* dx = x - deq(Q(x)) in fp64, stored as fp32.  Returns the number of elements whose
+ * difference is NOT exactly an fp32 value (expected 0 for bf16 inputs). */
+int64_t oracle_residual(const float *x, const double *deq, int64_t n, float *dx) {
+    int64_t inexact = 0;
+#pragma omp parallel for schedule(static) reduction(+ : inexact)
+    for (int64_t i = 0; i < n; ++i) {
+        double d = (double)x[i] - deq[i];
+        float f = (float)d;
+        if ((double)f != d) ++inexact;
+        dx[i] = f;
+    }
+    return inexact;
+}
+
+/* ---------------------------------------------------------------- masks S(.) */
+
+typedef struct { double key; int64_t idx; } keyed_t;
+
+/* larger key first; equal keys: lower index first */
+static int cmp_keyed(const void *pa, const void *pb) {
+    const keyed_t *a = (const keyed_t *)pa, *b = (const keyed_t *)pb;
+    if (a->key > b->key) return -1;
+    if (a->key < b->key) return 1;
+    return (a->idx < b->idx) ? -1 : (a->idx > b->idx);
+}
+
+static void set_bit(uint8_t *mask, int64_t K, int64_t m, int64_t k) {
+    mask[m * (K / 8) + (k >> 3)] |= (uint8_t)(1u << (k & 7));
+}
+
+/* Sum of squares with an exactness check (error-free two-sum): *exact is cleared
+ * if any partial sum rounded. */
+static double sumsq_add(double acc, double v, int *exact) {
+    double t = v * v; /* exact for the decoded grids: <= 12-bit significand */
+    double s = acc + t;
+    double bb = s - acc;
+    double err = (acc - (s - bb)) + (t - bb);
+    if (err != 0.0) *exact = 0;
+    return s;
+}
+
+/* v: decoded Q(dX) [M,K].  mask_bits[m][k>>3] bit (k&7) = kept.
+ * info[0] = 1 if all score sums were exact in fp64 (channel/block patterns), else 0;
+ * info[1] = relative gap between the last kept and first dropped score (channel/block), else 0.
+ * scores (optional, may be NULL): K channel scores or (M/32)*(K/64) block scores.
+ * Returns 0, -1 on a shape error, -2 on an unknown pattern. */
+int oracle_mask(const double *v, int64_t M, int64_t K, int pattern, uint8_t *mask_bits, double *info,
+                double *scores_out) {
+    if (K % 8) return -1;
+    memset(mask_bits, 0, (size_t)(M * (K / 8)));
+    info[0] = 1.0;
+    info[1] = 0.0;
+    switch (pattern) {
+    case S_NONE:
+        return 0;
+    case S_DENSE:
+        memset(mask_bits, 0xFF, (size_t)(M * (K / 8)));
+        return 0;
+    case S_2_4: {
+        /* Section 4.3 item (2): keep the 2 largest magnitudes of every 4 contiguous elements. */
+        if (K % 4) return -1;
+        for (int64_t m = 0; m < M; ++m)
+            for (int64_t g = 0; g < K / 4; ++g) {
+                keyed_t e[4];
+                for (int t = 0; t < 4; ++t) {
+                    e[t].key = fabs(v[m * K + 4 * g + t]);
+                    e[t].idx = t;
+                }
+                qsort(e, 4, sizeof(keyed_t), cmp_keyed);
+                set_bit(mask_bits, K, m, 4 * g + e[0].idx);
+                set_bit(mask_bits, K, m, 4 * g + e[1].idx);
+            }
+        return 0;
+    }
+    case S_ROW50: {
+        /* per row, the K/2 largest magnitudes (the benchmark configuration's wording of S_50%). */
+        keyed_t *e = (keyed_t *)malloc(sizeof(keyed_t) * (size_t)K);
+        for (int64_t m = 0; m < M; ++m) {
+            for (int64_t k = 0; k < K; ++k) {
+                e[k].key = fabs(v[m * K + k]);
+                e[k].idx = k;
+            }
+            qsort(e, (size_t)K, sizeof(keyed_t), cmp_keyed);
+            for (int64_t t = 0; t < K / 2; ++t) set_bit(mask_bits, K, m, e[t].idx);
+        }
+        free(e);
+        return 0;
+    }
+    case S_CHAN50: {
+        /* Section 4.3 item (1): keep the half of the channels (columns) with the largest L2 norm. */
+        keyed_t *e = (keyed_t *)malloc(sizeof(keyed_t) * (size_t)K);
+        int exact = 1;
+        for (int64_t k = 0; k < K; ++k) {
+            double acc = 0.0;
+            for (int64_t m = 0; m < M; ++m) acc = sumsq_add(acc, v[m * K + k], &exact);
+            e[k].key = acc;
+            e[k].idx = k;
+            if (scores_out) scores_out[k] = acc;
+        }
+        qsort(e, (size_t)K, sizeof(keyed_t), cmp_keyed);
+        int64_t keep = K / 2;
+        for (int64_t t = 0; t < keep; ++t)
+            for (int64_t m = 0; m < M; ++m) set_bit(mask_bits, K, m, e[t].idx);
+        info[0] = exact;
+        if (keep > 0 && keep < K && e[keep - 1].key > 0.0)
+            info[1] = (e[keep - 1].key - e[keep].key) / e[keep - 1].key;
+        free(e);
+        return 0;
+    }
+    case S_BLOCK32x64: {
+        /* Section 4.3 item (3): 32 token rows x 64 channels per block; keep the half of all
+         * blocks of the tensor with the largest L2 norm. */
+        if (M % BLK_ROWS || K % BLK_COLS) return -1;
+        int64_t nbr = M / BLK_ROWS, nbc = K / BLK_COLS, nb = nbr * nbc;
+        keyed_t *e = (keyed_t *)malloc(sizeof(keyed_t) * (size_t)nb);
+        int exact = 1;
+        for (int64_t a = 0; a < nbr; ++a)
+            for (int64_t b = 0; b < nbc; ++b) {
+                double acc = 0.0;
+                for (int64_t i = 0; i < BLK_ROWS; ++i)
+                    for (int64_t j = 0; j < BLK_COLS; ++j)
+                        acc = sumsq_add(acc, v[(a * BLK_ROWS + i) * K + b * BLK_COLS + j], &exact);
+                e[a * nbc + b].key = acc;
+                e[a * nbc + b].idx = a * nbc + b;
+                if (scores_out) scores_out[a * nbc + b] = acc;
+            }
+        qsort(e, (size_t)nb, sizeof(keyed_t), cmp_keyed);
+        int64_t keep = nb / 2;
+        for (int64_t t = 0; t < keep; ++t) {
+            int64_t a = e[t].idx / nbc, b = e[t].idx % nbc;
+            for (int64_t i = 0; i < BLK_ROWS; ++i)
+                for (int64_t j = 0; j < BLK_COLS; ++j) set_bit(mask_bits, K, a * BLK_ROWS + i, b * BLK_COLS + j);
+        }
+        info[0] = exact;
+        if (keep > 0 && keep < nb && e[keep - 1].key > 0.0)
+            info[1] = (e[keep - 1].key - e[keep].key) / e[keep - 1].key;
+        free(e);
+        return 0;
+    }
+    default:
+        return -2;
+    }
+}
+
+/* r_masked = mask ? r : 0 */
+void oracle_apply_mask(const double *r, const uint8_t *mask_bits, int64_t M, int64_t K, double *out) {
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t k = 0; k < K; ++k) {
+            int kept = (mask_bits[m * (K / 8) + (k >> 3)] >> (k & 7)) & 1;
+            out[m * K + k] = kept ? r[m * K + k] : 0.0;
+        }
+}
+
+/* ---------------------------------------------------------------- product, Eq. (5) */
+
+/* y[m][n] = sum_k a[m][k] w[n][k]  +  sum_k r[m][k] w[n][k]   (r may be NULL: Eq. (1)).
+ * abs_sum (optional) = sum_k |(a + r)[m][k] * w[n][k]|, the cancellation floor used by
+ * the tolerance.  a, r: [M,K]; w: [N,K]; y: [M,N]. */
+void oracle_matmul(const double *a, const double *r, const double *w, int64_t M, int64_t N, int64_t K, double *y,
+                   double *abs_sum) {
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        for (int64_t n = 0; n < N; ++n) {
+            double main_term = 0.0, res_term = 0.0, as = 0.0;
+            for (int64_t k = 0; k < K; ++k) main_term += a[m * K + k] * w[n * K + k];
+            if (r)
+                for (int64_t k = 0; k < K; ++k) res_term += r[m * K + k] * w[n * K + k];
+            y[m * N + n] = main_term + res_term;
+            if (abs_sum) {
+                for (int64_t k = 0; k < K; ++k) {
+                    double t = a[m * K + k] + (r ? r[m * K + k] : 0.0);
+                    as += fabs(t * w[n * K + k]);
+                }
+                abs_sum[m * N + n] = as;
+            }
+        }
+    }
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

@@ -1,0 +1,570 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked without a GPU.
+
+Each test is chosen so that a plausible mistake in the oracle (dropped term, wrong sign or
+index, transposed operand, wrong tie rule) fails at least one of them.  Nothing here retypes
+the oracle's own loops: properties are stated independently (exact rationals, brute force,
+library routines, hand-derived values).
+"""
+import itertools
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+from workloads import bf16_bits_to_f32, f32_to_bf16_bits
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+F = Fraction
+
+
+def nibbles(codes):
+    c = np.asarray(codes, dtype=np.uint8)
+    return np.stack([c & 15, c >> 4], axis=-1).reshape(c.shape[0], -1)
+
+
+def bf16_round(x):
+    return bf16_bits_to_f32(f32_to_bf16_bits(np.asarray(x, dtype=np.float32)))
+
+
+def gaussian_with_outliers(seed, rows, K, n_out=4, scale=64.0):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((rows, K)).astype(np.float32)
+    ch = rng.choice(K, n_out, replace=False)
+    x[:, ch] *= scale
+    return bf16_round(x)
+
+
+# ----------------------------------------------------------------- tables (Section 3)
+
+def test_s1p2_equals_e1m2_table():
+    # E1M2 with bias 1: exponent bit 0 -> subnormal 0.mm, exponent bit 1 -> 1.mm (times 2^0)
+    for code in range(16):
+        e, m = (code >> 2) & 1, code & 3
+        mag = F(m, 4) if e == 0 else 1 + F(m, 4)
+        want = -mag if code & 8 else mag
+        assert F(oracle.s1p2_value(code)) == want
+    assert [oracle.s1p2_value(q) for q in range(8)] == [0, .25, .5, .75, 1, 1.25, 1.5, 1.75]
+
+
+def test_e6m2_table_structure():
+    vals = [F(oracle.e6m2_value(s)) for s in range(256)]
+    assert all(b > a for a, b in zip(vals, vals[1:]))            # codes are monotone in value
+    assert vals[48 << 2] == 1                                    # bias 48
+    for s in range(256):
+        E, Mn = s >> 2, s & 3
+        assert vals[s] == F(4 + Mn, 4) * F(2) ** (E - 48)
+    assert vals[0] == F(2) ** -48 and vals[255] == F(7, 4) * 2 ** 15
+
+
+def test_e2m1_e8m0_tables_match_library(nvref):
+    for c in range(16):
+        assert oracle.e2m1_value(c) == nvref.nv_e2m1_to_float(c)
+        assert np.signbit(oracle.e2m1_value(c)) == bool(c & 8)
+    for c in range(255):
+        assert oracle.e8m0_value(c) == nvref.nv_e8m0_to_float(c)
+
+
+def test_e8m0_table_matches_torch():
+    import torch
+    b = torch.arange(255, dtype=torch.uint8)
+    v = b.view(torch.float8_e8m0fnu).to(torch.float32).numpy()
+    assert all(oracle.e8m0_value(c) == float(v[c]) for c in range(255))
+
+
+# ----------------------------------------------------------------- golden worked example
+
+def _load_worked_example():
+    rows, mask, mx, meta = [], None, [], {}
+    with open(os.path.join(GOLD, "hif4_worked_example.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if not line:
+                continue
+            t = line.split()
+            if t[0] in ("meta_x", "meta_r"):
+                meta[t[0]] = int(t[1], 16)
+            elif t[0] == "mask":
+                mask = [int(v, 16) for v in t[1:]]
+            elif t[0] == "mx_scale":
+                meta["mx_scale"] = [int(v) for v in t[1:]]
+            elif t[0] == "mx":
+                mx.append((int(t[1]), int(t[2])))
+            else:
+                rows.append((int(t[0]), float(t[1]), int(t[2]), float(t[3]), float(t[4]), int(t[5]), float(t[6])))
+    return rows, mask, mx, meta
+
+
+def test_worked_example_hif4_residual_mask():
+    rows, mask, mx, meta = _load_worked_example()
+    x = np.zeros((1, 64), dtype=np.float32)
+    for k, xv, *_ in rows:
+        x[0, k] = xv
+    out = oracle.quantize_residual_mask(x, oracle.S_2_4)
+    assert int(out["x_side"][0, 0]) == meta["meta_x"]
+    assert int(out["r_side"][0, 0]) == meta["meta_r"]
+    qx, qr = nibbles(out["x_codes"])[0], nibbles(out["r_codes"])[0]
+    listed = set()
+    for k, xv, cx, dqx, dx, cr, dqr in rows:
+        listed.add(k)
+        assert qx[k] == cx, k
+        assert out["a"][0, k] == dqx and np.signbit(out["a"][0, k]) == np.signbit(dqx)
+        assert out["dx"][0, k] == dx
+        assert qr[k] == cr, k
+        assert out["r"][0, k] == dqr
+    for k in range(64):
+        if k not in listed:
+            assert qx[k] == 0 and qr[k] == 0
+    assert list(out["mask"][0]) == mask
+
+
+def test_worked_example_mxfp4():
+    rows, mask, mx, meta = _load_worked_example()
+    x = np.zeros((1, 64), dtype=np.float32)
+    for k, xv, *_ in rows:
+        x[0, k] = xv
+    codes, scale = oracle.mxfp4_encode(x)
+    assert list(scale[0]) == meta["mx_scale"]
+    q = nibbles(codes)[0]
+    for k, c in mx:
+        assert q[k] == c, k
+
+
+# ----------------------------------------------------------------- HiF4 invariants (exact rationals)
+
+def _hif4_check_block(xb, cb, meta):
+    """No-clip, minimality and nearest-with-ties-to-even, stated as properties over exact rationals."""
+    s = meta & 255
+    S1 = F(4 + (s & 3), 4) * F(2) ** ((s >> 2) - 48)
+    ax = [abs(F(float(v))) for v in xb]
+    amax = max(ax)
+    if amax == 0:
+        assert s == 0
+    else:
+        if s < 255:
+            assert 7 * S1 >= amax                                   # level 1 does not clip
+        if s > 0:
+            sp = s - 1
+            assert 7 * F(4 + (sp & 3), 4) * F(2) ** ((sp >> 2) - 48) < amax   # ... and is minimal
+    for i in range(8):
+        e2 = (meta >> (8 + i)) & 1
+        g8 = max(ax[8 * i: 8 * i + 8])
+        # e2 = 0 would allow at most 1.75 * 2 * S1 (with e3 = 1)
+        assert (e2 == 1) == (g8 > F(7, 2) * S1)
+        for jj in range(2):
+            j = 2 * i + jj
+            e3 = (meta >> (16 + j)) & 1
+            g4 = max(ax[4 * j: 4 * j + 4])
+            top = F(7, 4) * S1 * 2 ** (e2 + e3)
+            if s < 255:
+                assert g4 <= top                                     # never clips
+            if e3 == 1:
+                assert g4 > F(7, 4) * S1 * 2 ** e2                    # lowering e3 would clip
+            step = S1 * 2 ** (e2 + e3) / 4
+            for k in range(4 * j, 4 * j + 4):
+                q, sign = cb[k] & 7, cb[k] >> 3
+                assert sign == int(np.signbit(xb[k]))
+                err = abs(ax[k] - q * step)
+                if s < 255 or ax[k] <= 7 * step:
+                    assert err <= step / 2
+                    if err == step / 2:
+                        assert q % 2 == 0                            # ties to even
+                else:
+                    assert q == 7                                     # saturation
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_hif4_invariants_random_blocks(seed):
+    x = gaussian_with_outliers(seed, 8, 256)
+    # mix in tiny, huge and exactly-zero blocks
+    x[0, :64] = 0
+    x[1, :64] *= np.float32(2.0 ** -60)
+    x[2, :64] *= np.float32(2.0 ** 12)
+    x[3, 64:128] = bf16_round(np.round(x[3, 64:128] * 4) / 4)      # many exact ties
+    codes, meta = oracle.hif4_encode(x)
+    q = nibbles(codes)
+    for r in range(x.shape[0]):
+        for b in range(x.shape[1] // 64):
+            _hif4_check_block(x[r, 64 * b: 64 * b + 64], q[r, 64 * b: 64 * b + 64], int(meta[r, b]))
+
+
+def test_hif4_scale_saturation_and_underflow():
+    x = np.zeros((2, 64), dtype=np.float32)
+    x[0, 5] = 3.0e38  # far above 7 * max S1: clamps to s = 255 and q = 7
+    x[1, 7] = 1e-30   # far below the smallest step: s = 0 and the element rounds to 0
+    codes, meta = oracle.hif4_encode(x)
+    q = nibbles(codes)
+    assert meta[0, 0] & 255 == 255 and q[0, 5] == 7
+    assert meta[1, 0] & 255 == 0 and q[1, 7] == 0
+    d = oracle.hif4_decode(codes, meta)
+    assert d[0, 5] == 7 * 1.75 * 2.0 ** 15
+
+
+def test_hif4_amax_group_invariant():
+    x = gaussian_with_outliers(5, 16, 512)
+    codes, meta = oracle.hif4_encode(x)
+    q = nibbles(codes) & 7
+    for r in range(16):
+        for b in range(8):
+            blk = np.abs(x[r, 64 * b: 64 * b + 64])
+            k = int(np.argmax(blk))
+            m = int(meta[r, b])
+            if m & 255:
+                # 7*S1(s-1) < amax and S1(s)/S1(s-1) <= 1.25  =>  amax > 5.6 * S1: top group uses both exponents
+                assert (m >> (8 + k // 8)) & 1 == 1 and (m >> (16 + k // 4)) & 1 == 1
+                assert q[r, 64 * b + k] >= 6
+
+
+def representable_hif4_blocks(seed, G, s_lo=1, s_hi=255):
+    """G blocks of values that ARE HiF4 values under scales that satisfy the encoder's own
+    minimality rules (every raised exponent is needed, the level-1 scale is the smallest that
+    covers the maximum), so that re-encoding must reproduce exactly these bits."""
+    rng = np.random.default_rng(seed)
+    x = np.zeros(64 * G, dtype=np.float64)
+    want_meta = np.zeros(G, dtype=np.uint32)
+    want_q = np.zeros(64 * G, dtype=np.uint8)
+    for b in range(G):
+        s = int(rng.integers(s_lo, s_hi))
+        S1 = float(F(4 + (s & 3), 4) * F(2) ** ((s >> 2) - 48))
+        e3 = rng.integers(0, 2, 16)
+        q = rng.integers(0, 8, 64)
+        sign = rng.integers(0, 2, 64)
+        top = int(rng.integers(0, 16))          # the 4-group that holds the block maximum 7*S1
+        e3[top] = 1
+        q[4 * top] = 7
+        # a raised level-2 exponent needs a raised level-3 group below it
+        e2 = np.array([int(rng.integers(0, 2)) if (e3[2 * i] or e3[2 * i + 1]) else 0 for i in range(8)])
+        e2[top // 2] = 1
+        for j in range(16):
+            if e3[j]:
+                q[4 * j + 1] = max(q[4 * j + 1], 4)   # the raised exponent must be needed (q >= 4)
+        want_meta[b] = s | sum(int(e2[i]) << (8 + i) for i in range(8)) | sum(int(e3[j]) << (16 + j) for j in range(16))
+        for k in range(64):
+            v = q[k] / 4.0 * 2.0 ** (int(e2[k // 8]) + int(e3[k // 4])) * S1
+            x[64 * b + k] = -v if sign[k] else v
+            want_q[64 * b + k] = (sign[k] << 3) | q[k]
+    return x, want_meta, want_q
+
+
+def test_hif4_round_trip_of_representable_blocks():
+    G = 200
+    x, want_meta, want_q = representable_hif4_blocks(7, G)
+    x = x.reshape(1, -1)
+    xf = x.astype(np.float32)
+    assert np.array_equal(xf.astype(np.float64), x)                 # representable values are fp32-exact
+    codes, meta = oracle.hif4_encode(xf)
+    assert np.array_equal(meta[0], want_meta)
+    assert np.array_equal(nibbles(codes)[0], want_q)
+    assert np.array_equal(oracle.hif4_decode(codes, meta), x)       # decode inverts it
+    # and the residual of a representable tensor is identically zero (Eq. 3)
+    assert not np.any(oracle.residual(xf, oracle.hif4_decode(codes, meta)))
+
+
+def test_hif4_rne_and_monotone_sweep():
+    # block whose scales are pinned by one element of magnitude 7 (S1 = 1, e2 = e3 = 1 in group 0);
+    # the probe sits in group 8 (e2 = e3 = 0 as long as it stays <= 1.75): step 1/4.
+    probes = np.arange(0, 1.75 + 1 / 64, 1 / 64)
+    x = np.zeros((len(probes), 64), dtype=np.float32)
+    x[:, 0] = 7.0
+    x[:, 40] = probes
+    codes, meta = oracle.hif4_encode(x)
+    assert np.all(meta == ((48 << 2) | (1 << 8) | (1 << 16)))
+    q = nibbles(codes)[:, 40]
+    assert np.all(np.diff(q.astype(int)) >= 0)
+    for p, qq in zip(probes, q):
+        t = F(float(p)) * 4
+        if t.denominator == 2:                    # exact midpoint -> even
+            assert qq % 2 == 0 and abs(qq - t) == F(1, 2)
+        else:
+            assert qq == round(t)
+    # negative probes mirror
+    x[:, 40] = -probes
+    codes2, _ = oracle.hif4_encode(x)
+    assert np.array_equal(nibbles(codes2)[:, 40], q | 8)
+
+
+def test_packing_nibble_order_and_meta_bits():
+    x = np.zeros((1, 64), dtype=np.float32)
+    x[0, 0], x[0, 1] = 1.75, -0.25          # S1 = 0.25 (7*.25 = 1.75): q0 = 7 at e2=e3=1 in group 0
+    codes, meta = oracle.hif4_encode(x)
+    # element 0 -> low nibble, element 1 -> high nibble of byte 0
+    assert codes[0, 0] & 15 == 7
+    assert codes[0, 0] >> 4 == (8 | 1)      # step in the raised group is 0.25*4/4 = 0.25 -> q = 1, negative
+    assert int(meta[0, 0]) & 255 == (46 << 2)
+    assert (int(meta[0, 0]) >> 8) & 255 == 1 and int(meta[0, 0]) >> 16 == 1
+
+
+# ----------------------------------------------------------------- MXFP4
+
+def test_mxfp4_element_rounding_matches_library(nvref):
+    # block scale pinned to 2^0 by an element of 4.0; the probe must not exceed 8 (would change the scale)
+    probes = np.concatenate([np.arange(0, 7.99, 1 / 32), [0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0, 7.0, 7.9]])
+    probes = probes.astype(np.float32)
+    x = np.zeros((len(probes), 32), dtype=np.float32)
+    x[:, 0] = 4.0
+    x[:, 9] = probes
+    x[1::2, 9] *= -1
+    codes, scale = oracle.mxfp4_encode(x)
+    assert np.all(scale == 127)
+    q = nibbles(codes)[:, 9]
+    for i, p in enumerate(x[:, 9]):
+        assert int(q[i]) == nvref.nv_float_to_e2m1(float(p)), p
+
+
+def test_mxfp4_scale_property():
+    x = gaussian_with_outliers(11, 8, 256)
+    x[0, :32] = 0
+    codes, scale = oracle.mxfp4_encode(x)
+    for r in range(8):
+        for b in range(8):
+            amax = float(np.abs(x[r, 32 * b: 32 * b + 32]).max())
+            if amax == 0:
+                assert scale[r, b] == 0
+                continue
+            t = F(amax) / F(2) ** (int(scale[r, b]) - 127)
+            assert 4 <= t < 8                      # the block maximum lands in E2M1's top binade
+    d = oracle.mxfp4_decode(codes, scale)
+    # decode is value(code) * 2^(scale-127), checked against the tables
+    q = nibbles(codes)
+    for (r, k) in [(1, 3), (2, 77), (7, 255)]:
+        assert d[r, k] == oracle.e2m1_value(int(q[r, k])) * oracle.e8m0_value(int(scale[r, k // 32]))
+
+
+def test_mxfp4_round_trip():
+    rng = np.random.default_rng(3)
+    G = 64
+    sc = rng.integers(100, 150, G)
+    q = rng.integers(0, 16, (G, 32))
+    q[:, 0] = 7 - (rng.integers(0, 2, G))          # top binade present (6 or 4): scale is recoverable
+    x = np.zeros((1, 32 * G))
+    for b in range(G):
+        for k in range(32):
+            x[0, 32 * b + k] = oracle.e2m1_value(int(q[b, k])) * oracle.e8m0_value(int(sc[b]))
+    codes, scale = oracle.mxfp4_encode(x.astype(np.float32))
+    assert np.array_equal(scale[0], sc)
+    assert np.array_equal(nibbles(codes)[0], q.reshape(-1))
+
+
+def test_hif4_is_more_accurate_than_mxfp4_on_outlier_data():
+    x = gaussian_with_outliers(21, 32, 1024, n_out=6)
+    xd = x.astype(np.float64)
+    eh = np.linalg.norm(xd - oracle.hif4_decode(*oracle.hif4_encode(x)))
+    em = np.linalg.norm(xd - oracle.mxfp4_decode(*oracle.mxfp4_encode(x)))
+    assert eh < em
+
+
+# ----------------------------------------------------------------- residual (Eq. 3) and bounds
+
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+def test_residual_identity_and_bound(fmt):
+    x = gaussian_with_outliers(4, 16, 512)
+    o = oracle.quantize_residual_mask(x, oracle.S_DENSE, fmt)
+    xd = x.astype(np.float64)
+    assert np.array_equal(o["dx"].astype(np.float64), xd - o["a"])          # Eq. (3), exactly
+    # the second quantization shrinks the error: ||x - a - r|| < ||x - a||
+    assert np.linalg.norm(xd - o["a"] - o["r"]) < 0.25 * np.linalg.norm(xd - o["a"])
+    if fmt == "hif4":
+        # |dx - r| <= step_r / 2 for every element (no clipping in the residual encode)
+        meta = o["r_side"]
+        for r in range(4):
+            for k in range(0, 512, 37):
+                m = int(meta[r, k // 64])
+                kk = k % 64
+                S1 = oracle.e6m2_value(m & 255)
+                step = S1 * 2.0 ** (((m >> (8 + kk // 8)) & 1) + ((m >> (16 + kk // 4)) & 1)) / 4
+                assert abs(float(o["dx"][r, k]) - o["r"][r, k]) <= step / 2
+
+
+def test_outliers_collapse_their_block_to_zero():
+    # Figure 1's effect: an outlier forces a large scale and the bulk of its block underflows
+    rng = np.random.default_rng(9)
+    x = bf16_round(rng.standard_normal((64, 64)).astype(np.float32))
+    xo = x.copy()
+    xo[:, 17] *= 64
+    z = lambda c: float(((nibbles(c) & 7) == 0).mean())
+    z_plain = z(oracle.hif4_encode(x)[0])
+    z_out = z(oracle.hif4_encode(xo)[0])
+    assert z_out > 0.5 > z_plain
+
+
+# ----------------------------------------------------------------- masks (Section 4.3)
+
+def _bits_to_bool(bits, K):
+    return np.unpackbits(bits, axis=1, bitorder="little")[:, :K].astype(bool)
+
+
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+def test_mask_counts(fmt):
+    M, K = 64, 256
+    x = gaussian_with_outliers(31, M, K)
+    for pattern in (oracle.S_2_4, oracle.S_ROW50, oracle.S_CHAN50, oracle.S_BLOCK, oracle.S_DENSE):
+        o = oracle.quantize_residual_mask(x, pattern, fmt)
+        mb = _bits_to_bool(o["mask"], K)
+        if pattern == oracle.S_2_4:
+            assert np.all(mb.reshape(M, K // 4, 4).sum(-1) == 2)
+        elif pattern == oracle.S_ROW50:
+            assert np.all(mb.sum(1) == K // 2)
+        elif pattern == oracle.S_CHAN50:
+            assert mb[0].sum() == K // 2 and np.all(mb == mb[0])
+        elif pattern == oracle.S_BLOCK:
+            blk = mb.reshape(M // 32, 32, K // 64, 64).transpose(0, 2, 1, 3).reshape(-1, 32 * 64)
+            assert np.all((blk.sum(1) == 0) | (blk.sum(1) == 2048))
+            assert (blk.sum(1) == 2048).sum() == (M // 32) * (K // 64) // 2
+        else:
+            assert mb.all()
+        # kept entries keep their value, dropped ones are zero
+        assert np.array_equal(o["r_masked"], np.where(mb, o["r"], 0.0))
+
+
+def _check_topk_valid(keys, kept):
+    """No dropped key exceeds a kept one; among equal boundary keys the lower index is kept."""
+    keys, kept = np.asarray(keys), np.asarray(kept, dtype=bool)
+    if kept.all() or not kept.any():
+        return
+    lo = keys[kept].min()
+    hi = keys[~kept].max()
+    assert hi <= lo
+    if hi == lo:
+        tied = np.nonzero(keys == lo)[0]
+        kt = kept[tied]
+        assert np.all(np.diff(kt.astype(int)) <= 0)      # kept ties come first
+
+
+def test_mask_optimality_bruteforce_small():
+    rng = np.random.default_rng(5)
+    M, K = 32, 128
+    # few distinct magnitudes => many ties
+    v = rng.integers(-3, 4, (M, K)).astype(np.float64) * 0.25
+    bits, _ = oracle.mask(v, oracle.S_2_4)
+    mb = _bits_to_bool(bits, K)
+    for m in range(M):
+        for g in range(K // 4):
+            grp = np.abs(v[m, 4 * g: 4 * g + 4])
+            # brute force over the 6 ways to keep 2 of 4: the kept set has the maximal key sum and,
+            # among those, the lexicographically smallest positions
+            best = max(itertools.combinations(range(4), 2), key=lambda c: (grp[list(c)].sum(), [-i for i in c]))
+            assert tuple(np.nonzero(mb[m, 4 * g: 4 * g + 4])[0]) == best
+    bits, _ = oracle.mask(v, oracle.S_ROW50)
+    mb = _bits_to_bool(bits, K)
+    for m in range(M):
+        _check_topk_valid(np.abs(v[m]), mb[m])
+    bits, info = oracle.mask(v, oracle.S_CHAN50, want_scores=True)
+    mb = _bits_to_bool(bits, K)
+    assert np.array_equal(info["scores"], (v ** 2).sum(0)) and info["exact"]
+    _check_topk_valid((v ** 2).sum(0), mb[0])
+    M2, K2 = 128, 256
+    v2 = rng.integers(-2, 3, (M2, K2)).astype(np.float64)
+    bits, info = oracle.mask(v2, oracle.S_BLOCK, want_scores=True)
+    mb = _bits_to_bool(bits, K2)
+    sc = (v2 ** 2).reshape(M2 // 32, 32, K2 // 64, 64).sum((1, 3)).reshape(-1)
+    assert np.array_equal(info["scores"], sc)
+    kept_blk = mb.reshape(M2 // 32, 32, K2 // 64, 64)[:, 0, :, 0].reshape(-1)
+    _check_topk_valid(sc, kept_blk)
+    assert kept_blk.sum() == len(sc) // 2
+
+
+def test_block_orientation_is_32_rows_by_64_columns():
+    v = np.zeros((64, 128))
+    v[0:32, 64:128] = 1.0      # one hot block at block-row 0, block-col 1
+    v[32:64, 0:64] = 0.5       # a weaker one at block-row 1, block-col 0
+    bits, _ = oracle.mask(v, oracle.S_BLOCK)
+    mb = _bits_to_bool(bits, 128)
+    assert mb[0:32, 64:128].all() and mb[32:64, 0:64].all() and mb.sum() == 2 * 2048
+
+
+def test_sparsifying_the_residual_costs_less_than_sparsifying_the_activation():
+    # Figure 4's observation, on synthetic data: 2:4 on Q(dX) loses less (absolute MSE) than 2:4 on Q(X)
+    x = gaussian_with_outliers(41, 32, 1024, n_out=6)
+    o = oracle.quantize_residual_mask(x, oracle.S_2_4)
+    a_bits, _ = oracle.mask(o["a"], oracle.S_2_4)
+    mse_a = np.mean((o["a"] - oracle.apply_mask(o["a"], a_bits)) ** 2)
+    mse_r = np.mean((o["r"] - o["r_masked"]) ** 2)
+    assert mse_r < mse_a
+
+
+# ----------------------------------------------------------------- product (Eqs. 1, 4, 5)
+
+def _to_frac(a):
+    return [[F(float(v)) for v in row] for row in a]
+
+
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_DENSE, oracle.S_2_4])
+def test_matmul_exact_rational_tiny(fmt, pattern):
+    M, K, N = 3, 128, 5
+    x = gaussian_with_outliers(51, M, K, n_out=2, scale=16.0)
+    rng = np.random.default_rng(52)
+    w = bf16_round(rng.standard_normal((N, K)).astype(np.float32) * 0.02)
+    o = oracle.resq_linear(x, w, pattern, fmt)
+    a, wv = _to_frac(o["a"]), _to_frac(o["w"])
+    r = _to_frac(o["r_masked"]) if pattern != oracle.S_NONE else [[F(0)] * K for _ in range(M)]
+    for m in range(M):
+        for n in range(N):
+            exact = sum((a[m][k] + r[m][k]) * wv[n][k] for k in range(K))
+            # fp64 over 128 exact products of ~12-bit significands with a narrow exponent range is exact
+            assert F(float(o["y"][m, n])) == exact
+            assert o["abs_sum"][m, n] >= abs(o["y"][m, n])
+    assert o["y"].shape == (M, N)
+
+
+def test_matmul_reduces_to_numpy_when_residual_vanishes():
+    rng = np.random.default_rng(61)
+    M, K, N = 8, 256, 12
+    # X made of decoded codes => Q(X) = X, dX = 0, every S gives the same Y = X W^T (Eqs. 1, 4, 5 coincide)
+    # (level-1 codes limited to 2^-8 .. 2^4 so that the fp64 sums stay well conditioned)
+    xq = representable_hif4_blocks(62, M * K // 64, 40 << 2, 52 << 2)[0].reshape(M, K).astype(np.float32)
+    assert np.array_equal(oracle.hif4_decode(*oracle.hif4_encode(xq)), xq.astype(np.float64))
+    w = bf16_round(rng.standard_normal((N, K)).astype(np.float32) * 0.02)
+    wq = oracle.hif4_decode(*oracle.hif4_encode(w))
+    ref = xq.astype(np.float64) @ wq.T
+    for pattern in (oracle.S_NONE, oracle.S_DENSE, oracle.S_2_4, oracle.S_ROW50):
+        o = oracle.resq_linear(xq, w, pattern)
+        np.testing.assert_allclose(o["y"], ref, rtol=1e-13, atol=1e-13)
+
+
+def test_dense_is_eq4_and_none_is_eq1():
+    x = gaussian_with_outliers(71, 8, 256)
+    rng = np.random.default_rng(72)
+    w = bf16_round(rng.standard_normal((16, 256)).astype(np.float32) * 0.02)
+    o_none = oracle.resq_linear(x, w, oracle.S_NONE)
+    o_dense = oracle.resq_linear(x, w, oracle.S_DENSE)
+    np.testing.assert_allclose(o_none["y"], o_none["a"] @ o_none["w"].T, rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(o_dense["y"], o_dense["a"] @ o_dense["w"].T + o_dense["r"] @ o_dense["w"].T,
+                               rtol=1e-13, atol=1e-13)
+    # and the correction does what the paper says it does: it moves Y toward X deq(W)^T
+    target = x.astype(np.float64) @ o_none["w"].T
+    o_24 = oracle.resq_linear(x, w, oracle.S_2_4)
+    e0 = np.linalg.norm(o_none["y"] - target)
+    e24 = np.linalg.norm(o_24["y"] - target)
+    ed = np.linalg.norm(o_dense["y"] - target)
+    assert ed < e24 < e0
+
+
+# ----------------------------------------------------------------- regression digest of a seeded tensor
+
+def test_seeded_digest():
+    """Statistics of a seeded tensor, first derived with an independent throw-away script under the
+    same reading and reproduced by this oracle; a change in any rule moves at least one of them."""
+    rng = np.random.default_rng(0)
+    X = rng.standard_normal((16, 2048)).astype(np.float32)
+    ch = rng.choice(2048, 8, replace=False)
+    assert sorted(int(c) for c in ch) == [79, 179, 520, 868, 1194, 1550, 1752, 1982]
+    X[:, ch] *= 64
+    X = bf16_round(X)
+    o = oracle.quantize_residual_mask(X, oracle.S_2_4)
+
+    def stats(codes, meta):
+        q = nibbles(codes)
+        return (int(((q & 7) == 0).sum()), int((q & 7).sum()), int((meta & 255).sum()),
+                sum(bin((int(m) >> 8) & 255).count("1") for m in meta.ravel()),
+                sum(bin(int(m) >> 16).count("1") for m in meta.ravel()))
+
+    assert stats(o["x_codes"], o["x_side"]) == (7496, 75391, 97397, 2429, 4637)
+    assert stats(o["r_codes"], o["r_side"]) == (2452, 111754, 89308, 2555, 5588)
+    assert int((nibbles(o["x_codes"]) >> 3).sum()) == 16425
+    XX = X.astype(np.float64)
+    rel = lambda e: float(np.linalg.norm(e) / np.linalg.norm(XX))
+    assert abs(rel(XX - o["a"]) - 0.0881) < 5e-4
+    assert abs(rel(XX - o["a"] - o["r"]) - 0.0076) < 5e-4
+    assert abs(rel(XX - o["a"] - o["r_masked"]) - 0.0346) < 5e-4
