@@ -1,0 +1,140 @@
+/*
+ * resq.h -- C ABI of the B200 (sm_100a) Rollout-ResQ FP4 linear layer.
+ *
+ *     Y  =  Q(X) Q(W)^T  +  S(Q(X - deq Q(X))) Q(W)^T            (paper Eq. (5))
+ *
+ * X is the activation [M, K] (paper: m x d), W the weight [N, K] (paper: n x d), Y [M, N]
+ * (Section 3, "Block-Scaled Quantization": Y = X W^T).  Q is a block-scaled 4-bit quantizer whose
+ * blocks run along K.  Two formats are provided, as in the paper: HiF4 (blocks of 64, E6M2 level-1
+ * scaler, E1 level-2 and level-3 scalers, S1P2 elements) and MXFP4 (blocks of 32, E8M0 scale,
+ * E2M1 elements), the latter as the comparison twin (`mxfp4_*`).
+ *
+ * Conventions for every call
+ *   - All tensor pointers are DEVICE pointers (the library never touches host data); row-major;
+ *     `ld*` is the row stride in ELEMENTS of the pointed-to type.  bf16 inputs must be 16-byte
+ *     aligned with ld a multiple of 8.  Packed outputs are dense (no stride).
+ *   - The caller owns every buffer; the library allocates no device memory.  Scratch comes from
+ *     the `workspace` argument, sized by the matching *_workspace_bytes query (256-byte aligned).
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *   - The return value is a resq_status.  Shape / null / alignment / workspace errors are detected
+ *     on the host before anything is launched.  Nothing throws.  resq_last_error() returns a
+ *     thread-local description of the most recent failure.
+ *   - Device-side waits are bounded; if one expires the kernel records RESQ_ERR_TIMEOUT in the
+ *     status word at the start of the workspace and exits normally; resq_check() reads it.
+ *
+ * Packed layouts (bit-exact contract; the paper fixes the field widths only, the rest is this
+ * library's reading, see the notes at each call)
+ *   HiF4   codes[row][K/2] u8 : element 2j in bits 3:0, element 2j+1 in bits 7:4; a code is
+ *                               sign<<3 | q, magnitude q/4 (S1P2 == E1M2: 0, .25, ..., 1.75).
+ *          meta [row][K/64] u32: bits 7:0 level-1 E6M2 code s = E<<2|Mn, S1 = (1+Mn/4) 2^(E-48);
+ *                               bit 8+i  = level-2 exponent of elements 8i..8i+7   (i = 0..7);
+ *                               bit 16+j = level-3 exponent of elements 4j..4j+3   (j = 0..15).
+ *          value = (-1)^sign (q/4) 2^(e2+e3) S1.
+ *   MXFP4  codes as above with E2M1 codes (0,.5,1,1.5,2,3,4,6); scale[row][K/32] u8 E8M0 (2^(c-127)).
+ *   mask   mask_bits[m][K/8] u8: bit (k&7) of byte k>>3 is 1 where S keeps element k of row m.
+ */
+#ifndef RESQ_H_
+#define RESQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define RESQ_API __attribute__((visibility("default")))
+#else
+#define RESQ_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RESQ_OK = 0,
+    RESQ_ERR_NULL = 1,      /* a required pointer is NULL */
+    RESQ_ERR_SHAPE = 2,     /* M,N,K <= 0; K % 64 (HiF4) or K % 32 (MXFP4); block pattern needs M % 32 == 0 */
+    RESQ_ERR_ALIGN = 3,     /* base pointer not 16-byte aligned, or ld not a multiple of 8 / smaller than K */
+    RESQ_ERR_WORKSPACE = 4, /* workspace NULL, misaligned or smaller than the query says */
+    RESQ_ERR_PATTERN = 5,   /* unknown pattern or output type */
+    RESQ_ERR_CUDA = 6,      /* a CUDA call or launch failed; text in resq_last_error() */
+    RESQ_ERR_TIMEOUT = 7    /* a bounded device-side wait expired (reported by resq_check) */
+} resq_status;
+
+/* The sparsity function S of Eq. (5) (Section 4.3). */
+typedef enum {
+    RESQ_S_NONE = 0,          /* no residual term: Eq. (1) */
+    RESQ_S_DENSE = 1,         /* S = identity: Eq. (4), "Rollout-ResQ-Dense" */
+    RESQ_S_2_4 = 2,           /* keep the 2 largest magnitudes of every 4 contiguous elements along K;
+                                 ties keep the lower index; always exactly 2 kept */
+    RESQ_S_ROW50 = 3,         /* per row, keep the K/2 largest magnitudes (ties: lower index) */
+    RESQ_S_CHAN50 = 4,        /* keep the K/2 channels (columns) with the largest L2 norm over all M rows */
+    RESQ_S_BLOCK32x64_50 = 5  /* keep floor(nb/2) of the nb aligned blocks of 32 rows x 64 channels with the
+                                 largest L2 norm, chosen over the whole tensor */
+} resq_pattern;
+
+typedef enum { RESQ_OUT_BF16 = 0, RESQ_OUT_F32 = 1 } resq_out;
+
+/* ---- size queries (host only, no CUDA calls) -------------------------------------------------- */
+RESQ_API size_t hif4_codes_bytes(int64_t rows, int64_t K);  /* rows*K/2 */
+RESQ_API size_t hif4_meta_bytes(int64_t rows, int64_t K);   /* rows*(K/64)*4 */
+RESQ_API size_t mxfp4_codes_bytes(int64_t rows, int64_t K); /* rows*K/2 */
+RESQ_API size_t mxfp4_scale_bytes(int64_t rows, int64_t K); /* rows*(K/32) */
+RESQ_API size_t resq_mask_bytes(int64_t M, int64_t K);      /* M*K/8 */
+/* Scratch for *_residual_mask (status word, channel / block scores, selection buffers). */
+RESQ_API size_t resq_residual_mask_workspace_bytes(int64_t M, int64_t K, int pattern);
+/* Scratch for *_resq_linear (the above plus the expanded activation operands of the GEMM and,
+ * for small M, split-K partial tiles). */
+RESQ_API size_t hif4_resq_workspace_bytes(int64_t M, int64_t N, int64_t K, int pattern);
+RESQ_API size_t mxfp4_resq_workspace_bytes(int64_t M, int64_t N, int64_t K, int pattern);
+
+/* ---- Q(W): pack a weight once per policy update (Section 3, Eq. (1): W_hat = Q(W)) -------------
+ * W_bf16 [N, K] with row stride ldw -> w_codes [N, K/2], w_meta [N, K/64] (HiF4) or w_scale [N, K/32].
+ * HiF4 scale rule (this library's reading; the paper gives the field formats only): level 1 is the
+ * smallest E6M2 value with 7*S1 >= max|block|; a level-2 / level-3 exponent is raised exactly when
+ * the group would otherwise clip; elements round to nearest, ties to even.  MXFP4: scale exponent
+ * floor(log2 max|block|) - 2, elements round to nearest even and saturate at 6. */
+RESQ_API int hif4_pack_weight(const void* W_bf16, int64_t N, int64_t K, int64_t ldw, void* w_codes, void* w_meta, void* stream);
+RESQ_API int mxfp4_pack_weight(const void* W_bf16, int64_t N, int64_t K, int64_t ldw, void* w_codes, void* w_scale, void* stream);
+
+/* ---- Q(X): on-the-fly activation quantizer (same operator Q applied to X, Eq. (1)) ------------- */
+RESQ_API int hif4_quantize_act(const void* X_bf16, int64_t M, int64_t K, int64_t ldx, void* x_codes, void* x_meta, void* stream);
+RESQ_API int mxfp4_quantize_act(const void* X_bf16, int64_t M, int64_t K, int64_t ldx, void* x_codes, void* x_scale, void* stream);
+
+/* ---- deq: decode packed data to fp32 [rows, K] (test helper; every HiF4 / MXFP4 value is fp32-exact) */
+RESQ_API int hif4_dequantize(const void* codes, const void* meta, int64_t rows, int64_t K, float* out, void* stream);
+RESQ_API int mxfp4_dequantize(const void* codes, const void* scale, int64_t rows, int64_t K, float* out, void* stream);
+
+/* ---- Q(X), dX = X - deq Q(X) (Eq. (3)), Q(dX) (Eq. (4)) and the selection S (Eq. (5), Section 4.3)
+ * in one pass over X.  Outputs (any of them may be NULL to skip it): Q(X), Q(dX) in the canonical
+ * dense layout, and mask_bits.  S acts on the decoded magnitudes of Q(dX); kept elements keep their
+ * value, dropped ones contribute zero.  For RESQ_S_NONE only Q(X) is written. */
+RESQ_API int resq_residual_mask(const void* X_bf16, int64_t M, int64_t K, int64_t ldx, int pattern,
+                       void* x_codes, void* x_meta, void* r_codes, void* r_meta, void* mask_bits,
+                       void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_residual_mask(const void* X_bf16, int64_t M, int64_t K, int64_t ldx, int pattern,
+                        void* x_codes, void* x_scale, void* r_codes, void* r_scale, void* mask_bits,
+                        void* workspace, size_t ws_bytes, void* stream);
+
+/* ---- the rollout projection, Eq. (5):  Y = Q(X) Q(W)^T + S(Q(dX)) Q(W)^T ------------------------
+ * X_bf16 [M, K] (ldx), packed weight from *_pack_weight, Y [M, N] (ldy) as bf16 (round-to-nearest-
+ * even of the fp32 accumulator) or fp32.  Products of decoded values are exact in fp32; only the
+ * accumulation rounds.  Both terms are accumulated into the same output tile. */
+RESQ_API int hif4_resq_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
+                     const void* w_codes, const void* w_meta, int64_t N,
+                     int pattern, void* Y, int out_dtype, int64_t ldy,
+                     void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_resq_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
+                      const void* w_codes, const void* w_scale, int64_t N,
+                      int pattern, void* Y, int out_dtype, int64_t ldy,
+                      void* workspace, size_t ws_bytes, void* stream);
+
+/* ---- status --------------------------------------------------------------------------------------
+ * resq_check synchronizes `stream` and returns the device status word kept at the start of
+ * `workspace` (RESQ_OK, or RESQ_ERR_TIMEOUT if a bounded wait expired in the last call that used it). */
+RESQ_API int resq_check(void* workspace, void* stream);
+RESQ_API const char* resq_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RESQ_H_ */

@@ -1,0 +1,198 @@
+"""Thin ctypes binding of the C ABI in include/resq.h (argument marshalling only).
+
+PyTorch supplies device memory (`tensor.data_ptr()`) and the stream; every step of the path
+runs in the CUDA library.  There is no CPU fallback: if the library is missing or a call fails,
+this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libresq.so")
+
+S_NONE, S_DENSE, S_2_4, S_ROW50, S_CHAN50, S_BLOCK = 0, 1, 2, 3, 4, 5
+OUT_BF16, OUT_F32 = 0, 1
+PATTERN_NAMES = {S_NONE: "none", S_DENSE: "dense", S_2_4: "2:4", S_ROW50: "row50", S_CHAN50: "chan50",
+                 S_BLOCK: "block32x64"}
+STATUS_NAMES = {0: "OK", 1: "ERR_NULL", 2: "ERR_SHAPE", 3: "ERR_ALIGN", 4: "ERR_WORKSPACE", 5: "ERR_PATTERN",
+                6: "ERR_CUDA", 7: "ERR_TIMEOUT"}
+
+# every symbol include/resq.h declares: (name, restype, argtypes)
+_i64, _vp, _ci, _sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+SYMBOLS = {
+    "hif4_codes_bytes": (_sz, [_i64, _i64]),
+    "hif4_meta_bytes": (_sz, [_i64, _i64]),
+    "mxfp4_codes_bytes": (_sz, [_i64, _i64]),
+    "mxfp4_scale_bytes": (_sz, [_i64, _i64]),
+    "resq_mask_bytes": (_sz, [_i64, _i64]),
+    "resq_residual_mask_workspace_bytes": (_sz, [_i64, _i64, _ci]),
+    "hif4_resq_workspace_bytes": (_sz, [_i64, _i64, _i64, _ci]),
+    "mxfp4_resq_workspace_bytes": (_sz, [_i64, _i64, _i64, _ci]),
+    "hif4_pack_weight": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
+    "mxfp4_pack_weight": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
+    "hif4_quantize_act": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
+    "mxfp4_quantize_act": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
+    "hif4_dequantize": (_ci, [_vp, _vp, _i64, _i64, _vp, _vp]),
+    "mxfp4_dequantize": (_ci, [_vp, _vp, _i64, _i64, _vp, _vp]),
+    "resq_residual_mask": (_ci, [_vp, _i64, _i64, _i64, _ci, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "mxfp4_residual_mask": (_ci, [_vp, _i64, _i64, _i64, _ci, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "hif4_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "mxfp4_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "resq_check": (_ci, [_vp, _vp]),
+    "resq_last_error": (ctypes.c_char_p, []),
+}
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+class ResqError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"resq: {STATUS_NAMES.get(status, status)}: {msg}")
+        self.status = status
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_26515_b200.build` "
+                               "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SYMBOLS.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def last_error() -> str:
+    return lib().resq_last_error().decode()
+
+
+def _check(status: int) -> None:
+    if status != 0:
+        raise ResqError(status, last_error())
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _side(fmt: str, rows: int, K: int, device) -> torch.Tensor:
+    if fmt == "hif4":
+        return torch.empty((rows, K // 64), dtype=torch.int32, device=device)
+    return torch.empty((rows, K // 32), dtype=torch.uint8, device=device)
+
+
+def _fn(fmt: str, hif4_name: str, mx_name: str):
+    if fmt not in ("hif4", "mxfp4"):
+        raise ValueError(f"unknown format {fmt!r}")
+    return getattr(lib(), hif4_name if fmt == "hif4" else mx_name)
+
+
+def _require_bf16_matrix(x: torch.Tensor, name: str) -> None:
+    if x.dtype != torch.bfloat16 or x.dim() != 2 or not x.is_cuda or x.stride(1) != 1:
+        raise ValueError(f"{name} must be a 2-D CUDA bf16 tensor with unit inner stride")
+
+
+# ------------------------------------------------------------------ size queries
+
+def residual_mask_workspace_bytes(M: int, K: int, pattern: int) -> int:
+    return int(lib().resq_residual_mask_workspace_bytes(M, K, pattern))
+
+
+def resq_workspace_bytes(M: int, N: int, K: int, pattern: int, fmt: str = "hif4") -> int:
+    return int(_fn(fmt, "hif4_resq_workspace_bytes", "mxfp4_resq_workspace_bytes")(M, N, K, pattern))
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+# ------------------------------------------------------------------ calls
+
+def pack_weight(W: torch.Tensor, fmt: str = "hif4", stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """*_pack_weight: W bf16 [N,K] -> (codes u8 [N,K/2], meta i32 [N,K/64] | scale u8 [N,K/32])."""
+    _require_bf16_matrix(W, "W")
+    N, K = W.shape
+    codes = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
+    side = _side(fmt, N, K, W.device)
+    _check(_fn(fmt, "hif4_pack_weight", "mxfp4_pack_weight")(W.data_ptr(), N, K, W.stride(0), codes.data_ptr(),
+                                                              side.data_ptr(), _stream(stream)))
+    return codes, side
+
+
+def quantize_act(X: torch.Tensor, fmt: str = "hif4", stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """*_quantize_act: X bf16 [M,K] -> (codes, meta | scale)."""
+    _require_bf16_matrix(X, "X")
+    M, K = X.shape
+    codes = torch.empty((M, K // 2), dtype=torch.uint8, device=X.device)
+    side = _side(fmt, M, K, X.device)
+    _check(_fn(fmt, "hif4_quantize_act", "mxfp4_quantize_act")(X.data_ptr(), M, K, X.stride(0), codes.data_ptr(),
+                                                                side.data_ptr(), _stream(stream)))
+    return codes, side
+
+
+def dequantize(codes: torch.Tensor, side: torch.Tensor, fmt: str = "hif4", stream=None) -> torch.Tensor:
+    rows, K = codes.shape[0], codes.shape[1] * 2
+    out = torch.empty((rows, K), dtype=torch.float32, device=codes.device)
+    _check(_fn(fmt, "hif4_dequantize", "mxfp4_dequantize")(codes.data_ptr(), side.data_ptr(), rows, K, out.data_ptr(),
+                                                            _stream(stream)))
+    return out
+
+
+def residual_mask(X: torch.Tensor, pattern: int, fmt: str = "hif4", workspace: Optional[torch.Tensor] = None,
+                  stream=None):
+    """resq_residual_mask / mxfp4_residual_mask -> dict(x_codes, x_side, r_codes, r_side, mask)."""
+    _require_bf16_matrix(X, "X")
+    M, K = X.shape
+    dev = X.device
+    out = {"x_codes": torch.empty((M, K // 2), dtype=torch.uint8, device=dev), "x_side": _side(fmt, M, K, dev),
+           "r_codes": None, "r_side": None, "mask": None}
+    if pattern != S_NONE:
+        out["r_codes"] = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
+        out["r_side"] = _side(fmt, M, K, dev)
+        out["mask"] = torch.empty((M, K // 8), dtype=torch.uint8, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(residual_mask_workspace_bytes(M, K, pattern), dev)
+    _check(_fn(fmt, "resq_residual_mask", "mxfp4_residual_mask")(
+        X.data_ptr(), M, K, X.stride(0), pattern, _ptr(out["x_codes"]), _ptr(out["x_side"]), _ptr(out["r_codes"]),
+        _ptr(out["r_side"]), _ptr(out["mask"]), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return out
+
+
+def resq_linear(X: torch.Tensor, w_codes: torch.Tensor, w_side: torch.Tensor, pattern: int, fmt: str = "hif4",
+                out_dtype: torch.dtype = torch.bfloat16, Y: Optional[torch.Tensor] = None,
+                workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """*_resq_linear: Y = Q(X) Q(W)^T + S(Q(X - deq Q(X))) Q(W)^T  (Eq. (5))."""
+    _require_bf16_matrix(X, "X")
+    M, K = X.shape
+    N = w_codes.shape[0]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=out_dtype, device=X.device)
+    if Y.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("Y must be bf16 or fp32")
+    if workspace is None:
+        workspace = alloc_workspace(resq_workspace_bytes(M, N, K, pattern, fmt), X.device)
+    _check(_fn(fmt, "hif4_resq_linear", "mxfp4_resq_linear")(
+        X.data_ptr(), M, K, X.stride(0), w_codes.data_ptr(), w_side.data_ptr(), N, pattern, Y.data_ptr(),
+        OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32, Y.stride(0), workspace.data_ptr(), workspace.numel(),
+        _stream(stream)))
+    return Y
+
+
+def check(workspace: torch.Tensor, stream=None) -> int:
+    """resq_check: synchronize and return the device status word."""
+    return int(lib().resq_check(workspace.data_ptr(), _stream(stream)))

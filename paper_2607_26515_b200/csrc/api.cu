@@ -1,0 +1,303 @@
+// C ABI of the ResQ library: argument checks, workspace carving, kernel sequencing.
+// The contract of every entry point is stated in include/resq.h.
+#include "common.cuh"
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+namespace resq {
+
+static thread_local char g_last_error[512] = "";
+
+void set_last_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_last_error, sizeof(g_last_error), fmt, ap);
+    va_end(ap);
+}
+
+int cuda_fail(cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return RESQ_OK;
+    set_last_error("%s: %s", what, cudaGetErrorString(e));
+    return RESQ_ERR_CUDA;
+}
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int block_of(int fmt) { return fmt == kHiF4 ? kHif4Block : kMxBlock; }
+
+int check_matrix(const void* p, int64_t rows, int64_t K, int64_t ld, int fmt, const char* name) {
+    if (!p) {
+        set_last_error("%s is NULL", name);
+        return RESQ_ERR_NULL;
+    }
+    if (rows <= 0 || K <= 0 || K % block_of(fmt) != 0) {
+        set_last_error("%s: rows=%lld K=%lld (K must be a positive multiple of %d)", name, (long long)rows, (long long)K,
+                       block_of(fmt));
+        return RESQ_ERR_SHAPE;
+    }
+    if (!aligned16(p) || ld < K || ld % 8 != 0) {
+        set_last_error("%s: needs a 16-byte aligned base and ld >= K, ld %% 8 == 0 (ld=%lld)", name, (long long)ld);
+        return RESQ_ERR_ALIGN;
+    }
+    return RESQ_OK;
+}
+
+int check_pattern(int pattern, int64_t M) {
+    if (pattern < RESQ_S_NONE || pattern > RESQ_S_BLOCK32x64_50) {
+        set_last_error("unknown pattern %d", pattern);
+        return RESQ_ERR_PATTERN;
+    }
+    if (pattern == RESQ_S_BLOCK32x64_50 && M % kBlkRows != 0) {
+        set_last_error("the 32x64 block pattern needs M %% 32 == 0 (M=%lld)", (long long)M);
+        return RESQ_ERR_SHAPE;
+    }
+    return RESQ_OK;
+}
+
+int check_workspace(const void* ws, size_t have, size_t need) {
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || have < need) {
+        set_last_error("workspace: need %zu bytes, 256-byte aligned (have %zu at %p)", need, have, ws);
+        return RESQ_ERR_WORKSPACE;
+    }
+    return RESQ_OK;
+}
+
+int quantize_only(int fmt, const void* X, int64_t rows, int64_t K, int64_t ld, void* codes, void* side, void* stream,
+                  const char* name) {
+    int rc = check_matrix(X, rows, K, ld, fmt, name);
+    if (rc) return rc;
+    if (!codes || !side) {
+        set_last_error("%s: output pointer is NULL", name);
+        return RESQ_ERR_NULL;
+    }
+    QuantArgs a;
+    memset(&a, 0, sizeof(a));
+    a.X = static_cast<const __nv_bfloat16*>(X);
+    a.M = rows;
+    a.K = K;
+    a.ldx = ld;
+    a.pattern = RESQ_S_NONE;
+    a.x_codes = static_cast<uint8_t*>(codes);
+    a.x_side = side;
+    return launch_quantize(fmt, a, static_cast<cudaStream_t>(stream));
+}
+
+int dequantize(int fmt, const void* codes, const void* side, int64_t rows, int64_t K, float* out, void* stream) {
+    if (!codes || !side || !out) {
+        set_last_error("dequantize: NULL pointer");
+        return RESQ_ERR_NULL;
+    }
+    if (rows <= 0 || K <= 0 || K % block_of(fmt) != 0) {
+        set_last_error("dequantize: bad shape");
+        return RESQ_ERR_SHAPE;
+    }
+    return launch_dequantize(fmt, static_cast<const uint8_t*>(codes), side, rows, K, out, static_cast<cudaStream_t>(stream));
+}
+
+// carve [header | scores | flags] from the front of a workspace
+void carve_quant_scratch(uint8_t* ws, int64_t M, int64_t K, int pattern, QuantArgs& a, size_t& used) {
+    a.status = reinterpret_cast<DeviceStatus*>(ws);
+    used = kWsHeader;
+    size_t n = 0;
+    if (pattern == RESQ_S_CHAN50) n = (size_t)K;
+    if (pattern == RESQ_S_BLOCK32x64_50) n = (size_t)(M / kBlkRows) * (size_t)(K / kBlkCols);
+    if (n) {
+        a.scores = reinterpret_cast<double*>(ws + used);
+        used += align_up(n * sizeof(double), 256);
+        a.keep_flags = ws + used;
+        used += align_up(n, 256);
+    }
+}
+
+int residual_mask(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, int pattern, void* x_codes, void* x_side,
+                  void* r_codes, void* r_side, void* mask_bits, void* workspace, size_t ws_bytes, void* stream) {
+    int rc = check_matrix(X, M, K, ldx, fmt, "X");
+    if (rc) return rc;
+    rc = check_pattern(pattern, M);
+    if (rc) return rc;
+    rc = check_workspace(workspace, ws_bytes, resq_residual_mask_workspace_bytes(M, K, pattern));
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kWsHeader, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(status)");
+    QuantArgs a;
+    memset(&a, 0, sizeof(a));
+    a.X = static_cast<const __nv_bfloat16*>(X);
+    a.M = M;
+    a.K = K;
+    a.ldx = ldx;
+    a.pattern = pattern;
+    a.x_codes = static_cast<uint8_t*>(x_codes);
+    a.x_side = x_side;
+    if (pattern != RESQ_S_NONE) {
+        a.r_codes = static_cast<uint8_t*>(r_codes);
+        a.r_side = r_side;
+        a.mask_bits = static_cast<uint8_t*>(mask_bits);
+    }
+    size_t used = 0;
+    carve_quant_scratch(static_cast<uint8_t*>(workspace), M, K, pattern, a, used);
+    return launch_quantize(fmt, a, st);
+}
+
+size_t linear_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K, int pattern) {
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    size_t b = kWsHeader + quant_scratch_bytes(M, K, pattern);
+    b += align_up((size_t)M * (size_t)K * 2, 256);                            // bf16 image of deq Q(X)
+    if (pattern != RESQ_S_NONE) b += align_up((size_t)M * (size_t)K * 2, 256);  // bf16 image of S(deq Q(dX))
+    int splits = fmt == kHiF4 ? gemm_hif4_pick_splits(M, N, K) : 1;
+    if (splits > 1) b += align_up((size_t)splits * (size_t)M * (size_t)N * 4, 256);
+    return b;
+}
+
+int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_side, int64_t N,
+           int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    int rc = check_matrix(X, M, K, ldx, fmt, "X");
+    if (rc) return rc;
+    rc = check_pattern(pattern, M);
+    if (rc) return rc;
+    if (!w_codes || !w_side || !Y) {
+        set_last_error("linear: NULL weight or output pointer");
+        return RESQ_ERR_NULL;
+    }
+    if (N <= 0) {
+        set_last_error("linear: N=%lld", (long long)N);
+        return RESQ_ERR_SHAPE;
+    }
+    if (out_dtype != RESQ_OUT_BF16 && out_dtype != RESQ_OUT_F32) {
+        set_last_error("unknown output type %d", out_dtype);
+        return RESQ_ERR_PATTERN;
+    }
+    if (!aligned16(Y) || !aligned16(w_codes) || !aligned16(w_side) || ldy < N ||
+        ldy % (out_dtype == RESQ_OUT_BF16 ? 8 : 4) != 0) {
+        set_last_error("linear: Y / weights need 16-byte aligned bases, ldy >= N and 16-byte aligned rows");
+        return RESQ_ERR_ALIGN;
+    }
+    rc = check_workspace(workspace, ws_bytes, linear_workspace_bytes(fmt, M, N, K, pattern));
+    if (rc) return rc;
+    if (fmt != kHiF4) {
+        set_last_error("the MXFP4 GEMM is not built yet");
+        return RESQ_ERR_PATTERN;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kWsHeader, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(status)");
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    QuantArgs a;
+    memset(&a, 0, sizeof(a));
+    a.X = static_cast<const __nv_bfloat16*>(X);
+    a.M = M;
+    a.K = K;
+    a.ldx = ldx;
+    a.pattern = pattern;
+    size_t used = 0;
+    carve_quant_scratch(ws, M, K, pattern, a, used);
+    a.a_bf16 = reinterpret_cast<__nv_bfloat16*>(ws + used);
+    used += align_up((size_t)M * (size_t)K * 2, 256);
+    if (pattern != RESQ_S_NONE) {
+        a.r_bf16 = reinterpret_cast<__nv_bfloat16*>(ws + used);
+        used += align_up((size_t)M * (size_t)K * 2, 256);
+    }
+    rc = launch_quantize(fmt, a, st);
+    if (rc) return rc;
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.a_bf16 = a.a_bf16;
+    g.r_bf16 = a.r_bf16;
+    g.w_codes = static_cast<const uint8_t*>(w_codes);
+    g.w_side = w_side;
+    g.M = M;
+    g.N = N;
+    g.K = K;
+    g.Y = Y;
+    g.out_dtype = out_dtype;
+    g.ldy = ldy;
+    g.splits = gemm_hif4_pick_splits(M, N, K);
+    g.splitk_partials = g.splits > 1 ? reinterpret_cast<float*>(ws + used) : nullptr;
+    g.status = a.status;
+    return launch_gemm_hif4(g, st);
+}
+
+}  // namespace
+}  // namespace resq
+
+using namespace resq;
+
+extern "C" {
+
+size_t hif4_codes_bytes(int64_t rows, int64_t K) { return rows > 0 && K > 0 ? (size_t)rows * (size_t)K / 2 : 0; }
+size_t hif4_meta_bytes(int64_t rows, int64_t K) { return rows > 0 && K > 0 ? (size_t)rows * (size_t)(K / kHif4Block) * 4 : 0; }
+size_t mxfp4_codes_bytes(int64_t rows, int64_t K) { return rows > 0 && K > 0 ? (size_t)rows * (size_t)K / 2 : 0; }
+size_t mxfp4_scale_bytes(int64_t rows, int64_t K) { return rows > 0 && K > 0 ? (size_t)rows * (size_t)(K / kMxBlock) : 0; }
+size_t resq_mask_bytes(int64_t M, int64_t K) { return M > 0 && K > 0 ? (size_t)M * (size_t)K / 8 : 0; }
+
+size_t resq_residual_mask_workspace_bytes(int64_t M, int64_t K, int pattern) {
+    if (M <= 0 || K <= 0) return kWsHeader;
+    return kWsHeader + quant_scratch_bytes(M, K, pattern);
+}
+size_t hif4_resq_workspace_bytes(int64_t M, int64_t N, int64_t K, int pattern) {
+    return linear_workspace_bytes(kHiF4, M, N, K, pattern);
+}
+size_t mxfp4_resq_workspace_bytes(int64_t M, int64_t N, int64_t K, int pattern) {
+    return linear_workspace_bytes(kMXFP4, M, N, K, pattern);
+}
+
+int hif4_pack_weight(const void* W, int64_t N, int64_t K, int64_t ldw, void* w_codes, void* w_meta, void* stream) {
+    return quantize_only(kHiF4, W, N, K, ldw, w_codes, w_meta, stream, "W");
+}
+int mxfp4_pack_weight(const void* W, int64_t N, int64_t K, int64_t ldw, void* w_codes, void* w_scale, void* stream) {
+    return quantize_only(kMXFP4, W, N, K, ldw, w_codes, w_scale, stream, "W");
+}
+int hif4_quantize_act(const void* X, int64_t M, int64_t K, int64_t ldx, void* x_codes, void* x_meta, void* stream) {
+    return quantize_only(kHiF4, X, M, K, ldx, x_codes, x_meta, stream, "X");
+}
+int mxfp4_quantize_act(const void* X, int64_t M, int64_t K, int64_t ldx, void* x_codes, void* x_scale, void* stream) {
+    return quantize_only(kMXFP4, X, M, K, ldx, x_codes, x_scale, stream, "X");
+}
+int hif4_dequantize(const void* codes, const void* meta, int64_t rows, int64_t K, float* out, void* stream) {
+    return dequantize(kHiF4, codes, meta, rows, K, out, stream);
+}
+int mxfp4_dequantize(const void* codes, const void* scale, int64_t rows, int64_t K, float* out, void* stream) {
+    return dequantize(kMXFP4, codes, scale, rows, K, out, stream);
+}
+
+int resq_residual_mask(const void* X, int64_t M, int64_t K, int64_t ldx, int pattern, void* x_codes, void* x_meta,
+                       void* r_codes, void* r_meta, void* mask_bits, void* workspace, size_t ws_bytes, void* stream) {
+    return residual_mask(kHiF4, X, M, K, ldx, pattern, x_codes, x_meta, r_codes, r_meta, mask_bits, workspace, ws_bytes,
+                         stream);
+}
+int mxfp4_residual_mask(const void* X, int64_t M, int64_t K, int64_t ldx, int pattern, void* x_codes, void* x_scale,
+                        void* r_codes, void* r_scale, void* mask_bits, void* workspace, size_t ws_bytes, void* stream) {
+    return residual_mask(kMXFP4, X, M, K, ldx, pattern, x_codes, x_scale, r_codes, r_scale, mask_bits, workspace,
+                         ws_bytes, stream);
+}
+
+int hif4_resq_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_meta, int64_t N,
+                     int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    return linear(kHiF4, X, M, K, ldx, w_codes, w_meta, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream);
+}
+int mxfp4_resq_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_scale,
+                      int64_t N, int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes,
+                      void* stream) {
+    return linear(kMXFP4, X, M, K, ldx, w_codes, w_scale, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream);
+}
+
+int resq_check(void* workspace, void* stream) {
+    if (!workspace) {
+        set_last_error("resq_check: workspace is NULL");
+        return RESQ_ERR_NULL;
+    }
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    DeviceStatus st;
+    e = cudaMemcpy(&st, workspace, sizeof(st), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
+    if (st.code != RESQ_OK) set_last_error("device status %d (wait %d gave up in block %d)", st.code, st.where, st.block);
+    return st.code;
+}
+
+const char* resq_last_error(void) { return g_last_error; }
+
+}  // extern "C"

@@ -1,0 +1,75 @@
+// Shared declarations of the ResQ CUDA library (sm_100a).  Internal; the public contract is include/resq.h.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "../../include/resq.h"
+
+namespace resq {
+
+enum Format : int { kHiF4 = 0, kMXFP4 = 1 };
+
+constexpr int kHif4Block = 64;
+constexpr int kMxBlock = 32;
+constexpr int kE6M2Bias = 48;      // S1 = (1 + Mn/4) * 2^(E - 48)
+constexpr int kBlkRows = 32;       // S^{32x64}: 32 token rows ...
+constexpr int kBlkCols = 64;       // ... by 64 channels
+constexpr size_t kWsHeader = 256;  // status word + padding at the start of every workspace
+
+// Device status word layout (first 16 bytes of the workspace).
+struct DeviceStatus {
+    int code;    // resq_status
+    int where;   // which wait gave up (kernel-specific tag)
+    int block;   // blockIdx.x of the reporter
+    int pad;
+};
+
+void set_last_error(const char* fmt, ...);
+int cuda_fail(cudaError_t e, const char* what);
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---- quantizer launch description (quantize.cu) ------------------------------------------------
+struct QuantArgs {
+    const __nv_bfloat16* X;
+    int64_t M, K, ldx;
+    int pattern;            // resq_pattern; RESQ_S_NONE => no residual work at all
+    // canonical packed outputs (any may be null)
+    uint8_t* x_codes;
+    void* x_side;           // u32 meta (HiF4) or u8 scale (MXFP4)
+    uint8_t* r_codes;
+    void* r_side;
+    uint8_t* mask_bits;
+    // expanded operands for the GEMM (any may be null): exact bf16 images of deq Q(X) and S(deq Q(dX))
+    __nv_bfloat16* a_bf16;  // [M, K]
+    __nv_bfloat16* r_bf16;  // [M, K]
+    // scratch
+    double* scores;         // CHAN50: [K]; BLOCK: [(M/32) * (K/64)]
+    uint8_t* keep_flags;    // CHAN50: [K]; BLOCK: [(M/32) * (K/64)]
+    DeviceStatus* status;
+};
+
+int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream);
+int launch_dequantize(int fmt, const uint8_t* codes, const void* side, int64_t rows, int64_t K, float* out,
+                      cudaStream_t stream);
+size_t quant_scratch_bytes(int64_t M, int64_t K, int pattern);  // scores + keep flags (without header)
+
+// ---- GEMM launch description (gemm_hif4.cu / gemm_mxfp4.cu) -------------------------------------
+struct GemmArgs {
+    const __nv_bfloat16* a_bf16;   // [M, K] exact bf16 image of deq Q(X)
+    const __nv_bfloat16* r_bf16;   // [M, K] masked residual image, or null (pattern NONE)
+    const uint8_t* w_codes;        // [N, K/2]
+    const void* w_side;            // [N, K/64] u32 or [N, K/32] u8
+    int64_t M, N, K;
+    void* Y;
+    int out_dtype;
+    int64_t ldy;
+    float* splitk_partials;        // [splits, M, N] fp32 when splits > 1
+    int splits;
+    DeviceStatus* status;
+};
+int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream);
+int gemm_hif4_pick_splits(int64_t M, int64_t N, int64_t K);
+
+}  // namespace resq
