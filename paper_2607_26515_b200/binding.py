@@ -181,7 +181,8 @@ def resq_linear(X: torch.Tensor, w_codes: torch.Tensor, w_side: torch.Tensor, pa
     M, K = X.shape
     N = w_codes.shape[0]
     if Y is None:
-        Y = torch.empty((M, N), dtype=out_dtype, device=X.device)
+        ld = (N + 7) // 8 * 8  # rows of Y start on 16-byte boundaries
+        Y = torch.empty((M, ld), dtype=out_dtype, device=X.device)[:, :N]
     if Y.dtype not in (torch.bfloat16, torch.float32):
         raise ValueError("Y must be bf16 or fp32")
     if workspace is None:

@@ -1,0 +1,105 @@
+"""Parity of hif4_resq_linear (Eq. (5)) with the CPU oracle, through the C ABI.
+
+Tolerance (fp32 accumulation on the GPU vs fp64 in the oracle; products are exact on both sides):
+    |y - y_ref| <= 2e-3 * |y_ref| + 1e-5 * sum_k |(a + r)[m,k] * w[n,k]|
+The second term is the cancellation floor: fp32 accumulation of K exact products errs by about
+sqrt(K) * 2^-24 of that sum.  bf16 output adds one rounding (2^-9 relative)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from workloads import CONFIGS, bf16_bits_to_f32, f32_to_bf16_bits, make_layer
+
+pytestmark = pytest.mark.gpu
+
+
+def rq():
+    import paper_2607_26515_b200 as m
+    return m
+
+
+def to_dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def synth_xw(seed, M, K, N, n_out=4, w_std=0.02):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    x[:, rng.choice(K, n_out, replace=False)] *= 50.0
+    w = (rng.standard_normal((N, K)) * w_std).astype(np.float32)
+    return f32_to_bf16_bits(x), f32_to_bf16_bits(w)
+
+
+def check_close(y, ref, abs_sum, bf16_out=False):
+    y = np.asarray(y, dtype=np.float64)
+    tol = 2e-3 * np.abs(ref) + 1e-5 * abs_sum
+    if bf16_out:
+        tol = tol + 2.0 ** -8 * np.abs(ref)
+    err = np.abs(y - ref)
+    bad = err > tol
+    assert not bad.any(), (f"{bad.sum()} of {bad.size} outside tolerance; worst ratio "
+                           f"{(err / np.maximum(tol, 1e-300)).max():.3g} at {np.unravel_index(np.argmax(err / np.maximum(tol, 1e-300)), err.shape)}")
+
+
+def run_case(xb, wb, pattern, fmt="hif4", out_dtype=torch.float32):
+    m = rq()
+    want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern, fmt)
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    M, K = xb.shape
+    N = wb.shape[0]
+    wsz = m.resq_workspace_bytes(M, N, K, pattern, fmt)
+    work = m.alloc_workspace(wsz)
+    y = m.resq_linear(to_dev(xb), wc, ws, pattern, fmt, out_dtype=out_dtype, workspace=work)
+    assert m.check(work) == 0, m.last_error()
+    check_close(y.float().cpu().numpy(), want["y"], want["abs_sum"], bf16_out=out_dtype == torch.bfloat16)
+    return y
+
+
+ALL = [oracle.S_NONE, oracle.S_DENSE, oracle.S_2_4, oracle.S_ROW50, oracle.S_CHAN50, oracle.S_BLOCK]
+
+
+@pytest.mark.parametrize("pattern", ALL)
+def test_linear_one_tile(pattern):
+    xb, wb = synth_xw(1, 128, 256, 256)
+    run_case(xb, wb, pattern)
+
+
+@pytest.mark.parametrize("pattern", ALL)
+@pytest.mark.parametrize("shape", [(64, 2048, 2048), (96, 192, 80), (160, 704, 328), (288, 1024, 1000), (32, 64, 16)])
+def test_linear_shapes(pattern, shape):
+    M, K, N = shape
+    xb, wb = synth_xw(M + N + pattern, M, K, N, n_out=max(1, K // 256))
+    run_case(xb, wb, pattern)
+
+
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4])
+def test_linear_bf16_output(pattern):
+    xb, wb = synth_xw(7, 200, 512, 520)
+    run_case(xb, wb, pattern, out_dtype=torch.bfloat16)
+
+
+def test_linear_config0_tiny():
+    cfg = CONFIGS[0]
+    xb, wb = make_layer(cfg, 0)
+    run_case(xb, wb, cfg.patterns[0])
+    run_case(xb, wb, cfg.patterns[0], out_dtype=torch.bfloat16)
+
+
+def test_linear_deterministic():
+    xb, wb = synth_xw(9, 256, 2048, 2560)
+    m = rq()
+    wc, ws = m.pack_weight(to_dev(wb))
+    y1 = m.resq_linear(to_dev(xb), wc, ws, m.S_2_4, out_dtype=torch.float32).clone()
+    y2 = m.resq_linear(to_dev(xb), wc, ws, m.S_2_4, out_dtype=torch.float32)
+    assert torch.equal(y1, y2)
+
+
+def test_linear_zero_input_gives_zero():
+    m = rq()
+    x = torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda")
+    _, wb = synth_xw(3, 8, 256, 64)
+    wc, ws = m.pack_weight(to_dev(wb))
+    for pattern in ALL:
+        y = m.resq_linear(x, wc, ws, pattern, out_dtype=torch.float32)
+        assert not y.any()
