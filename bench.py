@@ -1,0 +1,375 @@
+#!/usr/bin/env python
+"""Benchmark of the Rollout-ResQ FP4 linear path (Eq. (5)) on B200.
+
+A "step" is one pass of the whole hot path -- quantize X, residual, re-quantize, select, two-term
+GEMM against packed HiF4 weights -- over the four linears of one transformer block of the
+workload (default: the Qwen2.5-3B decode-shaped configuration, M = 256 tokens, S_2:4).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--pattern P] [--format F]
+    python bench.py --impl reference ...        # times the CPU oracle on a bounded sample
+
+Prints ONE JSON line on stdout (rank 0); `--verbose` adds a per-layer table on stderr.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from workloads import CONFIGS, make_activation, make_weight  # noqa: E402
+
+METRIC = "hif4_resq_linear TFLOP/s & GB/s at 1 B200; % of FP4-tensor/HBM roofline"
+L2_BYTES = 126 * 1024 * 1024
+PATTERN_IDS = {"none": 0, "dense": 1, "2:4": 2, "row50": 3, "chan50": 4, "block": 5}
+RHO = {0: 0.0, 1: 1.0, 2: 0.5, 3: 0.5, 4: 0.5, 5: 0.5}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------- algorithmic work
+
+def layer_flops(M, N, K, pattern):
+    """2 M N K (1 + rho): the dense term plus the kept half (or all) of the residual term (Section 5.4)."""
+    return 2.0 * M * N * K * (1.0 + RHO[pattern])
+
+
+def layer_bytes(M, N, K, pattern, fmt):
+    """Bytes the method must move per call: bf16 X in, packed W in, bf16 Y out."""
+    w_bits = 4.5 if fmt == "hif4" else 4.25
+    return 2.0 * M * K + w_bits / 8.0 * N * K + 2.0 * M * N
+
+
+# ----------------------------------------------------------------------------- clocks sampler
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._reader, daemon=True)
+        self.thread.start()
+
+    def _reader(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        rows = [r for (t, r) in self.rows if t0 - 0.05 <= t <= t1 + 0.15 and len(r) >= 9] or \
+               [r for (_, r) in self.rows if len(r) >= 9]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = [float(r[1]) for r in rows]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for r in rows for n, v in zip(names, r[5:9]) if v.lower().startswith("active")})
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": float(rows[0][2]), "reasons": reasons,
+                "samples": len(rows), "power_w_max": max(float(r[3]) for r in rows)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle timing
+
+def time_oracle(cfg, pattern, fmt, budget_s=20.0):
+    """Times the oracle, as it stands, on a bounded sample of the workload: every layer of the config, on
+    the first rows of X (all of them if that fits the budget).  Returns (TFLOP/s, cores, description, s)."""
+    import oracle
+    from workloads import bf16_bits_to_f32
+    threads = oracle.num_threads()
+    macs_per_row = sum(2.0 * l.K * l.N for l in cfg.layers)          # two fp64 sweeps per output element
+    rate = 0.6e9 * threads                                            # rough fp64 MAC/s of the plain triple loop
+    rows = int(max(32, min(cfg.M, budget_s * rate / macs_per_row)))
+    rows -= rows % 32
+    flops, dt = 0.0, 0.0
+    for li, spec in enumerate(cfg.layers):
+        x = bf16_bits_to_f32(make_activation(cfg, li, M=rows))
+        w = bf16_bits_to_f32(make_weight(cfg, li))
+        t0 = time.perf_counter()
+        oracle.resq_linear(x, w, pattern, fmt, want_abs=False)
+        dt += time.perf_counter() - t0
+        flops += layer_flops(rows, spec.N, spec.K, pattern)
+    sample = (f"{cfg.name}: all {len(cfg.layers)} layers, first {rows} of {cfg.M} token rows "
+              f"(weight packing, quantizer, masks and fp64 product all timed)")
+    return flops / dt / 1e12, threads, sample, dt
+
+
+# ----------------------------------------------------------------------------- main
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=1, help="index into the workload configs (default 1: 3B decode)")
+    ap.add_argument("--pattern", default=None, help="none|dense|2:4|row50|chan50|block (default: the config's)")
+    ap.add_argument("--format", default="hif4", choices=["hif4", "mxfp4"])
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--out-dtype", default="bf16", choices=["bf16", "f32"])
+    ap.add_argument("--layers", default=None, help="comma-separated subset of the config's layers (profiling aid)")
+    ap.add_argument("--tokens", type=int, default=None, help="override M (profiling aid; not the benchmark workload)")
+    ap.add_argument("--skip-e2e", action="store_true", help="skip the end-to-end and per-kernel passes (profiling aid)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--verbose", action="store_true")
+    args = ap.parse_args()
+
+    cfg = CONFIGS[args.config]
+    if args.layers or args.tokens:
+        import dataclasses
+        keep = args.layers.split(",") if args.layers else [l.name for l in cfg.layers]
+        cfg = dataclasses.replace(cfg, layers=tuple(l for l in cfg.layers if l.name in keep),
+                                  M=args.tokens or cfg.M, name=cfg.name + " (subset)")
+    pattern = PATTERN_IDS[args.pattern] if args.pattern else cfg.patterns[0]
+    pattern_name = {v: k for k, v in PATTERN_IDS.items()}[pattern]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    config_desc = {
+        "workload": f"{cfg.name}: M={cfg.M}, layers " + ", ".join(f"{l.name} {l.K}->{l.N}" for l in cfg.layers),
+        "pattern": pattern_name, "format": args.format, "out_dtype": args.out_dtype,
+        "parallelism": "replicas only (one independent copy of the step per GPU)",
+    }
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        vals = []
+        for _ in range(max(1, min(args.warmup, 1))):
+            time_oracle(cfg, pattern, args.format, budget_s=3.0)
+        info = None
+        for _ in range(max(1, min(args.steps, 3))):
+            info = time_oracle(cfg, pattern, args.format, budget_s=8.0)
+            vals.append(info[0])
+        v = statistics.median(vals)
+        line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "TFLOP/s", "n_gpus": args.gpus,
+                "steps": len(vals), "warmup": 1, "ms_per_step": info[3] * 1e3, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config_desc,
+                "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": info[1], "kind": "oracle", "sample": info[2]},
+                "e2e": {"value": v, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return
+
+    import torch
+    import paper_2607_26515_b200 as rq
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    rq.lib()  # fail loudly if the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    out_dtype = torch.bfloat16 if args.out_dtype == "bf16" else torch.float32
+    fmt = args.format
+
+    # ---- inputs: generated once on the host, packed once (weights are packed per policy update, not per call)
+    layers = []
+    w_bytes_total = 0
+    for li, spec in enumerate(cfg.layers):
+        xb = make_activation(cfg, li)
+        wb = make_weight(cfg, li)
+        x_host = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
+        w_dev = torch.from_numpy(wb.view(np.int16)).view(torch.bfloat16).to(dev)
+        wc, ws = rq.pack_weight(w_dev, fmt)
+        del w_dev
+        w_bytes_total += wc.numel() + ws.numel() * ws.element_size()
+        layers.append({"spec": spec, "x_host": x_host, "wc": wc, "ws": ws})
+    # rotate over enough copies of the packed weights that a step never finds them in L2
+    n_sets = max(2, int(np.ceil(1.5 * L2_BYTES / max(1, w_bytes_total))))
+    n_sets = min(n_sets, 16)
+    for L in layers:
+        spec = L["spec"]
+        L["w_sets"] = [(L["wc"], L["ws"])] + [(L["wc"].clone(), L["ws"].clone()) for _ in range(n_sets - 1)]
+        L["x_sets"] = [L["x_host"].to(dev) for _ in range(n_sets)]
+        L["y"] = torch.empty((cfg.M, spec.N), dtype=out_dtype, device=dev)
+        L["y_host"] = torch.empty((cfg.M, spec.N), dtype=out_dtype).pin_memory()
+        L["x_stage"] = torch.empty_like(L["x_sets"][0])
+        L["work"] = rq.alloc_workspace(rq.resq_workspace_bytes(cfg.M, spec.N, spec.K, pattern, fmt), dev)
+    config_desc["l2"] = (f"rotating {n_sets} copies of weights and activations "
+                         f"({n_sets * w_bytes_total / 1e6:.0f} MB of packed weights > 126 MB L2)")
+
+    def step(i):
+        k = i % n_sets
+        for L in layers:
+            wc, ws = L["w_sets"][k]
+            rq.resq_linear(L["x_sets"][k], wc, ws, pattern, fmt, Y=L["y"], workspace=L["work"])
+
+    def step_e2e(i):
+        k = i % n_sets
+        for L in layers:
+            wc, ws = L["w_sets"][k]
+            L["x_stage"].copy_(L["x_host"], non_blocking=True)           # host -> device, pinned
+            rq.resq_linear(L["x_stage"], wc, ws, pattern, fmt, Y=L["y"], workspace=L["work"])
+            L["y_host"].copy_(L["y"], non_blocking=True)                 # device -> host
+        torch.cuda.current_stream().synchronize()
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        barrier()
+        t1 = time.time()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, t0, t1
+
+    warmup = max(3, args.warmup)
+    for i in range(warmup):
+        step(i)
+    for L in layers:
+        if rq.check(L["work"]) != 0:
+            raise SystemExit("device status: " + rq.last_error())
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    launches0 = rq.kernel_launches()
+    ms, t0, t1 = timed(step, args.steps)
+    launches = rq.kernel_launches() - launches0
+    # keep the GPU busy a little longer so that the 100 ms sampler certainly sees the loaded state
+    t_load0 = time.time()
+    reps = 0
+    while time.time() - t_load0 < 0.6:
+        for i in range(20):
+            step(i)
+        torch.cuda.synchronize()
+        reps += 1
+    t_load1 = time.time()
+    clocks = sampler.stop(t0, t_load1) if rank == 0 else None
+
+    flops_step = sum(layer_flops(cfg.M, L["spec"].N, L["spec"].K, pattern) for L in layers)
+    bytes_step = sum(layer_bytes(cfg.M, L["spec"].N, L["spec"].K, pattern, fmt) for L in layers)
+    ms_per_step = ms / args.steps
+    tflops = world * flops_step / (ms_per_step * 1e-3) / 1e12
+    gbs = world * bytes_step / (ms_per_step * 1e-3) / 1e9
+
+    if args.skip_e2e:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": tflops, "unit": "TFLOP/s", "ms_per_step": ms_per_step,
+                              "config": config_desc, "note": "profiling aid run: no e2e / roofline passes"}))
+        return
+    # ---- end-to-end: host buffers, copies inside the timed region
+    for i in range(3):
+        step_e2e(i)
+    ms_e2e, _, _ = timed(step_e2e, args.steps)
+    e2e_tflops = world * flops_step / (ms_e2e / args.steps * 1e-3) / 1e12
+    h2d = sum(L["x_host"].numel() * 2 for L in layers)
+    d2h = sum(L["y_host"].numel() * L["y_host"].element_size() for L in layers)
+
+    # ---- per-kernel device time (CUDA events around every launch, on the launching stream)
+    rq.profile_enable(True)
+    rq.profile_read()
+    barrier()
+    for i in range(args.steps):
+        step(i)
+    torch.cuda.synchronize()
+    prof = rq.profile_read()
+    rq.profile_enable(False)
+    gemm_ms, gemm_n = prof["gemm"]
+    quant_ms, quant_n = prof["quantize"]
+    peaks, peak_kind = load_peaks()
+    gemm_tflops = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
+    roofline = {
+        "kernel": "gemm_hif4_kernel (tcgen05 kind::f16 on bf16-expanded HiF4)", "bound": "tensor",
+        "achieved": gemm_tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+        "frac": (gemm_tflops / peaks["bf16_tflops"]) if gemm_tflops else None,
+        "peak_source": f"bf16 burst, {peak_kind}", "traffic": None,
+        "avg_launch_us": gemm_ms * 1e3 / max(1, gemm_n), "launches": gemm_n,
+        "quantizer_avg_launch_us": quant_ms * 1e3 / max(1, quant_n),
+        "quantizer_share_of_kernel_time": quant_ms / max(1e-9, sum(v[0] for v in prof.values())),
+        "hbm_frac_of_step": gbs / world / peaks["hbm_gbs"],
+        "frac_of_fp8_nominal": (gemm_tflops / 4500.0) if gemm_tflops else None,
+        "frac_of_fp4_nominal": (gemm_tflops / 9000.0) if gemm_tflops else None,
+    }
+
+    if args.verbose and rank == 0:
+        rq.profile_enable(True)
+        for L in layers:
+            spec = L["spec"]
+            rq.profile_read()
+            for i in range(10):
+                wc, ws = L["w_sets"][i % n_sets]
+                rq.resq_linear(L["x_sets"][i % n_sets], wc, ws, pattern, fmt, Y=L["y"], workspace=L["work"])
+            torch.cuda.synchronize()
+            pr = rq.profile_read()
+            f = layer_flops(cfg.M, spec.N, spec.K, pattern)
+            g_us = pr["gemm"][0] * 100.0
+            print(f"[layer {spec.name:8s}] K={spec.K:6d} N={spec.N:6d}  quant {pr['quantize'][0]*100:8.1f} us  "
+                  f"select {pr['select'][0]*100:7.1f} us  gemm {g_us:8.1f} us  reduce {pr['splitk_reduce'][0]*100:6.1f} us  "
+                  f"gemm {f / (g_us * 1e-6) / 1e12:7.1f} TFLOP/s", file=sys.stderr)
+        rq.profile_enable(False)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, cores, sample, dt = time_oracle(cfg, pattern, fmt)
+        cpu_baseline = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample,
+                        "seconds": dt}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config_desc,
+            "gb_per_s": gbs, "clocks": clocks,
+            "e2e": {"value": e2e_tflops, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

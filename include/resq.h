@@ -134,6 +134,18 @@ RESQ_API int mxfp4_resq_linear(const void* X_bf16, int64_t M, int64_t K, int64_t
 RESQ_API int resq_check(void* workspace, void* stream);
 RESQ_API const char* resq_last_error(void);
 
+/* ---- diagnostics (no counterpart in the paper) -----------------------------------------------------
+ * resq_kernel_launches: number of kernels this library has launched in the process so far.
+ * resq_profile_enable(1): from now on every kernel launch is bracketed by a pair of CUDA events on its
+ * stream (this perturbs timing slightly; leave it off when measuring whole-call time).
+ * resq_profile_read: synchronizes on the recorded events, adds the device time (ms) and the number of
+ * launches per kernel kind into the two arrays of 4 entries (0 = quantizer/residual/mask pass,
+ * 1 = top-k select and mask apply, 2 = GEMM, 3 = split-K reduce; either array may be NULL) and
+ * clears the records. */
+RESQ_API int64_t resq_kernel_launches(void);
+RESQ_API int resq_profile_enable(int on);
+RESQ_API int resq_profile_read(double* ms_by_kind, int64_t* launches_by_kind);
+
 #ifdef __cplusplus
 }
 #endif

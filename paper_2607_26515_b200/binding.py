@@ -45,6 +45,9 @@ SYMBOLS = {
     "mxfp4_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "resq_check": (_ci, [_vp, _vp]),
     "resq_last_error": (ctypes.c_char_p, []),
+    "resq_kernel_launches": (_i64, []),
+    "resq_profile_enable": (_ci, [_ci]),
+    "resq_profile_read": (_ci, [_vp, _vp]),
 }
 
 _lib: Optional[ctypes.CDLL] = None
@@ -197,3 +200,25 @@ def resq_linear(X: torch.Tensor, w_codes: torch.Tensor, w_side: torch.Tensor, pa
 def check(workspace: torch.Tensor, stream=None) -> int:
     """resq_check: synchronize and return the device status word."""
     return int(lib().resq_check(workspace.data_ptr(), _stream(stream)))
+
+
+# ------------------------------------------------------------------ diagnostics
+
+KERNEL_KINDS = ("quantize", "select", "gemm", "splitk_reduce")
+
+
+def kernel_launches() -> int:
+    """resq_kernel_launches: kernels launched by the library in this process so far."""
+    return int(lib().resq_kernel_launches())
+
+
+def profile_enable(on: bool) -> None:
+    _check(lib().resq_profile_enable(1 if on else 0))
+
+
+def profile_read():
+    """resq_profile_read -> {kind: (device ms, launches)} since the last read."""
+    ms = (ctypes.c_double * 4)()
+    n = (ctypes.c_int64 * 4)()
+    _check(lib().resq_profile_read(ctypes.cast(ms, ctypes.c_void_p), ctypes.cast(n, ctypes.c_void_p)))
+    return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}

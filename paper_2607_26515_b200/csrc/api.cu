@@ -2,9 +2,12 @@
 // The contract of every entry point is stated in include/resq.h.
 #include "common.cuh"
 
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 namespace resq {
 
@@ -21,6 +24,37 @@ int cuda_fail(cudaError_t e, const char* what) {
     if (e == cudaSuccess) return RESQ_OK;
     set_last_error("%s: %s", what, cudaGetErrorString(e));
     return RESQ_ERR_CUDA;
+}
+
+// ---- diagnostics: launch counter and optional per-kernel event timing ---------------------------
+namespace {
+std::atomic<long long> g_launches{0};
+std::atomic<int> g_profile{0};
+struct ProfRec {
+    int kind;
+    cudaEvent_t start, stop;
+};
+std::mutex g_prof_mu;
+std::vector<ProfRec*> g_prof;
+}  // namespace
+
+LaunchScope::LaunchScope(int kind, cudaStream_t stream) : kind_(kind), stream_(stream), rec_(nullptr) {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (!g_profile.load(std::memory_order_relaxed)) return;
+    ProfRec* r = new ProfRec{kind, nullptr, nullptr};
+    if (cudaEventCreate(&r->start) != cudaSuccess || cudaEventCreate(&r->stop) != cudaSuccess) {
+        delete r;
+        return;
+    }
+    cudaEventRecord(r->start, stream);
+    rec_ = r;
+}
+LaunchScope::~LaunchScope() {
+    if (!rec_) return;
+    ProfRec* r = static_cast<ProfRec*>(rec_);
+    cudaEventRecord(r->stop, stream_);
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof.push_back(r);
 }
 
 namespace {
@@ -299,5 +333,39 @@ int resq_check(void* workspace, void* stream) {
 }
 
 const char* resq_last_error(void) { return g_last_error; }
+
+int64_t resq_kernel_launches(void) { return (int64_t)g_launches.load(); }
+
+int resq_profile_enable(int on) {
+    g_profile.store(on ? 1 : 0);
+    return RESQ_OK;
+}
+
+int resq_profile_read(double* ms_by_kind, int64_t* launches_by_kind) {
+    std::vector<ProfRec*> recs;
+    {
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        recs.swap(g_prof);
+    }
+    for (int k = 0; k < kNumKinds; ++k) {
+        if (ms_by_kind) ms_by_kind[k] = 0.0;
+        if (launches_by_kind) launches_by_kind[k] = 0;
+    }
+    int rc = RESQ_OK;
+    for (ProfRec* r : recs) {
+        float ms = 0.0f;
+        cudaError_t e = cudaEventSynchronize(r->stop);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, r->start, r->stop);
+        if (e != cudaSuccess) rc = cuda_fail(e, "profile event");
+        else {
+            if (ms_by_kind) ms_by_kind[r->kind] += (double)ms;
+            if (launches_by_kind) launches_by_kind[r->kind] += 1;
+        }
+        cudaEventDestroy(r->start);
+        cudaEventDestroy(r->stop);
+        delete r;
+    }
+    return rc;
+}
 
 }  // extern "C"

@@ -30,6 +30,17 @@ int cuda_fail(cudaError_t e, const char* what);
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Diagnostics (api.cu): every kernel launch of the library is counted; when profiling is enabled a
+// pair of CUDA events brackets each launch on its stream so that per-kernel device time can be read.
+enum KernelKind : int { kKindQuant = 0, kKindSelect = 1, kKindGemm = 2, kKindReduce = 3, kNumKinds = 4 };
+struct LaunchScope {
+    LaunchScope(int kind, cudaStream_t stream);
+    ~LaunchScope();
+    int kind_;
+    cudaStream_t stream_;
+    void* rec_;
+};
+
 // ---- quantizer launch description (quantize.cu) ------------------------------------------------
 struct QuantArgs {
     const __nv_bfloat16* X;

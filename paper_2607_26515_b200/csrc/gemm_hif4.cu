@@ -443,11 +443,15 @@ int launch_variant(const GemmArgs& g, const TileChoice& tc, cudaStream_t stream)
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute(gemm)");
     dim3 grid((unsigned)((g.N + tc.bn - 1) / tc.bn), (unsigned)((g.M + kBM * MT - 1) / (kBM * MT)), (unsigned)tc.splits);
-    kern<<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tr, tw, p);
+    {
+        LaunchScope scope(kKindGemm, stream);
+        kern<<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tr, tw, p);
+    }
     rc = cuda_fail(cudaGetLastError(), "gemm_hif4_kernel launch");
     if (rc) return rc;
     if (tc.splits > 1) {
         int64_t n = g.M * g.N;
+        LaunchScope scope(kKindReduce, stream);
         splitk_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(g.splitk_partials, tc.splits, g.M, g.N, g.Y,
                                                                              p.out_f32, g.ldy);
         rc = cuda_fail(cudaGetLastError(), "splitk_reduce_kernel launch");

@@ -456,6 +456,7 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
         auto kern = fmt == kHiF4 ? quant_row50_kernel<kHiF4> : quant_row50_kernel<kMXFP4>;
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(row50)");
+        LaunchScope scope(kKindQuant, stream);
         kern<<<(unsigned)a.M, kThreads, smem, stream>>>(a);
         return cuda_fail(cudaGetLastError(), "quant_row50_kernel launch");
     }
@@ -469,6 +470,8 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     const int rows_per_cta = pick_rows_per_cta(a.M, a.K, pattern);
     dim3 grid((unsigned)((a.M + rows_per_cta - 1) / rows_per_cta),
               (unsigned)((a.K + (int64_t)kWarpsPerCta * kColsPerWarp - 1) / ((int64_t)kWarpsPerCta * kColsPerWarp)));
+    {
+    LaunchScope scope(kKindQuant, stream);
     if (fmt == kHiF4) {
         if (residual) quant_stream_kernel<kHiF4, true><<<grid, kThreads, 0, stream>>>(a, rows_per_cta);
         else quant_stream_kernel<kHiF4, false><<<grid, kThreads, 0, stream>>>(a, rows_per_cta);
@@ -476,14 +479,17 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
         if (residual) quant_stream_kernel<kMXFP4, true><<<grid, kThreads, 0, stream>>>(a, rows_per_cta);
         else quant_stream_kernel<kMXFP4, false><<<grid, kThreads, 0, stream>>>(a, rows_per_cta);
     }
+    }
     int rc = cuda_fail(cudaGetLastError(), "quant_stream_kernel launch");
     if (rc) return rc;
     if (global_sel) {
-        topk_select_kernel<<<1, kSelThreads, 0, stream>>>(a.scores, (int)nscore, (int)(nscore / 2), a.keep_flags);
+        { LaunchScope scope(kKindSelect, stream);
+        topk_select_kernel<<<1, kSelThreads, 0, stream>>>(a.scores, (int)nscore, (int)(nscore / 2), a.keep_flags); }
         rc = cuda_fail(cudaGetLastError(), "topk_select_kernel launch");
         if (rc) return rc;
         if (a.mask_bits || a.r_bf16) {
             int64_t n = a.M * (a.K / 8);
+            LaunchScope scope(kKindSelect, stream);
             apply_global_mask_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(pattern, a.M, a.K, a.keep_flags,
                                                                                       a.mask_bits, a.r_bf16);
             rc = cuda_fail(cudaGetLastError(), "apply_global_mask_kernel launch");
@@ -496,6 +502,7 @@ int launch_dequantize(int fmt, const uint8_t* codes, const void* side, int64_t r
                       cudaStream_t stream) {
     int64_t n = rows * (K / 8);
     unsigned grid = (unsigned)((n + kThreads - 1) / kThreads);
+    LaunchScope scope(kKindQuant, stream);
     if (fmt == kHiF4) dequant_kernel<kHiF4><<<grid, kThreads, 0, stream>>>(codes, side, rows, K, out);
     else dequant_kernel<kMXFP4><<<grid, kThreads, 0, stream>>>(codes, side, rows, K, out);
     return cuda_fail(cudaGetLastError(), "dequant_kernel launch");
