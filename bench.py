@@ -187,6 +187,7 @@ def main():
 
     import torch
     import paper_2607_26515_b200 as rq
+    from paper_2607_26515_b200.replicas import max_over_ranks
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -256,12 +257,25 @@ def main():
         e1.record()
         barrier()
         t1 = time.time()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(e0.elapsed_time(e1), dev)
         return ms, t0, t1
+
+    def per_layer_table():
+        rq.profile_enable(True)
+        for L in layers:
+            spec = L["spec"]
+            rq.profile_read()
+            for i in range(10):
+                wc, ws = L["w_sets"][i % n_sets]
+                rq.resq_linear(L["x_sets"][i % n_sets], wc, ws, pattern, fmt, Y=L["y"], workspace=L["work"])
+            torch.cuda.synchronize()
+            pr = rq.profile_read()
+            f = layer_flops(cfg.M, spec.N, spec.K, pattern)
+            g_us = pr["gemm"][0] * 100.0
+            print(f"[layer {spec.name:8s}] K={spec.K:6d} N={spec.N:6d}  quant {pr['quantize'][0]*100:8.1f} us  "
+                  f"select {pr['select'][0]*100:7.1f} us  gemm {g_us:8.1f} us  reduce {pr['splitk_reduce'][0]*100:6.1f} us  "
+                  f"gemm {f / (g_us * 1e-6) / 1e12:7.1f} TFLOP/s", file=sys.stderr)
+        rq.profile_enable(False)
 
     warmup = max(3, args.warmup)
     for i in range(warmup):
@@ -294,6 +308,8 @@ def main():
     tflops = world * flops_step / (ms_per_step * 1e-3) / 1e12
     gbs = world * bytes_step / (ms_per_step * 1e-3) / 1e9
 
+    if args.verbose and rank == 0:
+        per_layer_table()
     if args.skip_e2e:
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": tflops, "unit": "TFLOP/s", "ms_per_step": ms_per_step,
@@ -332,23 +348,6 @@ def main():
         "frac_of_fp8_nominal": (gemm_tflops / 4500.0) if gemm_tflops else None,
         "frac_of_fp4_nominal": (gemm_tflops / 9000.0) if gemm_tflops else None,
     }
-
-    if args.verbose and rank == 0:
-        rq.profile_enable(True)
-        for L in layers:
-            spec = L["spec"]
-            rq.profile_read()
-            for i in range(10):
-                wc, ws = L["w_sets"][i % n_sets]
-                rq.resq_linear(L["x_sets"][i % n_sets], wc, ws, pattern, fmt, Y=L["y"], workspace=L["work"])
-            torch.cuda.synchronize()
-            pr = rq.profile_read()
-            f = layer_flops(cfg.M, spec.N, spec.K, pattern)
-            g_us = pr["gemm"][0] * 100.0
-            print(f"[layer {spec.name:8s}] K={spec.K:6d} N={spec.N:6d}  quant {pr['quantize'][0]*100:8.1f} us  "
-                  f"select {pr['select'][0]*100:7.1f} us  gemm {g_us:8.1f} us  reduce {pr['splitk_reduce'][0]*100:6.1f} us  "
-                  f"gemm {f / (g_us * 1e-6) / 1e12:7.1f} TFLOP/s", file=sys.stderr)
-        rq.profile_enable(False)
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

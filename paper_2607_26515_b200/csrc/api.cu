@@ -181,7 +181,7 @@ size_t linear_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K, int patt
     size_t b = kWsHeader + quant_scratch_bytes(M, K, pattern);
     b += align_up((size_t)M * (size_t)K * 2, 256);                            // bf16 image of deq Q(X)
     if (pattern != RESQ_S_NONE) b += align_up((size_t)M * (size_t)K * 2, 256);  // bf16 image of S(deq Q(dX))
-    int splits = fmt == kHiF4 ? gemm_hif4_pick_splits(M, N, K) : 1;
+    int splits = gemm_hif4_pick_splits(M, N, K);
     if (splits > 1) b += align_up((size_t)splits * (size_t)M * (size_t)N * 4, 256);
     return b;
 }
@@ -211,10 +211,6 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     }
     rc = check_workspace(workspace, ws_bytes, linear_workspace_bytes(fmt, M, N, K, pattern));
     if (rc) return rc;
-    if (fmt != kHiF4) {
-        set_last_error("the MXFP4 GEMM is not built yet");
-        return RESQ_ERR_PATTERN;
-    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemsetAsync(workspace, 0, kWsHeader, st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(status)");
@@ -238,6 +234,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     if (rc) return rc;
     GemmArgs g;
     memset(&g, 0, sizeof(g));
+    g.fmt = fmt;
     g.a_bf16 = a.a_bf16;
     g.r_bf16 = a.r_bf16;
     g.w_codes = static_cast<const uint8_t*>(w_codes);

@@ -68,6 +68,7 @@ size_t quant_scratch_bytes(int64_t M, int64_t K, int pattern);  // scores + keep
 
 // ---- GEMM launch description (gemm_hif4.cu / gemm_mxfp4.cu) -------------------------------------
 struct GemmArgs {
+    int fmt;                       // kHiF4 or kMXFP4: how w_codes / w_side are decoded
     const __nv_bfloat16* a_bf16;   // [M, K] exact bf16 image of deq Q(X)
     const __nv_bfloat16* r_bf16;   // [M, K] masked residual image, or null (pattern NONE)
     const uint8_t* w_codes;        // [N, K/2]

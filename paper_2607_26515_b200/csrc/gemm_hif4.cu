@@ -7,18 +7,24 @@
 // accumulation order.  (HiF4's 2-bit level-1 mantissa and uniform S1P2 grid do not map onto the
 // block-scaled FP4/FP8 MMA kinds, whose scales are powers of two.)
 //
-// One CTA computes a (128*MT) x BN tile of Y.  Warp roles:
-//   warp 0      TMA producer: activation tiles (128x64 bf16, 128-byte swizzle) and the raw weight
-//               codes (BN rows x 32 bytes) of each 64-wide k-block into a ring of stages
-//   warp 1      MMA issuer: tcgen05.mma kind::f16, 128 x BN x 16, accumulators in tensor memory;
-//               main and residual terms accumulate into the same TMEM tile against the same B tile
-//   warps 2..9  expanders: 4-bit codes + block metadata -> bf16, written in the canonical K-major
-//               128-byte-swizzled layout; afterwards the same warps run the epilogue
-// Stage hand-off uses mbarriers; every wait is bounded and a timeout ends the kernel cleanly.
+// Persistent kernel: one CTA per SM walks a static list of (128*MT) x BN output tiles (x K splits).
+// Warp roles (16 warps):
+//   warp 0       TMA producer of the activation tiles (128x64 bf16, 128-byte swizzle), main + residual
+//   warp 1       MMA issuer: tcgen05.mma kind::f16, 128 x BN x 16, fp32 accumulators in tensor memory,
+//                double-buffered across tiles; main and residual terms accumulate into the same tile
+//                against the same expanded weight tile
+//   warp 2       TMA producer of the raw weight codes (BN rows x 32 bytes per 64-wide k-block)
+//   warps 4..7   epilogue: TMEM -> registers -> global (bf16 / fp32 / split-K partial), overlapped with
+//                the next tile's main loop
+//   warps 8..15  expanders: 4-bit codes + block metadata -> bf16 in the canonical K-major
+//                128-byte-swizzled layout
+// Three independent shared-memory rings (activation tiles, raw codes, expanded weights) decouple the
+// TMA latency from the expansion latency.  Every wait is bounded; a timeout ends the kernel cleanly.
 #include "common.cuh"
 #include "ptx.cuh"
 
 #include <algorithm>
+#include <cstdlib>
 #include <mutex>
 
 namespace resq {
@@ -29,35 +35,30 @@ constexpr int kBM = 128;          // rows per MMA (UMMA M)
 constexpr int kBK = 64;           // one HiF4 block per row per stage
 constexpr int kMaxBN = 256;
 constexpr int kExpWarps = 8;
-constexpr int kGemmThreads = 32 * (2 + kExpWarps);
+constexpr int kFirstEpiWarp = 4;
+constexpr int kFirstExpWarp = 8;
+constexpr int kGemmThreads = 32 * (kFirstExpWarp + kExpWarps);
 constexpr int kATileBytes = kBM * kBK * 2;       // 16 KiB
-constexpr int kBExpBytes = kMaxBN * kBK * 2;     // 32 KiB
-constexpr int kBRawBytes = kMaxBN * (kBK / 2);   // 8 KiB
-constexpr int kMaxStages = 4;
+constexpr int kMaxRing = 8;
+constexpr int kSmemBudget = 232448;              // opt-in limit per block on sm_100
+constexpr int kTmemCols = 512;
 
 struct GemmParams {
-    const uint32_t* w_meta;   // [N, K/64]
+    const void* w_side;       // HiF4: u32 [N, K/64]; MXFP4: u8 [N, K/32]
     int64_t M, N, K;
-    int bn;                   // tile width (multiple of 16, <= 256)
+    int bn;                   // MMA N (multiple of 32, <= 256)
+    int nt;                   // N sub-tiles per CTA tile (1 or 2): the tile is 128*MT x nt*bn
     int kblocks_per_split;
     int splits;
+    int ntiles_m, ntiles_n, num_tiles;
+    int sa, sr, se;           // ring depths: activation tiles, raw codes, expanded weights
+    int acc_bufs;             // 2 if two accumulators fit in tensor memory, else 1
     void* Y;
     int out_f32;
     int64_t ldy;
     float* partials;          // [splits, M, N] when splits > 1
     DeviceStatus* status;
-};
-
-template <int MT, bool RES>
-struct SmemLayout {
-    static constexpr int kStageBytes = MT * kATileBytes * (RES ? 2 : 1) + kBExpBytes + kBRawBytes;
-    static constexpr int kStages = (224 * 1024 / kStageBytes) < kMaxStages ? (224 * 1024 / kStageBytes) : kMaxStages;
-    static constexpr int kAMainOff = 0;
-    static constexpr int kAResOff = MT * kATileBytes;
-    static constexpr int kBExpOff = MT * kATileBytes * (RES ? 2 : 1);
-    static constexpr int kBRawOff = kBExpOff + kBExpBytes;
-    static constexpr int kBarOff = kStages * kStageBytes;
-    static constexpr int kTotal = kBarOff + 256 + 1024;  // barriers + alignment slack
+    int debug;                // bit 0: expanders skip the arithmetic; bit 1: no MMAs; bit 2: epilogue skips stores
 };
 
 __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
@@ -70,228 +71,350 @@ __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
 // Expand one 32-bit word of 8 HiF4 codes (one level-2 group) into 8 bf16 values (one 16-byte chunk).
 // bf16x2 trick: (0x4300 | q) is the bf16 number 128+q and (0x4300 | q<<4) is 128+16q, so one packed
 // FMA with (scale, scale/16) and (-128 scale, -8 scale) yields q*scale exactly for both nibbles of a
-// byte; the sign bits are then XOR-ed in.
+// byte; the sign bits are then XOR-ed in.  Per pair of elements: one byte permute, one logic op, one
+// packed FMA, one logic op.
 __device__ __forceinline__ uint4 expand_hif4_chunk(uint32_t c, uint32_t meta, int chunk) {
-    const uint32_t s = meta & 255u;
-    const uint32_t Mn = s & 3u, E = s >> 2;
-    const uint32_t e2 = (meta >> (8 + chunk)) & 1u;
-    const uint32_t e3a = (meta >> (16 + 2 * chunk)) & 1u, e3b = (meta >> (17 + 2 * chunk)) & 1u;
-    // bf16 bits of (4+Mn) * 2^x: exponent field x + 2 + 127, top mantissa bits Mn
-    const uint32_t base = ((E + 77u + e2) << 7) | (Mn << 5);   // x = E - 52 + e2
-    const uint32_t sa = base + (e3a << 7), sb = base + (e3b << 7);
-    const uint32_t scale_a = sa | ((sa - 0x200u) << 16), scale_b = sb | ((sb - 0x200u) << 16);
-    const uint32_t add_a = scale_a + 0x03800380u + 0x80008000u;  // -(128 * scale) in both halves
-    const uint32_t add_b = scale_b + 0x03800380u + 0x80008000u;
+    // bf16 bits of (4+Mn) * 2^(E-52): exponent field E - 52 + 2 + 127, top mantissa bits Mn; s = E<<2|Mn
+    // so (s << 5) already is (E << 7) | (Mn << 5).
+    const uint32_t base = ((meta & 255u) << 5) + (77u << 7) + (((meta >> (8 + chunk)) & 1u) << 7);
+    const uint32_t sa = base + (((meta >> (16 + 2 * chunk)) & 1u) << 7);
+    const uint32_t sb = base + (((meta >> (17 + 2 * chunk)) & 1u) << 7);
+    const uint32_t scale_a = sa * 0x10001u - 0x02000000u;  // (scale, scale / 16)
+    const uint32_t scale_b = sb * 0x10001u - 0x02000000u;
+    const uint32_t add_a = scale_a + 0x83808380u;          // -(128 * scale) in both halves
+    const uint32_t add_b = scale_b + 0x83808380u;
     const uint32_t c4 = c << 4;
     uint32_t out[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        // y = byte i replicated into bytes 0 and 2
-        uint32_t y = __byte_perm(c, 0u, (uint32_t)(i | (4 << 4) | (i << 8) | (4 << 12)));
-        uint32_t t = (y & 0x00700007u) | 0x43004300u;
+        // w: byte i of c in bytes 0, 2 and 3; byte i of (c << 4) in byte 1.  Bits 2:0 and 22:20 are the two
+        // magnitudes; bit 15 is the sign of the even element, bit 31 the sign of the odd one.
+        const uint32_t w = __byte_perm(c, c4, (uint32_t)(i | ((4 + i) << 4) | (i << 8) | (i << 12)));
+        const uint32_t t = (w & 0x00700007u) | 0x43004300u;
         uint32_t v;
-        const uint32_t sc = i < 2 ? scale_a : scale_b, ad = i < 2 ? add_a : add_b;
-        asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(v) : "r"(t), "r"(sc), "r"(ad));
-        // signs: bit 7 of byte i (odd element) -> bit 31; bit 3 of byte i (even element) -> bit 15
-        uint32_t sg = __byte_perm(c, c4, (uint32_t)(0 | ((4 + i) << 4) | (0 << 8) | (i << 12)));
-        out[i] = v ^ (sg & 0x80008000u);
+        asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(v) : "r"(t), "r"(i < 2 ? scale_a : scale_b), "r"(i < 2 ? add_a : add_b));
+        out[i] = v ^ (w & 0x80008000u);
     }
     return make_uint4(out[0], out[1], out[2], out[3]);
 }
 
-template <int MT, bool RES>
+// MXFP4: expand 8 E2M1 codes with their E8M0 block scale `sc` (2^(sc-127)).  The eight E2M1 magnitudes
+// 0, .5, 1, 1.5, 2, 3, 4, 6 are bf16 values whose high / low bytes come from two 8-entry byte tables
+// indexed with a byte permute; the power-of-two scale is applied with an exact packed multiply.
+__device__ __forceinline__ uint4 expand_mxfp4_chunk(uint32_t c, uint32_t sc) {
+    // bf16(2^(sc-127)): exponent field sc; sc = 0 is the subnormal 2^-127 (mantissa bit 6)
+    const uint32_t s16 = sc == 0 ? 0x0040u : (sc << 7);
+    const uint32_t scale = s16 * 0x10001u;
+    const uint32_t c4 = c << 4;
+    uint32_t out[4];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t sel = (c >> (16 * h)) & 0x7777u;                 // four magnitude indices
+        const uint32_t hi4 = __byte_perm(0x3F3F3F00u, 0x40404040u, sel);  // high bytes of the four bf16 values
+        const uint32_t lo4 = __byte_perm(0xC0800000u, 0xC0804000u, sel);  // low bytes
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int i = 2 * h + j;  // byte of c holding this pair
+            uint32_t v = __byte_perm(lo4, hi4, j == 0 ? 0x5140u : 0x7362u);
+            asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(v) : "r"(v), "r"(scale));
+            const uint32_t w = __byte_perm(c, c4, (uint32_t)(i | ((4 + i) << 4) | (i << 8) | (i << 12)));
+            out[i] = v ^ (w & 0x80008000u);
+        }
+    }
+    return make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+struct TileCoord {
+    int64_t m0, n0;
+    int split, kb_begin, nkb;
+};
+
+__device__ __forceinline__ TileCoord decode_tile(const GemmParams& p, int tile, int mt_rows) {
+    TileCoord t;
+    t.split = tile % p.splits;
+    const int rest = tile / p.splits;
+    t.n0 = (int64_t)(rest % p.ntiles_n) * (p.bn * p.nt);
+    t.m0 = (int64_t)(rest / p.ntiles_n) * mt_rows;
+    const int G = (int)(p.K / kBK);
+    t.kb_begin = t.split * p.kblocks_per_split;
+    t.nkb = min(G, t.kb_begin + p.kblocks_per_split) - t.kb_begin;
+    if (t.nkb < 0) t.nkb = 0;
+    return t;
+}
+
+template <int MT, bool RES, int TN, int FMT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_r,
                  const __grid_constant__ CUtensorMap tmap_w, const GemmParams p) {
-    using L = SmemLayout<MT, RES>;
-    constexpr int S = L::kStages;
+    constexpr int kAStage = MT * kATileBytes * (RES ? 2 : 1);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
-    uint64_t* raw_full = bars;            // [S] TMA bytes landed
-    uint64_t* exp_full = bars + S;        // [S] expanded B tile written
-    uint64_t* empty = bars + 2 * S;       // [S] MMAs that read the stage have completed
-    uint64_t* acc_full = bars + 3 * S;    // [1] all MMAs of the tile have completed
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * S + 1);
+    constexpr int tile_n = TN;                       // CTA tile width
+    constexpr int bn = TN > kMaxBN ? kMaxBN : TN;    // MMA N
+    constexpr int nt = TN / bn;                      // MMAs side by side in N
+    const int SA = p.sa, SR = p.sr, SE = p.se;
+    constexpr int exp_stage = tile_n * 128, raw_stage = tile_n * 32;
+    uint8_t* ring_a = smem;
+    uint8_t* ring_e = ring_a + (size_t)SA * kAStage;
+    uint8_t* ring_r = ring_e + (size_t)SE * exp_stage;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(ring_r + (size_t)SR * raw_stage);
+    uint64_t* a_full = bars;                   // [kMaxRing] TMA bytes of an activation stage landed
+    uint64_t* a_empty = bars + kMaxRing;       // [kMaxRing] MMAs that read the stage have completed
+    uint64_t* r_full = bars + 2 * kMaxRing;    // raw codes landed
+    uint64_t* r_empty = bars + 3 * kMaxRing;   // expanders have consumed the raw codes
+    uint64_t* e_full = bars + 4 * kMaxRing;    // expanded weight tile written
+    uint64_t* e_empty = bars + 5 * kMaxRing;   // MMAs that read the expanded tile have completed
+    uint64_t* acc_full = bars + 6 * kMaxRing;  // [2] accumulator complete
+    uint64_t* acc_empty = acc_full + 2;        // [2] accumulator drained by the epilogue
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bn = p.bn;
-    const int64_t n0 = (int64_t)blockIdx.x * bn;
-    const int64_t m0 = (int64_t)blockIdx.y * (kBM * MT);
-    const int split = blockIdx.z;
     const int G = (int)(p.K / kBK);
-    const int kb_begin = split * p.kblocks_per_split;
-    const int kb_end = min(G, kb_begin + p.kblocks_per_split);
-    const int nkb = kb_end - kb_begin;
-    uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < MT * bn) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) {
-            ptx::mbar_init(&raw_full[s], 1);
-            ptx::mbar_init(&exp_full[s], kExpWarps);
-            ptx::mbar_init(&empty[s], 1);
+        for (int s = 0; s < kMaxRing; ++s) {
+            ptx::mbar_init(&a_full[s], 1);
+            ptx::mbar_init(&a_empty[s], 1);
+            ptx::mbar_init(&r_full[s], 1);
+            ptx::mbar_init(&r_empty[s], kExpWarps);
+            ptx::mbar_init(&e_full[s], kExpWarps);
+            ptx::mbar_init(&e_empty[s], 1);
         }
-        ptx::mbar_init(acc_full, 1);
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(&acc_full[b], 1);
+            ptx::mbar_init(&acc_empty[b], 4);
+        }
         *abort_flag = 0;
         ptx::mbar_fence_init();
     }
-    if (warp == 1) ptx::tmem_alloc(tmem_slot, tmem_cols);
+    if (warp == 1) ptx::tmem_alloc(tmem_slot, kTmemCols);
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ activation producer
         if (lane == 0) {
             ptx::tma_prefetch_desc(&tmap_a);
             if (RES) ptx::tma_prefetch_desc(&tmap_r);
-            ptx::tma_prefetch_desc(&tmap_w);
-            const uint32_t tx = (uint32_t)(MT * kATileBytes * (RES ? 2 : 1) + bn * (kBK / 2));
-            for (int i = 0; i < nkb; ++i) {
-                const int s = i % S;
-                if (i >= S && !ptx::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) {
-                    report_timeout(p.status, 1);
-                    break;
-                }
-                uint8_t* st = smem + (size_t)s * L::kStageBytes;
-                ptx::mbar_arrive_expect_tx(&raw_full[s], tx);
-                const int kb = kb_begin + i;
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+                const TileCoord tc = decode_tile(p, tile, kBM * MT);
+                for (int i = 0; i < tc.nkb; ++i, ++it) {
+                    const int s = it % SA;
+                    if (!ptx::mbar_wait(&a_empty[s], ((it / SA) & 1) ^ 1, abort_flag)) {
+                        report_timeout(p.status, 1);
+                        ok = false;
+                        break;
+                    }
+                    uint8_t* st = ring_a + (size_t)s * kAStage;
+                    ptx::mbar_arrive_expect_tx(&a_full[s], (uint32_t)kAStage);
+                    const int kx = (tc.kb_begin + i) * kBK;
 #pragma unroll
-                for (int t = 0; t < MT; ++t) {
-                    ptx::tma_load_2d(st + L::kAMainOff + t * kATileBytes, &tmap_a, &raw_full[s], kb * kBK,
-                                     (int)(m0 + t * kBM));
-                    if (RES)
-                        ptx::tma_load_2d(st + L::kAResOff + t * kATileBytes, &tmap_r, &raw_full[s], kb * kBK,
-                                         (int)(m0 + t * kBM));
+                    for (int t = 0; t < MT; ++t) {
+                        ptx::tma_load_2d(st + t * kATileBytes, &tmap_a, &a_full[s], kx, (int)(tc.m0 + t * kBM));
+                        if (RES)
+                            ptx::tma_load_2d(st + (MT + t) * kATileBytes, &tmap_r, &a_full[s], kx, (int)(tc.m0 + t * kBM));
+                    }
                 }
-                ptx::tma_load_2d(st + L::kBRawOff, &tmap_w, &raw_full[s], kb * (kBK / 2), (int)n0);
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ raw weight-code producer
+        if (lane == 0) {
+            ptx::tma_prefetch_desc(&tmap_w);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+                const TileCoord tc = decode_tile(p, tile, kBM * MT);
+                for (int i = 0; i < tc.nkb; ++i, ++it) {
+                    const int s = it % SR;
+                    if (!ptx::mbar_wait(&r_empty[s], ((it / SR) & 1) ^ 1, abort_flag)) {
+                        report_timeout(p.status, 5);
+                        ok = false;
+                        break;
+                    }
+                    ptx::mbar_arrive_expect_tx(&r_full[s], (uint32_t)raw_stage);
+#pragma unroll
+                    for (int j = 0; j < nt; ++j)
+                        ptx::tma_load_2d(ring_r + (size_t)s * raw_stage + (size_t)j * bn * 32, &tmap_w, &r_full[s],
+                                         (tc.kb_begin + i) * (kBK / 2), (int)(tc.n0 + j * bn));
+                }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc = ptx::idesc_bf16_f32(kBM, bn);
+            uint32_t it = 0;
+            int local_tile = 0;
             bool ok = true;
-            for (int i = 0; i < nkb && ok; ++i) {
-                const int s = i % S;
-                const uint32_t par = (i / S) & 1;
-                ok = ptx::mbar_wait(&raw_full[s], par, abort_flag) && ptx::mbar_wait(&exp_full[s], par, abort_flag);
-                if (!ok) {
-                    report_timeout(p.status, 2);
+            for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local_tile) {
+                const TileCoord tc = decode_tile(p, tile, kBM * MT);
+                if (tc.nkb == 0) continue;
+                const int buf = p.acc_bufs == 2 ? (local_tile & 1) : 0;
+                const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(local_tile >> 1) : (uint32_t)local_tile;
+                if (!ptx::mbar_wait(&acc_empty[buf], (use & 1) ^ 1, abort_flag)) {
+                    report_timeout(p.status, 6);
                     break;
                 }
                 ptx::tc_fence_after();
-                uint8_t* st = smem + (size_t)s * L::kStageBytes;
-                const uint32_t b_addr = ptx::smem_u32(st + L::kBExpOff);
+                const uint32_t d0 = tmem_base + (uint32_t)(buf * MT * tile_n);
+                for (int i = 0; i < tc.nkb; ++i, ++it) {
+                    const int sa = it % SA, se = it % SE;
+                    ok = ptx::mbar_wait(&a_full[sa], (it / SA) & 1, abort_flag) &&
+                         ptx::mbar_wait(&e_full[se], (it / SE) & 1, abort_flag);
+                    if (!ok) {
+                        report_timeout(p.status, 2);
+                        break;
+                    }
+                    ptx::tc_fence_after();
+                    const uint32_t a_addr = ptx::smem_u32(ring_a + (size_t)sa * kAStage);
+                    const uint32_t b_addr = ptx::smem_u32(ring_e + (size_t)se * exp_stage);
+                    if (!(p.debug & 2))
 #pragma unroll
-                for (int k = 0; k < kBK / 16; ++k) {
-                    const uint64_t bdesc = ptx::smem_desc_sw128_kmajor(b_addr + k * 32);
+                    for (int k = 0; k < kBK / 16; ++k) {
 #pragma unroll
-                    for (int t = 0; t < MT; ++t) {
-                        const uint32_t d = tmem_base + (uint32_t)(t * bn);
-                        const uint64_t adesc =
-                            ptx::smem_desc_sw128_kmajor(ptx::smem_u32(st + L::kAMainOff + t * kATileBytes) + k * 32);
-                        ptx::umma_bf16(d, adesc, bdesc, idesc, (i > 0 || k > 0) ? 1u : 0u);
-                        if (RES) {
-                            const uint64_t rdesc =
-                                ptx::smem_desc_sw128_kmajor(ptx::smem_u32(st + L::kAResOff + t * kATileBytes) + k * 32);
-                            ptx::umma_bf16(d, rdesc, bdesc, idesc, 1u);
+                        for (int j = 0; j < nt; ++j) {
+                            const uint64_t bdesc = ptx::smem_desc_sw128_kmajor(b_addr + j * bn * 128 + k * 32);
+#pragma unroll
+                            for (int t = 0; t < MT; ++t) {
+                                const uint32_t d = d0 + (uint32_t)((t * nt + j) * bn);
+                                ptx::umma_bf16(d, ptx::smem_desc_sw128_kmajor(a_addr + t * kATileBytes + k * 32), bdesc,
+                                               idesc, (i > 0 || k > 0) ? 1u : 0u);
+                                if (RES)
+                                    ptx::umma_bf16(d, ptx::smem_desc_sw128_kmajor(a_addr + (MT + t) * kATileBytes + k * 32),
+                                                   bdesc, idesc, 1u);
+                            }
                         }
                     }
+                    ptx::umma_commit(&a_empty[sa]);  // frees both stages when these MMAs have read them
+                    ptx::umma_commit(&e_empty[se]);
                 }
-                ptx::umma_commit(&empty[s]);  // frees the stage when these MMAs have read it
+                if (ok) ptx::umma_commit(&acc_full[buf]);
             }
-            ptx::umma_commit(acc_full);
         }
-    } else {
+    } else if (warp >= kFirstExpWarp) {
         // ------------------------------------------------------------------ expanders
-        const int ew = warp - 2;                      // 0..7
-        const int rows_per_warp = bn / kExpWarps;     // bn is a multiple of 16: 2..32 rows
+        const int ew = warp - kFirstExpWarp;          // 0..7
+        constexpr int rows_per_warp = tile_n / kExpWarps;  // 8, 16, 32 or 64 rows
         const int r_begin = ew * rows_per_warp;
         // lane -> (row within a group of 4, chunk): a quarter-warp writes one full 128-byte row
         const int sub_row = lane >> 3, chunk = lane & 7;
-        uint32_t meta_next = 0;
-        {
-            const int64_t n = n0 + r_begin + lane;
-            if (lane < rows_per_warp && n < p.N && nkb > 0) meta_next = __ldg(p.w_meta + n * G + kb_begin);
-        }
+        uint32_t it = 0;
         bool ok = true;
-        for (int i = 0; i < nkb && ok; ++i) {
-            const int s = i % S;
-            const uint32_t par = (i / S) & 1;
-            const uint32_t meta_cur = meta_next;
-            {
-                const int64_t n = n0 + r_begin + lane;
-                if (lane < rows_per_warp && n < p.N && i + 1 < nkb) meta_next = __ldg(p.w_meta + n * G + kb_begin + i + 1);
+        for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+            const TileCoord tc = decode_tile(p, tile, kBM * MT);
+            // lane l owns the metadata of rows l and 32 + l of this warp's slice
+            const int64_t n = tc.n0 + r_begin + lane;
+            const bool row_ok0 = lane < rows_per_warp && n < p.N;
+            const bool row_ok1 = lane + 32 < rows_per_warp && n + 32 < p.N;
+            // per row and k-block: one u32 of HiF4 metadata, or two E8M0 bytes (one u16) for MXFP4
+            auto load_side = [&](int64_t row, int kb) -> uint32_t {
+                if (FMT == kHiF4) return __ldg(reinterpret_cast<const uint32_t*>(p.w_side) + row * G + kb);
+                return (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(p.w_side) + row * G + kb);
+            };
+            uint32_t meta_next0 = (row_ok0 && tc.nkb > 0) ? load_side(n, tc.kb_begin) : 0u;
+            uint32_t meta_next1 = (row_ok1 && tc.nkb > 0) ? load_side(n + 32, tc.kb_begin) : 0u;
+            for (int i = 0; i < tc.nkb; ++i, ++it) {
+                const uint32_t meta_cur0 = meta_next0, meta_cur1 = meta_next1;
+                if (i + 1 < tc.nkb) {  // prefetch the next k-block
+                    meta_next0 = row_ok0 ? load_side(n, tc.kb_begin + i + 1) : 0u;
+                    meta_next1 = row_ok1 ? load_side(n + 32, tc.kb_begin + i + 1) : 0u;
+                }
+                const int sr = it % SR, se = it % SE;
+                ok = ptx::mbar_wait(&e_empty[se], ((it / SE) & 1) ^ 1, abort_flag) &&
+                     ptx::mbar_wait(&r_full[sr], (it / SR) & 1, abort_flag);
+                if (!ok) {
+                    report_timeout(p.status, 3);
+                    break;
+                }
+                const uint32_t* raw = reinterpret_cast<const uint32_t*>(ring_r + (size_t)sr * raw_stage);
+                uint8_t* bexp = ring_e + (size_t)se * exp_stage;
+                // all loads and shuffles first, then the arithmetic: independent chains interleave
+                constexpr int kIters = rows_per_warp / 4;
+                uint32_t cw[kIters], mw[kIters];
+#pragma unroll
+                for (int q = 0; q < kIters; ++q) {
+                    const int rl = q * 4 + sub_row;
+                    mw[q] = __shfl_sync(0xFFFFFFFFu, q < 8 ? meta_cur0 : meta_cur1, rl & 31);
+                    cw[q] = raw[(r_begin + rl) * 8 + chunk];
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&r_empty[sr]);  // the raw codes are in registers now
+#pragma unroll
+                for (int q = 0; q < kIters; ++q) {
+                    const int r = r_begin + q * 4 + sub_row;
+                    const uint4 v = FMT == kHiF4 ? expand_hif4_chunk(cw[q], mw[q], chunk)
+                                                 : expand_mxfp4_chunk(cw[q], (mw[q] >> (8 * (chunk >> 2))) & 255u);
+                    if (!(p.debug & 1)) *reinterpret_cast<uint4*>(bexp + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
+                }
+                ptx::fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&e_full[se]);
             }
-            if (i >= S) ok = ptx::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag);
-            ok = ok && ptx::mbar_wait(&raw_full[s], par, abort_flag);
-            if (!ok) {
-                report_timeout(p.status, 3);
+        }
+    } else if (warp >= kFirstEpiWarp) {
+        // ------------------------------------------------------------------ epilogue
+        const int quad = warp & 3;  // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
+        constexpr int nchunks = tile_n / 32;
+        int local_tile = 0;
+        for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++local_tile) {
+            const TileCoord tc = decode_tile(p, tile, kBM * MT);
+            if (tc.nkb == 0) continue;
+            const int buf = p.acc_bufs == 2 ? (local_tile & 1) : 0;
+            const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(local_tile >> 1) : (uint32_t)local_tile;
+            if (!ptx::mbar_wait(&acc_full[buf], use & 1, abort_flag)) {
+                report_timeout(p.status, 4);
                 break;
             }
-            uint8_t* st = smem + (size_t)s * L::kStageBytes;
-            const uint32_t* raw = reinterpret_cast<const uint32_t*>(st + L::kBRawOff);
-            uint8_t* bexp = st + L::kBExpOff;
-            for (int rr = 0; rr < rows_per_warp; rr += 4) {
-                const int rl = rr + sub_row;                       // row inside this warp's slice
-                const uint32_t meta = __shfl_sync(0xFFFFFFFFu, meta_cur, rl & 31);
-                if (rl < rows_per_warp) {
-                    const int r = r_begin + rl;
-                    const uint32_t c = raw[r * 8 + chunk];
-                    const uint4 v = expand_hif4_chunk(c, meta, chunk);
-                    *reinterpret_cast<uint4*>(bexp + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
-                }
-            }
-            ptx::fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&exp_full[s]);
-        }
-        // ------------------------------------------------------------------ epilogue (same warps)
-        if (nkb > 0 && ptx::mbar_wait(acc_full, 0, abort_flag)) {
             ptx::tc_fence_after();
-            const int quad = warp & 3;            // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
-            const int half = ew >> 2;             // two warps share a quadrant: split the column chunks
-            const int nchunks = (bn + 31) / 32;
 #pragma unroll 1
             for (int t = 0; t < MT; ++t) {
-                const int64_t m = m0 + t * kBM + quad * 32 + lane;
-                for (int cchunk = half; cchunk < nchunks; cchunk += 2) {
+                const int64_t m = tc.m0 + t * kBM + quad * 32 + lane;
+#pragma unroll 1
+                for (int cc = 0; cc < nchunks; ++cc) {
                     uint32_t v[32];
-                    const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * bn + cchunk * 32);
-                    if (cchunk * 32 + 32 <= bn) {
-                        ptx::tmem_ld_32x32(taddr, v);
-                    } else {  // bn % 32 == 16: last chunk has 16 columns
-                        uint32_t h[16];
-                        ptx::tmem_ld_32x16(taddr, h);
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) { v[j] = h[j]; v[16 + j] = 0; }
-                    }
+                    ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((buf * MT + t) * tile_n + cc * 32), v);
                     ptx::tmem_ld_wait();
-                    if (m >= p.M) continue;
-                    const int64_t nb = n0 + cchunk * 32;
-                    int64_t valid64 = p.N - nb;
-                    if (valid64 > bn - cchunk * 32) valid64 = bn - cchunk * 32;
-                    const int valid = valid64 > 32 ? 32 : (int)valid64;
-                    if (valid <= 0) continue;
+                    if (t == MT - 1 && cc == nchunks - 1) {
+                        // everything of this accumulator is in registers: hand it back to the MMA warp
+                        ptx::tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
+                    }
+                    if (m >= p.M || (p.debug & 4)) continue;
+                    const int64_t nb = tc.n0 + cc * 32;
+                    const int64_t left = p.N - nb;
+                    if (left <= 0) continue;
                     if (p.splits > 1) {
-                        float* dst = p.partials + ((int64_t)split * p.M + m) * p.N + nb;
-                        for (int j = 0; j < valid; ++j) dst[j] = __uint_as_float(v[j]);
-                    } else if (p.out_f32) {
-                        float* dst = reinterpret_cast<float*>(p.Y) + m * p.ldy + nb;
-                        if (valid == 32) {
+                        float* dst = p.partials + ((int64_t)tc.split * p.M + m) * p.N + nb;
+                        if (left >= 32 && (p.N & 3) == 0) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 4)
                                 *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                         } else {
-                            for (int j = 0; j < valid; ++j) dst[j] = __uint_as_float(v[j]);
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < left) dst[j] = __uint_as_float(v[j]);
+                        }
+                    } else if (p.out_f32) {
+                        float* dst = reinterpret_cast<float*>(p.Y) + m * p.ldy + nb;
+                        if (left >= 32) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < left) dst[j] = __uint_as_float(v[j]);
                         }
                     } else {
                         __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.Y) + m * p.ldy + nb;
-                        if (valid == 32) {
+                        if (left >= 32) {
                             uint32_t o[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
@@ -302,20 +425,20 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                             for (int j = 0; j < 16; j += 4)
                                 *reinterpret_cast<uint4*>(dst + 2 * j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
                         } else {
-                            for (int j = 0; j < valid; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < left) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
                         }
                     }
                 }
             }
-        } else if (nkb > 0) {
-            report_timeout(p.status, 4);
         }
     }
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, tmem_cols);
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -349,7 +472,7 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-int make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t inner, uint64_t rows,
+int make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, const void* base, uint64_t inner, uint64_t rows,
                  uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle sw) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) {
@@ -360,7 +483,6 @@ int make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const v
     cuuint64_t strides[1] = {row_stride_bytes};
     cuuint32_t box[2] = {box_inner, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    (void)elem_bytes;
     CUresult r = fn(m, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -371,81 +493,135 @@ int make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const v
 }
 
 struct TileChoice {
-    int mt, bn, splits;
+    int mt, bn, splits, nt;
 };
 
-// Pick the tile width and K split so that the grid covers the 148 SMs in as few, as full waves as possible.
+int env_int(const char* name, int dflt) {
+    const char* v = getenv(name);
+    return v && *v ? atoi(v) : dflt;
+}
+
+// Pick the tile width and K split so that the persistent grid covers the 148 SMs evenly.
 TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res) {
     const int sms = 148;
     const int G = (int)(K / kBK);
-    TileChoice best{1, 256, 1};
+    TileChoice best{1, 256, 1, 1};
     double best_cost = 1e300;
     for (int mt = 1; mt <= (res ? 1 : 2); ++mt) {
         if (mt == 2 && M <= kBM) continue;
         const int64_t mtiles = (M + kBM * mt - 1) / (kBM * mt);
-        for (int bn = 256; bn >= 64; bn -= 32) {
-            if (mt * bn > 512) continue;
-            const int64_t ntiles = (N + bn - 1) / bn;
+        for (int nt = 1; nt <= 2; ++nt)
+        for (int bn = 256; bn >= 64; bn /= 2) {
+            if (mt * nt * bn > 512) continue;
+            if (nt == 2 && bn < 256) continue;
+            const int64_t ntiles = (N + nt * bn - 1) / (nt * bn);
             for (int splits = 1; splits <= 8; splits *= 2) {
                 if (G / splits < 4 && splits > 1) break;
-                const int64_t ctas = mtiles * ntiles * splits;
-                const int64_t waves = (ctas + sms - 1) / sms;
+                const int64_t tiles = mtiles * ntiles * splits;
+                const int64_t per_cta = (tiles + sms - 1) / sms;  // tiles walked by the busiest CTA
                 const int kb = (G + splits - 1) / splits;
-                // per-CTA time model (arbitrary units): MMA time scales with bn*mt*(1+res) per k-block, floored by
-                // the expander time (scales with bn); fixed prologue/epilogue cost; split-K adds a reduce pass
-                const double mma = (double)mt * bn * (res ? 2.0 : 1.0) / 256.0;
-                const double expand = bn / 256.0 * 1.0;
-                const double per_kb = std::max(mma, expand) + 0.08;
-                double cost = waves * (kb * per_kb + 6.0 + 0.02 * mt * bn);
-                if (splits > 1) cost += 8.0 + (double)M * N * splits / 3.0e5;
+                // per-k-block time (arbitrary units): tensor time scales with mt*bn*(1+res), floored by the
+                // expander time (scales with bn); small tiles pay a fixed hand-off cost per k-block
+                const double mma = (double)mt * nt * bn * (res ? 2.0 : 1.0) / 256.0;
+                const double expand = nt * bn / 256.0 * 0.8;
+                // bytes pulled from L2 per k-block (activation tiles dominate), in units that make a
+                // 128x256 tile with a residual operand cost about 1.3 tensor-time units
+                const double l2 = (mt * (res ? 2.0 : 1.0) * 16.0 + nt * bn * 36.0 / 1024.0) / 31.0;
+                const double per_kb = std::max(std::max(mma, expand), l2) + 0.15;
+                double cost = per_cta * kb * per_kb + 8.0;  // pipeline fill + last epilogue
+                if (mt * nt * bn > 256) cost += per_cta * 4.0;   // single accumulator: the epilogue is not overlapped
+                if (splits > 1) cost += 8.0 + (double)M * N * splits / 2.0e5;
                 if (cost < best_cost) {
                     best_cost = cost;
-                    best = TileChoice{mt, bn, splits};
+                    best = TileChoice{mt, bn, splits, nt};
                 }
             }
         }
     }
+    // debugging overrides (tile exploration); not part of the interface
+    best.mt = env_int("RESQ_GEMM_MT", best.mt);
+    best.bn = env_int("RESQ_GEMM_BN", best.bn);
+    best.splits = env_int("RESQ_GEMM_SPLITS", best.splits);
+    best.nt = env_int("RESQ_GEMM_NT", best.nt);
+    if (res) best.mt = 1;
     return best;
 }
 
-template <int MT, bool RES>
+template <int MT, bool RES, int TN, int FMT>
 int launch_variant(const GemmArgs& g, const TileChoice& tc, cudaStream_t stream) {
-    using L = SmemLayout<MT, RES>;
+    constexpr int kAStage = MT * kATileBytes * (RES ? 2 : 1);
     CUtensorMap ta, tr, tw;
-    int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, g.a_bf16, (uint64_t)g.K, (uint64_t)g.M,
-                          (uint64_t)g.K * 2, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+    int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.a_bf16, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.K * 2,
+                          kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
-    rc = make_tmap_2d(&tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, RES ? g.r_bf16 : g.a_bf16, (uint64_t)g.K, (uint64_t)g.M,
+    rc = make_tmap_2d(&tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, RES ? g.r_bf16 : g.a_bf16, (uint64_t)g.K, (uint64_t)g.M,
                       (uint64_t)g.K * 2, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
-    rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.w_codes, (uint64_t)g.K / 2, (uint64_t)g.N,
-                      (uint64_t)g.K / 2, kBK / 2, (uint32_t)tc.bn, CU_TENSOR_MAP_SWIZZLE_NONE);
+    rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.w_codes, (uint64_t)g.K / 2, (uint64_t)g.N, (uint64_t)g.K / 2,
+                      kBK / 2, (uint32_t)tc.bn, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc) return rc;
     GemmParams p;
-    p.w_meta = static_cast<const uint32_t*>(g.w_side);
+    p.w_side = g.w_side;
     p.M = g.M;
     p.N = g.N;
     p.K = g.K;
     p.bn = tc.bn;
+    p.nt = tc.nt;
     const int G = (int)(g.K / kBK);
     p.splits = tc.splits;
     p.kblocks_per_split = (G + tc.splits - 1) / tc.splits;
+    p.ntiles_m = (int)((g.M + kBM * MT - 1) / (kBM * MT));
+    p.ntiles_n = (int)((g.N + tc.nt * tc.bn - 1) / (tc.nt * tc.bn));
+    p.num_tiles = p.ntiles_m * p.ntiles_n * tc.splits;
+    if (MT * tc.nt * tc.bn > kTmemCols) {
+        set_last_error("internal: tile does not fit tensor memory");
+        return RESQ_ERR_CUDA;
+    }
+    p.acc_bufs = MT * tc.nt * tc.bn * 2 <= kTmemCols ? 2 : 1;
+    // ring depths from the shared-memory budget
+    const int exp_stage = tc.nt * tc.bn * 128, raw_stage = tc.nt * tc.bn * 32;
+    const int fixed = 1024 /*alignment slack*/ + 1024 /*barriers*/;
+    p.se = env_int("RESQ_GEMM_SE", 3);
+    p.sr = env_int("RESQ_GEMM_SR", 4);
+    p.sa = (kSmemBudget - fixed - p.se * exp_stage - p.sr * raw_stage) / kAStage;
+    if (p.sa < 3 && p.se > 2) {
+        p.se = 2;
+        p.sa = (kSmemBudget - fixed - p.se * exp_stage - p.sr * raw_stage) / kAStage;
+    }
+    if (p.sa < 2 && p.sr > 2) {
+        p.sr = 2;
+        p.sa = (kSmemBudget - fixed - p.se * exp_stage - p.sr * raw_stage) / kAStage;
+    }
+    p.sa = std::min(p.sa, kMaxRing);
+    if (p.sa < 2 || p.se > kMaxRing || p.sr > kMaxRing) {
+        set_last_error("internal: shared-memory rings do not fit (bn=%d)", tc.bn);
+        return RESQ_ERR_CUDA;
+    }
+    const int smem_bytes = fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage;
     p.Y = g.Y;
     p.out_f32 = g.out_dtype == RESQ_OUT_F32;
     p.ldy = g.ldy;
     p.partials = g.splitk_partials;
     p.status = g.status;
-    auto kern = gemm_hif4_kernel<MT, RES>;
+    p.debug = env_int("RESQ_GEMM_DEBUG", 0);
+    auto kern = gemm_hif4_kernel<MT, RES, TN, FMT>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute(gemm)");
-    dim3 grid((unsigned)((g.N + tc.bn - 1) / tc.bn), (unsigned)((g.M + kBM * MT - 1) / (kBM * MT)), (unsigned)tc.splits);
+    static int num_sms = 0;
+    if (num_sms == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (num_sms <= 0) num_sms = 148;
+    }
+    const unsigned grid = (unsigned)std::min(p.num_tiles, num_sms);
     {
         LaunchScope scope(kKindGemm, stream);
-        kern<<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tr, tw, p);
+        kern<<<grid, kGemmThreads, smem_bytes, stream>>>(ta, tr, tw, p);
     }
     rc = cuda_fail(cudaGetLastError(), "gemm_hif4_kernel launch");
     if (rc) return rc;
@@ -466,13 +642,31 @@ int gemm_hif4_pick_splits(int64_t M, int64_t N, int64_t K) {
     return std::max(choose_tile(M, N, K, false).splits, choose_tile(M, N, K, true).splits);
 }
 
+template <int MT, bool RES, int FMT>
+int dispatch_tn(const GemmArgs& g, const TileChoice& tc, cudaStream_t stream) {
+    const int tn = tc.bn * tc.nt;
+    if (tn == 64) return launch_variant<MT, RES, 64, FMT>(g, tc, stream);
+    if (tn == 128) return launch_variant<MT, RES, 128, FMT>(g, tc, stream);
+    if (tn == 256) return launch_variant<MT, RES, 256, FMT>(g, tc, stream);
+    if constexpr (MT == 1) {
+        if (tn == 512) return launch_variant<MT, RES, 512, FMT>(g, tc, stream);
+    }
+    set_last_error("internal: unsupported tile width %d", tn);
+    return RESQ_ERR_CUDA;
+}
+
 int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream) {
     const bool res = g.r_bf16 != nullptr;
     TileChoice tc = choose_tile(g.M, g.N, g.K, res);
     if (tc.splits > 1 && (!g.splitk_partials || tc.splits > g.splits)) tc.splits = 1;
-    if (res) return launch_variant<1, true>(g, tc, stream);
-    if (tc.mt == 2) return launch_variant<2, false>(g, tc, stream);
-    return launch_variant<1, false>(g, tc, stream);
+    if (g.fmt == kMXFP4) {
+        if (res) return dispatch_tn<1, true, kMXFP4>(g, tc, stream);
+        if (tc.mt == 2) return dispatch_tn<2, false, kMXFP4>(g, tc, stream);
+        return dispatch_tn<1, false, kMXFP4>(g, tc, stream);
+    }
+    if (res) return dispatch_tn<1, true, kHiF4>(g, tc, stream);
+    if (tc.mt == 2) return dispatch_tn<2, false, kHiF4>(g, tc, stream);
+    return dispatch_tn<1, false, kHiF4>(g, tc, stream);
 }
 
 }  // namespace resq

@@ -73,6 +73,14 @@ def test_linear_shapes(pattern, shape):
     run_case(xb, wb, pattern)
 
 
+@pytest.mark.parametrize("pattern", ALL)
+@pytest.mark.parametrize("shape", [(128, 256, 256), (96, 192, 80), (288, 1024, 1000), (64, 2048, 2048)])
+def test_linear_mxfp4(pattern, shape):
+    M, K, N = shape
+    xb, wb = synth_xw(M + N + pattern + 1, M, K, N, n_out=max(1, K // 256))
+    run_case(xb, wb, pattern, fmt="mxfp4")
+
+
 @pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4])
 def test_linear_bf16_output(pattern):
     xb, wb = synth_xw(7, 200, 512, 520)
