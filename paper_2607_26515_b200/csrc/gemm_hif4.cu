@@ -124,6 +124,14 @@ __device__ __forceinline__ uint4 expand_mxfp4_chunk(uint32_t c, uint32_t sc) {
     return make_uint4(out[0], out[1], out[2], out[3]);
 }
 
+// Debug aid: cycles spent per role, summed over CTAs into the 64-bit counters that follow the status word.
+struct Trace {
+    unsigned long long* out;
+    long long t0;
+    __device__ __forceinline__ void begin() { if (out) t0 = clock64(); }
+    __device__ __forceinline__ void end(int slot) { if (out) atomicAdd(out + slot, (unsigned long long)(clock64() - t0)); }
+};
+
 struct TileCoord {
     int64_t m0, n0;
     int split, kb_begin, nkb;
@@ -193,6 +201,8 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    Trace tr{(p.debug & 16) ? reinterpret_cast<unsigned long long*>(p.status) + 8 : nullptr, 0};
+    const long long t_kernel0 = clock64();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ activation producer
@@ -205,12 +215,19 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 const TileCoord tc = decode_tile(p, tile, kBM * MT);
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
                     const int s = it % SA;
-                    if (!ptx::mbar_wait(&a_empty[s], ((it / SA) & 1) ^ 1, abort_flag)) {
+                    tr.begin();
+                    const bool got = ptx::mbar_wait(&a_empty[s], ((it / SA) & 1) ^ 1, abort_flag);
+                    tr.end(0);
+                    if (!got) {
                         report_timeout(p.status, 1);
                         ok = false;
                         break;
                     }
                     uint8_t* st = ring_a + (size_t)s * kAStage;
+                    if (p.debug & 8) {
+                        ptx::mbar_arrive(&a_full[s]);
+                        continue;
+                    }
                     ptx::mbar_arrive_expect_tx(&a_full[s], (uint32_t)kAStage);
                     const int kx = (tc.kb_begin + i) * kBK;
 #pragma unroll
@@ -232,10 +249,17 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 const TileCoord tc = decode_tile(p, tile, kBM * MT);
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
                     const int s = it % SR;
-                    if (!ptx::mbar_wait(&r_empty[s], ((it / SR) & 1) ^ 1, abort_flag)) {
+                    tr.begin();
+                    const bool got = ptx::mbar_wait(&r_empty[s], ((it / SR) & 1) ^ 1, abort_flag);
+                    tr.end(1);
+                    if (!got) {
                         report_timeout(p.status, 5);
                         ok = false;
                         break;
+                    }
+                    if (p.debug & 8) {
+                        ptx::mbar_arrive(&r_full[s]);
+                        continue;
                     }
                     ptx::mbar_arrive_expect_tx(&r_full[s], (uint32_t)raw_stage);
 #pragma unroll
@@ -257,7 +281,10 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 if (tc.nkb == 0) continue;
                 const int buf = p.acc_bufs == 2 ? (local_tile & 1) : 0;
                 const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(local_tile >> 1) : (uint32_t)local_tile;
-                if (!ptx::mbar_wait(&acc_empty[buf], (use & 1) ^ 1, abort_flag)) {
+                tr.begin();
+                const bool got_acc = ptx::mbar_wait(&acc_empty[buf], (use & 1) ^ 1, abort_flag);
+                tr.end(4);
+                if (!got_acc) {
                     report_timeout(p.status, 6);
                     break;
                 }
@@ -265,12 +292,17 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 const uint32_t d0 = tmem_base + (uint32_t)(buf * MT * tile_n);
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
                     const int sa = it % SA, se = it % SE;
-                    ok = ptx::mbar_wait(&a_full[sa], (it / SA) & 1, abort_flag) &&
-                         ptx::mbar_wait(&e_full[se], (it / SE) & 1, abort_flag);
+                    tr.begin();
+                    ok = ptx::mbar_wait(&a_full[sa], (it / SA) & 1, abort_flag);
+                    tr.end(2);
+                    tr.begin();
+                    ok = ok && ptx::mbar_wait(&e_full[se], (it / SE) & 1, abort_flag);
+                    tr.end(3);
                     if (!ok) {
                         report_timeout(p.status, 2);
                         break;
                     }
+                    tr.begin();
                     ptx::tc_fence_after();
                     const uint32_t a_addr = ptx::smem_u32(ring_a + (size_t)sa * kAStage);
                     const uint32_t b_addr = ptx::smem_u32(ring_e + (size_t)se * exp_stage);
@@ -293,6 +325,7 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     }
                     ptx::umma_commit(&a_empty[sa]);  // frees both stages when these MMAs have read them
                     ptx::umma_commit(&e_empty[se]);
+                    tr.end(5);
                 }
                 if (ok) ptx::umma_commit(&acc_full[buf]);
             }
@@ -326,8 +359,11 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     meta_next1 = row_ok1 ? load_side(n + 32, tc.kb_begin + i + 1) : 0u;
                 }
                 const int sr = it % SR, se = it % SE;
-                ok = ptx::mbar_wait(&e_empty[se], ((it / SE) & 1) ^ 1, abort_flag) &&
-                     ptx::mbar_wait(&r_full[sr], (it / SR) & 1, abort_flag);
+                if (ew == 0 && lane == 0) tr.begin();
+                ok = ptx::mbar_wait(&e_empty[se], ((it / SE) & 1) ^ 1, abort_flag);
+                if (ew == 0 && lane == 0) { tr.end(6); tr.begin(); }
+                ok = ok && ptx::mbar_wait(&r_full[sr], (it / SR) & 1, abort_flag);
+                if (ew == 0 && lane == 0) { tr.end(7); tr.begin(); }
                 if (!ok) {
                     report_timeout(p.status, 3);
                     break;
@@ -340,6 +376,7 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 #pragma unroll
                 for (int q = 0; q < kIters; ++q) {
                     const int rl = q * 4 + sub_row;
+                    if (p.debug & 64) { mw[q] = meta_cur0; cw[q] = meta_cur1; continue; }
                     mw[q] = __shfl_sync(0xFFFFFFFFu, q < 8 ? meta_cur0 : meta_cur1, rl & 31);
                     cw[q] = raw[(r_begin + rl) * 8 + chunk];
                 }
@@ -352,9 +389,10 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                                                  : expand_mxfp4_chunk(cw[q], (mw[q] >> (8 * (chunk >> 2))) & 255u);
                     if (!(p.debug & 1)) *reinterpret_cast<uint4*>(bexp + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
                 }
-                ptx::fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core
+                if (!(p.debug & 32)) ptx::fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&e_full[se]);
+                if (ew == 0 && lane == 0) tr.end(8);
             }
         }
     } else if (warp >= kFirstEpiWarp) {
@@ -367,7 +405,10 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             if (tc.nkb == 0) continue;
             const int buf = p.acc_bufs == 2 ? (local_tile & 1) : 0;
             const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(local_tile >> 1) : (uint32_t)local_tile;
-            if (!ptx::mbar_wait(&acc_full[buf], use & 1, abort_flag)) {
+            if (quad == 0 && lane == 0) tr.begin();
+            const bool got_full = ptx::mbar_wait(&acc_full[buf], use & 1, abort_flag);
+            if (quad == 0 && lane == 0) { tr.end(9); tr.begin(); }
+            if (!got_full) {
                 report_timeout(p.status, 4);
                 break;
             }
@@ -432,10 +473,15 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     }
                 }
             }
+            if (quad == 0 && lane == 0) tr.end(10);
         }
     }
     ptx::tc_fence_before();
     __syncthreads();
+    if (tr.out && threadIdx.x == 0) {
+        atomicAdd(tr.out + 11, (unsigned long long)(clock64() - t_kernel0));
+        atomicAdd(tr.out + 12, 1ull);
+    }
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
