@@ -115,6 +115,27 @@ RESQ_API int mxfp4_residual_mask(const void* X_bf16, int64_t M, int64_t K, int64
                         void* x_codes, void* x_scale, void* r_codes, void* r_scale, void* mask_bits,
                         void* workspace, size_t ws_bytes, void* stream);
 
+/* ---- the same pass for callers that cannot allocate device memory (the paper has no counterpart) ----
+ * Meant for hosts that cannot give the library a workspace: a server that handed all device memory to its
+ * own pool at start-up, a plugin invoked inside a serving loop where an allocation would stall the device,
+ * or a foreign-function caller that owns only its inputs and outputs.  Same inputs, outputs, patterns and
+ * results as resq_residual_mask (HiF4), but the scratch of the channel-wise and block-wise selections lives
+ * in a fixed device array inside the library image (about 290 KB, held by every GPU that loads the
+ * library until the process exits).  The call performs no cudaMalloc / cudaFree and uses no allocating
+ * library routine.
+ *   - Limit: at most RESQ_STATIC_SCRATCH_MAX_SCORES selection scores, i.e. K for RESQ_S_CHAN50 and
+ *     (M/32)*(K/64) for RESQ_S_BLOCK32x64_50; larger problems return RESQ_ERR_WORKSPACE with a message
+ *     (the other patterns need no scores and have no limit).
+ *   - The first call on each device looks up the array's device address (with that device current); make
+ *     that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the call clears
+ *     what has to start from zero itself.  Two calls whose kernels overlap on the GPU (different streams,
+ *     or different host threads) race on it: serialise them. */
+#define RESQ_STATIC_SCRATCH_MAX_SCORES 32768
+RESQ_API int resq_residual_mask_static(const void* X_bf16, int64_t M, int64_t K, int64_t ldx, int pattern,
+                                       void* x_codes, void* x_meta, void* r_codes, void* r_meta, void* mask_bits,
+                                       void* stream);
+
 /* ---- the rollout projection, Eq. (5):  Y = Q(X) Q(W)^T + S(Q(dX)) Q(W)^T ------------------------
  * X_bf16 [M, K] (ldx), packed weight from *_pack_weight, Y [M, N] (ldy) as bf16 (round-to-nearest-
  * even of the fp32 accumulator) or fp32.  Products of decoded values are exact in fp32; only the

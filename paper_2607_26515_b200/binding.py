@@ -41,6 +41,7 @@ SYMBOLS = {
     "mxfp4_dequantize": (_ci, [_vp, _vp, _i64, _i64, _vp, _vp]),
     "resq_residual_mask": (_ci, [_vp, _i64, _i64, _i64, _ci, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "mxfp4_residual_mask": (_ci, [_vp, _i64, _i64, _i64, _ci, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "resq_residual_mask_static": (_ci, [_vp, _i64, _i64, _i64, _ci, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hif4_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "mxfp4_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "resq_check": (_ci, [_vp, _vp]),
@@ -173,6 +174,28 @@ def residual_mask(X: torch.Tensor, pattern: int, fmt: str = "hif4", workspace: O
     _check(_fn(fmt, "resq_residual_mask", "mxfp4_residual_mask")(
         X.data_ptr(), M, K, X.stride(0), pattern, _ptr(out["x_codes"]), _ptr(out["x_side"]), _ptr(out["r_codes"]),
         _ptr(out["r_side"]), _ptr(out["mask"]), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return out
+
+
+STATIC_SCRATCH_MAX_SCORES = 32768
+
+
+def residual_mask_static(X: torch.Tensor, pattern: int, stream=None):
+    """resq_residual_mask_static: the HiF4 residual / mask pass without a caller workspace, for callers that
+    cannot allocate device memory; its selection scratch is a fixed array inside the library (at most
+    STATIC_SCRATCH_MAX_SCORES channel or block scores).  Calls that overlap on the GPU race on that array."""
+    _require_bf16_matrix(X, "X")
+    M, K = X.shape
+    dev = X.device
+    out = {"x_codes": torch.empty((M, K // 2), dtype=torch.uint8, device=dev), "x_side": _side("hif4", M, K, dev),
+           "r_codes": None, "r_side": None, "mask": None}
+    if pattern != S_NONE:
+        out["r_codes"] = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
+        out["r_side"] = _side("hif4", M, K, dev)
+        out["mask"] = torch.empty((M, K // 8), dtype=torch.uint8, device=dev)
+    _check(lib().resq_residual_mask_static(
+        X.data_ptr(), M, K, X.stride(0), pattern, _ptr(out["x_codes"]), _ptr(out["x_side"]), _ptr(out["r_codes"]),
+        _ptr(out["r_side"]), _ptr(out["mask"]), _stream(stream)))
     return out
 
 
