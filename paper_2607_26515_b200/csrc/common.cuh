@@ -1,5 +1,6 @@
 // Shared declarations of the ResQ CUDA library (sm_100a).  Internal; the public contract is include/resq.h.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -82,6 +83,9 @@ struct GemmArgs {
     DeviceStatus* status;
 };
 int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream);
+int make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, const void* base, uint64_t inner, uint64_t rows,
+                 uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle sw);
+int launch_splitk_reduce(const GemmArgs& g, int splits, cudaStream_t stream);
 int gemm_hif4_pick_splits(int64_t M, int64_t N, int64_t K);
 
 }  // namespace resq

@@ -22,6 +22,7 @@
 // TMA latency from the expansion latency.  Every wait is bounded; a timeout ends the kernel cleanly.
 #include "common.cuh"
 #include "ptx.cuh"
+#include "expand.cuh"
 
 #include <algorithm>
 #include <cstdlib>
@@ -66,62 +67,6 @@ __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
         st->where = where;
         st->block = (int)blockIdx.x;
     }
-}
-
-// Expand one 32-bit word of 8 HiF4 codes (one level-2 group) into 8 bf16 values (one 16-byte chunk).
-// bf16x2 trick: (0x4300 | q) is the bf16 number 128+q and (0x4300 | q<<4) is 128+16q, so one packed
-// FMA with (scale, scale/16) and (-128 scale, -8 scale) yields q*scale exactly for both nibbles of a
-// byte; the sign bits are then XOR-ed in.  Per pair of elements: one byte permute, one logic op, one
-// packed FMA, one logic op.
-__device__ __forceinline__ uint4 expand_hif4_chunk(uint32_t c, uint32_t meta, int chunk) {
-    // bf16 bits of (4+Mn) * 2^(E-52): exponent field E - 52 + 2 + 127, top mantissa bits Mn; s = E<<2|Mn
-    // so (s << 5) already is (E << 7) | (Mn << 5).
-    const uint32_t base = ((meta & 255u) << 5) + (77u << 7) + (((meta >> (8 + chunk)) & 1u) << 7);
-    const uint32_t sa = base + (((meta >> (16 + 2 * chunk)) & 1u) << 7);
-    const uint32_t sb = base + (((meta >> (17 + 2 * chunk)) & 1u) << 7);
-    const uint32_t scale_a = sa * 0x10001u - 0x02000000u;  // (scale, scale / 16)
-    const uint32_t scale_b = sb * 0x10001u - 0x02000000u;
-    const uint32_t add_a = scale_a + 0x83808380u;          // -(128 * scale) in both halves
-    const uint32_t add_b = scale_b + 0x83808380u;
-    const uint32_t c4 = c << 4;
-    uint32_t out[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        // w: byte i of c in bytes 0, 2 and 3; byte i of (c << 4) in byte 1.  Bits 2:0 and 22:20 are the two
-        // magnitudes; bit 15 is the sign of the even element, bit 31 the sign of the odd one.
-        const uint32_t w = __byte_perm(c, c4, (uint32_t)(i | ((4 + i) << 4) | (i << 8) | (i << 12)));
-        const uint32_t t = (w & 0x00700007u) | 0x43004300u;
-        uint32_t v;
-        asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(v) : "r"(t), "r"(i < 2 ? scale_a : scale_b), "r"(i < 2 ? add_a : add_b));
-        out[i] = v ^ (w & 0x80008000u);
-    }
-    return make_uint4(out[0], out[1], out[2], out[3]);
-}
-
-// MXFP4: expand 8 E2M1 codes with their E8M0 block scale `sc` (2^(sc-127)).  The eight E2M1 magnitudes
-// 0, .5, 1, 1.5, 2, 3, 4, 6 are bf16 values whose high / low bytes come from two 8-entry byte tables
-// indexed with a byte permute; the power-of-two scale is applied with an exact packed multiply.
-__device__ __forceinline__ uint4 expand_mxfp4_chunk(uint32_t c, uint32_t sc) {
-    // bf16(2^(sc-127)): exponent field sc; sc = 0 is the subnormal 2^-127 (mantissa bit 6)
-    const uint32_t s16 = sc == 0 ? 0x0040u : (sc << 7);
-    const uint32_t scale = s16 * 0x10001u;
-    const uint32_t c4 = c << 4;
-    uint32_t out[4];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const uint32_t sel = (c >> (16 * h)) & 0x7777u;                 // four magnitude indices
-        const uint32_t hi4 = __byte_perm(0x3F3F3F00u, 0x40404040u, sel);  // high bytes of the four bf16 values
-        const uint32_t lo4 = __byte_perm(0xC0800000u, 0xC0804000u, sel);  // low bytes
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const int i = 2 * h + j;  // byte of c holding this pair
-            uint32_t v = __byte_perm(lo4, hi4, j == 0 ? 0x5140u : 0x7362u);
-            asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(v) : "r"(v), "r"(scale));
-            const uint32_t w = __byte_perm(c, c4, (uint32_t)(i | ((4 + i) << 4) | (i << 8) | (i << 12)));
-            out[i] = v ^ (w & 0x80008000u);
-        }
-    }
-    return make_uint4(out[0], out[1], out[2], out[3]);
 }
 
 // Debug aid: cycles spent per role, summed over CTAs into the 64-bit counters that follow the status word.
@@ -347,8 +292,8 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             const bool row_ok1 = lane + 32 < rows_per_warp && n + 32 < p.N;
             // per row and k-block: one u32 of HiF4 metadata, or two E8M0 bytes (one u16) for MXFP4
             auto load_side = [&](int64_t row, int kb) -> uint32_t {
-                if (FMT == kHiF4) return __ldg(reinterpret_cast<const uint32_t*>(p.w_side) + row * G + kb);
-                return (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(p.w_side) + row * G + kb);
+                if (FMT == kHiF4) return ptx::ld_nc_u32(reinterpret_cast<const uint32_t*>(p.w_side) + row * G + kb);
+                return ptx::ld_nc_u16(reinterpret_cast<const uint16_t*>(p.w_side) + row * G + kb);
             };
             uint32_t meta_next0 = (row_ok0 && tc.nkb > 0) ? load_side(n, tc.kb_begin) : 0u;
             uint32_t meta_next1 = (row_ok1 && tc.nkb > 0) ? load_side(n + 32, tc.kb_begin) : 0u;
@@ -500,6 +445,8 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ partials, int spl
     else reinterpret_cast<__nv_bfloat16*>(Y)[m * ldy + n] = __float2bfloat16_rn(acc);
 }
 
+}  // namespace
+
 // ---- host side -----------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -538,8 +485,22 @@ int make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, const void* base, uint6
     return RESQ_OK;
 }
 
+int launch_splitk_reduce(const GemmArgs& g, int splits, cudaStream_t stream) {
+    if (splits <= 1) return RESQ_OK;
+    const int64_t n = g.M * g.N;
+    LaunchScope scope(kKindReduce, stream);
+    splitk_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(g.splitk_partials, splits, g.M, g.N, g.Y,
+                                                                         g.out_dtype == RESQ_OUT_F32, g.ldy);
+    return cuda_fail(cudaGetLastError(), "splitk_reduce_kernel launch");
+}
+
+int launch_gemm_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream);
+
+namespace {
+
 struct TileChoice {
     int mt, bn, splits, nt;
+    int pair_tn;  // > 0: use the CTA-pair kernel with a 256 x pair_tn tile
 };
 
 int env_int(const char* name, int dflt) {
@@ -551,7 +512,7 @@ int env_int(const char* name, int dflt) {
 TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res) {
     const int sms = 148;
     const int G = (int)(K / kBK);
-    TileChoice best{1, 256, 1, 1};
+    TileChoice best{1, 256, 1, 1, 0};
     double best_cost = 1e300;
     for (int mt = 1; mt <= (res ? 1 : 2); ++mt) {
         if (mt == 2 && M <= kBM) continue;
@@ -579,7 +540,32 @@ TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res) {
                 if (splits > 1) cost += 8.0 + (double)M * N * splits / 2.0e5;
                 if (cost < best_cost) {
                     best_cost = cost;
-                    best = TileChoice{mt, bn, splits, nt};
+                    best = TileChoice{mt, bn, splits, nt, 0};
+                }
+            }
+        }
+    }
+    // CTA pairs (256 x tn tiles, 74 pairs): same per-SM tensor time as a 128 x tn single-CTA tile, half the
+    // expansion work per SM
+    if (M > kBM && env_int("RESQ_GEMM_PAIR", 1)) {
+        const int64_t mtiles = (M + 2 * kBM - 1) / (2 * kBM);
+        for (int tn = 512; tn >= 128; tn /= 2) {
+            const int64_t ntiles = (N + tn - 1) / tn;
+            for (int splits = 1; splits <= 8; splits *= 2) {
+                if (G / splits < 4 && splits > 1) break;
+                const int64_t tiles = mtiles * ntiles * splits;
+                const int64_t per_pair = (tiles + sms / 2 - 1) / (sms / 2);
+                const int kb = (G + splits - 1) / splits;
+                const double mma = tn / 256.0 * (res ? 2.0 : 1.0);
+                const double expand = tn / 2 / 256.0 * 0.8;
+                const double l2 = ((res ? 2.0 : 1.0) * 16.0 + tn / 2 * 36.0 / 1024.0) / 31.0;
+                const double per_kb = std::max(std::max(mma, expand), l2) + 0.15;
+                double cost = per_pair * kb * per_kb + 8.0;
+                if (tn > 256) cost += per_pair * 4.0;
+                if (splits > 1) cost += 8.0 + (double)M * N * splits / 2.0e5;
+                if (cost < best_cost) {
+                    best_cost = cost;
+                    best = TileChoice{1, std::min(tn, 256), splits, tn > 256 ? 2 : 1, tn};
                 }
             }
         }
@@ -589,6 +575,8 @@ TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res) {
     best.bn = env_int("RESQ_GEMM_BN", best.bn);
     best.splits = env_int("RESQ_GEMM_SPLITS", best.splits);
     best.nt = env_int("RESQ_GEMM_NT", best.nt);
+    best.pair_tn = env_int("RESQ_GEMM_PAIR_TN", best.pair_tn);
+    if (M <= kBM) best.pair_tn = 0;
     if (res) best.mt = 1;
     return best;
 }
@@ -671,14 +659,7 @@ int launch_variant(const GemmArgs& g, const TileChoice& tc, cudaStream_t stream)
     }
     rc = cuda_fail(cudaGetLastError(), "gemm_hif4_kernel launch");
     if (rc) return rc;
-    if (tc.splits > 1) {
-        int64_t n = g.M * g.N;
-        LaunchScope scope(kKindReduce, stream);
-        splitk_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(g.splitk_partials, tc.splits, g.M, g.N, g.Y,
-                                                                             p.out_f32, g.ldy);
-        rc = cuda_fail(cudaGetLastError(), "splitk_reduce_kernel launch");
-    }
-    return rc;
+    return launch_splitk_reduce(g, tc.splits, stream);
 }
 
 }  // namespace
@@ -705,6 +686,7 @@ int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream) {
     const bool res = g.r_bf16 != nullptr;
     TileChoice tc = choose_tile(g.M, g.N, g.K, res);
     if (tc.splits > 1 && (!g.splitk_partials || tc.splits > g.splits)) tc.splits = 1;
+    if (tc.pair_tn > 0) return launch_gemm_pair(g, tc.pair_tn, tc.splits, stream);
     if (g.fmt == kMXFP4) {
         if (res) return dispatch_tn<1, true, kMXFP4>(g, tc, stream);
         if (tc.mt == 2) return dispatch_tn<2, false, kMXFP4>(g, tc, stream);

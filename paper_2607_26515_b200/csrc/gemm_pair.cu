@@ -1,0 +1,538 @@
+// CTA-pair version of the HiF4 / MXFP4 GEMM of Eq. (5) (see gemm_hif4.cu for the numerics).
+//
+// Two CTAs on neighbouring SMs (a cluster of 2) compute one 256 x TN output tile with
+// tcgen05.mma.cta_group::2: each CTA supplies the activation rows of its own 128 token rows and expands
+// only HALF of the weight tile; the tensor cores read the other half from the peer's shared memory.
+// Against the single-CTA kernel this halves the expansion work and the weight-side shared-memory fill per
+// SM, which is what bounds that kernel.  No TMA multicast is used: every TMA load targets the issuing
+// CTA's own shared memory; only mbarrier arrivals and tcgen05.commit cross the pair.
+//
+// Roles per CTA (16 warps): warp 0 activation TMA, warp 1 MMA issue (leader CTA only) + TMEM alloc,
+// warp 2 raw weight-code TMA, warps 4..7 epilogue, warps 8..15 expanders.  The leader's "full" barriers
+// collect arrivals from both CTAs; "empty" barriers are released in both CTAs by a commit multicast.
+#include "common.cuh"
+#include "ptx.cuh"
+#include "expand.cuh"
+
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+namespace resq {
+
+namespace {
+
+constexpr int kBM = 128;
+constexpr int kBK = 64;
+constexpr int kMaxBN = 256;
+constexpr int kExpWarps = 16;
+constexpr int kExpGroups = 4;                       // expander groups take k-blocks round-robin; each group
+                                                    // owns one slot of the expanded-weight ring (SE == groups)
+constexpr int kGroupWarps = kExpWarps / kExpGroups;
+constexpr int kFirstEpiWarp = 4;
+constexpr int kFirstExpWarp = 8;
+constexpr int kThreads = 32 * (kFirstExpWarp + kExpWarps);
+constexpr int kATileBytes = kBM * kBK * 2;
+constexpr int kMaxRing = 8;
+constexpr int kSmemBudget = 232448;
+constexpr int kTmemCols = 512;
+
+struct PairParams {
+    const void* w_side;
+    int64_t M, N, K;
+    int kblocks_per_split, splits;
+    int ntiles_m, ntiles_n, num_tiles;
+    int sa, sr, se, acc_bufs;
+    void* Y;
+    int out_f32;
+    int64_t ldy;
+    float* partials;
+    DeviceStatus* status;
+    int debug;
+    unsigned int* timeline;  // debug: device buffer for a per-role event log of pair 0 (or null)
+};
+
+__device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
+    if (atomicCAS(&st->code, 0, (int)RESQ_ERR_TIMEOUT) == 0) {
+        st->where = where;
+        st->block = (int)blockIdx.x;
+    }
+}
+
+struct Trace {
+    unsigned long long* out;
+    long long t0;
+    __device__ __forceinline__ void begin() { if (out) t0 = clock64(); }
+    __device__ __forceinline__ void end(int slot) { if (out) atomicAdd(out + slot, (unsigned long long)(clock64() - t0)); }
+};
+
+struct TileCoord {
+    int64_t m0, n0;
+    int split, kb_begin, nkb;
+};
+
+template <int TN>
+__device__ __forceinline__ TileCoord decode_tile(const PairParams& p, int tile) {
+    TileCoord t;
+    t.split = tile % p.splits;
+    const int rest = tile / p.splits;
+    t.n0 = (int64_t)(rest % p.ntiles_n) * TN;
+    t.m0 = (int64_t)(rest / p.ntiles_n) * (2 * kBM);
+    const int G = (int)(p.K / kBK);
+    t.kb_begin = t.split * p.kblocks_per_split;
+    t.nkb = min(G, t.kb_begin + p.kblocks_per_split) - t.kb_begin;
+    if (t.nkb < 0) t.nkb = 0;
+    return t;
+}
+
+// TN: width of the pair's output tile (the pair computes 256 x TN); bn = MMA N; each CTA expands TN/2 rows.
+template <bool RES, int TN, int FMT>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_r,
+                 const __grid_constant__ CUtensorMap tmap_w, const PairParams p) {
+    constexpr int kAStage = kATileBytes * (RES ? 2 : 1);
+    constexpr int bn = TN > kMaxBN ? kMaxBN : TN;  // MMA N
+    constexpr int nt = TN / bn;                    // MMAs side by side in N
+    constexpr int half = bn / 2;                   // rows of each MMA's weight tile held by one CTA
+    constexpr int my_rows = nt * half;             // rows this CTA expands per k-block
+    constexpr int exp_stage = my_rows * 128, raw_stage = my_rows * 32;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int SA = p.sa, SR = p.sr, SE = p.se;
+    uint8_t* ring_a = smem;
+    uint8_t* ring_e = ring_a + (size_t)SA * kAStage;
+    uint8_t* ring_r = ring_e + (size_t)SE * exp_stage;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(ring_r + (size_t)SR * raw_stage);
+    uint64_t* a_full = bars;                   // leader: both CTAs' activation stages landed
+    uint64_t* a_empty = bars + kMaxRing;       // each CTA: the MMAs that read the stage completed
+    uint64_t* r_full = bars + 2 * kMaxRing;    // each CTA: own raw codes landed
+    uint64_t* r_empty = bars + 3 * kMaxRing;   // each CTA: own expanders consumed them
+    uint64_t* e_full = bars + 4 * kMaxRing;    // leader: both CTAs' expanded halves written
+    uint64_t* e_empty = bars + 5 * kMaxRing;   // each CTA
+    uint64_t* acc_full = bars + 6 * kMaxRing;  // [2] each CTA
+    uint64_t* acc_empty = acc_full + 2;        // [2] leader: both epilogues drained
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    unsigned int* tlog = reinterpret_cast<unsigned int*>(tmem_slot + 4);  // [8 roles][32 iterations] (512 B)
+    const bool tl = p.timeline != nullptr && (blockIdx.x >> 1) == 0;
+    constexpr int kTl0 = 96;  // first logged iteration
+#define TLOG(role, it) do { if (tl && (it) >= kTl0 && (it) < kTl0 + 32) tlog[(role) * 32 + ((it) - kTl0)] = (unsigned int)clock64(); } while (0)
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();  // 0 = leader
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    const int G = (int)(p.K / kBK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxRing; ++s) {
+            ptx::mbar_init(&a_full[s], 2);                 // one arrive.expect_tx per CTA
+            ptx::mbar_init(&a_empty[s], 1);
+            ptx::mbar_init(&r_full[s], 1);
+            ptx::mbar_init(&r_empty[s], kGroupWarps);
+            ptx::mbar_init(&e_full[s], 2 * kGroupWarps);   // one expander group of each CTA
+            ptx::mbar_init(&e_empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(&acc_full[b], 1);
+            ptx::mbar_init(&acc_empty[b], 8);              // four epilogue warps per CTA
+        }
+        *abort_flag = 0;
+        ptx::mbar_fence_init();
+    }
+    if (warp == 1) ptx::tmem_alloc_pair(tmem_slot, kTmemCols);
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::cluster_sync();  // the peer's barriers exist before anything arrives on them
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    Trace tr{(p.debug & 16) ? reinterpret_cast<unsigned long long*>(p.status) + 8 : nullptr, 0};
+    const long long t_kernel0 = clock64();
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ activation producer (both CTAs)
+        if (lane == 0) {
+            ptx::tma_prefetch_desc(&tmap_a);
+            if (RES) ptx::tma_prefetch_desc(&tmap_r);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = pair; tile < p.num_tiles && ok; tile += npairs) {
+                const TileCoord tc = decode_tile<TN>(p, tile);
+                const int my_m = (int)(tc.m0 + rank * kBM);
+                for (int i = 0; i < tc.nkb; ++i, ++it) {
+                    const int s = it % SA;
+                    tr.begin();
+                    const bool got = ptx::mbar_wait(&a_empty[s], ((it / SA) & 1) ^ 1, abort_flag);
+                    tr.end(0);
+                    if (!got) {
+                        report_timeout(p.status, 1);
+                        ok = false;
+                        break;
+                    }
+                    uint8_t* st = ring_a + (size_t)s * kAStage;
+                    TLOG(0, it);
+                    const uint32_t full = ptx::map_to_cta(&a_full[s], 0);
+                    ptx::mbar_arrive_expect_tx_cluster(full, (uint32_t)kAStage);
+                    const int kx = (tc.kb_begin + i) * kBK;
+                    ptx::tma_load_2d_pair(st, &tmap_a, full, kx, my_m);
+                    if (RES) ptx::tma_load_2d_pair(st + kATileBytes, &tmap_r, full, kx, my_m);
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ raw weight-code producer (both CTAs)
+        if (lane == 0) {
+            ptx::tma_prefetch_desc(&tmap_w);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = pair; tile < p.num_tiles && ok; tile += npairs) {
+                const TileCoord tc = decode_tile<TN>(p, tile);
+                for (int i = 0; i < tc.nkb; ++i, ++it) {
+                    const int s = it % SR;
+                    tr.begin();
+                    const bool got = ptx::mbar_wait(&r_empty[s], ((it / SR) & 1) ^ 1, abort_flag);
+                    tr.end(1);
+                    if (!got) {
+                        report_timeout(p.status, 5);
+                        ok = false;
+                        break;
+                    }
+                    TLOG(1, it);
+                    ptx::mbar_arrive_expect_tx(&r_full[s], (uint32_t)raw_stage);
+#pragma unroll
+                    for (int j = 0; j < nt; ++j)
+                        ptx::tma_load_2d(ring_r + (size_t)s * raw_stage + (size_t)j * half * 32, &tmap_w, &r_full[s],
+                                         (tc.kb_begin + i) * (kBK / 2), (int)(tc.n0 + j * bn + rank * half));
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = ptx::idesc_bf16_f32(2 * kBM, bn);
+            uint32_t it = 0;
+            int local_tile = 0;
+            bool ok = true;
+            for (int tile = pair; tile < p.num_tiles && ok; tile += npairs, ++local_tile) {
+                const TileCoord tc = decode_tile<TN>(p, tile);
+                if (tc.nkb == 0) continue;
+                const int buf = p.acc_bufs == 2 ? (local_tile & 1) : 0;
+                const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(local_tile >> 1) : (uint32_t)local_tile;
+                tr.begin();
+                const bool got_acc = ptx::mbar_wait(&acc_empty[buf], (use & 1) ^ 1, abort_flag);
+                tr.end(4);
+                if (!got_acc) {
+                    report_timeout(p.status, 6);
+                    break;
+                }
+                ptx::tc_fence_after();
+                const uint32_t d0 = tmem_base + (uint32_t)(buf * TN);
+                for (int i = 0; i < tc.nkb; ++i, ++it) {
+                    const int sa = it % SA, se = it % SE;
+                    tr.begin();
+                    ok = ptx::mbar_wait(&a_full[sa], (it / SA) & 1, abort_flag);
+                    tr.end(2);
+                    tr.begin();
+                    ok = ok && ptx::mbar_wait(&e_full[se], (it / SE) & 1, abort_flag);
+                    tr.end(3);
+                    if (!ok) {
+                        report_timeout(p.status, 2);
+                        break;
+                    }
+                    tr.begin();
+                    TLOG(2, it);
+                    ptx::tc_fence_after();
+                    const uint32_t a_addr = ptx::smem_u32(ring_a + (size_t)sa * kAStage);
+                    const uint32_t b_addr = ptx::smem_u32(ring_e + (size_t)se * exp_stage);
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k) {
+#pragma unroll
+                        for (int j = 0; j < nt; ++j) {
+                            const uint64_t bdesc = ptx::smem_desc_sw128_kmajor(b_addr + j * half * 128 + k * 32);
+                            const uint32_t d = d0 + (uint32_t)(j * bn);
+                            ptx::umma_bf16_pair(d, ptx::smem_desc_sw128_kmajor(a_addr + k * 32), bdesc, idesc,
+                                                (i > 0 || k > 0) ? 1u : 0u);
+                            if (RES)
+                                ptx::umma_bf16_pair(d, ptx::smem_desc_sw128_kmajor(a_addr + kATileBytes + k * 32), bdesc,
+                                                    idesc, 1u);
+                        }
+                    }
+                    ptx::umma_commit_pair(&a_empty[sa], 3);  // frees the stages in both CTAs
+                    ptx::umma_commit_pair(&e_empty[se], 3);
+                    TLOG(3, it);
+                    tr.end(5);
+                }
+                if (ok) ptx::umma_commit_pair(&acc_full[buf], 3);
+            }
+        }
+    } else if (warp >= kFirstExpWarp) {
+        // ------------------------------------------------------------------ expanders (both CTAs, own half)
+        // Two groups of 8 warps take alternate k-blocks, so each group has two MMA periods for one block:
+        // the per-block synchronisation latency (two waits, two arrives, one proxy fence) stays off the
+        // critical path.
+        const int ew = (warp - kFirstExpWarp) % kGroupWarps;
+        const int grp = (warp - kFirstExpWarp) / kGroupWarps;
+        constexpr int rows_per_warp = my_rows / kGroupWarps;  // 8, 16 or 32
+        const int r_begin = ew * rows_per_warp;
+        const int sub_row = lane >> 3, chunk = lane & 7;
+        uint32_t it0 = 0;  // k-block counter at the start of the current tile
+        bool ok = true;
+        for (int tile = pair; tile < p.num_tiles && ok; tile += npairs) {
+            const TileCoord tc = decode_tile<TN>(p, tile);
+            // local row l (< my_rows) is weight row n0 + (l / half) * bn + rank * half + (l % half)
+            const int l = r_begin + lane;
+            const int64_t n = tc.n0 + (int64_t)(l / half) * bn + rank * half + (l % half);
+            const bool row_ok = lane < rows_per_warp && n < p.N;
+            auto load_side = [&](int kb) -> uint32_t {
+                if (FMT == kHiF4) return ptx::ld_nc_u32(reinterpret_cast<const uint32_t*>(p.w_side) + n * G + kb);
+                return ptx::ld_nc_u16(reinterpret_cast<const uint16_t*>(p.w_side) + n * G + kb);
+            };
+            // first k-block of this tile that belongs to this group
+            int i = (int)((grp + kExpGroups - (it0 % kExpGroups)) % kExpGroups);
+            uint32_t meta_next = (row_ok && i < tc.nkb) ? load_side(tc.kb_begin + i) : 0u;
+            for (; i < tc.nkb; i += kExpGroups) {
+                const uint32_t it = it0 + (uint32_t)i;
+                const uint32_t meta_cur = meta_next;
+                if (i + kExpGroups < tc.nkb) meta_next = row_ok ? load_side(tc.kb_begin + i + kExpGroups) : 0u;
+                const int sr = it % SR, se = it % SE;
+                if (ew == 0 && lane == 0 && grp == 0) tr.begin();
+                ok = ptx::mbar_wait(&e_empty[se], ((it / SE) & 1) ^ 1, abort_flag);
+                if (ew == 0 && lane == 0 && grp == 0) { tr.end(6); tr.begin(); TLOG(4, it); }
+                ok = ok && ptx::mbar_wait(&r_full[sr], (it / SR) & 1, abort_flag);
+                if (ew == 0 && lane == 0 && grp == 0) { tr.end(7); tr.begin(); TLOG(5, it); }
+                if (!ok) {
+                    report_timeout(p.status, 3);
+                    break;
+                }
+                const uint32_t* raw = reinterpret_cast<const uint32_t*>(ring_r + (size_t)sr * raw_stage);
+                uint8_t* bexp = ring_e + (size_t)se * exp_stage;
+                constexpr int kIters = rows_per_warp / 4;
+                uint32_t cw[kIters], mw[kIters];
+#pragma unroll
+                for (int q = 0; q < kIters; ++q) {
+                    const int rl = q * 4 + sub_row;
+                    mw[q] = __shfl_sync(0xFFFFFFFFu, meta_cur, rl & 31);
+                    cw[q] = raw[(r_begin + rl) * 8 + chunk];
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&r_empty[sr]);
+#pragma unroll
+                for (int q = 0; q < kIters; ++q) {
+                    const int r = r_begin + q * 4 + sub_row;
+                    const uint4 v = FMT == kHiF4 ? expand_hif4_chunk(cw[q], mw[q], chunk)
+                                                 : expand_mxfp4_chunk(cw[q], (mw[q] >> (8 * (chunk >> 2))) & 255u);
+                    *reinterpret_cast<uint4*>(bexp + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(&e_full[se], 0));
+                if (ew == 0 && lane == 0 && grp == 0) { tr.end(8); TLOG(6, it); }
+            }
+            it0 += (uint32_t)tc.nkb;
+        }
+    } else if (warp >= kFirstEpiWarp) {
+        // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
+        const int quad = warp & 3;
+        constexpr int nchunks = TN / 32;
+        int local_tile = 0;
+        for (int tile = pair; tile < p.num_tiles; tile += npairs, ++local_tile) {
+            const TileCoord tc = decode_tile<TN>(p, tile);
+            if (tc.nkb == 0) continue;
+            const int buf = p.acc_bufs == 2 ? (local_tile & 1) : 0;
+            const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(local_tile >> 1) : (uint32_t)local_tile;
+            if (quad == 0 && lane == 0) tr.begin();
+            const bool got_full = ptx::mbar_wait(&acc_full[buf], use & 1, abort_flag);
+            if (quad == 0 && lane == 0) { tr.end(9); tr.begin(); }
+            if (!got_full) {
+                report_timeout(p.status, 4);
+                break;
+            }
+            ptx::tc_fence_after();
+            const int64_t m = tc.m0 + rank * kBM + quad * 32 + lane;
+#pragma unroll 1
+            for (int cc = 0; cc < nchunks; ++cc) {
+                uint32_t v[32];
+                ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * TN + cc * 32), v);
+                ptx::tmem_ld_wait();
+                if (cc == nchunks - 1) {
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(&acc_empty[buf], 0));
+                }
+                if (m >= p.M) continue;
+                const int64_t nb = tc.n0 + cc * 32;
+                const int64_t left = p.N - nb;
+                if (left <= 0) continue;
+                if (p.splits > 1) {
+                    float* dst = p.partials + ((int64_t)tc.split * p.M + m) * p.N + nb;
+                    if (left >= 32 && (p.N & 3) == 0) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < left) dst[j] = __uint_as_float(v[j]);
+                    }
+                } else if (p.out_f32) {
+                    float* dst = reinterpret_cast<float*>(p.Y) + m * p.ldy + nb;
+                    if (left >= 32) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < left) dst[j] = __uint_as_float(v[j]);
+                    }
+                } else {
+                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.Y) + m * p.ldy + nb;
+                    if (left >= 32) {
+                        uint32_t o[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                            o[j] = *reinterpret_cast<uint32_t*>(&b);
+                        }
+                        if ((reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {  // two full 32-byte sectors per thread
+                            ptx::st_global_v8(dst, o[0], o[1], o[2], o[3], o[4], o[5], o[6], o[7]);
+                            ptx::st_global_v8(dst + 16, o[8], o[9], o[10], o[11], o[12], o[13], o[14], o[15]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4)
+                                *reinterpret_cast<uint4*>(dst + 2 * j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < left) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                    }
+                }
+            }
+            if (quad == 0 && lane == 0) tr.end(10);
+        }
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (tl && threadIdx.x < 256) p.timeline[blockIdx.x * 256 + threadIdx.x] = tlog[threadIdx.x];
+    ptx::cluster_sync();  // no CTA leaves while the peer may still signal its barriers or read its shared memory
+    if (tr.out && threadIdx.x == 0) {
+        atomicAdd(tr.out + 11, (unsigned long long)(clock64() - t_kernel0));
+        atomicAdd(tr.out + 12, 1ull);
+    }
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
+int env_int(const char* name, int dflt) {
+    const char* v = getenv(name);
+    return v && *v ? atoi(v) : dflt;
+}
+
+template <bool RES, int TN, int FMT>
+int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream) {
+    constexpr int kAStage = kATileBytes * (RES ? 2 : 1);
+    constexpr int bn = TN > kMaxBN ? kMaxBN : TN;
+    constexpr int nt = TN / bn;
+    constexpr int half = bn / 2;
+    constexpr int my_rows = nt * half;
+    CUtensorMap ta, tr, tw;
+    int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.a_bf16, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.K * 2,
+                          kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    rc = make_tmap_2d(&tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, RES ? g.r_bf16 : g.a_bf16, (uint64_t)g.K, (uint64_t)g.M,
+                      (uint64_t)g.K * 2, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.w_codes, (uint64_t)g.K / 2, (uint64_t)g.N, (uint64_t)g.K / 2,
+                      kBK / 2, (uint32_t)half, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (rc) return rc;
+    PairParams p;
+    p.w_side = g.w_side;
+    p.M = g.M;
+    p.N = g.N;
+    p.K = g.K;
+    const int G = (int)(g.K / kBK);
+    p.splits = splits;
+    p.kblocks_per_split = (G + splits - 1) / splits;
+    p.ntiles_m = (int)((g.M + 2 * kBM - 1) / (2 * kBM));
+    p.ntiles_n = (int)((g.N + TN - 1) / TN);
+    p.num_tiles = p.ntiles_m * p.ntiles_n * splits;
+    p.acc_bufs = TN * 2 <= kTmemCols ? 2 : 1;
+    constexpr int exp_stage = my_rows * 128, raw_stage = my_rows * 32;
+    const int fixed = 1024 + 1024;
+    p.se = kExpGroups;  // one slot per expander group (a group never runs two phases ahead on a slot)
+    p.sr = env_int("RESQ_GEMM_SR", 4);
+    p.sa = std::min(kMaxRing, (kSmemBudget - fixed - p.se * exp_stage - p.sr * raw_stage) / kAStage);
+    if (p.sa < 2 || p.se > kMaxRing || p.sr > kMaxRing) {
+        set_last_error("internal: shared-memory rings do not fit (pair tile %d)", TN);
+        return RESQ_ERR_CUDA;
+    }
+    const int smem_bytes = fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage;
+    p.Y = g.Y;
+    p.out_f32 = g.out_dtype == RESQ_OUT_F32;
+    p.ldy = g.ldy;
+    p.partials = g.splitk_partials;
+    p.status = g.status;
+    p.debug = env_int("RESQ_GEMM_DEBUG", 0);
+    {
+        const char* tp = getenv("RESQ_GEMM_TIMELINE_PTR");
+        p.timeline = tp && *tp ? reinterpret_cast<unsigned int*>(strtoull(tp, nullptr, 0)) : nullptr;
+    }
+    auto kern = gemm_pair_kernel<RES, TN, FMT>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute(gemm pair)");
+    static int num_sms = 0;
+    if (num_sms == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (num_sms <= 0) num_sms = 148;
+    }
+    const int max_pairs = num_sms / 2;
+    const int npairs = std::min(p.num_tiles, max_pairs);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)(2 * npairs), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
+    {
+        LaunchScope scope(kKindGemm, stream);
+        e = cudaLaunchKernelEx(&cfg, kern, ta, tr, tw, p);
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "gemm_pair_kernel launch");
+    return launch_splitk_reduce(g, splits, stream);
+}
+
+template <bool RES, int FMT>
+int dispatch_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
+    if (tn == 128) return launch_pair_variant<RES, 128, FMT>(g, splits, stream);
+    if (tn == 256) return launch_pair_variant<RES, 256, FMT>(g, splits, stream);
+    if (tn == 512) return launch_pair_variant<RES, 512, FMT>(g, splits, stream);
+    set_last_error("internal: unsupported pair tile width %d", tn);
+    return RESQ_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_gemm_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
+    const bool res = g.r_bf16 != nullptr;
+    if (g.fmt == kMXFP4) return res ? dispatch_pair<true, kMXFP4>(g, tn, splits, stream) : dispatch_pair<false, kMXFP4>(g, tn, splits, stream);
+    return res ? dispatch_pair<true, kHiF4>(g, tn, splits, stream) : dispatch_pair<false, kHiF4>(g, tn, splits, stream);
+}
+
+}  // namespace resq
