@@ -145,6 +145,7 @@ def main():
     ap.add_argument("--layers", default=None, help="comma-separated subset of the config's layers (profiling aid)")
     ap.add_argument("--tokens", type=int, default=None, help="override M (profiling aid; not the benchmark workload)")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the end-to-end and per-kernel passes (profiling aid)")
+    ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph per step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--verbose", action="store_true")
     args = ap.parse_args()
@@ -233,6 +234,26 @@ def main():
             wc, ws = L["w_sets"][k]
             rq.resq_linear(L["x_sets"][k], wc, ws, pattern, fmt, Y=L["y"], workspace=L["work"])
 
+    # One CUDA graph per rotation set: at decode sizes the step is a dozen short kernels and the host
+    # (tensor-map encoding, launches) would otherwise be the bottleneck.  Everything the library enqueues
+    # (memsets, kernels, cluster launches) is capturable; attributes were set during warm-up.
+    graphs = []
+
+    def build_graphs():
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for k in range(n_sets):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    step(k)
+                graphs.append(g)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+
+    def step_graph(i):
+        graphs[i % n_sets].replay()
+
     def step_e2e(i):
         k = i % n_sets
         for L in layers:
@@ -289,14 +310,23 @@ def main():
         sampler.start()
         time.sleep(0.25)
     launches0 = rq.kernel_launches()
-    ms, t0, t1 = timed(step, args.steps)
-    launches = rq.kernel_launches() - launches0
+    step(0)
+    launches_per_step = rq.kernel_launches() - launches0
+    use_graph = not args.no_graph
+    if use_graph:
+        build_graphs()
+        for i in range(3):
+            step_graph(i)
+    run_step = step_graph if use_graph else step
+    config_desc["launch"] = "one CUDA graph replay per step" if use_graph else "eager launches"
+    ms, t0, t1 = timed(run_step, args.steps)
+    launches = launches_per_step * args.steps
     # keep the GPU busy a little longer so that the 100 ms sampler certainly sees the loaded state
     t_load0 = time.time()
     reps = 0
     while time.time() - t_load0 < 0.6:
         for i in range(20):
-            step(i)
+            run_step(i)
         torch.cuda.synchronize()
         reps += 1
     t_load1 = time.time()

@@ -545,26 +545,26 @@ TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res) {
             }
         }
     }
-    // CTA pairs (256 x tn tiles, 74 pairs): same per-SM tensor time as a 128 x tn single-CTA tile, half the
-    // expansion work per SM
+    // CTA pairs (256 x tn tiles, 74 pairs) for everything taller than one MMA.  Cycle model fitted to
+    // in-kernel timelines: a k-block costs the tensor time of the tile or, for narrow tiles, the ~2400-cycle
+    // hand-off floor of the pipeline, plus ~600 cycles of barrier traffic; a tile costs ~8000 cycles of
+    // fill and epilogue; a K split costs a second launch plus the partial-tile traffic.
     if (M > kBM && env_int("RESQ_GEMM_PAIR", 1)) {
         const int64_t mtiles = (M + 2 * kBM - 1) / (2 * kBM);
+        double best_pair = 1e300;
         for (int tn = 512; tn >= 128; tn /= 2) {
             const int64_t ntiles = (N + tn - 1) / tn;
             for (int splits = 1; splits <= 8; splits *= 2) {
                 if (G / splits < 4 && splits > 1) break;
                 const int64_t tiles = mtiles * ntiles * splits;
-                const int64_t per_pair = (tiles + sms / 2 - 1) / (sms / 2);
+                const int64_t rounds = (tiles + sms / 2 - 1) / (sms / 2);
                 const int kb = (G + splits - 1) / splits;
-                const double mma = tn / 256.0 * (res ? 2.0 : 1.0);
-                const double expand = tn / 2 / 256.0 * 0.8;
-                const double l2 = ((res ? 2.0 : 1.0) * 16.0 + tn / 2 * 36.0 / 1024.0) / 31.0;
-                const double per_kb = std::max(std::max(mma, expand), l2) + 0.15;
-                double cost = per_pair * kb * per_kb + 8.0;
-                if (tn > 256) cost += per_pair * 4.0;
-                if (splits > 1) cost += 8.0 + (double)M * N * splits / 2.0e5;
-                if (cost < best_cost) {
-                    best_cost = cost;
+                const double mma = tn / 256.0 * (res ? 1024.0 : 512.0);
+                const double per_kb = std::max(mma, 2400.0) + 600.0;
+                double cost = rounds * (kb * per_kb + 8000.0);
+                if (splits > 1) cost += 15000.0 + (double)splits * M * N * 8.0 / 3000.0;
+                if (cost < best_pair) {
+                    best_pair = cost;
                     best = TileChoice{1, std::min(tn, 256), splits, tn > 256 ? 2 : 1, tn};
                 }
             }

@@ -279,21 +279,28 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         bool ok = true;
         for (int tile = pair; tile < p.num_tiles && ok; tile += npairs) {
             const TileCoord tc = decode_tile<TN>(p, tile);
-            // local row l (< my_rows) is weight row n0 + (l / half) * bn + rank * half + (l % half)
-            const int l = r_begin + lane;
-            const int64_t n = tc.n0 + (int64_t)(l / half) * bn + rank * half + (l % half);
-            const bool row_ok = lane < rows_per_warp && n < p.N;
-            auto load_side = [&](int kb) -> uint32_t {
+            // local row l (< my_rows) is weight row n0 + (l / half) * bn + rank * half + (l % half);
+            // lane l owns the metadata of rows l and 32 + l of this warp's slice
+            auto row_of = [&](int l) -> int64_t { return tc.n0 + (int64_t)(l / half) * bn + rank * half + (l % half); };
+            const int64_t n_a = row_of(r_begin + lane);
+            const int64_t n_b = row_of(r_begin + (rows_per_warp > 32 ? 32 + lane : lane));
+            const bool ok_a = lane < rows_per_warp && n_a < p.N;
+            const bool ok_b = rows_per_warp > 32 && n_b < p.N;
+            auto load_side = [&](int64_t n, int kb) -> uint32_t {
                 if (FMT == kHiF4) return ptx::ld_nc_u32(reinterpret_cast<const uint32_t*>(p.w_side) + n * G + kb);
                 return ptx::ld_nc_u16(reinterpret_cast<const uint16_t*>(p.w_side) + n * G + kb);
             };
             // first k-block of this tile that belongs to this group
             int i = (int)((grp + kExpGroups - (it0 % kExpGroups)) % kExpGroups);
-            uint32_t meta_next = (row_ok && i < tc.nkb) ? load_side(tc.kb_begin + i) : 0u;
+            uint32_t ma_next = (ok_a && i < tc.nkb) ? load_side(n_a, tc.kb_begin + i) : 0u;
+            uint32_t mb_next = (ok_b && i < tc.nkb) ? load_side(n_b, tc.kb_begin + i) : 0u;
             for (; i < tc.nkb; i += kExpGroups) {
                 const uint32_t it = it0 + (uint32_t)i;
-                const uint32_t meta_cur = meta_next;
-                if (i + kExpGroups < tc.nkb) meta_next = row_ok ? load_side(tc.kb_begin + i + kExpGroups) : 0u;
+                const uint32_t ma = ma_next, mb = mb_next;
+                if (i + kExpGroups < tc.nkb) {
+                    ma_next = ok_a ? load_side(n_a, tc.kb_begin + i + kExpGroups) : 0u;
+                    mb_next = ok_b ? load_side(n_b, tc.kb_begin + i + kExpGroups) : 0u;
+                }
                 const int sr = it % SR, se = it % SE;
                 if (ew == 0 && lane == 0 && grp == 0) tr.begin();
                 ok = ptx::mbar_wait(&e_empty[se], ((it / SE) & 1) ^ 1, abort_flag);
@@ -311,7 +318,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 #pragma unroll
                 for (int q = 0; q < kIters; ++q) {
                     const int rl = q * 4 + sub_row;
-                    mw[q] = __shfl_sync(0xFFFFFFFFu, meta_cur, rl & 31);
+                    mw[q] = __shfl_sync(0xFFFFFFFFu, q < 8 ? ma : mb, rl & 31);
                     cw[q] = raw[(r_begin + rl) * 8 + chunk];
                 }
                 __syncwarp();
@@ -463,7 +470,7 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream) {
     constexpr int exp_stage = my_rows * 128, raw_stage = my_rows * 32;
     const int fixed = 1024 + 1024;
     p.se = kExpGroups;  // one slot per expander group (a group never runs two phases ahead on a slot)
-    p.sr = env_int("RESQ_GEMM_SR", 4);
+    p.sr = kExpGroups;  // the groups read k-blocks i .. i+3 concurrently
     p.sa = std::min(kMaxRing, (kSmemBudget - fixed - p.se * exp_stage - p.sr * raw_stage) / kAStage);
     if (p.sa < 2 || p.se > kMaxRing || p.sr > kMaxRing) {
         set_last_error("internal: shared-memory rings do not fit (pair tile %d)", TN);

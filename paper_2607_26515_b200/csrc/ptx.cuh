@@ -51,13 +51,37 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  `abort_flag` (shared memory) lets one role's timeout release the others quickly.
 // Each failed try_wait has slept up to kSuspendHintNs, so the cap bounds the wait to about a second.
 constexpr uint32_t kMaxWaitPolls = 1u << 16;
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    // fast path: a few non-blocking tests (the phase is usually complete already in a well-fed pipeline)
+#pragma unroll 1
+    for (int i = 0; i < 4; ++i)
+        if (mbar_test_wait(bar, parity)) return true;
     for (uint32_t i = 0; i < kMaxWaitPolls; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 7u) == 7u && *abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
+}
+
+// Warp-collective bounded wait: lane 0 polls, the outcome is broadcast.  Keeps the number of threads that
+// hammer the barrier (and the shared-memory pipe) at one per warp.  All 32 lanes must call it.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    int ok = 0;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    return ok != 0;
 }
 
 // Read-only global loads that stay where they are written: the compiler must not sink them to their first
@@ -224,6 +248,17 @@ __device__ __forceinline__ uint64_t smem_desc_sw128_kmajor(uint32_t addr) {
     d |= (uint64_t)(1024 >> 4) << 32;         // stride byte offset between 8-row groups
     d |= (uint64_t)1 << 46;                   // descriptor version for sm_100
     d |= (uint64_t)2 << 61;                   // SWIZZLE_128B
+    return d;
+}
+// Same for rows of 64 bytes with the 64-byte swizzle (chunk index XOR ((row >> 1) & 3)); 8-row groups are
+// 512 bytes apart.  Used for half k-blocks (32 bf16 per row).
+__device__ __forceinline__ uint64_t smem_desc_sw64_kmajor(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(512 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)4 << 61;  // SWIZZLE_64B
     return d;
 }
 // Instruction descriptor for kind::f16 with bf16 A/B (both K-major) and fp32 accumulation.

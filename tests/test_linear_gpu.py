@@ -111,3 +111,74 @@ def test_linear_zero_input_gives_zero():
     for pattern in ALL:
         y = m.resq_linear(x, wc, ws, pattern, out_dtype=torch.float32)
         assert not y.any()
+
+
+# ----------------------------------------------------------------------------------------------
+# Every tile configuration of the GEMM on one shape that spans several tiles and ragged edges.
+# RESQ_GEMM_* are the library's debugging overrides of its tile heuristic (read at every call).
+
+TILE_CONFIGS = [
+    {"RESQ_GEMM_PAIR_TN": "512", "RESQ_GEMM_SPLITS": "1"},
+    {"RESQ_GEMM_PAIR_TN": "512", "RESQ_GEMM_SPLITS": "2"},
+    {"RESQ_GEMM_PAIR_TN": "256", "RESQ_GEMM_SPLITS": "1"},
+    {"RESQ_GEMM_PAIR_TN": "256", "RESQ_GEMM_SPLITS": "4"},
+    {"RESQ_GEMM_PAIR_TN": "128", "RESQ_GEMM_SPLITS": "1"},
+    {"RESQ_GEMM_PAIR": "0", "RESQ_GEMM_MT": "1", "RESQ_GEMM_BN": "64", "RESQ_GEMM_NT": "1", "RESQ_GEMM_SPLITS": "1"},
+    {"RESQ_GEMM_PAIR": "0", "RESQ_GEMM_MT": "1", "RESQ_GEMM_BN": "128", "RESQ_GEMM_NT": "1", "RESQ_GEMM_SPLITS": "2"},
+    {"RESQ_GEMM_PAIR": "0", "RESQ_GEMM_MT": "1", "RESQ_GEMM_BN": "256", "RESQ_GEMM_NT": "1", "RESQ_GEMM_SPLITS": "1"},
+    {"RESQ_GEMM_PAIR": "0", "RESQ_GEMM_MT": "1", "RESQ_GEMM_BN": "256", "RESQ_GEMM_NT": "2", "RESQ_GEMM_SPLITS": "1"},
+    {"RESQ_GEMM_PAIR": "0", "RESQ_GEMM_MT": "2", "RESQ_GEMM_BN": "256", "RESQ_GEMM_NT": "1", "RESQ_GEMM_SPLITS": "1"},
+]
+
+
+@pytest.fixture(scope="module")
+def tile_case():
+    M, K, N = 400, 1152, 1336          # 2 pair tiles in M (ragged), 18 k-blocks, N not a multiple of any tile
+    xb, wb = synth_xw(77, M, K, N, n_out=5)
+    want = {}
+    for pattern in (oracle.S_NONE, oracle.S_2_4):
+        for fmt in ("hif4", "mxfp4"):
+            want[(pattern, fmt)] = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern, fmt)
+    return xb, wb, want
+
+
+@pytest.mark.parametrize("cfg", TILE_CONFIGS, ids=lambda c: ",".join(f"{k[10:]}={v}" for k, v in c.items()))
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4])
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+def test_every_tile_configuration(tile_case, cfg, pattern, fmt, monkeypatch):
+    xb, wb, want = tile_case
+    if pattern != oracle.S_NONE and cfg.get("RESQ_GEMM_MT") == "2":
+        pytest.skip("two M tiles per CTA exist only without a residual operand")
+    for k, v in cfg.items():
+        monkeypatch.setenv(k, v)
+    m = rq()
+    M, K = xb.shape
+    N = wb.shape[0]
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    work = m.alloc_workspace(m.resq_workspace_bytes(M, N, K, pattern, fmt))
+    y = m.resq_linear(to_dev(xb), wc, ws, pattern, fmt, out_dtype=torch.float32, workspace=work)
+    assert m.check(work) == 0, m.last_error()
+    w = want[(pattern, fmt)]
+    check_close(y.cpu().numpy(), w["y"], w["abs_sum"])
+
+
+# ----------------------------------------------------------------------------------------------
+# Full benchmark sizes in the launch configuration bench.py times: the GPU computes the whole layer,
+# the oracle recomputes sampled token rows (the 2:4 and per-row selections are row-local).
+
+@pytest.mark.parametrize("cfg_idx,layer,pattern", [(1, 0, oracle.S_2_4), (1, 2, oracle.S_2_4), (1, 3, oracle.S_2_4),
+                                                   (2, 1, oracle.S_ROW50), (3, 0, oracle.S_2_4)])
+def test_full_size_layers_on_sampled_rows(cfg_idx, layer, pattern):
+    m = rq()
+    cfg = CONFIGS[cfg_idx]
+    xb, wb = make_layer(cfg, layer)
+    M, K = xb.shape
+    N = wb.shape[0]
+    wc, ws = m.pack_weight(to_dev(wb))
+    work = m.alloc_workspace(m.resq_workspace_bytes(M, N, K, pattern))
+    y = m.resq_linear(to_dev(xb), wc, ws, pattern, out_dtype=torch.bfloat16, workspace=work)
+    assert m.check(work) == 0, m.last_error()
+    rows = np.unique(np.concatenate([[0, 127, 128, M - 1], np.random.default_rng(5).integers(0, M, 12)]))
+    want = oracle.resq_linear(bf16_bits_to_f32(np.ascontiguousarray(xb[rows])), bf16_bits_to_f32(wb), pattern)
+    got = y[torch.from_numpy(rows).cuda()].float().cpu().numpy()
+    check_close(got, want["y"], want["abs_sum"], bf16_out=True)
