@@ -433,14 +433,39 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
 }
 
-// Sum the split-K partial tiles in a fixed order (split 0, 1, ...) and write Y.
+// Sum the split-K partial tiles in a fixed order (split 0, 1, ...) and write Y.  Four outputs per thread
+// (128-bit loads) when N is a multiple of 4.
 __global__ void splitk_reduce_kernel(const float* __restrict__ partials, int splits, int64_t M, int64_t N, void* Y,
                                      int out_f32, int64_t ldy) {
-    int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= M * N) return;
-    int64_t m = idx / N, n = idx % N;
+    const int64_t total = M * N;
+    if ((N & 3) == 0) {
+        const int64_t idx = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+        if (idx >= total) return;
+        const int64_t m = idx / N, n = idx % N;
+        float4 acc = *reinterpret_cast<const float4*>(partials + idx);
+        for (int s = 1; s < splits; ++s) {
+            const float4 t = *reinterpret_cast<const float4*>(partials + (int64_t)s * total + idx);
+            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+        }
+        if (out_f32) {
+            float* o = reinterpret_cast<float*>(Y) + m * ldy + n;
+            o[0] = acc.x; o[1] = acc.y; o[2] = acc.z; o[3] = acc.w;
+        } else {
+            __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(Y) + m * ldy + n;
+            __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+            if ((reinterpret_cast<uintptr_t>(o) & 7u) == 0) {
+                *reinterpret_cast<uint2*>(o) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+            } else {
+                o[0] = lo.x; o[1] = lo.y; o[2] = hi.x; o[3] = hi.y;
+            }
+        }
+        return;
+    }
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int64_t m = idx / N, n = idx % N;
     float acc = partials[idx];
-    for (int s = 1; s < splits; ++s) acc += partials[(int64_t)s * M * N + idx];
+    for (int s = 1; s < splits; ++s) acc += partials[(int64_t)s * total + idx];
     if (out_f32) reinterpret_cast<float*>(Y)[m * ldy + n] = acc;
     else reinterpret_cast<__nv_bfloat16*>(Y)[m * ldy + n] = __float2bfloat16_rn(acc);
 }
@@ -487,7 +512,7 @@ int make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, const void* base, uint6
 
 int launch_splitk_reduce(const GemmArgs& g, int splits, cudaStream_t stream) {
     if (splits <= 1) return RESQ_OK;
-    const int64_t n = g.M * g.N;
+    const int64_t n = (g.N & 3) == 0 ? g.M * g.N / 4 : g.M * g.N;
     LaunchScope scope(kKindReduce, stream);
     splitk_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(g.splitk_partials, splits, g.M, g.N, g.Y,
                                                                          g.out_dtype == RESQ_OUT_F32, g.ldy);
@@ -562,7 +587,7 @@ TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res) {
                 const double mma = tn / 256.0 * (res ? 1024.0 : 512.0);
                 const double per_kb = std::max(mma, 2400.0) + 600.0;
                 double cost = rounds * (kb * per_kb + 8000.0);
-                if (splits > 1) cost += 15000.0 + (double)splits * M * N * 8.0 / 3000.0;
+                if (splits > 1) cost += 15000.0 + (double)splits * M * N * 4.0 / 1200.0;  // partial tiles: ~1.6 KB/clk
                 if (cost < best_pair) {
                     best_pair = cost;
                     best = TileChoice{1, std::min(tn, 256), splits, tn > 256 ? 2 : 1, tn};

@@ -372,7 +372,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 if (left <= 0) continue;
                 if (p.splits > 1) {
                     float* dst = p.partials + ((int64_t)tc.split * p.M + m) * p.N + nb;
-                    if (left >= 32 && (p.N & 3) == 0) {
+                    if (left >= 32 && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8)
+                            ptx::st_global_v8(dst + j, v[j], v[j + 1], v[j + 2], v[j + 3], v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
+                    } else if (left >= 32 && (p.N & 3) == 0) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
                             *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -383,7 +387,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     }
                 } else if (p.out_f32) {
                     float* dst = reinterpret_cast<float*>(p.Y) + m * p.ldy + nb;
-                    if (left >= 32) {
+                    if (left >= 32 && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8)
+                            ptx::st_global_v8(dst + j, v[j], v[j + 1], v[j + 2], v[j + 3], v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
+                    } else if (left >= 32) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
                             *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);

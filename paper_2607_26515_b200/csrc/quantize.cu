@@ -186,16 +186,32 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(const double* 
             if (match) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
         }
         __syncthreads();
-        if (tid == 0) {
-            int remaining = s_remaining;
-            int b = 255;
-            for (; b > 0; --b) {
-                int c = (int)hist[b];
-                if (c >= remaining) break;
-                remaining -= c;
+        // pick the bucket that holds the remaining-th largest key: suffix sums of the histogram by one warp
+        if (tid < 32) {
+            const int remaining = s_remaining;
+            // lane l owns buckets 8l .. 8l+7; above[l] = number of keys in buckets of higher lanes
+            int mine = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mine += (int)hist[8 * tid + j];
+            int incl = mine;  // inclusive suffix sum over lanes >= l
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int t = __shfl_down_sync(0xFFFFFFFFu, incl, o);
+                if (tid + o < 32) incl += t;
             }
-            s_prefix = prefix | ((unsigned long long)b << shift);
-            s_remaining = remaining;  // how many are still to be taken among keys sharing the new prefix
+            const int above = incl - mine;
+            const bool here = above < remaining && incl >= remaining;  // exactly one lane
+            if (here) {
+                int rem = remaining - above;
+                int b = 8 * tid + 7;
+                for (; b > 8 * tid; --b) {
+                    int c = (int)hist[b];
+                    if (c >= rem) break;
+                    rem -= c;
+                }
+                s_prefix = prefix | ((unsigned long long)b << shift);
+                s_remaining = rem;  // how many are still to be taken among keys sharing the new prefix
+            }
         }
         __syncthreads();
     }
