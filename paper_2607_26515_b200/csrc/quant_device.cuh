@@ -19,35 +19,50 @@ __device__ __forceinline__ float pow2_from_biased(int biased) {  // 2^(biased-12
 // error below 2^-22, so an exact tie can land one ulp off .5.  Inputs have at most 8 significant
 // bits (bf16 activations, and residuals of bf16 activations), which keeps every non-tie at least
 // 2^-9 away from a half-integer; snapping to a 2^-14 grid first therefore restores exact ties
-// without creating new ones.  Returns the float whose low mantissa bits hold q.
+// without creating new ones.  The snap is the rounding of the fused multiply-add itself
+// (768 + r has ulp 2^-14); the second add rounds to an integer with ties to even.
+// Returns u = 1.5 * 2^23 + q: the low mantissa bits hold q (bit 3 is clear).
+constexpr float kMagicInt = 12582912.0f;  // 1.5 * 2^23
 __device__ __forceinline__ float rne_magic(float ax, float inv) {
-    float r = fminf(__fmul_rn(ax, inv), 7.25f);
-    r = __fadd_rn(__fadd_rn(r, 768.0f), -768.0f);  // 1.5 * 2^9: ulp 2^-14
-    return __fadd_rn(r, 12582912.0f);              // 1.5 * 2^23: ulp 1, round to nearest even
+    float t = fminf(__fmaf_rn(ax, inv, 768.0f), 775.25f);  // 768 = 1.5 * 2^9; clamp keeps q <= 7
+    return __fadd_rn(t, kMagicInt - 768.0f);
 }
+// Sum over i of 16^i (or 8^i for four 3-bit keys) of the magic constant's bit pattern, modulo 2^32: what an
+// integer multiply-accumulate over the raw float bits adds on top of the packed digits.
+constexpr uint32_t kMagicBits = 0x4B400000u;
+constexpr uint32_t kNibbleBias = (uint32_t)(((uint64_t)kMagicBits * 0x11111111ull) & 0xFFFFFFFFull);
+constexpr uint32_t kOctalBias = (uint32_t)(((uint64_t)kMagicBits * (1ull + 8ull + 64ull + 512ull)) & 0xFFFFFFFFull);
 
-// top-2-of-4 (Section 4.3, item (2)): keys are the 3-bit magnitudes of four codes packed in bits
-// 15:0 of c (element i at bits 4i+2:4i, sign bits ignored).  Larger key wins, equal keys keep the
-// lower index; exactly two bits of the result are set.
-__device__ __forceinline__ uint32_t top2of4(uint32_t c) {
-    int k0 = (int)(c & 7u) * 4 + 3;
-    int k1 = (int)((c >> 4) & 7u) * 4 + 2;
-    int k2 = (int)((c >> 8) & 7u) * 4 + 1;
-    int k3 = (int)((c >> 12) & 7u) * 4;
-    int g01 = k0 > k1, g02 = k0 > k2, g03 = k0 > k3, g12 = k1 > k2, g13 = k1 > k3, g23 = k2 > k3;
-    int w0 = g01 + g02 + g03;
-    int w1 = 1 - g01 + g12 + g13;
-    int w2 = 2 - g02 - g12 + g23;
-    int w3 = 3 - g03 - g13 - g23;
+// top-2-of-4 (Section 4.3, item (2)): keys are four 3-bit magnitudes.  Larger key wins, equal keys keep
+// the lower index; exactly two bits of the result are set.
+__host__ __device__ constexpr uint32_t top2of4_keys(int q0, int q1, int q2, int q3) {
+    const int k0 = q0 * 4 + 3, k1 = q1 * 4 + 2, k2 = q2 * 4 + 1, k3 = q3 * 4;
+    const int w0 = (k0 > k1) + (k0 > k2) + (k0 > k3);
+    const int w1 = (k1 > k0) + (k1 > k2) + (k1 > k3);
+    const int w2 = (k2 > k0) + (k2 > k1) + (k2 > k3);
+    const int w3 = (k3 > k0) + (k3 > k1) + (k3 > k2);
     return (uint32_t)((w0 >= 2) | ((w1 >= 2) << 1) | ((w2 >= 2) << 2) | ((w3 >= 2) << 3));
 }
+// c: four 4-bit codes (element i at bits 4i+2:4i, sign bits ignored).
+__device__ __forceinline__ uint32_t top2of4(uint32_t c) {
+    return top2of4_keys((int)(c & 7u), (int)((c >> 4) & 7u), (int)((c >> 8) & 7u), (int)((c >> 12) & 7u));
+}
+// The same as a 4096-entry table indexed by q0 | q1<<3 | q2<<6 | q3<<9, built at compile time.
+struct Top2Table {
+    uint8_t v[4096];
+    constexpr Top2Table() : v() {
+        for (int i = 0; i < 4096; ++i) v[i] = (uint8_t)top2of4_keys(i & 7, (i >> 3) & 7, (i >> 6) & 7, (i >> 9) & 7);
+    }
+};
+__device__ const Top2Table kTop2Table{};
 
 // ------------------------------------------------------------------------------------ HiF4
 // x: the lane's 8 values.  grp_mask: the 8 lanes of this block.  lane8: lane index inside the octet.
 // Out: codes (8 nibbles, element i at bits 4i+3:4i), meta (whole-block word, same in all 8 lanes),
-// deq (signed decoded values, exact in fp32).
+// deq (signed decoded values, exact in fp32), oct (q0 | q1<<3 | q2<<6 | q3<<9 of elements 0..3 in bits 11:0
+// and of elements 4..7 in bits 27:16: the indices of the top-2-of-4 table).
 __device__ __forceinline__ void hif4_encode_lane(const float (&x)[8], unsigned grp_mask, int lane8,
-                                                 uint32_t& codes, uint32_t& meta, float (&deq)[8]) {
+                                                 uint32_t& codes, uint32_t& meta, float (&deq)[8], uint32_t& oct) {
     float m4a = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
     float m4b = fmaxf(fmaxf(fabsf(x[4]), fabsf(x[5])), fmaxf(fabsf(x[6]), fabsf(x[7])));
     float m8 = fmaxf(m4a, m4b);
@@ -60,33 +75,35 @@ __device__ __forceinline__ void hif4_encode_lane(const float (&x)[8], unsigned g
     uint32_t mant = ab & 0x7FFFFFu;
     int s = 4 * (p + 45) + 1 + (mant > 0x0C0000u) + (mant > 0x280000u) + (mant > 0x440000u) + (mant > 0x600000u);
     s = min(max(s, 0), 255);
-    int E = s >> 2, Mn = s & 3;
-    float d = (float)(4 + Mn);
-    float S1 = d * pow2_from_biased(E - 50 + 127);  // (4+Mn) * 2^(E-50)
+    const uint32_t E = (uint32_t)s >> 2, Mn = (uint32_t)s & 3u;
+    // (4+Mn) * 2^x as fp32 bits: exponent field x + 2 + 127, top mantissa bits Mn
+    const uint32_t dbits = Mn << 21;
+    const float S1 = __uint_as_float(((E + 79u) << 23) | dbits);          // (4+Mn) * 2^(E-50)
     // levels 2 and 3: raise an exponent exactly when the group would clip without it
-    int e2 = m8 > 3.5f * S1;
-    float thr3 = 1.75f * S1 * (e2 ? 2.0f : 1.0f);
-    int e3a = m4a > thr3, e3b = m4b > thr3;
-    uint32_t mine = ((uint32_t)e2 << (8 + lane8)) | ((uint32_t)(e3a | (e3b << 1)) << (16 + 2 * lane8));
+    const uint32_t e2 = m8 > 3.5f * S1;
+    const float thr3 = 1.75f * __uint_as_float(((E + 79u + e2) << 23) | dbits);
+    const uint32_t e3a = m4a > thr3, e3b = m4b > thr3;
+    const uint32_t mine = (e2 << (8 + lane8)) | ((e3a | (e3b << 1)) << (16 + 2 * lane8));
     meta = __reduce_or_sync(grp_mask, mine) | (uint32_t)s;
-    // elements: step = (4+Mn) * 2^(E-52+e2+e3)
-    float rcp_d = Mn == 0 ? 0.25f : (Mn == 1 ? 0.2f : (Mn == 2 ? (1.0f / 6.0f) : (1.0f / 7.0f)));
-    int ja = E - 52 + e2 + e3a, jb = E - 52 + e2 + e3b;
-    float step_a = d * pow2_from_biased(ja + 127), step_b = d * pow2_from_biased(jb + 127);
-    float inv_a = rcp_d * pow2_from_biased(127 - ja), inv_b = rcp_d * pow2_from_biased(127 - jb);
-    uint32_t c = 0;
+    // elements: step = (4+Mn) * 2^(E-52+e2+e3); inv = fl(1/(4+Mn)) * 2^-(E-52+e2+e3) by exponent arithmetic
+    const uint32_t rcp_bits = Mn == 0 ? 0x3E800000u : (Mn == 1 ? 0x3E4CCCCDu : (Mn == 2 ? 0x3E2AAAABu : 0x3E124925u));
+    const uint32_t ea = E + 77u + e2 + e3a, eb = E + 77u + e2 + e3b;        // biased exponent of 2^(j+2)
+    const float step_a = __uint_as_float((ea << 23) | dbits), step_b = __uint_as_float((eb << 23) | dbits);
+    const float inv_a = __uint_as_float(rcp_bits - ((ea - 129u) << 23)), inv_b = __uint_as_float(rcp_bits - ((eb - 129u) << 23));
+    uint32_t c = 0, oa = 0, ob = 0;
 #pragma unroll
     for (int i = 7; i >= 0; --i) {
-        float step = i < 4 ? step_a : step_b;
-        float inv = i < 4 ? inv_a : inv_b;
-        float t = rne_magic(fabsf(x[i]), inv);
-        uint32_t xb = __float_as_uint(x[i]);
-        uint32_t nib = (__float_as_uint(t) & 7u) | ((xb >> 28) & 8u);
-        c = c * 16u + nib;
-        float qf = __fadd_rn(t, -12582912.0f);
+        const float step = i < 4 ? step_a : step_b;
+        const float inv = i < 4 ? inv_a : inv_b;
+        const float u = rne_magic(fabsf(x[i]), inv);
+        const uint32_t ub = __float_as_uint(u);
+        c = c * 16u + (ub | ((__float_as_uint(x[i]) >> 28) & 8u));
+        if (i < 4) oa = oa * 8u + ub; else ob = ob * 8u + ub;
+        const float qf = __fadd_rn(u, -kMagicInt);
         deq[i] = copysignf(__fmul_rn(qf, step), x[i]);
     }
-    codes = c;
+    codes = c - kNibbleBias;
+    oct = ((oa - kOctalBias) & 0xFFFu) | (((ob - kOctalBias) & 0xFFFu) << 16);
 }
 
 // decode one nibble word with its block meta (used by the dequantize helper)

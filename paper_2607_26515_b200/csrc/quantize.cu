@@ -31,7 +31,7 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& r, float (&x)[8]) {
 
 __device__ __forceinline__ uint32_t pack_bf16x2_exact(float lo, float hi) {
     // the values are bf16-representable: truncation is exact
-    return (__float_as_uint(lo) >> 16) | (__float_as_uint(hi) & 0xFFFF0000u);
+    return __byte_perm(__float_as_uint(lo), __float_as_uint(hi), 0x7632);
 }
 
 __device__ __forceinline__ uint4 ld_nc_16(const void* p) {
@@ -41,16 +41,29 @@ __device__ __forceinline__ uint4 ld_nc_16(const void* p) {
     return r;
 }
 
+// oct: the 3-bit magnitude keys of elements 0..3 in bits 11:0 and of elements 4..7 in bits 27:16
+// (indices of the top-2-of-4 table).
 template <int FMT>
 __device__ __forceinline__ void encode_lane(const float (&x)[8], int lane, uint32_t& codes, uint32_t& side,
-                                            float (&deq)[8]) {
+                                            float (&deq)[8], uint32_t& oct) {
     if (FMT == kHiF4) {
         unsigned m = 0xFFu << (lane & 24);
-        hif4_encode_lane(x, m, lane & 7, codes, side, deq);
+        hif4_encode_lane(x, m, lane & 7, codes, side, deq, oct);
     } else {
         unsigned m = 0xFu << (lane & 28);
         mxfp4_encode_lane(x, m, codes, side, deq);
+        uint32_t o = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            o |= ((codes >> (4 * i)) & 7u) << (3 * i);
+            o |= ((codes >> (16 + 4 * i)) & 7u) << (16 + 3 * i);
+        }
+        oct = o;
     }
+}
+
+__device__ __forceinline__ uint32_t top2_mask8(uint32_t oct) {
+    return (uint32_t)kTop2Table.v[oct & 0xFFFu] | ((uint32_t)kTop2Table.v[(oct >> 16) & 0xFFFu] << 4);
 }
 
 template <int FMT>
@@ -87,8 +100,8 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
         if (active && m + 1 < m_end) raw = ld_nc_16(a.X + (m + 1) * a.ldx + k0);  // prefetch the next row
         float x[8], deq[8];
         unpack_bf16x8(cur, x);
-        uint32_t codes, side;
-        encode_lane<FMT>(x, lane, codes, side, deq);
+        uint32_t codes, side, oct;
+        encode_lane<FMT>(x, lane, codes, side, deq, oct);
         if (active) {
             if (a.x_codes) *reinterpret_cast<uint32_t*>(a.x_codes + m * (a.K / 2) + k0 / 2) = codes;
             if (a.x_side) store_side<FMT>(a.x_side, m, a.K, k0, lane, side);
@@ -106,10 +119,10 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
         float dx[8], rdeq[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) dx[i] = __fsub_rn(x[i], deq[i]);
-        uint32_t rcodes, rside;
-        encode_lane<FMT>(dx, lane, rcodes, rside, rdeq);
+        uint32_t rcodes, rside, roct;
+        encode_lane<FMT>(dx, lane, rcodes, rside, rdeq, roct);
         uint32_t keep = 0xFFu;
-        if (pattern == RESQ_S_2_4) keep = top2of4(rcodes) | (top2of4(rcodes >> 16) << 4);
+        if (pattern == RESQ_S_2_4) keep = top2_mask8(roct);
         if (pattern == RESQ_S_CHAN50) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) chan_acc[i] += (double)rdeq[i] * (double)rdeq[i];
@@ -299,11 +312,11 @@ __global__ void __launch_bounds__(kThreads) quant_row50_kernel(QuantArgs a) {
         if (active) raw = ld_nc_16(a.X + m * a.ldx + k0);
         float x[8], deq[8], dx[8], rdeq[8];
         unpack_bf16x8(raw, x);
-        uint32_t codes, side, rcodes, rside;
-        encode_lane<FMT>(x, lane, codes, side, deq);
+        uint32_t codes, side, rcodes, rside, oct;
+        encode_lane<FMT>(x, lane, codes, side, deq, oct);
 #pragma unroll
         for (int i = 0; i < 8; ++i) dx[i] = __fsub_rn(x[i], deq[i]);
-        encode_lane<FMT>(dx, lane, rcodes, rside, rdeq);
+        encode_lane<FMT>(dx, lane, rcodes, rside, rdeq, oct);
         if (active) {
             if (a.x_codes) *reinterpret_cast<uint32_t*>(a.x_codes + m * (K / 2) + k0 / 2) = codes;
             if (a.x_side) store_side<FMT>(a.x_side, m, K, k0, lane, side);
