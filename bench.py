@@ -33,6 +33,8 @@ METRIC = "hif4_resq_linear TFLOP/s & GB/s at 1 B200; % of FP4-tensor/HBM rooflin
 L2_BYTES = 126 * 1024 * 1024
 PATTERN_IDS = {"none": 0, "dense": 1, "2:4": 2, "row50": 3, "chan50": 4, "block": 5}
 RHO = {0: 0.0, 1: 1.0, 2: 0.5, 3: 0.5, 4: 0.5, 5: 0.5}
+# mean DRAM bytes per GEMM launch from an ncu capture of the default workload (see profiles/)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {(1, 2, "hif4"): 15.3e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -367,10 +369,13 @@ def main():
     peaks, peak_kind = load_peaks()
     gemm_tflops = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
     roofline = {
-        "kernel": "gemm_hif4_kernel (tcgen05 kind::f16 on bf16-expanded HiF4)", "bound": "tensor",
+        "kernel": "gemm_pair_kernel (tcgen05.mma cta_group::2 kind::f16 on in-kernel bf16-expanded 4-bit weights)",
+        "bound": "tensor",
         "achieved": gemm_tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
         "frac": (gemm_tflops / peaks["bf16_tflops"]) if gemm_tflops else None,
-        "peak_source": f"bf16 burst, {peak_kind}", "traffic": None,
+        "peak_source": f"bf16 burst, {peak_kind}", "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.config, pattern, fmt)),
+        "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum, mean over the step's GEMM launches "
+                          "(profiles/gemm_pair_kernel_3b-decode_2to4.md); null for workloads not captured",
         "avg_launch_us": gemm_ms * 1e3 / max(1, gemm_n), "launches": gemm_n,
         "quantizer_avg_launch_us": quant_ms * 1e3 / max(1, quant_n),
         "quantizer_share_of_kernel_time": quant_ms / max(1e-9, sum(v[0] for v in prof.values())),
