@@ -147,6 +147,8 @@ def main():
     ap.add_argument("--layers", default=None, help="comma-separated subset of the config's layers (profiling aid)")
     ap.add_argument("--tokens", type=int, default=None, help="override M (profiling aid; not the benchmark workload)")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the end-to-end and per-kernel passes (profiling aid)")
+    ap.add_argument("--quantizer-sweep", action="store_true",
+                    help="bandwidth sweep of *_quantize_act over M x K (prints a table on stderr and one JSON line)")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph per step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--verbose", action="store_true")
@@ -203,6 +205,40 @@ def main():
 
     out_dtype = torch.bfloat16 if args.out_dtype == "bf16" else torch.float32
     fmt = args.format
+
+    if args.quantizer_sweep:
+        # hif4_quantize_act / mxfp4_quantize_act alone: read bf16 X, write packed codes + metadata.
+        peaks, peak_kind = load_peaks()
+        bpe = 2.0 + (0.5625 if fmt == "hif4" else 0.53125)
+        rows = []
+        for K in (2048, 18944):
+            for M in (256, 512, 1024, 2048, 4096, 8192, 16384, 32768):
+                nbuf = max(2, int(np.ceil(1.5 * L2_BYTES / (M * K * 2))))
+                nbuf = min(nbuf, 64)
+                xs = [torch.randn((M, K), device=dev, dtype=torch.float32).to(torch.bfloat16) for _ in range(nbuf)]
+                for i in range(3):
+                    rq.quantize_act(xs[i % nbuf], fmt)
+                torch.cuda.synchronize()
+                reps = max(10, min(200, int(2e9 / (M * K * bpe))))
+                codes = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(reps):
+                    rq.quantize_act(xs[i % nbuf], fmt)
+                e1.record()
+                torch.cuda.synchronize()
+                us = e0.elapsed_time(e1) * 1e3 / reps
+                gbs = M * K * bpe / (us * 1e-6) / 1e9
+                rows.append({"M": M, "K": K, "us": us, "GB/s": gbs, "frac_of_hbm": gbs / peaks["hbm_gbs"]})
+                print(f"[quantize_act {fmt}] M={M:6d} K={K:6d}  {us:9.1f} us  {gbs:8.1f} GB/s  "
+                      f"{100 * gbs / peaks['hbm_gbs']:5.1f} % of {peak_kind} copy rate", file=sys.stderr)
+                del xs, codes
+        best = max(rows, key=lambda r: r["GB/s"])
+        print(json.dumps({"metric": f"{fmt}_quantize_act GB/s (algorithmic {bpe} B/element)", "value": best["GB/s"],
+                          "unit": "GB/s", "roofline": {"bound": "hbm", "achieved": best["GB/s"], "peak": peaks["hbm_gbs"],
+                                                       "unit": "GB/s", "frac": best["frac_of_hbm"]},
+                          "sweep": rows, "data": "synthetic", "note": "includes launch overhead at small M"}))
+        return
 
     # ---- inputs: generated once on the host, packed once (weights are packed per policy update, not per call)
     layers = []

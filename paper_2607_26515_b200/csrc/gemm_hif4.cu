@@ -59,7 +59,7 @@ struct GemmParams {
     int64_t ldy;
     float* partials;          // [splits, M, N] when splits > 1
     DeviceStatus* status;
-    int debug;                // bit 0: expanders skip the arithmetic; bit 1: no MMAs; bit 2: epilogue skips stores
+    int debug;                // bit 4 (16): accumulate per-role cycle counters after the status word
 };
 
 __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
@@ -169,10 +169,6 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         break;
                     }
                     uint8_t* st = ring_a + (size_t)s * kAStage;
-                    if (p.debug & 8) {
-                        ptx::mbar_arrive(&a_full[s]);
-                        continue;
-                    }
                     ptx::mbar_arrive_expect_tx(&a_full[s], (uint32_t)kAStage);
                     const int kx = (tc.kb_begin + i) * kBK;
 #pragma unroll
@@ -201,10 +197,6 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         report_timeout(p.status, 5);
                         ok = false;
                         break;
-                    }
-                    if (p.debug & 8) {
-                        ptx::mbar_arrive(&r_full[s]);
-                        continue;
                     }
                     ptx::mbar_arrive_expect_tx(&r_full[s], (uint32_t)raw_stage);
 #pragma unroll
@@ -251,7 +243,6 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     ptx::tc_fence_after();
                     const uint32_t a_addr = ptx::smem_u32(ring_a + (size_t)sa * kAStage);
                     const uint32_t b_addr = ptx::smem_u32(ring_e + (size_t)se * exp_stage);
-                    if (!(p.debug & 2))
 #pragma unroll
                     for (int k = 0; k < kBK / 16; ++k) {
 #pragma unroll
@@ -321,7 +312,6 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 #pragma unroll
                 for (int q = 0; q < kIters; ++q) {
                     const int rl = q * 4 + sub_row;
-                    if (p.debug & 64) { mw[q] = meta_cur0; cw[q] = meta_cur1; continue; }
                     mw[q] = __shfl_sync(0xFFFFFFFFu, q < 8 ? meta_cur0 : meta_cur1, rl & 31);
                     cw[q] = raw[(r_begin + rl) * 8 + chunk];
                 }
@@ -332,9 +322,9 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     const int r = r_begin + q * 4 + sub_row;
                     const uint4 v = FMT == kHiF4 ? expand_hif4_chunk(cw[q], mw[q], chunk)
                                                  : expand_mxfp4_chunk(cw[q], (mw[q] >> (8 * (chunk >> 2))) & 255u);
-                    if (!(p.debug & 1)) *reinterpret_cast<uint4*>(bexp + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
+                    *reinterpret_cast<uint4*>(bexp + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
                 }
-                if (!(p.debug & 32)) ptx::fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core
+                ptx::fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&e_full[se]);
                 if (ew == 0 && lane == 0) tr.end(8);
@@ -372,7 +362,7 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
                     }
-                    if (m >= p.M || (p.debug & 4)) continue;
+                    if (m >= p.M) continue;
                     const int64_t nb = tc.n0 + cc * 32;
                     const int64_t left = p.N - nb;
                     if (left <= 0) continue;
