@@ -106,6 +106,77 @@ __device__ __forceinline__ void hif4_encode_lane(const float (&x)[8], unsigned g
     oct = ((oa - kOctalBias) & 0xFFFu) | (((ob - kOctalBias) & 0xFFFu) << 16);
 }
 
+// ---- streaming variant of the same encoder, arranged for instruction count -----------------------------
+// Sign bits of 8 elements as a nibble mask (bit 4e+3 for element e).  sw[i] carries the sign of element 2i
+// in bit 15 and of element 2i+1 in bit 31 (a pair of bf16 values, or any word with those two bits).
+__device__ __forceinline__ uint32_t sign_nibbles(const uint32_t (&sw)[4]) {
+    const uint32_t p01 = __byte_perm(sw[0], sw[1], 0x7351);  // high bytes: e0, e2 | e1, e3
+    const uint32_t p23 = __byte_perm(sw[2], sw[3], 0x7351);  //             e4, e6 | e5, e7
+    const uint32_t ev = __byte_perm(p01, p23, 0x5410);       // e0 e2 e4 e6: sign in bit 7 of bytes 0..3
+    const uint32_t od = __byte_perm(p01, p23, 0x7632);       // e1 e3 e5 e7
+    return ((ev >> 4) & 0x08080808u) | (od & 0x80808080u);   // element 2k -> bit 8k+3, 2k+1 -> bit 8k+7
+}
+
+// Element loop.  cm: magnitudes q as 8 nibbles; dq: decoded magnitudes q * step (exact); oct as above.
+// CLAMP is only needed when the level-1 code saturated (block maximum above 7 * S1max) or the block holds
+// a non-finite value: otherwise the scale rule guarantees |x| / step <= 7.
+template <bool CLAMP, bool DEQ, bool OCT>
+__device__ __forceinline__ void hif4_round_elements(const float (&x)[8], float inv_a, float inv_b, float step_a,
+                                                    float step_b, uint32_t& cm, float (&dq)[8], uint32_t& oct) {
+    const float nms_a = __fmul_rn(-kMagicInt, step_a), nms_b = __fmul_rn(-kMagicInt, step_b);  // exact
+    uint32_t c = 0, oa = 0, ob = 0;
+#pragma unroll
+    for (int i = 7; i >= 0; --i) {
+        const float inv = i < 4 ? inv_a : inv_b;
+        float t = __fmaf_rn(fabsf(x[i]), inv, 768.0f);
+        if (CLAMP) t = fminf(t, 775.25f);
+        const float u = __fadd_rn(t, kMagicInt - 768.0f);
+        const uint32_t ub = __float_as_uint(u);
+        c = c * 16u + ub;
+        if (OCT) {
+            if (i < 4) oa = oa * 8u + ub; else ob = ob * 8u + ub;
+        }
+        // (magic + q) * step - magic * step: the product is exact inside the fused multiply-add
+        if (DEQ) dq[i] = __fmaf_rn(u, i < 4 ? step_a : step_b, i < 4 ? nms_a : nms_b);
+    }
+    cm = c - kNibbleBias;
+    if (OCT) oct = ((oa - kOctalBias) & 0xFFFu) | (((ob - kOctalBias) & 0xFFFu) << 16);
+}
+
+constexpr uint32_t kHif4SatBits = 0x48C40000u;  // 401408 = 7 * 1.75 * 2^15: the largest block maximum level 1 covers
+
+// Same results as hif4_encode_lane, except that `dq` holds decoded MAGNITUDES and the signs come from sw.
+template <bool DEQ, bool OCT>
+__device__ __forceinline__ void hif4_encode_stream(const float (&x)[8], const uint32_t (&sw)[4], unsigned grp_mask,
+                                                   int lane8, uint32_t& codes, uint32_t& meta, float (&dq)[8],
+                                                   uint32_t& oct) {
+    const float m4a = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
+    const float m4b = fmaxf(fmaxf(fabsf(x[4]), fabsf(x[5])), fmaxf(fabsf(x[6]), fabsf(x[7])));
+    const float m8 = fmaxf(m4a, m4b);
+    const uint32_t ab = __reduce_max_sync(grp_mask, __float_as_uint(m8));
+    const uint32_t mant = ab & 0x7FFFFFu;
+    int s = 4 * (int)(ab >> 23) - 327 + (mant > 0x0C0000u) + (mant > 0x280000u) + (mant > 0x440000u) + (mant > 0x600000u);
+    s = min(max(s, 0), 255);
+    const uint32_t E = (uint32_t)s >> 2;
+    const uint32_t dbits = ((uint32_t)s & 3u) << 21;
+    const float S1 = __uint_as_float(((E + 79u) << 23) | dbits);          // (4+Mn) * 2^(E-50)
+    const uint32_t e2 = m8 > 3.5f * S1;
+    const float thr3 = 1.75f * __uint_as_float(((E + 79u + e2) << 23) | dbits);
+    const uint32_t e3a = m4a > thr3, e3b = m4b > thr3;
+    const uint32_t mine = (e2 << (8 + lane8)) | ((e3a | (e3b << 1)) << (16 + 2 * lane8));
+    meta = __reduce_or_sync(grp_mask, mine) | (uint32_t)s;
+    const float step_a = __uint_as_float(((E + 77u + e2 + e3a) << 23) | dbits);
+    const float step_b = __uint_as_float(((E + 77u + e2 + e3b) << 23) | dbits);
+    // 1/step to within one ulp: the rounding below snaps to a 2^-14 grid, far coarser than that error
+    float inv_a, inv_b;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv_a) : "f"(step_a));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv_b) : "f"(step_b));
+    uint32_t cm;
+    if (ab > kHif4SatBits) hif4_round_elements<true, DEQ, OCT>(x, inv_a, inv_b, step_a, step_b, cm, dq, oct);
+    else hif4_round_elements<false, DEQ, OCT>(x, inv_a, inv_b, step_a, step_b, cm, dq, oct);
+    codes = cm | sign_nibbles(sw);
+}
+
 // decode one nibble word with its block meta (used by the dequantize helper)
 __device__ __forceinline__ void hif4_decode_lane(uint32_t codes, uint32_t meta, int lane8, float (&v)[8]) {
     int s = meta & 255;

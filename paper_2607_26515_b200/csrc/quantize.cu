@@ -75,11 +75,23 @@ __device__ __forceinline__ void store_side(void* side_ptr, int64_t row, int64_t 
     }
 }
 
+// Per-pair keep masks for the bf16 image: word i is 0xFFFF in the half of every kept element of (2i, 2i+1).
+// n * 0x10204080 puts bit j of a nibble n into the top bit of byte j; the permute then replicates those bits.
+__device__ __forceinline__ void keep_words(uint32_t keep, uint32_t (&km)[4]) {
+    const uint32_t zl = (keep & 15u) * 0x10204080u, zh = (keep >> 4) * 0x10204080u;
+    // prmt selector nibbles with bit 3 set replicate the top bit of the selected byte
+    asm("prmt.b32 %0, %1, 0, 0x9988;" : "=r"(km[0]) : "r"(zl));
+    asm("prmt.b32 %0, %1, 0, 0xBBAA;" : "=r"(km[1]) : "r"(zl));
+    asm("prmt.b32 %0, %1, 0, 0x9988;" : "=r"(km[2]) : "r"(zh));
+    asm("prmt.b32 %0, %1, 0, 0xBBAA;" : "=r"(km[3]) : "r"(zh));
+}
+
 // ------------------------------------------------------------------------------------------------
 // Streaming kernel for the patterns whose selection is local to a row segment (NONE, DENSE, 2:4) and
 // first pass of the global ones (CHAN50, BLOCK: writes the unmasked residual and accumulates scores).
 // grid.y: groups of 8 warps, each warp owning 256 channels; grid.x: row chunks of `rows_per_cta`.
-template <int FMT, bool RESIDUAL>
+// IMG: the bf16 images for the GEMM are written (a_bf16, and r_bf16 when RESIDUAL).
+template <int FMT, bool RESIDUAL, bool IMG>
 __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int rows_per_cta) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t k0 = ((int64_t)blockIdx.y * kWarpsPerCta + warp) * kColsPerWarp + lane * 8;
@@ -87,6 +99,11 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
     const int64_t m_begin = (int64_t)blockIdx.x * rows_per_cta;
     const int64_t m_end = min(a.M, m_begin + rows_per_cta);
     const int pattern = a.pattern;
+    const unsigned grp = FMT == kHiF4 ? 0xFFu << (lane & 24) : 0xFu << (lane & 28);
+    const int lane8 = lane & 7;
+    const bool side_lane = FMT == kHiF4 ? (lane & 7) == 0 : (lane & 3) == 0;
+    const int64_t side_cols = a.K / (FMT == kHiF4 ? kHif4Block : kMxBlock);
+    const int64_t side_k = k0 / (FMT == kHiF4 ? kHif4Block : kMxBlock);
 
     double chan_acc[8];
     double blk_acc = 0.0;
@@ -96,21 +113,42 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
     uint4 raw = make_uint4(0, 0, 0, 0);
     if (active && m_begin < m_end) raw = ld_nc_16(a.X + m_begin * a.ldx + k0);
     for (int64_t m = m_begin; m < m_end; ++m) {
-        uint4 cur = raw;
+        const uint4 cur = raw;
         if (active && m + 1 < m_end) raw = ld_nc_16(a.X + (m + 1) * a.ldx + k0);  // prefetch the next row
+        const uint32_t w[4] = {cur.x, cur.y, cur.z, cur.w};
         float x[8], deq[8];
         unpack_bf16x8(cur, x);
         uint32_t codes, side, oct;
-        encode_lane<FMT>(x, lane, codes, side, deq, oct);
+        if constexpr (FMT == kHiF4) {
+            // deq holds magnitudes here; the signs are those of x
+            hif4_encode_stream<RESIDUAL || IMG, false>(x, w, grp, lane8, codes, side, deq, oct);
+        } else {
+            encode_lane<FMT>(x, lane, codes, side, deq, oct);
+        }
         if (active) {
             if (a.x_codes) *reinterpret_cast<uint32_t*>(a.x_codes + m * (a.K / 2) + k0 / 2) = codes;
-            if (a.x_side) store_side<FMT>(a.x_side, m, a.K, k0, lane, side);
-            if (a.a_bf16) {
+            if (a.x_side && side_lane) {
+                if (FMT == kHiF4) reinterpret_cast<uint32_t*>(a.x_side)[m * side_cols + side_k] = side;
+                else reinterpret_cast<uint8_t*>(a.x_side)[m * side_cols + side_k] = (uint8_t)side;
+            }
+        }
+        if constexpr (RESIDUAL && FMT == kHiF4) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) deq[i] = copysignf(deq[i], x[i]);
+        }
+        if constexpr (IMG) {
+            if (active) {
                 uint4 o;
                 o.x = pack_bf16x2_exact(deq[0], deq[1]);
                 o.y = pack_bf16x2_exact(deq[2], deq[3]);
                 o.z = pack_bf16x2_exact(deq[4], deq[5]);
                 o.w = pack_bf16x2_exact(deq[6], deq[7]);
+                if constexpr (!RESIDUAL && FMT == kHiF4) {
+                    o.x |= w[0] & 0x80008000u;
+                    o.y |= w[1] & 0x80008000u;
+                    o.z |= w[2] & 0x80008000u;
+                    o.w |= w[3] & 0x80008000u;
+                }
                 *reinterpret_cast<uint4*>(a.a_bf16 + m * a.K + k0) = o;
             }
         }
@@ -120,7 +158,14 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
 #pragma unroll
         for (int i = 0; i < 8; ++i) dx[i] = __fsub_rn(x[i], deq[i]);
         uint32_t rcodes, rside, roct;
-        encode_lane<FMT>(dx, lane, rcodes, rside, rdeq, roct);
+        uint32_t dw[4];  // signs of dx in bits 15 / 31
+        if constexpr (FMT == kHiF4) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) dw[i] = pack_bf16x2_exact(dx[2 * i], dx[2 * i + 1]);
+            hif4_encode_stream<true, true>(dx, dw, grp, lane8, rcodes, rside, rdeq, roct);  // rdeq: magnitudes
+        } else {
+            encode_lane<FMT>(dx, lane, rcodes, rside, rdeq, roct);
+        }
         uint32_t keep = 0xFFu;
         if (pattern == RESQ_S_2_4) keep = top2_mask8(roct);
         if (pattern == RESQ_S_CHAN50) {
@@ -142,19 +187,31 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
         }
         if (active) {
             if (a.r_codes) *reinterpret_cast<uint32_t*>(a.r_codes + m * (a.K / 2) + k0 / 2) = rcodes;
-            if (a.r_side) store_side<FMT>(a.r_side, m, a.K, k0, lane, rside);
+            if (a.r_side && side_lane) {
+                if (FMT == kHiF4) reinterpret_cast<uint32_t*>(a.r_side)[m * side_cols + side_k] = rside;
+                else reinterpret_cast<uint8_t*>(a.r_side)[m * side_cols + side_k] = (uint8_t)rside;
+            }
             const bool local = pattern == RESQ_S_DENSE || pattern == RESQ_S_2_4;
             if (a.mask_bits && local) a.mask_bits[m * (a.K / 8) + k0 / 8] = (uint8_t)keep;
-            if (a.r_bf16) {
+            if constexpr (IMG) {
                 // for the global patterns this is the unmasked image; the apply kernel zeroes dropped entries
-                float r[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) r[i] = ((keep >> i) & 1u) ? rdeq[i] : 0.0f;
+                uint32_t km[4];
+                keep_words(keep, km);
                 uint4 o;
-                o.x = pack_bf16x2_exact(r[0], r[1]);
-                o.y = pack_bf16x2_exact(r[2], r[3]);
-                o.z = pack_bf16x2_exact(r[4], r[5]);
-                o.w = pack_bf16x2_exact(r[6], r[7]);
+                o.x = pack_bf16x2_exact(rdeq[0], rdeq[1]);
+                o.y = pack_bf16x2_exact(rdeq[2], rdeq[3]);
+                o.z = pack_bf16x2_exact(rdeq[4], rdeq[5]);
+                o.w = pack_bf16x2_exact(rdeq[6], rdeq[7]);
+                if constexpr (FMT == kHiF4) {
+                    o.x |= dw[0] & 0x80008000u;
+                    o.y |= dw[1] & 0x80008000u;
+                    o.z |= dw[2] & 0x80008000u;
+                    o.w |= dw[3] & 0x80008000u;
+                }
+                o.x &= km[0];
+                o.y &= km[1];
+                o.z &= km[2];
+                o.w &= km[3];
                 *reinterpret_cast<uint4*>(a.r_bf16 + m * a.K + k0) = o;
             }
         }
@@ -164,6 +221,278 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
 #pragma unroll
         for (int i = 0; i < 8; ++i) atomicAdd(&a.scores[k0 + i], chan_acc[i]);
     }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Block-per-lane streaming kernel (HiF4; NONE, DENSE, 2:4, BLOCK32x64).  A lane owns one whole block of 64
+// values, so the block maximum, the level-1 scale and the metadata word need no cross-lane traffic and the
+// scale set-up is paid once per 64 values instead of once per 8.  A warp owns 32 consecutive blocks (2048
+// channels) of a row and walks down `rows_per_warp` rows.  Global accesses stay coalesced: rows arrive
+// through a double-buffered cp.async stage in shared memory, each block padded to 144 bytes so that the
+// 128-bit accesses of 8 neighbouring lanes fall on distinct banks; the bf16 images leave the same way.
+constexpr int kStagePitch = 144;                 // bytes per staged block (128 + 16 padding)
+constexpr int kStageBytes = 32 * kStagePitch;    // one row segment of a warp
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, bool valid) {
+    const int n = valid ? 16 : 0;  // 0: the destination is zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
+
+__device__ __forceinline__ uint4 lds_16(uint32_t addr) {
+    uint4 r;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+    return r;
+}
+__device__ __forceinline__ void sts_16(uint32_t addr, const uint4& v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+// Maxima of |v| over elements 0..3 and 4..7 of a chunk of 8 bf16 values, as bf16 bit patterns
+// (non-negative bf16 values order like their bit patterns).
+__device__ __forceinline__ void chunk_maxima(const uint32_t* w, uint32_t& mA, uint32_t& mB) {
+    const uint32_t p = max_u16x2(w[0] & 0x7FFF7FFFu, w[1] & 0x7FFF7FFFu);
+    const uint32_t q = max_u16x2(w[2] & 0x7FFF7FFFu, w[3] & 0x7FFF7FFFu);
+    mA = max(p & 0xFFFFu, p >> 16);
+    mB = max(q & 0xFFFFu, q >> 16);
+}
+
+// Level-1 scale of a block from its maximum (bf16 bits), plus what the per-group decisions need.
+struct Hif4BlockScale {
+    uint32_t s;          // level-1 code
+    uint32_t base_bits;  // fp32 bits of the element step (4+Mn) * 2^(E-52) with both exponents 0
+    uint32_t inv_bits;   // fp32 bits of 1/step (to within one ulp)
+    uint32_t thr2;       // bf16 bits of 3.5 * S1: a level-2 group above it needs e2 = 1
+    uint32_t thr3;       // bf16 bits of 1.75 * S1: a level-3 group above thr3 * 2^e2 needs e3 = 1
+    bool saturated;      // the block maximum exceeds what code 255 covers (or is not finite)
+};
+
+__device__ __forceinline__ Hif4BlockScale hif4_block_scale(uint32_t amax16) {
+    Hif4BlockScale b;
+    const uint32_t ab = amax16 << 16;
+    const uint32_t mant = ab & 0x7FFFFFu;
+    int s = 4 * (int)(ab >> 23) - 327 + (mant > 0x0C0000u) + (mant > 0x280000u) + (mant > 0x440000u) + (mant > 0x600000u);
+    s = min(max(s, 0), 255);
+    b.s = (uint32_t)s;
+    const uint32_t E = (uint32_t)s >> 2, dbits = ((uint32_t)s & 3u) << 21;
+    const float S1 = __uint_as_float(((E + 79u) << 23) | dbits);  // (4+Mn) * 2^(E-50)
+    b.thr2 = __float_as_uint(3.5f * S1) >> 16;                    // 14, 17.5, 21, 24.5 times a power of two: exact in bf16
+    b.thr3 = __float_as_uint(1.75f * S1) >> 16;
+    b.base_bits = ((E + 77u) << 23) | dbits;
+    float inv;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(__uint_as_float(b.base_bits)));
+    b.inv_bits = __float_as_uint(inv);
+    b.saturated = ab > kHif4SatBits;
+    return b;
+}
+
+// One chunk of 8 values (a level-2 group) of a block whose scale is known.  w: the values as bf16 pairs.
+// Returns the 8 codes; meta_bits: this chunk's e2 / e3 bits at their place in the metadata word.
+template <bool CLAMP, bool DEQ, bool OCT>
+__device__ __forceinline__ uint32_t hif4_encode_chunk(const uint32_t* w, const Hif4BlockScale& b, uint32_t mA, uint32_t mB,
+                                                      int c, uint32_t& meta_bits, float (&x)[8], float (&dq)[8],
+                                                      uint32_t& oct) {
+    const uint32_t e2 = max(mA, mB) > b.thr2;
+    const uint32_t t3 = b.thr3 + (e2 << 7);  // bf16 exponent + e2
+    const uint32_t e3a = mA > t3, e3b = mB > t3;
+    meta_bits = (e2 << (8 + c)) | ((e3a | (e3b << 1)) << (16 + 2 * c));
+    const uint32_t na = (e2 + e3a) << 23, nb = (e2 + e3b) << 23;
+    const float step_a = __uint_as_float(b.base_bits + na), step_b = __uint_as_float(b.base_bits + nb);
+    const float inv_a = __uint_as_float(b.inv_bits - na), inv_b = __uint_as_float(b.inv_bits - nb);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        x[2 * i] = __uint_as_float(w[i] << 16);
+        x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+    uint32_t cm;
+    hif4_round_elements<CLAMP, DEQ, OCT>(x, inv_a, inv_b, step_a, step_b, cm, dq, oct);
+    const uint32_t sw[4] = {w[0], w[1], w[2], w[3]};
+    return cm | sign_nibbles(sw);
+}
+
+// Encode the lane's block held in w[32] (bf16 pairs).  Outputs the 8 code words and the metadata word.
+// Per chunk, `sink(c, x, dq, oct)` receives the unpacked values, the decoded magnitudes and the top-2-of-4
+// table indices (only what DEQ / OCT ask for is defined).
+template <bool DEQ, bool OCT, typename Sink>
+__device__ __forceinline__ void hif4_encode_block(const uint32_t (&w)[32], uint32_t (&codes)[8], uint32_t& meta, Sink&& sink) {
+    uint32_t mA[8], mB[8];
+    uint32_t amax = 0;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        chunk_maxima(&w[4 * c], mA[c], mB[c]);
+        amax = max(amax, max(mA[c], mB[c]));
+    }
+    const Hif4BlockScale b = hif4_block_scale(amax);
+    uint32_t m = b.s;
+    if (b.saturated) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            float x[8], dq[8];
+            uint32_t mb, oct = 0;
+            codes[c] = hif4_encode_chunk<true, DEQ, OCT>(&w[4 * c], b, mA[c], mB[c], c, mb, x, dq, oct);
+            m |= mb;
+            sink(c, x, dq, oct);
+        }
+    } else {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            float x[8], dq[8];
+            uint32_t mb, oct = 0;
+            codes[c] = hif4_encode_chunk<false, DEQ, OCT>(&w[4 * c], b, mA[c], mB[c], c, mb, x, dq, oct);
+            m |= mb;
+            sink(c, x, dq, oct);
+        }
+    }
+    meta = m;
+}
+
+template <bool RESIDUAL, bool IMG>
+__global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, int rows_per_warp) {
+    extern __shared__ __align__(16) uint8_t smem_q[];
+    constexpr int kBufs = IMG ? 3 : 2;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t G = a.K / kHif4Block;
+    const int64_t ncg = (G + 31) / 32;                       // column groups of 32 blocks
+    const int64_t task = (int64_t)blockIdx.x * kWarpsPerCta + warp;
+    const int64_t cg = task % ncg;
+    const int64_t m_begin = (task / ncg) * rows_per_warp;
+    const int64_t m_end = min(a.M, m_begin + rows_per_warp);
+    if (m_begin >= m_end) return;                            // warps are independent: no CTA-wide barrier below
+    const uint32_t in0 = smem_u32(smem_q) + (uint32_t)(warp * kBufs * kStageBytes);
+    const uint32_t stage = in0 + 2 * kStageBytes;            // only with IMG
+    const int pattern = a.pattern;
+
+    // cooperative row copies: piece j of lane l is chunk (l & 7) of block 4j + (l >> 3)
+    const int cp_blk = lane >> 3, cp_ch = lane & 7;
+    const uint32_t cp_smem = (uint32_t)(cp_blk * kStagePitch + cp_ch * 16);
+    const int64_t cp_col = (cg * 32 + cp_blk) * kHif4Block + cp_ch * 8;  // first channel of piece 0
+    auto issue_row = [&](int64_t m, uint32_t buf) {
+        const __nv_bfloat16* src = a.X + m * a.ldx + cp_col;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const bool valid = cp_col + j * 4 * kHif4Block < a.K;
+            cp_async_16(buf + cp_smem + j * 4 * kStagePitch, valid ? (const void*)(src + j * 4 * kHif4Block) : (const void*)a.X, valid);
+        }
+    };
+    // write-out of a staged bf16 image row (same piece mapping)
+    auto drain_stage = [&](__nv_bfloat16* dst_row) {
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint4 v = lds_16(stage + cp_smem + j * 4 * kStagePitch);
+            if (cp_col + j * 4 * kHif4Block < a.K) *reinterpret_cast<uint4*>(dst_row + cp_col + j * 4 * kHif4Block) = v;
+        }
+        __syncwarp();
+    };
+
+    const int64_t blk = cg * 32 + lane;  // the lane's block within the row
+    const bool active = blk < G;
+    const uint32_t my_in = (uint32_t)(lane * kStagePitch);
+    double blk_acc = 0.0;
+
+    issue_row(m_begin, in0);
+    cp_async_commit();
+    if (m_begin + 1 < m_end) issue_row(m_begin + 1, in0 + kStageBytes);
+    cp_async_commit();
+    for (int64_t m = m_begin; m < m_end; ++m) {
+        const uint32_t buf = in0 + (uint32_t)(((m - m_begin) & 1) * kStageBytes);
+        cp_async_wait<1>();
+        __syncwarp();
+        uint32_t w[32];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint4 v = lds_16(buf + my_in + c * 16);
+            w[4 * c] = v.x; w[4 * c + 1] = v.y; w[4 * c + 2] = v.z; w[4 * c + 3] = v.w;
+        }
+        __syncwarp();
+        if (m + 2 < m_end) issue_row(m + 2, buf);
+        cp_async_commit();  // one group per row keeps the wait count uniform
+
+        uint32_t codes[8], meta;
+        // main encode; with RESIDUAL, w is overwritten by dX = X - deq Q(X) (Eq. (3)), exact in bf16
+        hif4_encode_block<RESIDUAL || IMG, false>(w, codes, meta, [&](int c, const float (&x)[8], const float (&dq)[8], uint32_t) {
+            if constexpr (RESIDUAL) {
+                float sd[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) sd[i] = copysignf(dq[i], x[i]);
+                if constexpr (IMG)
+                    sts_16(stage + my_in + c * 16, make_uint4(pack_bf16x2_exact(sd[0], sd[1]), pack_bf16x2_exact(sd[2], sd[3]),
+                                                              pack_bf16x2_exact(sd[4], sd[5]), pack_bf16x2_exact(sd[6], sd[7])));
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    w[4 * c + i] = pack_bf16x2_exact(__fsub_rn(x[2 * i], sd[2 * i]), __fsub_rn(x[2 * i + 1], sd[2 * i + 1]));
+            } else if constexpr (IMG) {
+                uint32_t img[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) img[i] = pack_bf16x2_exact(dq[2 * i], dq[2 * i + 1]) | (w[4 * c + i] & 0x80008000u);
+                sts_16(stage + my_in + c * 16, make_uint4(img[0], img[1], img[2], img[3]));
+            }
+        });
+        if (active) {
+            if (a.x_codes) {
+                uint4* p = reinterpret_cast<uint4*>(a.x_codes + m * (a.K / 2) + blk * 32);
+                p[0] = make_uint4(codes[0], codes[1], codes[2], codes[3]);
+                p[1] = make_uint4(codes[4], codes[5], codes[6], codes[7]);
+            }
+            if (a.x_side) reinterpret_cast<uint32_t*>(a.x_side)[m * G + blk] = meta;
+        }
+        if constexpr (IMG) drain_stage(a.a_bf16 + m * a.K);
+        if constexpr (RESIDUAL) {
+            uint32_t rcodes[8], rmeta, keep_lo = 0xFFFFFFFFu, keep_hi = 0xFFFFFFFFu;
+            float sq = 0.0f;
+            hif4_encode_block<true, true>(w, rcodes, rmeta, [&](int c, const float (&)[8], const float (&rdq)[8], uint32_t roct) {
+                uint32_t keep = 0xFFu;
+                if (pattern == RESQ_S_2_4) {
+                    keep = top2_mask8(roct);
+                    if (c < 4) keep_lo = (keep_lo & ~(0xFFu << (8 * c))) | (keep << (8 * c));
+                    else keep_hi = (keep_hi & ~(0xFFu << (8 * (c - 4)))) | (keep << (8 * (c - 4)));
+                }
+                if (pattern == RESQ_S_BLOCK32x64_50) {
+                    // 64 squares of at most 12 significant bits whose exponents differ by at most 4: exact in fp32
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) sq = __fmaf_rn(rdq[i], rdq[i], sq);
+                }
+                if constexpr (IMG) {
+                    // for BLOCK this is the unmasked image; the apply kernel zeroes dropped entries
+                    uint32_t km[4];
+                    keep_words(keep, km);
+                    uint32_t img[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        img[i] = (pack_bf16x2_exact(rdq[2 * i], rdq[2 * i + 1]) | (w[4 * c + i] & 0x80008000u)) & km[i];
+                    sts_16(stage + my_in + c * 16, make_uint4(img[0], img[1], img[2], img[3]));
+                }
+            });
+            if (pattern == RESQ_S_BLOCK32x64_50) {
+                blk_acc += (double)sq;
+                if (((m + 1) % kBlkRows) == 0 || m + 1 == m_end) {
+                    if (active) atomicAdd(&a.scores[(m / kBlkRows) * G + blk], blk_acc);
+                    blk_acc = 0.0;
+                }
+            }
+            if (active) {
+                if (a.r_codes) {
+                    uint4* p = reinterpret_cast<uint4*>(a.r_codes + m * (a.K / 2) + blk * 32);
+                    p[0] = make_uint4(rcodes[0], rcodes[1], rcodes[2], rcodes[3]);
+                    p[1] = make_uint4(rcodes[4], rcodes[5], rcodes[6], rcodes[7]);
+                }
+                if (a.r_side) reinterpret_cast<uint32_t*>(a.r_side)[m * G + blk] = rmeta;
+                const bool local = pattern == RESQ_S_DENSE || pattern == RESQ_S_2_4;
+                if (a.mask_bits && local) *reinterpret_cast<uint2*>(a.mask_bits + m * (a.K / 8) + blk * 8) = make_uint2(keep_lo, keep_hi);
+            }
+            if constexpr (IMG) drain_stage(a.r_bf16 + m * a.K);
+        }
+    }
+    cp_async_wait<0>();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -496,17 +825,58 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
         cudaError_t e = cudaMemsetAsync(a.scores, 0, (size_t)nscore * sizeof(double), stream);
         if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(scores)");
     }
+    // HiF4 with a row-local or block-wise selection: block-per-lane kernel (needs 16-byte aligned outputs)
+    auto al16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
+    // Worth it once there is a warp task (32 blocks of one row) for every warp slot of the machine; below
+    // that the finer-grained kernel (a lane per 8 values) finishes sooner.
+    const int64_t block_tasks = a.M * ((a.K / kHif4Block + 31) / 32);
+    if (fmt == kHiF4 && pattern != RESQ_S_CHAN50 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
+        al16(a.a_bf16) && al16(a.r_bf16)) {
+        const bool img = a.a_bf16 != nullptr;
+        const int64_t ncg = (a.K / kHif4Block + 31) / 32;
+        int rows_per_warp = 1;
+        while (rows_per_warp < 32 && (a.M / (rows_per_warp * 2)) * ncg >= 148 * 16 * 4) rows_per_warp *= 2;
+        const int64_t tasks = ((a.M + rows_per_warp - 1) / rows_per_warp) * ncg;
+        const unsigned ctas = (unsigned)((tasks + kWarpsPerCta - 1) / kWarpsPerCta);
+        const int smem = kWarpsPerCta * (img ? 3 : 2) * kStageBytes;
+        auto launch = [&](void (*kern)(QuantArgs, int)) -> int {
+            cudaError_t attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute(quant_block_kernel)");
+            LaunchScope scope(kKindQuant, stream);
+            kern<<<ctas, kThreads, smem, stream>>>(a, rows_per_warp);
+            return cuda_fail(cudaGetLastError(), "quant_block_kernel launch");
+        };
+        int rc = residual ? (img ? launch(quant_block_kernel<true, true>) : launch(quant_block_kernel<true, false>))
+                          : (img ? launch(quant_block_kernel<false, true>) : launch(quant_block_kernel<false, false>));
+        if (rc) return rc;
+        if (global_sel) {
+            { LaunchScope scope(kKindSelect, stream);
+            topk_select_kernel<<<1, kSelThreads, 0, stream>>>(a.scores, (int)nscore, (int)(nscore / 2), a.keep_flags); }
+            rc = cuda_fail(cudaGetLastError(), "topk_select_kernel launch");
+            if (rc) return rc;
+            if (a.mask_bits || a.r_bf16) {
+                int64_t n = a.M * (a.K / 8);
+                LaunchScope scope(kKindSelect, stream);
+                apply_global_mask_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(pattern, a.M, a.K, a.keep_flags,
+                                                                                          a.mask_bits, a.r_bf16);
+                rc = cuda_fail(cudaGetLastError(), "apply_global_mask_kernel launch");
+            }
+        }
+        return rc;
+    }
     const int rows_per_cta = pick_rows_per_cta(a.M, a.K, pattern);
     dim3 grid((unsigned)((a.M + rows_per_cta - 1) / rows_per_cta),
               (unsigned)((a.K + (int64_t)kWarpsPerCta * kColsPerWarp - 1) / ((int64_t)kWarpsPerCta * kColsPerWarp)));
     {
     LaunchScope scope(kKindQuant, stream);
+    const bool img = a.a_bf16 != nullptr;  // the GEMM path asks for both images (r_bf16 whenever there is a residual)
+    auto launch = [&](auto kern) { kern<<<grid, kThreads, 0, stream>>>(a, rows_per_cta); };
     if (fmt == kHiF4) {
-        if (residual) quant_stream_kernel<kHiF4, true><<<grid, kThreads, 0, stream>>>(a, rows_per_cta);
-        else quant_stream_kernel<kHiF4, false><<<grid, kThreads, 0, stream>>>(a, rows_per_cta);
+        if (residual) img ? launch(quant_stream_kernel<kHiF4, true, true>) : launch(quant_stream_kernel<kHiF4, true, false>);
+        else img ? launch(quant_stream_kernel<kHiF4, false, true>) : launch(quant_stream_kernel<kHiF4, false, false>);
     } else {
-        if (residual) quant_stream_kernel<kMXFP4, true><<<grid, kThreads, 0, stream>>>(a, rows_per_cta);
-        else quant_stream_kernel<kMXFP4, false><<<grid, kThreads, 0, stream>>>(a, rows_per_cta);
+        if (residual) img ? launch(quant_stream_kernel<kMXFP4, true, true>) : launch(quant_stream_kernel<kMXFP4, true, false>);
+        else img ? launch(quant_stream_kernel<kMXFP4, false, true>) : launch(quant_stream_kernel<kMXFP4, false, false>);
     }
     }
     int rc = cuda_fail(cudaGetLastError(), "quant_stream_kernel launch");

@@ -92,6 +92,26 @@ def test_residual_mask_bit_exact(fmt, pattern, shape):
     assert np.array_equal(mask, want["mask"])
 
 
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4, oracle.S_BLOCK])
+def test_many_rows_per_warp(pattern):
+    """Tall, narrow input: every warp of the streaming kernel walks several rows (prefetch ring, row tail)."""
+    M, K = 38400 + 32, 192
+    bits = synth(11 + pattern, M, K, n_out=4, extremes=pattern != oracle.S_BLOCK)
+    want = oracle.quantize_residual_mask(bf16_bits_to_f32(bits), pattern, "hif4")
+    if pattern == oracle.S_NONE:
+        codes, side = rq().quantize_act(to_dev(bits), "hif4")
+        assert np.array_equal(codes.cpu().numpy(), want["x_codes"]) and np.array_equal(side_np(side), want["x_side"])
+        return
+    got = rq().residual_mask(to_dev(bits), pattern, "hif4")
+    torch.cuda.synchronize()
+    for key in ("x_codes", "x_side", "r_codes", "r_side"):
+        assert np.array_equal(side_np(got[key]), want[key]), key
+    info = want["mask_info"]
+    if pattern == oracle.S_BLOCK and not (info["exact"] or info["margin"] > 2.0 ** -40):
+        pytest.skip("score sum not exactly representable in fp64 for this draw")
+    assert np.array_equal(got["mask"].cpu().numpy(), want["mask"])
+
+
 def test_residual_mask_ties_and_zero_rows():
     # all-equal magnitudes: every selection is decided by the lower-index rule
     M, K = 64, 256
