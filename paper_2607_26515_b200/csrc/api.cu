@@ -178,11 +178,10 @@ int residual_mask(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, int
 
 size_t linear_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K, int pattern) {
     if (M <= 0 || N <= 0 || K <= 0) return 0;
-    size_t b = kWsHeader + quant_scratch_bytes(M, K, pattern);
+    size_t b = kWsHeader + kWsFlags + quant_scratch_bytes(M, K, pattern);
     b += align_up((size_t)M * (size_t)K * 2, 256);                            // bf16 image of deq Q(X)
     if (pattern != RESQ_S_NONE) b += align_up((size_t)M * (size_t)K * 2, 256);  // bf16 image of S(deq Q(dX))
-    int splits = gemm_hif4_pick_splits(M, N, K);
-    if (splits > 1) b += align_up((size_t)splits * (size_t)M * (size_t)N * 4, 256);
+    b += align_up(gemm_hif4_scratch_bytes(M, N, K), 256);                     // fp32 partial tiles of a K split
     return b;
 }
 
@@ -212,7 +211,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     rc = check_workspace(workspace, ws_bytes, linear_workspace_bytes(fmt, M, N, K, pattern));
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemsetAsync(workspace, 0, kWsHeader, st);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kWsHeader + kWsFlags, st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(status)");
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     QuantArgs a;
@@ -223,7 +222,9 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     a.ldx = ldx;
     a.pattern = pattern;
     size_t used = 0;
-    carve_quant_scratch(ws, M, K, pattern, a, used);
+    carve_quant_scratch(ws + kWsFlags, M, K, pattern, a, used);
+    a.status = reinterpret_cast<DeviceStatus*>(ws);
+    used += kWsFlags;
     a.a_bf16 = reinterpret_cast<__nv_bfloat16*>(ws + used);
     used += align_up((size_t)M * (size_t)K * 2, 256);
     if (pattern != RESQ_S_NONE) {
@@ -245,8 +246,10 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     g.Y = Y;
     g.out_dtype = out_dtype;
     g.ldy = ldy;
-    g.splits = gemm_hif4_pick_splits(M, N, K);
-    g.splitk_partials = g.splits > 1 ? reinterpret_cast<float*>(ws + used) : nullptr;
+    g.partial_bytes = gemm_hif4_scratch_bytes(M, N, K);
+    g.splitk_partials = g.partial_bytes ? reinterpret_cast<float*>(ws + used) : nullptr;
+    g.splits = (int)(g.partial_bytes / ((size_t)M * (size_t)N * 4));
+    g.sk_flags = reinterpret_cast<unsigned int*>(ws + kWsHeader);
     g.status = a.status;
     return launch_gemm_hif4(g, st);
 }

@@ -17,6 +17,7 @@ constexpr int kE6M2Bias = 48;      // S1 = (1 + Mn/4) * 2^(E - 48)
 constexpr int kBlkRows = 32;       // S^{32x64}: 32 token rows ...
 constexpr int kBlkCols = 64;       // ... by 64 channels
 constexpr size_t kWsHeader = 256;  // status word + padding at the start of every workspace
+constexpr size_t kWsFlags = 2048;  // linear-layer workspaces: arrival counters of the K-streamed GEMM, right after the header
 
 // Device status word layout (first 16 bytes of the workspace).
 struct DeviceStatus {
@@ -78,8 +79,10 @@ struct GemmArgs {
     void* Y;
     int out_dtype;
     int64_t ldy;
-    float* splitk_partials;        // [splits, M, N] fp32 when splits > 1
-    int splits;
+    float* splitk_partials;        // fp32 scratch for partial tiles: [splits, M, N] slabs, or tile slots (K-streamed schedule)
+    int splits;                    // slabs that fit in splitk_partials
+    size_t partial_bytes;          // size of splitk_partials
+    unsigned int* sk_flags;        // kWsFlags bytes of zeroed counters (K-streamed schedule)
     DeviceStatus* status;
 };
 int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream);
@@ -87,5 +90,6 @@ int make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, const void* base, uint6
                  uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle sw);
 int launch_splitk_reduce(const GemmArgs& g, int splits, cudaStream_t stream);
 int gemm_hif4_pick_splits(int64_t M, int64_t N, int64_t K);
+size_t gemm_hif4_scratch_bytes(int64_t M, int64_t N, int64_t K);  // what splitk_partials must hold for this shape
 
 }  // namespace resq

@@ -25,6 +25,7 @@
 #include "expand.cuh"
 
 #include <algorithm>
+#include <cstdio>
 #include <cstdlib>
 #include <mutex>
 
@@ -510,6 +511,8 @@ int launch_splitk_reduce(const GemmArgs& g, int splits, cudaStream_t stream) {
 }
 
 int launch_gemm_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream);
+int launch_gemm_pair_streamk(const GemmArgs& g, cudaStream_t stream);
+size_t gemm_pair_streamk_scratch_bytes();
 
 namespace {
 
@@ -560,22 +563,26 @@ TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res) {
             }
         }
     }
-    // CTA pairs (256 x tn tiles, 74 pairs) for everything taller than one MMA.  Cycle model fitted to
-    // in-kernel timelines: a k-block costs the tensor time of the tile or, for narrow tiles, the ~2400-cycle
-    // hand-off floor of the pipeline, plus ~600 cycles of barrier traffic; a tile costs ~8000 cycles of
-    // fill and epilogue; a K split costs a second launch plus the partial-tile traffic.
+    // CTA pairs (256 x tn tiles, 74 pairs) for everything taller than one MMA.  Cycle model fitted to in-kernel
+    // timelines: a k-block costs the tensor time of the tile or, when the activation ring is shallow, the ring's
+    // round trip (stage freed -> TMA issued -> data landed -> MMA woken, ~6500 cycles when every pair pulls the
+    // same activation tiles) divided by its depth; a tile costs ~8000 cycles of fill and epilogue; a K split
+    // costs a second launch plus the partial-tile traffic.
     if (M > kBM && env_int("RESQ_GEMM_PAIR", 1)) {
         const int64_t mtiles = (M + 2 * kBM - 1) / (2 * kBM);
         double best_pair = 1e300;
-        for (int tn = 512; tn >= 128; tn /= 2) {
+        for (int tn : {512, 256, 128}) {
             const int64_t ntiles = (N + tn - 1) / tn;
+            const int groups = tn == 128 ? 4 : 3;                                    // as dispatched in gemm_pair.cu
+            const int ring = groups * (tn / 2) * 160;                                // expanded + raw stages
+            const int sa = std::min(8, (kSmemBudget - 2048 - ring) / (res ? 32768 : 16384));
             for (int splits = 1; splits <= 8; splits *= 2) {
                 if (G / splits < 4 && splits > 1) break;
                 const int64_t tiles = mtiles * ntiles * splits;
                 const int64_t rounds = (tiles + sms / 2 - 1) / (sms / 2);
                 const int kb = (G + splits - 1) / splits;
                 const double mma = tn / 256.0 * (res ? 1024.0 : 512.0);
-                const double per_kb = std::max(mma, 2400.0) + 600.0;
+                const double per_kb = std::max(mma, 6500.0 / sa) + 300.0;
                 double cost = rounds * (kb * per_kb + 8000.0);
                 if (splits > 1) cost += 15000.0 + (double)splits * M * N * 4.0 / 1200.0;  // partial tiles: ~1.6 KB/clk
                 if (cost < best_pair) {
@@ -679,6 +686,26 @@ int launch_variant(const GemmArgs& g, const TileChoice& tc, cudaStream_t stream)
 
 }  // namespace
 
+// K-streamed schedule of the pair kernel: used when there are too few 256 x 256 output tiles to give every CTA
+// pair whole tiles (decode-sized M): the (tile, k-block) units are dealt out evenly instead.
+bool gemm_use_streamk(int64_t M, int64_t N, int64_t K) {
+    if (M <= kBM || !env_int("RESQ_GEMM_PAIR", 1)) return false;
+    const int force = env_int("RESQ_GEMM_STREAMK", -1);
+    if (force >= 0) return force != 0;
+    if (env_int("RESQ_GEMM_PAIR_TN", 0) || env_int("RESQ_GEMM_SPLITS", 0)) return false;  // explicit tile exploration
+    const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + 255) / 256);
+    return tiles <= 74 / 2 && tiles * (K / kBK) >= 2;  // at least two pairs per tile: otherwise whole tiles per pair
+}
+
+size_t gemm_hif4_scratch_bytes(int64_t M, int64_t N, int64_t K) {
+    size_t classic = 0;
+    const int splits = gemm_hif4_pick_splits(M, N, K);
+    if (splits > 1) classic = (size_t)splits * (size_t)M * (size_t)N * 4;
+    // the K-streamed schedule may be switched on or off by the debugging overrides: size for both
+    const size_t sk = M > kBM ? gemm_pair_streamk_scratch_bytes() : 0;
+    return std::max(classic, sk);
+}
+
 int gemm_hif4_pick_splits(int64_t M, int64_t N, int64_t K) {
     // the workspace must cover the larger of the two possible choices (with / without residual)
     return std::max(choose_tile(M, N, K, false).splits, choose_tile(M, N, K, true).splits);
@@ -699,8 +726,14 @@ int dispatch_tn(const GemmArgs& g, const TileChoice& tc, cudaStream_t stream) {
 
 int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream) {
     const bool res = g.r_bf16 != nullptr;
+    if (gemm_use_streamk(g.M, g.N, g.K) && g.splitk_partials && g.sk_flags &&
+        g.partial_bytes >= gemm_pair_streamk_scratch_bytes())
+        return launch_gemm_pair_streamk(g, stream);
     TileChoice tc = choose_tile(g.M, g.N, g.K, res);
     if (tc.splits > 1 && (!g.splitk_partials || tc.splits > g.splits)) tc.splits = 1;
+    if (env_int("RESQ_GEMM_DEBUG", 0) & 1)
+        fprintf(stderr, "resq gemm M=%lld N=%lld K=%lld res=%d: pair_tn=%d mt=%d bn=%d nt=%d splits=%d\n", (long long)g.M,
+                (long long)g.N, (long long)g.K, (int)res, tc.pair_tn, tc.mt, tc.bn, tc.nt, tc.splits);
     if (tc.pair_tn > 0) return launch_gemm_pair(g, tc.pair_tn, tc.splits, stream);
     if (g.fmt == kMXFP4) {
         if (res) return dispatch_tn<1, true, kMXFP4>(g, tc, stream);

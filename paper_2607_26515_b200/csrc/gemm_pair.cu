@@ -7,8 +7,8 @@
 // SM, which is what bounds that kernel.  No TMA multicast is used: every TMA load targets the issuing
 // CTA's own shared memory; only mbarrier arrivals and tcgen05.commit cross the pair.
 //
-// Roles per CTA (16 warps): warp 0 activation TMA, warp 1 MMA issue (leader CTA only) + TMEM alloc,
-// warp 2 raw weight-code TMA, warps 4..7 epilogue, warps 8..15 expanders.  The leader's "full" barriers
+// Roles per CTA (24 warps): warp 0 activation TMA, warp 1 MMA issue (leader CTA only) + TMEM alloc,
+// warp 2 raw weight-code TMA, warps 4..7 epilogue, warps 8..23 expanders.  The leader's "full" barriers
 // collect arrivals from both CTAs; "empty" barriers are released in both CTAs by a commit multicast.
 #include "common.cuh"
 #include "ptx.cuh"
@@ -26,13 +26,15 @@ namespace {
 constexpr int kBM = 128;
 constexpr int kBK = 64;
 constexpr int kMaxBN = 256;
-constexpr int kExpWarps = 16;
-constexpr int kExpGroups = 4;                       // expander groups take k-blocks round-robin; each group
-                                                    // owns one slot of the expanded-weight ring (SE == groups)
-constexpr int kGroupWarps = kExpWarps / kExpGroups;
+constexpr int kGroupWarps = 4;                       // expander warps per group
+// Expander groups take k-blocks round-robin; each group owns one slot of the expanded-weight ring and of the
+// raw-code ring (SE == SR == groups).  The number of groups NG (four warps each) is a template parameter of the
+// kernel: more groups tolerate more hand-off latency on the weight side, fewer groups leave more shared memory
+// to the activation ring, whose round trip (stage freed -> TMA issued -> data landed -> MMAs issued) otherwise
+// bounds the k-block rate.
 constexpr int kFirstEpiWarp = 4;
 constexpr int kFirstExpWarp = 8;
-constexpr int kThreads = 32 * (kFirstExpWarp + kExpWarps);
+constexpr int pair_threads(int groups) { return 32 * (kFirstExpWarp + kGroupWarps * groups); }
 constexpr int kATileBytes = kBM * kBK * 2;
 constexpr int kMaxRing = 8;
 constexpr int kSmemBudget = 232448;
@@ -51,6 +53,12 @@ struct PairParams {
     DeviceStatus* status;
     int debug;
     unsigned int* timeline;  // debug: device buffer for a per-role event log of pair 0 (or null)
+    int timeline_first;      // debug: first k-block iteration that is logged
+    // K-streamed schedule (streamk != 0): the num_tiles * G (tile, k-block) units are dealt out evenly to the
+    // pairs; a pair's first and last segment may cover only part of a tile's K range and then go to fp32 slots
+    int streamk;
+    float* sk_slots;         // [2 * npairs][256][TN] fp32: slot 2p = first segment of pair p, 2p + 1 = its last
+    unsigned int* sk_flags;  // [num_tiles][2]: segments of the tile written, per CTA rank (zeroed before launch)
 };
 
 __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
@@ -70,6 +78,9 @@ struct Trace {
 struct TileCoord {
     int64_t m0, n0;
     int split, kb_begin, nkb;
+    int tile_id;   // K-streamed schedule: output tile of the segment
+    int slot;      //   and where its fp32 partial goes
+    bool partial;  // the segment does not cover the whole K range (or K is split): fp32 partial output
 };
 
 template <int TN>
@@ -83,17 +94,155 @@ __device__ __forceinline__ TileCoord decode_tile(const PairParams& p, int tile) 
     t.kb_begin = t.split * p.kblocks_per_split;
     t.nkb = min(G, t.kb_begin + p.kblocks_per_split) - t.kb_begin;
     if (t.nkb < 0) t.nkb = 0;
+    t.tile_id = rest;
+    t.slot = 0;
+    t.partial = p.splits > 1;
     return t;
 }
 
+// K-streamed schedule: pair q owns units [q * U / P, (q + 1) * U / P) of the U = num_tiles * G (tile, k-block)
+// units, tile-major.
+__device__ __forceinline__ int64_t sk_begin(int64_t U, int P, int q) { return (int64_t)q * U / P; }
+__device__ __forceinline__ int sk_pair_of(int64_t U, int P, int64_t u) { return (int)((((u + 1) * P) - 1) / U); }
+
+// Walks the work of one pair in the order every role of the kernel uses.
+template <int TN>
+struct SegIter {
+    const PairParams& p;
+    int pair, npairs, G;
+    int tile;            // tile schedule: next tile
+    int64_t u0, u, u1;   // K-streamed schedule: this pair's units
+    __device__ SegIter(const PairParams& p_, int pair_, int npairs_) : p(p_), pair(pair_), npairs(npairs_) {
+        G = (int)(p.K / kBK);
+        tile = pair;
+        if (p.streamk) {
+            const int64_t U = (int64_t)p.num_tiles * G;
+            u0 = u = sk_begin(U, npairs, pair);
+            u1 = sk_begin(U, npairs, pair + 1);
+        }
+    }
+    __device__ bool next(TileCoord& tc) {
+        if (!p.streamk) {
+            if (tile >= p.num_tiles) return false;
+            tc = decode_tile<TN>(p, tile);
+            tile += npairs;
+            return true;
+        }
+        if (u >= u1) return false;
+        const int t = (int)(u / G);
+        tc.tile_id = t;
+        tc.split = 0;
+        tc.kb_begin = (int)(u - (int64_t)t * G);
+        tc.nkb = (int)min((int64_t)(G - tc.kb_begin), u1 - u);
+        tc.n0 = (int64_t)(t % p.ntiles_n) * TN;
+        tc.m0 = (int64_t)(t / p.ntiles_n) * (2 * kBM);
+        tc.partial = tc.nkb < G;
+        tc.slot = 2 * pair + (u == u0 ? 0 : 1);
+        u += tc.nkb;
+        return true;
+    }
+};
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_cg_f4(const float* p) {
+    float4 v;
+    asm volatile("ld.global.cg.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+
+// End of the K-streamed kernel: the tiles whose K range this pair shared with other pairs are summed here.
+// The pairs that hold segments of a tile each reduce one column slice of it: they wait until all segments of
+// the tile are in their slots, then add them in k order (a fixed order: the result does not depend on timing).
+// Called by all threads of the CTA; the CTA of rank r handles rows r * 128 .. r * 128 + 127 of the tile.
+template <int TN>
+__device__ __forceinline__ void streamk_fixup(const PairParams& p, int pair, int npairs, int rank, volatile int* abort_flag,
+                                              volatile int* s_ok, int* s_slots) {
+    const int G = (int)(p.K / kBK);
+    const int64_t U = (int64_t)p.num_tiles * G;
+    const int64_t u0 = sk_begin(U, npairs, pair), u1 = sk_begin(U, npairs, pair + 1);
+    if (u1 <= u0) return;
+    const int t_first = (int)(u0 / G), t_last = (int)((u1 - 1) / G);
+    for (int which = 0; which < 2; ++which) {
+        const int t = which == 0 ? t_first : t_last;
+        if (which == 1 && t_last == t_first) break;
+        const int64_t tb = (int64_t)t * G, te = tb + G;
+        if (u0 <= tb && u1 >= te) continue;  // this pair computed the whole tile and wrote it out directly
+        const int pf = sk_pair_of(U, npairs, tb), pl = sk_pair_of(U, npairs, te - 1);
+        const int nseg = pl - pf + 1, j = pair - pf;
+        if (threadIdx.x == 0) {
+            int ok = *abort_flag ? 0 : 1;
+            const unsigned int* flag = p.sk_flags + t * 2 + rank;
+            for (int polls = 0; ok && ld_acquire_u32(flag) < (unsigned)nseg; ++polls) {
+                __nanosleep(200);
+                if (polls > (1 << 20)) {
+                    report_timeout(p.status, 7);
+                    ok = 0;
+                }
+            }
+            *s_ok = ok;
+        }
+        __syncthreads();
+        const bool ok = *s_ok != 0;
+        __syncthreads();
+        if (!ok) return;
+        // slot of every segment (k order), worked out once per tile
+        if ((int)threadIdx.x < nseg) {
+            const int q = pf + (int)threadIdx.x;
+            s_slots[threadIdx.x] = 2 * q + (sk_begin(U, npairs, q) >= tb ? 0 : 1);
+        }
+        __syncthreads();
+        // column slice j of nseg, in units of 4 columns
+        const int c0 = (int)((int64_t)j * (TN / 4) / nseg) * 4, c1 = (int)((int64_t)(j + 1) * (TN / 4) / nseg) * 4;
+        const int w4 = (c1 - c0) / 4;
+        const int64_t m_base = (int64_t)(t / p.ntiles_n) * (2 * kBM) + rank * kBM;
+        const int64_t n_base = (int64_t)(t % p.ntiles_n) * TN;
+        for (int item = threadIdx.x; item < kBM * w4; item += (int)blockDim.x) {
+            const int row = item / w4, c = c0 + (item % w4) * 4;
+            const int64_t m = m_base + row, n = n_base + c;
+            if (m >= p.M || n >= p.N) continue;
+            const float* src = p.sk_slots + ((size_t)rank * kBM + row) * TN + c;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int s0 = 0; s0 < nseg; s0 += 4) {
+                float4 v[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)  // the loads of a group of four segments are in flight together
+                    v[e] = s0 + e < nseg ? ld_cg_f4(src + (size_t)s_slots[s0 + e] * (2 * kBM) * TN) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    acc.x += v[e].x; acc.y += v[e].y; acc.z += v[e].z; acc.w += v[e].w;
+                }
+            }
+            const float o[4] = {acc.x, acc.y, acc.z, acc.w};
+            if (p.out_f32) {
+                float* dst = reinterpret_cast<float*>(p.Y) + m * p.ldy + n;
+                if (n + 3 < p.N) *reinterpret_cast<float4*>(dst) = acc;
+                else for (int e = 0; e < 4; ++e) if (n + e < p.N) dst[e] = o[e];
+            } else {
+                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.Y) + m * p.ldy + n;
+                if (n + 3 < p.N) {
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+                    *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+                } else {
+                    for (int e = 0; e < 4; ++e) if (n + e < p.N) dst[e] = __float2bfloat16_rn(o[e]);
+                }
+            }
+        }
+    }
+}
+
 // TN: width of the pair's output tile (the pair computes 256 x TN); bn = MMA N; each CTA expands TN/2 rows.
-template <bool RES, int TN, int FMT>
-__global__ void __launch_bounds__(kThreads, 1)
+template <bool RES, int TN, int FMT, int NG>
+__global__ void __launch_bounds__(pair_threads(NG), 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_r,
                  const __grid_constant__ CUtensorMap tmap_w, const PairParams p) {
+    constexpr int kExpGroups = NG;
     constexpr int kAStage = kATileBytes * (RES ? 2 : 1);
-    constexpr int bn = TN > kMaxBN ? kMaxBN : TN;  // MMA N
-    constexpr int nt = TN / bn;                    // MMAs side by side in N
+    constexpr int nt = TN > kMaxBN ? 2 : 1;           // MMAs side by side in N
+    constexpr int bn = TN / nt;                    // MMA N
     constexpr int half = bn / 2;                   // rows of each MMA's weight tile held by one CTA
     constexpr int my_rows = nt * half;             // rows this CTA expands per k-block
     constexpr int exp_stage = my_rows * 128, raw_stage = my_rows * 32;
@@ -116,7 +265,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     unsigned int* tlog = reinterpret_cast<unsigned int*>(tmem_slot + 4);  // [8 roles][32 iterations] (512 B)
     const bool tl = p.timeline != nullptr && (blockIdx.x >> 1) == 0;
-    constexpr int kTl0 = 96;  // first logged iteration
+    const int kTl0 = p.timeline_first;  // first logged iteration
 #define TLOG(role, it) do { if (tl && (it) >= kTl0 && (it) < kTl0 + 32) tlog[(role) * 32 + ((it) - kTl0)] = (unsigned int)clock64(); } while (0)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -156,8 +305,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             if (RES) ptx::tma_prefetch_desc(&tmap_r);
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = pair; tile < p.num_tiles && ok; tile += npairs) {
-                const TileCoord tc = decode_tile<TN>(p, tile);
+            SegIter<TN> si(p, pair, npairs);
+            TileCoord tc;
+            while (ok && si.next(tc)) {
                 const int my_m = (int)(tc.m0 + rank * kBM);
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
                     const int s = it % SA;
@@ -185,8 +335,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             ptx::tma_prefetch_desc(&tmap_w);
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = pair; tile < p.num_tiles && ok; tile += npairs) {
-                const TileCoord tc = decode_tile<TN>(p, tile);
+            SegIter<TN> si(p, pair, npairs);
+            TileCoord tc;
+            while (ok && si.next(tc)) {
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
                     const int s = it % SR;
                     tr.begin();
@@ -213,11 +364,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             uint32_t it = 0;
             int local_tile = 0;
             bool ok = true;
-            for (int tile = pair; tile < p.num_tiles && ok; tile += npairs, ++local_tile) {
-                const TileCoord tc = decode_tile<TN>(p, tile);
+            SegIter<TN> si(p, pair, npairs);
+            TileCoord tc;
+            while (ok && si.next(tc)) {
+                const int lt = local_tile++;
                 if (tc.nkb == 0) continue;
-                const int buf = p.acc_bufs == 2 ? (local_tile & 1) : 0;
-                const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(local_tile >> 1) : (uint32_t)local_tile;
+                const int buf = p.acc_bufs == 2 ? (lt & 1) : 0;
+                const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(lt >> 1) : (uint32_t)lt;
                 tr.begin();
                 const bool got_acc = ptx::mbar_wait(&acc_empty[buf], (use & 1) ^ 1, abort_flag);
                 tr.end(4);
@@ -232,6 +385,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     tr.begin();
                     ok = ptx::mbar_wait(&a_full[sa], (it / SA) & 1, abort_flag);
                     tr.end(2);
+                    TLOG(7, it);
                     tr.begin();
                     ok = ok && ptx::mbar_wait(&e_full[se], (it / SE) & 1, abort_flag);
                     tr.end(3);
@@ -277,8 +431,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         const int sub_row = lane >> 3, chunk = lane & 7;
         uint32_t it0 = 0;  // k-block counter at the start of the current tile
         bool ok = true;
-        for (int tile = pair; tile < p.num_tiles && ok; tile += npairs) {
-            const TileCoord tc = decode_tile<TN>(p, tile);
+        SegIter<TN> si(p, pair, npairs);
+        TileCoord tc;
+        while (ok && si.next(tc)) {
             // local row l (< my_rows) is weight row n0 + (l / half) * bn + rank * half + (l % half);
             // lane l owns the metadata of rows l and 32 + l of this warp's slice
             auto row_of = [&](int l) -> int64_t { return tc.n0 + (int64_t)(l / half) * bn + rank * half + (l % half); };
@@ -342,11 +497,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         const int quad = warp & 3;
         constexpr int nchunks = TN / 32;
         int local_tile = 0;
-        for (int tile = pair; tile < p.num_tiles; tile += npairs, ++local_tile) {
-            const TileCoord tc = decode_tile<TN>(p, tile);
+        SegIter<TN> si(p, pair, npairs);
+        TileCoord tc;
+        while (si.next(tc)) {
+            const int lt = local_tile++;
             if (tc.nkb == 0) continue;
-            const int buf = p.acc_bufs == 2 ? (local_tile & 1) : 0;
-            const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(local_tile >> 1) : (uint32_t)local_tile;
+            const int buf = p.acc_bufs == 2 ? (lt & 1) : 0;
+            const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(lt >> 1) : (uint32_t)lt;
             if (quad == 0 && lane == 0) tr.begin();
             const bool got_full = ptx::mbar_wait(&acc_full[buf], use & 1, abort_flag);
             if (quad == 0 && lane == 0) { tr.end(9); tr.begin(); }
@@ -365,6 +522,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(&acc_empty[buf], 0));
+                }
+                if (p.streamk && tc.partial) {
+                    // dense fp32 slot [256][TN]; rows / columns outside the matrix hold zeros
+                    float* dst = p.sk_slots + ((size_t)tc.slot * (2 * kBM) + rank * kBM + quad * 32 + lane) * TN + cc * 32;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8)
+                        ptx::st_global_v8(dst + j, v[j], v[j + 1], v[j + 2], v[j + 3], v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
+                    continue;
                 }
                 if (m >= p.M) continue;
                 const int64_t nb = tc.n0 + cc * 32;
@@ -424,11 +589,24 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     }
                 }
             }
+            if (p.streamk && tc.partial) {
+                // publish the slot: every epilogue thread fences its stores, then one thread counts the segment in
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (quad == 0 && lane == 0) atomicAdd(&p.sk_flags[tc.tile_id * 2 + (int)rank], 1u);
+            }
             if (quad == 0 && lane == 0) tr.end(10);
         }
     }
     ptx::tc_fence_before();
     __syncthreads();
+    if (p.streamk) {
+        if (threadIdx.x == 0) tr.begin();
+        // the activation ring is idle by now: its first bytes hold the slot list of the tile being summed
+        streamk_fixup<TN>(p, pair, npairs, (int)rank, abort_flag, reinterpret_cast<volatile int*>(tmem_slot + 2),
+                          reinterpret_cast<int*>(ring_a));
+        if (threadIdx.x == 0) tr.end(13);
+    }
     if (tl && threadIdx.x < 256) p.timeline[blockIdx.x * 256 + threadIdx.x] = tlog[threadIdx.x];
     ptx::cluster_sync();  // no CTA leaves while the peer may still signal its barriers or read its shared memory
     if (tr.out && threadIdx.x == 0) {
@@ -446,11 +624,15 @@ int env_int(const char* name, int dflt) {
     return v && *v ? atoi(v) : dflt;
 }
 
-template <bool RES, int TN, int FMT>
-int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream) {
+constexpr int kStreamKTN = 256;    // tile width of the K-streamed schedule (two accumulators fit in tensor memory)
+constexpr int kStreamKMaxPairs = 74;
+
+template <bool RES, int TN, int FMT, int NG>
+int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool streamk = false) {
+    constexpr int kExpGroups = NG;
     constexpr int kAStage = kATileBytes * (RES ? 2 : 1);
-    constexpr int bn = TN > kMaxBN ? kMaxBN : TN;
-    constexpr int nt = TN / bn;
+    constexpr int nt = TN > kMaxBN ? 2 : 1;
+    constexpr int bn = TN / nt;
     constexpr int half = bn / 2;
     constexpr int my_rows = nt * half;
     CUtensorMap ta, tr, tw;
@@ -475,6 +657,9 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream) {
     p.ntiles_n = (int)((g.N + TN - 1) / TN);
     p.num_tiles = p.ntiles_m * p.ntiles_n * splits;
     p.acc_bufs = TN * 2 <= kTmemCols ? 2 : 1;
+    p.streamk = streamk ? 1 : 0;
+    p.sk_slots = g.splitk_partials;
+    p.sk_flags = g.sk_flags;
     constexpr int exp_stage = my_rows * 128, raw_stage = my_rows * 32;
     const int fixed = 1024 + 1024;
     p.se = kExpGroups;  // one slot per expander group (a group never runs two phases ahead on a slot)
@@ -494,8 +679,9 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream) {
     {
         const char* tp = getenv("RESQ_GEMM_TIMELINE_PTR");
         p.timeline = tp && *tp ? reinterpret_cast<unsigned int*>(strtoull(tp, nullptr, 0)) : nullptr;
+        p.timeline_first = env_int("RESQ_GEMM_TIMELINE_FIRST", 96);
     }
-    auto kern = gemm_pair_kernel<RES, TN, FMT>;
+    auto kern = gemm_pair_kernel<RES, TN, FMT, NG>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -510,11 +696,27 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream) {
         if (num_sms <= 0) num_sms = 148;
     }
     const int max_pairs = num_sms / 2;
-    const int npairs = std::min(p.num_tiles, max_pairs);
+    int npairs = std::min(p.num_tiles, max_pairs);
+    if (streamk && (size_t)p.num_tiles * 2 * sizeof(unsigned int) > kWsFlags) {
+        set_last_error("internal: %d output tiles exceed the arrival counters of the K-streamed schedule", p.num_tiles);
+        return RESQ_ERR_CUDA;
+    }
+    if (streamk) {
+        // every pair gets at least two k-blocks; the pairs wait for one another at the end, so all of them
+        // must be resident at once
+        const int64_t units = (int64_t)p.num_tiles * G;
+        const int cap = std::min(max_pairs, kStreamKMaxPairs);
+        npairs = (int)std::min<int64_t>(cap, std::max<int64_t>(1, units / 2));
+        if (p.num_tiles <= cap) {
+            // few tiles: the same number of pairs for every tile, so that a pair works on one tile only
+            const int per_tile = std::max(1, std::min(cap / p.num_tiles, G / 2));
+            npairs = p.num_tiles * per_tile;
+        }
+    }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)(2 * npairs), 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.blockDim = dim3(pair_threads(NG), 1, 1);
     cfg.dynamicSmemBytes = (size_t)smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -525,24 +727,58 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e;
+    if (streamk) {
+        static int max_clusters = -1;  // co-resident clusters of this variant
+        if (max_clusters < 0) {
+            int n = 0;
+            e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaOccupancyMaxActiveClusters(gemm pair)");
+            max_clusters = n;
+        }
+        if (npairs > max_clusters) {
+            npairs = max_clusters;
+            cfg.gridDim = dim3((unsigned)(2 * npairs), 1, 1);
+        }
+        if (npairs < 1) {
+            set_last_error("gemm pair kernel: no cluster of two CTAs fits on this device");
+            return RESQ_ERR_CUDA;
+        }
+    }
     {
         LaunchScope scope(kKindGemm, stream);
         e = cudaLaunchKernelEx(&cfg, kern, ta, tr, tw, p);
     }
     if (e != cudaSuccess) return cuda_fail(e, "gemm_pair_kernel launch");
+    if (streamk) return RESQ_OK;
     return launch_splitk_reduce(g, splits, stream);
 }
 
 template <bool RES, int FMT>
 int dispatch_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
-    if (tn == 128) return launch_pair_variant<RES, 128, FMT>(g, splits, stream);
-    if (tn == 256) return launch_pair_variant<RES, 256, FMT>(g, splits, stream);
-    if (tn == 512) return launch_pair_variant<RES, 512, FMT>(g, splits, stream);
+    const int ng = env_int("RESQ_GEMM_GROUPS", 3);
+    if (tn == 128) return launch_pair_variant<RES, 128, FMT, 4>(g, splits, stream);
+    if (tn == 256 && ng == 3) return launch_pair_variant<RES, 256, FMT, 3>(g, splits, stream);
+    if (tn == 256) return launch_pair_variant<RES, 256, FMT, 4>(g, splits, stream);
+    if (tn == 512 && ng == 3) return launch_pair_variant<RES, 512, FMT, 3>(g, splits, stream);
+    if (tn == 512) return launch_pair_variant<RES, 512, FMT, 4>(g, splits, stream);
     set_last_error("internal: unsupported pair tile width %d", tn);
     return RESQ_ERR_CUDA;
 }
 
 }  // namespace
+
+size_t gemm_pair_streamk_scratch_bytes() {
+    return (size_t)2 * kStreamKMaxPairs * (2 * kBM) * kStreamKTN * sizeof(float);
+}
+
+int launch_gemm_pair_streamk(const GemmArgs& g, cudaStream_t stream) {
+    const bool res = g.r_bf16 != nullptr;
+    if (g.fmt == kMXFP4)
+        return res ? launch_pair_variant<true, kStreamKTN, kMXFP4, 3>(g, 1, stream, true)
+                   : launch_pair_variant<false, kStreamKTN, kMXFP4, 3>(g, 1, stream, true);
+    return res ? launch_pair_variant<true, kStreamKTN, kHiF4, 3>(g, 1, stream, true)
+               : launch_pair_variant<false, kStreamKTN, kHiF4, 3>(g, 1, stream, true);
+}
 
 int launch_gemm_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
     const bool res = g.r_bf16 != nullptr;
