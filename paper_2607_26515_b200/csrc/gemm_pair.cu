@@ -160,7 +160,7 @@ __device__ __forceinline__ float4 ld_cg_f4(const float* p) {
 // Called by all threads of the CTA; the CTA of rank r handles rows r * 128 .. r * 128 + 127 of the tile.
 template <int TN>
 __device__ __forceinline__ void streamk_fixup(const PairParams& p, int pair, int npairs, int rank, volatile int* abort_flag,
-                                              volatile int* s_ok, int* s_slots) {
+                                              volatile int* s_ok, int* s_slots, unsigned int* evt, long long t0) {
     const int G = (int)(p.K / kBK);
     const int64_t U = (int64_t)p.num_tiles * G;
     const int64_t u0 = sk_begin(U, npairs, pair), u1 = sk_begin(U, npairs, pair + 1);
@@ -189,6 +189,7 @@ __device__ __forceinline__ void streamk_fixup(const PairParams& p, int pair, int
         const bool ok = *s_ok != 0;
         __syncthreads();
         if (!ok) return;
+        if (evt && threadIdx.x == 0) evt[which] = (unsigned int)(clock64() - t0);
         // slot of every segment (k order), worked out once per tile
         if ((int)threadIdx.x < nseg) {
             const int q = pf + (int)threadIdx.x;
@@ -253,12 +254,16 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     uint8_t* ring_e = ring_a + (size_t)SA * kAStage;
     uint8_t* ring_r = ring_e + (size_t)SE * exp_stage;
     uint64_t* bars = reinterpret_cast<uint64_t*>(ring_r + (size_t)SR * raw_stage);
-    uint64_t* a_full = bars;                   // leader: both CTAs' activation stages landed
-    uint64_t* a_empty = bars + kMaxRing;       // each CTA: the MMAs that read the stage completed
+    // All three rings have one slot per expander group, and slot s of each holds k-block it = s (mod NG): one
+    // "full" barrier per slot collects the activation bytes of both CTAs and the arrivals of both CTAs' expander
+    // group, and one "empty" barrier per slot (a single commit) releases the activation stage and the expanded
+    // stage together.  The MMA thread thus does one wait and one commit per k-block.
+    uint64_t* a_full = bars;                   // leader: both CTAs' activation stages landed and expanded halves written
+    uint64_t* a_empty = bars + kMaxRing;       // each CTA: the MMAs that read the slot completed
     uint64_t* r_full = bars + 2 * kMaxRing;    // each CTA: own raw codes landed
     uint64_t* r_empty = bars + 3 * kMaxRing;   // each CTA: own expanders consumed them
-    uint64_t* e_full = bars + 4 * kMaxRing;    // leader: both CTAs' expanded halves written
-    uint64_t* e_empty = bars + 5 * kMaxRing;   // each CTA
+    uint64_t* e_full = a_full;                 // (same barriers: see above)
+    uint64_t* e_empty = a_empty;
     uint64_t* acc_full = bars + 6 * kMaxRing;  // [2] each CTA
     uint64_t* acc_empty = acc_full + 2;        // [2] leader: both epilogues drained
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
@@ -266,8 +271,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     unsigned int* tlog = reinterpret_cast<unsigned int*>(tmem_slot + 4);  // [8 roles][32 iterations] (512 B)
     const bool tl = p.timeline != nullptr && (blockIdx.x >> 1) == 0;
     const int kTl0 = p.timeline_first;  // first logged iteration
+#define EVT(k) do { if (tl) p.timeline[512 + (int)rank * 16 + (k)] = (unsigned int)(clock64() - t_kernel0); } while (0)
 #define TLOG(role, it) do { if (tl && (it) >= kTl0 && (it) < kTl0 + 32) tlog[(role) * 32 + ((it) - kTl0)] = (unsigned int)clock64(); } while (0)
 
+    const long long t_entry = clock64();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();  // 0 = leader
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
@@ -275,12 +282,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxRing; ++s) {
-            ptx::mbar_init(&a_full[s], 2);                 // one arrive.expect_tx per CTA
+            ptx::mbar_init(&a_full[s], 2 + 2 * kGroupWarps);  // an arrive.expect_tx and one expander group per CTA
             ptx::mbar_init(&a_empty[s], 1);
             ptx::mbar_init(&r_full[s], 1);
             ptx::mbar_init(&r_empty[s], kGroupWarps);
-            ptx::mbar_init(&e_full[s], 2 * kGroupWarps);   // one expander group of each CTA
-            ptx::mbar_init(&e_empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(&acc_full[b], 1);
@@ -297,6 +302,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     const uint32_t tmem_base = *tmem_slot;
     Trace tr{(p.debug & 16) ? reinterpret_cast<unsigned long long*>(p.status) + 8 : nullptr, 0};
     const long long t_kernel0 = clock64();
+    if (tl && threadIdx.x == 0) p.timeline[512 + (int)rank * 16] = (unsigned int)(t_kernel0 - t_entry);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ activation producer (both CTAs)
@@ -312,7 +318,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
                     const int s = it % SA;
                     tr.begin();
-                    const bool got = ptx::mbar_wait(&a_empty[s], ((it / SA) & 1) ^ 1, abort_flag);
+                    const bool got = ptx::mbar_wait_spin(&a_empty[s], ((it / SA) & 1) ^ 1, abort_flag);
                     tr.end(0);
                     if (!got) {
                         report_timeout(p.status, 1);
@@ -321,8 +327,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     }
                     uint8_t* st = ring_a + (size_t)s * kAStage;
                     TLOG(0, it);
+                    if (it == 0) EVT(1);
                     const uint32_t full = ptx::map_to_cta(&a_full[s], 0);
-                    ptx::mbar_arrive_expect_tx_cluster(full, (uint32_t)kAStage);
+                    ptx::mbar_arrive_expect_tx_cluster_relaxed(full, (uint32_t)kAStage);  // publishes nothing itself
                     const int kx = (tc.kb_begin + i) * kBK;
                     ptx::tma_load_2d_pair(st, &tmap_a, full, kx, my_m);
                     if (RES) ptx::tma_load_2d_pair(st + kATileBytes, &tmap_r, full, kx, my_m);
@@ -341,7 +348,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
                     const int s = it % SR;
                     tr.begin();
-                    const bool got = ptx::mbar_wait(&r_empty[s], ((it / SR) & 1) ^ 1, abort_flag);
+                    const bool got = ptx::mbar_wait_spin(&r_empty[s], ((it / SR) & 1) ^ 1, abort_flag);
                     tr.end(1);
                     if (!got) {
                         report_timeout(p.status, 5);
@@ -361,7 +368,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && rank == 0) {
             const uint32_t idesc = ptx::idesc_bf16_f32(2 * kBM, bn);
-            uint32_t it = 0;
+            const uint64_t desc0 = ptx::smem_desc_sw128_kmajor(0);  // everything but the start address
+            const uint32_t a_base16 = (ptx::smem_u32(ring_a) & 0x3FFFFu) >> 4, e_base16 = (ptx::smem_u32(ring_e) & 0x3FFFFu) >> 4;
+            uint32_t it = 0, sa = 0, pha = 0;  // ring slot and phase parity of this k-block
             int local_tile = 0;
             bool ok = true;
             SegIter<TN> si(p, pair, npairs);
@@ -372,7 +381,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 const int buf = p.acc_bufs == 2 ? (lt & 1) : 0;
                 const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(lt >> 1) : (uint32_t)lt;
                 tr.begin();
-                const bool got_acc = ptx::mbar_wait(&acc_empty[buf], (use & 1) ^ 1, abort_flag);
+                const bool got_acc = ptx::mbar_wait_spin(&acc_empty[buf], (use & 1) ^ 1, abort_flag);
                 tr.end(4);
                 if (!got_acc) {
                     report_timeout(p.status, 6);
@@ -381,42 +390,38 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 ptx::tc_fence_after();
                 const uint32_t d0 = tmem_base + (uint32_t)(buf * TN);
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
-                    const int sa = it % SA, se = it % SE;
+                    // This thread's instruction stream sits between the MMAs of consecutive k-blocks: stage
+                    // indices, phases and descriptors advance by additions only.
                     tr.begin();
-                    ok = ptx::mbar_wait(&a_full[sa], (it / SA) & 1, abort_flag);
+                    ok = ptx::mbar_wait_spin(&a_full[sa], pha, abort_flag);
                     tr.end(2);
-                    TLOG(7, it);
-                    tr.begin();
-                    ok = ok && ptx::mbar_wait(&e_full[se], (it / SE) & 1, abort_flag);
-                    tr.end(3);
                     if (!ok) {
                         report_timeout(p.status, 2);
                         break;
                     }
                     tr.begin();
                     TLOG(2, it);
+                    if (it == 0) EVT(2);
                     ptx::tc_fence_after();
-                    const uint32_t a_addr = ptx::smem_u32(ring_a + (size_t)sa * kAStage);
-                    const uint32_t b_addr = ptx::smem_u32(ring_e + (size_t)se * exp_stage);
+                    const uint64_t adesc = desc0 + (uint64_t)(a_base16 + sa * (uint32_t)(kAStage >> 4));
+                    const uint64_t bdesc = desc0 + (uint64_t)(e_base16 + sa * (uint32_t)(exp_stage >> 4));
 #pragma unroll
                     for (int k = 0; k < kBK / 16; ++k) {
 #pragma unroll
                         for (int j = 0; j < nt; ++j) {
-                            const uint64_t bdesc = ptx::smem_desc_sw128_kmajor(b_addr + j * half * 128 + k * 32);
+                            const uint64_t bd = bdesc + (uint64_t)((j * half * 128 + k * 32) >> 4);
                             const uint32_t d = d0 + (uint32_t)(j * bn);
-                            ptx::umma_bf16_pair(d, ptx::smem_desc_sw128_kmajor(a_addr + k * 32), bdesc, idesc,
-                                                (i > 0 || k > 0) ? 1u : 0u);
-                            if (RES)
-                                ptx::umma_bf16_pair(d, ptx::smem_desc_sw128_kmajor(a_addr + kATileBytes + k * 32), bdesc,
-                                                    idesc, 1u);
+                            ptx::umma_bf16_pair(d, adesc + (uint64_t)((k * 32) >> 4), bd, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                            if (RES) ptx::umma_bf16_pair(d, adesc + (uint64_t)((kATileBytes + k * 32) >> 4), bd, idesc, 1u);
                         }
                     }
-                    ptx::umma_commit_pair(&a_empty[sa], 3);  // frees the stages in both CTAs
-                    ptx::umma_commit_pair(&e_empty[se], 3);
+                    ptx::umma_commit_pair(&a_empty[sa], 3);  // frees the slot in both CTAs
+                    if (++sa == (uint32_t)SA) { sa = 0; pha ^= 1u; }
                     TLOG(3, it);
                     tr.end(5);
                 }
                 if (ok) ptx::umma_commit_pair(&acc_full[buf], 3);
+                EVT(3);
             }
         }
     } else if (warp >= kFirstExpWarp) {
@@ -506,7 +511,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(lt >> 1) : (uint32_t)lt;
             if (quad == 0 && lane == 0) tr.begin();
             const bool got_full = ptx::mbar_wait(&acc_full[buf], use & 1, abort_flag);
-            if (quad == 0 && lane == 0) { tr.end(9); tr.begin(); }
+            if (quad == 0 && lane == 0) { tr.end(9); tr.begin(); EVT(4); }
             if (!got_full) {
                 report_timeout(p.status, 4);
                 break;
@@ -595,7 +600,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (quad == 0 && lane == 0) atomicAdd(&p.sk_flags[tc.tile_id * 2 + (int)rank], 1u);
             }
-            if (quad == 0 && lane == 0) tr.end(10);
+            if (quad == 0 && lane == 0) { tr.end(10); EVT(5); }
         }
     }
     ptx::tc_fence_before();
@@ -604,8 +609,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         if (threadIdx.x == 0) tr.begin();
         // the activation ring is idle by now: its first bytes hold the slot list of the tile being summed
         streamk_fixup<TN>(p, pair, npairs, (int)rank, abort_flag, reinterpret_cast<volatile int*>(tmem_slot + 2),
-                          reinterpret_cast<int*>(ring_a));
-        if (threadIdx.x == 0) tr.end(13);
+                          reinterpret_cast<int*>(ring_a), tl ? p.timeline + 512 + (int)rank * 16 + 8 : nullptr, t_kernel0);
+        if (threadIdx.x == 0) { tr.end(13); EVT(7); }
     }
     if (tl && threadIdx.x < 256) p.timeline[blockIdx.x * 256 + threadIdx.x] = tlog[threadIdx.x];
     ptx::cluster_sync();  // no CTA leaves while the peer may still signal its barriers or read its shared memory
@@ -664,8 +669,8 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
     const int fixed = 1024 + 1024;
     p.se = kExpGroups;  // one slot per expander group (a group never runs two phases ahead on a slot)
     p.sr = kExpGroups;  // the groups read k-blocks i .. i+3 concurrently
-    p.sa = std::min(kMaxRing, (kSmemBudget - fixed - p.se * exp_stage - p.sr * raw_stage) / kAStage);
-    if (p.sa < 2 || p.se > kMaxRing || p.sr > kMaxRing) {
+    p.sa = kExpGroups;  // the activation ring shares its full / empty barriers with the expanded-weight ring
+    if (fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage > kSmemBudget) {
         set_last_error("internal: shared-memory rings do not fit (pair tile %d)", TN);
         return RESQ_ERR_CUDA;
     }
@@ -759,8 +764,7 @@ int dispatch_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
     if (tn == 128) return launch_pair_variant<RES, 128, FMT, 4>(g, splits, stream);
     if (tn == 256 && ng == 3) return launch_pair_variant<RES, 256, FMT, 3>(g, splits, stream);
     if (tn == 256) return launch_pair_variant<RES, 256, FMT, 4>(g, splits, stream);
-    if (tn == 512 && ng == 3) return launch_pair_variant<RES, 512, FMT, 3>(g, splits, stream);
-    if (tn == 512) return launch_pair_variant<RES, 512, FMT, 4>(g, splits, stream);
+    if (tn == 512) return launch_pair_variant<RES, 512, FMT, 3>(g, splits, stream);  // four slots would not fit
     set_last_error("internal: unsupported pair tile width %d", tn);
     return RESQ_ERR_CUDA;
 }

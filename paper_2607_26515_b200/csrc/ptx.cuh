@@ -75,6 +75,18 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return false;
 }
 
+// Bounded wait that never suspends the thread: for the single-thread roles (TMA producers, MMA issuer), whose
+// reaction time is on the critical path of the pipeline.  About 2^24 polls of ~25 cycles bound it to a fraction
+// of a second.
+__device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < (1u << 24); ++i) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((i & 1023u) == 1023u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
 // Warp-collective bounded wait: lane 0 polls, the outcome is broadcast.  Keeps the number of threads that
 // hammer the barrier (and the shared-memory pipe) at one per warp.  All 32 lanes must call it.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
@@ -193,6 +205,13 @@ __device__ __forceinline__ uint32_t map_to_cta(const void* p, uint32_t rank) {
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Remote arrive without cluster-scope release: for arrivals that publish no data of the issuing thread (an
+// expect_tx ahead of TMA loads, whose bytes are published by the complete_tx mechanism itself).  The release
+// form at cluster scope stalls the issuing thread for several hundred cycles.
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster_relaxed(uint32_t cluster_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes)
+                 : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes)
