@@ -5,6 +5,7 @@
 #include <atomic>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -37,6 +38,15 @@ struct ProfRec {
 std::mutex g_prof_mu;
 std::vector<ProfRec*> g_prof;
 }  // namespace
+
+bool pdl_enabled() {
+    static const int on = [] {
+        const char* v = getenv("RESQ_PDL");
+        return (v && *v) ? atoi(v) : 1;
+    }();
+    // event records between the kernels (profiling) would serialize them anyway
+    return on != 0 && !g_profile.load(std::memory_order_relaxed);
+}
 
 LaunchScope::LaunchScope(int kind, cudaStream_t stream) : kind_(kind), stream_(stream), rec_(nullptr) {
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -211,8 +221,6 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     rc = check_workspace(workspace, ws_bytes, linear_workspace_bytes(fmt, M, N, K, pattern));
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemsetAsync(workspace, 0, kWsHeader + kWsFlags, st);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(status)");
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     QuantArgs a;
     memset(&a, 0, sizeof(a));
@@ -224,6 +232,8 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     size_t used = 0;
     carve_quant_scratch(ws + kWsFlags, M, K, pattern, a, used);
     a.status = reinterpret_cast<DeviceStatus*>(ws);
+    a.clear_words = reinterpret_cast<uint32_t*>(ws);  // cleared by the quantizer kernel: no separate memset node
+    a.n_clear_words = (int)((kWsHeader + kWsFlags) / 4);
     used += kWsFlags;
     a.a_bf16 = reinterpret_cast<__nv_bfloat16*>(ws + used);
     used += align_up((size_t)M * (size_t)K * 2, 256);

@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <string.h>
 #include "../../include/resq.h"
 
 namespace resq {
@@ -43,6 +44,33 @@ struct LaunchScope {
     void* rec_;
 };
 
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// The kernels of one linear-layer call (and of consecutive calls on a stream) are launched with programmatic
+// stream serialization: a kernel may be scheduled, and run its set-up, while its predecessor drains.  Every
+// kernel launched this way executes pdl_wait() before it first touches global memory that an earlier kernel may
+// have written (or may still read), and pdl_trigger() as early as it likes.
+bool pdl_enabled();  // api.cu: environment switch RESQ_PDL (default on)
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 Args... args) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+#endif
+
 // ---- quantizer launch description (quantize.cu) ------------------------------------------------
 struct QuantArgs {
     const __nv_bfloat16* X;
@@ -61,6 +89,9 @@ struct QuantArgs {
     double* scores;         // CHAN50: [K]; BLOCK: [(M/32) * (K/64)]
     uint8_t* keep_flags;    // CHAN50: [K]; BLOCK: [(M/32) * (K/64)]
     DeviceStatus* status;
+    // words at the start of the workspace (status, counters of the GEMM) that the first kernel of the call clears
+    uint32_t* clear_words;
+    int n_clear_words;
 };
 
 int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream);

@@ -149,6 +149,9 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     const uint32_t tmem_base = *tmem_slot;
     Trace tr{(p.debug & 16) ? reinterpret_cast<unsigned long long*>(p.status) + 8 : nullptr, 0};
     const long long t_kernel0 = clock64();
+    // programmatic dependent launch: see gemm_pair.cu (the weight side does not depend on the quantizer)
+    pdl_trigger();
+    if (!(warp == 2 || warp >= kFirstExpWarp)) pdl_wait();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ activation producer
@@ -428,6 +431,8 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 // (128-bit loads) when N is a multiple of 4.
 __global__ void splitk_reduce_kernel(const float* __restrict__ partials, int splits, int64_t M, int64_t N, void* Y,
                                      int out_f32, int64_t ldy) {
+    pdl_wait();     // the partial tiles come from the GEMM kernel just before
+    pdl_trigger();
     const int64_t total = M * N;
     if ((N & 3) == 0) {
         const int64_t idx = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
@@ -505,9 +510,9 @@ int launch_splitk_reduce(const GemmArgs& g, int splits, cudaStream_t stream) {
     if (splits <= 1) return RESQ_OK;
     const int64_t n = (g.N & 3) == 0 ? g.M * g.N / 4 : g.M * g.N;
     LaunchScope scope(kKindReduce, stream);
-    splitk_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(g.splitk_partials, splits, g.M, g.N, g.Y,
-                                                                         g.out_dtype == RESQ_OUT_F32, g.ldy);
-    return cuda_fail(cudaGetLastError(), "splitk_reduce_kernel launch");
+    return cuda_fail(launch_kernel(splitk_reduce_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, stream,
+                                   (const float*)g.splitk_partials, splits, g.M, g.N, g.Y, (int)(g.out_dtype == RESQ_OUT_F32), g.ldy),
+                     "splitk_reduce_kernel launch");
 }
 
 int launch_gemm_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream);
@@ -677,9 +682,9 @@ int launch_variant(const GemmArgs& g, const TileChoice& tc, cudaStream_t stream)
     const unsigned grid = (unsigned)std::min(p.num_tiles, num_sms);
     {
         LaunchScope scope(kKindGemm, stream);
-        kern<<<grid, kGemmThreads, smem_bytes, stream>>>(ta, tr, tw, p);
+        rc = cuda_fail(launch_kernel(kern, dim3(grid), dim3(kGemmThreads), (size_t)smem_bytes, stream, ta, tr, tw, p),
+                       "gemm_hif4_kernel launch");
     }
-    rc = cuda_fail(cudaGetLastError(), "gemm_hif4_kernel launch");
     if (rc) return rc;
     return launch_splitk_reduce(g, tc.splits, stream);
 }

@@ -303,6 +303,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     Trace tr{(p.debug & 16) ? reinterpret_cast<unsigned long long*>(p.status) + 8 : nullptr, 0};
     const long long t_kernel0 = clock64();
     if (tl && threadIdx.x == 0) p.timeline[512 + (int)rank * 16] = (unsigned int)(t_kernel0 - t_entry);
+    // Programmatic dependent launch: the set-up above overlaps the tail of the quantizer kernel.  The weight side
+    // (raw-code producer, expanders) reads only the packed weights, which no kernel since the start of the
+    // quantizer writes, and starts at once; everything else waits for the quantizer's outputs.
+    pdl_trigger();
+    if (!(warp == 2 || warp >= kFirstExpWarp)) pdl_wait();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ activation producer (both CTAs)
@@ -724,13 +729,15 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
     cfg.blockDim = dim3(pair_threads(NG), 1, 1);
     cfg.dynamicSmemBytes = (size_t)smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
     cudaError_t e;
     if (streamk) {
         static int max_clusters = -1;  // co-resident clusters of this variant

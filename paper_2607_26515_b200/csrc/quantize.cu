@@ -93,6 +93,10 @@ __device__ __forceinline__ void keep_words(uint32_t keep, uint32_t (&km)[4]) {
 // IMG: the bf16 images for the GEMM are written (a_bf16, and r_bf16 when RESIDUAL).
 template <int FMT, bool RESIDUAL, bool IMG>
 __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int rows_per_cta) {
+    pdl_wait();     // nothing below may touch global memory before the previous kernel of the stream is done
+    pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
+    if (a.clear_words && blockIdx.x == 0 && blockIdx.y == 0)
+        for (int i = threadIdx.x; i < a.n_clear_words; i += blockDim.x) a.clear_words[i] = 0u;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t k0 = ((int64_t)blockIdx.y * kWarpsPerCta + warp) * kColsPerWarp + lane * 8;
     const bool active = k0 < a.K;  // whole blocks are active or not (K is a multiple of the block size)
@@ -357,6 +361,10 @@ __device__ __forceinline__ void hif4_encode_block(const uint32_t (&w)[32], uint3
 
 template <bool RESIDUAL, bool IMG>
 __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, int rows_per_warp) {
+    pdl_wait();     // nothing below may touch global memory before the previous kernel of the stream is done
+    pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
+    if (a.clear_words && blockIdx.x == 0 && blockIdx.y == 0)
+        for (int i = threadIdx.x; i < a.n_clear_words; i += blockDim.x) a.clear_words[i] = 0u;
     extern __shared__ __align__(16) uint8_t smem_q[];
     constexpr int kBufs = IMG ? 3 : 2;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -625,6 +633,10 @@ __global__ void apply_global_mask_kernel(int pattern, int64_t M, int64_t K, cons
 // shared memory, a 2-pass radix select finds the threshold, an index-ordered pass resolves ties.
 template <int FMT>
 __global__ void __launch_bounds__(kThreads) quant_row50_kernel(QuantArgs a) {
+    pdl_wait();     // nothing below may touch global memory before the previous kernel of the stream is done
+    pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
+    if (a.clear_words && blockIdx.x == 0 && blockIdx.y == 0)
+        for (int i = threadIdx.x; i < a.n_clear_words; i += blockDim.x) a.clear_words[i] = 0u;
     extern __shared__ __align__(16) uint16_t s_r[];  // [K] signed bf16 image of deq Q(dX)
     __shared__ unsigned hist[256];
     __shared__ unsigned s_prefix;
@@ -815,8 +827,7 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(row50)");
         LaunchScope scope(kKindQuant, stream);
-        kern<<<(unsigned)a.M, kThreads, smem, stream>>>(a);
-        return cuda_fail(cudaGetLastError(), "quant_row50_kernel launch");
+        return cuda_fail(launch_kernel(kern, dim3((unsigned)a.M), dim3(kThreads), smem, stream, a), "quant_row50_kernel launch");
     }
     const bool global_sel = pattern == RESQ_S_CHAN50 || pattern == RESQ_S_BLOCK32x64_50;
     int64_t nscore = 0;
@@ -843,8 +854,8 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
             cudaError_t attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
             if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute(quant_block_kernel)");
             LaunchScope scope(kKindQuant, stream);
-            kern<<<ctas, kThreads, smem, stream>>>(a, rows_per_warp);
-            return cuda_fail(cudaGetLastError(), "quant_block_kernel launch");
+            return cuda_fail(launch_kernel(kern, dim3(ctas), dim3(kThreads), (size_t)smem, stream, a, rows_per_warp),
+                             "quant_block_kernel launch");
         };
         int rc = residual ? (img ? launch(quant_block_kernel<true, true>) : launch(quant_block_kernel<true, false>))
                           : (img ? launch(quant_block_kernel<false, true>) : launch(quant_block_kernel<false, false>));
@@ -867,10 +878,11 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     const int rows_per_cta = pick_rows_per_cta(a.M, a.K, pattern);
     dim3 grid((unsigned)((a.M + rows_per_cta - 1) / rows_per_cta),
               (unsigned)((a.K + (int64_t)kWarpsPerCta * kColsPerWarp - 1) / ((int64_t)kWarpsPerCta * kColsPerWarp)));
+    cudaError_t launch_err = cudaSuccess;
     {
     LaunchScope scope(kKindQuant, stream);
     const bool img = a.a_bf16 != nullptr;  // the GEMM path asks for both images (r_bf16 whenever there is a residual)
-    auto launch = [&](auto kern) { kern<<<grid, kThreads, 0, stream>>>(a, rows_per_cta); };
+    auto launch = [&](void (*kern)(QuantArgs, int)) { launch_err = launch_kernel(kern, grid, dim3(kThreads), 0, stream, a, rows_per_cta); };
     if (fmt == kHiF4) {
         if (residual) img ? launch(quant_stream_kernel<kHiF4, true, true>) : launch(quant_stream_kernel<kHiF4, true, false>);
         else img ? launch(quant_stream_kernel<kHiF4, false, true>) : launch(quant_stream_kernel<kHiF4, false, false>);
@@ -879,7 +891,7 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
         else img ? launch(quant_stream_kernel<kMXFP4, false, true>) : launch(quant_stream_kernel<kMXFP4, false, false>);
     }
     }
-    int rc = cuda_fail(cudaGetLastError(), "quant_stream_kernel launch");
+    int rc = cuda_fail(launch_err, "quant_stream_kernel launch");
     if (rc) return rc;
     if (global_sel) {
         { LaunchScope scope(kKindSelect, stream);
