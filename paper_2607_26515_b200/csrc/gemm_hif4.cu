@@ -569,25 +569,22 @@ TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res) {
         }
     }
     // CTA pairs (256 x tn tiles, 74 pairs) for everything taller than one MMA.  Cycle model fitted to in-kernel
-    // timelines: a k-block costs the tensor time of the tile or, when the activation ring is shallow, the ring's
-    // round trip (stage freed -> TMA issued -> data landed -> MMA woken, ~6500 cycles when every pair pulls the
-    // same activation tiles) divided by its depth; a tile costs ~8000 cycles of fill and epilogue; a K split
-    // costs a second launch plus the partial-tile traffic.
+    // timelines: a k-block costs the tensor time of the tile, but not less than the ~1500 cycles the slot hand-off
+    // (commit -> producers -> data landed -> MMA thread) takes, plus ~350 cycles of MMA-thread work between
+    // k-blocks; a tile costs ~8000 cycles of fill and epilogue; a K split costs a second launch plus the
+    // partial-tile traffic.
     if (M > kBM && env_int("RESQ_GEMM_PAIR", 1)) {
         const int64_t mtiles = (M + 2 * kBM - 1) / (2 * kBM);
         double best_pair = 1e300;
-        for (int tn : {512, 256, 128}) {
+        for (int tn : {512, 384, 320, 256, 128}) {
             const int64_t ntiles = (N + tn - 1) / tn;
-            const int groups = tn == 128 ? 4 : 3;                                    // as dispatched in gemm_pair.cu
-            const int ring = groups * (tn / 2) * 160;                                // expanded + raw stages
-            const int sa = std::min(8, (kSmemBudget - 2048 - ring) / (res ? 32768 : 16384));
             for (int splits = 1; splits <= 8; splits *= 2) {
                 if (G / splits < 4 && splits > 1) break;
                 const int64_t tiles = mtiles * ntiles * splits;
                 const int64_t rounds = (tiles + sms / 2 - 1) / (sms / 2);
                 const int kb = (G + splits - 1) / splits;
                 const double mma = tn / 256.0 * (res ? 1024.0 : 512.0);
-                const double per_kb = std::max(mma, 6500.0 / sa) + 300.0;
+                const double per_kb = std::max(mma, 1500.0) + 350.0;
                 double cost = rounds * (kb * per_kb + 8000.0);
                 if (splits > 1) cost += 15000.0 + (double)splits * M * N * 4.0 / 1200.0;  // partial tiles: ~1.6 KB/clk
                 if (cost < best_pair) {

@@ -771,6 +771,8 @@ int dispatch_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
     if (tn == 128) return launch_pair_variant<RES, 128, FMT, 4>(g, splits, stream);
     if (tn == 256 && ng == 3) return launch_pair_variant<RES, 256, FMT, 3>(g, splits, stream);
     if (tn == 256) return launch_pair_variant<RES, 256, FMT, 4>(g, splits, stream);
+    if (tn == 320) return launch_pair_variant<RES, 320, FMT, 3>(g, splits, stream);
+    if (tn == 384) return launch_pair_variant<RES, 384, FMT, 3>(g, splits, stream);
     if (tn == 512) return launch_pair_variant<RES, 512, FMT, 3>(g, splits, stream);  // four slots would not fit
     set_last_error("internal: unsupported pair tile width %d", tn);
     return RESQ_ERR_CUDA;

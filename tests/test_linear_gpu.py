@@ -120,6 +120,10 @@ def test_linear_zero_input_gives_zero():
 TILE_CONFIGS = [
     {"RESQ_GEMM_PAIR_TN": "512", "RESQ_GEMM_SPLITS": "1"},
     {"RESQ_GEMM_PAIR_TN": "512", "RESQ_GEMM_SPLITS": "2"},
+    {"RESQ_GEMM_PAIR_TN": "384", "RESQ_GEMM_SPLITS": "1"},
+    {"RESQ_GEMM_PAIR_TN": "320", "RESQ_GEMM_SPLITS": "2"},
+    {"RESQ_GEMM_STREAMK": "1"},
+    {"RESQ_GEMM_STREAMK": "0"},
     {"RESQ_GEMM_PAIR_TN": "256", "RESQ_GEMM_SPLITS": "1"},
     {"RESQ_GEMM_PAIR_TN": "256", "RESQ_GEMM_SPLITS": "4"},
     {"RESQ_GEMM_PAIR_TN": "128", "RESQ_GEMM_SPLITS": "1"},
@@ -160,6 +164,24 @@ def test_every_tile_configuration(tile_case, cfg, pattern, fmt, monkeypatch):
     assert m.check(work) == 0, m.last_error()
     w = want[(pattern, fmt)]
     check_close(y.cpu().numpy(), w["y"], w["abs_sum"])
+
+
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_k_streamed_schedule_with_uneven_segments(monkeypatch, out_dtype):
+    """More output tiles than CTA pairs: the (tile, k-block) units are dealt out evenly, so pairs start and end in
+    the middle of a tile's K range and most tiles are summed from two or three partial segments."""
+    monkeypatch.setenv("RESQ_GEMM_STREAMK", "1")
+    m = rq()
+    M, K, N = 300, 320, 20000 - 24     # 2 x 79 tiles of 256 x 256, 5 k-blocks each; ragged in M and N
+    xb, wb = synth_xw(91, M, K, N, n_out=3)
+    want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), oracle.S_2_4)
+    wc, ws = m.pack_weight(to_dev(wb))
+    work = m.alloc_workspace(m.resq_workspace_bytes(M, N, K, oracle.S_2_4))
+    ys = [m.resq_linear(to_dev(xb), wc, ws, oracle.S_2_4, out_dtype=out_dtype, workspace=work) for _ in range(2)]
+    assert m.check(work) == 0, m.last_error()
+    assert torch.equal(ys[0], ys[1])   # fixed summation order: identical bits on every run
+    y = ys[0].float().cpu().numpy().astype(np.float64)
+    check_close(y, want["y"], want["abs_sum"], bf16_out=out_dtype == torch.bfloat16)
 
 
 # ----------------------------------------------------------------------------------------------
