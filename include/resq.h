@@ -149,6 +149,20 @@ RESQ_API int mxfp4_resq_linear(const void* X_bf16, int64_t M, int64_t K, int64_t
                       int pattern, void* Y, int out_dtype, int64_t ldy,
                       void* workspace, size_t ws_bytes, void* stream);
 
+/* Weight-only ablation of Table 1 ("W4A16"): Y = X deq(Q(W))^T, the bf16 activations are used as they are
+ * (no activation quantizer, no residual term); weights as produced by *_pack_weight.  Same argument rules,
+ * output types and error behaviour as *_resq_linear; workspace of resq_w4a16_workspace_bytes(M, N, K) bytes
+ * (status word, arrival counters, fp32 partial tiles of a K split), owned by the caller. */
+RESQ_API size_t resq_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K);
+RESQ_API int hif4_w4a16_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
+                      const void* w_codes, const void* w_meta, int64_t N,
+                      void* Y, int out_dtype, int64_t ldy,
+                      void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_w4a16_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
+                       const void* w_codes, const void* w_scale, int64_t N,
+                       void* Y, int out_dtype, int64_t ldy,
+                       void* workspace, size_t ws_bytes, void* stream);
+
 /* ---- status --------------------------------------------------------------------------------------
  * resq_check synchronizes `stream` and returns the device status word kept at the start of
  * `workspace` (RESQ_OK, or RESQ_ERR_TIMEOUT if a bounded wait expired in the last call that used it). */

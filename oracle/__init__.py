@@ -226,3 +226,12 @@ def resq_linear(x_f32: np.ndarray, w_f32: np.ndarray, pattern: int, fmt: str = "
     y, ab = matmul(out["a"], out.get("r_masked"), w, want_abs)
     out.update({"w_codes": w_codes, "w_side": w_side, "w": w, "y": y, "abs_sum": ab})
     return out
+
+
+def w4a16_linear(x_f32: np.ndarray, w_f32: np.ndarray, fmt: str = "hif4", want_abs: bool = True) -> Dict[str, np.ndarray]:
+    """Weight-only ablation (Table 1, W4A16): Y = X deq(Q(W))^T, activations as given (bf16 values)."""
+    w_codes, w_side = encode(fmt, _f32(w_f32))
+    w = decode(fmt, w_codes, w_side)
+    y, ab = matmul(np.asarray(x_f32, dtype=np.float64), None, w, want_abs)
+    return {"w_codes": w_codes, "w_side": w_side, "w": w, "y": y, "abs_sum": ab}
+

@@ -264,6 +264,62 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     return launch_gemm_hif4(g, st);
 }
 
+// Weight-only variant (Table 1, "W4A16"): Y = X deq(Q(W))^T with the bf16 activations used as they are.
+// Workspace: [header | counters | fp32 partial tiles].
+size_t w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    return kWsHeader + kWsFlags + align_up(gemm_hif4_scratch_bytes(M, N, K), 256);
+}
+
+int w4a16_linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_side, int64_t N,
+                 void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    int rc = check_matrix(X, M, K, ldx, fmt, "X");
+    if (rc) return rc;
+    if (!w_codes || !w_side || !Y) {
+        set_last_error("w4a16_linear: NULL weight or output pointer");
+        return RESQ_ERR_NULL;
+    }
+    if (N <= 0) {
+        set_last_error("w4a16_linear: N=%lld", (long long)N);
+        return RESQ_ERR_SHAPE;
+    }
+    if (out_dtype != RESQ_OUT_BF16 && out_dtype != RESQ_OUT_F32) {
+        set_last_error("unknown output type %d", out_dtype);
+        return RESQ_ERR_PATTERN;
+    }
+    if (!aligned16(Y) || !aligned16(w_codes) || !aligned16(w_side) || ldy < N ||
+        ldy % (out_dtype == RESQ_OUT_BF16 ? 8 : 4) != 0) {
+        set_last_error("w4a16_linear: Y / weights need 16-byte aligned bases, ldy >= N and 16-byte aligned rows");
+        return RESQ_ERR_ALIGN;
+    }
+    rc = check_workspace(workspace, ws_bytes, w4a16_workspace_bytes(M, N, K));
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kWsHeader + kWsFlags, st);  // no quantizer kernel to clear it
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(status)");
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.fmt = fmt;
+    g.a_bf16 = static_cast<const __nv_bfloat16*>(X);
+    g.r_bf16 = nullptr;
+    g.lda = ldx;
+    g.w_codes = static_cast<const uint8_t*>(w_codes);
+    g.w_side = w_side;
+    g.M = M;
+    g.N = N;
+    g.K = K;
+    g.Y = Y;
+    g.out_dtype = out_dtype;
+    g.ldy = ldy;
+    g.partial_bytes = gemm_hif4_scratch_bytes(M, N, K);
+    g.splitk_partials = g.partial_bytes ? reinterpret_cast<float*>(ws + kWsHeader + kWsFlags) : nullptr;
+    g.splits = (int)(g.partial_bytes / ((size_t)M * (size_t)N * 4));
+    g.sk_flags = reinterpret_cast<unsigned int*>(ws + kWsHeader);
+    g.status = reinterpret_cast<DeviceStatus*>(ws);
+    return launch_gemm_hif4(g, st);
+}
+
 }  // namespace
 }  // namespace resq
 
@@ -316,6 +372,16 @@ int mxfp4_residual_mask(const void* X, int64_t M, int64_t K, int64_t ldx, int pa
                         void* r_codes, void* r_scale, void* mask_bits, void* workspace, size_t ws_bytes, void* stream) {
     return residual_mask(kMXFP4, X, M, K, ldx, pattern, x_codes, x_scale, r_codes, r_scale, mask_bits, workspace,
                          ws_bytes, stream);
+}
+
+size_t resq_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) { return w4a16_workspace_bytes(M, N, K); }
+int hif4_w4a16_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_meta, int64_t N,
+                      void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    return w4a16_linear(kHiF4, X, M, K, ldx, w_codes, w_meta, N, Y, out_dtype, ldy, workspace, ws_bytes, stream);
+}
+int mxfp4_w4a16_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_scale, int64_t N,
+                       void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    return w4a16_linear(kMXFP4, X, M, K, ldx, w_codes, w_scale, N, Y, out_dtype, ldy, workspace, ws_bytes, stream);
 }
 
 int hif4_resq_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_meta, int64_t N,

@@ -107,6 +107,7 @@ struct GemmArgs {
     const uint8_t* w_codes;        // [N, K/2]
     const void* w_side;            // [N, K/64] u32 or [N, K/32] u8
     int64_t M, N, K;
+    int64_t lda;                   // row pitch of a_bf16 / r_bf16 in elements (0: K, the workspace images)
     void* Y;
     int out_dtype;
     int64_t ldy;

@@ -609,11 +609,11 @@ template <int MT, bool RES, int TN, int FMT>
 int launch_variant(const GemmArgs& g, const TileChoice& tc, cudaStream_t stream) {
     constexpr int kAStage = MT * kATileBytes * (RES ? 2 : 1);
     CUtensorMap ta, tr, tw;
-    int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.a_bf16, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.K * 2,
+    int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.a_bf16, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)(g.lda ? g.lda : g.K) * 2,
                           kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
     rc = make_tmap_2d(&tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, RES ? g.r_bf16 : g.a_bf16, (uint64_t)g.K, (uint64_t)g.M,
-                      (uint64_t)g.K * 2, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+                      (uint64_t)(g.lda ? g.lda : g.K) * 2, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
     rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.w_codes, (uint64_t)g.K / 2, (uint64_t)g.N, (uint64_t)g.K / 2,
                       kBK / 2, (uint32_t)tc.bn, CU_TENSOR_MAP_SWIZZLE_NONE);

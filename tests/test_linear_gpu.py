@@ -113,6 +113,25 @@ def test_linear_zero_input_gives_zero():
         assert not y.any()
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("shape", [(64, 256, 200), (300, 1152, 1336), (256, 2048, 2560)])
+def test_w4a16_linear_parity(fmt, shape):
+    """Weight-only variant: bf16 activations straight into the GEMM, strided input included."""
+    m = rq()
+    M, K, N = shape
+    xb, wb = synth_xw(5 * M + N, M, K, N, n_out=max(1, K // 256))
+    want = oracle.w4a16_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), fmt)
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    big = torch.zeros((M, K + 64), dtype=torch.bfloat16, device="cuda")
+    big[:, :K] = to_dev(xb)
+    for x in (to_dev(xb), big[:, :K]):
+        y = m.w4a16_linear(x, wc, ws, fmt, out_dtype=torch.float32)
+        torch.cuda.synchronize()
+        check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+    yb = m.w4a16_linear(to_dev(xb), wc, ws, fmt, out_dtype=torch.bfloat16)
+    check_close(yb.float().cpu().numpy(), want["y"], want["abs_sum"], bf16_out=True)
+
+
 # ----------------------------------------------------------------------------------------------
 # Every tile configuration of the GEMM on one shape that spans several tiles and ragged edges.
 # RESQ_GEMM_* are the library's debugging overrides of its tile heuristic (read at every call).

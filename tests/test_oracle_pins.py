@@ -541,6 +541,29 @@ def test_dense_is_eq4_and_none_is_eq1():
     assert ed < e24 < e0
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+def test_w4a16_exact_rational_tiny_and_limit_of_the_residual_series(fmt):
+    """Weight-only ablation (Table 1): exact rational check of the product on a tiny case; and it is what the
+    two-term product approaches: for activations that are already decoded codes (zero residual) the W4A4 path
+    and the W4A16 path coincide, otherwise W4A16 is the target that the residual term moves Y toward."""
+    M, K, N = 3, 128, 4
+    x = gaussian_with_outliers(81, M, K, n_out=2, scale=16.0)
+    rng = np.random.default_rng(82)
+    w = bf16_round(rng.standard_normal((N, K)).astype(np.float32) * 0.02)
+    o = oracle.w4a16_linear(x, w, fmt)
+    xv, wv = _to_frac(x.astype(np.float64)), _to_frac(o["w"])
+    for m in range(M):
+        for n in range(N):
+            assert F(float(o["y"][m, n])) == sum(xv[m][k] * wv[n][k] for k in range(K))
+    full = oracle.resq_linear(x, w, oracle.S_DENSE, fmt)
+    none = oracle.resq_linear(x, w, oracle.S_NONE, fmt)
+    assert np.linalg.norm(full["y"] - o["y"]) < np.linalg.norm(none["y"] - o["y"])
+    xq = oracle.decode(fmt, *oracle.encode(fmt, x)).astype(np.float32)
+    if np.array_equal(oracle.decode(fmt, *oracle.encode(fmt, xq)), xq.astype(np.float64)):
+        same = oracle.resq_linear(xq, w, oracle.S_2_4, fmt)
+        np.testing.assert_allclose(same["y"], oracle.w4a16_linear(xq, w, fmt)["y"], rtol=1e-13, atol=1e-13)
+
+
 # ----------------------------------------------------------------- regression digest of a seeded tensor
 
 def test_seeded_digest():
