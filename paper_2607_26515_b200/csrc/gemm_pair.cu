@@ -7,9 +7,12 @@
 // SM, which is what bounds that kernel.  No TMA multicast is used: every TMA load targets the issuing
 // CTA's own shared memory; only mbarrier arrivals and tcgen05.commit cross the pair.
 //
-// Roles per CTA (24 warps): warp 0 activation TMA, warp 1 MMA issue (leader CTA only) + TMEM alloc,
-// warp 2 raw weight-code TMA, warps 4..7 epilogue, warps 8..23 expanders.  The leader's "full" barriers
-// collect arrivals from both CTAs; "empty" barriers are released in both CTAs by a commit multicast.
+// Roles per CTA (8 + 4 * NG warps): warp 0 activation TMA, warp 1 MMA issue (leader CTA only) + TMEM alloc,
+// warp 2 raw weight-code TMA, warps 4..7 epilogue, warps 8.. expanders in NG groups of four.  The leader's
+// "full" barriers collect arrivals from both CTAs; "empty" barriers are released in both CTAs by a commit
+// multicast.  Two schedules: whole tiles per pair (optionally with a K split and a separate reduce kernel), or
+// K-streamed (the k-blocks of few tiles dealt out evenly; partial tiles go to fp32 slots and are summed in a
+// fixed order at the end of the same kernel).
 #include "common.cuh"
 #include "ptx.cuh"
 #include "expand.cuh"
@@ -27,11 +30,10 @@ constexpr int kBM = 128;
 constexpr int kBK = 64;
 constexpr int kMaxBN = 256;
 constexpr int kGroupWarps = 4;                       // expander warps per group
-// Expander groups take k-blocks round-robin; each group owns one slot of the expanded-weight ring and of the
-// raw-code ring (SE == SR == groups).  The number of groups NG (four warps each) is a template parameter of the
-// kernel: more groups tolerate more hand-off latency on the weight side, fewer groups leave more shared memory
-// to the activation ring, whose round trip (stage freed -> TMA issued -> data landed -> MMAs issued) otherwise
-// bounds the k-block rate.
+// Expander groups take k-blocks round-robin; group g owns slot g of all three rings (activation stages, raw
+// codes, expanded weights: SA == SE == SR == NG).  The number of groups NG (four warps each) is a template
+// parameter of the kernel: more groups tolerate more hand-off latency, fewer groups fit wider tiles into
+// shared memory (three slots of a 512-wide tile with a residual operand take 216 KB).
 constexpr int kFirstEpiWarp = 4;
 constexpr int kFirstExpWarp = 8;
 constexpr int pair_threads(int groups) { return 32 * (kFirstExpWarp + kGroupWarps * groups); }
@@ -431,7 +433,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         }
     } else if (warp >= kFirstExpWarp) {
         // ------------------------------------------------------------------ expanders (both CTAs, own half)
-        // Two groups of 8 warps take alternate k-blocks, so each group has two MMA periods for one block:
+        // NG groups of four warps take k-blocks round-robin, so each group has NG MMA periods for one block:
         // the per-block synchronisation latency (two waits, two arrives, one proxy fence) stays off the
         // critical path.
         const int ew = (warp - kFirstExpWarp) % kGroupWarps;
