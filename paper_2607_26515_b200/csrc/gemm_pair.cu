@@ -721,7 +721,9 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
         npairs = (int)std::min<int64_t>(cap, std::max<int64_t>(1, units / 2));
         if (p.num_tiles <= cap) {
             // few tiles: the same number of pairs for every tile, so that a pair works on one tile only
-            const int per_tile = std::max(1, std::min(cap / p.num_tiles, G / 2));
+            int per_tile = std::max(1, std::min(cap / p.num_tiles, G / 2));
+            const int forced = env_int("RESQ_GEMM_SK_PAIRS", 0);  // debugging override: pairs per tile
+            if (forced > 0) per_tile = std::max(1, std::min(forced, per_tile));
             npairs = p.num_tiles * per_tile;
         }
     }
