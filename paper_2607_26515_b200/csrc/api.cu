@@ -235,14 +235,50 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     a.clear_words = reinterpret_cast<uint32_t*>(ws);  // cleared by the quantizer kernel: no separate memset node
     a.n_clear_words = (int)((kWsHeader + kWsFlags) / 4);
     used += kWsFlags;
-    a.a_bf16 = reinterpret_cast<__nv_bfloat16*>(ws + used);
+    // MXFP4 with a row-local selection: the GEMM runs on the block-scaled FP4 pipe and takes packed codes and
+    // scales (they fit into the space of the bf16 images); every other case takes exact bf16 images.
+    const bool native = fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K) &&
+                        (pattern == RESQ_S_NONE || pattern == RESQ_S_DENSE || pattern == RESQ_S_2_4);
+    uint8_t* region_a = ws + used;
     used += align_up((size_t)M * (size_t)K * 2, 256);
+    uint8_t* region_r = nullptr;
     if (pattern != RESQ_S_NONE) {
-        a.r_bf16 = reinterpret_cast<__nv_bfloat16*>(ws + used);
+        region_r = ws + used;
         used += align_up((size_t)M * (size_t)K * 2, 256);
+    }
+    const size_t codes_bytes = align_up((size_t)M * (size_t)K / 2, 256);
+    if (native) {
+        a.x_codes = region_a;
+        a.x_side = region_a + codes_bytes;
+        if (region_r) {
+            a.r_codes = region_r;
+            a.r_side = region_r + codes_bytes;
+            a.mask_r_codes = 1;
+        }
+    } else {
+        a.a_bf16 = reinterpret_cast<__nv_bfloat16*>(region_a);
+        a.r_bf16 = reinterpret_cast<__nv_bfloat16*>(region_r);
     }
     rc = launch_quantize(fmt, a, st);
     if (rc) return rc;
+    if (native) {
+        Mxfp4NativeArgs n;
+        memset(&n, 0, sizeof(n));
+        n.a_codes = a.x_codes;
+        n.a_scale = static_cast<const uint8_t*>(a.x_side);
+        n.r_codes = a.r_codes;
+        n.r_scale = static_cast<const uint8_t*>(a.r_side);
+        n.w_codes = static_cast<const uint8_t*>(w_codes);
+        n.w_scale = static_cast<const uint8_t*>(w_side);
+        n.M = M;
+        n.N = N;
+        n.K = K;
+        n.Y = Y;
+        n.out_dtype = out_dtype;
+        n.ldy = ldy;
+        n.status = a.status;
+        return launch_gemm_mxfp4_native(n, st);
+    }
     GemmArgs g;
     memset(&g, 0, sizeof(g));
     g.fmt = fmt;

@@ -82,6 +82,7 @@ struct QuantArgs {
     uint8_t* r_codes;
     void* r_side;
     uint8_t* mask_bits;
+    int mask_r_codes;       // nonzero: r_codes receives S(Q(dX)) (dropped codes zeroed) instead of the canonical Q(dX)
     // expanded operands for the GEMM (any may be null): exact bf16 images of deq Q(X) and S(deq Q(dX))
     __nv_bfloat16* a_bf16;  // [M, K]
     __nv_bfloat16* r_bf16;  // [M, K]
@@ -118,6 +119,23 @@ struct GemmArgs {
     DeviceStatus* status;
 };
 int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream);
+
+// MXFP4 on the block-scaled FP4 tensor pipe (gemm_mxfp4.cu): operands stay packed E2M1 codes + E8M0 scales.
+struct Mxfp4NativeArgs {
+    const uint8_t* a_codes;   // [M, K/2]  Q(X)
+    const uint8_t* a_scale;   // [M, K/32]
+    const uint8_t* r_codes;   // [M, K/2]  S(Q(dX)) with the dropped codes zeroed, or null (pattern NONE)
+    const uint8_t* r_scale;   // [M, K/32]
+    const uint8_t* w_codes;   // [N, K/2]
+    const uint8_t* w_scale;   // [N, K/32]
+    int64_t M, N, K;
+    void* Y;
+    int out_dtype;
+    int64_t ldy;
+    DeviceStatus* status;
+};
+bool gemm_mxfp4_native_supported(int64_t M, int64_t N, int64_t K);
+int launch_gemm_mxfp4_native(const Mxfp4NativeArgs& g, cudaStream_t stream);
 int make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, const void* base, uint64_t inner, uint64_t rows,
                  uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle sw);
 int launch_splitk_reduce(const GemmArgs& g, int splits, cudaStream_t stream);

@@ -1,0 +1,400 @@
+// MXFP4 GEMM of Eq. (5) on the block-scaled FP4 tensor pipe:
+//     Y[m, n] = sum_k a[m, k] w[n, k]  +  sum_k r[m, k] w[n, k]
+// with a = Q(X), r = S(Q(dX)) and w = Q(W) all kept as packed E2M1 codes (two per byte, element 2j in the low
+// nibble) with one E8M0 scale per 32 values along K.  tcgen05.mma kind::mxf4.block_scale multiplies the 4-bit
+// operands straight from shared memory and applies the scales, which it reads from tensor memory: nothing is
+// expanded.  Selected entries of the residual are kept by zeroing the dropped codes (the quantizer does that).
+//
+// One CTA per SM walks 128 x 256 output tiles.  A stage is 256 values of K: 128 x 128 B of activation codes
+// (and as much for the residual), 256 x 128 B of weight codes, and their scales re-arranged into the 512-byte
+// atoms tcgen05.cp copies to tensor memory (32 rows x 16 B: byte r1 * 4 + g of row r0 is the scale of row
+// r0 + 32 * r1 for the g-th group of 32 values).
+// Warp roles (8 warps): 0 TMA producer, 1 MMA issue + TMEM allocation, 2..3 scale gather, 4..7 epilogue.
+// Every wait is bounded; a timeout ends the kernel cleanly (status word, abort flag).
+#include "common.cuh"
+#include "ptx.cuh"
+
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+namespace resq {
+
+namespace {
+
+constexpr int kBM = 128;            // rows per tile (UMMA M)
+constexpr int kBN = 256;            // columns per tile (UMMA N)
+constexpr int kBKe = 256;           // K values per stage
+constexpr int kRowBytes = kBKe / 2; // 128 B of codes per row per stage: one 128-byte-swizzled row
+constexpr int kThreadsNative = 256;
+constexpr int kATile = kBM * kRowBytes;       // 16 KiB
+constexpr int kBTile = kBN * kRowBytes;       // 32 KiB
+constexpr int kSfAtom = 512;                  // scales of 128 rows x 128 values of K
+constexpr int kSfA = 2 * kSfAtom;             // two atoms along K per stage
+constexpr int kSfB = 4 * kSfAtom;             // two along K x two along N
+constexpr int kAccCols = kBN;                 // fp32 accumulator columns
+constexpr int kSfSetCols = 32;                // tensor-memory columns of one stage's scales: A 8, residual 8, W 16
+constexpr int kTmemColsNative = 512;
+constexpr int kSmemBudgetNative = 232448;
+
+struct NativeParams {
+    const uint8_t* a_scale;   // [M, K/32]
+    const uint8_t* r_scale;   // [M, K/32] or null
+    const uint8_t* w_scale;   // [N, K/32]
+    int64_t M, N, K;
+    int ntiles_n, num_tiles;
+    void* Y;
+    int out_f32;
+    int64_t ldy;
+    DeviceStatus* status;
+};
+
+__device__ __forceinline__ void report_timeout_native(DeviceStatus* st, int where) {
+    if (atomicCAS(&st->code, 0, (int)RESQ_ERR_TIMEOUT) == 0) {
+        st->where = where;
+        st->block = (int)blockIdx.x;
+    }
+}
+
+// Instruction descriptor of kind::mxf4 (E2M1 x E2M1, E8M0 scales, K-major operands, M x N tile); the scale-factor
+// ids select which byte of a 32-bit tensor-memory column holds the first scale of this K step.
+__host__ __device__ constexpr uint32_t idesc_mxf4(int m, int n, uint32_t a_sf_id, uint32_t b_sf_id) {
+    return (b_sf_id << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(m >> 4) << 24) |
+           (a_sf_id << 29);
+}
+// Shared-memory descriptor of a 32 x 16 B scale atom (no swizzle: 8-row groups of 128 contiguous bytes).
+__device__ __forceinline__ uint64_t smem_desc_sf(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(128 >> 4) << 16;  // leading byte offset (one 16-byte column only)
+    d |= (uint64_t)(128 >> 4) << 32;  // stride between 8-row groups
+    d |= (uint64_t)1 << 46;
+    return d;
+}
+__device__ __forceinline__ void tmem_cp_sf(uint32_t taddr, uint64_t desc) {
+    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
+}
+__device__ __forceinline__ void umma_mxf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t sfa,
+                                          uint32_t sfb, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+        :
+        : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
+        : "memory");
+}
+
+template <bool RES>
+struct StageLayout {
+    static constexpr int kStagesN = RES ? 3 : 4;
+    static constexpr int kA = 0;
+    static constexpr int kAr = kATile;                                  // only with RES
+    static constexpr int kB = kATile * (RES ? 2 : 1);
+    static constexpr int kSfAOff = kB + kBTile;
+    static constexpr int kSfArOff = kSfAOff + kSfA;                      // only with RES
+    static constexpr int kSfBOff = kSfAOff + kSfA * (RES ? 2 : 1);
+    static constexpr int kBytes = kSfBOff + kSfB;
+    static constexpr uint32_t kTxBytes = (uint32_t)(kATile * (RES ? 2 : 1) + kBTile);
+};
+
+template <bool RES>
+__global__ void __launch_bounds__(kThreadsNative, 1)
+gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_r,
+                         const __grid_constant__ CUtensorMap tmap_w, const NativeParams p) {
+    using L = StageLayout<RES>;
+    constexpr int S = L::kStagesN;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * L::kBytes);
+    uint64_t* full = bars;            // [S] codes landed (TMA bytes) and scale atoms written (two gather warps)
+    uint64_t* empty = bars + 4;       // [S] the MMAs that read the stage completed
+    uint64_t* acc_full = bars + 8;    // accumulator complete
+    uint64_t* acc_empty = bars + 9;   // accumulator drained by the four epilogue warps
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nkb = (int)(p.K / kBKe);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            ptx::mbar_init(&full[s], 3);
+            ptx::mbar_init(&empty[s], 1);
+        }
+        ptx::mbar_init(acc_full, 1);
+        ptx::mbar_init(acc_empty, 4);
+        *abort_flag = 0;
+        ptx::mbar_fence_init();
+    }
+    if (warp == 1) ptx::tmem_alloc(tmem_slot, kTmemColsNative);
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    pdl_trigger();
+    pdl_wait();  // codes and scales of the activations come from the quantizer kernel just before
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            ptx::tma_prefetch_desc(&tmap_a);
+            if (RES) ptx::tma_prefetch_desc(&tmap_r);
+            ptx::tma_prefetch_desc(&tmap_w);
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile / p.ntiles_n) * kBM, n0 = (tile % p.ntiles_n) * kBN;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!ptx::mbar_wait_spin(&empty[s], ph ^ 1u, abort_flag)) {
+                        report_timeout_native(p.status, 1);
+                        ok = false;
+                        break;
+                    }
+                    uint8_t* st = smem + (size_t)s * L::kBytes;
+                    ptx::mbar_arrive_expect_tx(&full[s], L::kTxBytes);
+                    ptx::tma_load_2d(st + L::kA, &tmap_a, &full[s], kb * kRowBytes, m0);
+                    if (RES) ptx::tma_load_2d(st + L::kAr, &tmap_r, &full[s], kb * kRowBytes, m0);
+                    ptx::tma_load_2d(st + L::kB, &tmap_w, &full[s], kb * kRowBytes, n0);
+                    if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint64_t desc0 = ptx::smem_desc_sw128_kmajor(0);
+            const uint32_t smem_base16 = (ptx::smem_u32(smem) & 0x3FFFFu) >> 4;
+            uint32_t s = 0, ph = 0, it = 0;
+            int local_tile = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local_tile) {
+                if (!ptx::mbar_wait_spin(acc_empty, (uint32_t)(local_tile & 1) ^ 1u, abort_flag)) {
+                    report_timeout_native(p.status, 6);
+                    break;
+                }
+                ptx::tc_fence_after();
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    if (!ptx::mbar_wait_spin(&full[s], ph, abort_flag)) {
+                        report_timeout_native(p.status, 2);
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after();
+                    const uint32_t st = ptx::smem_u32(smem) + s * (uint32_t)L::kBytes;
+                    // scales of this stage -> tensor memory (two column sets alternate between stages)
+                    const uint32_t sf = tmem_base + (uint32_t)(kAccCols + (it & 1u) * kSfSetCols);
+#pragma unroll
+                    for (int ka = 0; ka < 2; ++ka) {
+                        tmem_cp_sf(sf + ka * 4, smem_desc_sf(st + L::kSfAOff + ka * kSfAtom));
+                        if (RES) tmem_cp_sf(sf + 8 + ka * 4, smem_desc_sf(st + L::kSfArOff + ka * kSfAtom));
+#pragma unroll
+                        for (int nb = 0; nb < 2; ++nb)
+                            tmem_cp_sf(sf + 16 + ka * 8 + nb * 4, smem_desc_sf(st + L::kSfBOff + (ka * 2 + nb) * kSfAtom));
+                    }
+                    const uint32_t st16 = smem_base16 + s * (uint32_t)(L::kBytes >> 4);
+                    const uint64_t adesc = desc0 + (uint64_t)(st16 + (L::kA >> 4));
+                    const uint64_t rdesc = desc0 + (uint64_t)(st16 + (L::kAr >> 4));
+                    const uint64_t bdesc = desc0 + (uint64_t)(st16 + (L::kB >> 4));
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4) {  // 64 values (32 B) of K per MMA: two scale groups
+                        const int ka = k4 >> 1;
+                        const uint32_t sfid = (uint32_t)(k4 & 1) * 2u;
+                        const uint32_t idesc = idesc_mxf4(kBM, kBN, sfid, sfid);
+                        const uint32_t sfa = sf + ka * 4 + (sfid << 30), sfb = sf + 16 + ka * 8 + (sfid << 30);
+                        umma_mxf4(tmem_base, adesc + (uint64_t)(2 * k4), bdesc + (uint64_t)(2 * k4), idesc, sfa, sfb,
+                                  (kb > 0 || k4 > 0) ? 1u : 0u);
+                        if (RES)
+                            umma_mxf4(tmem_base, rdesc + (uint64_t)(2 * k4), bdesc + (uint64_t)(2 * k4), idesc,
+                                      sf + 8 + ka * 4 + (sfid << 30), sfb, 1u);
+                    }
+                    ptx::umma_commit(&empty[s]);
+                    if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
+                }
+                if (ok) ptx::umma_commit(acc_full);
+            }
+        }
+    } else if (warp < 4) {
+        // ------------------------------------------------------------------ scale gather (64 threads)
+        const int t = (warp - 2) * 32 + lane;
+        const int64_t spr = p.K / 32;  // scale bytes per row
+        uint32_t s = 0, ph = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+            const int64_t m0 = (int64_t)(tile / p.ntiles_n) * kBM, n0 = (int64_t)(tile % p.ntiles_n) * kBN;
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!ptx::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) {
+                    report_timeout_native(p.status, 3);
+                    ok = false;
+                    break;
+                }
+                uint8_t* st = smem + (size_t)s * L::kBytes;
+                // row rr of a 128-row atom: 4 bytes at (rr % 32) * 16 + (rr / 32) * 4; 8 scale bytes per row and stage
+                auto put = [&](uint8_t* atoms, int rr, const uint8_t* src, bool valid) {
+                    uint2 v = make_uint2(0u, 0u);
+                    if (valid) v = *reinterpret_cast<const uint2*>(src);
+                    const int off = (rr & 31) * 16 + (rr >> 5) * 4;
+                    *reinterpret_cast<uint32_t*>(atoms + off) = v.x;
+                    *reinterpret_cast<uint32_t*>(atoms + kSfAtom + off) = v.y;
+                };
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const int rr = t + 64 * j;
+                    const int64_t m = m0 + rr;
+                    put(st + L::kSfAOff, rr, p.a_scale + m * spr + kb * 8, m < p.M);
+                    if (RES) put(st + L::kSfArOff, rr, p.r_scale + m * spr + kb * 8, m < p.M);
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int rn = t + 64 * j;  // row of the 256-row weight tile
+                    const int64_t n = n0 + rn;
+                    // atoms of W: (ka, nb) at (ka * 2 + nb) * 512: the two K atoms of one N half are 1024 B apart
+                    uint2 v = make_uint2(0u, 0u);
+                    if (n < p.N) v = *reinterpret_cast<const uint2*>(p.w_scale + n * spr + kb * 8);
+                    const int nb = rn >> 7, rr = rn & 127;
+                    const int off = (rr & 31) * 16 + (rr >> 5) * 4;
+                    *reinterpret_cast<uint32_t*>(st + L::kSfBOff + (0 * 2 + nb) * kSfAtom + off) = v.x;
+                    *reinterpret_cast<uint32_t*>(st + L::kSfBOff + (1 * 2 + nb) * kSfAtom + off) = v.y;
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&full[s]);
+                if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 4..7)
+        const int quad = warp & 3;
+        int local_tile = 0;
+        for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++local_tile) {
+            const int64_t m0 = (int64_t)(tile / p.ntiles_n) * kBM, n0 = (int64_t)(tile % p.ntiles_n) * kBN;
+            if (!ptx::mbar_wait(acc_full, (uint32_t)(local_tile & 1), abort_flag)) {
+                report_timeout_native(p.status, 4);
+                break;
+            }
+            ptx::tc_fence_after();
+            const int64_t m = m0 + quad * 32 + lane;
+#pragma unroll 1
+            for (int cc = 0; cc < kBN / 32; ++cc) {
+                uint32_t v[32];
+                ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(cc * 32), v);
+                ptx::tmem_ld_wait();
+                if (cc == kBN / 32 - 1) {
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(acc_empty);
+                }
+                if (m >= p.M) continue;
+                const int64_t nb = n0 + cc * 32;
+                const int64_t left = p.N - nb;
+                if (left <= 0) continue;
+                if (p.out_f32) {
+                    float* dst = reinterpret_cast<float*>(p.Y) + m * p.ldy + nb;
+                    if (left >= 32) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < left) dst[j] = __uint_as_float(v[j]);
+                    }
+                } else {
+                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.Y) + m * p.ldy + nb;
+                    if (left >= 32) {
+                        uint32_t o[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                            o[j] = *reinterpret_cast<uint32_t*>(&b);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4)
+                            *reinterpret_cast<uint4*>(dst + 2 * j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < left) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                    }
+                }
+            }
+        }
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, kTmemColsNative);
+    }
+}
+
+template <bool RES>
+int launch_native_variant(const Mxfp4NativeArgs& g, cudaStream_t stream) {
+    using L = StageLayout<RES>;
+    CUtensorMap ta, tr, tw;
+    int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.a_codes, (uint64_t)g.K / 2, (uint64_t)g.M, (uint64_t)g.K / 2,
+                          kRowBytes, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    rc = make_tmap_2d(&tr, CU_TENSOR_MAP_DATA_TYPE_UINT8, RES ? g.r_codes : g.a_codes, (uint64_t)g.K / 2, (uint64_t)g.M,
+                      (uint64_t)g.K / 2, kRowBytes, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.w_codes, (uint64_t)g.K / 2, (uint64_t)g.N, (uint64_t)g.K / 2,
+                      kRowBytes, kBN, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    NativeParams p;
+    p.a_scale = g.a_scale;
+    p.r_scale = g.r_scale;
+    p.w_scale = g.w_scale;
+    p.M = g.M;
+    p.N = g.N;
+    p.K = g.K;
+    p.ntiles_n = (int)((g.N + kBN - 1) / kBN);
+    p.num_tiles = (int)((g.M + kBM - 1) / kBM) * p.ntiles_n;
+    p.Y = g.Y;
+    p.out_f32 = g.out_dtype == RESQ_OUT_F32;
+    p.ldy = g.ldy;
+    p.status = g.status;
+    const int smem_bytes = 1024 + L::kStagesN * L::kBytes + 256;
+    static_assert(1024 + L::kStagesN * L::kBytes + 256 <= kSmemBudgetNative, "stages do not fit");
+    auto kern = gemm_mxfp4_native_kernel<RES>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes); });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute(gemm mxfp4)");
+    static int num_sms = 0;
+    if (num_sms == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (num_sms <= 0) num_sms = 148;
+    }
+    const unsigned grid = (unsigned)std::min(p.num_tiles, num_sms);
+    LaunchScope scope(kKindGemm, stream);
+    return cuda_fail(launch_kernel(kern, dim3(grid), dim3(kThreadsNative), (size_t)smem_bytes, stream, ta, tr, tw, p),
+                     "gemm_mxfp4_native_kernel launch");
+}
+
+}  // namespace
+
+bool gemm_mxfp4_native_supported(int64_t M, int64_t N, int64_t K) {
+    // RESQ_MXFP4_NATIVE: debugging override (0: never, 1: whenever the shape allows, unset: when it pays)
+    const char* v = getenv("RESQ_MXFP4_NATIVE");
+    const int mode = (v && *v) ? atoi(v) : -1;
+    if (mode == 0 || K % kBKe != 0) return false;
+    if (mode == 1) return true;
+    // no K split yet: needs enough 128 x 256 tiles to fill the machine (decode-sized calls keep the bf16 path)
+    const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
+    return tiles >= 148;
+}
+
+int launch_gemm_mxfp4_native(const Mxfp4NativeArgs& g, cudaStream_t stream) {
+    auto al8 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 7u) == 0; };
+    if (!al8(g.a_scale) || !al8(g.w_scale) || (g.r_scale && !al8(g.r_scale))) {
+        set_last_error("native MXFP4 GEMM: scale arrays must be 8-byte aligned");
+        return RESQ_ERR_ALIGN;
+    }
+    return g.r_codes ? launch_native_variant<true>(g, stream) : launch_native_variant<false>(g, stream);
+}
+
+}  // namespace resq

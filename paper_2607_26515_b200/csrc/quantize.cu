@@ -190,7 +190,16 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
             }
         }
         if (active) {
-            if (a.r_codes) *reinterpret_cast<uint32_t*>(a.r_codes + m * (a.K / 2) + k0 / 2) = rcodes;
+            if (a.r_codes) {
+                uint32_t rc = rcodes;
+                if (a.mask_r_codes) {  // operand form for the block-scaled FP4 GEMM: dropped entries become code 0
+                    uint32_t nib = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) nib |= ((keep >> i) & 1u) * (0xFu << (4 * i));
+                    rc &= nib;
+                }
+                *reinterpret_cast<uint32_t*>(a.r_codes + m * (a.K / 2) + k0 / 2) = rc;
+            }
             if (a.r_side && side_lane) {
                 if (FMT == kHiF4) reinterpret_cast<uint32_t*>(a.r_side)[m * side_cols + side_k] = rside;
                 else reinterpret_cast<uint8_t*>(a.r_side)[m * side_cols + side_k] = (uint8_t)rside;

@@ -185,6 +185,27 @@ def test_every_tile_configuration(tile_case, cfg, pattern, fmt, monkeypatch):
     check_close(y.cpu().numpy(), w["y"], w["abs_sum"])
 
 
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_DENSE, oracle.S_2_4])
+@pytest.mark.parametrize("shape", [(300, 512, 600), (128, 256, 256), (1000, 1024, 1300)])
+def test_mxfp4_block_scaled_fp4_gemm(monkeypatch, pattern, shape):
+    """MXFP4 on the block-scaled FP4 tensor pipe (packed codes + scales straight into tcgen05.mma kind::mxf4),
+    forced on for these small shapes; the same call with the path switched off must agree within tolerance too."""
+    m = rq()
+    M, K, N = shape
+    xb, wb = synth_xw(17 * M + N + pattern, M, K, N, n_out=max(1, K // 256))
+    want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern, "mxfp4")
+    wc, ws = m.pack_weight(to_dev(wb), "mxfp4")
+    work = m.alloc_workspace(m.resq_workspace_bytes(M, N, K, pattern, "mxfp4"))
+    for native in ("1", "0"):
+        monkeypatch.setenv("RESQ_MXFP4_NATIVE", native)
+        y = m.resq_linear(to_dev(xb), wc, ws, pattern, "mxfp4", out_dtype=torch.float32, workspace=work)
+        assert m.check(work) == 0, m.last_error()
+        check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+    monkeypatch.setenv("RESQ_MXFP4_NATIVE", "1")
+    yb = m.resq_linear(to_dev(xb), wc, ws, pattern, "mxfp4", out_dtype=torch.bfloat16, workspace=work)
+    check_close(yb.float().cpu().numpy(), want["y"], want["abs_sum"], bf16_out=True)
+
+
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_k_streamed_schedule_with_uneven_segments(monkeypatch, out_dtype):
     """More output tiles than CTA pairs: the (tile, k-block) units are dealt out evenly, so pairs start and end in
