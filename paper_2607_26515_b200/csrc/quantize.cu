@@ -368,7 +368,68 @@ __device__ __forceinline__ void hif4_encode_block(const uint32_t (&w)[32], uint3
     meta = m;
 }
 
-template <bool RESIDUAL, bool IMG>
+// MXFP4 counterpart: the lane's 64 values are two blocks of 32 (chunks 0..3 and 4..7), each with its own E8M0
+// scale; `scales` returns the two scale bytes.  Same element arithmetic as mxfp4_encode_lane (hardware E2M1
+// conversion of the exactly scaled values); dq: decoded magnitudes.
+template <bool DEQ, bool OCT, typename Sink>
+__device__ __forceinline__ void mxfp4_encode_block(const uint32_t (&w)[32], uint32_t (&codes)[8], uint32_t& scales, Sink&& sink) {
+    uint32_t m8[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        uint32_t mA, mB;
+        chunk_maxima(&w[4 * c], mA, mB);
+        m8[c] = max(mA, mB);
+    }
+    scales = 0;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t amax16 = max(max(m8[4 * h], m8[4 * h + 1]), max(m8[4 * h + 2], m8[4 * h + 3]));
+        const int sc = max((int)(amax16 >> 7) - 2, 0);  // bf16 exponent field of the block maximum, minus E2M1's top exponent
+        scales |= (uint32_t)sc << (8 * h);
+        const float inv = pow2_from_biased(254 - sc);
+        const float sf = e8m0_to_float(sc);
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+            const int c = 4 * h + cc;
+            float x[8], dq[8];
+            uint32_t packed4 = 0;
+#pragma unroll
+            for (int i = 3; i >= 0; --i) {
+                x[2 * i] = __uint_as_float(w[4 * c + i] << 16);
+                x[2 * i + 1] = __uint_as_float(w[4 * c + i] & 0xFFFF0000u);
+                const float lo = __fmul_rn(x[2 * i], inv), hi = __fmul_rn(x[2 * i + 1], inv);
+                uint16_t pk;
+                asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %1, %2; mov.b16 %0, {t, 0}; }" : "=h"(pk) : "f"(hi), "f"(lo));
+                if (DEQ) {
+                    uint32_t h2;
+                    asm("{ .reg .b8 t, z; mov.b16 {t, z}, %1; cvt.rn.f16x2.e2m1x2 %0, t; }" : "=r"(h2) : "h"(pk));
+                    const __half2 hv = *reinterpret_cast<__half2*>(&h2);
+                    dq[2 * i] = fabsf(__fmul_rn(__low2float(hv), sf));
+                    dq[2 * i + 1] = fabsf(__fmul_rn(__high2float(hv), sf));
+                }
+                packed4 = (packed4 << 8) | (uint32_t)(pk & 0xFF);
+            }
+            codes[c] = packed4;
+            uint32_t oct = 0;
+            if (OCT) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    oct |= ((packed4 >> (4 * i)) & 7u) << (3 * i);
+                    oct |= ((packed4 >> (16 + 4 * i)) & 7u) << (16 + 3 * i);
+                }
+            }
+            sink(c, x, dq, oct);
+        }
+    }
+}
+
+template <int FMT, bool DEQ, bool OCT, typename Sink>
+__device__ __forceinline__ void encode_block(const uint32_t (&w)[32], uint32_t (&codes)[8], uint32_t& side, Sink&& sink) {
+    if constexpr (FMT == kHiF4) hif4_encode_block<DEQ, OCT>(w, codes, side, sink);
+    else mxfp4_encode_block<DEQ, OCT>(w, codes, side, sink);
+}
+
+template <int FMT, bool RESIDUAL, bool IMG>
 __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, int rows_per_warp) {
     pdl_wait();     // nothing below may touch global memory before the previous kernel of the stream is done
     pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
@@ -436,7 +497,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
 
         uint32_t codes[8], meta;
         // main encode; with RESIDUAL, w is overwritten by dX = X - deq Q(X) (Eq. (3)), exact in bf16
-        hif4_encode_block<RESIDUAL || IMG, false>(w, codes, meta, [&](int c, const float (&x)[8], const float (&dq)[8], uint32_t) {
+        encode_block<FMT, RESIDUAL || IMG, false>(w, codes, meta, [&](int c, const float (&x)[8], const float (&dq)[8], uint32_t) {
             if constexpr (RESIDUAL) {
                 float sd[8];
 #pragma unroll
@@ -460,13 +521,16 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
                 p[0] = make_uint4(codes[0], codes[1], codes[2], codes[3]);
                 p[1] = make_uint4(codes[4], codes[5], codes[6], codes[7]);
             }
-            if (a.x_side) reinterpret_cast<uint32_t*>(a.x_side)[m * G + blk] = meta;
+            if (a.x_side) {
+                if constexpr (FMT == kHiF4) reinterpret_cast<uint32_t*>(a.x_side)[m * G + blk] = meta;
+                else *reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(a.x_side) + (m * G + blk) * 2) = (uint16_t)meta;
+            }
         }
         if constexpr (IMG) drain_stage(a.a_bf16 + m * a.K);
         if constexpr (RESIDUAL) {
             uint32_t rcodes[8], rmeta, keep_lo = 0xFFFFFFFFu, keep_hi = 0xFFFFFFFFu;
-            float sq = 0.0f;
-            hif4_encode_block<true, true>(w, rcodes, rmeta, [&](int c, const float (&)[8], const float (&rdq)[8], uint32_t roct) {
+            float sq0 = 0.0f, sq1 = 0.0f;  // per 32 values: exact in fp32 for both formats (see below)
+            encode_block<FMT, true, true>(w, rcodes, rmeta, [&](int c, const float (&)[8], const float (&rdq)[8], uint32_t roct) {
                 uint32_t keep = 0xFFu;
                 if (pattern == RESQ_S_2_4) {
                     keep = top2_mask8(roct);
@@ -474,9 +538,13 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
                     else keep_hi = (keep_hi & ~(0xFFu << (8 * (c - 4)))) | (keep << (8 * (c - 4)));
                 }
                 if (pattern == RESQ_S_BLOCK32x64_50) {
-                    // 64 squares of at most 12 significant bits whose exponents differ by at most 4: exact in fp32
+                    // 32 squares of at most 12 significant bits whose exponents differ by at most 4 (HiF4) or that
+                    // share one power-of-two scale (MXFP4): exact in fp32; the two halves may differ more (MXFP4)
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) sq = __fmaf_rn(rdq[i], rdq[i], sq);
+                    for (int i = 0; i < 8; ++i) {
+                        if (c < 4) sq0 = __fmaf_rn(rdq[i], rdq[i], sq0);
+                        else sq1 = __fmaf_rn(rdq[i], rdq[i], sq1);
+                    }
                 }
                 if constexpr (IMG) {
                     // for BLOCK this is the unmasked image; the apply kernel zeroes dropped entries
@@ -490,7 +558,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
                 }
             });
             if (pattern == RESQ_S_BLOCK32x64_50) {
-                blk_acc += (double)sq;
+                blk_acc += (double)sq0 + (double)sq1;
                 if (((m + 1) % kBlkRows) == 0 || m + 1 == m_end) {
                     if (active) atomicAdd(&a.scores[(m / kBlkRows) * G + blk], blk_acc);
                     blk_acc = 0.0;
@@ -498,11 +566,24 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
             }
             if (active) {
                 if (a.r_codes) {
+                    if (a.mask_r_codes) {  // operand form for the block-scaled FP4 GEMM: dropped entries become code 0
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const uint32_t keep = ((c < 4 ? keep_lo : keep_hi) >> (8 * (c & 3))) & 0xFFu;
+                            uint32_t nib = 0;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) nib |= ((keep >> i) & 1u) * (0xFu << (4 * i));
+                            rcodes[c] &= nib;
+                        }
+                    }
                     uint4* p = reinterpret_cast<uint4*>(a.r_codes + m * (a.K / 2) + blk * 32);
                     p[0] = make_uint4(rcodes[0], rcodes[1], rcodes[2], rcodes[3]);
                     p[1] = make_uint4(rcodes[4], rcodes[5], rcodes[6], rcodes[7]);
                 }
-                if (a.r_side) reinterpret_cast<uint32_t*>(a.r_side)[m * G + blk] = rmeta;
+                if (a.r_side) {
+                    if constexpr (FMT == kHiF4) reinterpret_cast<uint32_t*>(a.r_side)[m * G + blk] = rmeta;
+                    else *reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(a.r_side) + (m * G + blk) * 2) = (uint16_t)rmeta;
+                }
                 const bool local = pattern == RESQ_S_DENSE || pattern == RESQ_S_2_4;
                 if (a.mask_bits && local) *reinterpret_cast<uint2*>(a.mask_bits + m * (a.K / 8) + blk * 8) = make_uint2(keep_lo, keep_hi);
             }
@@ -845,12 +926,13 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
         cudaError_t e = cudaMemsetAsync(a.scores, 0, (size_t)nscore * sizeof(double), stream);
         if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(scores)");
     }
-    // HiF4 with a row-local or block-wise selection: block-per-lane kernel (needs 16-byte aligned outputs)
+    // row-local or block-wise selection on a large enough input: block-per-lane kernel (needs 16-byte aligned
+    // outputs and, for MXFP4, whole pairs of 32-value blocks)
     auto al16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
     // Worth it once there is a warp task (32 blocks of one row) for every warp slot of the machine; below
     // that the finer-grained kernel (a lane per 8 values) finishes sooner.
     const int64_t block_tasks = a.M * ((a.K / kHif4Block + 31) / 32);
-    if (fmt == kHiF4 && pattern != RESQ_S_CHAN50 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
+    if (pattern != RESQ_S_CHAN50 && a.K % kHif4Block == 0 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
         al16(a.a_bf16) && al16(a.r_bf16)) {
         const bool img = a.a_bf16 != nullptr;
         const int64_t ncg = (a.K / kHif4Block + 31) / 32;
@@ -866,8 +948,13 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
             return cuda_fail(launch_kernel(kern, dim3(ctas), dim3(kThreads), (size_t)smem, stream, a, rows_per_warp),
                              "quant_block_kernel launch");
         };
-        int rc = residual ? (img ? launch(quant_block_kernel<true, true>) : launch(quant_block_kernel<true, false>))
-                          : (img ? launch(quant_block_kernel<false, true>) : launch(quant_block_kernel<false, false>));
+        int rc;
+        if (fmt == kHiF4)
+            rc = residual ? (img ? launch(quant_block_kernel<kHiF4, true, true>) : launch(quant_block_kernel<kHiF4, true, false>))
+                          : (img ? launch(quant_block_kernel<kHiF4, false, true>) : launch(quant_block_kernel<kHiF4, false, false>));
+        else
+            rc = residual ? (img ? launch(quant_block_kernel<kMXFP4, true, true>) : launch(quant_block_kernel<kMXFP4, true, false>))
+                          : (img ? launch(quant_block_kernel<kMXFP4, false, true>) : launch(quant_block_kernel<kMXFP4, false, false>));
         if (rc) return rc;
         if (global_sel) {
             { LaunchScope scope(kKindSelect, stream);
