@@ -674,10 +674,15 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
     p.sk_flags = g.sk_flags;
     constexpr int exp_stage = my_rows * 128, raw_stage = my_rows * 32;
     const int fixed = 1024 + 1024;
-    p.se = kExpGroups;  // one slot per expander group (a group never runs two phases ahead on a slot)
-    p.sr = kExpGroups;  // the groups read k-blocks i .. i+3 concurrently
-    p.sa = kExpGroups;  // the activation ring shares its full / empty barriers with the expanded-weight ring
-    if (fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage > kSmemBudget) {
+    // Ring slots: a multiple of the number of expander groups (group g works on the slots s = g mod NG, so a slot
+    // is only ever written by one group).  With one slot per group the group's expansion of a k-block and the
+    // MMAs that read its previous k-block alternate; with two slots per group they overlap.  All three rings have
+    // the same depth (they share the slot's full / empty barriers).
+    const int slot_bytes = kAStage + exp_stage + raw_stage;
+    int per_group = (fixed + 2 * kExpGroups * slot_bytes <= kSmemBudget) ? 2 : 1;
+    per_group = std::max(1, std::min(per_group, env_int("RESQ_GEMM_SLOTS_PER_GROUP", 2)));
+    p.se = p.sr = p.sa = kExpGroups * per_group;
+    if (p.sa > kMaxRing || fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage > kSmemBudget) {
         set_last_error("internal: shared-memory rings do not fit (pair tile %d)", TN);
         return RESQ_ERR_CUDA;
     }
