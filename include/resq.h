@@ -139,7 +139,18 @@ RESQ_API int resq_residual_mask_static(const void* X_bf16, int64_t M, int64_t K,
 /* ---- the rollout projection, Eq. (5):  Y = Q(X) Q(W)^T + S(Q(dX)) Q(W)^T ------------------------
  * X_bf16 [M, K] (ldx), packed weight from *_pack_weight, Y [M, N] (ldy) as bf16 (round-to-nearest-
  * even of the fp32 accumulator) or fp32.  Products of decoded values are exact in fp32; only the
- * accumulation rounds.  Both terms are accumulated into the same output tile. */
+ * accumulation rounds.  Both terms are accumulated into the same output tile.
+ *   - The workspace holds the status word, arrival counters, the quantizer's outputs and fp32 partial
+ *     tiles of the call: a workspace must not be shared by calls whose kernels may overlap on the GPU.
+ *   - For decode-sized problems the GEMM kernel's CTAs wait for one another at its end (bounded) and are
+ *     sized to be resident all at once on an otherwise idle device.  Calls whose kernels overlap on the
+ *     same device (different streams) can therefore delay each other up to the bound and then end with
+ *     RESQ_ERR_TIMEOUT in the status word instead of a result: issue them on one stream.
+ *   - Consecutive calls on one stream overlap their kernels' set-up through programmatic dependent
+ *     launch; every kernel waits for its predecessor before it touches memory that one may have written.
+ *   - MXFP4 with pattern NONE / DENSE / 2:4, K a multiple of 256 and at least 148 output tiles of 128 x 256
+ *     runs on the block-scaled FP4 tensor pipe; everything else on the bf16 pipe.  Both are exact in the
+ *     products; they differ in accumulation order only. */
 RESQ_API int hif4_resq_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
                      const void* w_codes, const void* w_meta, int64_t N,
                      int pattern, void* Y, int out_dtype, int64_t ldy,
