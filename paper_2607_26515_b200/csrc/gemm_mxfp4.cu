@@ -217,51 +217,70 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         }
     } else if (warp < 4) {
         // ------------------------------------------------------------------ scale gather (64 threads)
+        // Each thread owns 2 activation rows (+ 2 residual rows) and 4 weight rows of the tile: 8 scale bytes per
+        // row and stage.  The loads of the next stage are issued before this stage's slot is waited for, so
+        // their latency (uncoalesced 8-byte reads) stays off the slot's critical path.
         const int t = (warp - 2) * 32 + lane;
         const int64_t spr = p.K / 32;  // scale bytes per row
         uint32_t s = 0, ph = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+        uint2 va[2], vr[2], vw[4];
+        auto load_scales = [&](int tile, int kb) {
             const int64_t m0 = (int64_t)(tile / p.ntiles_n) * kBM, n0 = (int64_t)(tile % p.ntiles_n) * kBN;
-            for (int kb = 0; kb < nkb; ++kb) {
-                if (!ptx::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) {
-                    report_timeout_native(p.status, 3);
-                    ok = false;
-                    break;
-                }
-                uint8_t* st = smem + (size_t)s * L::kBytes;
-                // row rr of a 128-row atom: 4 bytes at (rr % 32) * 16 + (rr / 32) * 4; 8 scale bytes per row and stage
-                auto put = [&](uint8_t* atoms, int rr, const uint8_t* src, bool valid) {
-                    uint2 v = make_uint2(0u, 0u);
-                    if (valid) v = *reinterpret_cast<const uint2*>(src);
-                    const int off = (rr & 31) * 16 + (rr >> 5) * 4;
-                    *reinterpret_cast<uint32_t*>(atoms + off) = v.x;
-                    *reinterpret_cast<uint32_t*>(atoms + kSfAtom + off) = v.y;
-                };
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const int rr = t + 64 * j;
-                    const int64_t m = m0 + rr;
-                    put(st + L::kSfAOff, rr, p.a_scale + m * spr + kb * 8, m < p.M);
-                    if (RES) put(st + L::kSfArOff, rr, p.r_scale + m * spr + kb * 8, m < p.M);
+            for (int j = 0; j < 2; ++j) {
+                const int64_t m = m0 + t + 64 * j;
+                va[j] = vr[j] = make_uint2(0u, 0u);
+                if (m < p.M) {
+                    va[j] = *reinterpret_cast<const uint2*>(p.a_scale + m * spr + kb * 8);
+                    if (RES) vr[j] = *reinterpret_cast<const uint2*>(p.r_scale + m * spr + kb * 8);
                 }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int rn = t + 64 * j;  // row of the 256-row weight tile
-                    const int64_t n = n0 + rn;
-                    // atoms of W: (ka, nb) at (ka * 2 + nb) * 512: the two K atoms of one N half are 1024 B apart
-                    uint2 v = make_uint2(0u, 0u);
-                    if (n < p.N) v = *reinterpret_cast<const uint2*>(p.w_scale + n * spr + kb * 8);
-                    const int nb = rn >> 7, rr = rn & 127;
-                    const int off = (rr & 31) * 16 + (rr >> 5) * 4;
-                    *reinterpret_cast<uint32_t*>(st + L::kSfBOff + (0 * 2 + nb) * kSfAtom + off) = v.x;
-                    *reinterpret_cast<uint32_t*>(st + L::kSfBOff + (1 * 2 + nb) * kSfAtom + off) = v.y;
-                }
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&full[s]);
-                if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
             }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int64_t n = n0 + t + 64 * j;
+                vw[j] = make_uint2(0u, 0u);
+                if (n < p.N) vw[j] = *reinterpret_cast<const uint2*>(p.w_scale + n * spr + kb * 8);
+            }
+        };
+        int tile = blockIdx.x, kb = 0;
+        if (tile < p.num_tiles) load_scales(tile, kb);
+        while (tile < p.num_tiles && ok) {
+            if (!ptx::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) {
+                report_timeout_native(p.status, 3);
+                ok = false;
+                break;
+            }
+            uint8_t* st = smem + (size_t)s * L::kBytes;
+            // row rr of a 128-row atom: 4 bytes at (rr % 32) * 16 + (rr / 32) * 4; the two K atoms are 512 B apart
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int rr = t + 64 * j;
+                const int off = (rr & 31) * 16 + (rr >> 5) * 4;
+                *reinterpret_cast<uint32_t*>(st + L::kSfAOff + off) = va[j].x;
+                *reinterpret_cast<uint32_t*>(st + L::kSfAOff + kSfAtom + off) = va[j].y;
+                if (RES) {
+                    *reinterpret_cast<uint32_t*>(st + L::kSfArOff + off) = vr[j].x;
+                    *reinterpret_cast<uint32_t*>(st + L::kSfArOff + kSfAtom + off) = vr[j].y;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int rn = t + 64 * j;  // row of the 256-row weight tile; atoms of W: (ka, nb) at (ka * 2 + nb) * 512
+                const int nb = rn >> 7, rr = rn & 127;
+                const int off = (rr & 31) * 16 + (rr >> 5) * 4;
+                *reinterpret_cast<uint32_t*>(st + L::kSfBOff + (0 * 2 + nb) * kSfAtom + off) = vw[j].x;
+                *reinterpret_cast<uint32_t*>(st + L::kSfBOff + (1 * 2 + nb) * kSfAtom + off) = vw[j].y;
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&full[s]);
+            if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
+            if (++kb == nkb) {
+                kb = 0;
+                tile += gridDim.x;
+            }
+            if (tile < p.num_tiles) load_scales(tile, kb);  // in flight while the next slot is awaited
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 4..7)
