@@ -134,7 +134,7 @@ struct Mxfp4NativeArgs {
     int64_t ldy;
     DeviceStatus* status;
 };
-bool gemm_mxfp4_native_supported(int64_t M, int64_t N, int64_t K);
+bool gemm_mxfp4_native_supported(int64_t M, int64_t N, int64_t K, bool res);
 int launch_gemm_mxfp4_native(const Mxfp4NativeArgs& g, cudaStream_t stream);
 int make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, const void* base, uint64_t inner, uint64_t rows,
                  uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle sw);

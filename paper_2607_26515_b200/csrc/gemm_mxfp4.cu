@@ -396,15 +396,19 @@ int launch_native_variant(const Mxfp4NativeArgs& g, cudaStream_t stream) {
 
 }  // namespace
 
-bool gemm_mxfp4_native_supported(int64_t M, int64_t N, int64_t K) {
+bool gemm_mxfp4_native_supported(int64_t M, int64_t N, int64_t K, bool res) {
     // RESQ_MXFP4_NATIVE: debugging override (0: never, 1: whenever the shape allows, unset: when it pays)
     const char* v = getenv("RESQ_MXFP4_NATIVE");
     const int mode = (v && *v) ? atoi(v) : -1;
     if (mode == 0 || K % kBKe != 0) return false;
     if (mode == 1) return true;
-    // no K split yet: needs enough 128 x 256 tiles to fill the machine (decode-sized calls keep the bf16 path)
+    // No K split here: a CTA walks the whole K range of its tiles, about 1.1 us per 256 values of K.  The bf16
+    // route splits K for decode-sized calls; its time is about 15 us plus the executed flops at 1 PFLOP/s.
+    // (Both fitted to the layer shapes of the 3B / 7B configurations at M = 256 ... 16384.)
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
-    return tiles >= 148;
+    const double t_native = 8.0 + (double)((tiles + 147) / 148) * (double)(K / kBKe) * 1.1;
+    const double t_bf16 = 15.0 + 2.0 * (double)M * (double)N * (double)K * (res ? 2.0 : 1.0) / 1.0e9;
+    return t_native < t_bf16;
 }
 
 int launch_gemm_mxfp4_native(const Mxfp4NativeArgs& g, cudaStream_t stream) {
