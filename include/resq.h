@@ -148,9 +148,9 @@ RESQ_API int resq_residual_mask_static(const void* X_bf16, int64_t M, int64_t K,
  *     RESQ_ERR_TIMEOUT in the status word instead of a result: issue them on one stream.
  *   - Consecutive calls on one stream overlap their kernels' set-up through programmatic dependent
  *     launch; every kernel waits for its predecessor before it touches memory that one may have written.
- *   - MXFP4 with pattern NONE / DENSE / 2:4, K a multiple of 256 and at least 148 output tiles of 128 x 256
- *     runs on the block-scaled FP4 tensor pipe; everything else on the bf16 pipe.  Both are exact in the
- *     products; they differ in accumulation order only. */
+ *   - MXFP4 with K a multiple of 256 runs on the block-scaled FP4 tensor pipe where that is faster (all but
+ *     long-K calls with few output tiles); everything else on the bf16 pipe.  Both are exact in the products;
+ *     they differ in accumulation order only. */
 RESQ_API int hif4_resq_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
                      const void* w_codes, const void* w_meta, int64_t N,
                      int pattern, void* Y, int out_dtype, int64_t ldy,

@@ -235,10 +235,9 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     a.clear_words = reinterpret_cast<uint32_t*>(ws);  // cleared by the quantizer kernel: no separate memset node
     a.n_clear_words = (int)((kWsHeader + kWsFlags) / 4);
     used += kWsFlags;
-    // MXFP4 with a row-local selection: the GEMM runs on the block-scaled FP4 pipe and takes packed codes and
-    // scales (they fit into the space of the bf16 images); every other case takes exact bf16 images.
-    const bool native = fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K, pattern != RESQ_S_NONE) &&
-                        (pattern == RESQ_S_NONE || pattern == RESQ_S_DENSE || pattern == RESQ_S_2_4);
+    // MXFP4 where it pays: the GEMM runs on the block-scaled FP4 pipe and takes packed codes and scales (they
+    // fit into the space of the bf16 images; the selection zeroes dropped codes); otherwise exact bf16 images.
+    const bool native = fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K, pattern != RESQ_S_NONE);
     uint8_t* region_a = ws + used;
     used += align_up((size_t)M * (size_t)K * 2, 256);
     uint8_t* region_r = nullptr;

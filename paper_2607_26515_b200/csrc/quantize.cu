@@ -684,7 +684,8 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(const double* 
 // Turn the kept-channel / kept-block flags into mask bits and zero the dropped entries of the GEMM's
 // residual operand.  One thread per 8 channels of one row.
 __global__ void apply_global_mask_kernel(int pattern, int64_t M, int64_t K, const uint8_t* __restrict__ flag,
-                                         uint8_t* __restrict__ mask_bits, __nv_bfloat16* __restrict__ r_bf16) {
+                                         uint8_t* __restrict__ mask_bits, __nv_bfloat16* __restrict__ r_bf16,
+                                         uint8_t* __restrict__ r_codes_masked) {
     int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     int64_t per_row = K / 8;
     if (idx >= M * per_row) return;
@@ -701,6 +702,13 @@ __global__ void apply_global_mask_kernel(int pattern, int64_t M, int64_t K, cons
         keep = flag[(m / kBlkRows) * (K / kBlkCols) + k0 / kBlkCols] ? 0xFFu : 0u;
     }
     if (mask_bits) mask_bits[idx] = (uint8_t)keep;
+    if (r_codes_masked && keep != 0xFFu) {  // operand form for the block-scaled FP4 GEMM: dropped entries become code 0
+        uint32_t nib = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) nib |= ((keep >> i) & 1u) * (0xFu << (4 * i));
+        uint32_t* c = reinterpret_cast<uint32_t*>(r_codes_masked + m * (K / 2) + k0 / 2);
+        *c &= nib;
+    }
     if (r_bf16 && keep != 0xFFu) {
         uint4* p = reinterpret_cast<uint4*>(r_bf16 + m * K + k0);
         uint4 v = keep == 0 ? make_uint4(0, 0, 0, 0) : *p;
@@ -840,6 +848,13 @@ __global__ void __launch_bounds__(kThreads) quant_row50_kernel(QuantArgs a) {
                 }
             }
             if (a.mask_bits) a.mask_bits[m * (K / 8) + k0 / 8] = (uint8_t)keep;
+            if (a.r_codes && a.mask_r_codes) {  // written earlier by this CTA (a barrier ago): zero the dropped codes
+                uint32_t nib = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) nib |= ((keep >> i) & 1u) * (0xFu << (4 * i));
+                uint32_t* c = reinterpret_cast<uint32_t*>(a.r_codes + m * (K / 2) + k0 / 2);
+                *c = __ldcg(c) & nib;
+            }
             if (a.r_bf16) {
                 uint32_t w[4];
 #pragma unroll
@@ -961,11 +976,12 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
             topk_select_kernel<<<1, kSelThreads, 0, stream>>>(a.scores, (int)nscore, (int)(nscore / 2), a.keep_flags); }
             rc = cuda_fail(cudaGetLastError(), "topk_select_kernel launch");
             if (rc) return rc;
-            if (a.mask_bits || a.r_bf16) {
+            if (a.mask_bits || a.r_bf16 || (a.r_codes && a.mask_r_codes)) {
                 int64_t n = a.M * (a.K / 8);
                 LaunchScope scope(kKindSelect, stream);
                 apply_global_mask_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(pattern, a.M, a.K, a.keep_flags,
-                                                                                          a.mask_bits, a.r_bf16);
+                                                                                          a.mask_bits, a.r_bf16,
+                                                                                          a.mask_r_codes ? a.r_codes : nullptr);
                 rc = cuda_fail(cudaGetLastError(), "apply_global_mask_kernel launch");
             }
         }
@@ -994,11 +1010,12 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
         topk_select_kernel<<<1, kSelThreads, 0, stream>>>(a.scores, (int)nscore, (int)(nscore / 2), a.keep_flags); }
         rc = cuda_fail(cudaGetLastError(), "topk_select_kernel launch");
         if (rc) return rc;
-        if (a.mask_bits || a.r_bf16) {
+        if (a.mask_bits || a.r_bf16 || (a.r_codes && a.mask_r_codes)) {
             int64_t n = a.M * (a.K / 8);
             LaunchScope scope(kKindSelect, stream);
             apply_global_mask_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(pattern, a.M, a.K, a.keep_flags,
-                                                                                      a.mask_bits, a.r_bf16);
+                                                                                      a.mask_bits, a.r_bf16,
+                                                                                      a.mask_r_codes ? a.r_codes : nullptr);
             rc = cuda_fail(cudaGetLastError(), "apply_global_mask_kernel launch");
         }
     }

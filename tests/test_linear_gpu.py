@@ -185,8 +185,8 @@ def test_every_tile_configuration(tile_case, cfg, pattern, fmt, monkeypatch):
     check_close(y.cpu().numpy(), w["y"], w["abs_sum"])
 
 
-@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_DENSE, oracle.S_2_4])
-@pytest.mark.parametrize("shape", [(300, 512, 600), (128, 256, 256), (1000, 1024, 1300)])
+@pytest.mark.parametrize("pattern", ALL)
+@pytest.mark.parametrize("shape", [(288, 512, 600), (128, 256, 256), (992, 1024, 1300)])
 def test_mxfp4_block_scaled_fp4_gemm(monkeypatch, pattern, shape):
     """MXFP4 on the block-scaled FP4 tensor pipe (packed codes + scales straight into tcgen05.mma kind::mxf4),
     forced on for these small shapes; the same call with the path switched off must agree within tolerance too."""
