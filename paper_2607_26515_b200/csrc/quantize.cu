@@ -594,6 +594,220 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
 }
 
 // ------------------------------------------------------------------------------------------------
+// ROW50 with a warp per row (block-per-lane encoders).  The row is walked in segments of 32 blocks; the signed
+// bf16 image of deq Q(dX) of the whole row stays in the warp's shared memory (same padded block layout as the
+// staging buffers), so that the K/2 largest magnitudes can be selected and the image masked before it leaves.
+// Selection: most significant bit first over the 15 magnitude bits, counting with warp reductions only; ties
+// at the threshold are kept lowest index first.  Shared memory per warp: (3 + segments) staging tiles.
+template <int FMT, bool IMG>
+__global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs a, int warps_per_cta) {
+    pdl_wait();
+    pdl_trigger();
+    if (a.clear_words && blockIdx.x == 0)
+        for (int i = threadIdx.x; i < a.n_clear_words; i += blockDim.x) a.clear_words[i] = 0u;
+    extern __shared__ __align__(16) uint8_t smem_q[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (warp >= warps_per_cta) return;  // warps are independent: no CTA-wide barrier below
+    const int64_t m = (int64_t)blockIdx.x * warps_per_cta + warp;
+    if (m >= a.M) return;
+    const int64_t G = a.K / kHif4Block;
+    const int nseg = (int)((G + 31) / 32);
+    const uint32_t base = smem_u32(smem_q) + (uint32_t)(warp * (3 + nseg) * kStageBytes);
+    const uint32_t in0 = base, stage = base + 2 * kStageBytes, rrow = base + 3 * kStageBytes;
+    const int cp_blk = lane >> 3, cp_ch = lane & 7;
+    const uint32_t cp_smem = (uint32_t)(cp_blk * kStagePitch + cp_ch * 16);
+    const uint32_t my_in = (uint32_t)(lane * kStagePitch);
+    auto seg_col = [&](int seg) -> int64_t { return ((int64_t)seg * 32 + cp_blk) * kHif4Block + cp_ch * 8; };
+    auto issue_seg = [&](int seg, uint32_t buf) {
+        const int64_t col = seg_col(seg);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const bool valid = col + j * 4 * kHif4Block < a.K;
+            cp_async_16(buf + cp_smem + j * 4 * kStagePitch,
+                        valid ? (const void*)(a.X + m * a.ldx + col + j * 4 * kHif4Block) : (const void*)a.X, valid);
+        }
+    };
+    auto drain = [&](uint32_t src, __nv_bfloat16* dst_row, int seg) {
+        const int64_t col = seg_col(seg);
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint4 v = lds_16(src + cp_smem + j * 4 * kStagePitch);
+            if (col + j * 4 * kHif4Block < a.K) *reinterpret_cast<uint4*>(dst_row + col + j * 4 * kHif4Block) = v;
+        }
+        __syncwarp();
+    };
+
+    // ---- phase A: both encodes, segment by segment
+    issue_seg(0, in0);
+    cp_async_commit();
+    if (nseg > 1) issue_seg(1, in0 + kStageBytes);
+    cp_async_commit();
+    for (int seg = 0; seg < nseg; ++seg) {
+        const uint32_t buf = in0 + (uint32_t)((seg & 1) * kStageBytes);
+        cp_async_wait<1>();
+        __syncwarp();
+        uint32_t w[32];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint4 v = lds_16(buf + my_in + c * 16);
+            w[4 * c] = v.x; w[4 * c + 1] = v.y; w[4 * c + 2] = v.z; w[4 * c + 3] = v.w;
+        }
+        __syncwarp();
+        if (seg + 2 < nseg) issue_seg(seg + 2, buf);
+        cp_async_commit();
+        const int64_t blk = (int64_t)seg * 32 + lane;
+        const bool active = blk < G;
+        uint32_t codes[8], side;
+        encode_block<FMT, true, false>(w, codes, side, [&](int c, const float (&x)[8], const float (&dq)[8], uint32_t) {
+            float sd[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sd[i] = copysignf(dq[i], x[i]);
+            if constexpr (IMG)
+                sts_16(stage + my_in + c * 16, make_uint4(pack_bf16x2_exact(sd[0], sd[1]), pack_bf16x2_exact(sd[2], sd[3]),
+                                                          pack_bf16x2_exact(sd[4], sd[5]), pack_bf16x2_exact(sd[6], sd[7])));
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                w[4 * c + i] = pack_bf16x2_exact(__fsub_rn(x[2 * i], sd[2 * i]), __fsub_rn(x[2 * i + 1], sd[2 * i + 1]));
+        });
+        if (active) {
+            if (a.x_codes) {
+                uint4* p = reinterpret_cast<uint4*>(a.x_codes + m * (a.K / 2) + blk * 32);
+                p[0] = make_uint4(codes[0], codes[1], codes[2], codes[3]);
+                p[1] = make_uint4(codes[4], codes[5], codes[6], codes[7]);
+            }
+            if (a.x_side) {
+                if constexpr (FMT == kHiF4) reinterpret_cast<uint32_t*>(a.x_side)[m * G + blk] = side;
+                else *reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(a.x_side) + (m * G + blk) * 2) = (uint16_t)side;
+            }
+        }
+        if constexpr (IMG) drain(stage, a.a_bf16 + m * a.K, seg);
+        uint32_t rcodes[8], rside;
+        const uint32_t rdst = rrow + (uint32_t)(seg * kStageBytes) + my_in;
+        encode_block<FMT, true, false>(w, rcodes, rside, [&](int c, const float (&)[8], const float (&rdq)[8], uint32_t) {
+            uint32_t img[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                img[i] = active ? (pack_bf16x2_exact(rdq[2 * i], rdq[2 * i + 1]) | (w[4 * c + i] & 0x80008000u)) : 0u;
+            sts_16(rdst + c * 16, make_uint4(img[0], img[1], img[2], img[3]));
+        });
+        if (active) {
+            if (a.r_codes) {
+                uint4* p = reinterpret_cast<uint4*>(a.r_codes + m * (a.K / 2) + blk * 32);
+                p[0] = make_uint4(rcodes[0], rcodes[1], rcodes[2], rcodes[3]);
+                p[1] = make_uint4(rcodes[4], rcodes[5], rcodes[6], rcodes[7]);
+            }
+            if (a.r_side) {
+                if constexpr (FMT == kHiF4) reinterpret_cast<uint32_t*>(a.r_side)[m * G + blk] = rside;
+                else *reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(a.r_side) + (m * G + blk) * 2) = (uint16_t)rside;
+            }
+        }
+    }
+    cp_async_wait<0>();
+    __syncwarp();
+
+    // ---- phase B: the (K/2)-th largest 15-bit magnitude of the row (inactive blocks hold zeros: they never win)
+    unsigned prefix = 0u;
+    int remaining = (int)(a.K / 2);
+    for (int b = 14; b >= 0; --b) {
+        const unsigned cand = prefix | (1u << b);
+        const uint32_t cand2 = (cand >> b) * 0x00010001u;
+        const uint32_t mask2 = (0x7FFFu >> b) * 0x00010001u;
+        int cnt = 0;
+        for (int seg = 0; seg < nseg; ++seg) {
+            const uint32_t src = rrow + (uint32_t)(seg * kStageBytes) + my_in;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint4 v = lds_16(src + c * 16);
+                const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t z = (((w4[i] & 0x7FFF7FFFu) >> b) & mask2) ^ cand2;
+                    cnt += ((z & 0xFFFFu) == 0u) + ((z >> 16) == 0u);
+                }
+            }
+        }
+        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+        if (cnt >= remaining) prefix = cand;
+        else remaining -= cnt;
+    }
+    const uint32_t T = prefix;   // threshold magnitude
+    int need = remaining;        // entries equal to T that are kept, lowest index first
+
+    // ---- phase C: masks in index order (segment, lane, position), masked image, masked codes
+    for (int seg = 0; seg < nseg; ++seg) {
+        const int64_t blk = (int64_t)seg * 32 + lane;
+        const bool active = blk < G;
+        const uint32_t src = rrow + (uint32_t)(seg * kStageBytes) + my_in;
+        uint32_t wv[32];
+        uint32_t gt[2] = {0u, 0u}, eq[2] = {0u, 0u};  // bit per element of the lane's block (low / high 32)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint4 v = lds_16(src + c * 16);
+            wv[4 * c] = v.x; wv[4 * c + 1] = v.y; wv[4 * c + 2] = v.z; wv[4 * c + 3] = v.w;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t klo = wv[4 * c + i] & 0x7FFFu, khi = (wv[4 * c + i] >> 16) & 0x7FFFu;
+                const int e = 8 * c + 2 * i;
+                gt[e >> 5] |= (uint32_t)(klo > T) << (e & 31);
+                gt[(e + 1) >> 5] |= (uint32_t)(khi > T) << ((e + 1) & 31);
+                eq[e >> 5] |= (uint32_t)(klo == T) << (e & 31);
+                eq[(e + 1) >> 5] |= (uint32_t)(khi == T) << ((e + 1) & 31);
+            }
+        }
+        if (!active) eq[0] = eq[1] = gt[0] = gt[1] = 0u;
+        const int mine = __popc(eq[0]) + __popc(eq[1]);
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        int quota = max(0, min(mine, need - (incl - mine)));  // how many of this lane's ties are kept
+        need = max(0, need - total);
+        uint32_t keep[2] = {gt[0], gt[1]};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t e = eq[h];
+            while (e && quota > 0) {  // lowest set bits first
+                const uint32_t low = e & (0u - e);
+                keep[h] |= low;
+                e ^= low;
+                --quota;
+            }
+        }
+        if (active) {
+            if (a.mask_bits) *reinterpret_cast<uint2*>(a.mask_bits + m * (a.K / 8) + blk * 8) = make_uint2(keep[0], keep[1]);
+            if (a.r_codes && a.mask_r_codes) {
+                uint4* p = reinterpret_cast<uint4*>(a.r_codes + m * (a.K / 2) + blk * 32);
+                uint4 c0 = __ldcg(p), c1 = __ldcg(p + 1);
+                uint32_t cw[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t k8 = (keep[c >> 2] >> (8 * (c & 3))) & 0xFFu;
+                    uint32_t nib = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) nib |= ((k8 >> i) & 1u) * (0xFu << (4 * i));
+                    cw[c] &= nib;
+                }
+                p[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+                p[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
+            }
+        }
+        if constexpr (IMG) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                uint32_t km[4];
+                keep_words((keep[c >> 2] >> (8 * (c & 3))) & 0xFFu, km);
+                sts_16(src + c * 16, make_uint4(wv[4 * c] & km[0], wv[4 * c + 1] & km[1], wv[4 * c + 2] & km[2], wv[4 * c + 3] & km[3]));
+            }
+            drain(rrow + (uint32_t)(seg * kStageBytes), a.r_bf16 + m * a.K, seg);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Exact top-`keep` of n non-negative fp64 scores, ties to the lower index.  One CTA: MSB-first radix
 // select over the 64-bit patterns (8 passes of 8 bits), then an index-ordered pass that admits the
 // first `need` entries equal to the threshold.
@@ -923,6 +1137,25 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     const int pattern = a.pattern;
     const bool residual = pattern != RESQ_S_NONE;
     if (pattern == RESQ_S_ROW50) {
+        // a warp per row with the block-per-lane encoders, if the row's image fits next to the staging tiles
+        auto al16r = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
+        const int nseg = (int)((a.K / kHif4Block + 31) / 32);
+        const int per_warp = (3 + nseg) * kStageBytes;
+        const int wpc = std::min(kWarpsPerCta, (220 * 1024) / per_warp);
+        // (measured: wins for rows of up to two segments; longer rows keep a whole CTA busy better)
+        if (a.K % kHif4Block == 0 && nseg <= 2 && wpc >= 1 && a.M >= 148 && al16r(a.x_codes) && al16r(a.r_codes) && al16r(a.mask_bits) &&
+            al16r(a.a_bf16) && al16r(a.r_bf16)) {
+            const bool img = a.a_bf16 != nullptr;
+            void (*kern)(QuantArgs, int) =
+                fmt == kHiF4 ? (img ? quant_row50_warp_kernel<kHiF4, true> : quant_row50_warp_kernel<kHiF4, false>)
+                             : (img ? quant_row50_warp_kernel<kMXFP4, true> : quant_row50_warp_kernel<kMXFP4, false>);
+            const int smem_w = wpc * per_warp;
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_w);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(row50 warp)");
+            LaunchScope scope(kKindQuant, stream);
+            return cuda_fail(launch_kernel(kern, dim3((unsigned)((a.M + wpc - 1) / wpc)), dim3(kThreads), (size_t)smem_w, stream, a, wpc),
+                             "quant_row50_warp_kernel launch");
+        }
         size_t smem = (size_t)a.K * sizeof(uint16_t);
         if (smem > 200 * 1024) {
             set_last_error("ROW50 supports K <= %d", 200 * 1024 / 2);

@@ -69,7 +69,7 @@ PATTERNS = [oracle.S_NONE, oracle.S_DENSE, oracle.S_2_4, oracle.S_ROW50, oracle.
 
 @pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
 @pytest.mark.parametrize("pattern", PATTERNS)
-@pytest.mark.parametrize("shape", [(32, 64), (64, 2048), (96, 3584), (256, 11008)])
+@pytest.mark.parametrize("shape", [(32, 64), (64, 2048), (96, 3584), (256, 11008), (320, 2048), (160, 4096 - 64)])
 def test_residual_mask_bit_exact(fmt, pattern, shape):
     M, K = shape
     # the 2^-70 / 2^20 blocks would make the fp64 score sums inexact: leave them out for the global patterns
