@@ -1,6 +1,7 @@
 // C ABI of the ResQ library: argument checks, workspace carving, kernel sequencing.
 // The contract of every entry point is stated in include/resq.h.
 #include "common.cuh"
+#include <algorithm>
 
 #include <atomic>
 #include <cstdarg>
@@ -186,11 +187,21 @@ int residual_mask(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, int
     return launch_quantize(fmt, a, st);
 }
 
+// Residual operand region: the bf16 image of S(deq Q(dX)), or (2:4 on the sparse MMA) the compressed image [M, K/2]
+// followed by the index metadata; sized for either.
+size_t sparse24_meta_bytes(int64_t M, int64_t K) { return (size_t)sparse24_rows128(M) * (size_t)sparse24_ka(K) * 2048; }
+size_t residual_region_bytes(int64_t M, int64_t K, int pattern) {
+    if (pattern == RESQ_S_NONE) return 0;
+    size_t b = (size_t)M * (size_t)K * 2;
+    if (pattern == RESQ_S_2_4) b = std::max(b, align_up((size_t)M * (size_t)K, 256) + sparse24_meta_bytes(M, K));
+    return align_up(b, 256);
+}
+
 size_t linear_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K, int pattern) {
     if (M <= 0 || N <= 0 || K <= 0) return 0;
     size_t b = kWsHeader + kWsFlags + quant_scratch_bytes(M, K, pattern);
     b += align_up((size_t)M * (size_t)K * 2, 256);                            // bf16 image of deq Q(X)
-    if (pattern != RESQ_S_NONE) b += align_up((size_t)M * (size_t)K * 2, 256);  // bf16 image of S(deq Q(dX))
+    b += residual_region_bytes(M, K, pattern);
     b += align_up(gemm_hif4_scratch_bytes(M, N, K), 256);                     // fp32 partial tiles of a K split
     return b;
 }
@@ -243,8 +254,10 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     uint8_t* region_r = nullptr;
     if (pattern != RESQ_S_NONE) {
         region_r = ws + used;
-        used += align_up((size_t)M * (size_t)K * 2, 256);
+        used += residual_region_bytes(M, K, pattern);
     }
+    // 2:4 on the CTA-pair kernel: the residual goes to the structured-sparse MMA in compressed form
+    const bool sparse24 = !native && pattern == RESQ_S_2_4 && gemm_sparse24_supported(M, N, K);
     const size_t codes_bytes = align_up((size_t)M * (size_t)K / 2, 256);
     if (native) {
         a.x_codes = region_a;
@@ -254,6 +267,12 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
             a.r_side = region_r + codes_bytes;
             a.mask_r_codes = 1;
         }
+    } else if (sparse24) {
+        a.a_bf16 = reinterpret_cast<__nv_bfloat16*>(region_a);
+        a.r_comp = reinterpret_cast<__nv_bfloat16*>(region_r);
+        a.r_meta = region_r + align_up((size_t)M * (size_t)K, 256);
+        a.meta_rows128 = sparse24_rows128(M);
+        a.meta_ka = sparse24_ka(K);
     } else {
         a.a_bf16 = reinterpret_cast<__nv_bfloat16*>(region_a);
         a.r_bf16 = reinterpret_cast<__nv_bfloat16*>(region_r);
@@ -283,6 +302,10 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     g.fmt = fmt;
     g.a_bf16 = a.a_bf16;
     g.r_bf16 = a.r_bf16;
+    g.r_comp = a.r_comp;
+    g.r_meta = a.r_meta;
+    g.meta_rows128 = a.meta_rows128;
+    g.meta_ka = a.meta_ka;
     g.w_codes = static_cast<const uint8_t*>(w_codes);
     g.w_side = w_side;
     g.M = M;

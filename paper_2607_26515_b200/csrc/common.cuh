@@ -86,6 +86,10 @@ struct QuantArgs {
     // expanded operands for the GEMM (any may be null): exact bf16 images of deq Q(X) and S(deq Q(dX))
     __nv_bfloat16* a_bf16;  // [M, K]
     __nv_bfloat16* r_bf16;  // [M, K]
+    // pattern 2:4 only, instead of r_bf16: the compressed image and its index metadata (see GemmArgs)
+    __nv_bfloat16* r_comp;  // [M, K/2]
+    uint8_t* r_meta;
+    int64_t meta_rows128, meta_ka;
     // scratch
     double* scores;         // CHAN50: [K]; BLOCK: [(M/32) * (K/64)]
     uint8_t* keep_flags;    // CHAN50: [K]; BLOCK: [(M/32) * (K/64)]
@@ -104,7 +108,11 @@ size_t quant_scratch_bytes(int64_t M, int64_t K, int pattern);  // scores + keep
 struct GemmArgs {
     int fmt;                       // kHiF4 or kMXFP4: how w_codes / w_side are decoded
     const __nv_bfloat16* a_bf16;   // [M, K] exact bf16 image of deq Q(X)
-    const __nv_bfloat16* r_bf16;   // [M, K] masked residual image, or null (pattern NONE)
+    const __nv_bfloat16* r_bf16;   // [M, K] masked residual image, or null (pattern NONE, or r_comp given)
+    // 2:4 residual in compressed form for the structured-sparse MMA (CTA-pair kernel only), instead of r_bf16:
+    const __nv_bfloat16* r_comp;   // [M, K/2] the two kept values of every four consecutive channels, in channel order
+    const uint8_t* r_meta;         // index metadata, sparse24_meta_offset() layout: meta_rows128 x meta_ka blocks of 2 KB
+    int64_t meta_rows128, meta_ka;
     const uint8_t* w_codes;        // [N, K/2]
     const void* w_side;            // [N, K/64] u32 or [N, K/32] u8
     int64_t M, N, K;
@@ -119,6 +127,18 @@ struct GemmArgs {
     DeviceStatus* status;
 };
 int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream);
+// Whether launch_gemm_hif4 takes the compressed 2:4 residual for this shape (the CTA-pair kernel runs it).
+bool gemm_sparse24_supported(int64_t M, int64_t N, int64_t K);
+// Layout of the 2:4 index metadata, fixed by the sparse MMA: blocks of 128 rows x 128 K positions (2 KB, row bands
+// outermost); inside a block, rows of 16 bytes: byte 16 * (m % 8 + 8 * ((k / 16) % 2) + 16 * (m / 16)) + 4 * (k / 32)
+// + 2 * ((m / 8) % 2) + (k / 8) % 2 holds the two 4-bit index pairs (idx0 | idx1 << 2, lower channels in the low
+// nibble) of channels k .. k + 7 of row m (m, k relative to the block).
+__host__ __device__ inline int64_t sparse24_meta_offset(int64_t m, int64_t k, int64_t ka) {
+    return ((m >> 7) * ka + (k >> 7)) * 2048 + ((m >> 4) & 7) * 256 + ((k >> 4) & 1) * 128 + (m & 7) * 16 + ((k >> 5) & 3) * 4 +
+           ((m >> 3) & 1) * 2 + ((k >> 3) & 1);
+}
+inline int64_t sparse24_rows128(int64_t M) { return (M + 255) / 256 * 2; }  // whole 256-row tiles of the pair kernel
+inline int64_t sparse24_ka(int64_t K) { return (K + 127) / 128; }
 
 // MXFP4 on the block-scaled FP4 tensor pipe (gemm_mxfp4.cu): operands stay packed E2M1 codes + E8M0 scales.
 struct Mxfp4NativeArgs {

@@ -532,7 +532,7 @@ int env_int(const char* name, int dflt) {
 }
 
 // Pick the tile width and K split so that the persistent grid covers the 148 SMs evenly.
-TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res) {
+TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res, bool sparse = false) {
     const int sms = 148;
     const int G = (int)(K / kBK);
     TileChoice best{1, 256, 1, 1, 0};
@@ -576,14 +576,16 @@ TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res) {
     if (M > kBM && env_int("RESQ_GEMM_PAIR", 1)) {
         const int64_t mtiles = (M + 2 * kBM - 1) / (2 * kBM);
         double best_pair = 1e300;
-        for (int tn : {512, 384, 320, 256, 128}) {
+        for (int tn : {512, 480, 384, 320, 256, 128}) {
+            // the sparse metadata needs a few tensor-memory columns: 480 instead of 512
+            if (sparse ? tn == 512 : tn == 480) continue;
             const int64_t ntiles = (N + tn - 1) / tn;
             for (int splits = 1; splits <= 8; splits *= 2) {
                 if (G / splits < 4 && splits > 1) break;
                 const int64_t tiles = mtiles * ntiles * splits;
                 const int64_t rounds = (tiles + sms / 2 - 1) / (sms / 2);
                 const int kb = (G + splits - 1) / splits;
-                const double mma = tn / 256.0 * (res ? 1024.0 : 512.0);
+                const double mma = tn / 256.0 * (sparse ? 768.0 : res ? 1024.0 : 512.0);
                 const double per_kb = std::max(mma, 1500.0) + 350.0;
                 double cost = rounds * (kb * per_kb + 8000.0);
                 if (splits > 1) cost += 15000.0 + (double)splits * M * N * 4.0 / 1200.0;  // partial tiles: ~1.6 KB/clk
@@ -699,6 +701,17 @@ bool gemm_use_streamk(int64_t M, int64_t N, int64_t K) {
     return tiles <= 74 / 2 && tiles * (K / kBK) >= 2;  // at least two pairs per tile: otherwise whole tiles per pair
 }
 
+// The 2:4 residual on the structured-sparse MMA is complete and tested but not the default: it halves the tensor
+// work of the residual term and shrinks its operand from 16 KB to 9 KB per k-block, yet the pair kernel is bound
+// by weight expansion and by shared-memory ingest rather than by tensor issue, the 512-wide tile has no
+// tensor-memory columns left for the metadata, and the quantizer pays for the compression.  Measured (M = 8192,
+// K = 2048): N = 22016 in 955 us instead of 1011 us, but N = 2048 in 150 us instead of 124 us (tile count); the
+// decode shapes lose 4 %.  RESQ_SPARSE24=1 switches it on.
+bool gemm_sparse24_supported(int64_t M, int64_t N, int64_t K) {
+    (void)N;
+    return M > kBM && K % kBK == 0 && env_int("RESQ_GEMM_PAIR", 1) && env_int("RESQ_SPARSE24", 0);
+}
+
 size_t gemm_hif4_scratch_bytes(int64_t M, int64_t N, int64_t K) {
     size_t classic = 0;
     const int splits = gemm_hif4_pick_splits(M, N, K);
@@ -710,7 +723,8 @@ size_t gemm_hif4_scratch_bytes(int64_t M, int64_t N, int64_t K) {
 
 int gemm_hif4_pick_splits(int64_t M, int64_t N, int64_t K) {
     // the workspace must cover the larger of the two possible choices (with / without residual)
-    return std::max(choose_tile(M, N, K, false).splits, choose_tile(M, N, K, true).splits);
+    return std::max(std::max(choose_tile(M, N, K, false).splits, choose_tile(M, N, K, true).splits),
+                    choose_tile(M, N, K, true, true).splits);
 }
 
 template <int MT, bool RES, int FMT>
@@ -727,15 +741,21 @@ int dispatch_tn(const GemmArgs& g, const TileChoice& tc, cudaStream_t stream) {
 }
 
 int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream) {
-    const bool res = g.r_bf16 != nullptr;
+    const bool res = g.r_bf16 != nullptr || g.r_comp != nullptr;
+    if (g.r_comp && !gemm_sparse24_supported(g.M, g.N, g.K)) {
+        set_last_error("internal: compressed residual given for a shape the pair kernel does not run");
+        return RESQ_ERR_CUDA;
+    }
     if (gemm_use_streamk(g.M, g.N, g.K) && g.splitk_partials && g.sk_flags &&
         g.partial_bytes >= gemm_pair_streamk_scratch_bytes())
         return launch_gemm_pair_streamk(g, stream);
-    TileChoice tc = choose_tile(g.M, g.N, g.K, res);
+    TileChoice tc = choose_tile(g.M, g.N, g.K, res, g.r_comp != nullptr);
     if (tc.splits > 1 && (!g.splitk_partials || tc.splits > g.splits)) tc.splits = 1;
     if (env_int("RESQ_GEMM_DEBUG", 0) & 1)
         fprintf(stderr, "resq gemm M=%lld N=%lld K=%lld res=%d: pair_tn=%d mt=%d bn=%d nt=%d splits=%d\n", (long long)g.M,
                 (long long)g.N, (long long)g.K, (int)res, tc.pair_tn, tc.mt, tc.bn, tc.nt, tc.splits);
+    if (g.r_comp && tc.pair_tn == 512) tc.pair_tn = 480;  // (a forced width) no tensor-memory columns left for the metadata
+    if (!g.r_comp && tc.pair_tn == 480) tc.pair_tn = 512;
     if (tc.pair_tn > 0) return launch_gemm_pair(g, tc.pair_tn, tc.splits, stream);
     if (g.fmt == kMXFP4) {
         if (res) return dispatch_tn<1, true, kMXFP4>(g, tc, stream);

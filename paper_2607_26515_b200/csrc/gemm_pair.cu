@@ -30,8 +30,9 @@ constexpr int kBM = 128;
 constexpr int kBK = 64;
 constexpr int kMaxBN = 256;
 constexpr int kGroupWarps = 4;                       // expander warps per group
-// Expander groups take k-blocks round-robin; group g owns slot g of all three rings (activation stages, raw
-// codes, expanded weights: SA == SE == SR == NG).  The number of groups NG (four warps each) is a template
+// Expander groups take k-blocks round-robin; k-block it uses slot it mod depth of each of the three rings
+// (activation stages, raw codes, expanded weights; the depths are at least NG, see launch_pair_variant).  The
+// number of groups NG (four warps each) is a template
 // parameter of the kernel: more groups tolerate more hand-off latency, fewer groups fit wider tiles into
 // shared memory (three slots of a 512-wide tile with a residual operand take 216 KB).
 constexpr int kFirstEpiWarp = 4;
@@ -48,6 +49,7 @@ struct PairParams {
     int kblocks_per_split, splits;
     int ntiles_m, ntiles_n, num_tiles;
     int sa, sr, se, acc_bufs;
+    int meta_ka;             // sparse residual: metadata blocks (128 K positions) per 128-row band
     void* Y;
     int out_f32;
     int64_t ldy;
@@ -237,13 +239,23 @@ __device__ __forceinline__ void streamk_fixup(const PairParams& p, int pair, int
     }
 }
 
+// Residual term of the kernel: none, a dense second A operand (the masked bf16 image), or the 2:4 compressed image
+// with its index metadata on the structured-sparse MMA (half the tensor work of the dense form).
+enum ResMode : int { kResNone = 0, kResDense = 1, kResSparse24 = 2 };
+constexpr int kSpTileBytes = kATileBytes / 2;  // compressed residual tile: 128 rows x 32 kept values (64-byte rows)
+constexpr int kSpMetaBytes = 2048;             // index metadata of 128 rows x 128 K positions (two k-blocks)
+constexpr int kSpTmemCol = kTmemCols - 8;      // two metadata buffers of four columns at the end of tensor memory
+__host__ __device__ constexpr int a_stage_bytes(int res) {
+    return res == kResDense ? 2 * kATileBytes : res == kResSparse24 ? kATileBytes + kSpTileBytes + kSpMetaBytes : kATileBytes;
+}
+
 // TN: width of the pair's output tile (the pair computes 256 x TN); bn = MMA N; each CTA expands TN/2 rows.
-template <bool RES, int TN, int FMT, int NG>
+template <int RES, int TN, int FMT, int NG>
 __global__ void __launch_bounds__(pair_threads(NG), 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_r,
-                 const __grid_constant__ CUtensorMap tmap_w, const PairParams p) {
+                 const __grid_constant__ CUtensorMap tmap_e, const __grid_constant__ CUtensorMap tmap_w, const PairParams p) {
     constexpr int kExpGroups = NG;
-    constexpr int kAStage = kATileBytes * (RES ? 2 : 1);
+    constexpr int kAStage = a_stage_bytes(RES);
     constexpr int nt = TN > kMaxBN ? 2 : 1;           // MMAs side by side in N
     constexpr int bn = TN / nt;                    // MMA N
     constexpr int half = bn / 2;                   // rows of each MMA's weight tile held by one CTA
@@ -315,7 +327,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         // ------------------------------------------------------------------ activation producer (both CTAs)
         if (lane == 0) {
             ptx::tma_prefetch_desc(&tmap_a);
-            if (RES) ptx::tma_prefetch_desc(&tmap_r);
+            if (RES != kResNone) ptx::tma_prefetch_desc(&tmap_r);
+            if (RES == kResSparse24) ptx::tma_prefetch_desc(&tmap_e);
             uint32_t it = 0;
             bool ok = true;
             SegIter<TN> si(p, pair, npairs);
@@ -323,9 +336,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             while (ok && si.next(tc)) {
                 const int my_m = (int)(tc.m0 + rank * kBM);
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
-                    const int s = it % SA;
+                    // The activation ring may be shallower than the ring of expanded weights whose barriers it shares
+                    // (barrier slot = k-block mod SE): slot it % SA is free once the MMAs of k-block it - SA, which
+                    // signal barrier (it - SA) % SE, completed.  (That barrier cannot run a phase ahead: its next
+                    // phase needs the k-block it - SA + SE >= it, which this thread has not loaded yet.)
+                    const int s = it % SA, sb = it % SE;
                     tr.begin();
-                    const bool got = ptx::mbar_wait_spin(&a_empty[s], ((it / SA) & 1) ^ 1, abort_flag);
+                    const uint32_t prev = it - (uint32_t)SA;
+                    const bool got = it < (uint32_t)SA || ptx::mbar_wait_spin(&a_empty[prev % SE], (prev / SE) & 1, abort_flag);
                     tr.end(0);
                     if (!got) {
                         report_timeout(p.status, 1);
@@ -335,11 +353,21 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     uint8_t* st = ring_a + (size_t)s * kAStage;
                     TLOG(0, it);
                     if (it == 0) EVT(1);
-                    const uint32_t full = ptx::map_to_cta(&a_full[s], 0);
-                    ptx::mbar_arrive_expect_tx_cluster_relaxed(full, (uint32_t)kAStage);  // publishes nothing itself
-                    const int kx = (tc.kb_begin + i) * kBK;
+                    const uint32_t full = ptx::map_to_cta(&a_full[sb], 0);
+                    const int kb = tc.kb_begin + i;
+                    // the metadata of two k-blocks travels with the even one (or with the first of a K range)
+                    const bool with_meta = RES == kResSparse24 && ((kb & 1) == 0 || i == 0);
+                    ptx::mbar_arrive_expect_tx_cluster_relaxed(  // publishes nothing itself
+                        full, (uint32_t)(kAStage - (RES == kResSparse24 && !with_meta ? kSpMetaBytes : 0)));
+                    const int kx = kb * kBK;
                     ptx::tma_load_2d_pair(st, &tmap_a, full, kx, my_m);
-                    if (RES) ptx::tma_load_2d_pair(st + kATileBytes, &tmap_r, full, kx, my_m);
+                    if (RES == kResDense) ptx::tma_load_2d_pair(st + kATileBytes, &tmap_r, full, kx, my_m);
+                    if (RES == kResSparse24) {
+                        ptx::tma_load_2d_pair(st + kATileBytes, &tmap_r, full, kx / 2, my_m);
+                        if (with_meta)  // rows of 256 bytes, eight per 128 x 128 block
+                            ptx::tma_load_2d_pair(st + kATileBytes + kSpTileBytes, &tmap_e, full, 0,
+                                                  ((my_m >> 7) * p.meta_ka + (kb >> 1)) * 8);
+                    }
                 }
             }
         }
@@ -376,8 +404,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         if (lane == 0 && rank == 0) {
             const uint32_t idesc = ptx::idesc_bf16_f32(2 * kBM, bn);
             const uint64_t desc0 = ptx::smem_desc_sw128_kmajor(0);  // everything but the start address
+            const uint64_t desc0_sp = ptx::smem_desc_sw64_kmajor(0);
+            const uint64_t desc0_e = ptx::smem_desc_rows16(0);
+            uint32_t ebuf = 0;  // metadata buffer (four tensor-memory columns) in use
             const uint32_t a_base16 = (ptx::smem_u32(ring_a) & 0x3FFFFu) >> 4, e_base16 = (ptx::smem_u32(ring_e) & 0x3FFFFu) >> 4;
-            uint32_t it = 0, sa = 0, pha = 0;  // ring slot and phase parity of this k-block
+            uint32_t it = 0, sa = 0, se = 0, pha = 0;  // activation slot, barrier / weight slot and its phase parity
             int local_tile = 0;
             bool ok = true;
             SegIter<TN> si(p, pair, npairs);
@@ -400,7 +431,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     // This thread's instruction stream sits between the MMAs of consecutive k-blocks: stage
                     // indices, phases and descriptors advance by additions only.
                     tr.begin();
-                    ok = ptx::mbar_wait_spin(&a_full[sa], pha, abort_flag);
+                    ok = ptx::mbar_wait_spin(&a_full[se], pha, abort_flag);
                     tr.end(2);
                     if (!ok) {
                         report_timeout(p.status, 2);
@@ -410,8 +441,19 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     TLOG(2, it);
                     if (it == 0) EVT(2);
                     ptx::tc_fence_after();
-                    const uint64_t adesc = desc0 + (uint64_t)(a_base16 + sa * (uint32_t)(kAStage >> 4));
-                    const uint64_t bdesc = desc0 + (uint64_t)(e_base16 + sa * (uint32_t)(exp_stage >> 4));
+                    const uint32_t a16 = a_base16 + sa * (uint32_t)(kAStage >> 4);
+                    const uint64_t adesc = desc0 + (uint64_t)a16;
+                    const uint64_t bdesc = desc0 + (uint64_t)(e_base16 + se * (uint32_t)(exp_stage >> 4));
+                    uint32_t e_col = 0;
+                    if (RES == kResSparse24) {
+                        const int kb = tc.kb_begin + i;
+                        if ((kb & 1) == 0 || i == 0) {
+                            ebuf ^= 1u;
+                            ptx::tmem_cp_128x128b_pair(tmem_base + (uint32_t)kSpTmemCol + 4u * ebuf,
+                                                       desc0_e + (uint64_t)(a16 + (uint32_t)((kATileBytes + kSpTileBytes) >> 4)));
+                        }
+                        e_col = tmem_base + (uint32_t)kSpTmemCol + 4u * ebuf + 2u * (uint32_t)(kb & 1);
+                    }
 #pragma unroll
                     for (int k = 0; k < kBK / 16; ++k) {
 #pragma unroll
@@ -419,11 +461,20 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                             const uint64_t bd = bdesc + (uint64_t)((j * half * 128 + k * 32) >> 4);
                             const uint32_t d = d0 + (uint32_t)(j * bn);
                             ptx::umma_bf16_pair(d, adesc + (uint64_t)((k * 32) >> 4), bd, idesc, (i > 0 || k > 0) ? 1u : 0u);
-                            if (RES) ptx::umma_bf16_pair(d, adesc + (uint64_t)((kATileBytes + k * 32) >> 4), bd, idesc, 1u);
+                            if (RES == kResDense)
+                                ptx::umma_bf16_pair(d, adesc + (uint64_t)((kATileBytes + k * 32) >> 4), bd, idesc, 1u);
+                            if (RES == kResSparse24 && (k & 1)) {
+                                // 32 K positions per instruction: 32 bytes of the compressed rows, 64 bytes of the weight rows
+                                const int k2 = k >> 1;
+                                ptx::umma_bf16_sp_pair(d, desc0_sp + (uint64_t)(a16 + (uint32_t)((kATileBytes + k2 * 32) >> 4)),
+                                                       bdesc + (uint64_t)((j * half * 128 + k2 * 64) >> 4), e_col,
+                                                       ptx::sparse_idesc(idesc, (uint32_t)k2), 1u);
+                            }
                         }
                     }
-                    ptx::umma_commit_pair(&a_empty[sa], 3);  // frees the slot in both CTAs
-                    if (++sa == (uint32_t)SA) { sa = 0; pha ^= 1u; }
+                    ptx::umma_commit_pair(&a_empty[se], 3);  // frees the slots in both CTAs
+                    if (++sa == (uint32_t)SA) sa = 0;
+                    if (++se == (uint32_t)SE) { se = 0; pha ^= 1u; }
                     TLOG(3, it);
                     tr.end(5);
                 }
@@ -639,25 +690,37 @@ int env_int(const char* name, int dflt) {
 constexpr int kStreamKTN = 256;    // tile width of the K-streamed schedule (two accumulators fit in tensor memory)
 constexpr int kStreamKMaxPairs = 74;
 
-template <bool RES, int TN, int FMT, int NG>
+template <int RES, int TN, int FMT, int NG>
 int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool streamk = false) {
     constexpr int kExpGroups = NG;
-    constexpr int kAStage = kATileBytes * (RES ? 2 : 1);
+    constexpr int kAStage = a_stage_bytes(RES);
     constexpr int nt = TN > kMaxBN ? 2 : 1;
     constexpr int bn = TN / nt;
     constexpr int half = bn / 2;
     constexpr int my_rows = nt * half;
-    CUtensorMap ta, tr, tw;
+    CUtensorMap ta, tr, te, tw;
     int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.a_bf16, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)(g.lda ? g.lda : g.K) * 2,
                           kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
-    rc = make_tmap_2d(&tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, RES ? g.r_bf16 : g.a_bf16, (uint64_t)g.K, (uint64_t)g.M,
-                      (uint64_t)(g.lda ? g.lda : g.K) * 2, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (RES == kResSparse24) {
+        // compressed residual image [M, K/2] in boxes of 32 values x 128 rows (64-byte rows, 64-byte swizzle) and its
+        // metadata blocks (2 KB per 128 rows x 128 K positions) as rows of 256 bytes
+        rc = make_tmap_2d(&tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.r_comp, (uint64_t)g.K / 2, (uint64_t)g.M, (uint64_t)g.K,
+                          kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_64B);
+        if (rc) return rc;
+        rc = make_tmap_2d(&te, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.r_meta, 256, (uint64_t)g.meta_rows128 * (uint64_t)g.meta_ka * 8, 256,
+                          256, 8, CU_TENSOR_MAP_SWIZZLE_NONE);
+    } else {
+        rc = make_tmap_2d(&tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, RES == kResDense ? g.r_bf16 : g.a_bf16, (uint64_t)g.K, (uint64_t)g.M,
+                          (uint64_t)(g.lda ? g.lda : g.K) * 2, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+        te = ta;
+    }
     if (rc) return rc;
     rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.w_codes, (uint64_t)g.K / 2, (uint64_t)g.N, (uint64_t)g.K / 2,
                       kBK / 2, (uint32_t)half, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc) return rc;
     PairParams p;
+    p.meta_ka = g.meta_ka;
     p.w_side = g.w_side;
     p.M = g.M;
     p.N = g.N;
@@ -668,25 +731,14 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
     p.ntiles_m = (int)((g.M + 2 * kBM - 1) / (2 * kBM));
     p.ntiles_n = (int)((g.N + TN - 1) / TN);
     p.num_tiles = p.ntiles_m * p.ntiles_n * splits;
-    p.acc_bufs = TN * 2 <= kTmemCols ? 2 : 1;
+    p.acc_bufs = TN * 2 <= (RES == kResSparse24 ? kSpTmemCol : kTmemCols) ? 2 : 1;
+    if (RES == kResSparse24 && TN > kSpTmemCol) {
+        set_last_error("internal: no tensor-memory columns left for the sparse metadata (pair tile %d)", TN);
+        return RESQ_ERR_CUDA;
+    }
     p.streamk = streamk ? 1 : 0;
     p.sk_slots = g.splitk_partials;
     p.sk_flags = g.sk_flags;
-    constexpr int exp_stage = my_rows * 128, raw_stage = my_rows * 32;
-    const int fixed = 1024 + 1024;
-    // Ring slots: a multiple of the number of expander groups (group g works on the slots s = g mod NG, so a slot
-    // is only ever written by one group).  With one slot per group the group's expansion of a k-block and the
-    // MMAs that read its previous k-block alternate; with two slots per group they overlap.  All three rings have
-    // the same depth (they share the slot's full / empty barriers).
-    const int slot_bytes = kAStage + exp_stage + raw_stage;
-    int per_group = (fixed + 2 * kExpGroups * slot_bytes <= kSmemBudget) ? 2 : 1;
-    per_group = std::max(1, std::min(per_group, env_int("RESQ_GEMM_SLOTS_PER_GROUP", 2)));
-    p.se = p.sr = p.sa = kExpGroups * per_group;
-    if (p.sa > kMaxRing || fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage > kSmemBudget) {
-        set_last_error("internal: shared-memory rings do not fit (pair tile %d)", TN);
-        return RESQ_ERR_CUDA;
-    }
-    const int smem_bytes = fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage;
     p.Y = g.Y;
     p.out_f32 = g.out_dtype == RESQ_OUT_F32;
     p.ldy = g.ldy;
@@ -732,6 +784,38 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
             npairs = p.num_tiles * per_tile;
         }
     }
+    constexpr int exp_stage = my_rows * 128, raw_stage = my_rows * 32;
+    const int fixed = 1024 + 1024;
+    // Ring slots: a multiple of the number of expander groups (group g works on the slots s = g mod NG, so a slot
+    // is only ever written by one group).  With one slot per group the group's expansion of a k-block and the
+    // MMAs that read its previous k-block alternate; with two slots per group they overlap.  All three rings have
+    // the same depth (they share the slot's full / empty barriers).
+    const int slot_bytes = kAStage + exp_stage + raw_stage;
+    int per_group = (fixed + 2 * kExpGroups * slot_bytes <= kSmemBudget) ? 2 : 1;
+    per_group = std::max(1, std::min(per_group, env_int("RESQ_GEMM_SLOTS_PER_GROUP", 2)));
+    p.se = p.sr = p.sa = kExpGroups * per_group;
+    // If two full slots per group do not fit, two expanded-weight slots per group with shallower activation and
+    // raw-code rings may: what matters is that a group can expand its next k-block while the MMAs still read
+    // its previous one.
+    // (Not for a handful of k-blocks per pair: the deeper ring only pays once the pipeline is in steady state.)
+    const int64_t kb_per_pair = streamk ? ((int64_t)p.num_tiles * G + npairs - 1) / npairs : p.kblocks_per_split;
+    if (per_group == 1 && kb_per_pair >= 8 && env_int("RESQ_GEMM_DEEP_E", 1)) {
+        // three activation slots cover the latency of their loads, one raw-code slot per group is enough, and
+        // the rest goes to expanded-weight slots (any number: a k-block's barrier slot is k-block mod SE)
+        const int sa2 = env_int("RESQ_GEMM_MIN_SA", 3), sr2 = kExpGroups;
+        const int left = kSmemBudget - fixed - sa2 * kAStage - sr2 * raw_stage;
+        const int se2 = std::min(std::min(left / exp_stage, 2 * kExpGroups), kMaxRing);
+        if (se2 > kExpGroups) {
+            p.se = se2;
+            p.sr = sr2;
+            p.sa = sa2;
+        }
+    }
+    if (p.sa > kMaxRing || fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage > kSmemBudget) {
+        set_last_error("internal: shared-memory rings do not fit (pair tile %d)", TN);
+        return RESQ_ERR_CUDA;
+    }
+    const int smem_bytes = fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)(2 * npairs), 1, 1);
@@ -767,14 +851,14 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
     }
     {
         LaunchScope scope(kKindGemm, stream);
-        e = cudaLaunchKernelEx(&cfg, kern, ta, tr, tw, p);
+        e = cudaLaunchKernelEx(&cfg, kern, ta, tr, te, tw, p);
     }
     if (e != cudaSuccess) return cuda_fail(e, "gemm_pair_kernel launch");
     if (streamk) return RESQ_OK;
     return launch_splitk_reduce(g, splits, stream);
 }
 
-template <bool RES, int FMT>
+template <int RES, int FMT>
 int dispatch_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
     const int ng = env_int("RESQ_GEMM_GROUPS", 3);
     if (tn == 128) return launch_pair_variant<RES, 128, FMT, 4>(g, splits, stream);
@@ -782,7 +866,11 @@ int dispatch_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
     if (tn == 256) return launch_pair_variant<RES, 256, FMT, 4>(g, splits, stream);
     if (tn == 320) return launch_pair_variant<RES, 320, FMT, 3>(g, splits, stream);
     if (tn == 384) return launch_pair_variant<RES, 384, FMT, 3>(g, splits, stream);
-    if (tn == 512) return launch_pair_variant<RES, 512, FMT, 3>(g, splits, stream);  // four slots would not fit
+    if constexpr (RES != kResSparse24) {  // 512 accumulator columns leave none for the sparse metadata
+        if (tn == 512) return launch_pair_variant<RES, 512, FMT, 3>(g, splits, stream);  // four slots would not fit
+    } else {
+        if (tn == 480) return launch_pair_variant<RES, 480, FMT, 3>(g, splits, stream);
+    }
     set_last_error("internal: unsupported pair tile width %d", tn);
     return RESQ_ERR_CUDA;
 }
@@ -793,19 +881,32 @@ size_t gemm_pair_streamk_scratch_bytes() {
     return (size_t)2 * kStreamKMaxPairs * (2 * kBM) * kStreamKTN * sizeof(float);
 }
 
+namespace {
+int res_mode(const GemmArgs& g) { return g.r_comp ? kResSparse24 : g.r_bf16 ? kResDense : kResNone; }
+template <int FMT>
+int streamk_fmt(const GemmArgs& g, cudaStream_t stream) {
+    switch (res_mode(g)) {
+        case kResSparse24: return launch_pair_variant<kResSparse24, kStreamKTN, FMT, 3>(g, 1, stream, true);
+        case kResDense: return launch_pair_variant<kResDense, kStreamKTN, FMT, 3>(g, 1, stream, true);
+        default: return launch_pair_variant<kResNone, kStreamKTN, FMT, 3>(g, 1, stream, true);
+    }
+}
+template <int FMT>
+int pair_fmt(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
+    switch (res_mode(g)) {
+        case kResSparse24: return dispatch_pair<kResSparse24, FMT>(g, tn, splits, stream);
+        case kResDense: return dispatch_pair<kResDense, FMT>(g, tn, splits, stream);
+        default: return dispatch_pair<kResNone, FMT>(g, tn, splits, stream);
+    }
+}
+}  // namespace
+
 int launch_gemm_pair_streamk(const GemmArgs& g, cudaStream_t stream) {
-    const bool res = g.r_bf16 != nullptr;
-    if (g.fmt == kMXFP4)
-        return res ? launch_pair_variant<true, kStreamKTN, kMXFP4, 3>(g, 1, stream, true)
-                   : launch_pair_variant<false, kStreamKTN, kMXFP4, 3>(g, 1, stream, true);
-    return res ? launch_pair_variant<true, kStreamKTN, kHiF4, 3>(g, 1, stream, true)
-               : launch_pair_variant<false, kStreamKTN, kHiF4, 3>(g, 1, stream, true);
+    return g.fmt == kMXFP4 ? streamk_fmt<kMXFP4>(g, stream) : streamk_fmt<kHiF4>(g, stream);
 }
 
 int launch_gemm_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
-    const bool res = g.r_bf16 != nullptr;
-    if (g.fmt == kMXFP4) return res ? dispatch_pair<true, kMXFP4>(g, tn, splits, stream) : dispatch_pair<false, kMXFP4>(g, tn, splits, stream);
-    return res ? dispatch_pair<true, kHiF4>(g, tn, splits, stream) : dispatch_pair<false, kHiF4>(g, tn, splits, stream);
+    return g.fmt == kMXFP4 ? pair_fmt<kMXFP4>(g, tn, splits, stream) : pair_fmt<kHiF4>(g, tn, splits, stream);
 }
 
 }  // namespace resq

@@ -247,6 +247,26 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc,
         : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Same with a 2:4 structured-sparse A: a_desc addresses the compressed tile (the two kept values of every four
+// consecutive K positions, K = 32 logical positions per instruction), tmem_e the even tensor-memory column of the
+// column pair that holds the index metadata of these 32 positions; bits 0-1 of idesc select the column of the
+// pair and bit 2 marks the instruction as sparse (sparse_idesc()).
+__device__ __forceinline__ void umma_bf16_sp_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t tmem_e,
+                                                  uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
+        :
+        : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(tmem_e), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Copy 128 rows of 16 bytes (row r at byte 16 r of a contiguous 2 KB block described by `desc`) from the shared
+// memory of each CTA of the pair into four 32-bit columns of its own tensor memory (lane r); one thread of the
+// leader issues it, ordered with the MMAs of the same thread.
+__device__ __forceinline__ void tmem_cp_128x128b_pair(uint32_t taddr, uint64_t desc) {
+    asm volatile("tcgen05.cp.cta_group::2.128x128b [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
+}
 // Arrive (once the MMAs issued so far have completed) on the mbarrier at the same offset in every CTA of
 // `cta_mask` (a commit-side multicast, not a TMA load).
 __device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mask) {
@@ -280,6 +300,15 @@ __device__ __forceinline__ uint64_t smem_desc_sw64_kmajor(uint32_t addr) {
     d |= (uint64_t)4 << 61;  // SWIZZLE_64B
     return d;
 }
+// Unswizzled rows of 16 bytes, 8-row groups 128 bytes apart (a contiguous block): source of tmem_cp_128x128b_pair.
+__device__ __forceinline__ uint64_t smem_desc_rows16(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(128 >> 4) << 16;
+    d |= (uint64_t)(128 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    return d;
+}
 // Instruction descriptor for kind::f16 with bf16 A/B (both K-major) and fp32 accumulation.
 __host__ __device__ constexpr uint32_t idesc_bf16_f32(int m, int n) {
     return (1u << 4)                      // D format: f32
@@ -288,6 +317,9 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int m, int n) {
            | ((uint32_t)(n >> 3) << 17)   // N / 8
            | ((uint32_t)(m >> 4) << 24);  // M / 16
 }
+
+// The same instruction with a 2:4 sparse A operand; `col` (0 or 1) selects the metadata column of the pair.
+__host__ __device__ constexpr uint32_t sparse_idesc(uint32_t idesc, uint32_t col) { return idesc | (1u << 2) | (col & 3u); }
 
 }  // namespace ptx
 }  // namespace resq

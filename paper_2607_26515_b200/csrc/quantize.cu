@@ -86,6 +86,27 @@ __device__ __forceinline__ void keep_words(uint32_t keep, uint32_t (&km)[4]) {
     asm("prmt.b32 %0, %1, 0, 0xBBAA;" : "=r"(km[3]) : "r"(zh));
 }
 
+// 2:4 compression of four consecutive bf16 values held in two words whose dropped halves are already zero:
+// returns the two kept values in channel order and the 4-bit index pair (idx0 | idx1 << 2) of the sparse MMA.
+// `nib` has exactly two bits set (the top-2-of-4 table guarantees it).
+__device__ __forceinline__ uint32_t compress24(uint32_t w0, uint32_t w1, uint32_t nib, uint32_t& idx) {
+    const uint32_t i0 = (uint32_t)__ffs((int)nib) - 1u, i1 = 31u - (uint32_t)__clz((int)nib);
+    idx = i0 | (i1 << 2);
+    // halves 0..3 of (w0, w1) are bytes (2h, 2h + 1)
+    return __byte_perm(w0, w1, (0x10u + 0x22u * i0) | ((0x10u + 0x22u * i1) << 8));
+}
+
+// Rows M .. (whole 256-row tiles) of the index metadata get a valid index pair (0, 1): the GEMM reads them next to
+// zero-filled values.  Every 16-bit piece (one row, 16 channels) is written on its own.
+__device__ __forceinline__ void fill_meta_pad(const QuantArgs& a, int64_t tid, int64_t nthreads) {
+    const int64_t pad_rows = a.meta_rows128 * 128 - a.M;
+    const int64_t pieces_per_row = a.meta_ka * 8;
+    for (int64_t i = tid; i < pad_rows * pieces_per_row; i += nthreads) {
+        const int64_t m = a.M + i / pieces_per_row, k = (i % pieces_per_row) * 16;
+        *reinterpret_cast<uint16_t*>(a.r_meta + sparse24_meta_offset(m, k, a.meta_ka)) = (uint16_t)0x4444u;
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Streaming kernel for the patterns whose selection is local to a row segment (NONE, DENSE, 2:4) and
 // first pass of the global ones (CHAN50, BLOCK: writes the unmasked residual and accumulates scores).
@@ -97,6 +118,9 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
     pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
     if (a.clear_words && blockIdx.x == 0 && blockIdx.y == 0)
         for (int i = threadIdx.x; i < a.n_clear_words; i += blockDim.x) a.clear_words[i] = 0u;
+    if (RESIDUAL && IMG && a.r_comp)
+        fill_meta_pad(a, ((int64_t)blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x,
+                      (int64_t)gridDim.x * gridDim.y * blockDim.x);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t k0 = ((int64_t)blockIdx.y * kWarpsPerCta + warp) * kColsPerWarp + lane * 8;
     const bool active = k0 < a.K;  // whole blocks are active or not (K is a multiple of the block size)
@@ -172,6 +196,24 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
         }
         uint32_t keep = 0xFFu;
         if (pattern == RESQ_S_2_4) keep = top2_mask8(roct);
+        uint32_t comp0 = 0, comp1 = 0, idx_byte = 0;
+        if constexpr (IMG) {
+            if (a.r_comp) {  // (2:4 only) compressed image: 8 bytes per lane, and one byte of index pairs
+                uint32_t km[4], o[4], ia, ib;
+                keep_words(keep, km);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    o[i] = pack_bf16x2_exact(rdeq[2 * i], rdeq[2 * i + 1]);
+                    if constexpr (FMT == kHiF4) o[i] |= dw[i] & 0x80008000u;
+                    o[i] &= km[i];
+                }
+                comp0 = compress24(o[0], o[1], keep & 15u, ia);
+                comp1 = compress24(o[2], o[3], keep >> 4, ib);
+                idx_byte = ia | (ib << 4);
+                // the even lane of a pair stores the 16-bit piece of 16 channels
+                idx_byte |= __shfl_down_sync(0xFFFFFFFFu, idx_byte, 1) << 8;
+            }
+        }
         if (pattern == RESQ_S_CHAN50) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) chan_acc[i] += (double)rdeq[i] * (double)rdeq[i];
@@ -207,6 +249,11 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
             const bool local = pattern == RESQ_S_DENSE || pattern == RESQ_S_2_4;
             if (a.mask_bits && local) a.mask_bits[m * (a.K / 8) + k0 / 8] = (uint8_t)keep;
             if constexpr (IMG) {
+              if (a.r_comp) {
+                *reinterpret_cast<uint2*>(a.r_comp + m * (a.K / 2) + k0 / 2) = make_uint2(comp0, comp1);
+                if ((lane & 1) == 0)
+                    *reinterpret_cast<uint16_t*>(a.r_meta + sparse24_meta_offset(m, k0, a.meta_ka)) = (uint16_t)idx_byte;
+              } else {
                 // for the global patterns this is the unmasked image; the apply kernel zeroes dropped entries
                 uint32_t km[4];
                 keep_words(keep, km);
@@ -226,6 +273,7 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
                 o.z &= km[2];
                 o.w &= km[3];
                 *reinterpret_cast<uint4*>(a.r_bf16 + m * a.K + k0) = o;
+              }
             }
         }
         }  // RESIDUAL
@@ -435,6 +483,8 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
     pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
     if (a.clear_words && blockIdx.x == 0 && blockIdx.y == 0)
         for (int i = threadIdx.x; i < a.n_clear_words; i += blockDim.x) a.clear_words[i] = 0u;
+    const bool comp = RESIDUAL && IMG && a.r_comp != nullptr;  // 2:4: compressed residual image + index metadata
+    if (comp) fill_meta_pad(a, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, (int64_t)gridDim.x * blockDim.x);
     extern __shared__ __align__(16) uint8_t smem_q[];
     constexpr int kBufs = IMG ? 3 : 2;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -468,6 +518,17 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
         for (int j = 0; j < 8; ++j) {
             const uint4 v = lds_16(stage + cp_smem + j * 4 * kStagePitch);
             if (cp_col + j * 4 * kHif4Block < a.K) *reinterpret_cast<uint4*>(dst_row + cp_col + j * 4 * kHif4Block) = v;
+        }
+        __syncwarp();
+    };
+    // same for a staged compressed row (64 bytes per block): piece j of lane l is chunk (l & 3) of block 8j + (l >> 2)
+    auto drain_stage_comp = [&](__nv_bfloat16* dst_row) {
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int b = 8 * j + (lane >> 2);
+            const uint4 v = lds_16(stage + (uint32_t)(b * kStagePitch + (lane & 3) * 16));
+            if (cg * 32 + b < G) *reinterpret_cast<uint4*>(dst_row + (cg * 32 + b) * (kHif4Block / 2) + (lane & 3) * 8) = v;
         }
         __syncwarp();
     };
@@ -529,6 +590,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
         if constexpr (IMG) drain_stage(a.a_bf16 + m * a.K);
         if constexpr (RESIDUAL) {
             uint32_t rcodes[8], rmeta, keep_lo = 0xFFFFFFFFu, keep_hi = 0xFFFFFFFFu;
+            uint32_t idx_lo = 0, idx_hi = 0;  // comp: index pairs of channels 0..31 and 32..63 of the block
             float sq0 = 0.0f, sq1 = 0.0f;  // per 32 values: exact in fp32 for both formats (see below)
             encode_block<FMT, true, true>(w, rcodes, rmeta, [&](int c, const float (&)[8], const float (&rdq)[8], uint32_t roct) {
                 uint32_t keep = 0xFFu;
@@ -554,7 +616,16 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
                         img[i] = (pack_bf16x2_exact(rdq[2 * i], rdq[2 * i + 1]) | (w[4 * c + i] & 0x80008000u)) & km[i];
-                    sts_16(stage + my_in + c * 16, make_uint4(img[0], img[1], img[2], img[3]));
+                    if (comp) {
+                        uint32_t ia, ib;
+                        const uint32_t c0 = compress24(img[0], img[1], keep & 15u, ia);
+                        const uint32_t c1 = compress24(img[2], img[3], keep >> 4, ib);
+                        asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(stage + my_in + c * 8), "r"(c0), "r"(c1) : "memory");
+                        if (c < 4) idx_lo |= (ia | (ib << 4)) << (8 * c);
+                        else idx_hi |= (ia | (ib << 4)) << (8 * (c - 4));
+                    } else {
+                        sts_16(stage + my_in + c * 16, make_uint4(img[0], img[1], img[2], img[3]));
+                    }
                 }
             });
             if (pattern == RESQ_S_BLOCK32x64_50) {
@@ -587,7 +658,22 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
                 const bool local = pattern == RESQ_S_DENSE || pattern == RESQ_S_2_4;
                 if (a.mask_bits && local) *reinterpret_cast<uint2*>(a.mask_bits + m * (a.K / 8) + blk * 8) = make_uint2(keep_lo, keep_hi);
             }
-            if constexpr (IMG) drain_stage(a.r_bf16 + m * a.K);
+            if constexpr (IMG) {
+                if (comp) {
+                    if (active) {
+                        // four 16-bit pieces (16 channels each); consecutive pieces alternate between the two halves
+                        // of a metadata block's row group and advance one 32-bit word every second piece
+                        uint8_t* e = a.r_meta + sparse24_meta_offset(m, blk * kHif4Block, a.meta_ka);
+                        *reinterpret_cast<uint16_t*>(e) = (uint16_t)idx_lo;
+                        *reinterpret_cast<uint16_t*>(e + 128) = (uint16_t)(idx_lo >> 16);
+                        *reinterpret_cast<uint16_t*>(e + 4) = (uint16_t)idx_hi;
+                        *reinterpret_cast<uint16_t*>(e + 132) = (uint16_t)(idx_hi >> 16);
+                    }
+                    drain_stage_comp(a.r_comp + m * (a.K / 2));
+                } else {
+                    drain_stage(a.r_bf16 + m * a.K);
+                }
+            }
         }
     }
     cp_async_wait<0>();
@@ -1181,7 +1267,7 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     // that the finer-grained kernel (a lane per 8 values) finishes sooner.
     const int64_t block_tasks = a.M * ((a.K / kHif4Block + 31) / 32);
     if (pattern != RESQ_S_CHAN50 && a.K % kHif4Block == 0 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
-        al16(a.a_bf16) && al16(a.r_bf16)) {
+        al16(a.a_bf16) && al16(a.r_bf16) && al16(a.r_comp)) {
         const bool img = a.a_bf16 != nullptr;
         const int64_t ncg = (a.K / kHif4Block + 31) / 32;
         int rows_per_warp = 1;

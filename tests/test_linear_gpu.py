@@ -185,6 +185,58 @@ def test_every_tile_configuration(tile_case, cfg, pattern, fmt, monkeypatch):
     check_close(y.cpu().numpy(), w["y"], w["abs_sum"])
 
 
+SPARSE_CONFIGS = [
+    {},
+    {"RESQ_GEMM_PAIR_TN": "480", "RESQ_GEMM_SPLITS": "1"},
+    {"RESQ_GEMM_PAIR_TN": "384", "RESQ_GEMM_SPLITS": "2"},
+    {"RESQ_GEMM_PAIR_TN": "320", "RESQ_GEMM_SPLITS": "4"},   # K ranges that start at odd k-blocks
+    {"RESQ_GEMM_PAIR_TN": "256", "RESQ_GEMM_SPLITS": "1", "RESQ_GEMM_DEEP_E": "0"},
+    {"RESQ_GEMM_PAIR_TN": "128", "RESQ_GEMM_SPLITS": "1"},
+    {"RESQ_GEMM_STREAMK": "1"},
+]
+
+
+@pytest.mark.parametrize("cfg", SPARSE_CONFIGS, ids=lambda c: ",".join(f"{k[10:]}={v}" for k, v in c.items()) or "default")
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+def test_two_to_four_residual_on_the_sparse_mma(tile_case, cfg, fmt, monkeypatch):
+    """S_2:4 with the residual in compressed form (two kept values of every four channels + index metadata) on
+    the structured-sparse tensor instruction: same result as the dense form, for every tile width that has room
+    for the metadata, split K ranges and the K-streamed schedule."""
+    xb, wb, want = tile_case
+    monkeypatch.setenv("RESQ_SPARSE24", "1")
+    monkeypatch.setenv("RESQ_MXFP4_NATIVE", "0")
+    for k, v in cfg.items():
+        monkeypatch.setenv(k, v)
+    m = rq()
+    M, K = xb.shape
+    N = wb.shape[0]
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    work = m.alloc_workspace(m.resq_workspace_bytes(M, N, K, oracle.S_2_4, fmt))
+    y = m.resq_linear(to_dev(xb), wc, ws, oracle.S_2_4, fmt, out_dtype=torch.float32, workspace=work)
+    assert m.check(work) == 0, m.last_error()
+    w = want[(oracle.S_2_4, fmt)]
+    check_close(y.cpu().numpy(), w["y"], w["abs_sum"])
+
+
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("shape", [(2400, 192, 200), (2500, 4160, 96)])
+def test_sparse_mma_with_the_block_per_lane_quantizer(shape, fmt, monkeypatch):
+    """Shapes large enough for the block-per-lane quantizer kernel (which compresses in its staging buffers): an odd
+    number of k-blocks (half-used metadata block), rows that are not a multiple of the 128-row metadata bands,
+    and a row longer than one warp segment."""
+    monkeypatch.setenv("RESQ_SPARSE24", "1")
+    monkeypatch.setenv("RESQ_MXFP4_NATIVE", "0")
+    m = rq()
+    M, K, N = shape
+    xb, wb = synth_xw(3 * M + K, M, K, N, n_out=max(1, K // 256))
+    want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), oracle.S_2_4, fmt)
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    work = m.alloc_workspace(m.resq_workspace_bytes(M, N, K, oracle.S_2_4, fmt))
+    y = m.resq_linear(to_dev(xb), wc, ws, oracle.S_2_4, fmt, out_dtype=torch.float32, workspace=work)
+    assert m.check(work) == 0, m.last_error()
+    check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+
+
 @pytest.mark.parametrize("pattern", ALL)
 @pytest.mark.parametrize("shape", [(288, 512, 600), (128, 256, 256), (992, 1024, 1300)])
 def test_mxfp4_block_scaled_fp4_gemm(monkeypatch, pattern, shape):
