@@ -174,6 +174,20 @@ RESQ_API int mxfp4_w4a16_linear(const void* X_bf16, int64_t M, int64_t K, int64_
                        void* Y, int out_dtype, int64_t ldy,
                        void* workspace, size_t ws_bytes, void* stream);
 
+/* Activation-only ablation of Table 1 ("W16A4"): Y = (deq Q(X) + S(deq Q(dX))) W^T with the weights in plain
+ * bf16 (W_bf16: [N, K] device, row pitch ldw elements, ldw >= K, ldw % 8 == 0, 16-byte aligned base); the
+ * activations go through the same quantizer, residual and selection as *_resq_linear (pattern RESQ_S_NONE gives
+ * the table's plain Q(X) W^T).  Same argument rules, output types, error behaviour and workspace
+ * (*_resq_workspace_bytes(M, N, K, pattern)) as *_resq_linear. */
+RESQ_API int hif4_w16a4_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
+                      const void* W_bf16, int64_t N, int64_t ldw,
+                      int pattern, void* Y, int out_dtype, int64_t ldy,
+                      void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_w16a4_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
+                       const void* W_bf16, int64_t N, int64_t ldw,
+                       int pattern, void* Y, int out_dtype, int64_t ldy,
+                       void* workspace, size_t ws_bytes, void* stream);
+
 /* ---- status --------------------------------------------------------------------------------------
  * resq_check synchronizes `stream` and returns the device status word kept at the start of
  * `workspace` (RESQ_OK, or RESQ_ERR_TIMEOUT if a bounded wait expired in the last call that used it). */

@@ -228,6 +228,16 @@ def resq_linear(x_f32: np.ndarray, w_f32: np.ndarray, pattern: int, fmt: str = "
     return out
 
 
+def w16a4_linear(x_f32: np.ndarray, w_f32: np.ndarray, pattern: int = S_NONE, fmt: str = "hif4",
+                 want_abs: bool = True) -> Dict[str, np.ndarray]:
+    """Activation-only ablation (Table 1, W16A4): the activations go through Q, Eq. (3) and S as in Eq. (5); the
+    weights are used as given (bf16 values): Y = (deq Q(X) + S(deq Q(dX))) W^T."""
+    out = quantize_residual_mask(x_f32, pattern, fmt)
+    y, ab = matmul(out["a"], out.get("r_masked"), np.asarray(w_f32, dtype=np.float64), want_abs)
+    out.update({"y": y, "abs_sum": ab})
+    return out
+
+
 def w4a16_linear(x_f32: np.ndarray, w_f32: np.ndarray, fmt: str = "hif4", want_abs: bool = True) -> Dict[str, np.ndarray]:
     """Weight-only ablation (Table 1, W4A16): Y = X deq(Q(W))^T, activations as given (bf16 values)."""
     w_codes, w_side = encode(fmt, _f32(w_f32))

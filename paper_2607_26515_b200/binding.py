@@ -47,6 +47,8 @@ SYMBOLS = {
     "resq_w4a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "hif4_w4a16_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
     "mxfp4_w4a16_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "hif4_w16a4_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "mxfp4_w16a4_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "resq_check": (_ci, [_vp, _vp]),
     "resq_last_error": (ctypes.c_char_p, []),
     "resq_kernel_launches": (_i64, []),
@@ -239,6 +241,30 @@ def w4a16_linear(X: torch.Tensor, w_codes: torch.Tensor, w_side: torch.Tensor, f
         workspace = alloc_workspace(int(lib().resq_w4a16_workspace_bytes(M, N, K)), X.device)
     _check(_fn(fmt, "hif4_w4a16_linear", "mxfp4_w4a16_linear")(
         X.data_ptr(), M, K, X.stride(0), w_codes.data_ptr(), w_side.data_ptr(), N, Y.data_ptr(),
+        OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32, Y.stride(0), workspace.data_ptr(), workspace.numel(),
+        _stream(stream)))
+    return Y
+
+
+def w16a4_linear(X: torch.Tensor, W: torch.Tensor, pattern: int = S_NONE, fmt: str = "hif4",
+                 out_dtype: torch.dtype = torch.bfloat16, Y: Optional[torch.Tensor] = None,
+                 workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """*_w16a4_linear: Y = (deq Q(X) + S(deq Q(dX))) W^T with plain bf16 weights (Table 1, W16A4)."""
+    _require_bf16_matrix(X, "X")
+    _require_bf16_matrix(W, "W")
+    M, K = X.shape
+    N = W.shape[0]
+    if W.shape[1] != K:
+        raise ValueError("W must be [N, K]")
+    if Y is None:
+        ld = (N + 7) // 8 * 8
+        Y = torch.empty((M, ld), dtype=out_dtype, device=X.device)[:, :N]
+    if Y.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("Y must be bf16 or fp32")
+    if workspace is None:
+        workspace = alloc_workspace(resq_workspace_bytes(M, N, K, pattern, fmt), X.device)
+    _check(_fn(fmt, "hif4_w16a4_linear", "mxfp4_w16a4_linear")(
+        X.data_ptr(), M, K, X.stride(0), W.data_ptr(), N, W.stride(0), pattern, Y.data_ptr(),
         OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32, Y.stride(0), workspace.data_ptr(), workspace.numel(),
         _stream(stream)))
     return Y

@@ -206,12 +206,26 @@ size_t linear_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K, int patt
     return b;
 }
 
+// w_bf16 != null: activation-only quantization (Table 1, "W16A4"): plain bf16 weights [N, K] with row pitch ldw
+// instead of the packed ones.
 int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_side, int64_t N,
-           int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+           int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream,
+           const void* w_bf16 = nullptr, int64_t ldw = 0) {
     int rc = check_matrix(X, M, K, ldx, fmt, "X");
     if (rc) return rc;
     rc = check_pattern(pattern, M);
     if (rc) return rc;
+    if (w_bf16) {
+        if (!Y) {
+            set_last_error("linear: NULL output pointer");
+            return RESQ_ERR_NULL;
+        }
+        if (!aligned16(w_bf16) || ldw < K || ldw % 8 != 0) {
+            set_last_error("linear: bf16 weights need a 16-byte aligned base, ldw >= K and 16-byte aligned rows");
+            return RESQ_ERR_ALIGN;
+        }
+        w_codes = w_side = w_bf16;  // (only to pass the checks on the packed operands below)
+    }
     if (!w_codes || !w_side || !Y) {
         set_last_error("linear: NULL weight or output pointer");
         return RESQ_ERR_NULL;
@@ -248,7 +262,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     used += kWsFlags;
     // MXFP4 where it pays: the GEMM runs on the block-scaled FP4 pipe and takes packed codes and scales (they
     // fit into the space of the bf16 images; the selection zeroes dropped codes); otherwise exact bf16 images.
-    const bool native = fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K, pattern != RESQ_S_NONE);
+    const bool native = !w_bf16 && fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K, pattern != RESQ_S_NONE);
     uint8_t* region_a = ws + used;
     used += align_up((size_t)M * (size_t)K * 2, 256);
     uint8_t* region_r = nullptr;
@@ -257,7 +271,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
         used += residual_region_bytes(M, K, pattern);
     }
     // 2:4 on the CTA-pair kernel: the residual goes to the structured-sparse MMA in compressed form
-    const bool sparse24 = !native && pattern == RESQ_S_2_4 && gemm_sparse24_supported(M, N, K);
+    const bool sparse24 = !w_bf16 && !native && pattern == RESQ_S_2_4 && gemm_sparse24_supported(M, N, K);
     const size_t codes_bytes = align_up((size_t)M * (size_t)K / 2, 256);
     if (native) {
         a.x_codes = region_a;
@@ -308,6 +322,8 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     g.meta_ka = a.meta_ka;
     g.w_codes = static_cast<const uint8_t*>(w_codes);
     g.w_side = w_side;
+    g.w_bf16 = static_cast<const __nv_bfloat16*>(w_bf16);
+    g.ldw = ldw;
     g.M = M;
     g.N = N;
     g.K = K;
@@ -430,6 +446,23 @@ int mxfp4_residual_mask(const void* X, int64_t M, int64_t K, int64_t ldx, int pa
                         void* r_codes, void* r_scale, void* mask_bits, void* workspace, size_t ws_bytes, void* stream) {
     return residual_mask(kMXFP4, X, M, K, ldx, pattern, x_codes, x_scale, r_codes, r_scale, mask_bits, workspace,
                          ws_bytes, stream);
+}
+
+int hif4_w16a4_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* W, int64_t N, int64_t ldw, int pattern,
+                      void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    if (!W) {
+        set_last_error("w16a4_linear: NULL weight pointer");
+        return RESQ_ERR_NULL;
+    }
+    return linear(kHiF4, X, M, K, ldx, nullptr, nullptr, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream, W, ldw);
+}
+int mxfp4_w16a4_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* W, int64_t N, int64_t ldw, int pattern,
+                       void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    if (!W) {
+        set_last_error("w16a4_linear: NULL weight pointer");
+        return RESQ_ERR_NULL;
+    }
+    return linear(kMXFP4, X, M, K, ldx, nullptr, nullptr, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream, W, ldw);
 }
 
 size_t resq_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) { return w4a16_workspace_bytes(M, N, K); }

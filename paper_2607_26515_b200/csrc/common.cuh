@@ -115,6 +115,8 @@ struct GemmArgs {
     int64_t meta_rows128, meta_ka;
     const uint8_t* w_codes;        // [N, K/2]
     const void* w_side;            // [N, K/64] u32 or [N, K/32] u8
+    const __nv_bfloat16* w_bf16;   // instead of w_codes / w_side: plain bf16 weights [N, K], row pitch ldw ("W16A4")
+    int64_t ldw;
     int64_t M, N, K;
     int64_t lda;                   // row pitch of a_bf16 / r_bf16 in elements (0: K, the workspace images)
     void* Y;

@@ -517,6 +517,7 @@ int launch_splitk_reduce(const GemmArgs& g, int splits, cudaStream_t stream) {
 
 int launch_gemm_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream);
 int launch_gemm_pair_streamk(const GemmArgs& g, cudaStream_t stream);
+int launch_gemm_pair_plainw(const GemmArgs& g, int tn, int splits, bool streamk, cudaStream_t stream);
 size_t gemm_pair_streamk_scratch_bytes();
 
 namespace {
@@ -746,9 +747,15 @@ int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream) {
         set_last_error("internal: compressed residual given for a shape the pair kernel does not run");
         return RESQ_ERR_CUDA;
     }
-    if (gemm_use_streamk(g.M, g.N, g.K) && g.splitk_partials && g.sk_flags &&
-        g.partial_bytes >= gemm_pair_streamk_scratch_bytes())
-        return launch_gemm_pair_streamk(g, stream);
+    const bool streamk = gemm_use_streamk(g.M, g.N, g.K) && g.splitk_partials && g.sk_flags &&
+                         g.partial_bytes >= gemm_pair_streamk_scratch_bytes();
+    if (g.w_bf16) {  // the CTA-pair kernel for every M (rows past M are zero-filled and never stored)
+        if (streamk) return launch_gemm_pair_plainw(g, 256, 1, true, stream);
+        const TileChoice c = g.M > kBM ? choose_tile(g.M, g.N, g.K, res) : TileChoice{1, 256, 1, 1, 256};
+        const int splits = (c.splits > 1 && g.splitk_partials && c.splits <= g.splits) ? c.splits : 1;
+        return launch_gemm_pair_plainw(g, c.pair_tn >= 384 ? 512 : 256, splits, false, stream);
+    }
+    if (streamk) return launch_gemm_pair_streamk(g, stream);
     TileChoice tc = choose_tile(g.M, g.N, g.K, res, g.r_comp != nullptr);
     if (tc.splits > 1 && (!g.splitk_partials || tc.splits > g.splits)) tc.splits = 1;
     if (env_int("RESQ_GEMM_DEBUG", 0) & 1)

@@ -239,6 +239,10 @@ __device__ __forceinline__ void streamk_fixup(const PairParams& p, int pair, int
     }
 }
 
+// Weight formats of the kernel: the two packed 4-bit formats (expanded in the kernel), or plain bf16 weights that
+// TMA writes straight into the slots of the expanded-weight ring (activation-only quantization, "W16A4").
+constexpr int kPlainW = 2;
+
 // Residual term of the kernel: none, a dense second A operand (the masked bf16 image), or the 2:4 compressed image
 // with its index metadata on the structured-sparse MMA (half the tensor work of the dense form).
 enum ResMode : int { kResNone = 0, kResDense = 1, kResSparse24 = 2 };
@@ -260,7 +264,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     constexpr int bn = TN / nt;                    // MMA N
     constexpr int half = bn / 2;                   // rows of each MMA's weight tile held by one CTA
     constexpr int my_rows = nt * half;             // rows this CTA expands per k-block
-    constexpr int exp_stage = my_rows * 128, raw_stage = my_rows * 32;
+    constexpr int exp_stage = my_rows * 128, raw_stage = FMT == kPlainW ? 0 : my_rows * 32;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int SA = p.sa, SR = p.sr, SE = p.se;
@@ -296,7 +300,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxRing; ++s) {
-            ptx::mbar_init(&a_full[s], 2 + 2 * kGroupWarps);  // an arrive.expect_tx and one expander group per CTA
+            // an arrive.expect_tx per CTA for the activations, and one expander group per CTA (packed weights) or a
+            // second arrive.expect_tx per CTA (bf16 weights)
+            ptx::mbar_init(&a_full[s], FMT == kPlainW ? 4 : 2 + 2 * kGroupWarps);
             ptx::mbar_init(&a_empty[s], 1);
             ptx::mbar_init(&r_full[s], 1);
             ptx::mbar_init(&r_empty[s], kGroupWarps);
@@ -380,6 +386,23 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             SegIter<TN> si(p, pair, npairs);
             TileCoord tc;
             while (ok && si.next(tc)) {
+                if constexpr (FMT == kPlainW) {
+                    // bf16 weights: this CTA's rows of the k-block go straight into the expanded-weight slot
+                    for (int i = 0; i < tc.nkb; ++i, ++it) {
+                        const int se = it % SE;
+                        if (!ptx::mbar_wait_spin(&e_empty[se], ((it / SE) & 1) ^ 1, abort_flag)) {
+                            report_timeout(p.status, 5);
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t full = ptx::map_to_cta(&e_full[se], 0);
+                        ptx::mbar_arrive_expect_tx_cluster_relaxed(full, (uint32_t)exp_stage);
+#pragma unroll
+                        for (int j = 0; j < nt; ++j)
+                            ptx::tma_load_2d_pair(ring_e + (size_t)se * exp_stage + (size_t)j * half * 128, &tmap_w, full,
+                                                  (tc.kb_begin + i) * kBK, (int)(tc.n0 + j * bn + rank * half));
+                    }
+                } else {
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
                     const int s = it % SR;
                     tr.begin();
@@ -396,6 +419,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     for (int j = 0; j < nt; ++j)
                         ptx::tma_load_2d(ring_r + (size_t)s * raw_stage + (size_t)j * half * 32, &tmap_w, &r_full[s],
                                          (tc.kb_begin + i) * (kBK / 2), (int)(tc.n0 + j * bn + rank * half));
+                }
                 }
             }
         }
@@ -482,7 +506,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 EVT(3);
             }
         }
-    } else if (warp >= kFirstExpWarp) {
+    } else if (warp >= kFirstExpWarp && FMT != kPlainW) {
         // ------------------------------------------------------------------ expanders (both CTAs, own half)
         // NG groups of four warps take k-blocks round-robin, so each group has NG MMA periods for one block:
         // the per-block synchronisation latency (two waits, two arrives, one proxy fence) stays off the
@@ -555,7 +579,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             }
             it0 += (uint32_t)tc.nkb;
         }
-    } else if (warp >= kFirstEpiWarp) {
+    } else if (warp >= kFirstEpiWarp && warp < kFirstExpWarp) {
         // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
         const int quad = warp & 3;
         constexpr int nchunks = TN / 32;
@@ -716,8 +740,12 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
         te = ta;
     }
     if (rc) return rc;
-    rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.w_codes, (uint64_t)g.K / 2, (uint64_t)g.N, (uint64_t)g.K / 2,
-                      kBK / 2, (uint32_t)half, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (FMT == kPlainW)
+        rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.w_bf16, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.ldw * 2, kBK,
+                          (uint32_t)half, CU_TENSOR_MAP_SWIZZLE_128B);
+    else
+        rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.w_codes, (uint64_t)g.K / 2, (uint64_t)g.N, (uint64_t)g.K / 2,
+                          kBK / 2, (uint32_t)half, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc) return rc;
     PairParams p;
     p.meta_ka = g.meta_ka;
@@ -784,7 +812,7 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
             npairs = p.num_tiles * per_tile;
         }
     }
-    constexpr int exp_stage = my_rows * 128, raw_stage = my_rows * 32;
+    constexpr int exp_stage = my_rows * 128, raw_stage = FMT == kPlainW ? 0 : my_rows * 32;  // (the kernel's raw ring is unused then)
     const int fixed = 1024 + 1024;
     // Ring slots: a multiple of the number of expander groups (group g works on the slots s = g mod NG, so a slot
     // is only ever written by one group).  With one slot per group the group's expansion of a k-block and the
@@ -809,6 +837,8 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
             p.se = se2;
             p.sr = sr2;
             p.sa = sa2;
+            // what is left over deepens the activation ring (its loads have ~2000 cycles of latency to cover)
+            while (p.sa < p.se && fixed + (p.sa + 1) * kAStage + p.se * exp_stage + p.sr * raw_stage <= kSmemBudget) ++p.sa;
         }
     }
     if (p.sa > kMaxRing || fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage > kSmemBudget) {
@@ -900,6 +930,20 @@ int pair_fmt(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
     }
 }
 }  // namespace
+
+// bf16 weights (no expansion): 256-wide tiles on the K-streamed schedule or for small problems, else 512-wide.
+int launch_gemm_pair_plainw(const GemmArgs& g, int tn, int splits, bool streamk, cudaStream_t stream) {
+    const int mode = res_mode(g);
+    if (mode == kResSparse24) {
+        set_last_error("internal: the bf16-weight GEMM takes the dense residual image");
+        return RESQ_ERR_CUDA;
+    }
+    if (streamk || tn <= 256)
+        return mode == kResDense ? launch_pair_variant<kResDense, 256, kPlainW, 3>(g, splits, stream, streamk)
+                                 : launch_pair_variant<kResNone, 256, kPlainW, 3>(g, splits, stream, streamk);
+    return mode == kResDense ? launch_pair_variant<kResDense, 512, kPlainW, 3>(g, splits, stream)
+                             : launch_pair_variant<kResNone, 512, kPlainW, 3>(g, splits, stream);
+}
 
 int launch_gemm_pair_streamk(const GemmArgs& g, cudaStream_t stream) {
     return g.fmt == kMXFP4 ? streamk_fmt<kMXFP4>(g, stream) : streamk_fmt<kHiF4>(g, stream);

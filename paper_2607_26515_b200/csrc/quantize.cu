@@ -907,6 +907,8 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(const double* 
     __shared__ int s_warp_count[kSelThreads / 32];
     __shared__ int s_base;
     const int tid = threadIdx.x;
+    pdl_wait();     // the scores come from the quantizer kernel just before
+    pdl_trigger();  // the mask pass may be scheduled (it waits for this kernel's flags)
     if (keep <= 0 || keep >= n) {
         for (int i = tid; i < n; i += kSelThreads) flag[i] = keep >= n ? 1 : 0;
         return;
@@ -920,10 +922,14 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(const double* 
         if (tid < 256) hist[tid] = 0u;
         __syncthreads();
         const unsigned long long prefix = s_prefix;
-        for (int i = tid; i < n; i += kSelThreads) {
-            unsigned long long key = (unsigned long long)__double_as_longlong(score[i]);
-            bool match = shift == 56 ? true : ((key ^ prefix) >> (shift + 8)) == 0ull;
-            if (match) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
+        // scores of one tensor mostly share their leading digits: lanes that hit the same bucket add once
+        for (int i0 = 0; i0 < n; i0 += kSelThreads) {
+            const int i = i0 + tid;
+            unsigned long long key = i < n ? (unsigned long long)__double_as_longlong(score[i]) : 0ull;
+            const bool match = i < n && (shift == 56 ? true : ((key ^ prefix) >> (shift + 8)) == 0ull);
+            const unsigned bucket = match ? (unsigned)(key >> shift) & 255u : 0xFFFFFFFFu;
+            const unsigned same = __match_any_sync(0xFFFFFFFFu, bucket);
+            if (match && (unsigned)(__ffs((int)same) - 1) == (unsigned)(tid & 31)) atomicAdd(&hist[bucket], (unsigned)__popc(same));
         }
         __syncthreads();
         // pick the bucket that holds the remaining-th largest key: suffix sums of the histogram by one warp
@@ -986,6 +992,8 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(const double* 
 __global__ void apply_global_mask_kernel(int pattern, int64_t M, int64_t K, const uint8_t* __restrict__ flag,
                                          uint8_t* __restrict__ mask_bits, __nv_bfloat16* __restrict__ r_bf16,
                                          uint8_t* __restrict__ r_codes_masked) {
+    pdl_wait();     // the keep flags come from the selection kernel just before
+    pdl_trigger();  // the GEMM may be scheduled and run its set-up
     int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     int64_t per_row = K / 8;
     if (idx >= M * per_row) return;
@@ -1219,6 +1227,27 @@ size_t quant_scratch_bytes(int64_t M, int64_t K, int pattern) {
     return align_up(n * sizeof(double), 256) + align_up(n, 256);
 }
 
+// Second and third kernel of the patterns with a tensor-wide selection (CHAN50, BLOCK): top half of the scores,
+// then the mask pass over the residual outputs.
+static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t stream) {
+    int rc;
+    {
+        LaunchScope scope(kKindSelect, stream);
+        rc = cuda_fail(launch_kernel(topk_select_kernel, dim3(1), dim3(kSelThreads), 0, stream, (const double*)a.scores, (int)nscore,
+                                     (int)(nscore / 2), a.keep_flags),
+                       "topk_select_kernel launch");
+    }
+    if (rc) return rc;
+    if (a.mask_bits || a.r_bf16 || (a.r_codes && a.mask_r_codes)) {
+        const int64_t n = a.M * (a.K / 8);
+        LaunchScope scope(kKindSelect, stream);
+        rc = cuda_fail(launch_kernel(apply_global_mask_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, stream, a.pattern, a.M,
+                                     a.K, (const uint8_t*)a.keep_flags, a.mask_bits, a.r_bf16, a.mask_r_codes ? a.r_codes : (uint8_t*)nullptr),
+                       "apply_global_mask_kernel launch");
+    }
+    return rc;
+}
+
 int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     const int pattern = a.pattern;
     const bool residual = pattern != RESQ_S_NONE;
@@ -1290,20 +1319,7 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
             rc = residual ? (img ? launch(quant_block_kernel<kMXFP4, true, true>) : launch(quant_block_kernel<kMXFP4, true, false>))
                           : (img ? launch(quant_block_kernel<kMXFP4, false, true>) : launch(quant_block_kernel<kMXFP4, false, false>));
         if (rc) return rc;
-        if (global_sel) {
-            { LaunchScope scope(kKindSelect, stream);
-            topk_select_kernel<<<1, kSelThreads, 0, stream>>>(a.scores, (int)nscore, (int)(nscore / 2), a.keep_flags); }
-            rc = cuda_fail(cudaGetLastError(), "topk_select_kernel launch");
-            if (rc) return rc;
-            if (a.mask_bits || a.r_bf16 || (a.r_codes && a.mask_r_codes)) {
-                int64_t n = a.M * (a.K / 8);
-                LaunchScope scope(kKindSelect, stream);
-                apply_global_mask_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(pattern, a.M, a.K, a.keep_flags,
-                                                                                          a.mask_bits, a.r_bf16,
-                                                                                          a.mask_r_codes ? a.r_codes : nullptr);
-                rc = cuda_fail(cudaGetLastError(), "apply_global_mask_kernel launch");
-            }
-        }
+        if (global_sel) rc = launch_global_select(a, nscore, stream);
         return rc;
     }
     const int rows_per_cta = pick_rows_per_cta(a.M, a.K, pattern);
@@ -1324,20 +1340,7 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     }
     int rc = cuda_fail(launch_err, "quant_stream_kernel launch");
     if (rc) return rc;
-    if (global_sel) {
-        { LaunchScope scope(kKindSelect, stream);
-        topk_select_kernel<<<1, kSelThreads, 0, stream>>>(a.scores, (int)nscore, (int)(nscore / 2), a.keep_flags); }
-        rc = cuda_fail(cudaGetLastError(), "topk_select_kernel launch");
-        if (rc) return rc;
-        if (a.mask_bits || a.r_bf16 || (a.r_codes && a.mask_r_codes)) {
-            int64_t n = a.M * (a.K / 8);
-            LaunchScope scope(kKindSelect, stream);
-            apply_global_mask_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(pattern, a.M, a.K, a.keep_flags,
-                                                                                      a.mask_bits, a.r_bf16,
-                                                                                      a.mask_r_codes ? a.r_codes : nullptr);
-            rc = cuda_fail(cudaGetLastError(), "apply_global_mask_kernel launch");
-        }
-    }
+    if (global_sel) rc = launch_global_select(a, nscore, stream);
     return rc;
 }
 

@@ -132,6 +132,36 @@ def test_w4a16_linear_parity(fmt, shape):
     check_close(yb.float().cpu().numpy(), want["y"], want["abs_sum"], bf16_out=True)
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4, oracle.S_BLOCK])
+@pytest.mark.parametrize("shape", [(64, 256, 200), (300, 1152, 1336), (1056, 512, 1100)])
+def test_w16a4_linear_parity(shape, pattern, fmt):
+    """Activation-only quantization (Table 1, W16A4): quantizer + residual + selection as in the main path, GEMM
+    against plain bf16 weights (TMA straight into the MMA operand ring); contiguous and strided weights."""
+    m = rq()
+    M, K, N = shape
+    if pattern == oracle.S_BLOCK and M % 32:
+        pytest.skip("block pattern needs M % 32 == 0")
+    xb, wb = synth_xw(7 * M + N + pattern, M, K, N, n_out=max(1, K // 256))
+    want = oracle.w16a4_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern, fmt)
+    wbig = torch.zeros((N, K + 72), dtype=torch.bfloat16, device="cuda")
+    wbig[:, :K] = to_dev(wb)
+    for w in (to_dev(wb), wbig[:, :K]):
+        y = m.w16a4_linear(to_dev(xb), w, pattern, fmt, out_dtype=torch.float32)
+        torch.cuda.synchronize()
+        check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+    yb = m.w16a4_linear(to_dev(xb), to_dev(wb), pattern, fmt, out_dtype=torch.bfloat16)
+    check_close(yb.float().cpu().numpy(), want["y"], want["abs_sum"], bf16_out=True)
+
+
+def test_w16a4_rejects_bad_weights():
+    m = rq()
+    x = torch.zeros((64, 256), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((32, 260), dtype=torch.bfloat16, device="cuda")[:, :256]   # row pitch not a multiple of 8
+    with pytest.raises(m.ResqError):
+        m.w16a4_linear(x, w)
+
+
 # ----------------------------------------------------------------------------------------------
 # Every tile configuration of the GEMM on one shape that spans several tiles and ragged edges.
 # RESQ_GEMM_* are the library's debugging overrides of its tile heuristic (read at every call).

@@ -564,6 +564,38 @@ def test_w4a16_exact_rational_tiny_and_limit_of_the_residual_series(fmt):
         np.testing.assert_allclose(same["y"], oracle.w4a16_linear(xq, w, fmt)["y"], rtol=1e-13, atol=1e-13)
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+def test_w16a4_exact_rational_tiny_and_fixed_points(fmt):
+    """Activation-only ablation (Table 1): the product is the exact rational sum over the decoded activation codes
+    (and kept residual codes) and the weights as given; activations that are already decoded codes pass through
+    unchanged, so the result is then the plain product X W^T; and with identity weights the output is the decoded
+    operand itself."""
+    M, K, N = 3, 128, 4
+    x = gaussian_with_outliers(91, M, K, n_out=2, scale=16.0)
+    rng = np.random.default_rng(92)
+    w = bf16_round(rng.standard_normal((N, K)).astype(np.float32) * 0.02)
+    for pattern in (oracle.S_NONE, oracle.S_2_4, oracle.S_DENSE):
+        o = oracle.w16a4_linear(x, w, pattern, fmt)
+        av, wv = _to_frac(o["a"]), _to_frac(w.astype(np.float64))
+        rv = _to_frac(o["r_masked"]) if pattern != oracle.S_NONE else None
+        for m in range(M):
+            for n in range(N):
+                want = sum(av[m][k] * wv[n][k] for k in range(K))
+                if rv is not None:
+                    want += sum(rv[m][k] * wv[n][k] for k in range(K))
+                assert F(float(o["y"][m, n])) == want
+    xq = oracle.decode(fmt, *oracle.encode(fmt, x)).astype(np.float32)
+    if np.array_equal(oracle.decode(fmt, *oracle.encode(fmt, xq)), xq.astype(np.float64)):
+        o = oracle.w16a4_linear(xq, w, oracle.S_DENSE, fmt)
+        np.testing.assert_allclose(o["y"], xq.astype(np.float64) @ w.astype(np.float64).T, rtol=1e-13, atol=1e-13)
+    eye = np.eye(K, dtype=np.float32)
+    o = oracle.w16a4_linear(x, eye, oracle.S_2_4, fmt)
+    assert np.array_equal(o["y"], o["a"] + o["r_masked"])
+    # the weights really stay unquantized: a weight between two 4-bit codes changes W4A4 but not this path's use of it
+    w_off = bf16_round(w * np.float32(1.0078125))
+    assert not np.array_equal(oracle.w16a4_linear(x, w_off, oracle.S_NONE, fmt)["y"], oracle.w16a4_linear(x, w, oracle.S_NONE, fmt)["y"])
+
+
 # ----------------------------------------------------------------- regression digest of a seeded tensor
 
 def test_seeded_digest():

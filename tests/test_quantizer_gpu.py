@@ -112,9 +112,11 @@ def test_many_rows_per_warp(pattern):
     assert np.array_equal(got["mask"].cpu().numpy(), want["mask"])
 
 
-def test_residual_mask_ties_and_zero_rows():
-    # all-equal magnitudes: every selection is decided by the lower-index rule
-    M, K = 64, 256
+@pytest.mark.parametrize("shape", [(64, 256), (64, 2304), (32, 8448)])
+def test_residual_mask_ties_and_zero_rows(shape):
+    # all-equal magnitudes: every selection is decided by the lower-index rule (the channel scores of the wider
+    # shapes span several register rows of the small selection kernel, the widest takes the general one)
+    M, K = shape
     x = np.full((M, K), 0.75, dtype=np.float32)
     x[:, ::2] *= -1
     x[5] = 0
