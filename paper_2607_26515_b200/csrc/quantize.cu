@@ -112,13 +112,14 @@ __device__ __forceinline__ void fill_meta_pad(const QuantArgs& a, int64_t tid, i
 // first pass of the global ones (CHAN50, BLOCK: writes the unmasked residual and accumulates scores).
 // grid.y: groups of 8 warps, each warp owning 256 channels; grid.x: row chunks of `rows_per_cta`.
 // IMG: the bf16 images for the GEMM are written (a_bf16, and r_bf16 when RESIDUAL).
-template <int FMT, bool RESIDUAL, bool IMG>
+// COMP (2:4 only): the residual image leaves in compressed form with its index metadata (a.r_comp, a.r_meta).
+template <int FMT, bool RESIDUAL, bool IMG, bool COMP = false>
 __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int rows_per_cta) {
     pdl_wait();     // nothing below may touch global memory before the previous kernel of the stream is done
     pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
     if (a.clear_words && blockIdx.x == 0 && blockIdx.y == 0)
         for (int i = threadIdx.x; i < a.n_clear_words; i += blockDim.x) a.clear_words[i] = 0u;
-    if (RESIDUAL && IMG && a.r_comp)
+    if constexpr (COMP)
         fill_meta_pad(a, ((int64_t)blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x,
                       (int64_t)gridDim.x * gridDim.y * blockDim.x);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -197,8 +198,8 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
         uint32_t keep = 0xFFu;
         if (pattern == RESQ_S_2_4) keep = top2_mask8(roct);
         uint32_t comp0 = 0, comp1 = 0, idx_byte = 0;
-        if constexpr (IMG) {
-            if (a.r_comp) {  // (2:4 only) compressed image: 8 bytes per lane, and one byte of index pairs
+        if constexpr (COMP) {
+            {  // compressed image: 8 bytes per lane, and one byte of index pairs
                 uint32_t km[4], o[4], ia, ib;
                 keep_words(keep, km);
 #pragma unroll
@@ -249,7 +250,7 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
             const bool local = pattern == RESQ_S_DENSE || pattern == RESQ_S_2_4;
             if (a.mask_bits && local) a.mask_bits[m * (a.K / 8) + k0 / 8] = (uint8_t)keep;
             if constexpr (IMG) {
-              if (a.r_comp) {
+              if constexpr (COMP) {
                 *reinterpret_cast<uint2*>(a.r_comp + m * (a.K / 2) + k0 / 2) = make_uint2(comp0, comp1);
                 if ((lane & 1) == 0)
                     *reinterpret_cast<uint16_t*>(a.r_meta + sparse24_meta_offset(m, k0, a.meta_ka)) = (uint16_t)idx_byte;
@@ -477,14 +478,14 @@ __device__ __forceinline__ void encode_block(const uint32_t (&w)[32], uint32_t (
     else mxfp4_encode_block<DEQ, OCT>(w, codes, side, sink);
 }
 
-template <int FMT, bool RESIDUAL, bool IMG>
+template <int FMT, bool RESIDUAL, bool IMG, bool COMP = false>
 __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, int rows_per_warp) {
     pdl_wait();     // nothing below may touch global memory before the previous kernel of the stream is done
     pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
     if (a.clear_words && blockIdx.x == 0 && blockIdx.y == 0)
         for (int i = threadIdx.x; i < a.n_clear_words; i += blockDim.x) a.clear_words[i] = 0u;
-    const bool comp = RESIDUAL && IMG && a.r_comp != nullptr;  // 2:4: compressed residual image + index metadata
-    if (comp) fill_meta_pad(a, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, (int64_t)gridDim.x * blockDim.x);
+    constexpr bool comp = COMP;  // 2:4: compressed residual image + index metadata
+    if constexpr (comp) fill_meta_pad(a, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, (int64_t)gridDim.x * blockDim.x);
     extern __shared__ __align__(16) uint8_t smem_q[];
     constexpr int kBufs = IMG ? 3 : 2;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -616,7 +617,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
                         img[i] = (pack_bf16x2_exact(rdq[2 * i], rdq[2 * i + 1]) | (w[4 * c + i] & 0x80008000u)) & km[i];
-                    if (comp) {
+                    if constexpr (comp) {
                         uint32_t ia, ib;
                         const uint32_t c0 = compress24(img[0], img[1], keep & 15u, ia);
                         const uint32_t c1 = compress24(img[2], img[3], keep >> 4, ib);
@@ -659,7 +660,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
                 if (a.mask_bits && local) *reinterpret_cast<uint2*>(a.mask_bits + m * (a.K / 8) + blk * 8) = make_uint2(keep_lo, keep_hi);
             }
             if constexpr (IMG) {
-                if (comp) {
+                if constexpr (comp) {
                     if (active) {
                         // four 16-bit pieces (16 channels each); consecutive pieces alternate between the two halves
                         // of a metadata block's row group and advance one 32-bit word every second piece
@@ -1313,10 +1314,12 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
         };
         int rc;
         if (fmt == kHiF4)
-            rc = residual ? (img ? launch(quant_block_kernel<kHiF4, true, true>) : launch(quant_block_kernel<kHiF4, true, false>))
+            rc = residual ? (a.r_comp ? launch(quant_block_kernel<kHiF4, true, true, true>)
+                                      : img ? launch(quant_block_kernel<kHiF4, true, true>) : launch(quant_block_kernel<kHiF4, true, false>))
                           : (img ? launch(quant_block_kernel<kHiF4, false, true>) : launch(quant_block_kernel<kHiF4, false, false>));
         else
-            rc = residual ? (img ? launch(quant_block_kernel<kMXFP4, true, true>) : launch(quant_block_kernel<kMXFP4, true, false>))
+            rc = residual ? (a.r_comp ? launch(quant_block_kernel<kMXFP4, true, true, true>)
+                                      : img ? launch(quant_block_kernel<kMXFP4, true, true>) : launch(quant_block_kernel<kMXFP4, true, false>))
                           : (img ? launch(quant_block_kernel<kMXFP4, false, true>) : launch(quant_block_kernel<kMXFP4, false, false>));
         if (rc) return rc;
         if (global_sel) rc = launch_global_select(a, nscore, stream);
@@ -1331,10 +1334,12 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     const bool img = a.a_bf16 != nullptr;  // the GEMM path asks for both images (r_bf16 whenever there is a residual)
     auto launch = [&](void (*kern)(QuantArgs, int)) { launch_err = launch_kernel(kern, grid, dim3(kThreads), 0, stream, a, rows_per_cta); };
     if (fmt == kHiF4) {
-        if (residual) img ? launch(quant_stream_kernel<kHiF4, true, true>) : launch(quant_stream_kernel<kHiF4, true, false>);
+        if (residual && a.r_comp) launch(quant_stream_kernel<kHiF4, true, true, true>);
+        else if (residual) img ? launch(quant_stream_kernel<kHiF4, true, true>) : launch(quant_stream_kernel<kHiF4, true, false>);
         else img ? launch(quant_stream_kernel<kHiF4, false, true>) : launch(quant_stream_kernel<kHiF4, false, false>);
     } else {
-        if (residual) img ? launch(quant_stream_kernel<kMXFP4, true, true>) : launch(quant_stream_kernel<kMXFP4, true, false>);
+        if (residual && a.r_comp) launch(quant_stream_kernel<kMXFP4, true, true, true>);
+        else if (residual) img ? launch(quant_stream_kernel<kMXFP4, true, true>) : launch(quant_stream_kernel<kMXFP4, true, false>);
         else img ? launch(quant_stream_kernel<kMXFP4, false, true>) : launch(quant_stream_kernel<kMXFP4, false, false>);
     }
     }
