@@ -174,6 +174,23 @@ RESQ_API int mxfp4_w4a16_linear(const void* X_bf16, int64_t M, int64_t K, int64_
                        void* Y, int out_dtype, int64_t ldy,
                        void* workspace, size_t ws_bytes, void* stream);
 
+/* Down projection with its producer fused into the quantizer pass: the input is GU_bf16 = [gate | up], [M, 2K]
+ * device (row pitch ldgu >= 2K elements, ldgu % 8 == 0, 16-byte aligned base), the layer's activations are
+ * X = bf16(SiLU(gate) * up), formed on the fly and never written to memory; everything after that is
+ * *_resq_linear on X (Eq. (5)).  The rounding of X to bf16 decides 4-bit codes, so SiLU is evaluated by a fixed
+ * fp32 procedure (every operation rounded to nearest even, no fused multiply-add): t = g * (-log2 e) clamped to
+ * [-126, 126], n = rint(t), f = t - n, p = 2^f by the degree-6 Taylor polynomial of exp(f ln 2) in Horner form,
+ * e = p * 2^n, s = g / (1 + e), X = bf16(s * u).  All selections but RESQ_S_ROW50 (RESQ_ERR_PATTERN).  Workspace,
+ * output and errors as *_resq_linear with the same (M, N, K, pattern). */
+RESQ_API int hif4_swiglu_resq_linear(const void* GU_bf16, int64_t M, int64_t K, int64_t ldgu,
+                            const void* w_codes, const void* w_meta, int64_t N,
+                            int pattern, void* Y, int out_dtype, int64_t ldy,
+                            void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_swiglu_resq_linear(const void* GU_bf16, int64_t M, int64_t K, int64_t ldgu,
+                             const void* w_codes, const void* w_scale, int64_t N,
+                             int pattern, void* Y, int out_dtype, int64_t ldy,
+                             void* workspace, size_t ws_bytes, void* stream);
+
 /* Activation-only ablation of Table 1 ("W16A4"): Y = (deq Q(X) + S(deq Q(dX))) W^T with the weights in plain
  * bf16 (W_bf16: [N, K] device, row pitch ldw elements, ldw >= K, ldw % 8 == 0, 16-byte aligned base); the
  * activations go through the same quantizer, residual and selection as *_resq_linear (pattern RESQ_S_NONE gives

@@ -245,3 +245,54 @@ def w4a16_linear(x_f32: np.ndarray, w_f32: np.ndarray, fmt: str = "hif4", want_a
     y, ab = matmul(np.asarray(x_f32, dtype=np.float64), None, w, want_abs)
     return {"w_codes": w_codes, "w_side": w_side, "w": w, "y": y, "abs_sum": ab}
 
+
+# ---- fused producer of the down projection: x = SiLU(gate) * up, rounded to bf16, then the path above ---------
+# The paper applies the method to the linear layers of every transformer block; the input of the down projection is
+# SiLU(g) * u of the gate / up projection outputs.  Its rounding to bf16 decides 4-bit codes, so the evaluation is
+# fixed here operation by operation in fp32 (every operation rounded to nearest even, no fused multiply-add), the
+# precision the fused kernel works in:
+#   t = g * (-log2 e), clamped to [-126, 126];  n = rint(t);  f = t - n;
+#   p = 2^f by the degree-6 Taylor polynomial of exp(f ln 2) in Horner form;  e = p * 2^n  (= exp(-g));
+#   s = g / (1 + e);   x = bf16(s * u).
+_LOG2E_NEG = np.float32(-1.4426950408889634)
+_EXP2_COEF = [np.float32(c) for c in (1.0, 0.6931471805599453, 0.2402265069591007, 0.05550410866482158,
+                                       0.009618129107628477, 0.0013333558146428443, 0.00015403530393381608)]
+
+
+def silu32(g: np.ndarray) -> np.ndarray:
+    """SiLU(g) = g / (1 + exp(-g)) by the fixed fp32 procedure above (relative error about 2e-7)."""
+    g = np.asarray(g, dtype=np.float32)
+    t = np.multiply(g, _LOG2E_NEG, dtype=np.float32)
+    t = np.minimum(np.maximum(t, np.float32(-126.0)), np.float32(126.0))
+    n = np.rint(t).astype(np.float32)
+    f = np.subtract(t, n, dtype=np.float32)
+    p = np.full_like(f, _EXP2_COEF[6])
+    for c in reversed(_EXP2_COEF[:6]):
+        p = np.add(np.multiply(p, f, dtype=np.float32), c, dtype=np.float32)
+    scale = ((n.astype(np.int32) + 127) << 23).astype(np.uint32).view(np.float32)  # 2^n, exact
+    e = np.multiply(p, scale, dtype=np.float32)
+    d = np.add(np.float32(1.0), e, dtype=np.float32)
+    return np.divide(g, d, dtype=np.float32)
+
+
+def _bf16_rne(x: np.ndarray) -> np.ndarray:
+    b = np.asarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    b = (b + 0x7FFF + ((b >> 16) & 1)) & 0xFFFF0000
+    return b.astype(np.uint32).view(np.float32)
+
+
+def swiglu_bf16(g: np.ndarray, u: np.ndarray) -> np.ndarray:
+    """x = bf16(SiLU(g) * u) for bf16-valued g, u (finite)."""
+    s = silu32(g)
+    return _bf16_rne(np.multiply(s, np.asarray(u, dtype=np.float32), dtype=np.float32))
+
+
+def swiglu_resq_linear(gu_f32: np.ndarray, w_f32: np.ndarray, pattern: int, fmt: str = "hif4",
+                       want_abs: bool = True) -> Dict[str, np.ndarray]:
+    """Down projection with its producer: gu = [gate | up] ([M, 2K]); Eq. (5) on x = bf16(SiLU(gate) * up)."""
+    gu = np.asarray(gu_f32, dtype=np.float32)
+    K = gu.shape[1] // 2
+    x = swiglu_bf16(gu[:, :K], gu[:, K:])
+    out = resq_linear(x, w_f32, pattern, fmt, want_abs)
+    out["x"] = x
+    return out

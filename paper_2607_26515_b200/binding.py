@@ -47,6 +47,8 @@ SYMBOLS = {
     "resq_w4a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "hif4_w4a16_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
     "mxfp4_w4a16_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "hif4_swiglu_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "mxfp4_swiglu_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "hif4_w16a4_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "mxfp4_w16a4_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "resq_check": (_ci, [_vp, _vp]),
@@ -241,6 +243,30 @@ def w4a16_linear(X: torch.Tensor, w_codes: torch.Tensor, w_side: torch.Tensor, f
         workspace = alloc_workspace(int(lib().resq_w4a16_workspace_bytes(M, N, K)), X.device)
     _check(_fn(fmt, "hif4_w4a16_linear", "mxfp4_w4a16_linear")(
         X.data_ptr(), M, K, X.stride(0), w_codes.data_ptr(), w_side.data_ptr(), N, Y.data_ptr(),
+        OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32, Y.stride(0), workspace.data_ptr(), workspace.numel(),
+        _stream(stream)))
+    return Y
+
+
+def swiglu_resq_linear(GU: torch.Tensor, w_codes: torch.Tensor, w_side: torch.Tensor, pattern: int, fmt: str = "hif4",
+                       out_dtype: torch.dtype = torch.bfloat16, Y: Optional[torch.Tensor] = None,
+                       workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """*_swiglu_resq_linear: Eq. (5) on X = bf16(SiLU(gate) * up) with GU = [gate | up], X never stored."""
+    _require_bf16_matrix(GU, "GU")
+    M, K2 = GU.shape
+    K = K2 // 2
+    N = w_codes.shape[0]
+    if K2 % 2 or w_codes.shape[1] * 2 != K:
+        raise ValueError("GU must be [M, 2K] for weights packed as [N, K/2]")
+    if Y is None:
+        ld = (N + 7) // 8 * 8
+        Y = torch.empty((M, ld), dtype=out_dtype, device=GU.device)[:, :N]
+    if Y.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("Y must be bf16 or fp32")
+    if workspace is None:
+        workspace = alloc_workspace(resq_workspace_bytes(M, N, K, pattern, fmt), GU.device)
+    _check(_fn(fmt, "hif4_swiglu_resq_linear", "mxfp4_swiglu_resq_linear")(
+        GU.data_ptr(), M, K, GU.stride(0), w_codes.data_ptr(), w_side.data_ptr(), N, pattern, Y.data_ptr(),
         OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32, Y.stride(0), workspace.data_ptr(), workspace.numel(),
         _stream(stream)))
     return Y

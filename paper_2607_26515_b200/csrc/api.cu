@@ -210,9 +210,17 @@ size_t linear_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K, int patt
 // instead of the packed ones.
 int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_side, int64_t N,
            int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream,
-           const void* w_bf16 = nullptr, int64_t ldw = 0) {
+           const void* w_bf16 = nullptr, int64_t ldw = 0, bool swiglu = false) {
     int rc = check_matrix(X, M, K, ldx, fmt, "X");
     if (rc) return rc;
+    if (swiglu && ldx < 2 * K) {  // X is [gate | up]: 2K columns
+        set_last_error("swiglu: the input needs 2K columns per row (ldx=%lld, K=%lld)", (long long)ldx, (long long)K);
+        return RESQ_ERR_SHAPE;
+    }
+    if (swiglu && pattern == RESQ_S_ROW50) {
+        set_last_error("the fused SiLU * up producer does not support the row-wise selection");
+        return RESQ_ERR_PATTERN;
+    }
     rc = check_pattern(pattern, M);
     if (rc) return rc;
     if (w_bf16) {
@@ -250,6 +258,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     QuantArgs a;
     memset(&a, 0, sizeof(a));
     a.X = static_cast<const __nv_bfloat16*>(X);
+    if (swiglu) a.X_up = a.X + K;
     a.M = M;
     a.K = K;
     a.ldx = ldx;
@@ -262,7 +271,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     used += kWsFlags;
     // MXFP4 where it pays: the GEMM runs on the block-scaled FP4 pipe and takes packed codes and scales (they
     // fit into the space of the bf16 images; the selection zeroes dropped codes); otherwise exact bf16 images.
-    const bool native = !w_bf16 && fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K, pattern != RESQ_S_NONE);
+    const bool native = !w_bf16 && !swiglu && fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K, pattern != RESQ_S_NONE);
     uint8_t* region_a = ws + used;
     used += align_up((size_t)M * (size_t)K * 2, 256);
     uint8_t* region_r = nullptr;
@@ -271,7 +280,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
         used += residual_region_bytes(M, K, pattern);
     }
     // 2:4 on the CTA-pair kernel: the residual goes to the structured-sparse MMA in compressed form
-    const bool sparse24 = !w_bf16 && !native && pattern == RESQ_S_2_4 && gemm_sparse24_supported(M, N, K);
+    const bool sparse24 = !w_bf16 && !swiglu && !native && pattern == RESQ_S_2_4 && gemm_sparse24_supported(M, N, K);
     const size_t codes_bytes = align_up((size_t)M * (size_t)K / 2, 256);
     if (native) {
         a.x_codes = region_a;
@@ -446,6 +455,19 @@ int mxfp4_residual_mask(const void* X, int64_t M, int64_t K, int64_t ldx, int pa
                         void* r_codes, void* r_scale, void* mask_bits, void* workspace, size_t ws_bytes, void* stream) {
     return residual_mask(kMXFP4, X, M, K, ldx, pattern, x_codes, x_scale, r_codes, r_scale, mask_bits, workspace,
                          ws_bytes, stream);
+}
+
+int hif4_swiglu_resq_linear(const void* GU, int64_t M, int64_t K, int64_t ldgu, const void* w_codes, const void* w_meta,
+                            int64_t N, int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes,
+                            void* stream) {
+    return linear(kHiF4, GU, M, K, ldgu, w_codes, w_meta, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream, nullptr, 0,
+                  true);
+}
+int mxfp4_swiglu_resq_linear(const void* GU, int64_t M, int64_t K, int64_t ldgu, const void* w_codes, const void* w_scale,
+                             int64_t N, int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes,
+                             void* stream) {
+    return linear(kMXFP4, GU, M, K, ldgu, w_codes, w_scale, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream, nullptr,
+                  0, true);
 }
 
 int hif4_w16a4_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* W, int64_t N, int64_t ldw, int pattern,

@@ -74,6 +74,7 @@ inline cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, 
 // ---- quantizer launch description (quantize.cu) ------------------------------------------------
 struct QuantArgs {
     const __nv_bfloat16* X;
+    const __nv_bfloat16* X_up;  // non-null: fused producer, the input is bf16(SiLU(X) * X_up) (same M, K, ldx)
     int64_t M, K, ldx;
     int pattern;            // resq_pattern; RESQ_S_NONE => no residual work at all
     // canonical packed outputs (any may be null)

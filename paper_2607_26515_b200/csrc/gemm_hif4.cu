@@ -533,6 +533,10 @@ int env_int(const char* name, int dflt) {
 }
 
 // Pick the tile width and K split so that the persistent grid covers the 148 SMs evenly.
+// Calls with at most this many rows take the single-CTA kernel (one 128-row MMA tile); the CTA-pair kernel computes
+// 256-row tiles whatever M is (rows past M are zero-filled and never stored).
+int pair_min_m() { return env_int("RESQ_GEMM_PAIR_MIN_M", kBM); }
+
 TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res, bool sparse = false) {
     const int sms = 148;
     const int G = (int)(K / kBK);
@@ -574,7 +578,7 @@ TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res, bool sparse = 
     // (commit -> producers -> data landed -> MMA thread) takes, plus ~350 cycles of MMA-thread work between
     // k-blocks; a tile costs ~8000 cycles of fill and epilogue; a K split costs a second launch plus the
     // partial-tile traffic.
-    if (M > kBM && env_int("RESQ_GEMM_PAIR", 1)) {
+    if (M > pair_min_m() && env_int("RESQ_GEMM_PAIR", 1)) {
         const int64_t mtiles = (M + 2 * kBM - 1) / (2 * kBM);
         double best_pair = 1e300;
         for (int tn : {512, 480, 384, 320, 256, 128}) {
@@ -603,7 +607,7 @@ TileChoice choose_tile(int64_t M, int64_t N, int64_t K, bool res, bool sparse = 
     best.splits = env_int("RESQ_GEMM_SPLITS", best.splits);
     best.nt = env_int("RESQ_GEMM_NT", best.nt);
     best.pair_tn = env_int("RESQ_GEMM_PAIR_TN", best.pair_tn);
-    if (M <= kBM) best.pair_tn = 0;
+    if (M <= pair_min_m()) best.pair_tn = 0;
     if (res) best.mt = 1;
     return best;
 }
@@ -694,7 +698,7 @@ int launch_variant(const GemmArgs& g, const TileChoice& tc, cudaStream_t stream)
 // K-streamed schedule of the pair kernel: used when there are too few 256 x 256 output tiles to give every CTA
 // pair whole tiles (decode-sized M): the (tile, k-block) units are dealt out evenly instead.
 bool gemm_use_streamk(int64_t M, int64_t N, int64_t K) {
-    if (M <= kBM || !env_int("RESQ_GEMM_PAIR", 1)) return false;
+    if (M <= pair_min_m() || !env_int("RESQ_GEMM_PAIR", 1)) return false;
     const int force = env_int("RESQ_GEMM_STREAMK", -1);
     if (force >= 0) return force != 0;
     if (env_int("RESQ_GEMM_PAIR_TN", 0) || env_int("RESQ_GEMM_SPLITS", 0)) return false;  // explicit tile exploration
@@ -718,7 +722,7 @@ size_t gemm_hif4_scratch_bytes(int64_t M, int64_t N, int64_t K) {
     const int splits = gemm_hif4_pick_splits(M, N, K);
     if (splits > 1) classic = (size_t)splits * (size_t)M * (size_t)N * 4;
     // the K-streamed schedule may be switched on or off by the debugging overrides: size for both
-    const size_t sk = M > kBM ? gemm_pair_streamk_scratch_bytes() : 0;
+    const size_t sk = gemm_pair_streamk_scratch_bytes();
     return std::max(classic, sk);
 }
 

@@ -112,8 +112,41 @@ __device__ __forceinline__ void fill_meta_pad(const QuantArgs& a, int64_t tid, i
 // first pass of the global ones (CHAN50, BLOCK: writes the unmasked residual and accumulates scores).
 // grid.y: groups of 8 warps, each warp owning 256 channels; grid.x: row chunks of `rows_per_cta`.
 // IMG: the bf16 images for the GEMM are written (a_bf16, and r_bf16 when RESIDUAL).
+// Fused producer of the down projection: x = bf16(SiLU(g) * u).  Its rounding decides 4-bit codes, so the evaluation
+// is fixed operation by operation (fp32, round to nearest even, no contraction into fused multiply-adds):
+//   t = g * (-log2 e) clamped to [-126, 126]; n = rint(t); f = t - n; p = 2^f by the degree-6 Taylor polynomial of
+//   exp(f ln 2) in Horner form; e = p * 2^n (= exp(-g)); s = g / (1 + e); x = bf16(s * u).
+__device__ __forceinline__ float silu32(float g) {
+    float t = __fmul_rn(g, -1.4426950408889634f);
+    t = fminf(fmaxf(t, -126.0f), 126.0f);
+    const float n = rintf(t);
+    const float f = __fsub_rn(t, n);
+    float p = 0.00015403530393381608f;
+    p = __fadd_rn(__fmul_rn(p, f), 0.0013333558146428443f);
+    p = __fadd_rn(__fmul_rn(p, f), 0.009618129107628477f);
+    p = __fadd_rn(__fmul_rn(p, f), 0.05550410866482158f);
+    p = __fadd_rn(__fmul_rn(p, f), 0.2402265069591007f);
+    p = __fadd_rn(__fmul_rn(p, f), 0.6931471805599453f);
+    p = __fadd_rn(__fmul_rn(p, f), 1.0f);
+    const float e = __fmul_rn(p, __int_as_float(((int)n + 127) << 23));
+    return __fdiv_rn(g, __fadd_rn(1.0f, e));
+}
+__device__ __forceinline__ uint4 swiglu_bf16x8(const uint4& graw, const uint4& uraw) {
+    float g[8], u[8];
+    unpack_bf16x8(graw, g);
+    unpack_bf16x8(uraw, u);
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 v = __floats2bfloat162_rn(__fmul_rn(silu32(g[2 * i]), u[2 * i]), __fmul_rn(silu32(g[2 * i + 1]), u[2 * i + 1]));
+        o[i] = *reinterpret_cast<const uint32_t*>(&v);
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 // COMP (2:4 only): the residual image leaves in compressed form with its index metadata (a.r_comp, a.r_meta).
-template <int FMT, bool RESIDUAL, bool IMG, bool COMP = false>
+// PROD: the input is x = bf16(SiLU(g) * u) of a.X (g) and a.X_up (u), computed on the fly (never stored).
+template <int FMT, bool RESIDUAL, bool IMG, bool COMP = false, bool PROD = false>
 __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int rows_per_cta) {
     pdl_wait();     // nothing below may touch global memory before the previous kernel of the stream is done
     pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
@@ -139,11 +172,18 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
 #pragma unroll
     for (int i = 0; i < 8; ++i) chan_acc[i] = 0.0;
 
-    uint4 raw = make_uint4(0, 0, 0, 0);
-    if (active && m_begin < m_end) raw = ld_nc_16(a.X + m_begin * a.ldx + k0);
+    uint4 raw = make_uint4(0, 0, 0, 0), raw_up = make_uint4(0, 0, 0, 0);
+    if (active && m_begin < m_end) {
+        raw = ld_nc_16(a.X + m_begin * a.ldx + k0);
+        if constexpr (PROD) raw_up = ld_nc_16(a.X_up + m_begin * a.ldx + k0);
+    }
     for (int64_t m = m_begin; m < m_end; ++m) {
-        const uint4 cur = raw;
-        if (active && m + 1 < m_end) raw = ld_nc_16(a.X + (m + 1) * a.ldx + k0);  // prefetch the next row
+        uint4 cur = raw;
+        if constexpr (PROD) cur = swiglu_bf16x8(raw, raw_up);
+        if (active && m + 1 < m_end) {  // prefetch the next row
+            raw = ld_nc_16(a.X + (m + 1) * a.ldx + k0);
+            if constexpr (PROD) raw_up = ld_nc_16(a.X_up + (m + 1) * a.ldx + k0);
+        }
         const uint32_t w[4] = {cur.x, cur.y, cur.z, cur.w};
         float x[8], deq[8];
         unpack_bf16x8(cur, x);
@@ -1252,6 +1292,10 @@ static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t
 int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     const int pattern = a.pattern;
     const bool residual = pattern != RESQ_S_NONE;
+    if (pattern == RESQ_S_ROW50 && a.X_up) {
+        set_last_error("the fused SiLU * up producer does not support the row-wise selection");
+        return RESQ_ERR_PATTERN;
+    }
     if (pattern == RESQ_S_ROW50) {
         // a warp per row with the block-per-lane encoders, if the row's image fits next to the staging tiles
         auto al16r = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
@@ -1296,7 +1340,7 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     // Worth it once there is a warp task (32 blocks of one row) for every warp slot of the machine; below
     // that the finer-grained kernel (a lane per 8 values) finishes sooner.
     const int64_t block_tasks = a.M * ((a.K / kHif4Block + 31) / 32);
-    if (pattern != RESQ_S_CHAN50 && a.K % kHif4Block == 0 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
+    if (!a.X_up && pattern != RESQ_S_CHAN50 && a.K % kHif4Block == 0 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
         al16(a.a_bf16) && al16(a.r_bf16) && al16(a.r_comp)) {
         const bool img = a.a_bf16 != nullptr;
         const int64_t ncg = (a.K / kHif4Block + 31) / 32;
@@ -1333,7 +1377,14 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     LaunchScope scope(kKindQuant, stream);
     const bool img = a.a_bf16 != nullptr;  // the GEMM path asks for both images (r_bf16 whenever there is a residual)
     auto launch = [&](void (*kern)(QuantArgs, int)) { launch_err = launch_kernel(kern, grid, dim3(kThreads), 0, stream, a, rows_per_cta); };
-    if (fmt == kHiF4) {
+    if (a.X_up) {  // fused producer: GEMM-feeding variants only
+        if (!img || a.r_comp) {
+            set_last_error("internal: the fused producer feeds the dense GEMM operand images only");
+            return RESQ_ERR_CUDA;
+        }
+        if (fmt == kHiF4) residual ? launch(quant_stream_kernel<kHiF4, true, true, false, true>) : launch(quant_stream_kernel<kHiF4, false, true, false, true>);
+        else residual ? launch(quant_stream_kernel<kMXFP4, true, true, false, true>) : launch(quant_stream_kernel<kMXFP4, false, true, false, true>);
+    } else if (fmt == kHiF4) {
         if (residual && a.r_comp) launch(quant_stream_kernel<kHiF4, true, true, true>);
         else if (residual) img ? launch(quant_stream_kernel<kHiF4, true, true>) : launch(quant_stream_kernel<kHiF4, true, false>);
         else img ? launch(quant_stream_kernel<kHiF4, false, true>) : launch(quant_stream_kernel<kHiF4, false, false>);

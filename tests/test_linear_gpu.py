@@ -154,6 +154,51 @@ def test_w16a4_linear_parity(shape, pattern, fmt):
     check_close(yb.float().cpu().numpy(), want["y"], want["abs_sum"], bf16_out=True)
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4, oracle.S_CHAN50, oracle.S_BLOCK])
+@pytest.mark.parametrize("shape", [(64, 256, 200), (320, 1152, 520)])
+def test_swiglu_fused_producer(shape, pattern, fmt):
+    """Down projection with SiLU(gate) * up folded into the quantizer pass: within tolerance of the oracle, and
+    bit-identical to the unfused call on the oracle's bf16 activations (so the fused producer rounds every
+    activation exactly as the fixed procedure says, extremes included)."""
+    m = rq()
+    M, K, N = shape
+    rng = np.random.default_rng(1000 * M + K + pattern)
+    gu = rng.standard_normal((M, 2 * K)).astype(np.float32) * 2.5
+    gu[0, :16] = [0.0, -0.0, 100.0, -100.0, 88.0, -88.0, 1e-20, -1e-20, 30.0, -30.0, 0.5, -0.5, 7.0, -7.0, 3e4, -3e4]
+    gu[1, K:K + 8] = [0.0, -0.0, 1e-30, -3e4, 3e4, 1.0, -1.0, 2.0 ** -126]
+    gub = f32_to_bf16_bits(gu)
+    _, wb = synth_xw(9 * M + N, 8, K, N, n_out=1)
+    want = oracle.swiglu_resq_linear(bf16_bits_to_f32(gub), bf16_bits_to_f32(wb), pattern, fmt)
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    import os
+    old = os.environ.get("RESQ_MXFP4_NATIVE")
+    os.environ["RESQ_MXFP4_NATIVE"] = "0"   # the unfused reference call takes the same GEMM route as the fused one
+    try:
+        y = m.swiglu_resq_linear(to_dev(gub), wc, ws, pattern, fmt, out_dtype=torch.float32)
+        x_dev = to_dev(f32_to_bf16_bits(want["x"]))
+        y_unfused = m.resq_linear(x_dev, wc, ws, pattern, fmt, out_dtype=torch.float32)
+        torch.cuda.synchronize()
+    finally:
+        if old is None:
+            os.environ.pop("RESQ_MXFP4_NATIVE", None)
+        else:
+            os.environ["RESQ_MXFP4_NATIVE"] = old
+    check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+    assert torch.equal(y, y_unfused)
+
+
+def test_swiglu_rejects_row50_and_narrow_input():
+    m = rq()
+    gu = torch.zeros((64, 512), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((32, 256), dtype=torch.bfloat16, device="cuda")
+    wc, ws = m.pack_weight(w)
+    with pytest.raises(m.ResqError):
+        m.swiglu_resq_linear(gu, wc, ws, m.S_ROW50)
+    with pytest.raises((m.ResqError, ValueError)):
+        m.swiglu_resq_linear(gu[:, :256], wc, ws, m.S_NONE)     # weights say K = 256 but only 256 columns of [gate | up]
+
+
 def test_w16a4_rejects_bad_weights():
     m = rq()
     x = torch.zeros((64, 256), dtype=torch.bfloat16, device="cuda")

@@ -596,6 +596,36 @@ def test_w16a4_exact_rational_tiny_and_fixed_points(fmt):
     assert not np.array_equal(oracle.w16a4_linear(x, w_off, oracle.S_NONE, fmt)["y"], oracle.w16a4_linear(x, w, oracle.S_NONE, fmt)["y"])
 
 
+def test_swiglu_producer_fixed_procedure():
+    """Fused producer of the down projection: SiLU by the fixed fp32 procedure agrees with the closed form
+    g / (1 + exp(-g)) in fp64 to fp32 accuracy; exact special cases; the product with `up` is a bf16 value; and the
+    fused layer is Eq. (5) on exactly that tensor."""
+    g = np.concatenate([np.linspace(-30, 30, 20001), np.random.default_rng(5).standard_normal(20000) * 4]).astype(np.float32)
+    g = bf16_round(g)
+    s = oracle.silu32(g).astype(np.float64)
+    ref = g.astype(np.float64) / (1.0 + np.exp(-g.astype(np.float64)))
+    assert np.all(np.abs(s - ref) <= 3e-6 * np.abs(ref) + 1e-37)
+    assert oracle.silu32(np.float32(0.0)) == 0.0
+    big = np.array([90.0, 128.0, 3.0e4], dtype=np.float32)
+    assert np.array_equal(oracle.silu32(big), big)                    # exp(-g) vanishes against 1
+    tiny = oracle.silu32(np.array([-90.0, -1.0e3], dtype=np.float32))
+    assert np.all(tiny <= 0) and np.all(tiny > -1e-30)                # saturates at g * 2^-126
+    assert np.all(np.diff(oracle.silu32(np.linspace(-1.0, 30, 4001).astype(np.float32))) >= 0)   # monotone right of the minimum
+    u = bf16_round(np.random.default_rng(6).standard_normal(g.shape).astype(np.float32))
+    x = oracle.swiglu_bf16(g, u)
+    assert np.array_equal(bf16_round(x), x)
+    exact = ref * u.astype(np.float64)
+    assert np.all(np.abs(x - exact) <= 2.0 ** -8 * np.abs(exact) + 1e-37)   # half a bf16 ulp plus the fp32 error
+    one = oracle.swiglu_bf16(g, np.ones_like(g))
+    assert np.array_equal(one, bf16_round(oracle.silu32(g)))
+    M, K, N = 4, 128, 3
+    gu = bf16_round(np.random.default_rng(7).standard_normal((M, 2 * K)).astype(np.float32) * 2)
+    w = bf16_round(np.random.default_rng(8).standard_normal((N, K)).astype(np.float32) * 0.02)
+    o = oracle.swiglu_resq_linear(gu, w, oracle.S_2_4)
+    assert np.array_equal(o["x"], oracle.swiglu_bf16(gu[:, :K], gu[:, K:]))
+    assert np.array_equal(o["y"], oracle.resq_linear(o["x"], w, oracle.S_2_4)["y"])
+
+
 # ----------------------------------------------------------------- regression digest of a seeded tensor
 
 def test_seeded_digest():
