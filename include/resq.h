@@ -191,6 +191,25 @@ RESQ_API int mxfp4_swiglu_resq_linear(const void* GU_bf16, int64_t M, int64_t K,
                              int pattern, void* Y, int out_dtype, int64_t ldy,
                              void* workspace, size_t ws_bytes, void* stream);
 
+/* Projection with its RMSNorm producer fused into the quantizer pass (qkv / gate_up inputs): H_bf16 [M, K] device
+ * (row pitch ldh), gamma_bf16 [K] device (16-byte aligned), the layer's activations are
+ * X[m,k] = bf16((H[m,k] * r[m]) * gamma[k]), r[m] = 1 / sqrt(sum_k H[m,k]^2 / K + eps), formed on the fly and
+ * never written to memory; everything after that is *_resq_linear on X.  Fixed evaluation: the sum of squares is
+ * the exact sum rounded once to fp32 (realised by a fixed-order fp64 sum of the exact squares), every later
+ * operation is correctly rounded fp32 (division, square root, division, two multiplies), no fused multiply-add.
+ * A small row kernel computes r (kept in the workspace) before the quantizer kernel.  All selections but
+ * RESQ_S_ROW50.  Workspace, output and errors as *_resq_linear with the same (M, N, K, pattern). */
+RESQ_API int hif4_rmsnorm_resq_linear(const void* H_bf16, int64_t M, int64_t K, int64_t ldh,
+                             const void* gamma_bf16, float eps,
+                             const void* w_codes, const void* w_meta, int64_t N,
+                             int pattern, void* Y, int out_dtype, int64_t ldy,
+                             void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_rmsnorm_resq_linear(const void* H_bf16, int64_t M, int64_t K, int64_t ldh,
+                              const void* gamma_bf16, float eps,
+                              const void* w_codes, const void* w_scale, int64_t N,
+                              int pattern, void* Y, int out_dtype, int64_t ldy,
+                              void* workspace, size_t ws_bytes, void* stream);
+
 /* Activation-only ablation of Table 1 ("W16A4"): Y = (deq Q(X) + S(deq Q(dX))) W^T with the weights in plain
  * bf16 (W_bf16: [N, K] device, row pitch ldw elements, ldw >= K, ldw % 8 == 0, 16-byte aligned base); the
  * activations go through the same quantizer, residual and selection as *_resq_linear (pattern RESQ_S_NONE gives

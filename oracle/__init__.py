@@ -296,3 +296,35 @@ def swiglu_resq_linear(gu_f32: np.ndarray, w_f32: np.ndarray, pattern: int, fmt:
     out = resq_linear(x, w_f32, pattern, fmt, want_abs)
     out["x"] = x
     return out
+
+
+# ---- fused producer of the qkv / gate_up projections: x = RMSNorm(h) * gamma, rounded to bf16 -------------------
+# Fixed evaluation (fp32, every operation rounded to nearest even): ss = the exact sum of squares of the row (the
+# squares of bf16 values are exact; the sum is taken exactly and rounded once to fp32), ms = ss / K, v = ms + eps,
+# r = 1 / sqrt(v) as a correctly rounded square root followed by a correctly rounded division, and
+# x[k] = bf16((h[k] * r) * gamma[k]).
+def rmsnorm_row_scale(h: np.ndarray, eps: float) -> np.ndarray:
+    import math
+    h = np.asarray(h, dtype=np.float32)
+    K = h.shape[1]
+    ss = np.array([math.fsum((float(v) * float(v) for v in row)) for row in h], dtype=np.float64).astype(np.float32)
+    ms = np.divide(ss, np.float32(K), dtype=np.float32)
+    v = np.add(ms, np.float32(eps), dtype=np.float32)
+    return np.divide(np.float32(1.0), np.sqrt(v, dtype=np.float32), dtype=np.float32)
+
+
+def rmsnorm_bf16(h: np.ndarray, gamma: np.ndarray, eps: float) -> np.ndarray:
+    """x = bf16((h * r_row) * gamma) for bf16-valued h [M, K] and gamma [K]."""
+    h = np.asarray(h, dtype=np.float32)
+    r = rmsnorm_row_scale(h, eps)
+    t = np.multiply(h, r[:, None], dtype=np.float32)
+    return _bf16_rne(np.multiply(t, np.asarray(gamma, dtype=np.float32)[None, :], dtype=np.float32))
+
+
+def rmsnorm_resq_linear(h_f32: np.ndarray, gamma_f32: np.ndarray, eps: float, w_f32: np.ndarray, pattern: int,
+                        fmt: str = "hif4", want_abs: bool = True) -> Dict[str, np.ndarray]:
+    """Projection with its RMSNorm producer: Eq. (5) on x = bf16(RMSNorm(h) * gamma)."""
+    x = rmsnorm_bf16(h_f32, gamma_f32, eps)
+    out = resq_linear(x, w_f32, pattern, fmt, want_abs)
+    out["x"] = x
+    return out

@@ -49,6 +49,8 @@ SYMBOLS = {
     "mxfp4_w4a16_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
     "hif4_swiglu_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "mxfp4_swiglu_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "hif4_rmsnorm_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, ctypes.c_float, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "mxfp4_rmsnorm_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, ctypes.c_float, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "hif4_w16a4_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "mxfp4_w16a4_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "resq_check": (_ci, [_vp, _vp]),
@@ -269,6 +271,29 @@ def swiglu_resq_linear(GU: torch.Tensor, w_codes: torch.Tensor, w_side: torch.Te
         GU.data_ptr(), M, K, GU.stride(0), w_codes.data_ptr(), w_side.data_ptr(), N, pattern, Y.data_ptr(),
         OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32, Y.stride(0), workspace.data_ptr(), workspace.numel(),
         _stream(stream)))
+    return Y
+
+
+def rmsnorm_resq_linear(H: torch.Tensor, gamma: torch.Tensor, eps: float, w_codes: torch.Tensor, w_side: torch.Tensor,
+                        pattern: int, fmt: str = "hif4", out_dtype: torch.dtype = torch.bfloat16,
+                        Y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """*_rmsnorm_resq_linear: Eq. (5) on X = bf16(RMSNorm(H) * gamma), X never stored."""
+    _require_bf16_matrix(H, "H")
+    M, K = H.shape
+    N = w_codes.shape[0]
+    if gamma.dtype != torch.bfloat16 or gamma.numel() != K or not gamma.is_contiguous():
+        raise ValueError("gamma must be a contiguous bf16 vector of K elements")
+    if Y is None:
+        ld = (N + 7) // 8 * 8
+        Y = torch.empty((M, ld), dtype=out_dtype, device=H.device)[:, :N]
+    if Y.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("Y must be bf16 or fp32")
+    if workspace is None:
+        workspace = alloc_workspace(resq_workspace_bytes(M, N, K, pattern, fmt), H.device)
+    _check(_fn(fmt, "hif4_rmsnorm_resq_linear", "mxfp4_rmsnorm_resq_linear")(
+        H.data_ptr(), M, K, H.stride(0), gamma.data_ptr(), float(eps), w_codes.data_ptr(), w_side.data_ptr(), N, pattern,
+        Y.data_ptr(), OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32, Y.stride(0), workspace.data_ptr(),
+        workspace.numel(), _stream(stream)))
     return Y
 
 

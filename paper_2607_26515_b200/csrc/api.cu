@@ -200,6 +200,7 @@ size_t residual_region_bytes(int64_t M, int64_t K, int pattern) {
 size_t linear_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K, int pattern) {
     if (M <= 0 || N <= 0 || K <= 0) return 0;
     size_t b = kWsHeader + kWsFlags + quant_scratch_bytes(M, K, pattern);
+    b += align_up((size_t)M * sizeof(float), 256);                            // row scales of the fused RMSNorm producer
     b += align_up((size_t)M * (size_t)K * 2, 256);                            // bf16 image of deq Q(X)
     b += residual_region_bytes(M, K, pattern);
     b += align_up(gemm_hif4_scratch_bytes(M, N, K), 256);                     // fp32 partial tiles of a K split
@@ -210,16 +211,20 @@ size_t linear_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K, int patt
 // instead of the packed ones.
 int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_side, int64_t N,
            int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream,
-           const void* w_bf16 = nullptr, int64_t ldw = 0, bool swiglu = false) {
+           const void* w_bf16 = nullptr, int64_t ldw = 0, bool swiglu = false, const void* gamma = nullptr, float eps = 0.0f) {
     int rc = check_matrix(X, M, K, ldx, fmt, "X");
     if (rc) return rc;
     if (swiglu && ldx < 2 * K) {  // X is [gate | up]: 2K columns
         set_last_error("swiglu: the input needs 2K columns per row (ldx=%lld, K=%lld)", (long long)ldx, (long long)K);
         return RESQ_ERR_SHAPE;
     }
-    if (swiglu && pattern == RESQ_S_ROW50) {
-        set_last_error("the fused SiLU * up producer does not support the row-wise selection");
+    if ((swiglu || gamma) && pattern == RESQ_S_ROW50) {
+        set_last_error("the fused producers do not support the row-wise selection");
         return RESQ_ERR_PATTERN;
+    }
+    if (gamma && (!aligned16(gamma) || !(eps >= 0.0f))) {
+        set_last_error("rmsnorm: gamma needs a 16-byte aligned base and eps must be >= 0");
+        return RESQ_ERR_ALIGN;
     }
     rc = check_pattern(pattern, M);
     if (rc) return rc;
@@ -269,9 +274,15 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     a.clear_words = reinterpret_cast<uint32_t*>(ws);  // cleared by the quantizer kernel: no separate memset node
     a.n_clear_words = (int)((kWsHeader + kWsFlags) / 4);
     used += kWsFlags;
+    if (gamma) {
+        a.gamma = static_cast<const __nv_bfloat16*>(gamma);
+        a.eps = eps;
+        a.row_scale = reinterpret_cast<float*>(ws + used);
+    }
+    used += align_up((size_t)M * sizeof(float), 256);
     // MXFP4 where it pays: the GEMM runs on the block-scaled FP4 pipe and takes packed codes and scales (they
     // fit into the space of the bf16 images; the selection zeroes dropped codes); otherwise exact bf16 images.
-    const bool native = !w_bf16 && !swiglu && fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K, pattern != RESQ_S_NONE);
+    const bool native = !w_bf16 && !swiglu && !gamma && fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K, pattern != RESQ_S_NONE);
     uint8_t* region_a = ws + used;
     used += align_up((size_t)M * (size_t)K * 2, 256);
     uint8_t* region_r = nullptr;
@@ -280,7 +291,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
         used += residual_region_bytes(M, K, pattern);
     }
     // 2:4 on the CTA-pair kernel: the residual goes to the structured-sparse MMA in compressed form
-    const bool sparse24 = !w_bf16 && !swiglu && !native && pattern == RESQ_S_2_4 && gemm_sparse24_supported(M, N, K);
+    const bool sparse24 = !w_bf16 && !swiglu && !gamma && !native && pattern == RESQ_S_2_4 && gemm_sparse24_supported(M, N, K);
     const size_t codes_bytes = align_up((size_t)M * (size_t)K / 2, 256);
     if (native) {
         a.x_codes = region_a;
@@ -468,6 +479,27 @@ int mxfp4_swiglu_resq_linear(const void* GU, int64_t M, int64_t K, int64_t ldgu,
                              void* stream) {
     return linear(kMXFP4, GU, M, K, ldgu, w_codes, w_scale, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream, nullptr,
                   0, true);
+}
+
+int hif4_rmsnorm_resq_linear(const void* H, int64_t M, int64_t K, int64_t ldh, const void* gamma, float eps, const void* w_codes,
+                             const void* w_meta, int64_t N, int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace,
+                             size_t ws_bytes, void* stream) {
+    if (!gamma) {
+        set_last_error("rmsnorm_resq_linear: NULL gamma");
+        return RESQ_ERR_NULL;
+    }
+    return linear(kHiF4, H, M, K, ldh, w_codes, w_meta, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream, nullptr, 0,
+                  false, gamma, eps);
+}
+int mxfp4_rmsnorm_resq_linear(const void* H, int64_t M, int64_t K, int64_t ldh, const void* gamma, float eps, const void* w_codes,
+                              const void* w_scale, int64_t N, int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace,
+                              size_t ws_bytes, void* stream) {
+    if (!gamma) {
+        set_last_error("rmsnorm_resq_linear: NULL gamma");
+        return RESQ_ERR_NULL;
+    }
+    return linear(kMXFP4, H, M, K, ldh, w_codes, w_scale, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream, nullptr, 0,
+                  false, gamma, eps);
 }
 
 int hif4_w16a4_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* W, int64_t N, int64_t ldw, int pattern,

@@ -75,6 +75,11 @@ inline cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, 
 struct QuantArgs {
     const __nv_bfloat16* X;
     const __nv_bfloat16* X_up;  // non-null: fused producer, the input is bf16(SiLU(X) * X_up) (same M, K, ldx)
+    // non-null: fused RMSNorm producer, the input is bf16((X * row_scale[m]) * gamma[k]); row_scale [M] fp32 is
+    // written by the row kernel that launch_quantize runs first (1 / sqrt(mean(X^2) + eps))
+    const __nv_bfloat16* gamma;
+    float* row_scale;
+    float eps;
     int64_t M, K, ldx;
     int pattern;            // resq_pattern; RESQ_S_NONE => no residual work at all
     // canonical packed outputs (any may be null)

@@ -12,7 +12,8 @@
 // "full" barriers collect arrivals from both CTAs; "empty" barriers are released in both CTAs by a commit
 // multicast.  Two schedules: whole tiles per pair (optionally with a K split and a separate reduce kernel), or
 // K-streamed (the k-blocks of few tiles dealt out evenly; partial tiles go to fp32 slots and are summed in a
-// fixed order at the end of the same kernel).
+// fixed order at the end of the same kernel).  Residual term: a second dense A operand, or (2:4) the compressed
+// operand on the structured-sparse MMA.  Weights: packed 4-bit codes expanded here, or plain bf16 by TMA.
 #include "common.cuh"
 #include "ptx.cuh"
 #include "expand.cuh"
@@ -30,11 +31,11 @@ constexpr int kBM = 128;
 constexpr int kBK = 64;
 constexpr int kMaxBN = 256;
 constexpr int kGroupWarps = 4;                       // expander warps per group
-// Expander groups take k-blocks round-robin; k-block it uses slot it mod depth of each of the three rings
-// (activation stages, raw codes, expanded weights; the depths are at least NG, see launch_pair_variant).  The
-// number of groups NG (four warps each) is a template
-// parameter of the kernel: more groups tolerate more hand-off latency, fewer groups fit wider tiles into
-// shared memory (three slots of a 512-wide tile with a residual operand take 216 KB).
+// Expander groups take k-blocks round-robin; k-block i uses slot i mod depth of each of the three rings
+// (activation stages, raw codes, expanded weights; depths of at least NG, chosen in launch_pair_variant).  The
+// number of groups NG (four warps each) is a template parameter of the kernel: more groups tolerate more
+// hand-off latency, fewer groups fit wider tiles into shared memory (three slots of a 512-wide tile with a
+// residual operand take 216 KB).
 constexpr int kFirstEpiWarp = 4;
 constexpr int kFirstExpWarp = 8;
 constexpr int pair_threads(int groups) { return 32 * (kFirstExpWarp + kGroupWarps * groups); }

@@ -87,15 +87,6 @@ __device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, v
     return false;
 }
 
-// Warp-collective bounded wait: lane 0 polls, the outcome is broadcast.  Keeps the number of threads that
-// hammer the barrier (and the shared-memory pipe) at one per warp.  All 32 lanes must call it.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    int ok = 0;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
-    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-    return ok != 0;
-}
-
 // Read-only global loads that stay where they are written: the compiler must not sink them to their first
 // use (they are issued one k-block ahead precisely to hide their latency).
 __device__ __forceinline__ uint32_t ld_nc_u32(const uint32_t* p) {

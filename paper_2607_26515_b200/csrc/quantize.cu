@@ -144,9 +144,37 @@ __device__ __forceinline__ uint4 swiglu_bf16x8(const uint4& graw, const uint4& u
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
+// Fused RMSNorm producer, first kernel: r[m] = 1 / sqrt(sum_k X[m,k]^2 / K + eps).  The squares of bf16 values are
+// exact; a warp sums its row in fp64 in a fixed order (lane-strided partial sums, then a shuffle tree), which is
+// the exact sum except beyond 2^-40 relative; everything after the one rounding to fp32 is correctly rounded fp32.
+__global__ void __launch_bounds__(256) rmsnorm_row_scale_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int64_t ldx,
+                                                                float eps, float* __restrict__ row_scale) {
+    pdl_wait();
+    pdl_trigger();
+    const int lane = threadIdx.x & 31;
+    const int64_t m = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (m >= M) return;
+    const __nv_bfloat16* row = X + m * ldx;
+    double acc = 0.0;
+    for (int64_t k = (int64_t)lane * 8; k < K; k += 256) {  // K is a multiple of 32, rows are 16-byte aligned
+        float x[8];
+        unpack_bf16x8(ld_nc_16(row + k), x);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc += (double)x[i] * (double)x[i];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    if (lane == 0) {
+        const float ss = (float)acc;  // round to nearest
+        const float v = __fadd_rn(__fdiv_rn(ss, (float)K), eps);
+        row_scale[m] = __fdiv_rn(1.0f, __fsqrt_rn(v));
+    }
+}
+
 // COMP (2:4 only): the residual image leaves in compressed form with its index metadata (a.r_comp, a.r_meta).
-// PROD: the input is x = bf16(SiLU(g) * u) of a.X (g) and a.X_up (u), computed on the fly (never stored).
-template <int FMT, bool RESIDUAL, bool IMG, bool COMP = false, bool PROD = false>
+// PROD = 1: the input is x = bf16(SiLU(g) * u) of a.X (g) and a.X_up (u); PROD = 2: x = bf16((X * r[m]) * gamma[k])
+// with the row scales of rmsnorm_row_scale_kernel; computed on the fly, never stored.
+template <int FMT, bool RESIDUAL, bool IMG, bool COMP = false, int PROD = 0>
 __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int rows_per_cta) {
     pdl_wait();     // nothing below may touch global memory before the previous kernel of the stream is done
     pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
@@ -173,16 +201,35 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
     for (int i = 0; i < 8; ++i) chan_acc[i] = 0.0;
 
     uint4 raw = make_uint4(0, 0, 0, 0), raw_up = make_uint4(0, 0, 0, 0);
+    float gam[8];
+    if constexpr (PROD == 2) {
+        if (active) unpack_bf16x8(ld_nc_16(a.gamma + k0), gam);
+    }
     if (active && m_begin < m_end) {
         raw = ld_nc_16(a.X + m_begin * a.ldx + k0);
-        if constexpr (PROD) raw_up = ld_nc_16(a.X_up + m_begin * a.ldx + k0);
+        if constexpr (PROD == 1) raw_up = ld_nc_16(a.X_up + m_begin * a.ldx + k0);
     }
     for (int64_t m = m_begin; m < m_end; ++m) {
         uint4 cur = raw;
-        if constexpr (PROD) cur = swiglu_bf16x8(raw, raw_up);
+        if constexpr (PROD == 1) cur = swiglu_bf16x8(raw, raw_up);
+        if constexpr (PROD == 2) {
+            if (active) {
+                const float r = a.row_scale[m];
+                float h[8];
+                unpack_bf16x8(raw, h);
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const __nv_bfloat162 v = __floats2bfloat162_rn(__fmul_rn(__fmul_rn(h[2 * i], r), gam[2 * i]),
+                                                                   __fmul_rn(__fmul_rn(h[2 * i + 1], r), gam[2 * i + 1]));
+                    o[i] = *reinterpret_cast<const uint32_t*>(&v);
+                }
+                cur = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
         if (active && m + 1 < m_end) {  // prefetch the next row
             raw = ld_nc_16(a.X + (m + 1) * a.ldx + k0);
-            if constexpr (PROD) raw_up = ld_nc_16(a.X_up + (m + 1) * a.ldx + k0);
+            if constexpr (PROD == 1) raw_up = ld_nc_16(a.X_up + (m + 1) * a.ldx + k0);
         }
         const uint32_t w[4] = {cur.x, cur.y, cur.z, cur.w};
         float x[8], deq[8];
@@ -1292,9 +1339,16 @@ static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t
 int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     const int pattern = a.pattern;
     const bool residual = pattern != RESQ_S_NONE;
-    if (pattern == RESQ_S_ROW50 && a.X_up) {
-        set_last_error("the fused SiLU * up producer does not support the row-wise selection");
+    if (pattern == RESQ_S_ROW50 && (a.X_up || a.gamma)) {
+        set_last_error("the fused producers do not support the row-wise selection");
         return RESQ_ERR_PATTERN;
+    }
+    if (a.gamma) {  // row scales first (the quantizer kernel waits for them through the programmatic dependency)
+        LaunchScope scope(kKindQuant, stream);
+        int rc0 = cuda_fail(launch_kernel(rmsnorm_row_scale_kernel, dim3((unsigned)((a.M + 7) / 8)), dim3(256), 0, stream, a.X, a.M, a.K,
+                                          a.ldx, a.eps, a.row_scale),
+                            "rmsnorm_row_scale_kernel launch");
+        if (rc0) return rc0;
     }
     if (pattern == RESQ_S_ROW50) {
         // a warp per row with the block-per-lane encoders, if the row's image fits next to the staging tiles
@@ -1340,7 +1394,7 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     // Worth it once there is a warp task (32 blocks of one row) for every warp slot of the machine; below
     // that the finer-grained kernel (a lane per 8 values) finishes sooner.
     const int64_t block_tasks = a.M * ((a.K / kHif4Block + 31) / 32);
-    if (!a.X_up && pattern != RESQ_S_CHAN50 && a.K % kHif4Block == 0 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
+    if (!a.X_up && !a.gamma && pattern != RESQ_S_CHAN50 && a.K % kHif4Block == 0 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
         al16(a.a_bf16) && al16(a.r_bf16) && al16(a.r_comp)) {
         const bool img = a.a_bf16 != nullptr;
         const int64_t ncg = (a.K / kHif4Block + 31) / 32;
@@ -1377,13 +1431,18 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     LaunchScope scope(kKindQuant, stream);
     const bool img = a.a_bf16 != nullptr;  // the GEMM path asks for both images (r_bf16 whenever there is a residual)
     auto launch = [&](void (*kern)(QuantArgs, int)) { launch_err = launch_kernel(kern, grid, dim3(kThreads), 0, stream, a, rows_per_cta); };
-    if (a.X_up) {  // fused producer: GEMM-feeding variants only
+    if (a.X_up || a.gamma) {  // fused producer: GEMM-feeding variants only
         if (!img || a.r_comp) {
             set_last_error("internal: the fused producer feeds the dense GEMM operand images only");
             return RESQ_ERR_CUDA;
         }
-        if (fmt == kHiF4) residual ? launch(quant_stream_kernel<kHiF4, true, true, false, true>) : launch(quant_stream_kernel<kHiF4, false, true, false, true>);
-        else residual ? launch(quant_stream_kernel<kMXFP4, true, true, false, true>) : launch(quant_stream_kernel<kMXFP4, false, true, false, true>);
+        if (a.X_up) {
+            if (fmt == kHiF4) residual ? launch(quant_stream_kernel<kHiF4, true, true, false, 1>) : launch(quant_stream_kernel<kHiF4, false, true, false, 1>);
+            else residual ? launch(quant_stream_kernel<kMXFP4, true, true, false, 1>) : launch(quant_stream_kernel<kMXFP4, false, true, false, 1>);
+        } else {
+            if (fmt == kHiF4) residual ? launch(quant_stream_kernel<kHiF4, true, true, false, 2>) : launch(quant_stream_kernel<kHiF4, false, true, false, 2>);
+            else residual ? launch(quant_stream_kernel<kMXFP4, true, true, false, 2>) : launch(quant_stream_kernel<kMXFP4, false, true, false, 2>);
+        }
     } else if (fmt == kHiF4) {
         if (residual && a.r_comp) launch(quant_stream_kernel<kHiF4, true, true, true>);
         else if (residual) img ? launch(quant_stream_kernel<kHiF4, true, true>) : launch(quant_stream_kernel<kHiF4, true, false>);

@@ -188,6 +188,41 @@ def test_swiglu_fused_producer(shape, pattern, fmt):
     assert torch.equal(y, y_unfused)
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4, oracle.S_BLOCK])
+@pytest.mark.parametrize("shape", [(64, 256, 200), (320, 1152, 520), (40, 4160, 96)])
+def test_rmsnorm_fused_producer(shape, pattern, fmt, monkeypatch):
+    """Projection with RMSNorm * gamma folded into the quantizer pass: within tolerance of the oracle, and
+    bit-identical to the unfused call on the oracle's bf16 activations (rows of very different magnitude, a zero
+    row, an outlier channel, a strided input)."""
+    m = rq()
+    M, K, N = shape
+    if pattern == oracle.S_BLOCK and M % 32:
+        pytest.skip("block pattern needs M % 32 == 0")
+    rng = np.random.default_rng(77 * M + K + pattern)
+    h = rng.standard_normal((M, K)).astype(np.float32)
+    h[:, 5] *= 60.0
+    h[1] *= 2.0 ** 20
+    h[2] *= 2.0 ** -20
+    h[3] = 0.0
+    hb = f32_to_bf16_bits(h)
+    gb = f32_to_bf16_bits((1.0 + 0.2 * rng.standard_normal(K)).astype(np.float32))
+    _, wb = synth_xw(5 * M + N, 8, K, N, n_out=1)
+    eps = 1e-6
+    want = oracle.rmsnorm_resq_linear(bf16_bits_to_f32(hb), bf16_bits_to_f32(gb), eps, bf16_bits_to_f32(wb), pattern, fmt)
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    monkeypatch.setenv("RESQ_MXFP4_NATIVE", "0")   # the unfused reference call takes the same GEMM route as the fused one
+    big = torch.zeros((M, K + 40), dtype=torch.bfloat16, device="cuda")
+    big[:, :K] = to_dev(hb)
+    x_dev = to_dev(f32_to_bf16_bits(want["x"]))
+    y_unfused = m.resq_linear(x_dev, wc, ws, pattern, fmt, out_dtype=torch.float32)
+    for hin in (to_dev(hb), big[:, :K]):
+        y = m.rmsnorm_resq_linear(hin, to_dev(gb), eps, wc, ws, pattern, fmt, out_dtype=torch.float32)
+        torch.cuda.synchronize()
+        check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+        assert torch.equal(y, y_unfused)
+
+
 def test_swiglu_rejects_row50_and_narrow_input():
     m = rq()
     gu = torch.zeros((64, 512), dtype=torch.bfloat16, device="cuda")

@@ -626,6 +626,42 @@ def test_swiglu_producer_fixed_procedure():
     assert np.array_equal(o["y"], oracle.resq_linear(o["x"], w, oracle.S_2_4)["y"])
 
 
+def test_rmsnorm_producer_fixed_procedure():
+    """Fused RMSNorm producer: the row scale against exact rational arithmetic (sum of squares exact, one rounding
+    to fp32, then correctly rounded fp32 operations), closed-form cases, and the bf16 output against the fp64
+    definition."""
+    import math
+    rng = np.random.default_rng(11)
+    h = bf16_round(rng.standard_normal((6, 96)).astype(np.float32) * np.float32(3.0))
+    h[1] *= np.float32(2.0 ** 40)       # the scale must not depend on the magnitude class of the row
+    h[2] = 0.0
+    eps = 1e-6
+    r = oracle.rmsnorm_row_scale(h, eps)
+    for m in range(h.shape[0]):
+        exact_ss = sum(F(float(v)) * F(float(v)) for v in h[m])
+        ss32 = np.float32(float(exact_ss))                      # Fraction -> float is correctly rounded; -> fp32 once more
+        if float(np.float64(float(exact_ss))) == float(exact_ss):   # exactly representable in fp64: no double rounding
+            v = np.float32(np.float32(ss32 / np.float32(96)) + np.float32(eps))
+            want = np.float32(np.float32(1.0) / np.float32(math.sqrt(float(v))))   # fp64 sqrt of an fp32 value rounds correctly to fp32
+            assert r[m] == want
+    assert r[2] == np.float32(np.float32(1.0) / np.sqrt(np.float32(eps)))          # zero row: 1 / sqrt(eps)
+    const = np.full((1, 64), 2.0, dtype=np.float32)
+    assert oracle.rmsnorm_row_scale(const, 0.0)[0] == np.float32(0.5)                # mean square 4 -> 1/2 exactly
+    assert np.array_equal(oracle.rmsnorm_bf16(const, np.full(64, 3.0, np.float32), 0.0), np.full((1, 64), 3.0, np.float32))
+    gamma = bf16_round(1.0 + 0.1 * rng.standard_normal(96).astype(np.float32))
+    x = oracle.rmsnorm_bf16(h, gamma, eps)
+    assert np.array_equal(bf16_round(x), x)
+    h64 = h.astype(np.float64)
+    ref = h64 / np.sqrt((h64 ** 2).mean(axis=1, keepdims=True) + eps) * gamma.astype(np.float64)
+    assert np.all(np.abs(x - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-30)
+    w = bf16_round(rng.standard_normal((3, 96)).astype(np.float32) * 0.02)
+    h2 = bf16_round(rng.standard_normal((4, 128)).astype(np.float32))
+    g2 = bf16_round(1.0 + 0.1 * rng.standard_normal(128).astype(np.float32))
+    w2 = bf16_round(rng.standard_normal((3, 128)).astype(np.float32) * 0.02)
+    o = oracle.rmsnorm_resq_linear(h2, g2, eps, w2, oracle.S_2_4)
+    assert np.array_equal(o["y"], oracle.resq_linear(oracle.rmsnorm_bf16(h2, g2, eps), w2, oracle.S_2_4)["y"])
+
+
 # ----------------------------------------------------------------- regression digest of a seeded tensor
 
 def test_seeded_digest():
