@@ -149,6 +149,9 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true", help="skip the end-to-end and per-kernel passes (profiling aid)")
     ap.add_argument("--quantizer-sweep", action="store_true",
                     help="bandwidth sweep of *_quantize_act over M x K (prints a table on stderr and one JSON line)")
+    ap.add_argument("--accuracy-contrast", action="store_true",
+                    help="relative error of plain FP4, the rotation baseline and the residual variants against the exact "
+                         "bf16 product on the config's synthetic outlier tensors (no timing)")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph per step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--verbose", action="store_true")
@@ -238,6 +241,41 @@ def main():
                           "unit": "GB/s", "roofline": {"bound": "hbm", "achieved": best["GB/s"], "peak": peaks["hbm_gbs"],
                                                        "unit": "GB/s", "frac": best["frac_of_hbm"]},
                           "sweep": rows, "data": "synthetic", "note": "includes launch overhead at small M"}))
+        return
+
+    if args.accuracy_contrast:
+        # What the residual correction buys against the rotation baseline on this workload's synthetic tensors
+        # (outlier channels as in the paper's Figure 1): relative Frobenius error of Y against the exact product of
+        # the bf16 operands (fp64 on the device; plumbing, not part of the path).
+        signs = 0x9E3779B97F4A7C15
+        table = {}
+        for li, spec in enumerate(cfg.layers):
+            rows = min(cfg.M, 256)
+            x = torch.from_numpy(make_activation(cfg, li)[:rows].view(np.int16)).view(torch.bfloat16).to(dev)
+            w = torch.from_numpy(make_weight(cfg, li).view(np.int16)).view(torch.bfloat16).to(dev)
+            exact = x.double() @ w.double().t()
+            norm = exact.norm().item()
+            wc, ws = rq.pack_weight(w, fmt)
+            wcr, wsr = rq.rht_pack_weight(w, signs, fmt)
+            err = {}
+            for name, pat in (("plain", rq.S_NONE), ("resq_2:4", rq.S_2_4), ("resq_chan50", rq.S_CHAN50),
+                              ("resq_block", rq.S_BLOCK), ("resq_dense", rq.S_DENSE)):
+                if pat == rq.S_BLOCK and rows % 32:
+                    continue
+                y = rq.resq_linear(x, wc, ws, pat, fmt, out_dtype=torch.float32)
+                err[name] = ((y.double() - exact).norm().item() / norm)
+            y = rq.rht_resq_linear(x, signs, wcr, wsr, rq.S_NONE, fmt, out_dtype=torch.float32)
+            err["rotation"] = ((y.double() - exact).norm().item() / norm)
+            y = rq.rht_resq_linear(x, signs, wcr, wsr, rq.S_2_4, fmt, out_dtype=torch.float32)
+            err["rotation+resq_2:4"] = ((y.double() - exact).norm().item() / norm)
+            y = rq.w16a4_linear(x, w, rq.S_NONE, fmt, out_dtype=torch.float32)
+            err["w16a4"] = ((y.double() - exact).norm().item() / norm)
+            y = rq.w4a16_linear(x, wc, ws, fmt, out_dtype=torch.float32)
+            err["w4a16"] = ((y.double() - exact).norm().item() / norm)
+            table[spec.name] = err
+            print(f"[contrast {fmt}] {spec.name:8s} " + "  ".join(f"{k} {v:.4f}" for k, v in err.items()), file=sys.stderr)
+        print(json.dumps({"metric": f"relative Frobenius error of Y against the exact bf16 product ({fmt})", "contrast": table,
+                          "data": "synthetic", "config": config_desc}))
         return
 
     # ---- inputs: generated once on the host, packed once (weights are packed per policy update, not per call)

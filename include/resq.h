@@ -210,6 +210,28 @@ RESQ_API int mxfp4_rmsnorm_resq_linear(const void* H_bf16, int64_t M, int64_t K,
                               int pattern, void* Y, int out_dtype, int64_t ldy,
                               void* workspace, size_t ws_bytes, void* stream);
 
+/* Rotation baseline (the randomized Hadamard transform the paper compares against, Section 5.1): per block of 64
+ * channels, x' = bf16((1/8) H64 (s * x)) with H64 the Sylvester Hadamard matrix and s in {+1, -1}^64 given by
+ * `signs` (bit j set: channel j of every block is negated); H64 / 8 is orthogonal, so rotating X and W alike leaves
+ * X W^T unchanged in exact arithmetic.  Fixed evaluation: in-place fast transform in fp32, strides 1, 2, 4, 8, 16,
+ * 32, each stage (a, b) -> (a + b, a - b) with a the lower channel, every operation rounded to nearest even, the
+ * scale exact.  K % 64 == 0 (both formats).  *_rht_pack_weight rotates and packs W (same outputs as
+ * *_pack_weight); *_rht_resq_linear rotates X in the quantizer pass (never stored) and then is *_resq_linear
+ * against weights packed with the same `signs`; all selections but RESQ_S_ROW50; pattern RESQ_S_NONE is the plain
+ * rotation baseline.  Workspace, outputs and errors as *_pack_weight / *_resq_linear. */
+RESQ_API int hif4_rht_pack_weight(const void* W_bf16, int64_t N, int64_t K, int64_t ldw, unsigned long long signs,
+                         void* w_codes, void* w_meta, void* stream);
+RESQ_API int mxfp4_rht_pack_weight(const void* W_bf16, int64_t N, int64_t K, int64_t ldw, unsigned long long signs,
+                          void* w_codes, void* w_scale, void* stream);
+RESQ_API int hif4_rht_resq_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx, unsigned long long signs,
+                         const void* w_codes, const void* w_meta, int64_t N,
+                         int pattern, void* Y, int out_dtype, int64_t ldy,
+                         void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_rht_resq_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx, unsigned long long signs,
+                          const void* w_codes, const void* w_scale, int64_t N,
+                          int pattern, void* Y, int out_dtype, int64_t ldy,
+                          void* workspace, size_t ws_bytes, void* stream);
+
 /* Activation-only ablation of Table 1 ("W16A4"): Y = (deq Q(X) + S(deq Q(dX))) W^T with the weights in plain
  * bf16 (W_bf16: [N, K] device, row pitch ldw elements, ldw >= K, ldw % 8 == 0, 16-byte aligned base); the
  * activations go through the same quantizer, residual and selection as *_resq_linear (pattern RESQ_S_NONE gives

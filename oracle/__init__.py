@@ -328,3 +328,36 @@ def rmsnorm_resq_linear(h_f32: np.ndarray, gamma_f32: np.ndarray, eps: float, w_
     out = resq_linear(x, w_f32, pattern, fmt, want_abs)
     out["x"] = x
     return out
+
+
+# ---- randomized Hadamard pre-transform (the rotation baseline the paper compares against) ----------------------
+# Per block of 64 channels: x' = bf16( (1/8) * H64 (s * x) ), s in {+1, -1}^64 given by the bits of `signs` (bit j
+# set = channel j of every block negated), H64 the Sylvester Hadamard matrix.  Evaluated as the in-place fast
+# transform in fp32: six stages with strides 1, 2, 4, 8, 16, 32, each replacing a pair (a, b) = (v[j], v[j + stride])
+# by (a + b, a - b), every operation rounded to nearest even; the scale 1/8 is exact.  H64 / 8 is orthogonal, so
+# rotating X and W alike leaves X W^T unchanged in exact arithmetic.
+def rht64_bf16(x: np.ndarray, signs: int) -> np.ndarray:
+    x = np.asarray(x, dtype=np.float32)
+    M, K = x.shape
+    assert K % 64 == 0
+    s = np.array([-1.0 if (signs >> j) & 1 else 1.0 for j in range(64)], dtype=np.float32)
+    v = np.multiply(x.reshape(M, K // 64, 64), s, dtype=np.float32)
+    stride = 1
+    while stride < 64:
+        v = v.reshape(M, K // 64, 64 // (2 * stride), 2, stride)
+        a, b = v[:, :, :, 0, :], v[:, :, :, 1, :]
+        v = np.stack([np.add(a, b, dtype=np.float32), np.subtract(a, b, dtype=np.float32)], axis=3)
+        stride *= 2
+    v = np.multiply(v.reshape(M, K), np.float32(0.125), dtype=np.float32)
+    return _bf16_rne(v)
+
+
+def rht_resq_linear(x_f32: np.ndarray, w_f32: np.ndarray, signs: int, pattern: int, fmt: str = "hif4",
+                    want_abs: bool = True) -> Dict[str, np.ndarray]:
+    """Rotation baseline: Eq. (5) on the rotated activations and the rotated weights."""
+    x = rht64_bf16(x_f32, signs)
+    w = rht64_bf16(w_f32, signs)
+    out = resq_linear(x, w, pattern, fmt, want_abs)
+    out["x"] = x
+    out["w_rot"] = w
+    return out

@@ -51,6 +51,10 @@ SYMBOLS = {
     "mxfp4_swiglu_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "hif4_rmsnorm_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, ctypes.c_float, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "mxfp4_rmsnorm_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, ctypes.c_float, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "hif4_rht_pack_weight": (_ci, [_vp, _i64, _i64, _i64, ctypes.c_ulonglong, _vp, _vp, _vp]),
+    "mxfp4_rht_pack_weight": (_ci, [_vp, _i64, _i64, _i64, ctypes.c_ulonglong, _vp, _vp, _vp]),
+    "hif4_rht_resq_linear": (_ci, [_vp, _i64, _i64, _i64, ctypes.c_ulonglong, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "mxfp4_rht_resq_linear": (_ci, [_vp, _i64, _i64, _i64, ctypes.c_ulonglong, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "hif4_w16a4_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "mxfp4_w16a4_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "resq_check": (_ci, [_vp, _vp]),
@@ -145,6 +149,38 @@ def pack_weight(W: torch.Tensor, fmt: str = "hif4", stream=None) -> Tuple[torch.
     _check(_fn(fmt, "hif4_pack_weight", "mxfp4_pack_weight")(W.data_ptr(), N, K, W.stride(0), codes.data_ptr(),
                                                               side.data_ptr(), _stream(stream)))
     return codes, side
+
+
+def rht_pack_weight(W: torch.Tensor, signs: int, fmt: str = "hif4", stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """*_rht_pack_weight: rotate every block of 64 channels by the randomized Hadamard transform, then pack."""
+    _require_bf16_matrix(W, "W")
+    N, K = W.shape
+    codes = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
+    side = _side(fmt, N, K, W.device)
+    _check(_fn(fmt, "hif4_rht_pack_weight", "mxfp4_rht_pack_weight")(W.data_ptr(), N, K, W.stride(0), signs & (2 ** 64 - 1),
+                                                                      codes.data_ptr(), side.data_ptr(), _stream(stream)))
+    return codes, side
+
+
+def rht_resq_linear(X: torch.Tensor, signs: int, w_codes: torch.Tensor, w_side: torch.Tensor, pattern: int = S_NONE,
+                    fmt: str = "hif4", out_dtype: torch.dtype = torch.bfloat16, Y: Optional[torch.Tensor] = None,
+                    workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """*_rht_resq_linear: Eq. (5) on the rotated activations against weights packed by rht_pack_weight."""
+    _require_bf16_matrix(X, "X")
+    M, K = X.shape
+    N = w_codes.shape[0]
+    if Y is None:
+        ld = (N + 7) // 8 * 8
+        Y = torch.empty((M, ld), dtype=out_dtype, device=X.device)[:, :N]
+    if Y.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("Y must be bf16 or fp32")
+    if workspace is None:
+        workspace = alloc_workspace(resq_workspace_bytes(M, N, K, pattern, fmt), X.device)
+    _check(_fn(fmt, "hif4_rht_resq_linear", "mxfp4_rht_resq_linear")(
+        X.data_ptr(), M, K, X.stride(0), signs & (2 ** 64 - 1), w_codes.data_ptr(), w_side.data_ptr(), N, pattern,
+        Y.data_ptr(), OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32, Y.stride(0), workspace.data_ptr(),
+        workspace.numel(), _stream(stream)))
+    return Y
 
 
 def quantize_act(X: torch.Tensor, fmt: str = "hif4", stream=None) -> Tuple[torch.Tensor, torch.Tensor]:

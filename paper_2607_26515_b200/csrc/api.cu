@@ -111,7 +111,7 @@ int check_workspace(const void* ws, size_t have, size_t need) {
 }
 
 int quantize_only(int fmt, const void* X, int64_t rows, int64_t K, int64_t ld, void* codes, void* side, void* stream,
-                  const char* name) {
+                  const char* name, bool rht = false, unsigned long long rht_signs = 0) {
     int rc = check_matrix(X, rows, K, ld, fmt, name);
     if (rc) return rc;
     if (!codes || !side) {
@@ -127,6 +127,14 @@ int quantize_only(int fmt, const void* X, int64_t rows, int64_t K, int64_t ld, v
     a.pattern = RESQ_S_NONE;
     a.x_codes = static_cast<uint8_t*>(codes);
     a.x_side = side;
+    if (rht) {
+        if (K % 64 != 0) {
+            set_last_error("%s: the Hadamard pre-transform needs K %% 64 == 0 (K=%lld)", name, (long long)K);
+            return RESQ_ERR_SHAPE;
+        }
+        a.rht = 1;
+        a.rht_signs = rht_signs;
+    }
     return launch_quantize(fmt, a, static_cast<cudaStream_t>(stream));
 }
 
@@ -211,14 +219,19 @@ size_t linear_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K, int patt
 // instead of the packed ones.
 int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_side, int64_t N,
            int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream,
-           const void* w_bf16 = nullptr, int64_t ldw = 0, bool swiglu = false, const void* gamma = nullptr, float eps = 0.0f) {
+           const void* w_bf16 = nullptr, int64_t ldw = 0, bool swiglu = false, const void* gamma = nullptr, float eps = 0.0f,
+           bool rht = false, unsigned long long rht_signs = 0) {
     int rc = check_matrix(X, M, K, ldx, fmt, "X");
     if (rc) return rc;
     if (swiglu && ldx < 2 * K) {  // X is [gate | up]: 2K columns
         set_last_error("swiglu: the input needs 2K columns per row (ldx=%lld, K=%lld)", (long long)ldx, (long long)K);
         return RESQ_ERR_SHAPE;
     }
-    if ((swiglu || gamma) && pattern == RESQ_S_ROW50) {
+    if (rht && K % 64 != 0) {
+        set_last_error("the Hadamard pre-transform needs K %% 64 == 0 (K=%lld)", (long long)K);
+        return RESQ_ERR_SHAPE;
+    }
+    if ((swiglu || gamma || rht) && pattern == RESQ_S_ROW50) {
         set_last_error("the fused producers do not support the row-wise selection");
         return RESQ_ERR_PATTERN;
     }
@@ -274,6 +287,10 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     a.clear_words = reinterpret_cast<uint32_t*>(ws);  // cleared by the quantizer kernel: no separate memset node
     a.n_clear_words = (int)((kWsHeader + kWsFlags) / 4);
     used += kWsFlags;
+    if (rht) {
+        a.rht = 1;
+        a.rht_signs = rht_signs;
+    }
     if (gamma) {
         a.gamma = static_cast<const __nv_bfloat16*>(gamma);
         a.eps = eps;
@@ -282,7 +299,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     used += align_up((size_t)M * sizeof(float), 256);
     // MXFP4 where it pays: the GEMM runs on the block-scaled FP4 pipe and takes packed codes and scales (they
     // fit into the space of the bf16 images; the selection zeroes dropped codes); otherwise exact bf16 images.
-    const bool native = !w_bf16 && !swiglu && !gamma && fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K, pattern != RESQ_S_NONE);
+    const bool native = !w_bf16 && !swiglu && !gamma && !rht && fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K, pattern != RESQ_S_NONE);
     uint8_t* region_a = ws + used;
     used += align_up((size_t)M * (size_t)K * 2, 256);
     uint8_t* region_r = nullptr;
@@ -291,7 +308,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
         used += residual_region_bytes(M, K, pattern);
     }
     // 2:4 on the CTA-pair kernel: the residual goes to the structured-sparse MMA in compressed form
-    const bool sparse24 = !w_bf16 && !swiglu && !gamma && !native && pattern == RESQ_S_2_4 && gemm_sparse24_supported(M, N, K);
+    const bool sparse24 = !w_bf16 && !swiglu && !gamma && !rht && !native && pattern == RESQ_S_2_4 && gemm_sparse24_supported(M, N, K);
     const size_t codes_bytes = align_up((size_t)M * (size_t)K / 2, 256);
     if (native) {
         a.x_codes = region_a;
@@ -479,6 +496,27 @@ int mxfp4_swiglu_resq_linear(const void* GU, int64_t M, int64_t K, int64_t ldgu,
                              void* stream) {
     return linear(kMXFP4, GU, M, K, ldgu, w_codes, w_scale, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream, nullptr,
                   0, true);
+}
+
+int hif4_rht_pack_weight(const void* W, int64_t N, int64_t K, int64_t ldw, unsigned long long signs, void* w_codes, void* w_meta,
+                         void* stream) {
+    return quantize_only(kHiF4, W, N, K, ldw, w_codes, w_meta, stream, "W", true, signs);
+}
+int mxfp4_rht_pack_weight(const void* W, int64_t N, int64_t K, int64_t ldw, unsigned long long signs, void* w_codes, void* w_scale,
+                          void* stream) {
+    return quantize_only(kMXFP4, W, N, K, ldw, w_codes, w_scale, stream, "W", true, signs);
+}
+int hif4_rht_resq_linear(const void* X, int64_t M, int64_t K, int64_t ldx, unsigned long long signs, const void* w_codes,
+                         const void* w_meta, int64_t N, int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace,
+                         size_t ws_bytes, void* stream) {
+    return linear(kHiF4, X, M, K, ldx, w_codes, w_meta, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream, nullptr, 0,
+                  false, nullptr, 0.0f, true, signs);
+}
+int mxfp4_rht_resq_linear(const void* X, int64_t M, int64_t K, int64_t ldx, unsigned long long signs, const void* w_codes,
+                          const void* w_scale, int64_t N, int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace,
+                          size_t ws_bytes, void* stream) {
+    return linear(kMXFP4, X, M, K, ldx, w_codes, w_scale, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream, nullptr, 0,
+                  false, nullptr, 0.0f, true, signs);
 }
 
 int hif4_rmsnorm_resq_linear(const void* H, int64_t M, int64_t K, int64_t ldh, const void* gamma, float eps, const void* w_codes,

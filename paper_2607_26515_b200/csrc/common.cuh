@@ -80,6 +80,10 @@ struct QuantArgs {
     const __nv_bfloat16* gamma;
     float* row_scale;
     float eps;
+    // rht != 0: randomized Hadamard pre-transform, the input is bf16((1/8) H64 (s * X)) per block of 64 channels,
+    // bit j of rht_signs negates channel j of every block (K % 64 == 0)
+    int rht;
+    unsigned long long rht_signs;
     int64_t M, K, ldx;
     int pattern;            // resq_pattern; RESQ_S_NONE => no residual work at all
     // canonical packed outputs (any may be null)

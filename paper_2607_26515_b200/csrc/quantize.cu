@@ -171,8 +171,46 @@ __global__ void __launch_bounds__(256) rmsnorm_row_scale_kernel(const __nv_bfloa
     }
 }
 
+// Randomized Hadamard pre-transform of one block of 64 channels held by an aligned octet of lanes (8 values per
+// lane): x' = bf16((1/8) H64 (s * x)).  In-place fast transform in fp32, strides 1, 2, 4 inside the lane and 8, 16, 32
+// across lanes, each stage (a, b) -> (a + b, a - b) with a the lower channel; every operation rounded to nearest
+// (no contraction), so the result is the same on every implementation that keeps this order.
+__device__ __forceinline__ uint4 rht64_bf16x8(const uint4& raw, unsigned long long signs, int lane) {
+    float v[8];
+    unpack_bf16x8(raw, v);
+    const uint32_t sb = (uint32_t)(signs >> (8 * (lane & 7))) & 0xFFu;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = ((sb >> i) & 1u) ? -v[i] : v[i];
+#pragma unroll
+    for (int h = 1; h < 8; h <<= 1) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if ((i & h) == 0) {
+                const float a = v[i], b = v[i + h];
+                v[i] = __fadd_rn(a, b);
+                v[i + h] = __fsub_rn(a, b);
+            }
+        }
+    }
+#pragma unroll
+    for (int d = 1; d < 8; d <<= 1) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float other = __shfl_xor_sync(0xFFFFFFFFu, v[i], d);
+            v[i] = (lane & d) ? __fsub_rn(other, v[i]) : __fadd_rn(v[i], other);
+        }
+    }
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 p = __floats2bfloat162_rn(__fmul_rn(v[2 * i], 0.125f), __fmul_rn(v[2 * i + 1], 0.125f));
+        o[i] = *reinterpret_cast<const uint32_t*>(&p);
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 // COMP (2:4 only): the residual image leaves in compressed form with its index metadata (a.r_comp, a.r_meta).
-// PROD = 1: the input is x = bf16(SiLU(g) * u) of a.X (g) and a.X_up (u); PROD = 2: x = bf16((X * r[m]) * gamma[k])
+// PROD = 3: the input is the randomized Hadamard transform of X (rht64_bf16x8).  PROD = 1: the input is x = bf16(SiLU(g) * u) of a.X (g) and a.X_up (u); PROD = 2: x = bf16((X * r[m]) * gamma[k])
 // with the row scales of rmsnorm_row_scale_kernel; computed on the fly, never stored.
 template <int FMT, bool RESIDUAL, bool IMG, bool COMP = false, int PROD = 0>
 __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int rows_per_cta) {
@@ -212,6 +250,7 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
     for (int64_t m = m_begin; m < m_end; ++m) {
         uint4 cur = raw;
         if constexpr (PROD == 1) cur = swiglu_bf16x8(raw, raw_up);
+        if constexpr (PROD == 3) cur = rht64_bf16x8(raw, a.rht_signs, lane);  // all lanes: the octets exchange values
         if constexpr (PROD == 2) {
             if (active) {
                 const float r = a.row_scale[m];
@@ -1339,7 +1378,7 @@ static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t
 int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     const int pattern = a.pattern;
     const bool residual = pattern != RESQ_S_NONE;
-    if (pattern == RESQ_S_ROW50 && (a.X_up || a.gamma)) {
+    if (pattern == RESQ_S_ROW50 && (a.X_up || a.gamma || a.rht)) {
         set_last_error("the fused producers do not support the row-wise selection");
         return RESQ_ERR_PATTERN;
     }
@@ -1394,7 +1433,7 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     // Worth it once there is a warp task (32 blocks of one row) for every warp slot of the machine; below
     // that the finer-grained kernel (a lane per 8 values) finishes sooner.
     const int64_t block_tasks = a.M * ((a.K / kHif4Block + 31) / 32);
-    if (!a.X_up && !a.gamma && pattern != RESQ_S_CHAN50 && a.K % kHif4Block == 0 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
+    if (!a.X_up && !a.gamma && !a.rht && pattern != RESQ_S_CHAN50 && a.K % kHif4Block == 0 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
         al16(a.a_bf16) && al16(a.r_bf16) && al16(a.r_comp)) {
         const bool img = a.a_bf16 != nullptr;
         const int64_t ncg = (a.K / kHif4Block + 31) / 32;
@@ -1431,7 +1470,19 @@ int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
     LaunchScope scope(kKindQuant, stream);
     const bool img = a.a_bf16 != nullptr;  // the GEMM path asks for both images (r_bf16 whenever there is a residual)
     auto launch = [&](void (*kern)(QuantArgs, int)) { launch_err = launch_kernel(kern, grid, dim3(kThreads), 0, stream, a, rows_per_cta); };
-    if (a.X_up || a.gamma) {  // fused producer: GEMM-feeding variants only
+    if (a.rht) {  // rotation baseline: weight packing (plain outputs) or the GEMM-feeding variants
+        if (a.r_comp || (!img && residual)) {
+            set_last_error("internal: the Hadamard pre-transform feeds weight packing or the dense GEMM operand images");
+            return RESQ_ERR_CUDA;
+        }
+        if (fmt == kHiF4) {
+            if (!img) launch(quant_stream_kernel<kHiF4, false, false, false, 3>);
+            else residual ? launch(quant_stream_kernel<kHiF4, true, true, false, 3>) : launch(quant_stream_kernel<kHiF4, false, true, false, 3>);
+        } else {
+            if (!img) launch(quant_stream_kernel<kMXFP4, false, false, false, 3>);
+            else residual ? launch(quant_stream_kernel<kMXFP4, true, true, false, 3>) : launch(quant_stream_kernel<kMXFP4, false, true, false, 3>);
+        }
+    } else if (a.X_up || a.gamma) {  // fused producer: GEMM-feeding variants only
         if (!img || a.r_comp) {
             set_last_error("internal: the fused producer feeds the dense GEMM operand images only");
             return RESQ_ERR_CUDA;

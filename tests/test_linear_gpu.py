@@ -223,6 +223,30 @@ def test_rmsnorm_fused_producer(shape, pattern, fmt, monkeypatch):
         assert torch.equal(y, y_unfused)
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4, oracle.S_CHAN50])
+@pytest.mark.parametrize("shape", [(64, 256, 200), (300, 1152, 520)])
+def test_randomized_hadamard_baseline(shape, pattern, fmt, monkeypatch):
+    """Rotation baseline: weights rotated and packed by *_rht_pack_weight are bit-identical to packing the oracle's
+    rotated weights; the rotated layer is within tolerance of the oracle and bit-identical to the plain call on the
+    oracle's rotated activations."""
+    m = rq()
+    M, K, N = shape
+    signs = 0x9E3779B97F4A7C15
+    xb, wb = synth_xw(13 * M + N + pattern, M, K, N, n_out=max(1, K // 256))
+    want = oracle.rht_resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), signs, pattern, fmt)
+    wc, ws = m.rht_pack_weight(to_dev(wb), signs, fmt)
+    wc2, ws2 = m.pack_weight(to_dev(f32_to_bf16_bits(want["w_rot"])), fmt)
+    assert torch.equal(wc, wc2) and torch.equal(ws, ws2)
+    assert np.array_equal(wc.cpu().numpy(), want["w_codes"])
+    monkeypatch.setenv("RESQ_MXFP4_NATIVE", "0")   # the plain reference call takes the same GEMM route
+    y = m.rht_resq_linear(to_dev(xb), signs, wc, ws, pattern, fmt, out_dtype=torch.float32)
+    y_plain = m.resq_linear(to_dev(f32_to_bf16_bits(want["x"])), wc, ws, pattern, fmt, out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+    assert torch.equal(y, y_plain)
+
+
 def test_swiglu_rejects_row50_and_narrow_input():
     m = rq()
     gu = torch.zeros((64, 512), dtype=torch.bfloat16, device="cuda")

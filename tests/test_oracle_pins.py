@@ -662,6 +662,40 @@ def test_rmsnorm_producer_fixed_procedure():
     assert np.array_equal(o["y"], oracle.resq_linear(oracle.rmsnorm_bf16(h2, g2, eps), w2, oracle.S_2_4)["y"])
 
 
+def test_randomized_hadamard_transform():
+    """Rotation baseline: the fast transform equals the Sylvester Hadamard matrix product (exact on small integers),
+    is orthogonal (applying it twice with the signs moved to the other side returns the input; the dot product of
+    two rotated vectors equals that of the originals), spreads an outlier over its block, and the rotated layer is
+    Eq. (5) on the rotated operands."""
+    from scipy.linalg import hadamard
+    H = hadamard(64).astype(np.float64)
+    rng = np.random.default_rng(21)
+    signs = int(rng.integers(0, 2 ** 63)) | (1 << 63)
+    s = np.array([-1.0 if (signs >> j) & 1 else 1.0 for j in range(64)])
+    x = rng.integers(-8, 9, (5, 192)).astype(np.float32)
+    got = oracle.rht64_bf16(x, signs)
+    want = np.concatenate([(x[:, b * 64:(b + 1) * 64] * s) @ H.T / 8 for b in range(3)], axis=1)
+    assert np.array_equal(got, want)                                     # small integers: every step exact
+    back = oracle.rht64_bf16(got, 0) * s[None, :].repeat(3, axis=0).reshape(1, 192)   # H/8 is symmetric and orthogonal
+    assert np.array_equal(back, x)
+    y = rng.integers(-8, 9, (5, 192)).astype(np.float32)
+    assert np.array_equal((oracle.rht64_bf16(y, signs).astype(np.float64) * got).sum(axis=1), (x.astype(np.float64) * y).sum(axis=1))
+    g = bf16_round(rng.standard_normal((4, 128)).astype(np.float32))
+    g[:, 7] *= 80.0
+    r = oracle.rht64_bf16(g, signs).astype(np.float64)
+    ref = np.concatenate([(g[:, b * 64:(b + 1) * 64].astype(np.float64) * s) @ H.T / 8 for b in range(2)], axis=1)
+    assert np.all(np.abs(r - ref) <= 2.0 ** -8 * np.abs(ref) + 2.0 ** -20 * np.abs(g).max())
+    crest = lambda v: np.abs(v[:, :64]).max(axis=1) / np.sqrt((v[:, :64] ** 2).mean(axis=1))
+    assert np.all(crest(r) < 0.5 * crest(g.astype(np.float64)))           # the outlier is spread over its block
+    w = bf16_round(rng.standard_normal((3, 128)).astype(np.float32) * 0.02)
+    o = oracle.rht_resq_linear(g, w, signs, oracle.S_NONE)
+    assert np.array_equal(o["y"], oracle.resq_linear(oracle.rht64_bf16(g, signs), oracle.rht64_bf16(w, signs), oracle.S_NONE)["y"])
+    # what the baseline is for: on a tensor with outlier channels the rotated FP4 product is closer to the exact one
+    exact = g.astype(np.float64) @ w.astype(np.float64).T
+    plain = oracle.resq_linear(g, w, oracle.S_NONE)["y"]
+    assert np.linalg.norm(o["y"] - exact) < np.linalg.norm(plain - exact)
+
+
 # ----------------------------------------------------------------- regression digest of a seeded tensor
 
 def test_seeded_digest():
