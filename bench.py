@@ -32,7 +32,12 @@ from workloads import CONFIGS, make_activation, make_weight  # noqa: E402
 METRIC = "hif4_resq_linear TFLOP/s & GB/s at 1 B200; % of FP4-tensor/HBM roofline"
 L2_BYTES = 126 * 1024 * 1024
 PATTERN_IDS = {"none": 0, "dense": 1, "2:4": 2, "row50": 3, "chan50": 4, "block": 5}
+# sparsity sweep: the selecting patterns with 1/4 or 3/4 kept (RESQ_KEEP_QUARTERS)
+for _name, _base in (("{}:4", 2), ("row{}", 3), ("chan{}", 4), ("block{}", 5)):
+    for _q in (1, 3):
+        PATTERN_IDS[_name.format(_q if _base == 2 else 25 * _q)] = _base | (_q << 8)
 RHO = {0: 0.0, 1: 1.0, 2: 0.5, 3: 0.5, 4: 0.5, 5: 0.5}
+RHO.update({p: (p >> 8) / 4.0 for p in PATTERN_IDS.values() if p >> 8})
 # mean DRAM bytes per GEMM launch from an ncu capture of the default workload (see profiles/)
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {(1, 2, "hif4"): 15.3e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -140,7 +145,9 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=1, help="index into the workload configs (default 1: 3B decode)")
-    ap.add_argument("--pattern", default=None, help="none|dense|2:4|row50|chan50|block (default: the config's)")
+    ap.add_argument("--pattern", default=None,
+                    help="none|dense|2:4|row50|chan50|block (default: the config's); sparsity sweep: 1:4|3:4|row25|row75|"
+                         "chan25|chan75|block25|block75")
     ap.add_argument("--format", default="hif4", choices=["hif4", "mxfp4"])
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--out-dtype", default="bf16", choices=["bf16", "f32"])
@@ -258,9 +265,10 @@ def main():
             wc, ws = rq.pack_weight(w, fmt)
             wcr, wsr = rq.rht_pack_weight(w, signs, fmt)
             err = {}
-            for name, pat in (("plain", rq.S_NONE), ("resq_2:4", rq.S_2_4), ("resq_chan50", rq.S_CHAN50),
+            for name, pat in (("plain", rq.S_NONE), ("resq_1:4", rq.keep_quarters(rq.S_2_4, 1)), ("resq_2:4", rq.S_2_4),
+                              ("resq_3:4", rq.keep_quarters(rq.S_2_4, 3)), ("resq_chan50", rq.S_CHAN50),
                               ("resq_block", rq.S_BLOCK), ("resq_dense", rq.S_DENSE)):
-                if pat == rq.S_BLOCK and rows % 32:
+                if (pat & 0xFF) == rq.S_BLOCK and rows % 32:
                     continue
                 y = rq.resq_linear(x, wc, ws, pat, fmt, out_dtype=torch.float32)
                 err[name] = ((y.double() - exact).norm().item() / norm)

@@ -72,6 +72,13 @@ typedef enum {
                                  largest L2 norm, chosen over the whole tensor */
 } resq_pattern;
 
+/* Sparsity sweep (the paper evaluates 50 % and names other ratios as open, Section 6): a selecting pattern combined
+ * with RESQ_KEEP_QUARTERS(q), q = 1, 2 or 3, keeps q/4 instead of 1/2: the q largest of every 4 (RESQ_S_2_4, i.e.
+ * 1:4 / 2:4 / 3:4), floor(K q / 4) entries per row (RESQ_S_ROW50), floor(K q / 4) channels (RESQ_S_CHAN50),
+ * floor(nb q / 4) blocks (RESQ_S_BLOCK32x64_50); same tie rules.  Accepted wherever a pattern argument is; q = 2 is
+ * the pattern itself. */
+#define RESQ_KEEP_QUARTERS(q) ((int)(q) << 8)
+
 typedef enum { RESQ_OUT_BF16 = 0, RESQ_OUT_F32 = 1 } resq_out;
 
 /* ---- size queries (host only, no CUDA calls) -------------------------------------------------- */

@@ -23,6 +23,12 @@ _LIB = os.path.join(_HERE, "libresq_oracle.so")
 
 S_NONE, S_DENSE, S_2_4, S_ROW50, S_CHAN50, S_BLOCK = 0, 1, 2, 3, 4, 5
 
+
+def keep_quarters(pattern: int, q: int) -> int:
+    """Sparsity sweep: the pattern with q/4 of the entries kept instead of one half (q = 1, 2, 3)."""
+    return pattern | (q << 8)
+
+
 _lib = None
 
 
@@ -165,9 +171,9 @@ def mask(v: np.ndarray, pattern: int, want_scores: bool = False):
     bits = np.empty((M, K // 8), dtype=np.uint8)
     info = np.zeros(2, dtype=np.float64)
     scores = None
-    if want_scores and pattern == S_CHAN50:
+    if want_scores and (pattern & 0xFF) == S_CHAN50:
         scores = np.zeros(K, dtype=np.float64)
-    if want_scores and pattern == S_BLOCK:
+    if want_scores and (pattern & 0xFF) == S_BLOCK:
         scores = np.zeros((M // 32) * (K // 64), dtype=np.float64)
     rc = lib().oracle_mask(_p(v), M, K, int(pattern), _p(bits), _p(info), _p(scores))
     if rc == -1:

@@ -288,6 +288,11 @@ int oracle_mask(const double *v, int64_t M, int64_t K, int pattern, uint8_t *mas
     memset(mask_bits, 0, (size_t)(M * (K / 8)));
     info[0] = 1.0;
     info[1] = 0.0;
+    /* sparsity sweep: bits 8.. of the pattern give the kept share in quarters (0 = the paper's one half) */
+    int quarters = (pattern >> 8) & 0xFF;
+    if (quarters == 0) quarters = 2;
+    if (quarters > 3 || pattern < 0 || (pattern >> 16)) return -2;
+    pattern &= 0xFF;
     switch (pattern) {
     case S_NONE:
         return 0;
@@ -305,8 +310,7 @@ int oracle_mask(const double *v, int64_t M, int64_t K, int pattern, uint8_t *mas
                     e[t].idx = t;
                 }
                 qsort(e, 4, sizeof(keyed_t), cmp_keyed);
-                set_bit(mask_bits, K, m, 4 * g + e[0].idx);
-                set_bit(mask_bits, K, m, 4 * g + e[1].idx);
+                for (int t = 0; t < quarters; ++t) set_bit(mask_bits, K, m, 4 * g + e[t].idx);
             }
         return 0;
     }
@@ -319,7 +323,7 @@ int oracle_mask(const double *v, int64_t M, int64_t K, int pattern, uint8_t *mas
                 e[k].idx = k;
             }
             qsort(e, (size_t)K, sizeof(keyed_t), cmp_keyed);
-            for (int64_t t = 0; t < K / 2; ++t) set_bit(mask_bits, K, m, e[t].idx);
+            for (int64_t t = 0; t < K * quarters / 4; ++t) set_bit(mask_bits, K, m, e[t].idx);
         }
         free(e);
         return 0;
@@ -336,7 +340,7 @@ int oracle_mask(const double *v, int64_t M, int64_t K, int pattern, uint8_t *mas
             if (scores_out) scores_out[k] = acc;
         }
         qsort(e, (size_t)K, sizeof(keyed_t), cmp_keyed);
-        int64_t keep = K / 2;
+        int64_t keep = K * quarters / 4;
         for (int64_t t = 0; t < keep; ++t)
             for (int64_t m = 0; m < M; ++m) set_bit(mask_bits, K, m, e[t].idx);
         info[0] = exact;
@@ -363,7 +367,7 @@ int oracle_mask(const double *v, int64_t M, int64_t K, int pattern, uint8_t *mas
                 if (scores_out) scores_out[a * nbc + b] = acc;
             }
         qsort(e, (size_t)nb, sizeof(keyed_t), cmp_keyed);
-        int64_t keep = nb / 2;
+        int64_t keep = nb * quarters / 4;
         for (int64_t t = 0; t < keep; ++t) {
             int64_t a = e[t].idx / nbc, b = e[t].idx % nbc;
             for (int64_t i = 0; i < BLK_ROWS; ++i)

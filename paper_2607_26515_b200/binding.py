@@ -140,6 +140,11 @@ def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
 
 # ------------------------------------------------------------------ calls
 
+def keep_quarters(pattern: int, q: int) -> int:
+    """RESQ_KEEP_QUARTERS: the pattern with q/4 of the entries kept instead of one half (q = 1, 2, 3)."""
+    return pattern | (q << 8)
+
+
 def pack_weight(W: torch.Tensor, fmt: str = "hif4", stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
     """*_pack_weight: W bf16 [N,K] -> (codes u8 [N,K/2], meta i32 [N,K/64] | scale u8 [N,K/32])."""
     _require_bf16_matrix(W, "W")

@@ -90,6 +90,23 @@ int check_matrix(const void* p, int64_t rows, int64_t K, int64_t ld, int fmt, co
     return RESQ_OK;
 }
 
+// A pattern argument is a base pattern, optionally combined with RESQ_KEEP_QUARTERS(q): splits it in place.
+int split_pattern(int* pattern, int* quarters) {
+    const int q = (*pattern >> 8) & 0xFF;
+    if (*pattern < 0 || (*pattern >> 16) != 0 || q > 3) {
+        set_last_error("unknown pattern %d", *pattern);
+        return RESQ_ERR_PATTERN;
+    }
+    *quarters = q == 0 ? 2 : q;
+    *pattern &= 0xFF;
+    if (q != 0 && (*pattern == RESQ_S_NONE || *pattern == RESQ_S_DENSE)) {
+        set_last_error("RESQ_KEEP_QUARTERS applies to the selecting patterns only");
+        return RESQ_ERR_PATTERN;
+    }
+    return RESQ_OK;
+}
+int base_pattern(int pattern) { return pattern < 0 ? pattern : pattern & 0xFF; }
+
 int check_pattern(int pattern, int64_t M) {
     if (pattern < RESQ_S_NONE || pattern > RESQ_S_BLOCK32x64_50) {
         set_last_error("unknown pattern %d", pattern);
@@ -169,6 +186,9 @@ int residual_mask(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, int
                   void* r_codes, void* r_side, void* mask_bits, void* workspace, size_t ws_bytes, void* stream) {
     int rc = check_matrix(X, M, K, ldx, fmt, "X");
     if (rc) return rc;
+    int quarters = 2;
+    rc = split_pattern(&pattern, &quarters);
+    if (rc) return rc;
     rc = check_pattern(pattern, M);
     if (rc) return rc;
     rc = check_workspace(workspace, ws_bytes, resq_residual_mask_workspace_bytes(M, K, pattern));
@@ -183,6 +203,7 @@ int residual_mask(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, int
     a.K = K;
     a.ldx = ldx;
     a.pattern = pattern;
+    a.keep_quarters = quarters;
     a.x_codes = static_cast<uint8_t*>(x_codes);
     a.x_side = x_side;
     if (pattern != RESQ_S_NONE) {
@@ -222,6 +243,9 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
            const void* w_bf16 = nullptr, int64_t ldw = 0, bool swiglu = false, const void* gamma = nullptr, float eps = 0.0f,
            bool rht = false, unsigned long long rht_signs = 0) {
     int rc = check_matrix(X, M, K, ldx, fmt, "X");
+    if (rc) return rc;
+    int quarters = 2;
+    rc = split_pattern(&pattern, &quarters);
     if (rc) return rc;
     if (swiglu && ldx < 2 * K) {  // X is [gate | up]: 2K columns
         set_last_error("swiglu: the input needs 2K columns per row (ldx=%lld, K=%lld)", (long long)ldx, (long long)K);
@@ -281,6 +305,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     a.K = K;
     a.ldx = ldx;
     a.pattern = pattern;
+    a.keep_quarters = quarters;
     size_t used = 0;
     carve_quant_scratch(ws + kWsFlags, M, K, pattern, a, used);
     a.status = reinterpret_cast<DeviceStatus*>(ws);
@@ -308,7 +333,8 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
         used += residual_region_bytes(M, K, pattern);
     }
     // 2:4 on the CTA-pair kernel: the residual goes to the structured-sparse MMA in compressed form
-    const bool sparse24 = !w_bf16 && !swiglu && !gamma && !rht && !native && pattern == RESQ_S_2_4 && gemm_sparse24_supported(M, N, K);
+    const bool sparse24 = !w_bf16 && !swiglu && !gamma && !rht && !native && pattern == RESQ_S_2_4 && quarters == 2 &&
+                          gemm_sparse24_supported(M, N, K);
     const size_t codes_bytes = align_up((size_t)M * (size_t)K / 2, 256);
     if (native) {
         a.x_codes = region_a;
@@ -446,13 +472,13 @@ size_t resq_mask_bytes(int64_t M, int64_t K) { return M > 0 && K > 0 ? (size_t)M
 
 size_t resq_residual_mask_workspace_bytes(int64_t M, int64_t K, int pattern) {
     if (M <= 0 || K <= 0) return kWsHeader;
-    return kWsHeader + quant_scratch_bytes(M, K, pattern);
+    return kWsHeader + quant_scratch_bytes(M, K, base_pattern(pattern));
 }
 size_t hif4_resq_workspace_bytes(int64_t M, int64_t N, int64_t K, int pattern) {
-    return linear_workspace_bytes(kHiF4, M, N, K, pattern);
+    return linear_workspace_bytes(kHiF4, M, N, K, base_pattern(pattern));
 }
 size_t mxfp4_resq_workspace_bytes(int64_t M, int64_t N, int64_t K, int pattern) {
-    return linear_workspace_bytes(kMXFP4, M, N, K, pattern);
+    return linear_workspace_bytes(kMXFP4, M, N, K, base_pattern(pattern));
 }
 
 int hif4_pack_weight(const void* W, int64_t N, int64_t K, int64_t ldw, void* w_codes, void* w_meta, void* stream) {

@@ -33,28 +33,35 @@ constexpr uint32_t kMagicBits = 0x4B400000u;
 constexpr uint32_t kNibbleBias = (uint32_t)(((uint64_t)kMagicBits * 0x11111111ull) & 0xFFFFFFFFull);
 constexpr uint32_t kOctalBias = (uint32_t)(((uint64_t)kMagicBits * (1ull + 8ull + 64ull + 512ull)) & 0xFFFFFFFFull);
 
-// top-2-of-4 (Section 4.3, item (2)): keys are four 3-bit magnitudes.  Larger key wins, equal keys keep
-// the lower index; exactly two bits of the result are set.
-__host__ __device__ constexpr uint32_t top2of4_keys(int q0, int q1, int q2, int q3) {
+// top-n-of-4 (Section 4.3, item (2) is n = 2): keys are four 3-bit magnitudes.  Larger key wins, equal keys keep
+// the lower index; exactly n bits of the result are set.
+__host__ __device__ constexpr uint32_t topnof4_keys(int q0, int q1, int q2, int q3, int n) {
     const int k0 = q0 * 4 + 3, k1 = q1 * 4 + 2, k2 = q2 * 4 + 1, k3 = q3 * 4;
     const int w0 = (k0 > k1) + (k0 > k2) + (k0 > k3);
     const int w1 = (k1 > k0) + (k1 > k2) + (k1 > k3);
     const int w2 = (k2 > k0) + (k2 > k1) + (k2 > k3);
     const int w3 = (k3 > k0) + (k3 > k1) + (k3 > k2);
-    return (uint32_t)((w0 >= 2) | ((w1 >= 2) << 1) | ((w2 >= 2) << 2) | ((w3 >= 2) << 3));
+    const int need = 4 - n;  // an element is kept if it beats at least this many of the others
+    return (uint32_t)((w0 >= need) | ((w1 >= need) << 1) | ((w2 >= need) << 2) | ((w3 >= need) << 3));
 }
+__host__ __device__ constexpr uint32_t top2of4_keys(int q0, int q1, int q2, int q3) { return topnof4_keys(q0, q1, q2, q3, 2); }
 // c: four 4-bit codes (element i at bits 4i+2:4i, sign bits ignored).
 __device__ __forceinline__ uint32_t top2of4(uint32_t c) {
     return top2of4_keys((int)(c & 7u), (int)((c >> 4) & 7u), (int)((c >> 8) & 7u), (int)((c >> 12) & 7u));
 }
-// The same as a 4096-entry table indexed by q0 | q1<<3 | q2<<6 | q3<<9, built at compile time.
-struct Top2Table {
-    uint8_t v[4096];
-    constexpr Top2Table() : v() {
-        for (int i = 0; i < 4096; ++i) v[i] = (uint8_t)top2of4_keys(i & 7, (i >> 3) & 7, (i >> 6) & 7, (i >> 9) & 7);
+// The same as a 4096-entry table indexed by q0 | q1<<3 | q2<<6 | q3<<9, built at compile time: the keep nibbles of
+// n = 1, 2, 3 in bits 3:0, 7:4, 11:8 of an entry.
+struct TopNTable {
+    uint16_t v[4096];
+    constexpr TopNTable() : v() {
+        for (int i = 0; i < 4096; ++i) {
+            const int q0 = i & 7, q1 = (i >> 3) & 7, q2 = (i >> 6) & 7, q3 = (i >> 9) & 7;
+            v[i] = (uint16_t)(topnof4_keys(q0, q1, q2, q3, 1) | (topnof4_keys(q0, q1, q2, q3, 2) << 4) |
+                              (topnof4_keys(q0, q1, q2, q3, 3) << 8));
+        }
     }
 };
-__device__ const Top2Table kTop2Table{};
+__device__ const TopNTable kTopNTable{};
 
 // ------------------------------------------------------------------------------------ HiF4
 // x: the lane's 8 values.  grp_mask: the 8 lanes of this block.  lane8: lane index inside the octet.

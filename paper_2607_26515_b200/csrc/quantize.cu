@@ -62,8 +62,9 @@ __device__ __forceinline__ void encode_lane(const float (&x)[8], int lane, uint3
     }
 }
 
-__device__ __forceinline__ uint32_t top2_mask8(uint32_t oct) {
-    return (uint32_t)kTop2Table.v[oct & 0xFFFu] | ((uint32_t)kTop2Table.v[(oct >> 16) & 0xFFFu] << 4);
+// keep mask of the lane's two groups of four; nsh = 4 * (n - 1) selects the n-of-4 nibble of the table entries
+__device__ __forceinline__ uint32_t topn_mask8(uint32_t oct, int nsh) {
+    return (((uint32_t)kTopNTable.v[oct & 0xFFFu] >> nsh) & 15u) | ((((uint32_t)kTopNTable.v[(oct >> 16) & 0xFFFu] >> nsh) & 15u) << 4);
 }
 
 template <int FMT>
@@ -322,7 +323,7 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
             encode_lane<FMT>(dx, lane, rcodes, rside, rdeq, roct);
         }
         uint32_t keep = 0xFFu;
-        if (pattern == RESQ_S_2_4) keep = top2_mask8(roct);
+        if (pattern == RESQ_S_2_4) keep = topn_mask8(roct, 4 * (a.keep_quarters - 1));
         uint32_t comp0 = 0, comp1 = 0, idx_byte = 0;
         if constexpr (COMP) {
             {  // compressed image: 8 bytes per lane, and one byte of index pairs
@@ -625,6 +626,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
     const uint32_t in0 = smem_u32(smem_q) + (uint32_t)(warp * kBufs * kStageBytes);
     const uint32_t stage = in0 + 2 * kStageBytes;            // only with IMG
     const int pattern = a.pattern;
+    const int nsh = 4 * (a.keep_quarters - 1);               // n-of-4 selection: which nibble of the table entries
 
     // cooperative row copies: piece j of lane l is chunk (l & 7) of block 4j + (l >> 3)
     const int cp_blk = lane >> 3, cp_ch = lane & 7;
@@ -722,7 +724,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
             encode_block<FMT, true, true>(w, rcodes, rmeta, [&](int c, const float (&)[8], const float (&rdq)[8], uint32_t roct) {
                 uint32_t keep = 0xFFu;
                 if (pattern == RESQ_S_2_4) {
-                    keep = top2_mask8(roct);
+                    keep = topn_mask8(roct, nsh);
                     if (c < 4) keep_lo = (keep_lo & ~(0xFFu << (8 * c))) | (keep << (8 * c));
                     else keep_hi = (keep_hi & ~(0xFFu << (8 * (c - 4)))) | (keep << (8 * (c - 4)));
                 }
@@ -921,7 +923,7 @@ __global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs
 
     // ---- phase B: the (K/2)-th largest 15-bit magnitude of the row (inactive blocks hold zeros: they never win)
     unsigned prefix = 0u;
-    int remaining = (int)(a.K / 2);
+    int remaining = (int)(a.K * a.keep_quarters / 4);
     for (int b = 14; b >= 0; --b) {
         const unsigned cand = prefix | (1u << b);
         const uint32_t cand2 = (cand >> b) * 0x00010001u;
@@ -1213,7 +1215,7 @@ __global__ void __launch_bounds__(kThreads) quant_row50_kernel(QuantArgs a) {
     }
     if (tid == 0) {
         s_prefix = 0u;
-        s_remaining = (int)(K / 2);
+        s_remaining = (int)(K * a.keep_quarters / 4);
     }
     __syncthreads();
     // radix select on the 15-bit magnitude: bits 14:8 then 7:0
@@ -1361,7 +1363,7 @@ static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t
     {
         LaunchScope scope(kKindSelect, stream);
         rc = cuda_fail(launch_kernel(topk_select_kernel, dim3(1), dim3(kSelThreads), 0, stream, (const double*)a.scores, (int)nscore,
-                                     (int)(nscore / 2), a.keep_flags),
+                                     (int)(nscore * a.keep_quarters / 4), a.keep_flags),
                        "topk_select_kernel launch");
     }
     if (rc) return rc;
@@ -1375,7 +1377,13 @@ static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t
     return rc;
 }
 
-int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream) {
+int launch_quantize(int fmt, const QuantArgs& a_in, cudaStream_t stream) {
+    QuantArgs a = a_in;
+    if (a.keep_quarters < 1 || a.keep_quarters > 3) a.keep_quarters = 2;  // the paper's 50 %
+    if (a.r_comp && a.keep_quarters != 2) {
+        set_last_error("internal: the compressed residual operand exists for 2:4 only");
+        return RESQ_ERR_CUDA;
+    }
     const int pattern = a.pattern;
     const bool residual = pattern != RESQ_S_NONE;
     if (pattern == RESQ_S_ROW50 && (a.X_up || a.gamma || a.rht)) {

@@ -247,6 +247,29 @@ def test_randomized_hadamard_baseline(shape, pattern, fmt, monkeypatch):
     assert torch.equal(y, y_plain)
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("q", [1, 3])
+@pytest.mark.parametrize("base", [oracle.S_2_4, oracle.S_ROW50, oracle.S_CHAN50, oracle.S_BLOCK])
+def test_sparsity_sweep_linear(base, q, fmt):
+    """The layer with 1/4 and 3/4 of the residual kept (both GEMM routes of the MXFP4 twin)."""
+    m = rq()
+    M, K, N = 288, 512, 600
+    pattern = oracle.keep_quarters(base, q)
+    xb, wb = synth_xw(3 * base + q, M, K, N, n_out=2)
+    want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern, fmt)
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    work = m.alloc_workspace(m.resq_workspace_bytes(M, N, K, pattern, fmt))
+    import os
+    for native in (("1", "0") if fmt == "mxfp4" else ("0",)):
+        os.environ["RESQ_MXFP4_NATIVE"] = native
+        try:
+            y = m.resq_linear(to_dev(xb), wc, ws, pattern, fmt, out_dtype=torch.float32, workspace=work)
+            assert m.check(work) == 0, m.last_error()
+        finally:
+            os.environ.pop("RESQ_MXFP4_NATIVE", None)
+        check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+
+
 def test_swiglu_rejects_row50_and_narrow_input():
     m = rq()
     gu = torch.zeros((64, 512), dtype=torch.bfloat16, device="cuda")

@@ -696,6 +696,54 @@ def test_randomized_hadamard_transform():
     assert np.linalg.norm(o["y"] - exact) < np.linalg.norm(plain - exact)
 
 
+@pytest.mark.parametrize("q", [1, 3])
+def test_sparsity_sweep_masks(q):
+    """Kept share q/4 instead of one half: exact counts for every selecting pattern, brute-force optimality (no
+    kept magnitude / score is smaller than a dropped one, ties resolved toward the lower index) and nesting
+    (the kept set grows with q)."""
+    rng = np.random.default_rng(40 + q)
+    M, K = 64, 256
+    v = np.round(rng.standard_normal((M, K)) * 3).astype(np.float64) / 4      # many ties
+    v[5] = 0.0
+    def unpack(bits):
+        return np.unpackbits(bits, axis=1, bitorder="little").astype(bool)
+    for base in (oracle.S_2_4, oracle.S_ROW50, oracle.S_CHAN50, oracle.S_BLOCK):
+        bits, _ = oracle.mask(v, oracle.keep_quarters(base, q))
+        kept = unpack(bits)
+        half = unpack(oracle.mask(v, base)[0])
+        same = unpack(oracle.mask(v, oracle.keep_quarters(base, 2))[0])
+        assert np.array_equal(half, same)
+        assert np.all(kept <= half) if q == 1 else np.all(half <= kept)          # nested selections
+        a = np.abs(v)
+        if base == oracle.S_2_4:
+            g = kept.reshape(M, K // 4, 4)
+            assert np.all(g.sum(axis=2) == q)
+            ag = a.reshape(M, K // 4, 4)
+            for m in range(M):
+                for j in range(K // 4):
+                    order = sorted(range(4), key=lambda t: (-ag[m, j, t], t))
+                    assert sorted(order[:q]) == list(np.nonzero(g[m, j])[0])
+        elif base == oracle.S_ROW50:
+            assert np.all(kept.sum(axis=1) == K * q // 4)
+            for m in range(M):
+                order = sorted(range(K), key=lambda t: (-a[m, t], t))
+                assert sorted(order[:K * q // 4]) == list(np.nonzero(kept[m])[0])
+        elif base == oracle.S_CHAN50:
+            assert np.all(kept == kept[0]) and kept[0].sum() == K * q // 4
+            score = (v ** 2).sum(axis=0)
+            order = sorted(range(K), key=lambda t: (-score[t], t))
+            assert sorted(order[:K * q // 4]) == list(np.nonzero(kept[0])[0])
+        else:
+            blocks = kept.reshape(M // 32, 32, K // 64, 64)
+            per = blocks.all(axis=(1, 3))
+            assert np.array_equal(per, blocks.any(axis=(1, 3))) and per.sum() == per.size * q // 4
+            score = (v ** 2).reshape(M // 32, 32, K // 64, 64).sum(axis=(1, 3)).reshape(-1)
+            order = sorted(range(score.size), key=lambda t: (-score[t], t))
+            assert sorted(order[:score.size * q // 4]) == list(np.nonzero(per.reshape(-1))[0])
+    with pytest.raises(ValueError):
+        oracle.mask(v, oracle.S_2_4 | (4 << 8))
+
+
 # ----------------------------------------------------------------- regression digest of a seeded tensor
 
 def test_seeded_digest():

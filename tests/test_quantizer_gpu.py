@@ -92,6 +92,26 @@ def test_residual_mask_bit_exact(fmt, pattern, shape):
     assert np.array_equal(mask, want["mask"])
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("q", [1, 3])
+@pytest.mark.parametrize("base", [oracle.S_2_4, oracle.S_ROW50, oracle.S_CHAN50, oracle.S_BLOCK])
+@pytest.mark.parametrize("shape", [(64, 256), (320, 2048), (2432, 192), (32, 4160)])
+def test_sparsity_sweep_masks_bit_exact(shape, base, q, fmt):
+    """Kept share 1/4 and 3/4 (1:4 / 3:4, row-, channel- and block-wise): masks bit-exact against the oracle on
+    shapes that reach every quantizer kernel (chunk-per-lane, block-per-lane, both row-wise kernels)."""
+    M, K = shape
+    pattern = oracle.keep_quarters(base, q)
+    bits = synth(M + K + base + q, M, K, n_out=max(1, K // 256), extremes=base not in (oracle.S_CHAN50, oracle.S_BLOCK))
+    want = oracle.quantize_residual_mask(bf16_bits_to_f32(bits), pattern, fmt)
+    got = rq().residual_mask(to_dev(bits), pattern, fmt)
+    torch.cuda.synchronize()
+    assert np.array_equal(got["r_codes"].cpu().numpy(), want["r_codes"])
+    info = want["mask_info"]
+    if base in (oracle.S_CHAN50, oracle.S_BLOCK) and not (info["exact"] or info["margin"] > 2.0 ** -40):
+        pytest.skip("selection scores not exactly summable and boundary margin too small")
+    assert np.array_equal(got["mask"].cpu().numpy(), want["mask"])
+
+
 @pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4, oracle.S_BLOCK])
 def test_many_rows_per_warp(pattern):
     """Tall, narrow input: every warp of the streaming kernel walks several rows (prefetch ring, row tail)."""
