@@ -278,6 +278,8 @@ def main():
             err["rotation+resq_2:4"] = ((y.double() - exact).norm().item() / norm)
             y = rq.w16a4_linear(x, w, rq.S_NONE, fmt, out_dtype=torch.float32)
             err["w16a4"] = ((y.double() - exact).norm().item() / norm)
+            y = rq.w4a8_linear(x, wc, ws, fmt, out_dtype=torch.float32)
+            err["w4a8"] = ((y.double() - exact).norm().item() / norm)
             y = rq.w4a16_linear(x, wc, ws, fmt, out_dtype=torch.float32)
             err["w4a16"] = ((y.double() - exact).norm().item() / norm)
             table[spec.name] = err

@@ -181,6 +181,23 @@ RESQ_API int mxfp4_w4a16_linear(const void* X_bf16, int64_t M, int64_t K, int64_
                        void* Y, int out_dtype, int64_t ldy,
                        void* workspace, size_t ws_bytes, void* stream);
 
+/* Weight-and-8-bit-activation ablation of Table 1 ("W4A8"): Y = deq(Q8(X)) deq(Q(W))^T.  The paper names the
+ * ablation but not the 8-bit format; this library's reading is MXFP8 with E4M3 elements as the OCP microscaling
+ * specification defines it: blocks of 32 along K, one E8M0 scale 2^(floor(log2 amax) - 8) per block (all-zero
+ * block: scale code 0), elements rounded to the nearest E4M3 value (ties to even, subnormals below 2^-6) and
+ * saturated at +-448; used with both weight formats.  K % 32 == 0 (K % 64 == 0 with HiF4 weights).  No residual
+ * term.  Decoded activations below 2^-126 in magnitude lose bits (the GEMM operand is bf16).  Same argument
+ * rules, output types and error behaviour as *_resq_linear; workspace of resq_w4a8_workspace_bytes(M, N, K). */
+RESQ_API size_t resq_w4a8_workspace_bytes(int64_t M, int64_t N, int64_t K);
+RESQ_API int hif4_w4a8_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
+                     const void* w_codes, const void* w_meta, int64_t N,
+                     void* Y, int out_dtype, int64_t ldy,
+                     void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_w4a8_linear(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
+                      const void* w_codes, const void* w_scale, int64_t N,
+                      void* Y, int out_dtype, int64_t ldy,
+                      void* workspace, size_t ws_bytes, void* stream);
+
 /* Down projection with its producer fused into the quantizer pass: the input is GU_bf16 = [gate | up], [M, 2K]
  * device (row pitch ldgu >= 2K elements, ldgu % 8 == 0, 16-byte aligned base), the layer's activations are
  * X = bf16(SiLU(gate) * up), formed on the fly and never written to memory; everything after that is

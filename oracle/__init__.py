@@ -367,3 +367,53 @@ def rht_resq_linear(x_f32: np.ndarray, w_f32: np.ndarray, signs: int, pattern: i
     out["x"] = x
     out["w_rot"] = w
     return out
+
+
+# ---- 8-bit activations for the "W4A8" ablation of Table 1 -----------------------------------------------------
+# The paper names the ablation but not the 8-bit format.  Reading of this project: MXFP8 with E4M3 elements as the
+# OCP microscaling specification defines it -- blocks of 32 along K, one E8M0 power-of-two scale
+# 2^(floor(log2 amax) - 8) per block (8 = exponent of the largest E4M3 value, 448 = 1.75 * 2^8; all-zero block:
+# scale code 0), elements rounded to the nearest E4M3 value (4 exponent bits, bias 7, 3 mantissa bits, subnormals
+# below 2^-6, ties to even) and saturated at +-448.  Used for both weight formats.
+def e4m3_value(code: int) -> float:
+    s = -1.0 if code & 0x80 else 1.0
+    e, m = (code >> 3) & 15, code & 7
+    if e == 15 and m == 7:
+        return float("nan")
+    return s * (m / 8.0 * 2.0 ** -6 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7))
+
+
+def mxfp8_e4m3_quantize(x: np.ndarray):
+    """x float32 [rows, K] -> (codes uint8 [rows, K], scale uint8 [rows, K/32], decoded float64 [rows, K])."""
+    x = np.asarray(x, dtype=np.float64)
+    rows, K = x.shape
+    if K % 32:
+        raise ValueError("MXFP8 needs K % 32 == 0")
+    xb = x.reshape(rows, K // 32, 32)
+    amax = np.abs(xb).max(axis=2)
+    e = np.full(amax.shape, -127, dtype=np.int64)
+    nz = amax > 0
+    # floor(log2 amax) through frexp (exact at powers of two)
+    _, ex = np.frexp(amax[nz])
+    e[nz] = np.clip(ex.astype(np.int64) - 1 - 8, -127, 127)
+    t = np.abs(xb) / np.exp2(e.astype(np.float64))[:, :, None]            # exact scaling
+    # spacing of the E4M3 grid at t: 2^-9 below 2^-6, else 2^(floor(log2 t) - 3)
+    _, tex = np.frexp(np.maximum(t, 2.0 ** -6))
+    step = np.exp2((tex - 1 - 3).astype(np.float64))
+    q = np.minimum(np.rint(t / step) * step, 448.0)                        # rint: ties to even; exact quotient
+    deq = np.copysign(q, xb) * np.exp2(e.astype(np.float64))[:, :, None]
+    # codes (for the table pins): sign | exponent field | mantissa
+    _, qex = np.frexp(np.maximum(q, 2.0 ** -7))
+    ef = np.where(q < 2.0 ** -6, 0, qex - 1 + 7)
+    mf = np.where(q < 2.0 ** -6, np.rint(q * 2.0 ** 9), np.rint((q / np.exp2((qex - 1).astype(np.float64)) - 1.0) * 8))
+    codes = ((np.signbit(xb).astype(np.int64) << 7) | (ef.astype(np.int64) << 3) | mf.astype(np.int64)).astype(np.uint8)
+    return codes.reshape(rows, K), (e + 127).astype(np.uint8), deq.reshape(rows, K)
+
+
+def w4a8_linear(x_f32: np.ndarray, w_f32: np.ndarray, fmt: str = "hif4", want_abs: bool = True) -> Dict[str, np.ndarray]:
+    """Table 1, W4A8: Y = deq(Q8(X)) deq(Q4(W))^T with MXFP8-E4M3 activations and 4-bit weights."""
+    codes, scale, a = mxfp8_e4m3_quantize(x_f32)
+    w_codes, w_side = encode(fmt, _f32(w_f32))
+    w = decode(fmt, w_codes, w_side)
+    y, ab = matmul(a, None, w, want_abs)
+    return {"a_codes": codes, "a_scale": scale, "a": a, "w": w, "y": y, "abs_sum": ab}

@@ -45,6 +45,9 @@ SYMBOLS = {
     "hif4_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "mxfp4_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "resq_w4a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "resq_w4a8_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "hif4_w4a8_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "mxfp4_w4a8_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
     "hif4_w4a16_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
     "mxfp4_w4a16_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
     "hif4_swiglu_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
@@ -335,6 +338,27 @@ def rmsnorm_resq_linear(H: torch.Tensor, gamma: torch.Tensor, eps: float, w_code
         H.data_ptr(), M, K, H.stride(0), gamma.data_ptr(), float(eps), w_codes.data_ptr(), w_side.data_ptr(), N, pattern,
         Y.data_ptr(), OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32, Y.stride(0), workspace.data_ptr(),
         workspace.numel(), _stream(stream)))
+    return Y
+
+
+def w4a8_linear(X: torch.Tensor, w_codes: torch.Tensor, w_side: torch.Tensor, fmt: str = "hif4",
+                out_dtype: torch.dtype = torch.bfloat16, Y: Optional[torch.Tensor] = None,
+                workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """*_w4a8_linear: Y = deq(MXFP8-E4M3(X)) deq(Q(W))^T (Table 1, W4A8; the 8-bit format is this library's reading)."""
+    _require_bf16_matrix(X, "X")
+    M, K = X.shape
+    N = w_codes.shape[0]
+    if Y is None:
+        ld = (N + 7) // 8 * 8
+        Y = torch.empty((M, ld), dtype=out_dtype, device=X.device)[:, :N]
+    if Y.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("Y must be bf16 or fp32")
+    if workspace is None:
+        workspace = alloc_workspace(int(lib().resq_w4a8_workspace_bytes(M, N, K)), X.device)
+    _check(_fn(fmt, "hif4_w4a8_linear", "mxfp4_w4a8_linear")(
+        X.data_ptr(), M, K, X.stride(0), w_codes.data_ptr(), w_side.data_ptr(), N, Y.data_ptr(),
+        OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32, Y.stride(0), workspace.data_ptr(), workspace.numel(),
+        _stream(stream)))
     return Y
 
 

@@ -457,6 +457,67 @@ int w4a16_linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, cons
     return launch_gemm_hif4(g, st);
 }
 
+// "W4A8" (Table 1): 8-bit activations (MXFP8-E4M3, see include/resq.h) against the packed 4-bit weights.
+// Workspace: [header | counters | bf16 image of the decoded activations | fp32 partial tiles].
+size_t w4a8_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    return kWsHeader + kWsFlags + align_up((size_t)M * (size_t)K * 2, 256) + align_up(gemm_hif4_scratch_bytes(M, N, K), 256);
+}
+
+int w4a8_linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_side, int64_t N,
+                void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    int rc = check_matrix(X, M, K, ldx, fmt, "X");
+    if (rc) return rc;
+    if (K % 32 != 0) {
+        set_last_error("w4a8_linear: K must be a multiple of 32 (K=%lld)", (long long)K);
+        return RESQ_ERR_SHAPE;
+    }
+    if (!w_codes || !w_side || !Y) {
+        set_last_error("w4a8_linear: NULL weight or output pointer");
+        return RESQ_ERR_NULL;
+    }
+    if (N <= 0) {
+        set_last_error("w4a8_linear: N=%lld", (long long)N);
+        return RESQ_ERR_SHAPE;
+    }
+    if (out_dtype != RESQ_OUT_BF16 && out_dtype != RESQ_OUT_F32) {
+        set_last_error("unknown output type %d", out_dtype);
+        return RESQ_ERR_PATTERN;
+    }
+    if (!aligned16(Y) || !aligned16(w_codes) || !aligned16(w_side) || ldy < N ||
+        ldy % (out_dtype == RESQ_OUT_BF16 ? 8 : 4) != 0) {
+        set_last_error("w4a8_linear: Y / weights need 16-byte aligned bases, ldy >= N and 16-byte aligned rows");
+        return RESQ_ERR_ALIGN;
+    }
+    rc = check_workspace(workspace, ws_bytes, w4a8_workspace_bytes(M, N, K));
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    __nv_bfloat16* img = reinterpret_cast<__nv_bfloat16*>(ws + kWsHeader + kWsFlags);
+    rc = launch_quantize_mxfp8_image(static_cast<const __nv_bfloat16*>(X), M, K, ldx, img, reinterpret_cast<uint32_t*>(ws),
+                                     (int)((kWsHeader + kWsFlags) / 4), st);
+    if (rc) return rc;
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.fmt = fmt;
+    g.a_bf16 = img;
+    g.w_codes = static_cast<const uint8_t*>(w_codes);
+    g.w_side = w_side;
+    g.M = M;
+    g.N = N;
+    g.K = K;
+    g.Y = Y;
+    g.out_dtype = out_dtype;
+    g.ldy = ldy;
+    g.partial_bytes = gemm_hif4_scratch_bytes(M, N, K);
+    g.splitk_partials = g.partial_bytes ? reinterpret_cast<float*>(ws + kWsHeader + kWsFlags + align_up((size_t)M * (size_t)K * 2, 256))
+                                        : nullptr;
+    g.splits = (int)(g.partial_bytes / ((size_t)M * (size_t)N * 4));
+    g.sk_flags = reinterpret_cast<unsigned int*>(ws + kWsHeader);
+    g.status = reinterpret_cast<DeviceStatus*>(ws);
+    return launch_gemm_hif4(g, st);
+}
+
 }  // namespace
 }  // namespace resq
 
@@ -581,6 +642,16 @@ int mxfp4_w16a4_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const v
         return RESQ_ERR_NULL;
     }
     return linear(kMXFP4, X, M, K, ldx, nullptr, nullptr, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream, W, ldw);
+}
+
+size_t resq_w4a8_workspace_bytes(int64_t M, int64_t N, int64_t K) { return w4a8_workspace_bytes(M, N, K); }
+int hif4_w4a8_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_meta, int64_t N, void* Y,
+                     int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    return w4a8_linear(kHiF4, X, M, K, ldx, w_codes, w_meta, N, Y, out_dtype, ldy, workspace, ws_bytes, stream);
+}
+int mxfp4_w4a8_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* w_codes, const void* w_scale, int64_t N, void* Y,
+                      int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    return w4a8_linear(kMXFP4, X, M, K, ldx, w_codes, w_scale, N, Y, out_dtype, ldy, workspace, ws_bytes, stream);
 }
 
 size_t resq_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) { return w4a16_workspace_bytes(M, N, K); }

@@ -1356,6 +1356,60 @@ size_t quant_scratch_bytes(int64_t M, int64_t K, int pattern) {
     return align_up(n * sizeof(double), 256) + align_up(n, 256);
 }
 
+// 8-bit activations of the "W4A8" ablation: MXFP8 with E4M3 elements (blocks of 32 along K, E8M0 scale
+// 2^(floor(log2 amax) - 8), elements rounded to nearest even and saturated at 448).  Only the decoded image is
+// needed (the GEMM takes a bf16 operand; an E4M3 value times a power of two is exact in bf16).  A lane owns 8
+// values, an aligned quad of lanes a block.
+__global__ void __launch_bounds__(kThreads) quant_mxfp8_image_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K,
+                                                                     int64_t ldx, __nv_bfloat16* __restrict__ img,
+                                                                     uint32_t* clear_words, int n_clear_words) {
+    pdl_wait();
+    pdl_trigger();
+    if (clear_words && blockIdx.x == 0)
+        for (int i = threadIdx.x; i < n_clear_words; i += blockDim.x) clear_words[i] = 0u;
+    const int lane = threadIdx.x & 31;
+    const int64_t chunks_per_row = K / 8;
+    const int64_t total = M * chunks_per_row;  // K % 32 == 0: whole quads are in range or not
+    for (int64_t c0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) - lane; c0 < total; c0 += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t c = c0 + lane;
+        const bool active = c < total;
+        const int64_t m = active ? c / chunks_per_row : 0, k0 = active ? (c % chunks_per_row) * 8 : 0;
+        float x[8];
+        uint4 raw = make_uint4(0, 0, 0, 0);
+        if (active) raw = ld_nc_16(X + m * ldx + k0);
+        unpack_bf16x8(raw, x);
+        float m8 = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) m8 = fmaxf(m8, fabsf(x[i]));
+        const uint32_t ab = __reduce_max_sync(0xFu << (lane & 28), __float_as_uint(m8));
+        const int e = ab == 0u ? -127 : max((int)(ab >> 23) - 127 - 8, -127);
+        const float inv = __uint_as_float((uint32_t)(127 - e) << 23);                          // 2^-e, exact
+        const float scale = __uint_as_float(e == -127 ? 0x00400000u : (uint32_t)(e + 127) << 23);  // 2^e
+        uint32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint16_t pk;
+            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pk) : "f"(__fmul_rn(x[2 * i + 1], inv)), "f"(__fmul_rn(x[2 * i], inv)));
+            uint32_t h2;
+            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(pk));
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+            const __nv_bfloat162 b = __floats2bfloat162_rn(__fmul_rn(f.x, scale), __fmul_rn(f.y, scale));
+            o[i] = *reinterpret_cast<const uint32_t*>(&b);
+        }
+        if (active) *reinterpret_cast<uint4*>(img + m * K + k0) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+int launch_quantize_mxfp8_image(const __nv_bfloat16* X, int64_t M, int64_t K, int64_t ldx, __nv_bfloat16* img, uint32_t* clear_words,
+                                int n_clear_words, cudaStream_t stream) {
+    const int64_t threads = M * (K / 8);
+    const unsigned ctas = (unsigned)std::min<int64_t>((threads + kThreads - 1) / kThreads, 148 * 16);
+    LaunchScope scope(kKindQuant, stream);
+    return cuda_fail(launch_kernel(quant_mxfp8_image_kernel, dim3(ctas), dim3(kThreads), 0, stream, X, M, K, ldx, img, clear_words,
+                                   n_clear_words),
+                     "quant_mxfp8_image_kernel launch");
+}
+
 // Second and third kernel of the patterns with a tensor-wide selection (CHAN50, BLOCK): top half of the scores,
 // then the mask pass over the residual outputs.
 static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t stream) {

@@ -270,6 +270,35 @@ def test_sparsity_sweep_linear(base, q, fmt):
         check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("shape", [(64, 256, 200), (300, 1152, 520), (1056, 512, 1100)])
+def test_w4a8_linear_parity(shape, fmt):
+    """W4A8 (Table 1) with MXFP8-E4M3 activations: within tolerance of the oracle and bit-identical to the W4A16
+    call on the oracle's decoded 8-bit activations (so every activation is quantized exactly as the oracle does:
+    block scales, ties, saturation, zero blocks, an outlier that pushes its block into the subnormal codes)."""
+    m = rq()
+    M, K, N = shape
+    xb, wb = synth_xw(19 * M + N, M, K, N, n_out=max(1, K // 256))
+    xf = bf16_bits_to_f32(xb).copy()
+    xf[0, :32] = 0.0
+    xf[1, 7] *= 300.0
+    xf[2, :64] = np.float32(448.0) * np.float32(2.0 ** -3)       # exactly at the largest code
+    xb = f32_to_bf16_bits(xf)
+    want = oracle.w4a8_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), fmt)
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    big = torch.zeros((M, K + 24), dtype=torch.bfloat16, device="cuda")
+    big[:, :K] = to_dev(xb)
+    a_dev = to_dev(f32_to_bf16_bits(want["a"].astype(np.float32)))
+    y_ref = m.w4a16_linear(a_dev, wc, ws, fmt, out_dtype=torch.float32)
+    for x in (to_dev(xb), big[:, :K]):
+        y = m.w4a8_linear(x, wc, ws, fmt, out_dtype=torch.float32)
+        torch.cuda.synchronize()
+        check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+        assert torch.equal(y, y_ref)
+    yb = m.w4a8_linear(to_dev(xb), wc, ws, fmt, out_dtype=torch.bfloat16)
+    check_close(yb.float().cpu().numpy(), want["y"], want["abs_sum"], bf16_out=True)
+
+
 def test_swiglu_rejects_row50_and_narrow_input():
     m = rq()
     gu = torch.zeros((64, 512), dtype=torch.bfloat16, device="cuda")

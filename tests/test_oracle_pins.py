@@ -744,6 +744,49 @@ def test_sparsity_sweep_masks(q):
         oracle.mask(v, oracle.S_2_4 | (4 << 8))
 
 
+def test_mxfp8_e4m3_activations_for_w4a8():
+    """8-bit activations of the W4A8 ablation (this project's reading: MXFP8, E4M3 elements): the value table and
+    the element rounding against torch's float8_e4m3fn, the scale property 256 <= amax / 2^e < 512, saturation,
+    round trip of representable blocks, and the exact rational product on a tiny case."""
+    import torch
+    codes = np.arange(256, dtype=np.uint8)
+    tv = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float32).numpy()
+    ov = np.array([oracle.e4m3_value(int(c)) for c in codes])
+    assert np.array_equal(np.isnan(tv), np.isnan(ov)) and np.array_equal(tv[~np.isnan(tv)], ov[~np.isnan(ov)])
+    rng = np.random.default_rng(31)
+    x = bf16_round((rng.standard_normal((16, 128)) * np.exp2(rng.integers(-20, 20, (16, 1)))).astype(np.float32))
+    x[3, :32] = 0.0
+    x[4, 5] *= 300.0                                                     # an outlier: the rest of its block goes subnormal
+    c, sc, deq = oracle.mxfp8_e4m3_quantize(x)
+    e = sc.astype(np.int64) - 127
+    amax = np.abs(x.reshape(16, 4, 32)).max(axis=2).astype(np.float64)
+    nz = amax > 0
+    r = amax[nz] / np.exp2(e[nz].astype(np.float64))
+    assert np.all((r >= 256) & (r < 512)) and np.all(sc[~nz] == 0)
+    t = (x.reshape(16, 4, 32).astype(np.float64) / np.exp2(e.astype(np.float64))[:, :, None]).astype(np.float32)
+    tt = torch.from_numpy(t).clamp(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8).numpy().reshape(16, 128)
+    same = (tt & 0x7F) == (c & 0x7F)                                     # (torch keeps the sign of a rounded-to-zero value too)
+    assert np.all(same) and np.array_equal(tt >> 7, c >> 7)
+    dec = np.array([oracle.e4m3_value(int(v)) for v in c.reshape(-1)]).reshape(16, 4, 32) * np.exp2(e.astype(np.float64))[:, :, None]
+    assert np.array_equal(dec.reshape(16, 128), deq)
+    assert np.all(np.abs(deq) <= 448 * np.exp2(e.astype(np.float64)).repeat(32, axis=1))
+    assert np.all(np.abs(deq - x) <= np.maximum(2.0 ** -4 * np.abs(x), 2.0 ** -10 * np.exp2(e.astype(np.float64)).repeat(32, axis=1)) + 64 * np.exp2(e.astype(np.float64)).repeat(32, axis=1) * (np.abs(x) > 448 * np.exp2(e.astype(np.float64)).repeat(32, axis=1)))
+    c2, sc2, deq2 = oracle.mxfp8_e4m3_quantize(deq.astype(np.float32))  # representable blocks come back unchanged
+    assert np.array_equal(deq2, deq)
+    M, K, N = 3, 64, 4
+    xs = bf16_round(rng.standard_normal((M, K)).astype(np.float32))
+    w = bf16_round(rng.standard_normal((N, K)).astype(np.float32) * 0.02)
+    o = oracle.w4a8_linear(xs, w, "hif4")
+    av, wv = _to_frac(o["a"]), _to_frac(o["w"])
+    for m in range(M):
+        for n in range(N):
+            assert F(float(o["y"][m, n])) == sum(av[m][k] * wv[n][k] for k in range(K))
+    # 8-bit activations sit between the 4-bit and the unquantized ones
+    exact = oracle.w4a16_linear(xs, w, "hif4")["y"]
+    four = oracle.resq_linear(xs, w, oracle.S_NONE, "hif4")["y"]
+    assert np.linalg.norm(o["y"] - exact) < np.linalg.norm(four - exact)
+
+
 # ----------------------------------------------------------------- regression digest of a seeded tensor
 
 def test_seeded_digest():
