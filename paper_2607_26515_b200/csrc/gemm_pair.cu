@@ -601,18 +601,25 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             }
             ptx::tc_fence_after();
             const int64_t m = tc.m0 + rank * kBM + quad * 32 + lane;
+            // a warp whose 32 rows all lie past M (decode-sized calls fill a fraction of the 256-row tile) has
+            // nothing to read or store: it only hands the accumulator back
+            const bool warp_has_rows = tc.m0 + rank * kBM + quad * 32 < p.M;
 #pragma unroll 1
-            for (int cc = 0; cc < nchunks; ++cc) {
+            for (int cc = warp_has_rows ? 0 : nchunks - 1; cc < nchunks; ++cc) {
                 uint32_t v[32];
-                ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * TN + cc * 32), v);
-                ptx::tmem_ld_wait();
+                if (warp_has_rows) {
+                    ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * TN + cc * 32), v);
+                    ptx::tmem_ld_wait();
+                }
                 if (cc == nchunks - 1) {
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(&acc_empty[buf], 0));
                 }
+                if (!warp_has_rows) continue;
                 if (p.streamk && tc.partial) {
-                    // dense fp32 slot [256][TN]; rows / columns outside the matrix hold zeros
+                    // fp32 slot [256][TN]; the sum reads rows below M only, so rows past M are not written
+                    if (m >= p.M) continue;
                     float* dst = p.sk_slots + ((size_t)tc.slot * (2 * kBM) + rank * kBM + quad * 32 + lane) * TN + cc * 32;
 #pragma unroll
                     for (int j = 0; j < 32; j += 8)
