@@ -814,32 +814,47 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
 // staging buffers), so that the K/2 largest magnitudes can be selected and the image masked before it leaves.
 // Selection: most significant bit first over the 15 magnitude bits, counting with warp reductions only; ties
 // at the threshold are kept lowest index first.  Shared memory per warp: (3 + segments) staging tiles.
-template <int FMT, bool IMG>
+// WPR = 1: a warp per row (rows of up to two segments).  WPR = 8: the eight warps of a CTA share one row (up to 16
+// segments, warp w takes segments w and w + 8); the per-bit counts and the tie counts of the segments are summed
+// through shared memory with one CTA barrier each.
+template <int FMT, bool IMG, int WPR>
 __global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs a, int warps_per_cta) {
     pdl_wait();
     pdl_trigger();
     if (a.clear_words && blockIdx.x == 0)
         for (int i = threadIdx.x; i < a.n_clear_words; i += blockDim.x) a.clear_words[i] = 0u;
     extern __shared__ __align__(16) uint8_t smem_q[];
+    __shared__ int s_cnt[2][16];   // WPR > 1: candidates with bit b set, summed over the row's warps (alternating per row)
+    __shared__ int s_ties[16];     // WPR > 1: entries equal to the threshold, per segment
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (warp >= warps_per_cta) return;  // warps are independent: no CTA-wide barrier below
-    const int64_t m = (int64_t)blockIdx.x * warps_per_cta + warp;
-    if (m >= a.M) return;
+    const int wr = WPR == 1 ? 0 : warp;  // rank of the warp in its row's team
+    if (WPR == 1 && warp >= warps_per_cta) return;  // warps are independent: no CTA-wide barrier below
+    // WPR > 1: the CTA walks rows blockIdx.x, blockIdx.x + gridDim.x, ... and loads the next row while it selects
+    int64_t m = WPR == 1 ? (int64_t)blockIdx.x * warps_per_cta + warp : (int64_t)blockIdx.x;
+    const int64_t m_step = WPR == 1 ? a.M : (int64_t)gridDim.x;
+    if (WPR == 1 && m >= a.M) return;
+    if (WPR > 1) {
+        if (threadIdx.x < 32) s_cnt[threadIdx.x >> 4][threadIdx.x & 15] = 0;
+        __syncthreads();
+    }
     const int64_t G = a.K / kHif4Block;
-    const int nseg = (int)((G + 31) / 32);
-    const uint32_t base = smem_u32(smem_q) + (uint32_t)(warp * (3 + nseg) * kStageBytes);
+    const int nseg_row = (int)((G + 31) / 32);                                   // segments of the row
+    const int nseg = WPR == 1 ? nseg_row : max(0, (nseg_row - wr + WPR - 1) / WPR);  // segments of this warp (at most 2)
+    const int seg_cap = WPR == 1 ? nseg_row : (nseg_row + WPR - 1) / WPR;           // row-image tiles per warp
+    auto gseg = [&](int ls) -> int { return wr + ls * WPR; };                      // local -> row segment
+    const uint32_t base = smem_u32(smem_q) + (uint32_t)(warp * (3 + seg_cap) * kStageBytes);
     const uint32_t in0 = base, stage = base + 2 * kStageBytes, rrow = base + 3 * kStageBytes;
     const int cp_blk = lane >> 3, cp_ch = lane & 7;
     const uint32_t cp_smem = (uint32_t)(cp_blk * kStagePitch + cp_ch * 16);
     const uint32_t my_in = (uint32_t)(lane * kStagePitch);
     auto seg_col = [&](int seg) -> int64_t { return ((int64_t)seg * 32 + cp_blk) * kHif4Block + cp_ch * 8; };
-    auto issue_seg = [&](int seg, uint32_t buf) {
+    auto issue_seg = [&](int seg, uint32_t buf, int64_t row) {
         const int64_t col = seg_col(seg);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const bool valid = col + j * 4 * kHif4Block < a.K;
             cp_async_16(buf + cp_smem + j * 4 * kStagePitch,
-                        valid ? (const void*)(a.X + m * a.ldx + col + j * 4 * kHif4Block) : (const void*)a.X, valid);
+                        valid ? (const void*)(a.X + row * a.ldx + col + j * 4 * kHif4Block) : (const void*)a.X, valid);
         }
     };
     auto drain = [&](uint32_t src, __nv_bfloat16* dst_row, int seg) {
@@ -853,13 +868,20 @@ __global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs
         __syncwarp();
     };
 
+    bool loaded = false;  // the first two segments of row m are already on their way
+    for (int row_it = 0; m < a.M; m += m_step, ++row_it) {
+    int* const cnt_row = s_cnt[row_it & 1];
+    if (WPR > 1 && row_it > 0 && threadIdx.x < 16) s_cnt[(row_it + 1) & 1][threadIdx.x] = 0;  // for the next row
     // ---- phase A: both encodes, segment by segment
-    issue_seg(0, in0);
-    cp_async_commit();
-    if (nseg > 1) issue_seg(1, in0 + kStageBytes);
-    cp_async_commit();
-    for (int seg = 0; seg < nseg; ++seg) {
-        const uint32_t buf = in0 + (uint32_t)((seg & 1) * kStageBytes);
+    if (!loaded) {
+        if (nseg > 0) issue_seg(gseg(0), in0, m);
+        cp_async_commit();
+        if (nseg > 1) issue_seg(gseg(1), in0 + kStageBytes, m);
+        cp_async_commit();
+    }
+    for (int ls = 0; ls < nseg; ++ls) {
+        const int seg = gseg(ls);
+        const uint32_t buf = in0 + (uint32_t)((ls & 1) * kStageBytes);
         cp_async_wait<1>();
         __syncwarp();
         uint32_t w[32];
@@ -869,7 +891,7 @@ __global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs
             w[4 * c] = v.x; w[4 * c + 1] = v.y; w[4 * c + 2] = v.z; w[4 * c + 3] = v.w;
         }
         __syncwarp();
-        if (seg + 2 < nseg) issue_seg(seg + 2, buf);
+        if (ls + 2 < nseg) issue_seg(gseg(ls + 2), buf, m);
         cp_async_commit();
         const int64_t blk = (int64_t)seg * 32 + lane;
         const bool active = blk < G;
@@ -898,7 +920,7 @@ __global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs
         }
         if constexpr (IMG) drain(stage, a.a_bf16 + m * a.K, seg);
         uint32_t rcodes[8], rside;
-        const uint32_t rdst = rrow + (uint32_t)(seg * kStageBytes) + my_in;
+        const uint32_t rdst = rrow + (uint32_t)(ls * kStageBytes) + my_in;
         encode_block<FMT, true, false>(w, rcodes, rside, [&](int c, const float (&)[8], const float (&rdq)[8], uint32_t) {
             uint32_t img[4];
 #pragma unroll
@@ -920,57 +942,125 @@ __global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs
     }
     cp_async_wait<0>();
     __syncwarp();
+    loaded = false;
+    if (WPR > 1 && m + m_step < a.M) {  // the input staging tiles are free: the next row loads during phases B and C
+        if (nseg > 0) issue_seg(gseg(0), in0, m + m_step);
+        cp_async_commit();
+        if (nseg > 1) issue_seg(gseg(1), in0 + kStageBytes, m + m_step);
+        cp_async_commit();
+        loaded = true;
+    }
 
-    // ---- phase B: the (K/2)-th largest 15-bit magnitude of the row (inactive blocks hold zeros: they never win)
-    unsigned prefix = 0u;
-    int remaining = (int)(a.K * a.keep_quarters / 4);
-    for (int b = 14; b >= 0; --b) {
-        const unsigned cand = prefix | (1u << b);
-        const uint32_t cand2 = (cand >> b) * 0x00010001u;
-        const uint32_t mask2 = (0x7FFFu >> b) * 0x00010001u;
-        int cnt = 0;
-        for (int seg = 0; seg < nseg; ++seg) {
+    // ---- phase B: the keep-th largest 15-bit magnitude of the row, on bit planes.  The lane's 64 magnitudes of a
+    // segment are 32 words of two 16-bit halves: a 32 x 32 bit-matrix transpose turns them into planes -- word b
+    // holds bit b of the even elements (element 2r at bit r), word 16 + b that of the odd elements.  The most-
+    // significant-bit-first select then costs two population counts and a warp sum per bit; the sets "equal to the
+    // threshold" and "greater" fall out as masks.
+    constexpr int kMaxSeg = 2;                    // the launcher sends longer rows to the CTA-per-row kernel
+    uint32_t plane[kMaxSeg][32];
+    uint32_t c_even[kMaxSeg], c_odd[kMaxSeg], g_even[kMaxSeg], g_odd[kMaxSeg];
+#pragma unroll
+    for (int seg = 0; seg < kMaxSeg; ++seg) {
+        c_even[seg] = c_odd[seg] = g_even[seg] = g_odd[seg] = 0u;
+        if (seg < nseg) {
             const uint32_t src = rrow + (uint32_t)(seg * kStageBytes) + my_in;
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const uint4 v = lds_16(src + c * 16);
-                const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+                plane[seg][4 * c] = v.x; plane[seg][4 * c + 1] = v.y; plane[seg][4 * c + 2] = v.z; plane[seg][4 * c + 3] = v.w;
+            }
+            // transpose: afterwards bit r of word c is bit c of the former word r
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t z = (((w4[i] & 0x7FFF7FFFu) >> b) & mask2) ^ cand2;
-                    cnt += ((z & 0xFFFFu) == 0u) + ((z >> 16) == 0u);
+            for (int lg = 4; lg >= 0; --lg) {
+                const int j = 1 << lg;
+                const uint32_t msk = j == 16 ? 0x0000FFFFu : j == 8 ? 0x00FF00FFu : j == 4 ? 0x0F0F0F0Fu : j == 2 ? 0x33333333u : 0x55555555u;
+#pragma unroll
+                for (int k = 0; k < 32; ++k) {
+                    if ((k & j) == 0) {
+                        const uint32_t t = ((plane[seg][k] >> j) ^ plane[seg][k + j]) & msk;
+                        plane[seg][k] ^= t << j;
+                        plane[seg][k + j] ^= t;
+                    }
+                }
+            }
+            const bool seg_active = (int64_t)gseg(seg) * 32 + lane < G;
+            c_even[seg] = c_odd[seg] = seg_active ? 0xFFFFFFFFu : 0u;   // candidates: every element of an existing block
+        }
+    }
+    int remaining = (int)(a.K * a.keep_quarters / 4);
+#pragma unroll
+    for (int b = 14; b >= 0; --b) {
+        int cnt = 0;
+#pragma unroll
+        for (int seg = 0; seg < kMaxSeg; ++seg)
+            if (seg < nseg) cnt += __popc(c_even[seg] & plane[seg][b]) + __popc(c_odd[seg] & plane[seg][16 + b]);
+        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+        if (WPR > 1) {
+            if (lane == 0 && cnt) atomicAdd(&cnt_row[b], cnt);
+            __syncthreads();
+            cnt = cnt_row[b];
+        }
+        const bool take = cnt >= remaining;       // the threshold has this bit set: candidates without it fall below
+        if (!take) remaining -= cnt;
+#pragma unroll
+        for (int seg = 0; seg < kMaxSeg; ++seg) {
+            if (seg < nseg) {
+                const uint32_t one_e = c_even[seg] & plane[seg][b], one_o = c_odd[seg] & plane[seg][16 + b];
+                if (take) {
+                    c_even[seg] = one_e;
+                    c_odd[seg] = one_o;
+                } else {                          // candidates with the bit are above the threshold
+                    g_even[seg] |= one_e;
+                    g_odd[seg] |= one_o;
+                    c_even[seg] ^= one_e;
+                    c_odd[seg] ^= one_o;
                 }
             }
         }
-        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
-        if (cnt >= remaining) prefix = cand;
-        else remaining -= cnt;
     }
-    const uint32_t T = prefix;   // threshold magnitude
-    int need = remaining;        // entries equal to T that are kept, lowest index first
+    int need = remaining;        // entries equal to the threshold that are kept, lowest index first
+    // masks of even / odd elements -> element order (element e at bit e of a 64-bit mask)
+    auto spread16 = [](uint32_t x) -> uint32_t {
+        x &= 0xFFFFu;
+        x = (x | (x << 8)) & 0x00FF00FFu;
+        x = (x | (x << 4)) & 0x0F0F0F0Fu;
+        x = (x | (x << 2)) & 0x33333333u;
+        x = (x | (x << 1)) & 0x55555555u;
+        return x;
+    };
 
     // ---- phase C: masks in index order (segment, lane, position), masked image, masked codes
-    for (int seg = 0; seg < nseg; ++seg) {
+    const int need_row = need;
+    if (WPR > 1) {  // ties of every segment of the row, so that each warp knows how many come before its segments
+#pragma unroll
+        for (int ls = 0; ls < kMaxSeg; ++ls)
+            if (ls < nseg) {
+                const int t = __reduce_add_sync(0xFFFFFFFFu, __popc(c_even[ls]) + __popc(c_odd[ls]));
+                if (lane == 0) s_ties[gseg(ls)] = t;
+            }
+        __syncthreads();
+    }
+    for (int ls = 0; ls < nseg; ++ls) {
+        const int seg = gseg(ls);
+        if (WPR > 1) {
+            int before = 0;
+            for (int q = 0; q < seg; ++q) before += s_ties[q];
+            need = max(0, need_row - before);
+        }
         const int64_t blk = (int64_t)seg * 32 + lane;
         const bool active = blk < G;
-        const uint32_t src = rrow + (uint32_t)(seg * kStageBytes) + my_in;
+        const uint32_t src = rrow + (uint32_t)(ls * kStageBytes) + my_in;
         uint32_t wv[32];
-        uint32_t gt[2] = {0u, 0u}, eq[2] = {0u, 0u};  // bit per element of the lane's block (low / high 32)
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
             const uint4 v = lds_16(src + c * 16);
             wv[4 * c] = v.x; wv[4 * c + 1] = v.y; wv[4 * c + 2] = v.z; wv[4 * c + 3] = v.w;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t klo = wv[4 * c + i] & 0x7FFFu, khi = (wv[4 * c + i] >> 16) & 0x7FFFu;
-                const int e = 8 * c + 2 * i;
-                gt[e >> 5] |= (uint32_t)(klo > T) << (e & 31);
-                gt[(e + 1) >> 5] |= (uint32_t)(khi > T) << ((e + 1) & 31);
-                eq[e >> 5] |= (uint32_t)(klo == T) << (e & 31);
-                eq[(e + 1) >> 5] |= (uint32_t)(khi == T) << ((e + 1) & 31);
-            }
         }
-        if (!active) eq[0] = eq[1] = gt[0] = gt[1] = 0u;
+        // bit per element of the lane's block (low / high 32): greater than / equal to the threshold
+        const uint32_t ce = ls == 0 ? c_even[0] : c_even[1], co = ls == 0 ? c_odd[0] : c_odd[1];
+        const uint32_t ge = ls == 0 ? g_even[0] : g_even[1], go = ls == 0 ? g_odd[0] : g_odd[1];
+        uint32_t gt[2] = {spread16(ge) | (spread16(go) << 1), spread16(ge >> 16) | (spread16(go >> 16) << 1)};
+        uint32_t eq[2] = {spread16(ce) | (spread16(co) << 1), spread16(ce >> 16) | (spread16(co >> 16) << 1)};
         const int mine = __popc(eq[0]) + __popc(eq[1]);
         int incl = mine;
 #pragma unroll
@@ -1017,9 +1107,10 @@ __global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs
                 keep_words((keep[c >> 2] >> (8 * (c & 3))) & 0xFFu, km);
                 sts_16(src + c * 16, make_uint4(wv[4 * c] & km[0], wv[4 * c + 1] & km[1], wv[4 * c + 2] & km[2], wv[4 * c + 3] & km[3]));
             }
-            drain(rrow + (uint32_t)(seg * kStageBytes), a.r_bf16 + m * a.K, seg);
+            drain(rrow + (uint32_t)(ls * kStageBytes), a.r_bf16 + m * a.K, seg);
         }
     }
+    }  // rows of this CTA
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1335,6 +1426,12 @@ __global__ void __launch_bounds__(kThreads) dequant_kernel(const uint8_t* __rest
     o[1] = make_float4(v[4], v[5], v[6], v[7]);
 }
 
+// debugging override: RESQ_ROW50_TEAM=0 sends long rows to the older CTA-per-row kernel
+bool env_flag_row50_team() {
+    const char* v = getenv("RESQ_ROW50_TEAM");
+    return !(v && *v == '0');
+}
+
 int pick_rows_per_cta(int64_t M, int64_t K, int pattern) {
     // enough CTAs to fill 148 SMs several times over, but long enough row loops to amortize set-up
     int64_t col_ctas = (K + (int64_t)kWarpsPerCta * kColsPerWarp - 1) / ((int64_t)kWarpsPerCta * kColsPerWarp);
@@ -1457,19 +1554,31 @@ int launch_quantize(int fmt, const QuantArgs& a_in, cudaStream_t stream) {
         const int nseg = (int)((a.K / kHif4Block + 31) / 32);
         const int per_warp = (3 + nseg) * kStageBytes;
         const int wpc = std::min(kWarpsPerCta, (220 * 1024) / per_warp);
-        // (measured: wins for rows of up to two segments; longer rows keep a whole CTA busy better)
-        if (a.K % kHif4Block == 0 && nseg <= 2 && wpc >= 1 && a.M >= 148 && al16r(a.x_codes) && al16r(a.r_codes) && al16r(a.mask_bits) &&
-            al16r(a.a_bf16) && al16r(a.r_bf16)) {
-            const bool img = a.a_bf16 != nullptr;
+        const bool aligned = al16r(a.x_codes) && al16r(a.r_codes) && al16r(a.mask_bits) && al16r(a.a_bf16) && al16r(a.r_bf16);
+        const bool img = a.a_bf16 != nullptr;
+        if (a.K % kHif4Block == 0 && nseg <= 2 && wpc >= 1 && a.M >= 148 && aligned) {
             void (*kern)(QuantArgs, int) =
-                fmt == kHiF4 ? (img ? quant_row50_warp_kernel<kHiF4, true> : quant_row50_warp_kernel<kHiF4, false>)
-                             : (img ? quant_row50_warp_kernel<kMXFP4, true> : quant_row50_warp_kernel<kMXFP4, false>);
+                fmt == kHiF4 ? (img ? quant_row50_warp_kernel<kHiF4, true, 1> : quant_row50_warp_kernel<kHiF4, false, 1>)
+                             : (img ? quant_row50_warp_kernel<kMXFP4, true, 1> : quant_row50_warp_kernel<kMXFP4, false, 1>);
             const int smem_w = wpc * per_warp;
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_w);
             if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(row50 warp)");
             LaunchScope scope(kKindQuant, stream);
             return cuda_fail(launch_kernel(kern, dim3((unsigned)((a.M + wpc - 1) / wpc)), dim3(kThreads), (size_t)smem_w, stream, a, wpc),
                              "quant_row50_warp_kernel launch");
+        }
+        // longer rows (up to 16 segments): the eight warps of a CTA share a row
+        if (a.K % kHif4Block == 0 && nseg <= 2 * kWarpsPerCta && aligned && env_flag_row50_team()) {
+            void (*kern)(QuantArgs, int) =
+                fmt == kHiF4 ? (img ? quant_row50_warp_kernel<kHiF4, true, kWarpsPerCta> : quant_row50_warp_kernel<kHiF4, false, kWarpsPerCta>)
+                             : (img ? quant_row50_warp_kernel<kMXFP4, true, kWarpsPerCta> : quant_row50_warp_kernel<kMXFP4, false, kWarpsPerCta>);
+            const int smem_t = kWarpsPerCta * (3 + (nseg + kWarpsPerCta - 1) / kWarpsPerCta) * kStageBytes;
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_t);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(row50 team)");
+            LaunchScope scope(kKindQuant, stream);
+            const unsigned ctas = (unsigned)std::min<int64_t>(a.M, 148);  // one resident CTA per SM, rows strided
+            return cuda_fail(launch_kernel(kern, dim3(ctas), dim3(kThreads), (size_t)smem_t, stream, a, kWarpsPerCta),
+                             "quant_row50_warp_kernel (team) launch");
         }
         size_t smem = (size_t)a.K * sizeof(uint16_t);
         if (smem > 200 * 1024) {
