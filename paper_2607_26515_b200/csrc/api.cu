@@ -179,6 +179,10 @@ void carve_quant_scratch(uint8_t* ws, int64_t M, int64_t K, int pattern, QuantAr
         used += align_up(n * sizeof(double), 256);
         a.keep_flags = ws + used;
         used += align_up(n, 256);
+        if ((int64_t)n > kSelGridMin) {
+            a.sel_hist = reinterpret_cast<uint32_t*>(ws + used);
+            used += kSelGridScratch;
+        }
     }
 }
 

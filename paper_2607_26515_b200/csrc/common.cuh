@@ -104,6 +104,9 @@ struct QuantArgs {
     // scratch
     double* scores;         // CHAN50: [K]; BLOCK: [(M/32) * (K/64)]
     uint8_t* keep_flags;    // CHAN50: [K]; BLOCK: [(M/32) * (K/64)]
+    // more than kSelGridMin scores: the selection runs as a few grid-wide kernels over 16-bit digits and needs a
+    // histogram of 65536 counters plus a small state block (kSelGridScratch bytes); null: single-CTA selection
+    uint32_t* sel_hist;
     DeviceStatus* status;
     // words at the start of the workspace (status, counters of the GEMM) that the first kernel of the call clears
     uint32_t* clear_words;
@@ -116,7 +119,9 @@ int launch_quantize_mxfp8_image(const __nv_bfloat16* X, int64_t M, int64_t K, in
                                 int n_clear_words, cudaStream_t stream);
 int launch_dequantize(int fmt, const uint8_t* codes, const void* side, int64_t rows, int64_t K, float* out,
                       cudaStream_t stream);
-size_t quant_scratch_bytes(int64_t M, int64_t K, int pattern);  // scores + keep flags (without header)
+size_t quant_scratch_bytes(int64_t M, int64_t K, int pattern);  // scores + keep flags [+ histogram] (without header)
+constexpr int64_t kSelGridMin = 24576;                         // selections with more scores than this use the grid-wide kernels
+constexpr size_t kSelGridScratch = 65536 * 4 + 256;            // histogram + state
 
 // ---- GEMM launch description (gemm_hif4.cu / gemm_mxfp4.cu) -------------------------------------
 struct GemmArgs {

@@ -1450,7 +1450,7 @@ size_t quant_scratch_bytes(int64_t M, int64_t K, int pattern) {
     if (pattern == RESQ_S_CHAN50) n = (size_t)K;
     if (pattern == RESQ_S_BLOCK32x64_50) n = (size_t)(M / kBlkRows) * (size_t)(K / kBlkCols);
     if (n == 0) return 0;
-    return align_up(n * sizeof(double), 256) + align_up(n, 256);
+    return align_up(n * sizeof(double), 256) + align_up(n, 256) + ((int64_t)n > kSelGridMin ? kSelGridScratch : 0);
 }
 
 // 8-bit activations of the "W4A8" ablation: MXFP8 with E4M3 elements (blocks of 32 along K, E8M0 scale
@@ -1507,14 +1507,176 @@ int launch_quantize_mxfp8_image(const __nv_bfloat16* X, int64_t M, int64_t K, in
                      "quant_mxfp8_image_kernel launch");
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same exact selection for many scores (tens of thousands of blocks at prefill sizes), where one CTA re-reading
+// all keys eight times is the bottleneck: four passes over 16-bit digits, each a grid-wide histogram kernel
+// (global counters) and a one-CTA kernel that finds the bucket of the keep-th largest key and clears the counters
+// for the next pass; then a grid-wide flag kernel.  Ties at the threshold are kept lowest index first: when not all
+// of them are kept (rare) a one-CTA pass orders them.  State block after the histogram: [0..1] prefix (u64),
+// [2] remaining, [3] entries equal to the threshold.
+struct SelState {
+    unsigned long long prefix;
+    int remaining;
+    int equal;
+};
+
+__global__ void __launch_bounds__(256) sel_grid_init_kernel(uint32_t* hist, SelState* st, int keep) {
+    pdl_wait();
+    pdl_trigger();
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 65536; i += gridDim.x * blockDim.x) hist[i] = 0u;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        st->prefix = 0ull;
+        st->remaining = keep;
+        st->equal = 0;
+    }
+}
+
+__global__ void __launch_bounds__(256) sel_grid_hist_kernel(const double* __restrict__ score, int n, int shift, uint32_t* hist,
+                                                            const SelState* st) {
+    pdl_wait();
+    pdl_trigger();
+    const unsigned long long prefix = st->prefix;
+    for (int i0 = blockIdx.x * blockDim.x; i0 < n; i0 += gridDim.x * blockDim.x) {
+        const int i = i0 + threadIdx.x;
+        const unsigned long long key = i < n ? (unsigned long long)__double_as_longlong(score[i]) : 0ull;
+        const bool match = i < n && (shift == 48 ? true : ((key ^ prefix) >> (shift + 16)) == 0ull);
+        const unsigned bucket = match ? (unsigned)(key >> shift) & 0xFFFFu : 0xFFFFFFFFu;
+        const unsigned same = __match_any_sync(0xFFFFFFFFu, bucket);  // neighbouring scores often share the digit
+        if (match && (unsigned)(__ffs((int)same) - 1) == (threadIdx.x & 31u)) atomicAdd(&hist[bucket], (unsigned)__popc(same));
+    }
+}
+
+// One CTA of 1024 threads: thread t owns buckets 64 t .. 64 t + 63.
+__global__ void __launch_bounds__(1024) sel_grid_scan_kernel(uint32_t* hist, SelState* st, int shift) {
+    __shared__ int s_part[1024];
+    pdl_wait();
+    pdl_trigger();
+    const int tid = threadIdx.x;
+    uint32_t h[64];
+    int mine = 0;
+#pragma unroll
+    for (int j = 0; j < 64; j += 4) {
+        const uint4 v = *reinterpret_cast<const uint4*>(hist + 64 * tid + j);
+        h[j] = v.x; h[j + 1] = v.y; h[j + 2] = v.z; h[j + 3] = v.w;
+        mine += (int)(v.x + v.y + v.z + v.w);
+    }
+#pragma unroll
+    for (int j = 0; j < 64; j += 4) *reinterpret_cast<uint4*>(hist + 64 * tid + j) = make_uint4(0, 0, 0, 0);  // for the next pass
+    s_part[tid] = mine;
+    __syncthreads();
+    // inclusive suffix sums over threads (keys in higher buckets are larger)
+    for (int o = 1; o < 1024; o <<= 1) {
+        const int t = tid + o < 1024 ? s_part[tid + o] : 0;
+        __syncthreads();
+        s_part[tid] += t;
+        __syncthreads();
+    }
+    const int remaining = st->remaining;
+    const int incl = s_part[tid], above = incl - mine;
+    __syncthreads();
+    if (above < remaining && incl >= remaining) {  // exactly one thread
+        int rem = remaining - above;
+        int b = 63;
+        for (; b > 0; --b) {
+            const int c = (int)h[b];
+            if (c >= rem) break;
+            rem -= c;
+        }
+        st->prefix |= (unsigned long long)(64 * tid + b) << shift;
+        st->remaining = rem;
+        st->equal = (int)h[b];
+    }
+}
+
+__global__ void __launch_bounds__(256) sel_grid_flag_kernel(const double* __restrict__ score, int n, const SelState* st,
+                                                            uint8_t* __restrict__ flag) {
+    pdl_wait();
+    pdl_trigger();
+    const unsigned long long T = st->prefix;
+    const bool all_ties = st->remaining == st->equal;  // every entry equal to the threshold is kept
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const unsigned long long key = (unsigned long long)__double_as_longlong(score[i]);
+        flag[i] = (key > T || (key == T && all_ties)) ? 1 : 0;
+    }
+}
+
+// Only when some but not all ties are kept: one CTA walks the scores in index order and admits the first `remaining`.
+__global__ void __launch_bounds__(kSelThreads) sel_grid_ties_kernel(const double* __restrict__ score, int n, const SelState* st,
+                                                                    uint8_t* __restrict__ flag) {
+    __shared__ int s_warp_count[kSelThreads / 32];
+    __shared__ int s_base;
+    pdl_wait();
+    pdl_trigger();
+    if (st->remaining == st->equal) return;
+    const unsigned long long T = st->prefix;
+    const int need = st->remaining;
+    const int tid = threadIdx.x;
+    if (tid == 0) s_base = 0;
+    __syncthreads();
+    for (int i0 = 0; i0 < n; i0 += kSelThreads) {
+        const int i = i0 + tid;
+        const bool eq = i < n && (unsigned long long)__double_as_longlong(score[i]) == T;
+        const unsigned bal = __ballot_sync(0xFFFFFFFFu, eq);
+        const int lane = tid & 31, w = tid >> 5;
+        if (lane == 0) s_warp_count[w] = __popc(bal);
+        __syncthreads();
+        int before = s_base;
+        for (int j = 0; j < w; ++j) before += s_warp_count[j];
+        before += __popc(bal & ((1u << lane) - 1u));
+        if (eq && before < need) flag[i] = 1;
+        __syncthreads();
+        if (tid == 0) {
+            int tot = 0;
+            for (int j = 0; j < kSelThreads / 32; ++j) tot += s_warp_count[j];
+            s_base += tot;
+        }
+        __syncthreads();
+    }
+}
+
 // Second and third kernel of the patterns with a tensor-wide selection (CHAN50, BLOCK): top half of the scores,
 // then the mask pass over the residual outputs.
 static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t stream) {
-    int rc;
-    {
+    int rc = RESQ_OK;
+    const int keep = (int)(nscore * a.keep_quarters / 4);
+    const char* grid_env = getenv("RESQ_SEL_GRID");  // debugging override: 0 keeps the one-CTA selection
+    if (a.sel_hist && nscore > kSelGridMin && keep > 0 && keep < nscore && !(grid_env && *grid_env == '0')) {
+        SelState* st = reinterpret_cast<SelState*>(a.sel_hist + 65536);
+        const unsigned grid = (unsigned)std::min<int64_t>((nscore + 255) / 256, 148 * 4);
+        {
+            LaunchScope scope(kKindSelect, stream);
+            rc = cuda_fail(launch_kernel(sel_grid_init_kernel, dim3(64), dim3(256), 0, stream, a.sel_hist, st, keep),
+                           "sel_grid_init_kernel launch");
+        }
+        for (int shift = 48; shift >= 0 && !rc; shift -= 16) {
+            {
+                LaunchScope scope(kKindSelect, stream);
+                rc = cuda_fail(launch_kernel(sel_grid_hist_kernel, dim3(grid), dim3(256), 0, stream, (const double*)a.scores, (int)nscore,
+                                             shift, a.sel_hist, (const SelState*)st),
+                               "sel_grid_hist_kernel launch");
+            }
+            if (!rc) {
+                LaunchScope scope(kKindSelect, stream);
+                rc = cuda_fail(launch_kernel(sel_grid_scan_kernel, dim3(1), dim3(1024), 0, stream, a.sel_hist, st, shift),
+                               "sel_grid_scan_kernel launch");
+            }
+        }
+        if (!rc) {
+            LaunchScope scope(kKindSelect, stream);
+            rc = cuda_fail(launch_kernel(sel_grid_flag_kernel, dim3(grid), dim3(256), 0, stream, (const double*)a.scores, (int)nscore,
+                                         (const SelState*)st, a.keep_flags),
+                           "sel_grid_flag_kernel launch");
+        }
+        if (!rc) {
+            LaunchScope scope(kKindSelect, stream);
+            rc = cuda_fail(launch_kernel(sel_grid_ties_kernel, dim3(1), dim3(kSelThreads), 0, stream, (const double*)a.scores, (int)nscore,
+                                         (const SelState*)st, a.keep_flags),
+                           "sel_grid_ties_kernel launch");
+        }
+    } else {
         LaunchScope scope(kKindSelect, stream);
         rc = cuda_fail(launch_kernel(topk_select_kernel, dim3(1), dim3(kSelThreads), 0, stream, (const double*)a.scores, (int)nscore,
-                                     (int)(nscore * a.keep_quarters / 4), a.keep_flags),
+                                     keep, a.keep_flags),
                        "topk_select_kernel launch");
     }
     if (rc) return rc;

@@ -112,6 +112,22 @@ def test_sparsity_sweep_masks_bit_exact(shape, base, q, fmt):
     assert np.array_equal(got["mask"].cpu().numpy(), want["mask"])
 
 
+@pytest.mark.parametrize("q", [1, 2, 3])
+@pytest.mark.parametrize("case", [(oracle.S_BLOCK, 4096, 12352), (oracle.S_CHAN50, 32, 24704)])
+def test_selection_over_many_scores(case, q):
+    """More than 24576 block / channel scores: the selection runs as grid-wide kernels over 16-bit digits."""
+    base, M, K = case
+    pattern = oracle.keep_quarters(base, q)
+    bits = synth(5 * M + K + q, M, K, n_out=max(1, K // 256), extremes=False)
+    want = oracle.quantize_residual_mask(bf16_bits_to_f32(bits), pattern, "hif4")
+    got = rq().residual_mask(to_dev(bits), pattern, "hif4")
+    torch.cuda.synchronize()
+    info = want["mask_info"]
+    if not (info["exact"] or info["margin"] > 2.0 ** -40):
+        pytest.skip("selection scores not exactly summable and boundary margin too small")
+    assert np.array_equal(got["mask"].cpu().numpy(), want["mask"])
+
+
 @pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4, oracle.S_BLOCK])
 def test_many_rows_per_warp(pattern):
     """Tall, narrow input: every warp of the streaming kernel walks several rows (prefetch ring, row tail)."""
@@ -132,10 +148,10 @@ def test_many_rows_per_warp(pattern):
     assert np.array_equal(got["mask"].cpu().numpy(), want["mask"])
 
 
-@pytest.mark.parametrize("shape", [(64, 256), (64, 2304), (32, 8448)])
+@pytest.mark.parametrize("shape", [(64, 256), (64, 2304), (32, 24640)])
 def test_residual_mask_ties_and_zero_rows(shape):
-    # all-equal magnitudes: every selection is decided by the lower-index rule (the channel scores of the wider
-    # shapes span several register rows of the small selection kernel, the widest takes the general one)
+    # all-equal magnitudes: every selection is decided by the lower-index rule (the widest shape has more channel
+    # scores than one CTA selects: grid-wide kernels, including their ordered pass over the ties)
     M, K = shape
     x = np.full((M, K), 0.75, dtype=np.float32)
     x[:, ::2] *= -1
