@@ -814,11 +814,13 @@ __global__ void __launch_bounds__(kThreads, 2) quant_block_kernel(QuantArgs a, i
 // staging buffers), so that the K/2 largest magnitudes can be selected and the image masked before it leaves.
 // Selection: most significant bit first over the 15 magnitude bits, counting with warp reductions only; ties
 // at the threshold are kept lowest index first.  Shared memory per warp: (3 + segments) staging tiles.
-// WPR = 1: a warp per row (rows of up to two segments).  WPR = 8: the eight warps of a CTA share one row (up to 16
-// segments, warp w takes segments w and w + 8); the per-bit counts and the tie counts of the segments are summed
-// through shared memory with one CTA barrier each.
-template <int FMT, bool IMG, int WPR>
-__global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs a, int warps_per_cta) {
+// WPR = 1: a warp per row (rows of up to two segments, MAXSEG = 2).  WPR = 8 or 16: the warps of a CTA share one row,
+// one segment per warp (MAXSEG = 1: fewer registers and two shared-memory tiles per warp, so that two 8-warp CTAs
+// fit on an SM); the per-bit counts and the tie counts of the segments are summed through shared memory with one
+// CTA barrier each.
+template <int FMT, bool IMG, int WPR, int MAXSEG>
+__global__ void __launch_bounds__(WPR == 16 ? 512 : kThreads, (WPR != 16 && MAXSEG == 1) ? 2 : 1)
+quant_row50_warp_kernel(QuantArgs a, int warps_per_cta) {
     pdl_wait();
     pdl_trigger();
     if (a.clear_words && blockIdx.x == 0)
@@ -842,8 +844,11 @@ __global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs
     const int nseg = WPR == 1 ? nseg_row : max(0, (nseg_row - wr + WPR - 1) / WPR);  // segments of this warp (at most 2)
     const int seg_cap = WPR == 1 ? nseg_row : (nseg_row + WPR - 1) / WPR;           // row-image tiles per warp
     auto gseg = [&](int ls) -> int { return wr + ls * WPR; };                      // local -> row segment
-    const uint32_t base = smem_u32(smem_q) + (uint32_t)(warp * (3 + seg_cap) * kStageBytes);
-    const uint32_t in0 = base, stage = base + 2 * kStageBytes, rrow = base + 3 * kStageBytes;
+    // tiles per warp: two input stages, the image stage and the row image; with one segment per warp the input
+    // tile doubles as the image stage (it is in registers before the encode writes the image)
+    const uint32_t base = smem_u32(smem_q) + (uint32_t)(warp * (MAXSEG == 1 ? 2 : 3 + seg_cap) * kStageBytes);
+    const uint32_t in0 = base, stage = MAXSEG == 1 ? base : base + 2 * kStageBytes,
+                   rrow = MAXSEG == 1 ? base + kStageBytes : base + 3 * kStageBytes;
     const int cp_blk = lane >> 3, cp_ch = lane & 7;
     const uint32_t cp_smem = (uint32_t)(cp_blk * kStagePitch + cp_ch * 16);
     const uint32_t my_in = (uint32_t)(lane * kStagePitch);
@@ -956,7 +961,7 @@ __global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs
     // holds bit b of the even elements (element 2r at bit r), word 16 + b that of the odd elements.  The most-
     // significant-bit-first select then costs two population counts and a warp sum per bit; the sets "equal to the
     // threshold" and "greater" fall out as masks.
-    constexpr int kMaxSeg = 2;                    // the launcher sends longer rows to the CTA-per-row kernel
+    constexpr int kMaxSeg = MAXSEG;               // segments per warp (the launcher picks the variant)
     uint32_t plane[kMaxSeg][32];
     uint32_t c_even[kMaxSeg], c_odd[kMaxSeg], g_even[kMaxSeg], g_odd[kMaxSeg];
 #pragma unroll
@@ -1057,8 +1062,8 @@ __global__ void __launch_bounds__(kThreads, 1) quant_row50_warp_kernel(QuantArgs
             wv[4 * c] = v.x; wv[4 * c + 1] = v.y; wv[4 * c + 2] = v.z; wv[4 * c + 3] = v.w;
         }
         // bit per element of the lane's block (low / high 32): greater than / equal to the threshold
-        const uint32_t ce = ls == 0 ? c_even[0] : c_even[1], co = ls == 0 ? c_odd[0] : c_odd[1];
-        const uint32_t ge = ls == 0 ? g_even[0] : g_even[1], go = ls == 0 ? g_odd[0] : g_odd[1];
+        const uint32_t ce = ls == 0 ? c_even[0] : c_even[kMaxSeg - 1], co = ls == 0 ? c_odd[0] : c_odd[kMaxSeg - 1];
+        const uint32_t ge = ls == 0 ? g_even[0] : g_even[kMaxSeg - 1], go = ls == 0 ? g_odd[0] : g_odd[kMaxSeg - 1];
         uint32_t gt[2] = {spread16(ge) | (spread16(go) << 1), spread16(ge >> 16) | (spread16(go >> 16) << 1)};
         uint32_t eq[2] = {spread16(ce) | (spread16(co) << 1), spread16(ce >> 16) | (spread16(co >> 16) << 1)};
         const int mine = __popc(eq[0]) + __popc(eq[1]);
@@ -1719,27 +1724,37 @@ int launch_quantize(int fmt, const QuantArgs& a_in, cudaStream_t stream) {
         const bool aligned = al16r(a.x_codes) && al16r(a.r_codes) && al16r(a.mask_bits) && al16r(a.a_bf16) && al16r(a.r_bf16);
         const bool img = a.a_bf16 != nullptr;
         if (a.K % kHif4Block == 0 && nseg <= 2 && wpc >= 1 && a.M >= 148 && aligned) {
-            void (*kern)(QuantArgs, int) =
-                fmt == kHiF4 ? (img ? quant_row50_warp_kernel<kHiF4, true, 1> : quant_row50_warp_kernel<kHiF4, false, 1>)
-                             : (img ? quant_row50_warp_kernel<kMXFP4, true, 1> : quant_row50_warp_kernel<kMXFP4, false, 1>);
-            const int smem_w = wpc * per_warp;
+            void (*kern)(QuantArgs, int);
+            if (nseg == 1)  // one segment: the lean variant (128 registers, two tiles per warp: two CTAs per SM)
+                kern = fmt == kHiF4 ? (img ? quant_row50_warp_kernel<kHiF4, true, 1, 1> : quant_row50_warp_kernel<kHiF4, false, 1, 1>)
+                                    : (img ? quant_row50_warp_kernel<kMXFP4, true, 1, 1> : quant_row50_warp_kernel<kMXFP4, false, 1, 1>);
+            else
+                kern = fmt == kHiF4 ? (img ? quant_row50_warp_kernel<kHiF4, true, 1, 2> : quant_row50_warp_kernel<kHiF4, false, 1, 2>)
+                                    : (img ? quant_row50_warp_kernel<kMXFP4, true, 1, 2> : quant_row50_warp_kernel<kMXFP4, false, 1, 2>);
+            const int smem_w = nseg == 1 ? wpc * 2 * kStageBytes : wpc * per_warp;
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_w);
             if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(row50 warp)");
             LaunchScope scope(kKindQuant, stream);
             return cuda_fail(launch_kernel(kern, dim3((unsigned)((a.M + wpc - 1) / wpc)), dim3(kThreads), (size_t)smem_w, stream, a, wpc),
                              "quant_row50_warp_kernel launch");
         }
-        // longer rows (up to 16 segments): the eight warps of a CTA share a row
-        if (a.K % kHif4Block == 0 && nseg <= 2 * kWarpsPerCta && aligned && env_flag_row50_team()) {
-            void (*kern)(QuantArgs, int) =
-                fmt == kHiF4 ? (img ? quant_row50_warp_kernel<kHiF4, true, kWarpsPerCta> : quant_row50_warp_kernel<kHiF4, false, kWarpsPerCta>)
-                             : (img ? quant_row50_warp_kernel<kMXFP4, true, kWarpsPerCta> : quant_row50_warp_kernel<kMXFP4, false, kWarpsPerCta>);
-            const int smem_t = kWarpsPerCta * (3 + (nseg + kWarpsPerCta - 1) / kWarpsPerCta) * kStageBytes;
+        // longer rows (up to 16 segments): the warps of a persistent CTA share a row, one segment each
+        if (a.K % kHif4Block == 0 && nseg <= 16 && aligned && env_flag_row50_team()) {
+            const bool wide = nseg > kWarpsPerCta;  // 16 warps per CTA instead of 8
+            void (*kern)(QuantArgs, int);
+            if (wide)
+                kern = fmt == kHiF4 ? (img ? quant_row50_warp_kernel<kHiF4, true, 16, 1> : quant_row50_warp_kernel<kHiF4, false, 16, 1>)
+                                    : (img ? quant_row50_warp_kernel<kMXFP4, true, 16, 1> : quant_row50_warp_kernel<kMXFP4, false, 16, 1>);
+            else
+                kern = fmt == kHiF4 ? (img ? quant_row50_warp_kernel<kHiF4, true, 8, 1> : quant_row50_warp_kernel<kHiF4, false, 8, 1>)
+                                    : (img ? quant_row50_warp_kernel<kMXFP4, true, 8, 1> : quant_row50_warp_kernel<kMXFP4, false, 8, 1>);
+            const int warps = wide ? 16 : 8;
+            const int smem_t = warps * 2 * kStageBytes;
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_t);
             if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(row50 team)");
             LaunchScope scope(kKindQuant, stream);
-            const unsigned ctas = (unsigned)std::min<int64_t>(a.M, 148);  // one resident CTA per SM, rows strided
-            return cuda_fail(launch_kernel(kern, dim3(ctas), dim3(kThreads), (size_t)smem_t, stream, a, kWarpsPerCta),
+            const unsigned ctas = (unsigned)std::min<int64_t>(a.M, wide ? 148 : 296);  // resident CTAs, rows strided
+            return cuda_fail(launch_kernel(kern, dim3(ctas), dim3(32 * warps), (size_t)smem_t, stream, a, warps),
                              "quant_row50_warp_kernel (team) launch");
         }
         size_t smem = (size_t)a.K * sizeof(uint16_t);
