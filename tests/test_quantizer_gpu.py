@@ -112,6 +112,22 @@ def test_sparsity_sweep_masks_bit_exact(shape, base, q, fmt):
     assert np.array_equal(got["mask"].cpu().numpy(), want["mask"])
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("shape", [(700, 4160), (416, 18944), (1300, 2048), (900, 3584)])
+def test_row_selection_persistent_ctas(shape, fmt):
+    """Row-wise selection with more rows than resident CTAs (each CTA or warp walks several rows, the next row
+    loading while the current one is selected), for every variant: one warp per row (one and two segments),
+    8-warp and 16-warp teams per row."""
+    M, K = shape
+    bits = synth(9 * M + K, M, K, n_out=max(1, K // 256), extremes=True)
+    want = oracle.quantize_residual_mask(bf16_bits_to_f32(bits), oracle.S_ROW50, fmt)
+    got = rq().residual_mask(to_dev(bits), oracle.S_ROW50, fmt)
+    torch.cuda.synchronize()
+    for key in ("x_codes", "x_side", "r_codes", "r_side"):
+        assert np.array_equal(side_np(got[key]), want[key]), key
+    assert np.array_equal(got["mask"].cpu().numpy(), want["mask"])
+
+
 @pytest.mark.parametrize("q", [1, 2, 3])
 @pytest.mark.parametrize("case", [(oracle.S_BLOCK, 4096, 12352), (oracle.S_CHAN50, 32, 24704)])
 def test_selection_over_many_scores(case, q):
