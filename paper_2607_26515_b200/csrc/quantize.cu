@@ -1431,6 +1431,11 @@ __global__ void __launch_bounds__(kThreads) dequant_kernel(const uint8_t* __rest
     o[1] = make_float4(v[4], v[5], v[6], v[7]);
 }
 
+bool getenv_is_zero(const char* name) {
+    const char* v = getenv(name);
+    return v && *v == '0';
+}
+
 // debugging override: RESQ_ROW50_TEAM=0 sends long rows to the older CTA-per-row kernel
 bool env_flag_row50_team() {
     const char* v = getenv("RESQ_ROW50_TEAM");
@@ -1639,6 +1644,33 @@ __global__ void __launch_bounds__(kSelThreads) sel_grid_ties_kernel(const double
     }
 }
 
+// Channel scores of CHAN50 from the (unmasked) bf16 residual image the block-per-lane quantizer has just written
+// (still in L2 for all but the largest inputs): a thread owns 8 channels and a strip of rows; the squares of the
+// decoded values are exact, the strip sums run in fp64, one atomic per channel and strip.
+constexpr int kChanStripRows = 64;
+__global__ void __launch_bounds__(256) chan_score_kernel(const __nv_bfloat16* __restrict__ img, int64_t M, int64_t K,
+                                                         double* __restrict__ scores) {
+    pdl_wait();
+    pdl_trigger();
+    const int64_t per_row = K / 8;
+    const int64_t strips = (M + kChanStripRows - 1) / kChanStripRows;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= per_row * strips) return;
+    const int64_t k0 = (idx % per_row) * 8, m0 = (idx / per_row) * kChanStripRows;
+    const int64_t m1 = min(M, m0 + kChanStripRows);
+    double acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.0;
+    for (int64_t m = m0; m < m1; ++m) {
+        float v[8];
+        unpack_bf16x8(__ldcg(reinterpret_cast<const uint4*>(img + m * K + k0)), v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] += (double)v[i] * (double)v[i];
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) atomicAdd(&scores[k0 + i], acc[i]);
+}
+
 // Second and third kernel of the patterns with a tensor-wide selection (CHAN50, BLOCK): top half of the scores,
 // then the mask pass over the residual outputs.
 static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t stream) {
@@ -1781,7 +1813,9 @@ int launch_quantize(int fmt, const QuantArgs& a_in, cudaStream_t stream) {
     // Worth it once there is a warp task (32 blocks of one row) for every warp slot of the machine; below
     // that the finer-grained kernel (a lane per 8 values) finishes sooner.
     const int64_t block_tasks = a.M * ((a.K / kHif4Block + 31) / 32);
-    if (!a.X_up && !a.gamma && !a.rht && pattern != RESQ_S_CHAN50 && a.K % kHif4Block == 0 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
+    // (CHAN50 only when the residual image is written: its channel scores are then summed from the image)
+    const bool chan_from_image = pattern == RESQ_S_CHAN50 && a.r_bf16 != nullptr && !getenv_is_zero("RESQ_CHAN_FROM_IMAGE");
+    if (!a.X_up && !a.gamma && !a.rht && (pattern != RESQ_S_CHAN50 || chan_from_image) && a.K % kHif4Block == 0 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
         al16(a.a_bf16) && al16(a.r_bf16) && al16(a.r_comp)) {
         const bool img = a.a_bf16 != nullptr;
         const int64_t ncg = (a.K / kHif4Block + 31) / 32;
@@ -1807,6 +1841,14 @@ int launch_quantize(int fmt, const QuantArgs& a_in, cudaStream_t stream) {
                                       : img ? launch(quant_block_kernel<kMXFP4, true, true>) : launch(quant_block_kernel<kMXFP4, true, false>))
                           : (img ? launch(quant_block_kernel<kMXFP4, false, true>) : launch(quant_block_kernel<kMXFP4, false, false>));
         if (rc) return rc;
+        if (chan_from_image) {
+            const int64_t nthreads = (a.K / 8) * ((a.M + kChanStripRows - 1) / kChanStripRows);
+            LaunchScope scope(kKindSelect, stream);
+            rc = cuda_fail(launch_kernel(chan_score_kernel, dim3((unsigned)((nthreads + 255) / 256)), dim3(256), 0, stream,
+                                         (const __nv_bfloat16*)a.r_bf16, a.M, a.K, a.scores),
+                           "chan_score_kernel launch");
+            if (rc) return rc;
+        }
         if (global_sel) rc = launch_global_select(a, nscore, stream);
         return rc;
     }

@@ -299,6 +299,28 @@ def test_w4a8_linear_parity(shape, fmt):
     check_close(yb.float().cpu().numpy(), want["y"], want["abs_sum"], bf16_out=True)
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("q", [2, 1])
+def test_channel_selection_through_the_block_quantizer(fmt, q, monkeypatch):
+    """CHAN50 on an input large enough for the block-per-lane quantizer: the channel scores are then summed from the
+    residual image by a kernel of their own; same result as the chunk-per-lane path, which keeps them in registers."""
+    m = rq()
+    M, K, N = 2432, 1152, 264
+    pattern = oracle.keep_quarters(oracle.S_CHAN50, q)
+    xb, wb = synth_xw(4242 + q, M, K, N, n_out=4)
+    want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern, fmt)
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    monkeypatch.setenv("RESQ_MXFP4_NATIVE", "0")
+    y = m.resq_linear(to_dev(xb), wc, ws, pattern, fmt, out_dtype=torch.float32)
+    monkeypatch.setenv("RESQ_CHAN_FROM_IMAGE", "0")
+    y_old = m.resq_linear(to_dev(xb), wc, ws, pattern, fmt, out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    info = want["mask_info"]
+    if info["exact"] or info["margin"] > 2.0 ** -40:
+        check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+        assert torch.equal(y, y_old)
+
+
 def test_swiglu_rejects_row50_and_narrow_input():
     m = rq()
     gu = torch.zeros((64, 512), dtype=torch.bfloat16, device="cuda")
