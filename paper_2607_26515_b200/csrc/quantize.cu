@@ -1124,16 +1124,14 @@ quant_row50_warp_kernel(QuantArgs a, int warps_per_cta) {
 // first `need` entries equal to the threshold.
 constexpr int kSelThreads = 1024;
 
-__global__ void __launch_bounds__(kSelThreads) topk_select_kernel(const double* __restrict__ score, int n, int keep,
-                                                                 uint8_t* __restrict__ flag) {
+// (All kSelThreads threads of a CTA call it; `flag` may point to global or to shared memory.)
+__device__ __forceinline__ void topk_select_cta(const double* __restrict__ score, int n, int keep, uint8_t* flag) {
     __shared__ unsigned hist[256];
     __shared__ unsigned long long s_prefix;
     __shared__ int s_remaining;
     __shared__ int s_warp_count[kSelThreads / 32];
     __shared__ int s_base;
     const int tid = threadIdx.x;
-    pdl_wait();     // the scores come from the quantizer kernel just before
-    pdl_trigger();  // the mask pass may be scheduled (it waits for this kernel's flags)
     if (keep <= 0 || keep >= n) {
         for (int i = tid; i < n; i += kSelThreads) flag[i] = keep >= n ? 1 : 0;
         return;
@@ -1212,14 +1210,19 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(const double* 
     }
 }
 
+__global__ void __launch_bounds__(kSelThreads) topk_select_kernel(const double* __restrict__ score, int n, int keep,
+                                                                 uint8_t* __restrict__ flag) {
+    pdl_wait();     // the scores come from the quantizer kernel just before
+    pdl_trigger();  // the mask pass may be scheduled (it waits for this kernel's flags)
+    topk_select_cta(score, n, keep, flag);
+}
+
 // Turn the kept-channel / kept-block flags into mask bits and zero the dropped entries of the GEMM's
 // residual operand.  One thread per 8 channels of one row.
-__global__ void apply_global_mask_kernel(int pattern, int64_t M, int64_t K, const uint8_t* __restrict__ flag,
-                                         uint8_t* __restrict__ mask_bits, __nv_bfloat16* __restrict__ r_bf16,
-                                         uint8_t* __restrict__ r_codes_masked) {
-    pdl_wait();     // the keep flags come from the selection kernel just before
-    pdl_trigger();  // the GEMM may be scheduled and run its set-up
-    int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+// One item of the mask pass: 8 consecutive channels of one row (`flag`: global or shared memory).
+__device__ __forceinline__ void apply_mask_item(int64_t idx, int pattern, int64_t M, int64_t K, const uint8_t* flag,
+                                                uint8_t* __restrict__ mask_bits, __nv_bfloat16* __restrict__ r_bf16,
+                                                uint8_t* __restrict__ r_codes_masked) {
     int64_t per_row = K / 8;
     if (idx >= M * per_row) return;
     int64_t m = idx / per_row, k0 = (idx % per_row) * 8;
@@ -1256,6 +1259,14 @@ __global__ void apply_global_mask_kernel(int pattern, int64_t M, int64_t K, cons
         }
         *p = v;
     }
+}
+
+__global__ void apply_global_mask_kernel(int pattern, int64_t M, int64_t K, const uint8_t* __restrict__ flag,
+                                         uint8_t* __restrict__ mask_bits, __nv_bfloat16* __restrict__ r_bf16,
+                                         uint8_t* __restrict__ r_codes_masked) {
+    pdl_wait();     // the keep flags come from the selection kernel just before
+    pdl_trigger();  // the GEMM may be scheduled and run its set-up
+    apply_mask_item((int64_t)blockIdx.x * blockDim.x + threadIdx.x, pattern, M, K, flag, mask_bits, r_bf16, r_codes_masked);
 }
 
 // ------------------------------------------------------------------------------------------------
