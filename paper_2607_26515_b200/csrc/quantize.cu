@@ -1658,17 +1658,16 @@ __global__ void __launch_bounds__(kSelThreads) sel_grid_ties_kernel(const double
 // Channel scores of CHAN50 from the (unmasked) bf16 residual image the block-per-lane quantizer has just written
 // (still in L2 for all but the largest inputs): a thread owns 8 channels and a strip of rows; the squares of the
 // decoded values are exact, the strip sums run in fp64, one atomic per channel and strip.
-constexpr int kChanStripRows = 64;
 __global__ void __launch_bounds__(256) chan_score_kernel(const __nv_bfloat16* __restrict__ img, int64_t M, int64_t K,
-                                                         double* __restrict__ scores) {
+                                                         double* __restrict__ scores, int strip_rows) {
     pdl_wait();
     pdl_trigger();
     const int64_t per_row = K / 8;
-    const int64_t strips = (M + kChanStripRows - 1) / kChanStripRows;
+    const int64_t strips = (M + strip_rows - 1) / strip_rows;
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= per_row * strips) return;
-    const int64_t k0 = (idx % per_row) * 8, m0 = (idx / per_row) * kChanStripRows;
-    const int64_t m1 = min(M, m0 + kChanStripRows);
+    const int64_t k0 = (idx % per_row) * 8, m0 = (idx / per_row) * strip_rows;
+    const int64_t m1 = min(M, m0 + strip_rows);
     double acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.0;
@@ -1826,7 +1825,9 @@ int launch_quantize(int fmt, const QuantArgs& a_in, cudaStream_t stream) {
     const int64_t block_tasks = a.M * ((a.K / kHif4Block + 31) / 32);
     // (CHAN50 only when the residual image is written: its channel scores are then summed from the image)
     const bool chan_from_image = pattern == RESQ_S_CHAN50 && a.r_bf16 != nullptr && !getenv_is_zero("RESQ_CHAN_FROM_IMAGE");
-    if (!a.X_up && !a.gamma && !a.rht && (pattern != RESQ_S_CHAN50 || chan_from_image) && a.K % kHif4Block == 0 && block_tasks >= 148 * 16 && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
+    // (the chunk-per-lane kernel pays for CHAN50 with fp64 atomics per row and channel: the block kernel takes over earlier)
+    const int64_t min_block_tasks = chan_from_image ? 148 : 148 * 16;
+    if (!a.X_up && !a.gamma && !a.rht && (pattern != RESQ_S_CHAN50 || chan_from_image) && a.K % kHif4Block == 0 && block_tasks >= min_block_tasks && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
         al16(a.a_bf16) && al16(a.r_bf16) && al16(a.r_comp)) {
         const bool img = a.a_bf16 != nullptr;
         const int64_t ncg = (a.K / kHif4Block + 31) / 32;
@@ -1853,10 +1854,13 @@ int launch_quantize(int fmt, const QuantArgs& a_in, cudaStream_t stream) {
                           : (img ? launch(quant_block_kernel<kMXFP4, false, true>) : launch(quant_block_kernel<kMXFP4, false, false>));
         if (rc) return rc;
         if (chan_from_image) {
-            const int64_t nthreads = (a.K / 8) * ((a.M + kChanStripRows - 1) / kChanStripRows);
+            // strips of rows per thread: long enough to amortise the atomics, short enough for a few threads per lane slot
+            int strip = 64;
+            while (strip > 4 && (a.K / 8) * ((a.M + strip - 1) / strip) < 148 * 512) strip /= 2;
+            const int64_t nthreads = (a.K / 8) * ((a.M + strip - 1) / strip);
             LaunchScope scope(kKindSelect, stream);
             rc = cuda_fail(launch_kernel(chan_score_kernel, dim3((unsigned)((nthreads + 255) / 256)), dim3(256), 0, stream,
-                                         (const __nv_bfloat16*)a.r_bf16, a.M, a.K, a.scores),
+                                         (const __nv_bfloat16*)a.r_bf16, a.M, a.K, a.scores, strip),
                            "chan_score_kernel launch");
             if (rc) return rc;
         }
