@@ -812,8 +812,13 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
         const int64_t units = (int64_t)p.num_tiles * G;
         const int cap = std::min(max_pairs, kStreamKMaxPairs);
         npairs = (int)std::min<int64_t>(cap, std::max<int64_t>(1, units / 2));
-        if (p.num_tiles <= cap) {
-            // few tiles: the same number of pairs for every tile, so that a pair works on one tile only
+        // Few tiles: the same number of pairs for every tile, so that a pair works on one tile only -- unless that
+        // leaves more than 15 % of the pairs idle on long K ranges (measured: 18944 -> 3584 at M = 512, 28 tiles:
+        // 154 -> 134 us with the units dealt out evenly; short K ranges lose more in the second partial tile).
+        const int per_tile_aligned = std::max(1, std::min(cap / std::max(1, p.num_tiles), G / 2));
+        const bool idle_pairs = p.num_tiles * per_tile_aligned * 100 < cap * 85 && units / cap >= 64;
+        const int force_unaligned = env_int("RESQ_GEMM_SK_UNALIGNED", -1);  // debugging override
+        if (p.num_tiles <= cap && !(force_unaligned >= 0 ? force_unaligned != 0 : idle_pairs)) {
             int per_tile = std::max(1, std::min(cap / p.num_tiles, G / 2));
             const int forced = env_int("RESQ_GEMM_SK_PAIRS", 0);  // debugging override: pairs per tile
             if (forced > 0) per_tile = std::max(1, std::min(forced, per_tile));
