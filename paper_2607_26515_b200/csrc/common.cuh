@@ -145,6 +145,7 @@ struct GemmArgs {
     int splits;                    // slabs that fit in splitk_partials
     size_t partial_bytes;          // size of splitk_partials
     unsigned int* sk_flags;        // kWsFlags bytes of zeroed counters (K-streamed schedule)
+    int tile_limit;                // > 0: whole-tile schedule of the pair kernel stops after this many output tiles
     DeviceStatus* status;
 };
 int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream);

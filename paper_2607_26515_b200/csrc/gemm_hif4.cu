@@ -767,7 +767,37 @@ int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream) {
                 (long long)g.N, (long long)g.K, (int)res, tc.pair_tn, tc.mt, tc.bn, tc.nt, tc.splits);
     if (g.r_comp && tc.pair_tn == 512) tc.pair_tn = 480;  // (a forced width) no tensor-memory columns left for the metadata
     if (!g.r_comp && tc.pair_tn == 480) tc.pair_tn = 512;
-    if (tc.pair_tn > 0) return launch_gemm_pair(g, tc.pair_tn, tc.splits, stream);
+    if (tc.pair_tn > 0) {
+        // Whole tiles in rounds of 74: a last round with a handful of tiles keeps most pairs idle for a whole tile
+        // time.  When those tiles are the end of the last row of tiles, they are a rectangle of the output: it is
+        // cut off and computed by a second call (decode-sized: the K-streamed schedule spreads it over all pairs).
+        const int64_t mtiles = (g.M + 2 * kBM - 1) / (2 * kBM), ntiles = (g.N + tc.pair_tn - 1) / tc.pair_tn;
+        const int64_t tiles = mtiles * ntiles, tail = tiles % 74;
+        if (tc.splits == 1 && !g.r_comp && tiles > 74 && tail > 0 && tail <= ntiles && tail * 3 <= 74 && g.tile_limit == 0 &&
+            env_int("RESQ_GEMM_TAIL_SPLIT", 1)) {
+            GemmArgs main_part = g, tail_part = g;
+            main_part.tile_limit = (int)(tiles - tail);
+            int rc = launch_gemm_pair(main_part, tc.pair_tn, 1, stream);
+            if (rc) return rc;
+            const int64_t m0 = (mtiles - 1) * 2 * kBM, n0 = (ntiles - tail) * tc.pair_tn;
+            const int64_t lda = g.lda ? g.lda : g.K;
+            tail_part.a_bf16 = g.a_bf16 + m0 * lda;
+            if (g.r_bf16) tail_part.r_bf16 = g.r_bf16 + m0 * lda;
+            tail_part.lda = lda;
+            if (g.w_bf16) {
+                tail_part.w_bf16 = g.w_bf16 + n0 * g.ldw;
+            } else {
+                tail_part.w_codes = g.w_codes + n0 * (g.K / 2);
+                tail_part.w_side = static_cast<const uint8_t*>(g.w_side) + n0 * (g.fmt == kHiF4 ? (g.K / kBK) * 4 : g.K / 32);
+            }
+            tail_part.M = g.M - m0;
+            tail_part.N = g.N - n0;
+            tail_part.Y = static_cast<uint8_t*>(g.Y) + (m0 * g.ldy + n0) * (g.out_dtype == RESQ_OUT_F32 ? 4 : 2);
+            tail_part.tile_limit = -1;  // (no further cutting)
+            return launch_gemm_hif4(tail_part, stream);
+        }
+        return launch_gemm_pair(g, tc.pair_tn, tc.splits, stream);
+    }
     if (g.fmt == kMXFP4) {
         if (res) return dispatch_tn<1, true, kMXFP4>(g, tc, stream);
         if (tc.mt == 2) return dispatch_tn<2, false, kMXFP4>(g, tc, stream);

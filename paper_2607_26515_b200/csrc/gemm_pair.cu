@@ -767,6 +767,7 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
     p.ntiles_m = (int)((g.M + 2 * kBM - 1) / (2 * kBM));
     p.ntiles_n = (int)((g.N + TN - 1) / TN);
     p.num_tiles = p.ntiles_m * p.ntiles_n * splits;
+    if (g.tile_limit > 0 && !streamk) p.num_tiles = std::min(p.num_tiles, g.tile_limit * splits);
     p.acc_bufs = TN * 2 <= (RES == kResSparse24 ? kSpTmemCol : kTmemCols) ? 2 : 1;
     if (RES == kResSparse24 && TN > kSpTmemCol) {
         set_last_error("internal: no tensor-memory columns left for the sparse metadata (pair tile %d)", TN);

@@ -321,6 +321,28 @@ def test_channel_selection_through_the_block_quantizer(fmt, q, monkeypatch):
         assert torch.equal(y, y_old)
 
 
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4])
+def test_last_round_of_tiles_as_a_second_call(pattern, fmt, monkeypatch):
+    """80 output tiles of 256 x 512 on 74 CTA pairs: the six tiles of the second round are the end of the last row of
+    tiles and are computed by a second, decode-sized call on sub-matrices of X, W and Y (ragged in M and N)."""
+    m = rq()
+    M, K, N = 2560 - 40, 256, 4096 - 24
+    monkeypatch.setenv("RESQ_GEMM_PAIR_TN", "512")
+    monkeypatch.setenv("RESQ_GEMM_SPLITS", "1")
+    monkeypatch.setenv("RESQ_MXFP4_NATIVE", "0")
+    xb, wb = synth_xw(31 + pattern, M, K, N, n_out=2)
+    want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern, fmt)
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    work = m.alloc_workspace(m.resq_workspace_bytes(M, N, K, pattern, fmt))
+    for cut in ("1", "0"):
+        monkeypatch.setenv("RESQ_GEMM_TAIL_SPLIT", cut)
+        for out_dtype in (torch.float32, torch.bfloat16):
+            y = m.resq_linear(to_dev(xb), wc, ws, pattern, fmt, out_dtype=out_dtype, workspace=work)
+            assert m.check(work) == 0, m.last_error()
+            check_close(y.float().cpu().numpy(), want["y"], want["abs_sum"], bf16_out=out_dtype == torch.bfloat16)
+
+
 def test_swiglu_rejects_row50_and_narrow_input():
     m = rq()
     gu = torch.zeros((64, 512), dtype=torch.bfloat16, device="cuda")
