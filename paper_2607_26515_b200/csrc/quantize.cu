@@ -1655,6 +1655,47 @@ __global__ void __launch_bounds__(kSelThreads) sel_grid_ties_kernel(const double
     }
 }
 
+// The same exact selection for at most 1024 scores (block scores of decode-sized calls): one key per thread, a
+// bitonic sort of (score, index) in descending score / ascending index order -- strides below 32 by shuffles, the
+// others through shared memory -- after which the thread at position p holds the p-th entry of the ranking.
+__global__ void __launch_bounds__(1024) topk_sort1024_kernel(const double* __restrict__ score, int n, int keep,
+                                                             uint8_t* __restrict__ flag) {
+    __shared__ unsigned long long s_key[1024];
+    __shared__ int s_idx[1024];
+    pdl_wait();
+    pdl_trigger();
+    const int tid = threadIdx.x;
+    unsigned long long key = tid < n ? (unsigned long long)__double_as_longlong(score[tid]) : 0ull;  // scores are >= 0
+    int idx = tid;  // padding entries: key 0 and the highest indices, so they rank last
+    for (int k = 2; k <= 1024; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            unsigned long long pk;
+            int pi;
+            if (j < 32) {
+                pk = __shfl_xor_sync(0xFFFFFFFFu, key, j);
+                pi = __shfl_xor_sync(0xFFFFFFFFu, idx, j);
+            } else {
+                s_key[tid] = key;
+                s_idx[tid] = idx;
+                __syncthreads();
+                pk = s_key[tid ^ j];
+                pi = s_idx[tid ^ j];
+                __syncthreads();
+            }
+            // "mine ranks before the partner's": larger score, or equal score and lower index
+            const bool mine_first = key > pk || (key == pk && idx < pi);
+            const bool lower = (tid & j) == 0;          // this thread is the lower position of the pair
+            const bool ranked_order = (tid & k) == 0;   // this sub-sequence is being put in ranking order
+            const bool keep_mine = (lower == ranked_order) ? mine_first : !mine_first;
+            if (!keep_mine) {
+                key = pk;
+                idx = pi;
+            }
+        }
+    }
+    if (idx < n) flag[idx] = tid < keep ? 1 : 0;
+}
+
 // Channel scores of CHAN50 from the (unmasked) bf16 residual image the block-per-lane quantizer has just written
 // (still in L2 for all but the largest inputs): a thread owns 8 channels and a strip of rows; the squares of the
 // decoded values are exact, the strip sums run in fp64, one atomic per channel and strip.
@@ -1720,6 +1761,11 @@ static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t
                                          (const SelState*)st, a.keep_flags),
                            "sel_grid_ties_kernel launch");
         }
+    } else if (nscore <= 1024 && !getenv_is_zero("RESQ_SEL_SORT")) {
+        LaunchScope scope(kKindSelect, stream);
+        rc = cuda_fail(launch_kernel(topk_sort1024_kernel, dim3(1), dim3(1024), 0, stream, (const double*)a.scores, (int)nscore, keep,
+                                     a.keep_flags),
+                       "topk_sort1024_kernel launch");
     } else {
         LaunchScope scope(kKindSelect, stream);
         rc = cuda_fail(launch_kernel(topk_select_kernel, dim3(1), dim3(kSelThreads), 0, stream, (const double*)a.scores, (int)nscore,
