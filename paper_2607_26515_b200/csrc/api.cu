@@ -233,10 +233,10 @@ size_t residual_region_bytes(int64_t M, int64_t K, int pattern) {
 size_t linear_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K, int pattern) {
     if (M <= 0 || N <= 0 || K <= 0) return 0;
     size_t b = kWsHeader + kWsFlags + quant_scratch_bytes(M, K, pattern);
-    b += align_up((size_t)M * sizeof(float), 256);                            // row scales of the fused RMSNorm producer
     b += align_up((size_t)M * (size_t)K * 2, 256);                            // bf16 image of deq Q(X)
     b += residual_region_bytes(M, K, pattern);
     b += align_up(gemm_hif4_scratch_bytes(M, N, K), 256);                     // fp32 partial tiles of a K split
+    b += align_up((size_t)M * sizeof(float), 256);                            // row scales of the fused RMSNorm producer
     return b;
 }
 
@@ -320,12 +320,6 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
         a.rht = 1;
         a.rht_signs = rht_signs;
     }
-    if (gamma) {
-        a.gamma = static_cast<const __nv_bfloat16*>(gamma);
-        a.eps = eps;
-        a.row_scale = reinterpret_cast<float*>(ws + used);
-    }
-    used += align_up((size_t)M * sizeof(float), 256);
     // MXFP4 where it pays: the GEMM runs on the block-scaled FP4 pipe and takes packed codes and scales (they
     // fit into the space of the bf16 images; the selection zeroes dropped codes); otherwise exact bf16 images.
     const bool native = !w_bf16 && !swiglu && !gamma && !rht && fmt == kMXFP4 && gemm_mxfp4_native_supported(M, N, K, pattern != RESQ_S_NONE);
@@ -335,6 +329,11 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     if (pattern != RESQ_S_NONE) {
         region_r = ws + used;
         used += residual_region_bytes(M, K, pattern);
+    }
+    if (gamma) {  // row scales of the fused RMSNorm producer: last region, behind the fp32 partial tiles
+        a.gamma = static_cast<const __nv_bfloat16*>(gamma);
+        a.eps = eps;
+        a.row_scale = reinterpret_cast<float*>(ws + used + align_up(gemm_hif4_scratch_bytes(M, N, K), 256));
     }
     // 2:4 on the CTA-pair kernel: the residual goes to the structured-sparse MMA in compressed form
     const bool sparse24 = !w_bf16 && !swiglu && !gamma && !rht && !native && pattern == RESQ_S_2_4 && quarters == 2 &&
