@@ -29,6 +29,12 @@ def keep_quarters(pattern: int, q: int) -> int:
     return pattern | (q << 8)
 
 
+def per_strip(pattern: int) -> int:
+    """The 32x64 block pattern with the selection taken inside every strip of 32 token rows (each strip keeps
+    floor(nbc q / 4) of its K/64 blocks) instead of over the whole tensor: the load-balanced alternative."""
+    return pattern | (1 << 12)
+
+
 _lib = None
 
 

@@ -289,10 +289,13 @@ int oracle_mask(const double *v, int64_t M, int64_t K, int pattern, uint8_t *mas
     info[0] = 1.0;
     info[1] = 0.0;
     /* sparsity sweep: bits 8.. of the pattern give the kept share in quarters (0 = the paper's one half) */
-    int quarters = (pattern >> 8) & 0xFF;
+    int quarters = (pattern >> 8) & 0xF;
+    /* bit 12: the block pattern selects within every strip of 32 token rows instead of over the tensor */
+    int per_strip = (pattern >> 12) & 1;
     if (quarters == 0) quarters = 2;
-    if (quarters > 3 || pattern < 0 || (pattern >> 16)) return -2;
+    if (quarters > 3 || pattern < 0 || (pattern >> 13)) return -2;
     pattern &= 0xFF;
+    if (per_strip && pattern != S_BLOCK32x64) return -2;
     switch (pattern) {
     case S_NONE:
         return 0;
@@ -366,6 +369,29 @@ int oracle_mask(const double *v, int64_t M, int64_t K, int pattern, uint8_t *mas
                 e[a * nbc + b].idx = a * nbc + b;
                 if (scores_out) scores_out[a * nbc + b] = acc;
             }
+        if (per_strip) {
+            /* the alternative with equal work per strip: every strip of 32 rows keeps the floor(nbc q / 4)
+             * blocks of its own with the largest norm (ties: lower column block first) */
+            int64_t keep_s = nbc * quarters / 4;
+            double margin = -1.0;
+            for (int64_t a = 0; a < nbr; ++a) {
+                keyed_t *es = e + a * nbc;
+                qsort(es, (size_t)nbc, sizeof(keyed_t), cmp_keyed);
+                for (int64_t t = 0; t < keep_s; ++t) {
+                    int64_t b = es[t].idx % nbc;
+                    for (int64_t i = 0; i < BLK_ROWS; ++i)
+                        for (int64_t j = 0; j < BLK_COLS; ++j) set_bit(mask_bits, K, a * BLK_ROWS + i, b * BLK_COLS + j);
+                }
+                if (keep_s > 0 && keep_s < nbc && es[keep_s - 1].key > 0.0) {
+                    double g = (es[keep_s - 1].key - es[keep_s].key) / es[keep_s - 1].key;
+                    if (margin < 0.0 || g < margin) margin = g;
+                }
+            }
+            info[0] = exact;
+            info[1] = margin < 0.0 ? 0.0 : margin; /* smallest relative gap at a strip's cut */
+            free(e);
+            return 0;
+        }
         qsort(e, (size_t)nb, sizeof(keyed_t), cmp_keyed);
         int64_t keep = nb * quarters / 4;
         for (int64_t t = 0; t < keep; ++t) {

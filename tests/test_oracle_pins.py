@@ -744,6 +744,51 @@ def test_sparsity_sweep_masks(q):
         oracle.mask(v, oracle.S_2_4 | (4 << 8))
 
 
+@pytest.mark.parametrize("q", [1, 2, 3])
+def test_block_selection_per_strip(q):
+    """The 32x64 block pattern with the selection inside every strip of 32 token rows: whole blocks only, exactly
+    floor(nbc q / 4) per strip, no kept block of a strip scores below a dropped one of the same strip (ties to
+    the lower column block), a single strip reduces to the tensor-wide selection, and strips of very different
+    loudness separate the two definitions (tensor-wide keeps the loud strips whole, per-strip keeps its share in
+    each)."""
+    rng = np.random.default_rng(70 + q)
+    M, K = 128, 640                                                            # 4 strips x 10 column blocks
+    v = np.round(rng.standard_normal((M, K)) * 2).astype(np.float64) / 2
+    v[32:64] = 0.0                                                             # a strip of ties at zero
+    v[64:96, 64:192] = v[64:96, 192:320]                                       # equal scores inside a strip
+    v[96:] *= 1024.0                                                           # a loud strip
+    def blocks_of(bits):
+        kept = np.unpackbits(bits, axis=1, bitorder="little").astype(bool).reshape(M // 32, 32, K // 64, 64)
+        per = kept.all(axis=(1, 3))
+        assert np.array_equal(per, kept.any(axis=(1, 3)))                      # whole blocks only
+        return per
+    pat = oracle.keep_quarters(oracle.per_strip(oracle.S_BLOCK), q)
+    bits, info = oracle.mask(v, pat)
+    per = blocks_of(bits)
+    nbc = K // 64
+    assert info["exact"] and np.all(per.sum(axis=1) == nbc * q // 4)
+    score = np.array([[sum(Fraction(x) ** 2 for x in v[32 * a:32 * a + 32, 64 * b:64 * b + 64].ravel())
+                       for b in range(nbc)] for a in range(M // 32)], dtype=object)   # exact rational scores
+    for a in range(M // 32):
+        order = sorted(range(nbc), key=lambda b: (-score[a, b], b))
+        assert sorted(order[:nbc * q // 4]) == list(np.nonzero(per[a])[0])
+    # one strip alone: the same blocks as the tensor-wide definition on that strip
+    for a in range(M // 32):
+        alone = np.unpackbits(oracle.mask(v[32 * a:32 * a + 32], oracle.keep_quarters(oracle.S_BLOCK, q))[0], axis=1,
+                              bitorder="little").astype(bool).reshape(32, nbc, 64).all(axis=(0, 2))
+        assert np.array_equal(alone, per[a])
+    # the tensor-wide selection is a different set here: it keeps every block of the loud strip first
+    glob = blocks_of(oracle.mask(v, oracle.keep_quarters(oracle.S_BLOCK, q))[0])
+    assert glob.sum() == (M // 32) * nbc * q // 4 and glob[3].all() and not per[3].all()
+    # nesting with q, and the flag belongs to the block pattern only
+    if q > 1:
+        smaller = blocks_of(oracle.mask(v, oracle.keep_quarters(oracle.per_strip(oracle.S_BLOCK), q - 1))[0])
+        assert np.all(smaller <= per)
+    for other in (oracle.S_2_4, oracle.S_ROW50, oracle.S_CHAN50, oracle.S_DENSE):
+        with pytest.raises(ValueError):
+            oracle.mask(v, oracle.per_strip(other))
+
+
 def test_mxfp8_e4m3_activations_for_w4a8():
     """8-bit activations of the W4A8 ablation (this project's reading: MXFP8, E4M3 elements): the value table and
     the element rounding against torch's float8_e4m3fn, the scale property 256 <= amax / 2^e < 512, saturation,
