@@ -36,8 +36,9 @@ PATTERN_IDS = {"none": 0, "dense": 1, "2:4": 2, "row50": 3, "chan50": 4, "block"
 for _name, _base in (("{}:4", 2), ("row{}", 3), ("chan{}", 4), ("block{}", 5)):
     for _q in (1, 3):
         PATTERN_IDS[_name.format(_q if _base == 2 else 25 * _q)] = _base | (_q << 8)
+PATTERN_IDS["block-strip"] = 5 | (1 << 12)  # block selection inside every strip of 32 rows (RESQ_BLOCK_PER_STRIP)
 RHO = {0: 0.0, 1: 1.0, 2: 0.5, 3: 0.5, 4: 0.5, 5: 0.5}
-RHO.update({p: (p >> 8) / 4.0 for p in PATTERN_IDS.values() if p >> 8})
+RHO.update({p: ((p >> 8) & 0xF) / 4.0 if (p >> 8) & 0xF else 0.5 for p in PATTERN_IDS.values() if p >> 8})
 # mean DRAM bytes per GEMM launch from an ncu capture of the default workload (see profiles/)
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {(1, 2, "hif4"): 15.3e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -147,7 +148,7 @@ def main():
     ap.add_argument("--config", type=int, default=1, help="index into the workload configs (default 1: 3B decode)")
     ap.add_argument("--pattern", default=None,
                     help="none|dense|2:4|row50|chan50|block (default: the config's); sparsity sweep: 1:4|3:4|row25|row75|"
-                         "chan25|chan75|block25|block75")
+                         "chan25|chan75|block25|block75|block-strip")
     ap.add_argument("--format", default="hif4", choices=["hif4", "mxfp4"])
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--out-dtype", default="bf16", choices=["bf16", "f32"])

@@ -79,6 +79,13 @@ typedef enum {
  * the pattern itself. */
 #define RESQ_KEEP_QUARTERS(q) ((int)(q) << 8)
 
+/* Load-balanced alternative of the block pattern (Section 4.3 item 3 selects over the whole tensor):
+ * RESQ_S_BLOCK32x64_50 | RESQ_BLOCK_PER_STRIP selects inside every strip of 32 token rows -- each strip keeps the
+ * floor((K/64) q / 4) of its own K/64 blocks with the largest sum of squares (ties: lower column block first), so
+ * every strip of an M tile carries the same residual work.  May be combined with RESQ_KEEP_QUARTERS; with any other
+ * pattern it is RESQ_ERR_PATTERN. */
+#define RESQ_BLOCK_PER_STRIP (1 << 12)
+
 typedef enum { RESQ_OUT_BF16 = 0, RESQ_OUT_F32 = 1 } resq_out;
 
 /* ---- size queries (host only, no CUDA calls) -------------------------------------------------- */

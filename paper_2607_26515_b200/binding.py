@@ -148,6 +148,11 @@ def keep_quarters(pattern: int, q: int) -> int:
     return pattern | (q << 8)
 
 
+def per_strip(pattern: int) -> int:
+    """RESQ_BLOCK_PER_STRIP: the 32x64 block pattern with the selection taken inside every strip of 32 token rows."""
+    return pattern | (1 << 12)
+
+
 def pack_weight(W: torch.Tensor, fmt: str = "hif4", stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
     """*_pack_weight: W bf16 [N,K] -> (codes u8 [N,K/2], meta i32 [N,K/64] | scale u8 [N,K/32])."""
     _require_bf16_matrix(W, "W")

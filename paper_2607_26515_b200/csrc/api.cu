@@ -91,16 +91,22 @@ int check_matrix(const void* p, int64_t rows, int64_t K, int64_t ld, int fmt, co
 }
 
 // A pattern argument is a base pattern, optionally combined with RESQ_KEEP_QUARTERS(q): splits it in place.
-int split_pattern(int* pattern, int* quarters) {
-    const int q = (*pattern >> 8) & 0xFF;
-    if (*pattern < 0 || (*pattern >> 16) != 0 || q > 3) {
+int split_pattern(int* pattern, int* quarters, int* per_strip) {
+    const int q = (*pattern >> 8) & 0xF;
+    const int strip = (*pattern >> 12) & 1;
+    if (*pattern < 0 || (*pattern >> 13) != 0 || q > 3) {
         set_last_error("unknown pattern %d", *pattern);
         return RESQ_ERR_PATTERN;
     }
     *quarters = q == 0 ? 2 : q;
+    *per_strip = strip;
     *pattern &= 0xFF;
     if (q != 0 && (*pattern == RESQ_S_NONE || *pattern == RESQ_S_DENSE)) {
         set_last_error("RESQ_KEEP_QUARTERS applies to the selecting patterns only");
+        return RESQ_ERR_PATTERN;
+    }
+    if (strip && *pattern != RESQ_S_BLOCK32x64_50) {
+        set_last_error("RESQ_BLOCK_PER_STRIP applies to RESQ_S_BLOCK32x64_50 only");
         return RESQ_ERR_PATTERN;
     }
     return RESQ_OK;
@@ -190,8 +196,8 @@ int residual_mask(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, int
                   void* r_codes, void* r_side, void* mask_bits, void* workspace, size_t ws_bytes, void* stream) {
     int rc = check_matrix(X, M, K, ldx, fmt, "X");
     if (rc) return rc;
-    int quarters = 2;
-    rc = split_pattern(&pattern, &quarters);
+    int quarters = 2, per_strip = 0;
+    rc = split_pattern(&pattern, &quarters, &per_strip);
     if (rc) return rc;
     rc = check_pattern(pattern, M);
     if (rc) return rc;
@@ -208,6 +214,7 @@ int residual_mask(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, int
     a.ldx = ldx;
     a.pattern = pattern;
     a.keep_quarters = quarters;
+    a.per_strip = per_strip;
     a.x_codes = static_cast<uint8_t*>(x_codes);
     a.x_side = x_side;
     if (pattern != RESQ_S_NONE) {
@@ -248,8 +255,8 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
            bool rht = false, unsigned long long rht_signs = 0) {
     int rc = check_matrix(X, M, K, ldx, fmt, "X");
     if (rc) return rc;
-    int quarters = 2;
-    rc = split_pattern(&pattern, &quarters);
+    int quarters = 2, per_strip = 0;
+    rc = split_pattern(&pattern, &quarters, &per_strip);
     if (rc) return rc;
     if (swiglu && ldx < 2 * K) {  // X is [gate | up]: 2K columns
         set_last_error("swiglu: the input needs 2K columns per row (ldx=%lld, K=%lld)", (long long)ldx, (long long)K);
@@ -310,6 +317,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     a.ldx = ldx;
     a.pattern = pattern;
     a.keep_quarters = quarters;
+    a.per_strip = per_strip;
     size_t used = 0;
     carve_quant_scratch(ws + kWsFlags, M, K, pattern, a, used);
     a.status = reinterpret_cast<DeviceStatus*>(ws);

@@ -87,6 +87,7 @@ struct QuantArgs {
     int64_t M, K, ldx;
     int pattern;            // resq_pattern (base value); RESQ_S_NONE => no residual work at all
     int keep_quarters;      // kept share of the selection in quarters: 1, 2 (the paper's 50 %; also for 0) or 3
+    int per_strip;          // block pattern: select inside every strip of 32 rows instead of over the tensor
     // canonical packed outputs (any may be null)
     uint8_t* x_codes;
     void* x_side;           // u32 meta (HiF4) or u8 scale (MXFP4)

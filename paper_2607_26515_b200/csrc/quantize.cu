@@ -1214,7 +1214,8 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(const double* 
                                                                  uint8_t* __restrict__ flag) {
     pdl_wait();     // the scores come from the quantizer kernel just before
     pdl_trigger();  // the mask pass may be scheduled (it waits for this kernel's flags)
-    topk_select_cta(score, n, keep, flag);
+    // one independent selection of n scores per CTA (a single CTA for the tensor-wide rules)
+    topk_select_cta(score + (int64_t)blockIdx.x * n, n, keep, flag + (int64_t)blockIdx.x * n);
 }
 
 // Turn the kept-channel / kept-block flags into mask bits and zero the dropped entries of the GEMM's
@@ -1655,9 +1656,10 @@ __global__ void __launch_bounds__(kSelThreads) sel_grid_ties_kernel(const double
     }
 }
 
-// The same exact selection for at most 1024 scores (block scores of decode-sized calls): one key per thread, a
-// bitonic sort of (score, index) in descending score / ascending index order -- strides below 32 by shuffles, the
-// others through shared memory -- after which the thread at position p holds the p-th entry of the ranking.
+// The same exact selection for at most 1024 scores (block scores of decode-sized calls, the blocks of one strip):
+// one key per thread, a bitonic sort of (score, index) in descending score / ascending index order -- strides below
+// 32 by shuffles, the others through shared memory -- after which the thread at position p holds the p-th entry of
+// the ranking.  The CTA has as many threads as the sort network has inputs (the power of two at or above n).
 __global__ void __launch_bounds__(1024) topk_sort1024_kernel(const double* __restrict__ score, int n, int keep,
                                                              uint8_t* __restrict__ flag) {
     __shared__ unsigned long long s_key[1024];
@@ -1665,9 +1667,12 @@ __global__ void __launch_bounds__(1024) topk_sort1024_kernel(const double* __res
     pdl_wait();
     pdl_trigger();
     const int tid = threadIdx.x;
+    score += (int64_t)blockIdx.x * n;  // one independent selection of n scores per CTA
+    flag += (int64_t)blockIdx.x * n;
     unsigned long long key = tid < n ? (unsigned long long)__double_as_longlong(score[tid]) : 0ull;  // scores are >= 0
     int idx = tid;  // padding entries: key 0 and the highest indices, so they rank last
-    for (int k = 2; k <= 1024; k <<= 1) {
+    const int np2 = blockDim.x;  // a power of two >= n (at least a warp): the sort network's size
+    for (int k = 2; k <= np2; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
             unsigned long long pk;
             int pi;
@@ -1726,9 +1731,13 @@ __global__ void __launch_bounds__(256) chan_score_kernel(const __nv_bfloat16* __
 // then the mask pass over the residual outputs.
 static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t stream) {
     int rc = RESQ_OK;
+    // per-strip block rule: one selection of K/64 scores per strip of 32 rows (the scores of a strip are contiguous)
+    const bool strips = a.per_strip && a.pattern == RESQ_S_BLOCK32x64_50;
+    const unsigned nsel = strips ? (unsigned)(a.M / kBlkRows) : 1u;
+    if (strips) nscore = a.K / kBlkCols;
     const int keep = (int)(nscore * a.keep_quarters / 4);
     const char* grid_env = getenv("RESQ_SEL_GRID");  // debugging override: 0 keeps the one-CTA selection
-    if (a.sel_hist && nscore > kSelGridMin && keep > 0 && keep < nscore && !(grid_env && *grid_env == '0')) {
+    if (!strips && a.sel_hist && nscore > kSelGridMin && keep > 0 && keep < nscore && !(grid_env && *grid_env == '0')) {
         SelState* st = reinterpret_cast<SelState*>(a.sel_hist + 65536);
         const unsigned grid = (unsigned)std::min<int64_t>((nscore + 255) / 256, 148 * 4);
         {
@@ -1763,12 +1772,14 @@ static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t
         }
     } else if (nscore <= 1024 && !getenv_is_zero("RESQ_SEL_SORT")) {
         LaunchScope scope(kKindSelect, stream);
-        rc = cuda_fail(launch_kernel(topk_sort1024_kernel, dim3(1), dim3(1024), 0, stream, (const double*)a.scores, (int)nscore, keep,
+        unsigned np2 = 32;
+        while ((int64_t)np2 < nscore) np2 <<= 1;
+        rc = cuda_fail(launch_kernel(topk_sort1024_kernel, dim3(nsel), dim3(np2), 0, stream, (const double*)a.scores, (int)nscore, keep,
                                      a.keep_flags),
                        "topk_sort1024_kernel launch");
     } else {
         LaunchScope scope(kKindSelect, stream);
-        rc = cuda_fail(launch_kernel(topk_select_kernel, dim3(1), dim3(kSelThreads), 0, stream, (const double*)a.scores, (int)nscore,
+        rc = cuda_fail(launch_kernel(topk_select_kernel, dim3(nsel), dim3(kSelThreads), 0, stream, (const double*)a.scores, (int)nscore,
                                      keep, a.keep_flags),
                        "topk_select_kernel launch");
     }

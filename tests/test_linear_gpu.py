@@ -271,6 +271,28 @@ def test_sparsity_sweep_linear(base, q, fmt):
 
 
 @pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("shape", [(288, 512, 600), (1024, 2048, 1100)])
+def test_block_per_strip_linear(shape, fmt):
+    """The layer with the block selection taken per strip of 32 token rows (both GEMM routes of the MXFP4 twin)."""
+    m = rq()
+    M, K, N = shape
+    pattern = oracle.per_strip(oracle.S_BLOCK)
+    xb, wb = synth_xw(7 * M + N, M, K, N, n_out=2)
+    want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern, fmt)
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    work = m.alloc_workspace(m.resq_workspace_bytes(M, N, K, pattern, fmt))
+    import os
+    for native in (("1", "0") if fmt == "mxfp4" else ("0",)):
+        os.environ["RESQ_MXFP4_NATIVE"] = native
+        try:
+            y = m.resq_linear(to_dev(xb), wc, ws, pattern, fmt, out_dtype=torch.float32, workspace=work)
+            assert m.check(work) == 0, m.last_error()
+        finally:
+            os.environ.pop("RESQ_MXFP4_NATIVE", None)
+        check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+
+
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
 @pytest.mark.parametrize("shape", [(64, 256, 200), (300, 1152, 520), (1056, 512, 1100)])
 def test_w4a8_linear_parity(shape, fmt):
     """W4A8 (Table 1) with MXFP8-E4M3 activations: within tolerance of the oracle and bit-identical to the W4A16

@@ -113,6 +113,37 @@ def test_sparsity_sweep_masks_bit_exact(shape, base, q, fmt):
 
 
 @pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("q", [1, 2, 3])
+@pytest.mark.parametrize("shape", [(32, 64), (64, 256), (320, 2048), (2432, 192), (96, 18944), (4096, 1024)])
+def test_block_selection_per_strip_bit_exact(shape, q, fmt):
+    """Block pattern with the selection inside every strip of 32 token rows: codes and masks bit-exact against
+    the oracle on shapes that reach both quantizer kernels, from one block per strip (nothing or everything
+    kept) to 296 blocks per strip and 128 strips."""
+    M, K = shape
+    pattern = oracle.keep_quarters(oracle.per_strip(oracle.S_BLOCK), q)
+    bits = synth(5 * M + K + q, M, K, n_out=max(1, K // 256), extremes=False)
+    want = oracle.quantize_residual_mask(bf16_bits_to_f32(bits), pattern, fmt)
+    got = rq().residual_mask(to_dev(bits), pattern, fmt)
+    torch.cuda.synchronize()
+    for key in ("x_codes", "x_side", "r_codes", "r_side"):
+        assert np.array_equal(side_np(got[key]), want[key]), key
+    info = want["mask_info"]
+    if not (info["exact"] or info["margin"] > 2.0 ** -40):
+        pytest.skip("selection scores not exactly summable and boundary margin too small")
+    mask = got["mask"].cpu().numpy()
+    assert np.array_equal(mask, want["mask"])
+    kept = np.unpackbits(mask, axis=1, bitorder="little").reshape(M // 32, 32, K // 64, 64).all(axis=(1, 3))
+    assert np.all(kept.sum(axis=1) == (K // 64) * q // 4)
+
+
+def test_per_strip_flag_is_for_the_block_pattern_only():
+    bits = synth(3, 64, 256)
+    for base in (oracle.S_2_4, oracle.S_ROW50, oracle.S_CHAN50, oracle.S_DENSE, oracle.S_NONE):
+        with pytest.raises(Exception):
+            rq().residual_mask(to_dev(bits), oracle.per_strip(base), "hif4")
+
+
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
 @pytest.mark.parametrize("shape", [(700, 4160), (416, 18944), (1300, 2048), (900, 3584)])
 def test_row_selection_persistent_ctas(shape, fmt):
     """Row-wise selection with more rows than resident CTAs (each CTA or warp walks several rows, the next row
