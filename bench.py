@@ -341,13 +341,52 @@ def main():
     def step_graph(i):
         graphs[i % n_sets].replay()
 
-    def step_e2e(i):
+    # End to end: every step copies each layer's activations from pinned host memory, runs the layer through the
+    # public call and reads its output back.  The layers of a step are independent calls, so their copies run on
+    # two copy streams beside the compute stream (input of the next layer and output of the previous one overlap
+    # the current layer's kernels); the layer with the largest output goes first.  A step ends when every output
+    # is in host memory.
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    e2e_order = sorted(layers, key=lambda L: -L["y"].numel())
+
+    def step_e2e(i, capturing=False):
         k = i % n_sets
-        for L in layers:
+        main = torch.cuda.current_stream()
+        s_in.wait_stream(main)    # earlier work on the inputs' staging buffers is done (previous steps were synchronized)
+        for L in e2e_order:
+            with torch.cuda.stream(s_in):
+                L["x_stage"].copy_(L["x_host"], non_blocking=True)       # host -> device, pinned
+                L["ev_in"] = s_in.record_event()
+        for L in e2e_order:
             wc, ws = L["w_sets"][k]
-            L["x_stage"].copy_(L["x_host"], non_blocking=True)           # host -> device, pinned
+            main.wait_event(L["ev_in"])
             rq.resq_linear(L["x_stage"], wc, ws, pattern, fmt, Y=L["y"], workspace=L["work"])
-            L["y_host"].copy_(L["y"], non_blocking=True)                 # device -> host
+            ev = main.record_event()
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev)
+                L["y_host"].copy_(L["y"], non_blocking=True)             # device -> host
+        if capturing:
+            main.wait_stream(s_out)   # join the copy branches into the captured stream
+        else:
+            s_out.synchronize()
+            main.synchronize()
+
+    e2e_graphs = []
+
+    def build_e2e_graphs():
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for k in range(n_sets):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    step_e2e(k, capturing=True)
+                e2e_graphs.append(g)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+
+    def step_e2e_graph(i):
+        e2e_graphs[i % n_sets].replay()       # copies in, kernels and copies out: one graph launch per step
         torch.cuda.current_stream().synchronize()
 
     def barrier():
@@ -435,7 +474,19 @@ def main():
     # ---- end-to-end: host buffers, copies inside the timed region
     for i in range(3):
         step_e2e(i)
-    ms_e2e, _, _ = timed(step_e2e, args.steps)
+    run_e2e = step_e2e
+    if use_graph:
+        build_e2e_graphs()
+        run_e2e = step_e2e_graph
+        for i in range(3):
+            run_e2e(i)
+    for L in layers:  # the pipelined copies delivered what the device holds
+        if not torch.equal(L["y_host"], L["y"].cpu()) or not torch.equal(L["x_stage"].cpu(), L["x_host"]):
+            raise RuntimeError(f"end-to-end step: host copy of layer {L['spec'].name} differs from the device tensor")
+    ms_e2e, _, _ = timed(run_e2e, args.steps)
+    if os.environ.get("RESQ_BENCH_E2E_BOTH"):  # aid: the eager-launch figure beside the graph one
+        ms_eager, _, _ = timed(step_e2e, args.steps)
+        print(f"e2e eager {ms_eager / args.steps:.4f} ms  graph {ms_e2e / args.steps:.4f} ms", file=sys.stderr)
     e2e_tflops = world * flops_step / (ms_e2e / args.steps * 1e-3) / 1e12
     h2d = sum(L["x_host"].numel() * 2 for L in layers)
     d2h = sum(L["y_host"].numel() * L["y_host"].element_size() for L in layers)
