@@ -75,6 +75,11 @@ def test_host_side_argument_errors_need_no_device(lib):
     assert lib.resq_residual_mask(fake, 40, 64, 64, 5, fake, fake, fake, fake, fake, fake, 1 << 20, None) == 2
     assert lib.resq_residual_mask(fake, 32, 64, 64, 9, fake, fake, fake, fake, fake, fake, 1 << 20, None) == 5
     assert lib.resq_residual_mask(fake, 32, 64, 64, 4, fake, fake, fake, fake, fake, None, 0, None) == 4
+    # pattern modifiers: kept share in quarters (bits 8..11: 1..3, selecting patterns only), per-strip flag
+    # (bit 12: block pattern only), nothing above
+    for bad in (2 | (4 << 8), 0 | (1 << 8), 1 | (3 << 8), 2 | (1 << 12), 3 | (1 << 12), 4 | (1 << 12), 5 | (1 << 13), -1):
+        assert lib.resq_residual_mask(fake, 32, 64, 64, bad, fake, fake, fake, fake, fake, fake, 1 << 20, None) == 5, bad
+    assert lib.resq_residual_mask(fake, 40, 64, 64, 5 | (1 << 12), fake, fake, fake, fake, fake, fake, 1 << 20, None) == 2
     lib.hif4_resq_linear.argtypes = [vp, i64, i64, i64, vp, vp, i64, ci, vp, ci, i64, vp, sz, vp]
     assert lib.hif4_resq_linear(fake, 32, 64, 64, fake, fake, 0, 0, fake, 0, 64, fake, 1 << 20, None) == 2
     assert lib.hif4_resq_linear(fake, 32, 64, 64, fake, fake, 64, 0, fake, 7, 64, fake, 1 << 20, None) == 5
