@@ -844,7 +844,7 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
     if (per_group == 1 && kb_per_pair >= 8 && env_int("RESQ_GEMM_DEEP_E", 1)) {
         // three activation slots cover the latency of their loads, one raw-code slot per group is enough, and
         // the rest goes to expanded-weight slots (any number: a k-block's barrier slot is k-block mod SE)
-        const int sa2 = env_int("RESQ_GEMM_MIN_SA", 3), sr2 = kExpGroups;
+        const int sa2 = env_int("RESQ_GEMM_MIN_SA", 3), sr2 = std::max(kExpGroups, std::min(env_int("RESQ_GEMM_MIN_SR", kExpGroups), kMaxRing));
         const int left = kSmemBudget - fixed - sa2 * kAStage - sr2 * raw_stage;
         const int se2 = std::min(std::min(left / exp_stage, 2 * kExpGroups), kMaxRing);
         if (se2 > kExpGroups) {
