@@ -703,7 +703,12 @@ bool gemm_use_streamk(int64_t M, int64_t N, int64_t K) {
     if (force >= 0) return force != 0;
     if (env_int("RESQ_GEMM_PAIR_TN", 0) || env_int("RESQ_GEMM_SPLITS", 0)) return false;  // explicit tile exploration
     const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + 255) / 256);
-    return tiles <= 74 / 2 && tiles * (K / kBK) >= 2;  // at least two pairs per tile: otherwise whole tiles per pair
+    if (tiles <= 74 / 2 && tiles * (K / kBK) >= 2) return true;  // at least two pairs per tile: otherwise whole tiles per pair
+    // Opt-in (RESQ_GEMM_HYBRID=1): one whole 256-wide tile per pair and a last round of at most half the pairs whose
+    // k-blocks are dealt out over all pairs in the same kernel.  Measured slower than one round of wider tiles
+    // (M = 256, 2048 -> 22016: 67.6 us against 55.0 us per call): the fp32 partial tiles of the last round cost more
+    // than the narrower MMA instructions of the 320-wide tile.
+    return tiles > 74 && tiles <= 74 + 74 / 2 && K / kBK >= 16 && env_int("RESQ_GEMM_HYBRID", 0);
 }
 
 // The 2:4 residual on the structured-sparse MMA is complete and tested but not the default: it halves the tensor

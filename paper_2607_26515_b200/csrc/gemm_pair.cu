@@ -62,6 +62,10 @@ struct PairParams {
     // K-streamed schedule (streamk != 0): the num_tiles * G (tile, k-block) units are dealt out evenly to the
     // pairs; a pair's first and last segment may cover only part of a tile's K range and then go to fp32 slots
     int streamk;
+    // With more tiles than pairs the first dp_tiles tiles (a multiple of the number of pairs) are computed whole,
+    // one per pair and round, and written out directly; only the k-blocks of the remaining tiles are dealt out.
+    int dp_tiles;
+    int sk_pairs;            // pairs 0 .. sk_pairs-1 share the dealt-out units (at least two k-blocks each)
     float* sk_slots;         // [2 * npairs][256][TN] fp32: slot 2p = first segment of pair p, 2p + 1 = its last
     unsigned int* sk_flags;  // [num_tiles][2]: segments of the tile written, per CTA rank (zeroed before launch)
 };
@@ -121,9 +125,12 @@ struct SegIter {
         G = (int)(p.K / kBK);
         tile = pair;
         if (p.streamk) {
-            const int64_t U = (int64_t)p.num_tiles * G;
-            u0 = u = sk_begin(U, npairs, pair);
-            u1 = sk_begin(U, npairs, pair + 1);
+            const int64_t U = (int64_t)(p.num_tiles - p.dp_tiles) * G;  // units of the tiles that are dealt out
+            u0 = u = u1 = 0;
+            if (pair < p.sk_pairs) {
+                u0 = u = sk_begin(U, p.sk_pairs, pair);
+                u1 = sk_begin(U, p.sk_pairs, pair + 1);
+            }
         }
     }
     __device__ bool next(TileCoord& tc) {
@@ -133,11 +140,24 @@ struct SegIter {
             tile += npairs;
             return true;
         }
+        if (tile < p.dp_tiles) {  // whole tiles first
+            tc.tile_id = tile;
+            tc.split = 0;
+            tc.kb_begin = 0;
+            tc.nkb = G;
+            tc.n0 = (int64_t)(tile % p.ntiles_n) * TN;
+            tc.m0 = (int64_t)(tile / p.ntiles_n) * (2 * kBM);
+            tc.partial = false;
+            tc.slot = 0;
+            tile += npairs;
+            return true;
+        }
         if (u >= u1) return false;
-        const int t = (int)(u / G);
+        const int tr = (int)(u / G);     // among the tiles that are dealt out
+        const int t = p.dp_tiles + tr;
         tc.tile_id = t;
         tc.split = 0;
-        tc.kb_begin = (int)(u - (int64_t)t * G);
+        tc.kb_begin = (int)(u - (int64_t)tr * G);
         tc.nkb = (int)min((int64_t)(G - tc.kb_begin), u1 - u);
         tc.n0 = (int64_t)(t % p.ntiles_n) * TN;
         tc.m0 = (int64_t)(t / p.ntiles_n) * (2 * kBM);
@@ -167,14 +187,17 @@ template <int TN>
 __device__ __forceinline__ void streamk_fixup(const PairParams& p, int pair, int npairs, int rank, volatile int* abort_flag,
                                               volatile int* s_ok, int* s_slots, unsigned int* evt, long long t0) {
     const int G = (int)(p.K / kBK);
-    const int64_t U = (int64_t)p.num_tiles * G;
+    const int64_t U = (int64_t)(p.num_tiles - p.dp_tiles) * G;
+    if (pair >= p.sk_pairs) return;
+    npairs = p.sk_pairs;  // the pairs that share the dealt-out units
     const int64_t u0 = sk_begin(U, npairs, pair), u1 = sk_begin(U, npairs, pair + 1);
     if (u1 <= u0) return;
-    const int t_first = (int)(u0 / G), t_last = (int)((u1 - 1) / G);
+    const int t_first = (int)(u0 / G), t_last = (int)((u1 - 1) / G);  // among the tiles that are dealt out
     for (int which = 0; which < 2; ++which) {
-        const int t = which == 0 ? t_first : t_last;
+        const int tr = which == 0 ? t_first : t_last;
         if (which == 1 && t_last == t_first) break;
-        const int64_t tb = (int64_t)t * G, te = tb + G;
+        const int t = p.dp_tiles + tr;  // output tile
+        const int64_t tb = (int64_t)tr * G, te = tb + G;
         if (u0 <= tb && u1 >= te) continue;  // this pair computed the whole tile and wrote it out directly
         const int pf = sk_pair_of(U, npairs, tb), pl = sk_pair_of(U, npairs, te - 1);
         const int nseg = pl - pf + 1, j = pair - pf;
@@ -774,6 +797,8 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
         return RESQ_ERR_CUDA;
     }
     p.streamk = streamk ? 1 : 0;
+    p.dp_tiles = 0;
+    p.sk_pairs = 0;
     p.sk_slots = g.splitk_partials;
     p.sk_flags = g.sk_flags;
     p.Y = g.Y;
@@ -892,6 +917,9 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
             set_last_error("gemm pair kernel: no cluster of two CTAs fits on this device");
             return RESQ_ERR_CUDA;
         }
+        // more tiles than pairs: whole rounds of tiles first, only the last, incomplete round is dealt out by k-blocks
+        if (p.num_tiles > npairs) p.dp_tiles = (p.num_tiles / npairs) * npairs;
+        p.sk_pairs = (int)std::max<int64_t>(1, std::min<int64_t>(npairs, (int64_t)(p.num_tiles - p.dp_tiles) * G / 2));
     }
     {
         LaunchScope scope(kKindGemm, stream);

@@ -270,6 +270,26 @@ def test_sparsity_sweep_linear(base, q, fmt):
         check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
 
 
+@pytest.mark.parametrize("case", [(256, 1024, 22016, oracle.S_2_4), (200, 1024, 20000, oracle.S_NONE),
+                                  (512, 1024, 11000, oracle.S_DENSE), (256, 1088, 37888, oracle.S_2_4)])
+def test_whole_tiles_then_dealt_out_k_blocks(case, monkeypatch):
+    """K-streamed schedule with more tiles than CTA pairs (opt-in): whole rounds of tiles are computed one per pair
+    and written directly, only the last round's k-blocks are dealt out and summed from fp32 slots.  One round plus a
+    remainder, two M tiles, a ragged last tile, and two whole rounds with no remainder."""
+    m = rq()
+    M, K, N, pattern = case
+    monkeypatch.setenv("RESQ_GEMM_HYBRID", "1")
+    if N > 30000:
+        monkeypatch.setenv("RESQ_GEMM_STREAMK", "1")   # 148 tiles: two whole rounds
+    xb, wb = synth_xw(M + N, M, K, N, n_out=2)
+    want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern, "hif4")
+    wc, ws = m.pack_weight(to_dev(wb), "hif4")
+    work = m.alloc_workspace(m.resq_workspace_bytes(M, N, K, pattern, "hif4"))
+    y = m.resq_linear(to_dev(xb), wc, ws, pattern, "hif4", out_dtype=torch.float32, workspace=work)
+    assert m.check(work) == 0, m.last_error()
+    check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+
+
 @pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
 @pytest.mark.parametrize("shape", [(288, 512, 600), (1024, 2048, 1100)])
 def test_block_per_strip_linear(shape, fmt):
@@ -512,8 +532,9 @@ def test_mxfp4_block_scaled_fp4_gemm(monkeypatch, pattern, shape):
 
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_k_streamed_schedule_with_uneven_segments(monkeypatch, out_dtype):
-    """More output tiles than CTA pairs: the (tile, k-block) units are dealt out evenly, so pairs start and end in
-    the middle of a tile's K range and most tiles are summed from two or three partial segments."""
+    """More output tiles than CTA pairs with a short K range: two whole rounds of tiles, then the 50 k-blocks of the
+    last ten tiles are dealt out to 25 pairs (two each), so those tiles are summed from two or three partial
+    segments while the other pairs have nothing left to do."""
     monkeypatch.setenv("RESQ_GEMM_STREAMK", "1")
     m = rq()
     M, K, N = 300, 320, 20000 - 24     # 2 x 79 tiles of 256 x 256, 5 k-blocks each; ragged in M and N
