@@ -2,8 +2,12 @@
 """Benchmark of the Rollout-ResQ FP4 linear path (Eq. (5)) on B200.
 
 A "step" is one pass of the whole hot path -- quantize X, residual, re-quantize, select, two-term
-GEMM against packed HiF4 weights -- over the four linears of one transformer block of the
-workload (default: the Qwen2.5-3B decode-shaped configuration, M = 256 tokens, S_2:4).
+GEMM against packed HiF4 weights -- over the four linears of one transformer block of the workload.
+The headline workload is the largest single-GPU configuration, the Qwen2.5-Math-7B prefill-shaped
+block (M = 16384 tokens) with the S_2:4 residual; the same JSON line carries the other
+configurations (`per_config`), the residual patterns and the MXFP4 twin on the headline workload
+(`per_pattern`), a true decode sweep M = 16 ... 128 with its HBM fraction (`decode_sweep`) and the
+quantizer-only bandwidth sweep (`quantizer_sweep`).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--pattern P] [--format F]
     python bench.py --impl reference ...        # times the CPU oracle on a bounded sample
@@ -13,6 +17,7 @@ Prints ONE JSON line on stdout (rank 0); `--verbose` adds a per-layer table on s
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -27,9 +32,32 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from workloads import CONFIGS, make_activation, make_weight  # noqa: E402
+from workloads import CONFIGS  # noqa: E402
+from workloads import make_activation as _make_activation, make_weight as _make_weight  # noqa: E402
+
+_HOST_TENSORS = {}
+
+
+def make_activation(cfg, li, M=None):
+    """The seeded activation of a layer, generated once per process (the 7B prefill tensors take seconds to draw)."""
+    key = ("x", cfg.index, cfg.layers[li].name, cfg.M if M is None else M)
+    if key not in _HOST_TENSORS:
+        base = CONFIGS[cfg.index]  # (cfg may be a subset of its layers or carry another M: seeds follow the base config)
+        _HOST_TENSORS[key] = _make_activation(base, [l.name for l in base.layers].index(cfg.layers[li].name),
+                                              cfg.M if M is None else M)
+    return _HOST_TENSORS[key]
+
+
+def make_weight(cfg, li):
+    key = ("w", cfg.index, cfg.layers[li].name)
+    if key not in _HOST_TENSORS:
+        _HOST_TENSORS[key] = _make_weight(CONFIGS[cfg.index], [l.name for l in CONFIGS[cfg.index].layers].index(cfg.layers[li].name))
+    return _HOST_TENSORS[key]
+
 
 METRIC = "hif4_resq_linear TFLOP/s & GB/s at 1 B200; % of FP4-tensor/HBM roofline"
+HEADLINE_CONFIG = 4       # the largest single-GPU configuration (7B prefill, M = 16384)
+HEADLINE_PATTERN = "2:4"  # the paper's main variant, Rollout-ResQ-S_2:4
 L2_BYTES = 126 * 1024 * 1024
 PATTERN_IDS = {"none": 0, "dense": 1, "2:4": 2, "row50": 3, "chan50": 4, "block": 5}
 # sparsity sweep: the selecting patterns with 1/4 or 3/4 kept (RESQ_KEEP_QUARTERS)
@@ -37,10 +65,12 @@ for _name, _base in (("{}:4", 2), ("row{}", 3), ("chan{}", 4), ("block{}", 5)):
     for _q in (1, 3):
         PATTERN_IDS[_name.format(_q if _base == 2 else 25 * _q)] = _base | (_q << 8)
 PATTERN_IDS["block-strip"] = 5 | (1 << 12)  # block selection inside every strip of 32 rows (RESQ_BLOCK_PER_STRIP)
+PATTERN_NAMES = {v: k for k, v in PATTERN_IDS.items()}
 RHO = {0: 0.0, 1: 1.0, 2: 0.5, 3: 0.5, 4: 0.5, 5: 0.5}
 RHO.update({p: ((p >> 8) & 0xF) / 4.0 if (p >> 8) & 0xF else 0.5 for p in PATTERN_IDS.values() if p >> 8})
-# mean DRAM bytes per GEMM launch from an ncu capture of the default workload (see profiles/)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {(1, 2, "hif4"): 15.3e6}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the dominant GEMM kernel from ncu captures
+# of single layers (summaries with their commands under profiles/), keyed by (config, layer, pattern id, format)
+NCU_TRAFFIC = {}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -64,6 +94,13 @@ def layer_bytes(M, N, K, pattern, fmt):
     """Bytes the method must move per call: bf16 X in, packed W in, bf16 Y out."""
     w_bits = 4.5 if fmt == "hif4" else 4.25
     return 2.0 * M * K + w_bits / 8.0 * N * K + 2.0 * M * N
+
+
+def gemm_bytes(M, N, K, pattern, fmt):
+    """Algorithmic bytes of the GEMM launch alone: packed W, packed Q(X), the packed (2:4: compressed) residual, bf16 Y."""
+    side = 0.5625 if fmt == "hif4" else 0.53125
+    res = {0: 0.0, 1: side, 2: side - 0.125}.get(pattern & 0xFF, side - 0.125)
+    return side * N * K + (side + res) * M * K + 2.0 * M * N
 
 
 # ----------------------------------------------------------------------------- clocks sampler
@@ -94,16 +131,11 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
-    def stop(self, t0: float, t1: float):
+    def window(self, t0: float, t1: float):
+        """Summary of the samples taken between two wall-clock instants (the sampler keeps running)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            pass
-        rows = [r for (t, r) in self.rows if t0 - 0.05 <= t <= t1 + 0.15 and len(r) >= 9] or \
-               [r for (_, r) in self.rows if len(r) >= 9]
+        rows = [r for (t, r) in list(self.rows) if t0 - 0.05 <= t <= t1 + 0.15 and len(r) >= 9]
         if not rows:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
         sm = [float(r[1]) for r in rows]
@@ -112,12 +144,21 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(sm), "sm_max_mhz": float(rows[0][2]), "reasons": reasons,
                 "samples": len(rows), "power_w_max": max(float(r[3]) for r in rows)}
 
+    def stop(self):
+        if self.proc is None:
+            return
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+
 
 # ----------------------------------------------------------------------------- CPU oracle timing
 
-def time_oracle(cfg, pattern, fmt, budget_s=20.0):
-    """Times the oracle, as it stands, on a bounded sample of the workload: every layer of the config, on
-    the first rows of X (all of them if that fits the budget).  Returns (TFLOP/s, cores, description, s)."""
+def oracle_sample(cfg, budget_s):
+    """A bounded sample of the workload for the CPU oracle: every layer of the config, the first rows of X (all of
+    them if that fits the budget).  Returns (rows, [(X f32, W f32, spec)])."""
     import oracle
     from workloads import bf16_bits_to_f32
     threads = oracle.num_threads()
@@ -125,38 +166,140 @@ def time_oracle(cfg, pattern, fmt, budget_s=20.0):
     rate = 0.6e9 * threads                                            # rough fp64 MAC/s of the plain triple loop
     rows = int(max(32, min(cfg.M, budget_s * rate / macs_per_row)))
     rows -= rows % 32
+    tensors = [(bf16_bits_to_f32(make_activation(cfg, li, M=rows)), bf16_bits_to_f32(make_weight(cfg, li)), spec)
+               for li, spec in enumerate(cfg.layers)]
+    return rows, tensors
+
+
+def time_oracle(cfg, pattern, fmt, rows, tensors):
+    """Times the oracle, as it stands, on the sample.  Returns (TFLOP/s, cores, description, seconds)."""
+    import oracle
     flops, dt = 0.0, 0.0
-    for li, spec in enumerate(cfg.layers):
-        x = bf16_bits_to_f32(make_activation(cfg, li, M=rows))
-        w = bf16_bits_to_f32(make_weight(cfg, li))
+    for x, w, spec in tensors:
         t0 = time.perf_counter()
         oracle.resq_linear(x, w, pattern, fmt, want_abs=False)
         dt += time.perf_counter() - t0
         flops += layer_flops(rows, spec.N, spec.K, pattern)
     sample = (f"{cfg.name}: all {len(cfg.layers)} layers, first {rows} of {cfg.M} token rows "
               f"(weight packing, quantizer, masks and fp64 product all timed)")
-    return flops / dt / 1e12, threads, sample, dt
+    return flops / dt / 1e12, oracle.num_threads(), sample, dt
 
 
-# ----------------------------------------------------------------------------- main
+# ----------------------------------------------------------------------------- one workload on the device
+
+class Workload:
+    """The tensors of one configuration on the device, and the step over its layers."""
+
+    def __init__(self, rq, torch, dev, cfg, pattern, fmt, out_dtype, host_copies=False):
+        self.rq, self.torch, self.dev, self.cfg, self.pattern, self.fmt = rq, torch, dev, cfg, pattern, fmt
+        self.layers = []
+        w_bytes_total = 0
+        for li, spec in enumerate(cfg.layers):
+            xb = make_activation(cfg, li)
+            wb = make_weight(cfg, li)
+            x_host = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16)
+            if host_copies:
+                x_host = x_host.pin_memory()
+            w_dev = torch.from_numpy(wb.view(np.int16)).view(torch.bfloat16).to(dev)
+            wc, ws = rq.pack_weight(w_dev, fmt)
+            del w_dev
+            w_bytes_total += wc.numel() + ws.numel() * ws.element_size()
+            self.layers.append({"spec": spec, "x_host": x_host, "wc": wc, "ws": ws})
+        # rotate over enough copies of the packed weights that a step never finds them in L2
+        act_bytes = sum(cfg.M * l.K * 2 for l in cfg.layers)
+        n_sets = max(2, int(np.ceil(1.5 * L2_BYTES / max(1, w_bytes_total + act_bytes))))
+        self.n_sets = n_sets = min(n_sets, 16)
+        for L in self.layers:
+            spec = L["spec"]
+            L["w_sets"] = [(L["wc"], L["ws"])] + [(L["wc"].clone(), L["ws"].clone()) for _ in range(n_sets - 1)]
+            L["x_sets"] = [L["x_host"].to(dev) for _ in range(n_sets)]
+            L["y"] = torch.empty((cfg.M, spec.N), dtype=out_dtype, device=dev)
+            L["work"] = rq.alloc_workspace(rq.resq_workspace_bytes(cfg.M, spec.N, spec.K, pattern, fmt), dev)
+            if host_copies:
+                L["y_host"] = torch.empty((cfg.M, spec.N), dtype=out_dtype).pin_memory()
+                L["x_stage"] = torch.empty_like(L["x_sets"][0])
+        self.l2_note = (f"rotating {n_sets} copies of weights and activations "
+                        f"({n_sets * (w_bytes_total + act_bytes) / 1e6:.0f} MB > 126 MB L2)")
+        self.w_bytes_total = w_bytes_total
+        self.graphs = []
+        self.flops_step = sum(layer_flops(cfg.M, L["spec"].N, L["spec"].K, pattern) for L in self.layers)
+        self.bytes_step = sum(layer_bytes(cfg.M, L["spec"].N, L["spec"].K, pattern, fmt) for L in self.layers)
+
+    def step(self, i):
+        k = i % self.n_sets
+        for L in self.layers:
+            wc, ws = L["w_sets"][k]
+            self.rq.resq_linear(L["x_sets"][k], wc, ws, self.pattern, self.fmt, Y=L["y"], workspace=L["work"])
+
+    def check(self):
+        for L in self.layers:
+            if self.rq.check(L["work"]) != 0:
+                raise SystemExit("device status: " + self.rq.last_error())
+
+    # One CUDA graph per rotation set: at decode sizes the step is a handful of short kernels and the host
+    # (tensor-map encoding, launches) would otherwise be the bottleneck.  Everything the library enqueues
+    # is capturable; attributes were set during warm-up.
+    def build_graphs(self, fn=None, into=None):
+        torch = self.torch
+        into = self.graphs if into is None else into
+        fn = fn or self.step
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for k in range(self.n_sets):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    fn(k)
+                into.append(g)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+
+    def step_graph(self, i):
+        self.graphs[i % self.n_sets].replay()
+
+    def profile(self, steps):
+        """Per-kernel device time: CUDA events around every launch on the launching stream (a separate pass: the event
+        records serialize the kernels and switch the programmatic dependent launch off, so these are upper bounds)."""
+        rq, torch = self.rq, self.torch
+        rq.profile_enable(True)
+        rq.profile_read()
+        torch.cuda.synchronize()
+        per_layer = []
+        for L in self.layers:
+            for i in range(steps):
+                wc, ws = L["w_sets"][i % self.n_sets]
+                rq.resq_linear(L["x_sets"][i % self.n_sets], wc, ws, self.pattern, self.fmt, Y=L["y"], workspace=L["work"])
+            torch.cuda.synchronize()
+            pr = rq.profile_read()
+            per_layer.append({k: (v[0] / steps, v[1] // steps) for k, v in pr.items()})
+        rq.profile_enable(False)
+        return per_layer
+
+    def free(self):
+        self.graphs.clear()
+        self.layers.clear()
+        self.torch.cuda.empty_cache()
+
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=1, help="index into the workload configs (default 1: 3B decode)")
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=HEADLINE_CONFIG,
+                    help="index into the workload configs (default 4: 7B prefill, the largest single-GPU configuration)")
     ap.add_argument("--pattern", default=None,
-                    help="none|dense|2:4|row50|chan50|block (default: the config's); sparsity sweep: 1:4|3:4|row25|row75|"
-                         "chan25|chan75|block25|block75|block-strip")
+                    help="none|dense|2:4|row50|chan50|block (default: 2:4 on config 4, else the config's); sparsity sweep: "
+                         "1:4|3:4|row25|row75|chan25|chan75|block25|block75|block-strip")
     ap.add_argument("--format", default="hif4", choices=["hif4", "mxfp4"])
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--out-dtype", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--layers", default=None, help="comma-separated subset of the config's layers (profiling aid)")
     ap.add_argument("--tokens", type=int, default=None, help="override M (profiling aid; not the benchmark workload)")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the end-to-end and per-kernel passes (profiling aid)")
+    ap.add_argument("--headline-only", action="store_true", help="skip per_config / per_pattern / sweeps")
     ap.add_argument("--quantizer-sweep", action="store_true",
-                    help="bandwidth sweep of *_quantize_act over M x K (prints a table on stderr and one JSON line)")
+                    help="only the bandwidth sweep of *_quantize_act over M x K (table on stderr and one JSON line)")
     ap.add_argument("--accuracy-contrast", action="store_true",
                     help="relative error of plain FP4, the rotation baseline and the residual variants against the exact "
                          "bf16 product on the config's synthetic outlier tensors (no timing)")
@@ -166,18 +309,21 @@ def main():
     args = ap.parse_args()
 
     cfg = CONFIGS[args.config]
-    if args.layers or args.tokens:
-        import dataclasses
+    subset = bool(args.layers or args.tokens)
+    if subset:
         keep = args.layers.split(",") if args.layers else [l.name for l in cfg.layers]
         cfg = dataclasses.replace(cfg, layers=tuple(l for l in cfg.layers if l.name in keep),
                                   M=args.tokens or cfg.M, name=cfg.name + " (subset)")
-    pattern = PATTERN_IDS[args.pattern] if args.pattern else cfg.patterns[0]
-    pattern_name = {v: k for k, v in PATTERN_IDS.items()}[pattern]
+    if args.pattern:
+        pattern = PATTERN_IDS[args.pattern]
+    else:
+        pattern = PATTERN_IDS[HEADLINE_PATTERN] if args.config == HEADLINE_CONFIG else cfg.patterns[0]
+    pattern_name = PATTERN_NAMES[pattern]
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     config_desc = {
-        "workload": f"{cfg.name}: M={cfg.M}, layers " + ", ".join(f"{l.name} {l.K}->{l.N}" for l in cfg.layers),
+        "workload": f"config {args.config} ({cfg.name}): M={cfg.M}, layers " + ", ".join(f"{l.name} {l.K}->{l.N}" for l in cfg.layers),
         "pattern": pattern_name, "format": args.format, "out_dtype": args.out_dtype,
         "parallelism": "replicas only (one independent copy of the step per GPU)",
     }
@@ -185,12 +331,12 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return
-        vals = []
+        rows, tensors = oracle_sample(cfg, budget_s=8.0)
+        vals, info = [], None
         for _ in range(max(1, min(args.warmup, 1))):
-            time_oracle(cfg, pattern, args.format, budget_s=3.0)
-        info = None
+            time_oracle(cfg, pattern, args.format, rows, tensors)
         for _ in range(max(1, min(args.steps, 3))):
-            info = time_oracle(cfg, pattern, args.format, budget_s=8.0)
+            info = time_oracle(cfg, pattern, args.format, rows, tensors)
             vals.append(info[0])
         v = statistics.median(vals)
         line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "TFLOP/s", "n_gpus": args.gpus,
@@ -216,22 +362,20 @@ def main():
 
     out_dtype = torch.bfloat16 if args.out_dtype == "bf16" else torch.float32
     fmt = args.format
+    peaks, peak_kind = load_peaks()
 
-    if args.quantizer_sweep:
-        # hif4_quantize_act / mxfp4_quantize_act alone: read bf16 X, write packed codes + metadata.
-        peaks, peak_kind = load_peaks()
+    def quantizer_sweep(fmt, Ms, verbose):
+        """*_quantize_act alone: read bf16 X, write packed codes + metadata; rotating inputs larger than L2."""
         bpe = 2.0 + (0.5625 if fmt == "hif4" else 0.53125)
         rows = []
         for K in (2048, 18944):
-            for M in (256, 512, 1024, 2048, 4096, 8192, 16384, 32768):
-                nbuf = max(2, int(np.ceil(1.5 * L2_BYTES / (M * K * 2))))
-                nbuf = min(nbuf, 64)
+            for M in Ms:
+                nbuf = min(64, max(2, int(np.ceil(1.5 * L2_BYTES / (M * K * 2)))))
                 xs = [torch.randn((M, K), device=dev, dtype=torch.float32).to(torch.bfloat16) for _ in range(nbuf)]
                 for i in range(3):
                     rq.quantize_act(xs[i % nbuf], fmt)
                 torch.cuda.synchronize()
                 reps = max(10, min(200, int(2e9 / (M * K * bpe))))
-                codes = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
                 for i in range(reps):
@@ -240,10 +384,15 @@ def main():
                 torch.cuda.synchronize()
                 us = e0.elapsed_time(e1) * 1e3 / reps
                 gbs = M * K * bpe / (us * 1e-6) / 1e9
-                rows.append({"M": M, "K": K, "us": us, "GB/s": gbs, "frac_of_hbm": gbs / peaks["hbm_gbs"]})
-                print(f"[quantize_act {fmt}] M={M:6d} K={K:6d}  {us:9.1f} us  {gbs:8.1f} GB/s  "
-                      f"{100 * gbs / peaks['hbm_gbs']:5.1f} % of {peak_kind} copy rate", file=sys.stderr)
-                del xs, codes
+                rows.append({"M": M, "K": K, "us": round(us, 2), "GB/s": round(gbs, 1), "frac_of_hbm": round(gbs / peaks["hbm_gbs"], 4)})
+                if verbose:
+                    print(f"[quantize_act {fmt}] M={M:6d} K={K:6d}  {us:9.1f} us  {gbs:8.1f} GB/s  "
+                          f"{100 * gbs / peaks['hbm_gbs']:5.1f} % of {peak_kind} copy rate", file=sys.stderr)
+                del xs
+        return bpe, rows
+
+    if args.quantizer_sweep:
+        bpe, rows = quantizer_sweep(fmt, (256, 512, 1024, 2048, 4096, 8192, 16384, 32768), True)
         best = max(rows, key=lambda r: r["GB/s"])
         print(json.dumps({"metric": f"{fmt}_quantize_act GB/s (algorithmic {bpe} B/element)", "value": best["GB/s"],
                           "unit": "GB/s", "roofline": {"bound": "hbm", "achieved": best["GB/s"], "peak": peaks["hbm_gbs"],
@@ -289,106 +438,6 @@ def main():
                           "data": "synthetic", "config": config_desc}))
         return
 
-    # ---- inputs: generated once on the host, packed once (weights are packed per policy update, not per call)
-    layers = []
-    w_bytes_total = 0
-    for li, spec in enumerate(cfg.layers):
-        xb = make_activation(cfg, li)
-        wb = make_weight(cfg, li)
-        x_host = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
-        w_dev = torch.from_numpy(wb.view(np.int16)).view(torch.bfloat16).to(dev)
-        wc, ws = rq.pack_weight(w_dev, fmt)
-        del w_dev
-        w_bytes_total += wc.numel() + ws.numel() * ws.element_size()
-        layers.append({"spec": spec, "x_host": x_host, "wc": wc, "ws": ws})
-    # rotate over enough copies of the packed weights that a step never finds them in L2
-    n_sets = max(2, int(np.ceil(1.5 * L2_BYTES / max(1, w_bytes_total))))
-    n_sets = min(n_sets, 16)
-    for L in layers:
-        spec = L["spec"]
-        L["w_sets"] = [(L["wc"], L["ws"])] + [(L["wc"].clone(), L["ws"].clone()) for _ in range(n_sets - 1)]
-        L["x_sets"] = [L["x_host"].to(dev) for _ in range(n_sets)]
-        L["y"] = torch.empty((cfg.M, spec.N), dtype=out_dtype, device=dev)
-        L["y_host"] = torch.empty((cfg.M, spec.N), dtype=out_dtype).pin_memory()
-        L["x_stage"] = torch.empty_like(L["x_sets"][0])
-        L["work"] = rq.alloc_workspace(rq.resq_workspace_bytes(cfg.M, spec.N, spec.K, pattern, fmt), dev)
-    config_desc["l2"] = (f"rotating {n_sets} copies of weights and activations "
-                         f"({n_sets * w_bytes_total / 1e6:.0f} MB of packed weights > 126 MB L2)")
-
-    def step(i):
-        k = i % n_sets
-        for L in layers:
-            wc, ws = L["w_sets"][k]
-            rq.resq_linear(L["x_sets"][k], wc, ws, pattern, fmt, Y=L["y"], workspace=L["work"])
-
-    # One CUDA graph per rotation set: at decode sizes the step is a dozen short kernels and the host
-    # (tensor-map encoding, launches) would otherwise be the bottleneck.  Everything the library enqueues
-    # (memsets, kernels, cluster launches) is capturable; attributes were set during warm-up.
-    graphs = []
-
-    def build_graphs():
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            for k in range(n_sets):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=side):
-                    step(k)
-                graphs.append(g)
-        torch.cuda.current_stream().wait_stream(side)
-        torch.cuda.synchronize()
-
-    def step_graph(i):
-        graphs[i % n_sets].replay()
-
-    # End to end: every step copies each layer's activations from pinned host memory, runs the layer through the
-    # public call and reads its output back.  The layers of a step are independent calls, so their copies run on
-    # two copy streams beside the compute stream (input of the next layer and output of the previous one overlap
-    # the current layer's kernels); the layer with the largest output goes first.  A step ends when every output
-    # is in host memory.
-    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
-    e2e_order = sorted(layers, key=lambda L: -L["y"].numel())
-
-    def step_e2e(i, capturing=False):
-        k = i % n_sets
-        main = torch.cuda.current_stream()
-        s_in.wait_stream(main)    # earlier work on the inputs' staging buffers is done (previous steps were synchronized)
-        for L in e2e_order:
-            with torch.cuda.stream(s_in):
-                L["x_stage"].copy_(L["x_host"], non_blocking=True)       # host -> device, pinned
-                L["ev_in"] = s_in.record_event()
-        for L in e2e_order:
-            wc, ws = L["w_sets"][k]
-            main.wait_event(L["ev_in"])
-            rq.resq_linear(L["x_stage"], wc, ws, pattern, fmt, Y=L["y"], workspace=L["work"])
-            ev = main.record_event()
-            with torch.cuda.stream(s_out):
-                s_out.wait_event(ev)
-                L["y_host"].copy_(L["y"], non_blocking=True)             # device -> host
-        if capturing:
-            main.wait_stream(s_out)   # join the copy branches into the captured stream
-        else:
-            s_out.synchronize()
-            main.synchronize()
-
-    e2e_graphs = []
-
-    def build_e2e_graphs():
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            for k in range(n_sets):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=side):
-                    step_e2e(k, capturing=True)
-                e2e_graphs.append(g)
-        torch.cuda.current_stream().wait_stream(side)
-        torch.cuda.synchronize()
-
-    def step_e2e_graph(i):
-        e2e_graphs[i % n_sets].replay()       # copies in, kernels and copies out: one graph launch per step
-        torch.cuda.current_stream().synchronize()
-
     def barrier():
         if world > 1:
             torch.distributed.barrier()
@@ -407,143 +456,251 @@ def main():
         ms = max_over_ranks(e0.elapsed_time(e1), dev)
         return ms, t0, t1
 
-    def per_layer_table():
-        rq.profile_enable(True)
-        for L in layers:
-            spec = L["spec"]
-            rq.profile_read()
-            for i in range(10):
-                wc, ws = L["w_sets"][i % n_sets]
-                rq.resq_linear(L["x_sets"][i % n_sets], wc, ws, pattern, fmt, Y=L["y"], workspace=L["work"])
-            torch.cuda.synchronize()
-            pr = rq.profile_read()
-            f = layer_flops(cfg.M, spec.N, spec.K, pattern)
-            g_us = pr["gemm"][0] * 100.0
-            print(f"[layer {spec.name:8s}] K={spec.K:6d} N={spec.N:6d}  quant {pr['quantize'][0]*100:8.1f} us  "
-                  f"select {pr['select'][0]*100:7.1f} us  gemm {g_us:8.1f} us  reduce {pr['splitk_reduce'][0]*100:6.1f} us  "
-                  f"gemm {f / (g_us * 1e-6) / 1e12:7.1f} TFLOP/s", file=sys.stderr)
-        rq.profile_enable(False)
-
+    use_graph = not args.no_graph
     warmup = max(3, args.warmup)
-    for i in range(warmup):
-        step(i)
-    for L in layers:
-        if rq.check(L["work"]) != 0:
-            raise SystemExit("device status: " + rq.last_error())
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
+    def tensor_peak_for(fmt_, clocks):
+        """Denominator of the GEMM roofline: the measured bf16 peak -- the sustained figure when the clock record of
+        the timed region shows the power-capped regime (sw_power_cap active or SM clock well below its maximum), the
+        burst figure otherwise; the block-scaled FP4 route takes it times the nominal FP4 : bf16 ratio (9 : 2.25)."""
+        capped = bool(clocks) and clocks.get("sm_mhz") and (
+            "sw_power_cap" in clocks.get("reasons", []) or clocks["sm_mhz"] < 0.85 * clocks["sm_max_mhz"])
+        key = "bf16_tflops_sustained" if capped and peaks.get("bf16_tflops_sustained") else "bf16_tflops"
+        p = float(peaks[key])
+        src = f"bf16 {'sustained' if key.endswith('sustained') else 'burst'}, of {peak_kind}"
+        if fmt_ == "mxfp4":
+            return p * 4.0, src + " x 4 (nominal FP4 : bf16 ratio)"
+        return p, src
+
+    def measure(cfg_, pattern_, fmt_, steps, sampler=None, e2e=False, verbose=False):
+        """Times `steps` steps of one workload (value), then the per-kernel pass; optionally the end-to-end pass."""
+        wl = Workload(rq, torch, dev, cfg_, pattern_, fmt_, out_dtype, host_copies=e2e)
+        for i in range(warmup):
+            wl.step(i)
+        wl.check()
+        launches0 = rq.kernel_launches()
+        wl.step(0)
+        launches_per_step = rq.kernel_launches() - launches0
+        run_step = wl.step
+        if use_graph:
+            wl.build_graphs()
+            for i in range(3):
+                wl.step_graph(i)
+            run_step = wl.step_graph
+        ms, t0, t1 = timed(run_step, steps)
+        # keep the GPU busy a little longer so that the 100 ms sampler certainly sees the loaded state
+        clocks = None
+        if sampler is not None:
+            t_load0 = time.time()
+            while time.time() - t_load0 < 0.6:
+                for i in range(max(1, min(20, int(20.0 / max(ms / steps, 1e-3))))):
+                    run_step(i)
+                torch.cuda.synchronize()
+            clocks = sampler.window(t0, time.time())
+        wl.check()
+        ms_per_step = ms / steps
+        res = {
+            "ms_per_step": ms_per_step, "launches_per_step": int(launches_per_step),
+            "tflops": world * wl.flops_step / (ms_per_step * 1e-3) / 1e12,
+            "gbs": world * wl.bytes_step / (ms_per_step * 1e-3) / 1e9,
+            "clocks": clocks, "l2": wl.l2_note, "flops_step": wl.flops_step, "bytes_step": wl.bytes_step,
+        }
+        if not args.skip_e2e:
+            per_layer = wl.profile(min(steps, 10))
+            kinds = ("quantize", "select", "gemm", "splitk_reduce")
+            tot = {k: sum(pl[k][0] for pl in per_layer) for k in kinds}
+            n = {k: sum(pl[k][1] for pl in per_layer) for k in kinds}
+            kernel_ms = sum(tot.values())
+            res.update({"gemm_ms": tot["gemm"], "gemm_launches": n["gemm"], "quant_ms": tot["quantize"], "quant_launches": n["quantize"],
+                        "select_ms": tot["select"], "reduce_ms": tot["splitk_reduce"], "kernel_ms": kernel_ms,
+                        "per_layer": [{"layer": L["spec"].name, "K": L["spec"].K, "N": L["spec"].N,
+                                       "quant_us": round(pl["quantize"][0] * 1e3, 1), "select_us": round(pl["select"][0] * 1e3, 1),
+                                       "gemm_us": round((pl["gemm"][0] + pl["splitk_reduce"][0]) * 1e3, 1),
+                                       "gemm_tflops": round(layer_flops(cfg_.M, L["spec"].N, L["spec"].K, pattern_) /
+                                                            max(1e-9, (pl["gemm"][0] + pl["splitk_reduce"][0]) * 1e-3) / 1e12, 1)}
+                                      for L, pl in zip(wl.layers, per_layer)]})
+            if verbose:
+                for row in res["per_layer"]:
+                    print(f"[layer {row['layer']:8s}] K={row['K']:6d} N={row['N']:6d}  quant {row['quant_us']:8.1f} us  "
+                          f"select {row['select_us']:7.1f} us  gemm {row['gemm_us']:8.1f} us  {row['gemm_tflops']:7.1f} TFLOP/s",
+                          file=sys.stderr)
+        if e2e:
+            res["e2e"] = measure_e2e(wl, steps)
+        wl.free()
+        del wl
+        return res
+
+    def measure_e2e(wl, steps):
+        # End to end: every step copies each layer's activations from pinned host memory, runs the layer through the
+        # public call and reads its output back.  The layers of a step are independent calls, so their copies run on
+        # two copy streams beside the compute stream (input of the next layer and output of the previous one overlap
+        # the current layer's kernels); the layer with the largest output goes first.  A step ends when every output
+        # is in host memory.
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        order = sorted(wl.layers, key=lambda L: -L["y"].numel())
+
+        def step_e2e(i, capturing=False):
+            k = i % wl.n_sets
+            main_s = torch.cuda.current_stream()
+            s_in.wait_stream(main_s)    # earlier work on the staging buffers is done (previous steps were synchronized)
+            for L in order:
+                with torch.cuda.stream(s_in):
+                    L["x_stage"].copy_(L["x_host"], non_blocking=True)       # host -> device, pinned
+                    L["ev_in"] = s_in.record_event()
+            for L in order:
+                wc, ws = L["w_sets"][k]
+                main_s.wait_event(L["ev_in"])
+                rq.resq_linear(L["x_stage"], wc, ws, wl.pattern, wl.fmt, Y=L["y"], workspace=L["work"])
+                ev = main_s.record_event()
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev)
+                    L["y_host"].copy_(L["y"], non_blocking=True)             # device -> host
+            if capturing:
+                main_s.wait_stream(s_out)   # join the copy branches into the captured stream
+            else:
+                s_out.synchronize()
+                main_s.synchronize()
+
+        for i in range(3):
+            step_e2e(i)
+        run = step_e2e
+        if use_graph:
+            graphs = []
+            wl.build_graphs(lambda k: step_e2e(k, capturing=True), into=graphs)
+
+            def run(i):
+                graphs[i % wl.n_sets].replay()       # copies in, kernels and copies out: one graph launch per step
+                torch.cuda.current_stream().synchronize()
+            for i in range(3):
+                run(i)
+        for L in wl.layers:  # the pipelined copies delivered what the device holds
+            if not torch.equal(L["y_host"], L["y"].cpu()) or not torch.equal(L["x_stage"].cpu(), L["x_host"]):
+                raise RuntimeError(f"end-to-end step: host copy of layer {L['spec'].name} differs from the device tensor")
+        ms_e2e, _, _ = timed(run, steps)
+        h2d = sum(L["x_host"].numel() * 2 for L in wl.layers)
+        d2h = sum(L["y_host"].numel() * L["y_host"].element_size() for L in wl.layers)
+        return {"value": world * wl.flops_step / (ms_e2e / steps * 1e-3) / 1e12, "unit": "TFLOP/s",
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / steps}
+
+    def gemm_roofline(res, fmt_):
+        """Roofline object of the dominant kernel (the GEMM) from a measure() result."""
+        if "gemm_ms" not in res:
+            return None
+        tensor_peak, peak_src = tensor_peak_for(fmt_, res.get("clocks"))
+        # the event-bracketed durations are upper bounds; the step itself bounds them from above as well
+        gemm_ms = min(res["gemm_ms"] + res["reduce_ms"], res["ms_per_step"])
+        bracketed = res["gemm_ms"] + res["reduce_ms"] > res["ms_per_step"]
+        t = res["flops_step"] / (gemm_ms * 1e-3) / 1e12
+        return {"bound": "tensor", "achieved": t, "peak": tensor_peak, "unit": "TFLOP/s", "frac": t / tensor_peak,
+                "peak_source": peak_src,
+                "duration": "sum of the GEMM launches of a step, CUDA events around every launch" +
+                            (" (exceeded the graph-replayed step: the whole step time is used, an upper bound)" if bracketed else ""),
+                "gemm_ms_per_step": gemm_ms, "launches_per_step": res["gemm_launches"],
+                "avg_launch_us": gemm_ms * 1e3 / max(1, res["gemm_launches"]),
+                "quantizer_avg_launch_us": res["quant_ms"] * 1e3 / max(1, res["quant_launches"]),
+                "quantizer_share_of_kernel_time": res["quant_ms"] / max(1e-9, res["kernel_ms"]),
+                "select_share_of_kernel_time": res["select_ms"] / max(1e-9, res["kernel_ms"]),
+                "hbm_frac_of_step": res["gbs"] / world / peaks["hbm_gbs"],
+                "frac_of_bf16_burst": t / (peaks["bf16_tflops"] * (4.0 if fmt_ == "mxfp4" else 1.0)),
+                "frac_of_fp8_nominal": t / 4500.0, "frac_of_fp4_nominal": t / 9000.0}
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
         sampler.start()
         time.sleep(0.25)
-    launches0 = rq.kernel_launches()
-    step(0)
-    launches_per_step = rq.kernel_launches() - launches0
-    use_graph = not args.no_graph
-    if use_graph:
-        build_graphs()
-        for i in range(3):
-            step_graph(i)
-    run_step = step_graph if use_graph else step
+
+    # ---- headline workload
+    head = measure(cfg, pattern, fmt, args.steps, sampler=sampler, e2e=not args.skip_e2e, verbose=args.verbose)
+    config_desc["l2"] = head["l2"]
     config_desc["launch"] = "one CUDA graph replay per step" if use_graph else "eager launches"
-    ms, t0, t1 = timed(run_step, args.steps)
-    launches = launches_per_step * args.steps
-    # keep the GPU busy a little longer so that the 100 ms sampler certainly sees the loaded state
-    t_load0 = time.time()
-    reps = 0
-    while time.time() - t_load0 < 0.6:
-        for i in range(20):
-            run_step(i)
-        torch.cuda.synchronize()
-        reps += 1
-    t_load1 = time.time()
-    clocks = sampler.stop(t0, t_load1) if rank == 0 else None
-
-    flops_step = sum(layer_flops(cfg.M, L["spec"].N, L["spec"].K, pattern) for L in layers)
-    bytes_step = sum(layer_bytes(cfg.M, L["spec"].N, L["spec"].K, pattern, fmt) for L in layers)
-    ms_per_step = ms / args.steps
-    tflops = world * flops_step / (ms_per_step * 1e-3) / 1e12
-    gbs = world * bytes_step / (ms_per_step * 1e-3) / 1e9
-
-    if args.verbose and rank == 0:
-        per_layer_table()
     if args.skip_e2e:
         if rank == 0:
-            print(json.dumps({"metric": METRIC, "value": tflops, "unit": "TFLOP/s", "ms_per_step": ms_per_step,
+            print(json.dumps({"metric": METRIC, "value": head["tflops"], "unit": "TFLOP/s", "ms_per_step": head["ms_per_step"],
                               "config": config_desc, "note": "profiling aid run: no e2e / roofline passes"}))
+        if sampler:
+            sampler.stop()
         return
-    # ---- end-to-end: host buffers, copies inside the timed region
-    for i in range(3):
-        step_e2e(i)
-    run_e2e = step_e2e
-    if use_graph:
-        build_e2e_graphs()
-        run_e2e = step_e2e_graph
-        for i in range(3):
-            run_e2e(i)
-    for L in layers:  # the pipelined copies delivered what the device holds
-        if not torch.equal(L["y_host"], L["y"].cpu()) or not torch.equal(L["x_stage"].cpu(), L["x_host"]):
-            raise RuntimeError(f"end-to-end step: host copy of layer {L['spec'].name} differs from the device tensor")
-    ms_e2e, _, _ = timed(run_e2e, args.steps)
-    if os.environ.get("RESQ_BENCH_E2E_BOTH"):  # aid: the eager-launch figure beside the graph one
-        ms_eager, _, _ = timed(step_e2e, args.steps)
-        print(f"e2e eager {ms_eager / args.steps:.4f} ms  graph {ms_e2e / args.steps:.4f} ms", file=sys.stderr)
-    e2e_tflops = world * flops_step / (ms_e2e / args.steps * 1e-3) / 1e12
-    h2d = sum(L["x_host"].numel() * 2 for L in layers)
-    d2h = sum(L["y_host"].numel() * L["y_host"].element_size() for L in layers)
-
-    # ---- per-kernel device time (CUDA events around every launch, on the launching stream)
-    rq.profile_enable(True)
-    rq.profile_read()
-    barrier()
-    for i in range(args.steps):
-        step(i)
-    torch.cuda.synchronize()
-    prof = rq.profile_read()
-    rq.profile_enable(False)
-    gemm_ms, gemm_n = prof["gemm"]
-    quant_ms, quant_n = prof["quantize"]
-    peaks, peak_kind = load_peaks()
-    gemm_tflops = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
+    roofline = gemm_roofline(head, fmt)
     if fmt == "mxfp4":
-        # block-scaled FP4 pipe: the measured bf16 peak times the nominal FP4 : bf16 ratio (9 : 2.25 PFLOP/s)
-        kernel_name = "gemm_mxfp4_native_kernel (tcgen05.mma kind::mxf4.block_scale on packed E2M1 codes; bf16 route for some layers)"
-        tensor_peak, peak_src = peaks["bf16_tflops"] * 4.0, f"bf16 burst ({peak_kind}) x 4 (nominal FP4 : bf16 ratio)"
+        roofline["kernel"] = "gemm_mxfp4_native_kernel (tcgen05.mma kind::mxf4.block_scale on packed E2M1 codes; bf16 route for some layers)"
     else:
-        kernel_name = "gemm_pair_kernel (tcgen05.mma cta_group::2 kind::f16 on in-kernel bf16-expanded 4-bit weights)"
-        tensor_peak, peak_src = peaks["bf16_tflops"], f"bf16 burst, {peak_kind}"
-    roofline = {
-        "kernel": kernel_name,
-        "bound": "tensor",
-        "achieved": gemm_tflops, "peak": tensor_peak, "unit": "TFLOP/s",
-        "frac": (gemm_tflops / tensor_peak) if gemm_tflops else None,
-        "peak_source": peak_src, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.config, pattern, fmt)),
-        "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum, mean over the step's GEMM launches "
-                          "(profiles/gemm_pair_kernel_3b-decode_2to4.md); null for workloads not captured",
-        "avg_launch_us": gemm_ms * 1e3 / max(1, gemm_n), "launches": gemm_n,
-        "quantizer_avg_launch_us": quant_ms * 1e3 / max(1, quant_n),
-        "quantizer_share_of_kernel_time": quant_ms / max(1e-9, sum(v[0] for v in prof.values())),
-        "hbm_frac_of_step": gbs / world / peaks["hbm_gbs"],
-        "frac_of_fp8_nominal": (gemm_tflops / 4500.0) if gemm_tflops else None,
-        "frac_of_fp4_nominal": (gemm_tflops / 9000.0) if gemm_tflops else None,
-    }
+        roofline["kernel"] = "gemm_pair_kernel (tcgen05.mma cta_group::2 kind::f16 on in-kernel bf16-expanded 4-bit weights)"
+    dom = max(head["per_layer"], key=lambda r: r["gemm_us"])
+    tr = NCU_TRAFFIC.get((args.config, dom["layer"], pattern, fmt)) if not subset else None
+    roofline["traffic"] = tr["bytes"] if tr else None
+    roofline["traffic_source"] = (tr["source"] if tr else "no ncu capture of this workload's dominant launch") + \
+        f"; dominant launch: {dom['layer']}, algorithmic bytes {gemm_bytes(cfg.M, dom['N'], dom['K'], pattern, fmt):.4g}"
+    roofline["per_layer"] = head["per_layer"]
+
+    extras = {}
+    if rank == 0 and world == 1 and not args.headline_only and not subset:
+        n_small = max(10, min(args.steps, 20))
+        # ---- the other configurations with their named patterns (configs 0-3; the headline is config 4)
+        per_config = []
+        for ci in range(len(CONFIGS)):
+            if ci == args.config:
+                continue
+            c = CONFIGS[ci]
+            r = measure(c, c.patterns[0], "hif4", n_small, sampler=sampler)
+            rf = gemm_roofline(r, "hif4")
+            per_config.append({"config": ci, "name": c.name, "M": c.M, "pattern": PATTERN_NAMES[c.patterns[0]], "format": "hif4",
+                               "ms_per_step": r["ms_per_step"], "tflops": r["tflops"], "gb_per_s": r["gbs"],
+                               "gemm_frac_of_peak": rf["frac"], "peak_source": rf["peak_source"],
+                               "quantizer_share": rf["quantizer_share_of_kernel_time"], "select_share": rf["select_share_of_kernel_time"],
+                               "launches_per_step": r["launches_per_step"], "clocks": r["clocks"], "per_layer": r["per_layer"]})
+        extras["per_config"] = per_config
+        # ---- residual patterns and the MXFP4 twin on the headline workload
+        per_pattern = []
+        for name, f in (("none", "hif4"), ("dense", "hif4"), ("row50", "hif4"), ("chan50", "hif4"), ("block", "hif4"),
+                        ("2:4", "mxfp4"), ("dense", "mxfp4")):
+            if PATTERN_IDS[name] == pattern and f == fmt:
+                continue
+            r = measure(cfg, PATTERN_IDS[name], f, max(3, min(args.steps, 5)), sampler=sampler)
+            rf = gemm_roofline(r, f)
+            per_pattern.append({"pattern": name, "format": f, "ms_per_step": r["ms_per_step"], "tflops": r["tflops"],
+                                "gemm_ms_per_step": rf["gemm_ms_per_step"], "gemm_frac_of_peak": rf["frac"],
+                                "peak_source": rf["peak_source"], "quant_ms": r["quant_ms"], "select_ms": r["select_ms"]})
+        extras["per_pattern"] = per_pattern
+        none = next((p for p in per_pattern if p["pattern"] == "none" and p["format"] == fmt), None)
+        if none:
+            extras["residual_overhead_over_plain"] = {
+                "whole_step": head["ms_per_step"] / none["ms_per_step"] - 1.0,
+                "gemm_only": roofline["gemm_ms_per_step"] / none["gemm_ms_per_step"] - 1.0, "pattern": pattern_name}
+        # ---- true decode: M = 16 ... 128 on the 3B layers, where weight streaming from HBM is the roof
+        sweep = []
+        c1 = CONFIGS[1]
+        for M in (16, 32, 64, 128, 256):
+            cM = dataclasses.replace(c1, M=M, name=f"{c1.name} M={M}")
+            r = measure(cM, PATTERN_IDS["2:4"], "hif4", n_small)
+            sweep.append({"M": M, "us_per_step": r["ms_per_step"] * 1e3, "tflops": r["tflops"], "gb_per_s": r["gbs"],
+                          "frac_of_hbm": r["gbs"] / peaks["hbm_gbs"], "launches_per_step": r["launches_per_step"]})
+        extras["decode_sweep"] = {"workload": "config 1 layers, S_2:4, HiF4; algorithmic bytes = bf16 X + packed W + bf16 Y",
+                                  "hbm_peak_gbs": peaks["hbm_gbs"], "points": sweep}
+        # ---- quantizer alone
+        bpe, rows = quantizer_sweep("hif4", (256, 1024, 4096, 16384, 32768), args.verbose)
+        extras["quantizer_sweep"] = {"kernel": "hif4_quantize_act", "bytes_per_element": bpe, "hbm_peak_gbs": peaks["hbm_gbs"],
+                                     "best": max(rows, key=lambda r: r["GB/s"]), "worst": min(rows, key=lambda r: r["GB/s"]),
+                                     "points": rows}
+    if sampler:
+        sampler.stop()
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, cores, sample, dt = time_oracle(cfg, pattern, fmt)
+        rows, tensors = oracle_sample(cfg, budget_s=20.0)
+        v, cores, sample, dt = time_oracle(cfg, pattern, fmt, rows, tensors)
         cpu_baseline = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample,
                         "seconds": dt}
 
     if rank == 0:
         line = {
-            "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "metric": METRIC, "value": head["tflops"], "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if fmt == "hif4" else "fp4 (e2m1, ue8m0 block scales) / bf16",
             "data": "synthetic", "config": config_desc,
-            "gb_per_s": gbs, "clocks": clocks,
-            "e2e": {"value": e2e_tflops, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": ms_e2e / args.steps},
-            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "gb_per_s": head["gbs"], "clocks": head["clocks"], "e2e": head["e2e"],
+            "gpu_launches": int(head["launches_per_step"] * args.steps), "roofline": roofline, "cpu_baseline": cpu_baseline,
         }
+        line.update(extras)
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()

@@ -12,7 +12,11 @@
  * Conventions for every call
  *   - All tensor pointers are DEVICE pointers (the library never touches host data); row-major;
  *     `ld*` is the row stride in ELEMENTS of the pointed-to type.  bf16 inputs must be 16-byte
- *     aligned with ld a multiple of 8.  Packed outputs are dense (no stride).
+ *     aligned with ld a multiple of 8.  Packed outputs are dense (no stride); codes, metadata and
+ *     scale outputs must be 4-byte aligned (they are written with 32-bit / 16-bit stores), mask_bits
+ *     may start at any byte.  A misaligned pointer is RESQ_ERR_ALIGN, found on the host.
+ *   - The RESQ_* environment variables are debugging overrides of the kernel choices; they are read only
+ *     when RESQ_DEBUG is set to a non-zero value at the library's first call, otherwise never.
  *   - The caller owns every buffer; the library allocates no device memory.  Scratch comes from
  *     the `workspace` argument, sized by the matching *_workspace_bytes query (256-byte aligned).
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream).
@@ -132,13 +136,13 @@ RESQ_API int mxfp4_residual_mask(const void* X_bf16, int64_t M, int64_t K, int64
 /* ---- the same pass for callers that cannot allocate device memory (the paper has no counterpart) ----
  * Meant for hosts that cannot give the library a workspace: a server that handed all device memory to its
  * own pool at start-up, a plugin invoked inside a serving loop where an allocation would stall the device,
- * or a foreign-function caller that owns only its inputs and outputs.  Same inputs, outputs, patterns and
- * results as resq_residual_mask (HiF4), but the scratch of the channel-wise and block-wise selections lives
+ * or a foreign-function caller that owns only its inputs and outputs.  Same inputs, outputs, patterns (the
+ * RESQ_KEEP_QUARTERS and RESQ_BLOCK_PER_STRIP modifiers included) and results as resq_residual_mask (HiF4), but the scratch of the channel-wise and block-wise selections lives
  * in a fixed device array inside the library image (about 290 KB, held by every GPU that loads the
  * library until the process exits).  The call performs no cudaMalloc / cudaFree and uses no allocating
  * library routine.
  *   - Limit: at most RESQ_STATIC_SCRATCH_MAX_SCORES selection scores, i.e. K for RESQ_S_CHAN50 and
- *     (M/32)*(K/64) for RESQ_S_BLOCK32x64_50; larger problems return RESQ_ERR_WORKSPACE with a message
+ *     (M/32)*(K/64) for RESQ_S_BLOCK32x64_50 (with or without RESQ_BLOCK_PER_STRIP); larger problems return RESQ_ERR_WORKSPACE with a message
  *     (the other patterns need no scores and have no limit).
  *   - The first call on each device looks up the array's device address (with that device current); make
  *     that first call before starting any stream capture.
@@ -290,8 +294,15 @@ RESQ_API const char* resq_last_error(void);
  * resq_profile_read: synchronizes on the recorded events, adds the device time (ms) and the number of
  * launches per kernel kind into the two arrays of 4 entries (0 = quantizer/residual/mask pass,
  * 1 = top-k select and mask apply, 2 = GEMM, 3 = split-K reduce; either array may be NULL) and
- * clears the records. */
+ * clears the records.
+ * resq_debug_expire_next_wait(1): test hook for the RESQ_ERR_TIMEOUT path.  The next decode-sized GEMM launch of
+ * the process (K-streamed schedule: M > 128 and few output tiles) waits at its end for one partial tile more than
+ * its CTAs can deliver, with a poll limit of about a millisecond: the bounded wait runs out, the kernel records
+ * RESQ_ERR_TIMEOUT in the status word, leaves through its normal exit (tensor memory freed, no output for the
+ * tiles it was summing) and the context stays usable; resq_check then returns RESQ_ERR_TIMEOUT and the next call
+ * on the same workspace is an ordinary one.  Nothing faults or hangs.  (0 withdraws an unconsumed request.) */
 RESQ_API int64_t resq_kernel_launches(void);
+RESQ_API int resq_debug_expire_next_wait(int on);
 RESQ_API int resq_profile_enable(int on);
 RESQ_API int resq_profile_read(double* ms_by_kind, int64_t* launches_by_kind);
 

@@ -63,6 +63,7 @@ SYMBOLS = {
     "resq_check": (_ci, [_vp, _vp]),
     "resq_last_error": (ctypes.c_char_p, []),
     "resq_kernel_launches": (_i64, []),
+    "resq_debug_expire_next_wait": (_ci, [_ci]),
     "resq_profile_enable": (_ci, [_ci]),
     "resq_profile_read": (_ci, [_vp, _vp]),
 }
@@ -404,6 +405,11 @@ KERNEL_KINDS = ("quantize", "select", "gemm", "splitk_reduce")
 def kernel_launches() -> int:
     """resq_kernel_launches: kernels launched by the library in this process so far."""
     return int(lib().resq_kernel_launches())
+
+
+def debug_expire_next_wait(on: bool = True) -> None:
+    """resq_debug_expire_next_wait: the next decode-sized GEMM launch lets its bounded wait run out (test hook)."""
+    _check(lib().resq_debug_expire_next_wait(1 if on else 0))
 
 
 def profile_enable(on: bool) -> None:

@@ -8,7 +8,10 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <mutex>
+#include <tuple>
+#include <utility>
 #include <vector>
 
 namespace resq {
@@ -40,11 +43,77 @@ std::mutex g_prof_mu;
 std::vector<ProfRec*> g_prof;
 }  // namespace
 
-bool pdl_enabled() {
-    static const int on = [] {
-        const char* v = getenv("RESQ_PDL");
-        return (v && *v) ? atoi(v) : 1;
+bool debug_overrides() {
+    static const bool on = [] {
+        const char* v = getenv("RESQ_DEBUG");
+        return v && *v && *v != '0';
     }();
+    return on;
+}
+int env_int(const char* name, int dflt) {
+    if (!debug_overrides()) return dflt;
+    const char* v = getenv(name);
+    return v && *v ? atoi(v) : dflt;
+}
+bool env_is_zero(const char* name) {
+    if (!debug_overrides()) return false;
+    const char* v = getenv(name);
+    return v && *v == '0';
+}
+
+int device_sm_count() {
+    constexpr int kMaxDev = 64;
+    static std::mutex mu;
+    static int sms[kMaxDev] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return 148;
+    std::lock_guard<std::mutex> lk(mu);
+    if (sms[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        sms[dev] = n;
+    }
+    return sms[dev];
+}
+
+namespace {
+std::mutex g_dev_mu;
+std::map<std::pair<int, const void*>, int> g_smem_opt_in;                    // (device, function) -> bytes set
+std::map<std::tuple<int, const void*, size_t>, int> g_max_clusters;         // (device, function, smem) -> clusters
+}  // namespace
+
+int ensure_dynamic_smem(const void* func, int bytes, const char* what) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    std::lock_guard<std::mutex> lk(g_dev_mu);
+    int& have = g_smem_opt_in[std::make_pair(dev, func)];
+    if (have >= bytes) return RESQ_OK;
+    e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return cuda_fail(e, what);
+    have = bytes;
+    return RESQ_OK;
+}
+
+int max_active_clusters(const void* func, const cudaLaunchConfig_t* cfg, int* out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    std::lock_guard<std::mutex> lk(g_dev_mu);
+    const auto key = std::make_tuple(dev, func, cfg->dynamicSmemBytes);
+    auto it = g_max_clusters.find(key);
+    if (it == g_max_clusters.end()) {
+        int n = 0;
+        e = cudaOccupancyMaxActiveClusters(&n, func, cfg);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaOccupancyMaxActiveClusters");
+        it = g_max_clusters.emplace(key, n).first;
+    }
+    *out = it->second;
+    return RESQ_OK;
+}
+
+bool pdl_enabled() {
+    static const int on = env_int("RESQ_PDL", 1);
     // event records between the kernels (profiling) would serialize them anyway
     return on != 0 && !g_profile.load(std::memory_order_relaxed);
 }
@@ -66,6 +135,50 @@ LaunchScope::~LaunchScope() {
     cudaEventRecord(r->stop, stream_);
     std::lock_guard<std::mutex> lk(g_prof_mu);
     g_prof.push_back(r);
+}
+
+// A pattern argument is a base pattern, optionally combined with RESQ_KEEP_QUARTERS(q): splits it in place.
+int split_pattern(int* pattern, int* quarters, int* per_strip) {
+    const int q = (*pattern >> 8) & 0xF;
+    const int strip = (*pattern >> 12) & 1;
+    if (*pattern < 0 || (*pattern >> 13) != 0 || q > 3) {
+        set_last_error("unknown pattern %d", *pattern);
+        return RESQ_ERR_PATTERN;
+    }
+    *quarters = q == 0 ? 2 : q;
+    *per_strip = strip;
+    *pattern &= 0xFF;
+    if (q != 0 && (*pattern == RESQ_S_NONE || *pattern == RESQ_S_DENSE)) {
+        set_last_error("RESQ_KEEP_QUARTERS applies to the selecting patterns only");
+        return RESQ_ERR_PATTERN;
+    }
+    if (strip && *pattern != RESQ_S_BLOCK32x64_50) {
+        set_last_error("RESQ_BLOCK_PER_STRIP applies to RESQ_S_BLOCK32x64_50 only");
+        return RESQ_ERR_PATTERN;
+    }
+    return RESQ_OK;
+}
+int check_pattern(int pattern, int64_t M) {
+    if (pattern < RESQ_S_NONE || pattern > RESQ_S_BLOCK32x64_50) {
+        set_last_error("unknown pattern %d", pattern);
+        return RESQ_ERR_PATTERN;
+    }
+    if (pattern == RESQ_S_BLOCK32x64_50 && M % kBlkRows != 0) {
+        set_last_error("the 32x64 block pattern needs M %% 32 == 0 (M=%lld)", (long long)M);
+        return RESQ_ERR_SHAPE;
+    }
+    return RESQ_OK;
+}
+
+int check_packed_outputs(const void* x_codes, const void* x_side, const void* r_codes, const void* r_side) {
+    const void* ptrs[4] = {x_codes, x_side, r_codes, r_side};
+    const char* names[4] = {"x_codes", "x_meta / x_scale", "r_codes", "r_meta / r_scale"};
+    for (int i = 0; i < 4; ++i)
+        if (ptrs[i] && (reinterpret_cast<uintptr_t>(ptrs[i]) & 3u) != 0) {
+            set_last_error("%s must be 4-byte aligned (%p)", names[i], ptrs[i]);
+            return RESQ_ERR_ALIGN;
+        }
+    return RESQ_OK;
 }
 
 namespace {
@@ -90,40 +203,7 @@ int check_matrix(const void* p, int64_t rows, int64_t K, int64_t ld, int fmt, co
     return RESQ_OK;
 }
 
-// A pattern argument is a base pattern, optionally combined with RESQ_KEEP_QUARTERS(q): splits it in place.
-int split_pattern(int* pattern, int* quarters, int* per_strip) {
-    const int q = (*pattern >> 8) & 0xF;
-    const int strip = (*pattern >> 12) & 1;
-    if (*pattern < 0 || (*pattern >> 13) != 0 || q > 3) {
-        set_last_error("unknown pattern %d", *pattern);
-        return RESQ_ERR_PATTERN;
-    }
-    *quarters = q == 0 ? 2 : q;
-    *per_strip = strip;
-    *pattern &= 0xFF;
-    if (q != 0 && (*pattern == RESQ_S_NONE || *pattern == RESQ_S_DENSE)) {
-        set_last_error("RESQ_KEEP_QUARTERS applies to the selecting patterns only");
-        return RESQ_ERR_PATTERN;
-    }
-    if (strip && *pattern != RESQ_S_BLOCK32x64_50) {
-        set_last_error("RESQ_BLOCK_PER_STRIP applies to RESQ_S_BLOCK32x64_50 only");
-        return RESQ_ERR_PATTERN;
-    }
-    return RESQ_OK;
-}
 int base_pattern(int pattern) { return pattern < 0 ? pattern : pattern & 0xFF; }
-
-int check_pattern(int pattern, int64_t M) {
-    if (pattern < RESQ_S_NONE || pattern > RESQ_S_BLOCK32x64_50) {
-        set_last_error("unknown pattern %d", pattern);
-        return RESQ_ERR_PATTERN;
-    }
-    if (pattern == RESQ_S_BLOCK32x64_50 && M % kBlkRows != 0) {
-        set_last_error("the 32x64 block pattern needs M %% 32 == 0 (M=%lld)", (long long)M);
-        return RESQ_ERR_SHAPE;
-    }
-    return RESQ_OK;
-}
 
 int check_workspace(const void* ws, size_t have, size_t need) {
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || have < need) {
@@ -141,6 +221,8 @@ int quantize_only(int fmt, const void* X, int64_t rows, int64_t K, int64_t ld, v
         set_last_error("%s: output pointer is NULL", name);
         return RESQ_ERR_NULL;
     }
+    rc = check_packed_outputs(codes, side, nullptr, nullptr);
+    if (rc) return rc;
     QuantArgs a;
     memset(&a, 0, sizeof(a));
     a.X = static_cast<const __nv_bfloat16*>(X);
@@ -200,6 +282,8 @@ int residual_mask(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, int
     rc = split_pattern(&pattern, &quarters, &per_strip);
     if (rc) return rc;
     rc = check_pattern(pattern, M);
+    if (rc) return rc;
+    rc = check_packed_outputs(x_codes, x_side, r_codes, r_side);
     if (rc) return rc;
     rc = check_workspace(workspace, ws_bytes, resq_residual_mask_workspace_bytes(M, K, pattern));
     if (rc) return rc;
@@ -700,6 +784,11 @@ int resq_check(void* workspace, void* stream) {
 }
 
 const char* resq_last_error(void) { return g_last_error; }
+
+int resq_debug_expire_next_wait(int on) {
+    debug_expire_next_wait(on);
+    return RESQ_OK;
+}
 
 int64_t resq_kernel_launches(void) { return (int64_t)g_launches.load(); }
 

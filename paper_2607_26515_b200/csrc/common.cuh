@@ -31,6 +31,27 @@ struct DeviceStatus {
 void set_last_error(const char* fmt, ...);
 int cuda_fail(cudaError_t e, const char* what);
 
+// Debugging overrides (tile widths, schedules, kernel choices: the RESQ_* variables the tests use to reach every
+// variant) are honoured only when RESQ_DEBUG is set to a non-zero value in the environment at the library's first
+// call; otherwise no call reads the environment and every override has its default.
+bool debug_overrides();
+int env_int(const char* name, int dflt);       // the variable's integer value if overrides are on and it is set
+bool env_is_zero(const char* name);            // overrides on and the variable starts with '0'
+
+// Per-device facts the launchers need (looked up once per device, under a mutex).
+int device_sm_count();                         // of the current device
+// Opts `func` into `bytes` of dynamic shared memory on the current device (once per device and function).
+int ensure_dynamic_smem(const void* func, int bytes, const char* what);
+// cudaOccupancyMaxActiveClusters of `func` under `cfg`, cached per device, function and shared-memory size.
+int max_active_clusters(const void* func, const cudaLaunchConfig_t* cfg, int* out);
+
+// Argument checks shared by the entry points (api.cu).
+int split_pattern(int* pattern, int* quarters, int* per_strip);  // strips RESQ_KEEP_QUARTERS / RESQ_BLOCK_PER_STRIP
+int check_pattern(int base_pattern, int64_t M);
+// Packed outputs are written with 32-bit stores (codes, HiF4 metadata) or 16-bit stores (MXFP4 scales): every
+// non-null packed output must be 4-byte aligned, else RESQ_ERR_ALIGN.
+int check_packed_outputs(const void* x_codes, const void* x_side, const void* r_codes, const void* r_side);
+
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Diagnostics (api.cu): every kernel launch of the library is counted; when profiling is enabled a
@@ -150,6 +171,8 @@ struct GemmArgs {
     DeviceStatus* status;
 };
 int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream);
+// Test hook behind resq_debug_expire_next_wait (gemm_pair.cu).
+void debug_expire_next_wait(int on);
 // Whether launch_gemm_hif4 takes the compressed 2:4 residual for this shape (the CTA-pair kernel runs it).
 bool gemm_sparse24_supported(int64_t M, int64_t N, int64_t K);
 // Layout of the 2:4 index metadata, fixed by the sparse MMA: blocks of 128 rows x 128 K positions (2 KB, row bands

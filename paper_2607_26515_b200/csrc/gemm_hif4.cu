@@ -60,7 +60,9 @@ struct GemmParams {
     int64_t ldy;
     float* partials;          // [splits, M, N] when splits > 1
     DeviceStatus* status;
+#ifdef RESQ_TIMELINE
     int debug;                // bit 4 (16): accumulate per-role cycle counters after the status word
+#endif
 };
 
 __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
@@ -70,13 +72,21 @@ __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
     }
 }
 
-// Debug aid: cycles spent per role, summed over CTAs into the 64-bit counters that follow the status word.
+// Profiling builds (-DRESQ_TIMELINE) only: cycles spent per role, summed over CTAs into the 64-bit counters that
+// follow the status word.  The shipped kernels carry no instrumentation.
+#ifdef RESQ_TIMELINE
 struct Trace {
     unsigned long long* out;
     long long t0;
     __device__ __forceinline__ void begin() { if (out) t0 = clock64(); }
     __device__ __forceinline__ void end(int slot) { if (out) atomicAdd(out + slot, (unsigned long long)(clock64() - t0)); }
 };
+#else
+struct Trace {
+    __device__ __forceinline__ void begin() {}
+    __device__ __forceinline__ void end(int) {}
+};
+#endif
 
 struct TileCoord {
     int64_t m0, n0;
@@ -147,8 +157,12 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+#ifdef RESQ_TIMELINE
     Trace tr{(p.debug & 16) ? reinterpret_cast<unsigned long long*>(p.status) + 8 : nullptr, 0};
     const long long t_kernel0 = clock64();
+#else
+    Trace tr;
+#endif
     // programmatic dependent launch: see gemm_pair.cu (the weight side does not depend on the quantizer)
     pdl_trigger();
     if (!(warp == 2 || warp >= kFirstExpWarp)) pdl_wait();
@@ -417,10 +431,12 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
     ptx::tc_fence_before();
     __syncthreads();
+#ifdef RESQ_TIMELINE
     if (tr.out && threadIdx.x == 0) {
         atomicAdd(tr.out + 11, (unsigned long long)(clock64() - t_kernel0));
         atomicAdd(tr.out + 12, 1ull);
     }
+#endif
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
@@ -526,11 +542,6 @@ struct TileChoice {
     int mt, bn, splits, nt;
     int pair_tn;  // > 0: use the CTA-pair kernel with a 256 x pair_tn tile
 };
-
-int env_int(const char* name, int dflt) {
-    const char* v = getenv(name);
-    return v && *v ? atoi(v) : dflt;
-}
 
 // Pick the tile width and K split so that the persistent grid covers the 148 SMs evenly.
 // Calls with at most this many rows take the single-CTA kernel (one 128-row MMA tile); the CTA-pair kernel computes
@@ -668,21 +679,13 @@ int launch_variant(const GemmArgs& g, const TileChoice& tc, cudaStream_t stream)
     p.ldy = g.ldy;
     p.partials = g.splitk_partials;
     p.status = g.status;
+#ifdef RESQ_TIMELINE
     p.debug = env_int("RESQ_GEMM_DEBUG", 0);
+#endif
     auto kern = gemm_hif4_kernel<MT, RES, TN, FMT>;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-    });
-    if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute(gemm)");
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-        if (num_sms <= 0) num_sms = 148;
-    }
+    rc = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), kSmemBudget, "cudaFuncSetAttribute(gemm)");
+    if (rc) return rc;
+    const int num_sms = device_sm_count();
     const unsigned grid = (unsigned)std::min(p.num_tiles, num_sms);
     {
         LaunchScope scope(kKindGemm, stream);

@@ -377,17 +377,9 @@ int launch_native_variant(const Mxfp4NativeArgs& g, cudaStream_t stream) {
     const int smem_bytes = 1024 + L::kStagesN * L::kBytes + 256;
     static_assert(1024 + L::kStagesN * L::kBytes + 256 <= kSmemBudgetNative, "stages do not fit");
     auto kern = gemm_mxfp4_native_kernel<RES>;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes); });
-    if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute(gemm mxfp4)");
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-        if (num_sms <= 0) num_sms = 148;
-    }
+    rc = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem_bytes, "cudaFuncSetAttribute(gemm mxfp4)");
+    if (rc) return rc;
+    const int num_sms = device_sm_count();
     const unsigned grid = (unsigned)std::min(p.num_tiles, num_sms);
     LaunchScope scope(kKindGemm, stream);
     return cuda_fail(launch_kernel(kern, dim3(grid), dim3(kThreadsNative), (size_t)smem_bytes, stream, ta, tr, tw, p),
@@ -398,8 +390,7 @@ int launch_native_variant(const Mxfp4NativeArgs& g, cudaStream_t stream) {
 
 bool gemm_mxfp4_native_supported(int64_t M, int64_t N, int64_t K, bool res) {
     // RESQ_MXFP4_NATIVE: debugging override (0: never, 1: whenever the shape allows, unset: when it pays)
-    const char* v = getenv("RESQ_MXFP4_NATIVE");
-    const int mode = (v && *v) ? atoi(v) : -1;
+    const int mode = env_int("RESQ_MXFP4_NATIVE", -1);
     if (mode == 0 || K % kBKe != 0) return false;
     if (mode == 1) return true;
     // No K split here: a CTA walks the whole K range of its tiles, about 1.1 us per 256 values of K.  The bf16

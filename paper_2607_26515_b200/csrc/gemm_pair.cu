@@ -19,6 +19,7 @@
 #include "expand.cuh"
 
 #include <algorithm>
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -56,9 +57,11 @@ struct PairParams {
     int64_t ldy;
     float* partials;
     DeviceStatus* status;
+#ifdef RESQ_TIMELINE
     int debug;
-    unsigned int* timeline;  // debug: device buffer for a per-role event log of pair 0 (or null)
-    int timeline_first;      // debug: first k-block iteration that is logged
+    unsigned int* timeline;  // device buffer for a per-role event log of pair 0 (or null)
+    int timeline_first;      // first k-block iteration that is logged
+#endif
     // K-streamed schedule (streamk != 0): the num_tiles * G (tile, k-block) units are dealt out evenly to the
     // pairs; a pair's first and last segment may cover only part of a tile's K range and then go to fp32 slots
     int streamk;
@@ -68,6 +71,8 @@ struct PairParams {
     int sk_pairs;            // pairs 0 .. sk_pairs-1 share the dealt-out units (at least two k-blocks each)
     float* sk_slots;         // [2 * npairs][256][TN] fp32: slot 2p = first segment of pair p, 2p + 1 = its last
     unsigned int* sk_flags;  // [num_tiles][2]: segments of the tile written, per CTA rank (zeroed before launch)
+    int sk_poll_limit;       // polls (about 0.3 us each) before the wait for a tile's segments gives up
+    int sk_extra;            // test hook (resq_debug_expire_next_wait): arrivals awaited beyond those that can come
 };
 
 __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
@@ -77,12 +82,21 @@ __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
     }
 }
 
+// In-kernel instrumentation (cycle counters per role, an event log of pair 0) exists only in builds with
+// -DRESQ_TIMELINE, which the profiling experiments use; the shipped kernels carry none of it.
+#ifdef RESQ_TIMELINE
 struct Trace {
     unsigned long long* out;
     long long t0;
     __device__ __forceinline__ void begin() { if (out) t0 = clock64(); }
     __device__ __forceinline__ void end(int slot) { if (out) atomicAdd(out + slot, (unsigned long long)(clock64() - t0)); }
 };
+#else
+struct Trace {
+    __device__ __forceinline__ void begin() {}
+    __device__ __forceinline__ void end(int) {}
+};
+#endif
 
 struct TileCoord {
     int64_t m0, n0;
@@ -204,9 +218,9 @@ __device__ __forceinline__ void streamk_fixup(const PairParams& p, int pair, int
         if (threadIdx.x == 0) {
             int ok = *abort_flag ? 0 : 1;
             const unsigned int* flag = p.sk_flags + t * 2 + rank;
-            for (int polls = 0; ok && ld_acquire_u32(flag) < (unsigned)nseg; ++polls) {
+            for (int polls = 0; ok && ld_acquire_u32(flag) < (unsigned)(nseg + p.sk_extra); ++polls) {
                 __nanosleep(200);
-                if (polls > (1 << 20)) {
+                if (polls > p.sk_poll_limit) {
                     report_timeout(p.status, 7);
                     ok = 0;
                 }
@@ -310,13 +324,17 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     uint64_t* acc_empty = acc_full + 2;        // [2] leader: both epilogues drained
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+#ifdef RESQ_TIMELINE
     unsigned int* tlog = reinterpret_cast<unsigned int*>(tmem_slot + 4);  // [8 roles][32 iterations] (512 B)
     const bool tl = p.timeline != nullptr && (blockIdx.x >> 1) == 0;
     const int kTl0 = p.timeline_first;  // first logged iteration
 #define EVT(k) do { if (tl) p.timeline[512 + (int)rank * 16 + (k)] = (unsigned int)(clock64() - t_kernel0); } while (0)
 #define TLOG(role, it) do { if (tl && (it) >= kTl0 && (it) < kTl0 + 32) tlog[(role) * 32 + ((it) - kTl0)] = (unsigned int)clock64(); } while (0)
-
     const long long t_entry = clock64();
+#else
+#define EVT(k) do { } while (0)
+#define TLOG(role, it) do { } while (0)
+#endif
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();  // 0 = leader
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
@@ -344,9 +362,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     ptx::cluster_sync();  // the peer's barriers exist before anything arrives on them
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+#ifdef RESQ_TIMELINE
     Trace tr{(p.debug & 16) ? reinterpret_cast<unsigned long long*>(p.status) + 8 : nullptr, 0};
     const long long t_kernel0 = clock64();
     if (tl && threadIdx.x == 0) p.timeline[512 + (int)rank * 16] = (unsigned int)(t_kernel0 - t_entry);
+#else
+    Trace tr;
+#endif
     // Programmatic dependent launch: the set-up above overlaps the tail of the quantizer kernel.  The weight side
     // (raw-code producer, expanders) reads only the packed weights, which no kernel since the start of the
     // quantizer writes, and starts at once; everything else waits for the quantizer's outputs.
@@ -721,26 +743,32 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     if (p.streamk) {
         if (threadIdx.x == 0) tr.begin();
         // the activation ring is idle by now: its first bytes hold the slot list of the tile being summed
+#ifdef RESQ_TIMELINE
         streamk_fixup<TN>(p, pair, npairs, (int)rank, abort_flag, reinterpret_cast<volatile int*>(tmem_slot + 2),
                           reinterpret_cast<int*>(ring_a), tl ? p.timeline + 512 + (int)rank * 16 + 8 : nullptr, t_kernel0);
+#else
+        streamk_fixup<TN>(p, pair, npairs, (int)rank, abort_flag, reinterpret_cast<volatile int*>(tmem_slot + 2),
+                          reinterpret_cast<int*>(ring_a), nullptr, 0);
+#endif
         if (threadIdx.x == 0) { tr.end(13); EVT(7); }
     }
+#ifdef RESQ_TIMELINE
     if (tl && threadIdx.x < 256) p.timeline[blockIdx.x * 256 + threadIdx.x] = tlog[threadIdx.x];
+#endif
     ptx::cluster_sync();  // no CTA leaves while the peer may still signal its barriers or read its shared memory
+#ifdef RESQ_TIMELINE
     if (tr.out && threadIdx.x == 0) {
         atomicAdd(tr.out + 11, (unsigned long long)(clock64() - t_kernel0));
         atomicAdd(tr.out + 12, 1ull);
     }
+#endif
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
     }
 }
 
-int env_int(const char* name, int dflt) {
-    const char* v = getenv(name);
-    return v && *v ? atoi(v) : dflt;
-}
+std::atomic<int> g_expire_next_wait{0};
 
 constexpr int kStreamKTN = 256;    // tile width of the K-streamed schedule (two accumulators fit in tensor memory)
 constexpr int kStreamKMaxPairs = 74;
@@ -801,32 +829,29 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
     p.sk_pairs = 0;
     p.sk_slots = g.splitk_partials;
     p.sk_flags = g.sk_flags;
+    p.sk_poll_limit = 1 << 20;
+    p.sk_extra = 0;
+    if (streamk && g_expire_next_wait.exchange(0)) {  // test hook: this launch's wait for the segments cannot be met
+        p.sk_poll_limit = 1 << 12;
+        p.sk_extra = 1;
+    }
     p.Y = g.Y;
     p.out_f32 = g.out_dtype == RESQ_OUT_F32;
     p.ldy = g.ldy;
     p.partials = g.splitk_partials;
     p.status = g.status;
+#ifdef RESQ_TIMELINE
     p.debug = env_int("RESQ_GEMM_DEBUG", 0);
     {
         const char* tp = getenv("RESQ_GEMM_TIMELINE_PTR");
         p.timeline = tp && *tp ? reinterpret_cast<unsigned int*>(strtoull(tp, nullptr, 0)) : nullptr;
         p.timeline_first = env_int("RESQ_GEMM_TIMELINE_FIRST", 96);
     }
+#endif
     auto kern = gemm_pair_kernel<RES, TN, FMT, NG>;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-    });
-    if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute(gemm pair)");
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-        if (num_sms <= 0) num_sms = 148;
-    }
-    const int max_pairs = num_sms / 2;
+    rc = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), kSmemBudget, "cudaFuncSetAttribute(gemm pair)");
+    if (rc) return rc;
+    const int max_pairs = device_sm_count() / 2;
     int npairs = std::min(p.num_tiles, max_pairs);
     if (streamk && (size_t)p.num_tiles * 2 * sizeof(unsigned int) > kWsFlags) {
         set_last_error("internal: %d output tiles exceed the arrival counters of the K-streamed schedule", p.num_tiles);
@@ -902,13 +927,9 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
     cfg.numAttrs = pdl_enabled() ? 2 : 1;
     cudaError_t e;
     if (streamk) {
-        static int max_clusters = -1;  // co-resident clusters of this variant
-        if (max_clusters < 0) {
-            int n = 0;
-            e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
-            if (e != cudaSuccess) return cuda_fail(e, "cudaOccupancyMaxActiveClusters(gemm pair)");
-            max_clusters = n;
-        }
+        int max_clusters = 0;  // co-resident clusters of this variant with this much shared memory
+        rc = max_active_clusters(reinterpret_cast<const void*>(kern), &cfg, &max_clusters);
+        if (rc) return rc;
         if (npairs > max_clusters) {
             npairs = max_clusters;
             cfg.gridDim = dim3((unsigned)(2 * npairs), 1, 1);
@@ -948,6 +969,8 @@ int dispatch_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
 }
 
 }  // namespace
+
+void debug_expire_next_wait(int on) { g_expire_next_wait.store(on ? 1 : 0); }
 
 size_t gemm_pair_streamk_scratch_bytes() {
     return (size_t)2 * kStreamKMaxPairs * (2 * kBM) * kStreamKTN * sizeof(float);

@@ -1443,16 +1443,10 @@ __global__ void __launch_bounds__(kThreads) dequant_kernel(const uint8_t* __rest
     o[1] = make_float4(v[4], v[5], v[6], v[7]);
 }
 
-bool getenv_is_zero(const char* name) {
-    const char* v = getenv(name);
-    return v && *v == '0';
-}
-
-// debugging override: RESQ_ROW50_TEAM=0 sends long rows to the older CTA-per-row kernel
-bool env_flag_row50_team() {
-    const char* v = getenv("RESQ_ROW50_TEAM");
-    return !(v && *v == '0');
-}
+// debugging overrides (honoured only under RESQ_DEBUG, see common.cuh)
+bool getenv_is_zero(const char* name) { return env_is_zero(name); }
+// RESQ_ROW50_TEAM=0 sends long rows to the older CTA-per-row kernel
+bool env_flag_row50_team() { return !env_is_zero("RESQ_ROW50_TEAM"); }
 
 int pick_rows_per_cta(int64_t M, int64_t K, int pattern) {
     // enough CTAs to fill 148 SMs several times over, but long enough row loops to amortize set-up
@@ -1736,8 +1730,8 @@ static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t
     const unsigned nsel = strips ? (unsigned)(a.M / kBlkRows) : 1u;
     if (strips) nscore = a.K / kBlkCols;
     const int keep = (int)(nscore * a.keep_quarters / 4);
-    const char* grid_env = getenv("RESQ_SEL_GRID");  // debugging override: 0 keeps the one-CTA selection
-    if (!strips && a.sel_hist && nscore > kSelGridMin && keep > 0 && keep < nscore && !(grid_env && *grid_env == '0')) {
+    // (debugging override RESQ_SEL_GRID=0 keeps the one-CTA selection)
+    if (!strips && a.sel_hist && nscore > kSelGridMin && keep > 0 && keep < nscore && !env_is_zero("RESQ_SEL_GRID")) {
         SelState* st = reinterpret_cast<SelState*>(a.sel_hist + 65536);
         const unsigned grid = (unsigned)std::min<int64_t>((nscore + 255) / 256, 148 * 4);
         {
@@ -1820,7 +1814,8 @@ int launch_quantize(int fmt, const QuantArgs& a_in, cudaStream_t stream) {
         const int nseg = (int)((a.K / kHif4Block + 31) / 32);
         const int per_warp = (3 + nseg) * kStageBytes;
         const int wpc = std::min(kWarpsPerCta, (220 * 1024) / per_warp);
-        const bool aligned = al16r(a.x_codes) && al16r(a.r_codes) && al16r(a.mask_bits) && al16r(a.a_bf16) && al16r(a.r_bf16);
+        const bool aligned = al16r(a.x_codes) && al16r(a.r_codes) && al16r(a.mask_bits) && al16r(a.x_side) && al16r(a.r_side) &&
+                             al16r(a.a_bf16) && al16r(a.r_bf16);
         const bool img = a.a_bf16 != nullptr;
         if (a.K % kHif4Block == 0 && nseg <= 2 && wpc >= 1 && a.M >= 148 && aligned) {
             void (*kern)(QuantArgs, int);
@@ -1885,7 +1880,7 @@ int launch_quantize(int fmt, const QuantArgs& a_in, cudaStream_t stream) {
     // (the chunk-per-lane kernel pays for CHAN50 with fp64 atomics per row and channel: the block kernel takes over earlier)
     const int64_t min_block_tasks = chan_from_image ? 148 : 148 * 16;
     if (!a.X_up && !a.gamma && !a.rht && (pattern != RESQ_S_CHAN50 || chan_from_image) && a.K % kHif4Block == 0 && block_tasks >= min_block_tasks && al16(a.x_codes) && al16(a.r_codes) && al16(a.mask_bits) &&
-        al16(a.a_bf16) && al16(a.r_bf16) && al16(a.r_comp)) {
+        al16(a.x_side) && al16(a.r_side) && al16(a.a_bf16) && al16(a.r_bf16) && al16(a.r_comp)) {
         const bool img = a.a_bf16 != nullptr;
         const int64_t ncg = (a.K / kHif4Block + 31) / 32;
         int rows_per_warp = 1;

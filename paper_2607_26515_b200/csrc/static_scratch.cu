@@ -64,14 +64,14 @@ extern "C" int resq_residual_mask_static(const void* X, int64_t M, int64_t K, in
         set_last_error("X: needs a 16-byte aligned base and ld >= K, ld %% 8 == 0 (ld=%lld)", (long long)ldx);
         return RESQ_ERR_ALIGN;
     }
-    if (pattern < RESQ_S_NONE || pattern > RESQ_S_BLOCK32x64_50) {
-        set_last_error("unknown pattern %d", pattern);
-        return RESQ_ERR_PATTERN;
-    }
-    if (pattern == RESQ_S_BLOCK32x64_50 && M % kBlkRows != 0) {
-        set_last_error("the 32x64 block pattern needs M %% 32 == 0 (M=%lld)", (long long)M);
-        return RESQ_ERR_SHAPE;
-    }
+    // the same pattern rules as resq_residual_mask: RESQ_KEEP_QUARTERS and RESQ_BLOCK_PER_STRIP are honoured
+    int quarters = 2, per_strip = 0;
+    int rc = split_pattern(&pattern, &quarters, &per_strip);
+    if (rc) return rc;
+    rc = check_pattern(pattern, M);
+    if (rc) return rc;
+    rc = check_packed_outputs(x_codes, x_meta, r_codes, r_meta);
+    if (rc) return rc;
     size_t nscores = 0;
     if (pattern == RESQ_S_CHAN50) nscores = (size_t)K;
     if (pattern == RESQ_S_BLOCK32x64_50) nscores = (size_t)(M / kBlkRows) * (size_t)(K / kBlkCols);
@@ -82,7 +82,7 @@ extern "C" int resq_residual_mask_static(const void* X, int64_t M, int64_t K, in
         return RESQ_ERR_WORKSPACE;
     }
     unsigned char* scratch = nullptr;
-    int rc = static_scratch_for_current_device(&scratch);
+    rc = static_scratch_for_current_device(&scratch);
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the array keeps whatever the previous call left: the status header is cleared here, the scores are
@@ -96,6 +96,8 @@ extern "C" int resq_residual_mask_static(const void* X, int64_t M, int64_t K, in
     a.K = K;
     a.ldx = ldx;
     a.pattern = pattern;
+    a.keep_quarters = quarters;
+    a.per_strip = per_strip;
     a.x_codes = static_cast<uint8_t*>(x_codes);
     a.x_side = x_meta;
     if (pattern != RESQ_S_NONE) {

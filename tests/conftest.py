@@ -6,6 +6,9 @@ import sys
 import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+# the library honours its RESQ_* debugging overrides (which the tests use to reach every kernel variant) only when
+# this is set before its first call
+os.environ.setdefault("RESQ_DEBUG", "1")
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 

@@ -80,6 +80,29 @@ def test_host_side_argument_errors_need_no_device(lib):
     for bad in (2 | (4 << 8), 0 | (1 << 8), 1 | (3 << 8), 2 | (1 << 12), 3 | (1 << 12), 4 | (1 << 12), 5 | (1 << 13), -1):
         assert lib.resq_residual_mask(fake, 32, 64, 64, bad, fake, fake, fake, fake, fake, fake, 1 << 20, None) == 5, bad
     assert lib.resq_residual_mask(fake, 40, 64, 64, 5 | (1 << 12), fake, fake, fake, fake, fake, fake, 1 << 20, None) == 2
+    # packed outputs are written with 32-bit / 16-bit stores: codes, metadata and scales must be 4-byte aligned
+    # (a sub-buffer at an odd offset is refused on the host, not found by a misaligned-address fault)
+    odd, half = ctypes.c_void_p(0x1001), ctypes.c_void_p(0x1002)
+    assert lib.hif4_quantize_act(fake, 4, 64, 64, odd, fake, None) == 3
+    assert lib.hif4_quantize_act(fake, 4, 64, 64, fake, half, None) == 3
+    assert b"4-byte aligned" in lib.resq_last_error()
+    lib.mxfp4_pack_weight.argtypes = [vp, i64, i64, i64, vp, vp, vp]
+    assert lib.mxfp4_pack_weight(fake, 4, 64, 64, fake, odd, None) == 3
+    for slot in range(4):    # x_codes, x_meta, r_codes, r_meta in turn
+        outs = [fake] * 4
+        outs[slot] = half
+        assert lib.resq_residual_mask(fake, 32, 64, 64, 2, *outs, fake, fake, 1 << 20, None) == 3, slot
+    lib.mxfp4_residual_mask.argtypes = lib.resq_residual_mask.argtypes
+    assert lib.mxfp4_residual_mask(fake, 32, 64, 64, 2, fake, odd, fake, fake, fake, fake, 1 << 20, None) == 3
+    lib.resq_residual_mask_static.argtypes = [vp, i64, i64, i64, ci, vp, vp, vp, vp, vp, vp]
+    assert lib.resq_residual_mask_static(fake, 32, 64, 64, 2, fake, fake, half, fake, fake, None) == 3
+    # the allocation-free variant takes the same pattern modifiers and refuses the same combinations
+    for bad in (2 | (4 << 8), 0 | (1 << 8), 2 | (1 << 12), 5 | (1 << 13), -1, 9):
+        assert lib.resq_residual_mask_static(fake, 32, 64, 64, bad, fake, fake, fake, fake, fake, None) == 5, bad
+    assert lib.resq_residual_mask_static(fake, 40, 64, 64, 5 | (1 << 12), fake, fake, fake, fake, fake, None) == 2
+    # its size limit (32768 scores) is checked on the host: one block column too many
+    assert lib.resq_residual_mask_static(fake, 32, 32768 + 64, 32768 + 64, 4, fake, fake, fake, fake, fake, None) == 4
+    assert b"32768" in lib.resq_last_error()
     lib.hif4_resq_linear.argtypes = [vp, i64, i64, i64, vp, vp, i64, ci, vp, ci, i64, vp, sz, vp]
     assert lib.hif4_resq_linear(fake, 32, 64, 64, fake, fake, 0, 0, fake, 0, 64, fake, 1 << 20, None) == 2
     assert lib.hif4_resq_linear(fake, 32, 64, 64, fake, fake, 64, 0, fake, 7, 64, fake, 1 << 20, None) == 5

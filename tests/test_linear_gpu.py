@@ -569,3 +569,31 @@ def test_full_size_layers_on_sampled_rows(cfg_idx, layer, pattern):
     want = oracle.resq_linear(bf16_bits_to_f32(np.ascontiguousarray(xb[rows])), bf16_bits_to_f32(wb), pattern)
     got = y[torch.from_numpy(rows).cuda()].float().cpu().numpy()
     check_close(got, want["y"], want["abs_sum"], bf16_out=True)
+
+
+def test_bounded_wait_expires_and_the_context_stays_usable():
+    """RESQ_ERR_TIMEOUT path: the test hook makes the decode-sized GEMM wait for a partial tile that cannot come.  The
+    bounded wait gives up, the kernel records the status and exits normally (nothing faults, nothing hangs),
+    resq_check reports it, and the next call on the same workspace is an ordinary, correct one."""
+    m = rq()
+    xb, wb = make_layer(CONFIGS[1], 1, N=512)   # M = 256, K = 2048: CTA-pair kernel, K-streamed schedule
+    pattern = oracle.S_2_4
+    want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern)
+    wc, ws = m.pack_weight(to_dev(wb))
+    M, K = xb.shape
+    work = m.alloc_workspace(m.resq_workspace_bytes(M, 512, K, pattern))
+    x = to_dev(xb)
+    m.debug_expire_next_wait(True)
+    m.resq_linear(x, wc, ws, pattern, out_dtype=torch.float32, workspace=work)
+    assert m.check(work) == 7                     # RESQ_ERR_TIMEOUT
+    assert "wait 7" in m.last_error()             # the wait for the other pairs' segments
+    torch.cuda.synchronize()                      # the context is intact
+    for _ in range(2):
+        y = m.resq_linear(x, wc, ws, pattern, out_dtype=torch.float32, workspace=work)
+        assert m.check(work) == 0, m.last_error()
+        check_close(y.cpu().numpy(), want["y"], want["abs_sum"])
+    # a request that no launch consumed can be withdrawn
+    m.debug_expire_next_wait(True)
+    m.debug_expire_next_wait(False)
+    y = m.resq_linear(x, wc, ws, pattern, out_dtype=torch.float32, workspace=work)
+    assert m.check(work) == 0

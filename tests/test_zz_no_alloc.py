@@ -45,6 +45,37 @@ def test_static_scratch_matches_workspace_variant_twice(pattern):
     _same(want1, got1b)
 
 
+@pytest.mark.parametrize("pattern", ["chan25", "block-strip", "block-strip75", "1:4"])
+def test_static_scratch_takes_the_pattern_modifiers(pattern):
+    """Kept share in quarters and the per-strip block rule: the same masks as the workspace variant."""
+    import paper_2607_26515_b200 as rq
+    pat = {"chan25": rq.keep_quarters(rq.S_CHAN50, 1), "block-strip": rq.per_strip(rq.S_BLOCK),
+           "block-strip75": rq.keep_quarters(rq.per_strip(rq.S_BLOCK), 3), "1:4": rq.keep_quarters(rq.S_2_4, 1)}[pattern]
+    for seed, (M, K) in enumerate([(256, 4096), (96, 1024)]):
+        x = _inputs(10 + seed, M, K)
+        want = rq.residual_mask(x, pat)
+        got = rq.residual_mask_static(x, pat)
+        torch.cuda.synchronize()
+        _same(want, got)
+
+
+def test_static_scratch_at_its_largest_selection():
+    """32768 channel scores is the limit: accepted, and selected by the one-CTA kernel (the workspace variant uses
+    the grid-wide selection from 24577 scores on): both must keep the same channels."""
+    import paper_2607_26515_b200 as rq
+    K = rq.STATIC_SCRATCH_MAX_SCORES
+    x = _inputs(5, 32, K)
+    want = rq.residual_mask(x, rq.S_CHAN50)
+    for _ in range(2):
+        got = rq.residual_mask_static(x, rq.S_CHAN50)
+        torch.cuda.synchronize()
+        _same(want, got)
+    xl = torch.zeros((32, K + 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(rq.ResqError) as e:
+        rq.residual_mask_static(xl, rq.S_CHAN50)
+    assert e.value.status == 4
+
+
 def test_static_scratch_rejects_problems_beyond_its_size():
     import paper_2607_26515_b200 as rq
     K = 64 * 1024   # 65536 channel scores > 32768
