@@ -178,6 +178,39 @@ RESQ_API int mxfp4_resq_linear(const void* X_bf16, int64_t M, int64_t K, int64_t
                       int pattern, void* Y, int out_dtype, int64_t ldy,
                       void* workspace, size_t ws_bytes, void* stream);
 
+/* ---- several independent projections of Eq. (5) in one call (the paper treats one projection; the grouping is this
+ * library's, for decode-sized problems) -----------------------------------------------------------------------------
+ * At a few hundred token rows a single projection cannot fill the device: its launch, pipeline fill and the sum of its
+ * partial tiles cost more than its arithmetic.  A group of up to RESQ_MAX_GROUP projections that do not depend on one
+ * another (the q/k/v, gate and up projections of a block, the experts of a mixture, the layers of several models)
+ * runs as ONE quantizer launch and ONE GEMM launch whose CTA pairs walk the output tiles of all problems: whole tiles
+ * first, the k-blocks of the remaining tiles dealt out evenly, partial tiles summed in a fixed order inside the kernel
+ * (bit-identical results run to run).  Each problem is exactly *_resq_linear: same quantizer, residual and selection,
+ * results within the same tolerance (the fp32 summation order over K differs from the single call's).
+ *   - `problems` is a HOST array read during the call; its tensor pointers are device pointers with the alignment
+ *     rules of *_resq_linear; M, N, K may differ from problem to problem; any M >= 1.
+ *   - pattern: RESQ_S_NONE, RESQ_S_DENSE or RESQ_S_2_4 (with RESQ_KEEP_QUARTERS), one for the whole group; the
+ *     selections that look beyond a token row (ROW50, CHAN50, BLOCK) are RESQ_ERR_PATTERN here.
+ *   - workspace of *_resq_group_workspace_bytes(problems, count, pattern) bytes, owned by the caller; status word,
+ *     bounded waits and resq_check as for *_resq_linear (the CTAs of the GEMM wait for one another at its end: issue
+ *     overlapping calls on one stream). */
+#define RESQ_MAX_GROUP 8
+typedef struct resq_problem {
+    const void* X_bf16;  /* [M, K] device, row pitch ldx */
+    int64_t M, K, ldx;
+    const void* w_codes; /* [N, K/2] from *_pack_weight */
+    const void* w_side;  /* HiF4: w_meta [N, K/64] u32; MXFP4: w_scale [N, K/32] u8 */
+    int64_t N;
+    void* Y;             /* [M, N] device, row pitch ldy; bf16 or fp32 as out_dtype says */
+    int64_t ldy;
+} resq_problem;
+RESQ_API size_t hif4_resq_group_workspace_bytes(const resq_problem* problems, int count, int pattern);
+RESQ_API size_t mxfp4_resq_group_workspace_bytes(const resq_problem* problems, int count, int pattern);
+RESQ_API int hif4_resq_linear_group(const resq_problem* problems, int count, int pattern, int out_dtype,
+                           void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_resq_linear_group(const resq_problem* problems, int count, int pattern, int out_dtype,
+                            void* workspace, size_t ws_bytes, void* stream);
+
 /* Weight-only ablation of Table 1 ("W4A16"): Y = X deq(Q(W))^T, the bf16 activations are used as they are
  * (no activation quantizer, no residual term); weights as produced by *_pack_weight.  Same argument rules,
  * output types and error behaviour as *_resq_linear; workspace of resq_w4a16_workspace_bytes(M, N, K) bytes

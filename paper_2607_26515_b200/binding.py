@@ -44,6 +44,10 @@ SYMBOLS = {
     "resq_residual_mask_static": (_ci, [_vp, _i64, _i64, _i64, _ci, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hif4_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
     "mxfp4_resq_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "hif4_resq_group_workspace_bytes": (_sz, [_vp, _ci, _ci]),
+    "mxfp4_resq_group_workspace_bytes": (_sz, [_vp, _ci, _ci]),
+    "hif4_resq_linear_group": (_ci, [_vp, _ci, _ci, _ci, _vp, _sz, _vp]),
+    "mxfp4_resq_linear_group": (_ci, [_vp, _ci, _ci, _ci, _vp, _sz, _vp]),
     "resq_w4a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "resq_w4a8_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "hif4_w4a8_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
@@ -277,6 +281,54 @@ def resq_linear(X: torch.Tensor, w_codes: torch.Tensor, w_side: torch.Tensor, pa
         OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32, Y.stride(0), workspace.data_ptr(), workspace.numel(),
         _stream(stream)))
     return Y
+
+
+class _Problem(ctypes.Structure):
+    """struct resq_problem of include/resq.h."""
+    _fields_ = [("X_bf16", _vp), ("M", _i64), ("K", _i64), ("ldx", _i64), ("w_codes", _vp), ("w_side", _vp), ("N", _i64),
+                ("Y", _vp), ("ldy", _i64)]
+
+
+MAX_GROUP = 8
+
+
+def _problem_array(problems, out_dtype):
+    """problems: sequence of (X, w_codes, w_side) or (X, w_codes, w_side, Y) -> (ctypes array, list of Y)."""
+    arr = (_Problem * len(problems))()
+    ys = []
+    for i, pr in enumerate(problems):
+        X, wc, ws = pr[0], pr[1], pr[2]
+        _require_bf16_matrix(X, "X")
+        M, K = X.shape
+        N = wc.shape[0]
+        Y = pr[3] if len(pr) > 3 and pr[3] is not None else torch.empty((M, (N + 7) // 8 * 8), dtype=out_dtype, device=X.device)[:, :N]
+        if Y.dtype != out_dtype:
+            raise ValueError("every Y of a group has the group's output type")
+        ys.append(Y)
+        arr[i] = _Problem(X.data_ptr(), M, K, X.stride(0), wc.data_ptr(), ws.data_ptr(), N, Y.data_ptr(), Y.stride(0))
+    return arr, ys
+
+
+def resq_group_workspace_bytes(problems, pattern: int, fmt: str = "hif4", out_dtype: torch.dtype = torch.bfloat16) -> int:
+    arr, _ = _problem_array(problems, out_dtype)
+    return int(_fn(fmt, "hif4_resq_group_workspace_bytes", "mxfp4_resq_group_workspace_bytes")(
+        ctypes.cast(arr, _vp), len(problems), pattern))
+
+
+def resq_linear_group(problems, pattern: int, fmt: str = "hif4", out_dtype: torch.dtype = torch.bfloat16,
+                      workspace: Optional[torch.Tensor] = None, stream=None):
+    """*_resq_linear_group: up to MAX_GROUP independent projections of Eq. (5) in one quantizer launch and one GEMM
+    launch.  problems: sequence of (X, w_codes, w_side[, Y]); returns the list of outputs."""
+    if out_dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("Y must be bf16 or fp32")
+    arr, ys = _problem_array(problems, out_dtype)
+    fn_b = _fn(fmt, "hif4_resq_group_workspace_bytes", "mxfp4_resq_group_workspace_bytes")
+    if workspace is None:
+        workspace = alloc_workspace(int(fn_b(ctypes.cast(arr, _vp), len(problems), pattern)), problems[0][0].device)
+    _check(_fn(fmt, "hif4_resq_linear_group", "mxfp4_resq_linear_group")(
+        ctypes.cast(arr, _vp), len(problems), pattern, OUT_BF16 if out_dtype == torch.bfloat16 else OUT_F32,
+        workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return ys
 
 
 def w4a16_linear(X: torch.Tensor, w_codes: torch.Tensor, w_side: torch.Tensor, fmt: str = "hif4",

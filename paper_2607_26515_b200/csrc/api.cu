@@ -496,6 +496,123 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     return launch_gemm_hif4(g, st);
 }
 
+// ---- a group of independent projections in one quantizer launch and one GEMM launch ---------------------------
+// Workspace: [header | counters | per problem: image of deq Q(X), residual operand | fp32 partial-tile slots].
+size_t group_workspace_bytes(const resq_problem* pr, int count, int pattern) {
+    if (!pr || count < 1 || count > kMaxQuantGroup) return 0;
+    size_t b = kWsHeader + kWsFlags;
+    for (int i = 0; i < count; ++i) {
+        if (pr[i].M <= 0 || pr[i].N <= 0 || pr[i].K <= 0) return 0;
+        b += align_up((size_t)pr[i].M * (size_t)pr[i].K * 2, 256) + residual_region_bytes(pr[i].M, pr[i].K, pattern);
+    }
+    return b + align_up(gemm_pair_streamk_scratch_bytes(), 256);
+}
+
+int linear_group(int fmt, const resq_problem* pr, int count, int pattern, int out_dtype, void* workspace, size_t ws_bytes,
+                 void* stream) {
+    if (!pr) {
+        set_last_error("linear_group: problems is NULL");
+        return RESQ_ERR_NULL;
+    }
+    if (count < 1 || count > kMaxQuantGroup) {
+        set_last_error("linear_group: a group holds 1 to %d problems (got %d)", kMaxQuantGroup, count);
+        return RESQ_ERR_SHAPE;
+    }
+    int quarters = 2, per_strip = 0;
+    int rc = split_pattern(&pattern, &quarters, &per_strip);
+    if (rc) return rc;
+    if (pattern != RESQ_S_NONE && pattern != RESQ_S_DENSE && pattern != RESQ_S_2_4) {
+        set_last_error("linear_group takes the selections that are local to a token row (none, dense, n:4); the row-wise, "
+                       "channel-wise and block-wise selections run through *_resq_linear");
+        return RESQ_ERR_PATTERN;
+    }
+    if (out_dtype != RESQ_OUT_BF16 && out_dtype != RESQ_OUT_F32) {
+        set_last_error("unknown output type %d", out_dtype);
+        return RESQ_ERR_PATTERN;
+    }
+    for (int i = 0; i < count; ++i) {
+        rc = check_matrix(pr[i].X_bf16, pr[i].M, pr[i].K, pr[i].ldx, fmt, "X");
+        if (rc) return rc;
+        if (!pr[i].w_codes || !pr[i].w_side || !pr[i].Y) {
+            set_last_error("linear_group: NULL weight or output pointer in problem %d", i);
+            return RESQ_ERR_NULL;
+        }
+        if (pr[i].N <= 0) {
+            set_last_error("linear_group: N=%lld in problem %d", (long long)pr[i].N, i);
+            return RESQ_ERR_SHAPE;
+        }
+        if (!aligned16(pr[i].Y) || !aligned16(pr[i].w_codes) || !aligned16(pr[i].w_side) || pr[i].ldy < pr[i].N ||
+            pr[i].ldy % (out_dtype == RESQ_OUT_BF16 ? 8 : 4) != 0) {
+            set_last_error("linear_group: Y / weights need 16-byte aligned bases, ldy >= N and 16-byte aligned rows (problem %d)", i);
+            return RESQ_ERR_ALIGN;
+        }
+    }
+    rc = check_workspace(workspace, ws_bytes, group_workspace_bytes(pr, count, pattern));
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    QuantArgs qa[kMaxQuantGroup];
+    GemmArgs ga[kMaxQuantGroup];
+    size_t used = kWsHeader + kWsFlags;
+    bool sparse24 = pattern == RESQ_S_2_4 && quarters == 2;
+    for (int i = 0; i < count && sparse24; ++i) sparse24 = gemm_sparse24_supported(256, pr[i].N, pr[i].K);
+    for (int i = 0; i < count; ++i) {
+        QuantArgs& a = qa[i];
+        memset(&a, 0, sizeof(a));
+        a.X = static_cast<const __nv_bfloat16*>(pr[i].X_bf16);
+        a.M = pr[i].M;
+        a.K = pr[i].K;
+        a.ldx = pr[i].ldx;
+        a.pattern = pattern;
+        a.keep_quarters = quarters;
+        a.status = reinterpret_cast<DeviceStatus*>(ws);
+        if (i == 0) {  // cleared by the quantizer kernel: no separate memset node
+            a.clear_words = reinterpret_cast<uint32_t*>(ws);
+            a.n_clear_words = (int)((kWsHeader + kWsFlags) / 4);
+        }
+        a.a_bf16 = reinterpret_cast<__nv_bfloat16*>(ws + used);
+        used += align_up((size_t)a.M * (size_t)a.K * 2, 256);
+        if (pattern != RESQ_S_NONE) {
+            uint8_t* region_r = ws + used;
+            used += residual_region_bytes(a.M, a.K, pattern);
+            if (sparse24) {
+                a.r_comp = reinterpret_cast<__nv_bfloat16*>(region_r);
+                a.r_meta = region_r + align_up((size_t)a.M * (size_t)a.K, 256);
+                a.meta_rows128 = sparse24_rows128(a.M);
+                a.meta_ka = sparse24_ka(a.K);
+            } else {
+                a.r_bf16 = reinterpret_cast<__nv_bfloat16*>(region_r);
+            }
+        }
+    }
+    for (int i = 0; i < count; ++i) {
+        GemmArgs& g = ga[i];
+        memset(&g, 0, sizeof(g));
+        g.fmt = fmt;
+        g.a_bf16 = qa[i].a_bf16;
+        g.r_bf16 = qa[i].r_bf16;
+        g.r_comp = qa[i].r_comp;
+        g.r_meta = qa[i].r_meta;
+        g.meta_rows128 = qa[i].meta_rows128;
+        g.meta_ka = qa[i].meta_ka;
+        g.w_codes = static_cast<const uint8_t*>(pr[i].w_codes);
+        g.w_side = pr[i].w_side;
+        g.M = pr[i].M;
+        g.N = pr[i].N;
+        g.K = pr[i].K;
+        g.Y = pr[i].Y;
+        g.out_dtype = out_dtype;
+        g.ldy = pr[i].ldy;
+        g.partial_bytes = gemm_pair_streamk_scratch_bytes();
+        g.splitk_partials = reinterpret_cast<float*>(ws + used);
+        g.sk_flags = reinterpret_cast<unsigned int*>(ws + kWsHeader);
+        g.status = reinterpret_cast<DeviceStatus*>(ws);
+    }
+    rc = launch_quantize_group(fmt, qa, count, st);
+    if (rc) return rc;
+    return launch_gemm_pair_group(ga, count, st);
+}
+
 // Weight-only variant (Table 1, "W4A16"): Y = X deq(Q(W))^T with the bf16 activations used as they are.
 // Workspace: [header | counters | fp32 partial tiles].
 size_t w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
@@ -767,6 +884,21 @@ int mxfp4_resq_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const vo
                       int64_t N, int pattern, void* Y, int out_dtype, int64_t ldy, void* workspace, size_t ws_bytes,
                       void* stream) {
     return linear(kMXFP4, X, M, K, ldx, w_codes, w_scale, N, pattern, Y, out_dtype, ldy, workspace, ws_bytes, stream);
+}
+
+size_t hif4_resq_group_workspace_bytes(const resq_problem* problems, int count, int pattern) {
+    return group_workspace_bytes(problems, count, base_pattern(pattern));
+}
+size_t mxfp4_resq_group_workspace_bytes(const resq_problem* problems, int count, int pattern) {
+    return group_workspace_bytes(problems, count, base_pattern(pattern));
+}
+int hif4_resq_linear_group(const resq_problem* problems, int count, int pattern, int out_dtype, void* workspace, size_t ws_bytes,
+                           void* stream) {
+    return linear_group(kHiF4, problems, count, pattern, out_dtype, workspace, ws_bytes, stream);
+}
+int mxfp4_resq_linear_group(const resq_problem* problems, int count, int pattern, int out_dtype, void* workspace, size_t ws_bytes,
+                            void* stream) {
+    return linear_group(kMXFP4, problems, count, pattern, out_dtype, workspace, ws_bytes, stream);
 }
 
 int resq_check(void* workspace, void* stream) {

@@ -136,6 +136,8 @@ struct QuantArgs {
 };
 
 int launch_quantize(int fmt, const QuantArgs& a, cudaStream_t stream);
+constexpr int kMaxQuantGroup = 8;  // problems per grouped launch (quantizer and GEMM alike)
+int launch_quantize_group(int fmt, const QuantArgs* a, int count, cudaStream_t stream);
 // "W4A8": the decoded bf16 image of MXFP8-E4M3 quantized activations (blocks of 32, E8M0 scale), for the GEMM
 int launch_quantize_mxfp8_image(const __nv_bfloat16* X, int64_t M, int64_t K, int64_t ldx, __nv_bfloat16* img, uint32_t* clear_words,
                                 int n_clear_words, cudaStream_t stream);
@@ -171,6 +173,10 @@ struct GemmArgs {
     DeviceStatus* status;
 };
 int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream);
+// A group of independent problems (same format, residual mode and output type) as one launch of the CTA-pair kernel on
+// the K-streamed schedule; status word, arrival counters and partial-tile slots are those of g[0] (gemm_pair.cu).
+int launch_gemm_pair_group(const GemmArgs* g, int count, cudaStream_t stream);
+size_t gemm_pair_streamk_scratch_bytes();
 // Test hook behind resq_debug_expire_next_wait (gemm_pair.cu).
 void debug_expire_next_wait(int on);
 // Whether launch_gemm_hif4 takes the compressed 2:4 residual for this shape (the CTA-pair kernel runs it).

@@ -333,6 +333,9 @@ gemm_hif4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     mw[q] = __shfl_sync(0xFFFFFFFFu, q < 8 ? meta_cur0 : meta_cur1, rl & 31);
                     cw[q] = raw[(r_begin + rl) * 8 + chunk];
                 }
+                // the reads above (generic proxy) are ordered before the TMA producer's next load into this slot (async
+                // proxy) by a proxy fence; see gemm_pair.cu
+                ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&r_empty[sr]);  // the raw codes are in registers now
 #pragma unroll

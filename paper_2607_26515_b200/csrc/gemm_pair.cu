@@ -20,9 +20,11 @@
 
 #include <algorithm>
 #include <atomic>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 namespace resq {
 
@@ -45,16 +47,35 @@ constexpr int kMaxRing = 8;
 constexpr int kSmemBudget = 232448;
 constexpr int kTmemCols = 512;
 
-struct PairParams {
+// One launch computes one problem (NP = 1) or a group of independent problems that share the residual mode, the weight
+// format and the output type (NP = kMaxGroup): the tiles of all problems form one list, problem after problem.
+constexpr int kMaxGroup = kMaxQuantGroup;
+
+struct PairProblem {
     const void* w_side;
-    int64_t M, N, K;
-    int kblocks_per_split, splits;
-    int ntiles_m, ntiles_n, num_tiles;
-    int sa, sr, se, acc_bufs;
-    int meta_ka;             // sparse residual: metadata blocks (128 K positions) per 128-row band
     void* Y;
-    int out_f32;
     int64_t ldy;
+    int M, N, G;             // token rows, output columns, k-blocks (K / 64)
+    int ntiles_n;
+    int tile_base;           // position of the problem's first tile in the launch's tile list
+    int dealt_first;         // K-streamed schedule: first tile of the problem whose k-blocks are dealt out (else whole)
+    int64_t unit_base;       //   and the (tile, k-block) units of the dealt tiles of the problems before it
+    int meta_ka;             // sparse residual: metadata blocks (128 K positions) per 128-row band
+};
+
+template <int NP>
+struct PairMaps {
+    CUtensorMap a[NP], r[NP], e[NP], w[NP];
+};
+
+template <int NP>
+struct PairParams {
+    PairProblem pr[NP];
+    int nprob;
+    int kblocks_per_split, splits;
+    int num_tiles;
+    int sa, sr, se, acc_bufs;
+    int out_f32;
     float* partials;
     DeviceStatus* status;
 #ifdef RESQ_TIMELINE
@@ -62,15 +83,17 @@ struct PairParams {
     unsigned int* timeline;  // device buffer for a per-role event log of pair 0 (or null)
     int timeline_first;      // first k-block iteration that is logged
 #endif
-    // K-streamed schedule (streamk != 0): the num_tiles * G (tile, k-block) units are dealt out evenly to the
-    // pairs; a pair's first and last segment may cover only part of a tile's K range and then go to fp32 slots
+    // K-streamed schedule (streamk != 0): the first dp_tiles tiles of the list are computed whole, tile t by pair
+    // t mod npairs, and written out directly; the sk_units (tile, k-block) units of the remaining tiles are dealt
+    // out in contiguous ranges: the pairs below sk_first (those that hold one whole tile more) take sk_hi units
+    // each, the pairs sk_first .. sk_first + sk_pairs - 1 share the rest evenly.  A range may start and end inside
+    // a tile's K range: such segments go to fp32 slots and are summed at the end of the kernel.
     int streamk;
-    // With more tiles than pairs the first dp_tiles tiles (a multiple of the number of pairs) are computed whole,
-    // one per pair and round, and written out directly; only the k-blocks of the remaining tiles are dealt out.
     int dp_tiles;
-    int sk_pairs;            // pairs 0 .. sk_pairs-1 share the dealt-out units (at least two k-blocks each)
+    int sk_first, sk_hi, sk_pairs;
+    int64_t sk_units;
     float* sk_slots;         // [2 * npairs][256][TN] fp32: slot 2p = first segment of pair p, 2p + 1 = its last
-    unsigned int* sk_flags;  // [num_tiles][2]: segments of the tile written, per CTA rank (zeroed before launch)
+    unsigned int* sk_flags;  // [dealt tiles][2]: segments of the tile written, per CTA rank (zeroed before launch)
     int sk_poll_limit;       // polls (about 0.3 us each) before the wait for a tile's segments gives up
     int sk_extra;            // test hook (resq_debug_expire_next_wait): arrivals awaited beyond those that can come
 };
@@ -101,19 +124,33 @@ struct Trace {
 struct TileCoord {
     int64_t m0, n0;
     int split, kb_begin, nkb;
-    int tile_id;   // K-streamed schedule: output tile of the segment
+    int prob;      // problem of the tile
+    int tile_id;   // K-streamed schedule: index of the segment's tile among the dealt tiles
     int slot;      //   and where its fp32 partial goes
     bool partial;  // the segment does not cover the whole K range (or K is split): fp32 partial output
 };
 
-template <int TN>
-__device__ __forceinline__ TileCoord decode_tile(const PairParams& p, int tile) {
+// Problem that holds tile t of the launch's tile list (t below the total).
+template <int NP>
+__device__ __forceinline__ int problem_of_tile(const PairParams<NP>& p, int t) {
+    int q = 0;
+    if constexpr (NP > 1) {
+#pragma unroll 1
+        while (q + 1 < p.nprob && t >= p.pr[q + 1].tile_base) ++q;
+    }
+    return q;
+}
+
+// Whole-tile schedule of a single problem (tile list entry = (output tile, K split)).
+template <int TN, int NP>
+__device__ __forceinline__ TileCoord decode_tile(const PairParams<NP>& p, int tile) {
     TileCoord t;
     t.split = tile % p.splits;
     const int rest = tile / p.splits;
-    t.n0 = (int64_t)(rest % p.ntiles_n) * TN;
-    t.m0 = (int64_t)(rest / p.ntiles_n) * (2 * kBM);
-    const int G = (int)(p.K / kBK);
+    t.prob = 0;
+    t.n0 = (int64_t)(rest % p.pr[0].ntiles_n) * TN;
+    t.m0 = (int64_t)(rest / p.pr[0].ntiles_n) * (2 * kBM);
+    const int G = p.pr[0].G;
     t.kb_begin = t.split * p.kblocks_per_split;
     t.nkb = min(G, t.kb_begin + p.kblocks_per_split) - t.kb_begin;
     if (t.nkb < 0) t.nkb = 0;
@@ -123,28 +160,48 @@ __device__ __forceinline__ TileCoord decode_tile(const PairParams& p, int tile) 
     return t;
 }
 
-// K-streamed schedule: pair q owns units [q * U / P, (q + 1) * U / P) of the U = num_tiles * G (tile, k-block)
-// units, tile-major.
-__device__ __forceinline__ int64_t sk_begin(int64_t U, int P, int q) { return (int64_t)q * U / P; }
-__device__ __forceinline__ int sk_pair_of(int64_t U, int P, int64_t u) { return (int)((((u + 1) * P) - 1) / U); }
+// K-streamed schedule: first dealt unit of pair q (q may be one past the last pair), and the pair that owns unit u.
+template <int NP>
+__device__ __forceinline__ int64_t sk_begin(const PairParams<NP>& p, int q) {
+    if (q < p.sk_first) return (int64_t)q * p.sk_hi;
+    const int64_t head = (int64_t)p.sk_first * p.sk_hi;
+    if (q >= p.sk_first + p.sk_pairs) return p.sk_units;
+    return head + (int64_t)(q - p.sk_first) * (p.sk_units - head) / p.sk_pairs;
+}
+template <int NP>
+__device__ __forceinline__ int sk_pair_of(const PairParams<NP>& p, int64_t u) {
+    const int64_t head = (int64_t)p.sk_first * p.sk_hi;
+    if (u < head) return (int)(u / p.sk_hi);
+    return p.sk_first + (int)((((u - head + 1) * p.sk_pairs) - 1) / (p.sk_units - head));
+}
+// Dealt unit u -> problem, tile of the launch's list and k-block.
+template <int NP>
+__device__ __forceinline__ void sk_locate(const PairParams<NP>& p, int64_t u, int& prob, int& tile, int& kb) {
+    int q = 0;
+    if constexpr (NP > 1) {
+#pragma unroll 1
+        while (q + 1 < p.nprob && u >= p.pr[q + 1].unit_base) ++q;
+    }
+    const int64_t rel = u - p.pr[q].unit_base;
+    const int tr = (int)(rel / p.pr[q].G);
+    prob = q;
+    tile = p.pr[q].dealt_first + tr;
+    kb = (int)(rel - (int64_t)tr * p.pr[q].G);
+}
 
 // Walks the work of one pair in the order every role of the kernel uses.
-template <int TN>
+template <int TN, int NP>
 struct SegIter {
-    const PairParams& p;
-    int pair, npairs, G;
-    int tile;            // tile schedule: next tile
-    int64_t u0, u, u1;   // K-streamed schedule: this pair's units
-    __device__ SegIter(const PairParams& p_, int pair_, int npairs_) : p(p_), pair(pair_), npairs(npairs_) {
-        G = (int)(p.K / kBK);
+    const PairParams<NP>& p;
+    int pair, npairs;
+    int tile;            // next whole tile
+    int64_t u0, u, u1;   // K-streamed schedule: this pair's dealt units
+    __device__ SegIter(const PairParams<NP>& p_, int pair_, int npairs_) : p(p_), pair(pair_), npairs(npairs_) {
         tile = pair;
+        u0 = u = u1 = 0;
         if (p.streamk) {
-            const int64_t U = (int64_t)(p.num_tiles - p.dp_tiles) * G;  // units of the tiles that are dealt out
-            u0 = u = u1 = 0;
-            if (pair < p.sk_pairs) {
-                u0 = u = sk_begin(U, p.sk_pairs, pair);
-                u1 = sk_begin(U, p.sk_pairs, pair + 1);
-            }
+            u0 = u = sk_begin(p, pair);
+            u1 = sk_begin(p, pair + 1);
         }
     }
     __device__ bool next(TileCoord& tc) {
@@ -155,27 +212,32 @@ struct SegIter {
             return true;
         }
         if (tile < p.dp_tiles) {  // whole tiles first
-            tc.tile_id = tile;
+            const int q = problem_of_tile(p, tile);
+            const int tl = tile - p.pr[q].tile_base;
+            tc.prob = q;
+            tc.tile_id = 0;
             tc.split = 0;
             tc.kb_begin = 0;
-            tc.nkb = G;
-            tc.n0 = (int64_t)(tile % p.ntiles_n) * TN;
-            tc.m0 = (int64_t)(tile / p.ntiles_n) * (2 * kBM);
+            tc.nkb = p.pr[q].G;
+            tc.n0 = (int64_t)(tl % p.pr[q].ntiles_n) * TN;
+            tc.m0 = (int64_t)(tl / p.pr[q].ntiles_n) * (2 * kBM);
             tc.partial = false;
             tc.slot = 0;
             tile += npairs;
             return true;
         }
         if (u >= u1) return false;
-        const int tr = (int)(u / G);     // among the tiles that are dealt out
-        const int t = p.dp_tiles + tr;
-        tc.tile_id = t;
+        int q, t, kb;
+        sk_locate(p, u, q, t, kb);
+        const int tl = t - p.pr[q].tile_base;
+        tc.prob = q;
+        tc.tile_id = t - p.dp_tiles;
         tc.split = 0;
-        tc.kb_begin = (int)(u - (int64_t)tr * G);
-        tc.nkb = (int)min((int64_t)(G - tc.kb_begin), u1 - u);
-        tc.n0 = (int64_t)(t % p.ntiles_n) * TN;
-        tc.m0 = (int64_t)(t / p.ntiles_n) * (2 * kBM);
-        tc.partial = tc.nkb < G;
+        tc.kb_begin = kb;
+        tc.nkb = (int)min((int64_t)(p.pr[q].G - kb), u1 - u);
+        tc.n0 = (int64_t)(tl % p.pr[q].ntiles_n) * TN;
+        tc.m0 = (int64_t)(tl / p.pr[q].ntiles_n) * (2 * kBM);
+        tc.partial = tc.nkb < p.pr[q].G;
         tc.slot = 2 * pair + (u == u0 ? 0 : 1);
         u += tc.nkb;
         return true;
@@ -197,27 +259,26 @@ __device__ __forceinline__ float4 ld_cg_f4(const float* p) {
 // The pairs that hold segments of a tile each reduce one column slice of it: they wait until all segments of
 // the tile are in their slots, then add them in k order (a fixed order: the result does not depend on timing).
 // Called by all threads of the CTA; the CTA of rank r handles rows r * 128 .. r * 128 + 127 of the tile.
-template <int TN>
-__device__ __forceinline__ void streamk_fixup(const PairParams& p, int pair, int npairs, int rank, volatile int* abort_flag,
+template <int TN, int NP>
+__device__ __forceinline__ void streamk_fixup(const PairParams<NP>& p, int pair, int rank, volatile int* abort_flag,
                                               volatile int* s_ok, int* s_slots, unsigned int* evt, long long t0) {
-    const int G = (int)(p.K / kBK);
-    const int64_t U = (int64_t)(p.num_tiles - p.dp_tiles) * G;
-    if (pair >= p.sk_pairs) return;
-    npairs = p.sk_pairs;  // the pairs that share the dealt-out units
-    const int64_t u0 = sk_begin(U, npairs, pair), u1 = sk_begin(U, npairs, pair + 1);
+    const int64_t u0 = sk_begin(p, pair), u1 = sk_begin(p, pair + 1);
     if (u1 <= u0) return;
-    const int t_first = (int)(u0 / G), t_last = (int)((u1 - 1) / G);  // among the tiles that are dealt out
+    int q_first, t_first, q_last, t_last, kb_unused;
+    sk_locate(p, u0, q_first, t_first, kb_unused);
+    sk_locate(p, u1 - 1, q_last, t_last, kb_unused);
     for (int which = 0; which < 2; ++which) {
-        const int tr = which == 0 ? t_first : t_last;
+        const int t = which == 0 ? t_first : t_last;  // tile of the launch's list
+        const int q = which == 0 ? q_first : q_last;
         if (which == 1 && t_last == t_first) break;
-        const int t = p.dp_tiles + tr;  // output tile
-        const int64_t tb = (int64_t)tr * G, te = tb + G;
+        const PairProblem& pb = p.pr[q];
+        const int64_t tb = pb.unit_base + (int64_t)(t - pb.dealt_first) * pb.G, te = tb + pb.G;
         if (u0 <= tb && u1 >= te) continue;  // this pair computed the whole tile and wrote it out directly
-        const int pf = sk_pair_of(U, npairs, tb), pl = sk_pair_of(U, npairs, te - 1);
+        const int pf = sk_pair_of(p, tb), pl = sk_pair_of(p, te - 1);
         const int nseg = pl - pf + 1, j = pair - pf;
         if (threadIdx.x == 0) {
             int ok = *abort_flag ? 0 : 1;
-            const unsigned int* flag = p.sk_flags + t * 2 + rank;
+            const unsigned int* flag = p.sk_flags + (t - p.dp_tiles) * 2 + rank;
             for (int polls = 0; ok && ld_acquire_u32(flag) < (unsigned)(nseg + p.sk_extra); ++polls) {
                 __nanosleep(200);
                 if (polls > p.sk_poll_limit) {
@@ -234,19 +295,20 @@ __device__ __forceinline__ void streamk_fixup(const PairParams& p, int pair, int
         if (evt && threadIdx.x == 0) evt[which] = (unsigned int)(clock64() - t0);
         // slot of every segment (k order), worked out once per tile
         if ((int)threadIdx.x < nseg) {
-            const int q = pf + (int)threadIdx.x;
-            s_slots[threadIdx.x] = 2 * q + (sk_begin(U, npairs, q) >= tb ? 0 : 1);
+            const int sq = pf + (int)threadIdx.x;
+            s_slots[threadIdx.x] = 2 * sq + (sk_begin(p, sq) >= tb ? 0 : 1);
         }
         __syncthreads();
         // column slice j of nseg, in units of 4 columns
         const int c0 = (int)((int64_t)j * (TN / 4) / nseg) * 4, c1 = (int)((int64_t)(j + 1) * (TN / 4) / nseg) * 4;
         const int w4 = (c1 - c0) / 4;
-        const int64_t m_base = (int64_t)(t / p.ntiles_n) * (2 * kBM) + rank * kBM;
-        const int64_t n_base = (int64_t)(t % p.ntiles_n) * TN;
+        const int tl = t - pb.tile_base;
+        const int64_t m_base = (int64_t)(tl / pb.ntiles_n) * (2 * kBM) + rank * kBM;
+        const int64_t n_base = (int64_t)(tl % pb.ntiles_n) * TN;
         for (int item = threadIdx.x; item < kBM * w4; item += (int)blockDim.x) {
             const int row = item / w4, c = c0 + (item % w4) * 4;
             const int64_t m = m_base + row, n = n_base + c;
-            if (m >= p.M || n >= p.N) continue;
+            if (m >= pb.M || n >= pb.N) continue;
             const float* src = p.sk_slots + ((size_t)rank * kBM + row) * TN + c;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int s0 = 0; s0 < nseg; s0 += 4) {
@@ -261,19 +323,20 @@ __device__ __forceinline__ void streamk_fixup(const PairParams& p, int pair, int
             }
             const float o[4] = {acc.x, acc.y, acc.z, acc.w};
             if (p.out_f32) {
-                float* dst = reinterpret_cast<float*>(p.Y) + m * p.ldy + n;
-                if (n + 3 < p.N) *reinterpret_cast<float4*>(dst) = acc;
-                else for (int e = 0; e < 4; ++e) if (n + e < p.N) dst[e] = o[e];
+                float* dst = reinterpret_cast<float*>(pb.Y) + m * pb.ldy + n;
+                if (n + 3 < pb.N) *reinterpret_cast<float4*>(dst) = acc;
+                else for (int e = 0; e < 4; ++e) if (n + e < pb.N) dst[e] = o[e];
             } else {
-                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.Y) + m * p.ldy + n;
-                if (n + 3 < p.N) {
+                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(pb.Y) + m * pb.ldy + n;
+                if (n + 3 < pb.N) {
                     __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
                     *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
                 } else {
-                    for (int e = 0; e < 4; ++e) if (n + e < p.N) dst[e] = __float2bfloat16_rn(o[e]);
+                    for (int e = 0; e < 4; ++e) if (n + e < pb.N) dst[e] = __float2bfloat16_rn(o[e]);
                 }
             }
         }
+        __syncthreads();  // the slot list is rewritten for the next tile
     }
 }
 
@@ -292,10 +355,9 @@ __host__ __device__ constexpr int a_stage_bytes(int res) {
 }
 
 // TN: width of the pair's output tile (the pair computes 256 x TN); bn = MMA N; each CTA expands TN/2 rows.
-template <int RES, int TN, int FMT, int NG>
+template <int RES, int TN, int FMT, int NG, int NP>
 __global__ void __launch_bounds__(pair_threads(NG), 1)
-gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_r,
-                 const __grid_constant__ CUtensorMap tmap_e, const __grid_constant__ CUtensorMap tmap_w, const PairParams p) {
+gemm_pair_kernel(const __grid_constant__ PairMaps<NP> maps, const __grid_constant__ PairParams<NP> p) {
     constexpr int kExpGroups = NG;
     constexpr int kAStage = a_stage_bytes(RES);
     constexpr int nt = TN > kMaxBN ? 2 : 1;           // MMAs side by side in N
@@ -338,7 +400,6 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();  // 0 = leader
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
-    const int G = (int)(p.K / kBK);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxRing; ++s) {
@@ -363,8 +424,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 #ifdef RESQ_TIMELINE
-    Trace tr{(p.debug & 16) ? reinterpret_cast<unsigned long long*>(p.status) + 8 : nullptr, 0};
     const long long t_kernel0 = clock64();
+    Trace tr{(p.debug & 16) ? reinterpret_cast<unsigned long long*>(p.status) + 8 : nullptr, 0};
     if (tl && threadIdx.x == 0) p.timeline[512 + (int)rank * 16] = (unsigned int)(t_kernel0 - t_entry);
 #else
     Trace tr;
@@ -378,15 +439,21 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------------ activation producer (both CTAs)
         if (lane == 0) {
-            ptx::tma_prefetch_desc(&tmap_a);
-            if (RES != kResNone) ptx::tma_prefetch_desc(&tmap_r);
-            if (RES == kResSparse24) ptx::tma_prefetch_desc(&tmap_e);
+            for (int q = 0; q < (NP > 1 ? p.nprob : 1); ++q) {
+                ptx::tma_prefetch_desc(&maps.a[q]);
+                if (RES != kResNone) ptx::tma_prefetch_desc(&maps.r[q]);
+                if (RES == kResSparse24) ptx::tma_prefetch_desc(&maps.e[q]);
+            }
             uint32_t it = 0;
             bool ok = true;
-            SegIter<TN> si(p, pair, npairs);
+            SegIter<TN, NP> si(p, pair, npairs);
             TileCoord tc;
             while (ok && si.next(tc)) {
                 const int my_m = (int)(tc.m0 + rank * kBM);
+                const CUtensorMap* tmap_a = &maps.a[tc.prob];
+                const CUtensorMap* tmap_r = &maps.r[tc.prob];
+                const CUtensorMap* tmap_e = &maps.e[tc.prob];
+                const int meta_ka = p.pr[tc.prob].meta_ka;
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
                     // The activation ring may be shallower than the ring of expanded weights whose barriers it shares
                     // (barrier slot = k-block mod SE): slot it % SA is free once the MMAs of k-block it - SA, which
@@ -412,13 +479,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     ptx::mbar_arrive_expect_tx_cluster_relaxed(  // publishes nothing itself
                         full, (uint32_t)(kAStage - (RES == kResSparse24 && !with_meta ? kSpMetaBytes : 0)));
                     const int kx = kb * kBK;
-                    ptx::tma_load_2d_pair(st, &tmap_a, full, kx, my_m);
-                    if (RES == kResDense) ptx::tma_load_2d_pair(st + kATileBytes, &tmap_r, full, kx, my_m);
+                    ptx::tma_load_2d_pair(st, tmap_a, full, kx, my_m);
+                    if (RES == kResDense) ptx::tma_load_2d_pair(st + kATileBytes, tmap_r, full, kx, my_m);
                     if (RES == kResSparse24) {
-                        ptx::tma_load_2d_pair(st + kATileBytes, &tmap_r, full, kx / 2, my_m);
+                        ptx::tma_load_2d_pair(st + kATileBytes, tmap_r, full, kx / 2, my_m);
                         if (with_meta)  // rows of 256 bytes, eight per 128 x 128 block
-                            ptx::tma_load_2d_pair(st + kATileBytes + kSpTileBytes, &tmap_e, full, 0,
-                                                  ((my_m >> 7) * p.meta_ka + (kb >> 1)) * 8);
+                            ptx::tma_load_2d_pair(st + kATileBytes + kSpTileBytes, tmap_e, full, 0,
+                                                  ((my_m >> 7) * meta_ka + (kb >> 1)) * 8);
                     }
                 }
             }
@@ -426,12 +493,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     } else if (warp == 2) {
         // ------------------------------------------------------------------ raw weight-code producer (both CTAs)
         if (lane == 0) {
-            ptx::tma_prefetch_desc(&tmap_w);
+            for (int q = 0; q < (NP > 1 ? p.nprob : 1); ++q) ptx::tma_prefetch_desc(&maps.w[q]);
             uint32_t it = 0;
             bool ok = true;
-            SegIter<TN> si(p, pair, npairs);
+            SegIter<TN, NP> si(p, pair, npairs);
             TileCoord tc;
             while (ok && si.next(tc)) {
+                const CUtensorMap* tmap_w = &maps.w[tc.prob];
                 if constexpr (FMT == kPlainW) {
                     // bf16 weights: this CTA's rows of the k-block go straight into the expanded-weight slot
                     for (int i = 0; i < tc.nkb; ++i, ++it) {
@@ -445,7 +513,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         ptx::mbar_arrive_expect_tx_cluster_relaxed(full, (uint32_t)exp_stage);
 #pragma unroll
                         for (int j = 0; j < nt; ++j)
-                            ptx::tma_load_2d_pair(ring_e + (size_t)se * exp_stage + (size_t)j * half * 128, &tmap_w, full,
+                            ptx::tma_load_2d_pair(ring_e + (size_t)se * exp_stage + (size_t)j * half * 128, tmap_w, full,
                                                   (tc.kb_begin + i) * kBK, (int)(tc.n0 + j * bn + rank * half));
                     }
                 } else {
@@ -463,7 +531,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     ptx::mbar_arrive_expect_tx(&r_full[s], (uint32_t)raw_stage);
 #pragma unroll
                     for (int j = 0; j < nt; ++j)
-                        ptx::tma_load_2d(ring_r + (size_t)s * raw_stage + (size_t)j * half * 32, &tmap_w, &r_full[s],
+                        ptx::tma_load_2d(ring_r + (size_t)s * raw_stage + (size_t)j * half * 32, tmap_w, &r_full[s],
                                          (tc.kb_begin + i) * (kBK / 2), (int)(tc.n0 + j * bn + rank * half));
                 }
                 }
@@ -481,7 +549,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             uint32_t it = 0, sa = 0, se = 0, pha = 0;  // activation slot, barrier / weight slot and its phase parity
             int local_tile = 0;
             bool ok = true;
-            SegIter<TN> si(p, pair, npairs);
+            SegIter<TN, NP> si(p, pair, npairs);
             TileCoord tc;
             while (ok && si.next(tc)) {
                 const int lt = local_tile++;
@@ -564,7 +632,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         const int sub_row = lane >> 3, chunk = lane & 7;
         uint32_t it0 = 0;  // k-block counter at the start of the current tile
         bool ok = true;
-        SegIter<TN> si(p, pair, npairs);
+        SegIter<TN, NP> si(p, pair, npairs);
         TileCoord tc;
         while (ok && si.next(tc)) {
             // local row l (< my_rows) is weight row n0 + (l / half) * bn + rank * half + (l % half);
@@ -572,11 +640,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             auto row_of = [&](int l) -> int64_t { return tc.n0 + (int64_t)(l / half) * bn + rank * half + (l % half); };
             const int64_t n_a = row_of(r_begin + lane);
             const int64_t n_b = row_of(r_begin + (rows_per_warp > 32 ? 32 + lane : lane));
-            const bool ok_a = lane < rows_per_warp && n_a < p.N;
-            const bool ok_b = rows_per_warp > 32 && n_b < p.N;
+            const PairProblem& pb = p.pr[tc.prob];
+            const int64_t G = pb.G;
+            const void* w_side = pb.w_side;
+            const bool ok_a = lane < rows_per_warp && n_a < pb.N;
+            const bool ok_b = rows_per_warp > 32 && n_b < pb.N;
             auto load_side = [&](int64_t n, int kb) -> uint32_t {
-                if (FMT == kHiF4) return ptx::ld_nc_u32(reinterpret_cast<const uint32_t*>(p.w_side) + n * G + kb);
-                return ptx::ld_nc_u16(reinterpret_cast<const uint16_t*>(p.w_side) + n * G + kb);
+                if (FMT == kHiF4) return ptx::ld_nc_u32(reinterpret_cast<const uint32_t*>(w_side) + n * G + kb);
+                return ptx::ld_nc_u16(reinterpret_cast<const uint16_t*>(w_side) + n * G + kb);
             };
             // first k-block of this tile that belongs to this group
             int i = (int)((grp + kExpGroups - (it0 % kExpGroups)) % kExpGroups);
@@ -609,6 +680,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     mw[q] = __shfl_sync(0xFFFFFFFFu, q < 8 ? ma : mb, rl & 31);
                     cw[q] = raw[(r_begin + rl) * 8 + chunk];
                 }
+                // The raw slot goes back to the TMA producer, whose next load overwrites it through the async proxy: the
+                // reads above (generic proxy) are ordered before that by a proxy fence.  Without it the loads of the
+                // later rows were found to execute after the arrive, late enough to read 128-byte pieces of the next
+                // k-block's codes (wrong expanded rows in groups of four).
+                ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&r_empty[sr]);
 #pragma unroll
@@ -630,11 +706,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         const int quad = warp & 3;
         constexpr int nchunks = TN / 32;
         int local_tile = 0;
-        SegIter<TN> si(p, pair, npairs);
+        SegIter<TN, NP> si(p, pair, npairs);
         TileCoord tc;
         while (si.next(tc)) {
             const int lt = local_tile++;
             if (tc.nkb == 0) continue;
+            const PairProblem& pb = p.pr[tc.prob];
+            const int64_t pM = pb.M, pN = pb.N, ldy = pb.ldy;
             const int buf = p.acc_bufs == 2 ? (lt & 1) : 0;
             const uint32_t use = p.acc_bufs == 2 ? (uint32_t)(lt >> 1) : (uint32_t)lt;
             if (quad == 0 && lane == 0) tr.begin();
@@ -648,7 +726,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             const int64_t m = tc.m0 + rank * kBM + quad * 32 + lane;
             // a warp whose 32 rows all lie past M (decode-sized calls fill a fraction of the 256-row tile) has
             // nothing to read or store: it only hands the accumulator back
-            const bool warp_has_rows = tc.m0 + rank * kBM + quad * 32 < p.M;
+            const bool warp_has_rows = tc.m0 + rank * kBM + quad * 32 < pM;
 #pragma unroll 1
             for (int cc = warp_has_rows ? 0 : nchunks - 1; cc < nchunks; ++cc) {
                 uint32_t v[32];
@@ -664,24 +742,24 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 if (!warp_has_rows) continue;
                 if (p.streamk && tc.partial) {
                     // fp32 slot [256][TN]; the sum reads rows below M only, so rows past M are not written
-                    if (m >= p.M) continue;
+                    if (m >= pM) continue;
                     float* dst = p.sk_slots + ((size_t)tc.slot * (2 * kBM) + rank * kBM + quad * 32 + lane) * TN + cc * 32;
 #pragma unroll
                     for (int j = 0; j < 32; j += 8)
                         ptx::st_global_v8(dst + j, v[j], v[j + 1], v[j + 2], v[j + 3], v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
                     continue;
                 }
-                if (m >= p.M) continue;
+                if (m >= pM) continue;
                 const int64_t nb = tc.n0 + cc * 32;
-                const int64_t left = p.N - nb;
+                const int64_t left = pN - nb;
                 if (left <= 0) continue;
                 if (p.splits > 1) {
-                    float* dst = p.partials + ((int64_t)tc.split * p.M + m) * p.N + nb;
+                    float* dst = p.partials + ((int64_t)tc.split * pM + m) * pN + nb;
                     if (left >= 32 && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 8)
                             ptx::st_global_v8(dst + j, v[j], v[j + 1], v[j + 2], v[j + 3], v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
-                    } else if (left >= 32 && (p.N & 3) == 0) {
+                    } else if (left >= 32 && (pN & 3) == 0) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
                             *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -691,7 +769,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                             if (j < left) dst[j] = __uint_as_float(v[j]);
                     }
                 } else if (p.out_f32) {
-                    float* dst = reinterpret_cast<float*>(p.Y) + m * p.ldy + nb;
+                    float* dst = reinterpret_cast<float*>(pb.Y) + m * ldy + nb;
                     if (left >= 32 && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 8)
@@ -706,7 +784,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                             if (j < left) dst[j] = __uint_as_float(v[j]);
                     }
                 } else {
-                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.Y) + m * p.ldy + nb;
+                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(pb.Y) + m * ldy + nb;
                     if (left >= 32) {
                         uint32_t o[16];
 #pragma unroll
@@ -744,10 +822,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         if (threadIdx.x == 0) tr.begin();
         // the activation ring is idle by now: its first bytes hold the slot list of the tile being summed
 #ifdef RESQ_TIMELINE
-        streamk_fixup<TN>(p, pair, npairs, (int)rank, abort_flag, reinterpret_cast<volatile int*>(tmem_slot + 2),
+        streamk_fixup<TN>(p, pair, (int)rank, abort_flag, reinterpret_cast<volatile int*>(tmem_slot + 2),
                           reinterpret_cast<int*>(ring_a), tl ? p.timeline + 512 + (int)rank * 16 + 8 : nullptr, t_kernel0);
 #else
-        streamk_fixup<TN>(p, pair, npairs, (int)rank, abort_flag, reinterpret_cast<volatile int*>(tmem_slot + 2),
+        streamk_fixup<TN>(p, pair, (int)rank, abort_flag, reinterpret_cast<volatile int*>(tmem_slot + 2),
                           reinterpret_cast<int*>(ring_a), nullptr, 0);
 #endif
         if (threadIdx.x == 0) { tr.end(13); EVT(7); }
@@ -773,60 +851,117 @@ std::atomic<int> g_expire_next_wait{0};
 constexpr int kStreamKTN = 256;    // tile width of the K-streamed schedule (two accumulators fit in tensor memory)
 constexpr int kStreamKMaxPairs = 74;
 
-template <int RES, int TN, int FMT, int NG>
-int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool streamk = false) {
-    constexpr int kExpGroups = NG;
-    constexpr int kAStage = a_stage_bytes(RES);
+// Tensor maps of one problem: activation image, residual operand (dense image, or compressed image + index metadata),
+// weights (packed codes, or plain bf16 rows).
+template <int RES, int TN, int FMT>
+int make_problem_maps(const GemmArgs& g, CUtensorMap* ta, CUtensorMap* tr, CUtensorMap* te, CUtensorMap* tw) {
     constexpr int nt = TN > kMaxBN ? 2 : 1;
-    constexpr int bn = TN / nt;
-    constexpr int half = bn / 2;
-    constexpr int my_rows = nt * half;
-    CUtensorMap ta, tr, te, tw;
-    int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.a_bf16, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)(g.lda ? g.lda : g.K) * 2,
+    constexpr int half = TN / nt / 2;
+    int rc = make_tmap_2d(ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.a_bf16, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)(g.lda ? g.lda : g.K) * 2,
                           kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
     if (RES == kResSparse24) {
         // compressed residual image [M, K/2] in boxes of 32 values x 128 rows (64-byte rows, 64-byte swizzle) and its
         // metadata blocks (2 KB per 128 rows x 128 K positions) as rows of 256 bytes
-        rc = make_tmap_2d(&tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.r_comp, (uint64_t)g.K / 2, (uint64_t)g.M, (uint64_t)g.K,
+        rc = make_tmap_2d(tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.r_comp, (uint64_t)g.K / 2, (uint64_t)g.M, (uint64_t)g.K,
                           kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_64B);
         if (rc) return rc;
-        rc = make_tmap_2d(&te, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.r_meta, 256, (uint64_t)g.meta_rows128 * (uint64_t)g.meta_ka * 8, 256,
+        rc = make_tmap_2d(te, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.r_meta, 256, (uint64_t)g.meta_rows128 * (uint64_t)g.meta_ka * 8, 256,
                           256, 8, CU_TENSOR_MAP_SWIZZLE_NONE);
     } else {
-        rc = make_tmap_2d(&tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, RES == kResDense ? g.r_bf16 : g.a_bf16, (uint64_t)g.K, (uint64_t)g.M,
+        rc = make_tmap_2d(tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, RES == kResDense ? g.r_bf16 : g.a_bf16, (uint64_t)g.K, (uint64_t)g.M,
                           (uint64_t)(g.lda ? g.lda : g.K) * 2, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
-        te = ta;
+        *te = *ta;
     }
     if (rc) return rc;
     if (FMT == kPlainW)
-        rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.w_bf16, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.ldw * 2, kBK,
-                          (uint32_t)half, CU_TENSOR_MAP_SWIZZLE_128B);
-    else
-        rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.w_codes, (uint64_t)g.K / 2, (uint64_t)g.N, (uint64_t)g.K / 2,
-                          kBK / 2, (uint32_t)half, CU_TENSOR_MAP_SWIZZLE_NONE);
-    if (rc) return rc;
-    PairParams p;
-    p.meta_ka = g.meta_ka;
-    p.w_side = g.w_side;
-    p.M = g.M;
-    p.N = g.N;
-    p.K = g.K;
-    const int G = (int)(g.K / kBK);
-    p.splits = splits;
-    p.kblocks_per_split = (G + splits - 1) / splits;
-    p.ntiles_m = (int)((g.M + 2 * kBM - 1) / (2 * kBM));
-    p.ntiles_n = (int)((g.N + TN - 1) / TN);
-    p.num_tiles = p.ntiles_m * p.ntiles_n * splits;
-    if (g.tile_limit > 0 && !streamk) p.num_tiles = std::min(p.num_tiles, g.tile_limit * splits);
-    p.acc_bufs = TN * 2 <= (RES == kResSparse24 ? kSpTmemCol : kTmemCols) ? 2 : 1;
-    if (RES == kResSparse24 && TN > kSpTmemCol) {
-        set_last_error("internal: no tensor-memory columns left for the sparse metadata (pair tile %d)", TN);
+        return make_tmap_2d(tw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.w_bf16, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.ldw * 2, kBK,
+                            (uint32_t)half, CU_TENSOR_MAP_SWIZZLE_128B);
+    return make_tmap_2d(tw, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.w_codes, (uint64_t)g.K / 2, (uint64_t)g.N, (uint64_t)g.K / 2,
+                        kBK / 2, (uint32_t)half, CU_TENSOR_MAP_SWIZZLE_NONE);
+}
+
+template <int TN>
+void fill_problem(PairProblem& pb, const GemmArgs& g) {
+    pb.w_side = g.w_side;
+    pb.Y = g.Y;
+    pb.ldy = g.ldy;
+    pb.M = (int)g.M;
+    pb.N = (int)g.N;
+    pb.G = (int)(g.K / kBK);
+    pb.ntiles_n = (int)((g.N + TN - 1) / TN);
+    pb.tile_base = 0;
+    pb.dealt_first = 0;
+    pb.unit_base = 0;
+    pb.meta_ka = (int)g.meta_ka;
+}
+
+// Ring depths from the shared-memory budget.  Ring slots: a multiple of the number of expander groups (group g works
+// on the slots s = g mod NG, so a slot is only ever written by one group).  With one slot per group the group's
+// expansion of a k-block and the MMAs that read its previous k-block alternate; with two slots per group they
+// overlap.  `kb_per_pair`: k-blocks a pair walks in a row (a deeper ring only pays once the pipeline is in steady state).
+template <int RES, int TN, int FMT, int NG, int NP>
+int pick_rings(PairParams<NP>& p, int64_t kb_per_pair, int* smem_bytes) {
+    constexpr int kExpGroups = NG;
+    constexpr int kAStage = a_stage_bytes(RES);
+    constexpr int nt = TN > kMaxBN ? 2 : 1;
+    constexpr int my_rows = nt * (TN / nt / 2);
+    constexpr int exp_stage = my_rows * 128, raw_stage = FMT == kPlainW ? 0 : my_rows * 32;  // (the kernel's raw ring is unused then)
+    const int fixed = 1024 + 1024;
+    const int slot_bytes = kAStage + exp_stage + raw_stage;
+    int per_group = (fixed + 2 * kExpGroups * slot_bytes <= kSmemBudget) ? 2 : 1;
+    per_group = std::max(1, std::min(per_group, env_int("RESQ_GEMM_SLOTS_PER_GROUP", 2)));
+    p.se = p.sr = p.sa = kExpGroups * per_group;
+    // If two full slots per group do not fit, two expanded-weight slots per group with shallower activation and
+    // raw-code rings may: what matters is that a group can expand its next k-block while the MMAs still read
+    // its previous one.
+    if (per_group == 1 && kb_per_pair >= 8 && env_int("RESQ_GEMM_DEEP_E", 1)) {
+        // three activation slots cover the latency of their loads, one raw-code slot per group is enough, and
+        // the rest goes to expanded-weight slots (any number: a k-block's barrier slot is k-block mod SE)
+        const int sa2 = env_int("RESQ_GEMM_MIN_SA", 3), sr2 = std::max(kExpGroups, std::min(env_int("RESQ_GEMM_MIN_SR", kExpGroups), kMaxRing));
+        const int left = kSmemBudget - fixed - sa2 * kAStage - sr2 * raw_stage;
+        const int se2 = std::min(std::min(left / exp_stage, 2 * kExpGroups), kMaxRing);
+        if (se2 > kExpGroups) {
+            p.se = se2;
+            p.sr = sr2;
+            p.sa = sa2;
+            // what is left over deepens the activation ring (its loads have ~2000 cycles of latency to cover)
+            while (p.sa < p.se && fixed + (p.sa + 1) * kAStage + p.se * exp_stage + p.sr * raw_stage <= kSmemBudget) ++p.sa;
+        }
+    }
+    if (p.sa > kMaxRing || fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage > kSmemBudget) {
+        set_last_error("internal: shared-memory rings do not fit (pair tile %d)", TN);
         return RESQ_ERR_CUDA;
     }
+    *smem_bytes = fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage;
+    return RESQ_OK;
+}
+
+template <int NG>
+void pair_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute (&attr)[2], int npairs, int smem_bytes, cudaStream_t stream) {
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)(2 * npairs), 1, 1);
+    cfg.blockDim = dim3(pair_threads(NG), 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = stream;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
+}
+
+template <int NP>
+void common_params(PairParams<NP>& p, const GemmArgs& g, bool streamk) {
     p.streamk = streamk ? 1 : 0;
     p.dp_tiles = 0;
+    p.sk_first = 0;
+    p.sk_hi = 0;
     p.sk_pairs = 0;
+    p.sk_units = 0;
     p.sk_slots = g.splitk_partials;
     p.sk_flags = g.sk_flags;
     p.sk_poll_limit = 1 << 20;
@@ -835,9 +970,7 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
         p.sk_poll_limit = 1 << 12;
         p.sk_extra = 1;
     }
-    p.Y = g.Y;
     p.out_f32 = g.out_dtype == RESQ_OUT_F32;
-    p.ldy = g.ldy;
     p.partials = g.splitk_partials;
     p.status = g.status;
 #ifdef RESQ_TIMELINE
@@ -848,15 +981,34 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
         p.timeline_first = env_int("RESQ_GEMM_TIMELINE_FIRST", 96);
     }
 #endif
-    auto kern = gemm_pair_kernel<RES, TN, FMT, NG>;
+}
+
+template <int RES, int TN, int FMT, int NG>
+int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool streamk = false) {
+    PairMaps<1> maps;
+    int rc = make_problem_maps<RES, TN, FMT>(g, &maps.a[0], &maps.r[0], &maps.e[0], &maps.w[0]);
+    if (rc) return rc;
+    PairParams<1> p;
+    memset(&p, 0, sizeof(p));
+    p.nprob = 1;
+    fill_problem<TN>(p.pr[0], g);
+    const int G = p.pr[0].G;
+    p.splits = splits;
+    p.kblocks_per_split = (G + splits - 1) / splits;
+    const int ntiles_m = (int)((g.M + 2 * kBM - 1) / (2 * kBM));
+    p.num_tiles = ntiles_m * p.pr[0].ntiles_n * splits;
+    if (g.tile_limit > 0 && !streamk) p.num_tiles = std::min(p.num_tiles, g.tile_limit * splits);
+    p.acc_bufs = TN * 2 <= (RES == kResSparse24 ? kSpTmemCol : kTmemCols) ? 2 : 1;
+    if (RES == kResSparse24 && TN > kSpTmemCol) {
+        set_last_error("internal: no tensor-memory columns left for the sparse metadata (pair tile %d)", TN);
+        return RESQ_ERR_CUDA;
+    }
+    common_params(p, g, streamk);
+    auto kern = gemm_pair_kernel<RES, TN, FMT, NG, 1>;
     rc = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), kSmemBudget, "cudaFuncSetAttribute(gemm pair)");
     if (rc) return rc;
     const int max_pairs = device_sm_count() / 2;
     int npairs = std::min(p.num_tiles, max_pairs);
-    if (streamk && (size_t)p.num_tiles * 2 * sizeof(unsigned int) > kWsFlags) {
-        set_last_error("internal: %d output tiles exceed the arrival counters of the K-streamed schedule", p.num_tiles);
-        return RESQ_ERR_CUDA;
-    }
     if (streamk) {
         // every pair gets at least two k-blocks; the pairs wait for one another at the end, so all of them
         // must be resident at once
@@ -876,55 +1028,13 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
             npairs = p.num_tiles * per_tile;
         }
     }
-    constexpr int exp_stage = my_rows * 128, raw_stage = FMT == kPlainW ? 0 : my_rows * 32;  // (the kernel's raw ring is unused then)
-    const int fixed = 1024 + 1024;
-    // Ring slots: a multiple of the number of expander groups (group g works on the slots s = g mod NG, so a slot
-    // is only ever written by one group).  With one slot per group the group's expansion of a k-block and the
-    // MMAs that read its previous k-block alternate; with two slots per group they overlap.  All three rings have
-    // the same depth (they share the slot's full / empty barriers).
-    const int slot_bytes = kAStage + exp_stage + raw_stage;
-    int per_group = (fixed + 2 * kExpGroups * slot_bytes <= kSmemBudget) ? 2 : 1;
-    per_group = std::max(1, std::min(per_group, env_int("RESQ_GEMM_SLOTS_PER_GROUP", 2)));
-    p.se = p.sr = p.sa = kExpGroups * per_group;
-    // If two full slots per group do not fit, two expanded-weight slots per group with shallower activation and
-    // raw-code rings may: what matters is that a group can expand its next k-block while the MMAs still read
-    // its previous one.
-    // (Not for a handful of k-blocks per pair: the deeper ring only pays once the pipeline is in steady state.)
     const int64_t kb_per_pair = streamk ? ((int64_t)p.num_tiles * G + npairs - 1) / npairs : p.kblocks_per_split;
-    if (per_group == 1 && kb_per_pair >= 8 && env_int("RESQ_GEMM_DEEP_E", 1)) {
-        // three activation slots cover the latency of their loads, one raw-code slot per group is enough, and
-        // the rest goes to expanded-weight slots (any number: a k-block's barrier slot is k-block mod SE)
-        const int sa2 = env_int("RESQ_GEMM_MIN_SA", 3), sr2 = std::max(kExpGroups, std::min(env_int("RESQ_GEMM_MIN_SR", kExpGroups), kMaxRing));
-        const int left = kSmemBudget - fixed - sa2 * kAStage - sr2 * raw_stage;
-        const int se2 = std::min(std::min(left / exp_stage, 2 * kExpGroups), kMaxRing);
-        if (se2 > kExpGroups) {
-            p.se = se2;
-            p.sr = sr2;
-            p.sa = sa2;
-            // what is left over deepens the activation ring (its loads have ~2000 cycles of latency to cover)
-            while (p.sa < p.se && fixed + (p.sa + 1) * kAStage + p.se * exp_stage + p.sr * raw_stage <= kSmemBudget) ++p.sa;
-        }
-    }
-    if (p.sa > kMaxRing || fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage > kSmemBudget) {
-        set_last_error("internal: shared-memory rings do not fit (pair tile %d)", TN);
-        return RESQ_ERR_CUDA;
-    }
-    const int smem_bytes = fixed + p.sa * kAStage + p.se * exp_stage + p.sr * raw_stage;
+    int smem_bytes = 0;
+    rc = pick_rings<RES, TN, FMT, NG>(p, kb_per_pair, &smem_bytes);
+    if (rc) return rc;
     cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = dim3((unsigned)(2 * npairs), 1, 1);
-    cfg.blockDim = dim3(pair_threads(NG), 1, 1);
-    cfg.dynamicSmemBytes = (size_t)smem_bytes;
-    cfg.stream = stream;
     cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = pdl_enabled() ? 2 : 1;
+    pair_launch_config<NG>(cfg, attr, npairs, smem_bytes, stream);
     cudaError_t e;
     if (streamk) {
         int max_clusters = 0;  // co-resident clusters of this variant with this much shared memory
@@ -940,15 +1050,216 @@ int launch_pair_variant(const GemmArgs& g, int splits, cudaStream_t stream, bool
         }
         // more tiles than pairs: whole rounds of tiles first, only the last, incomplete round is dealt out by k-blocks
         if (p.num_tiles > npairs) p.dp_tiles = (p.num_tiles / npairs) * npairs;
-        p.sk_pairs = (int)std::max<int64_t>(1, std::min<int64_t>(npairs, (int64_t)(p.num_tiles - p.dp_tiles) * G / 2));
+        const int dealt_tiles = p.num_tiles - p.dp_tiles;
+        p.pr[0].dealt_first = p.dp_tiles;
+        p.sk_units = (int64_t)dealt_tiles * G;
+        p.sk_pairs = (int)std::max<int64_t>(1, std::min<int64_t>(npairs, p.sk_units / 2));
+        if ((size_t)dealt_tiles * 2 * sizeof(unsigned int) > kWsFlags) {
+            set_last_error("internal: %d dealt tiles exceed the arrival counters of the K-streamed schedule", dealt_tiles);
+            return RESQ_ERR_CUDA;
+        }
     }
     {
         LaunchScope scope(kKindGemm, stream);
-        e = cudaLaunchKernelEx(&cfg, kern, ta, tr, te, tw, p);
+        e = cudaLaunchKernelEx(&cfg, kern, maps, p);
     }
     if (e != cudaSuccess) return cuda_fail(e, "gemm_pair_kernel launch");
     if (streamk) return RESQ_OK;
     return launch_splitk_reduce(g, splits, stream);
+}
+
+// ---- a group of independent problems in one launch ----------------------------------------------------------
+// The tiles of all problems (256 x 256) form one list; the launch walks it with the K-streamed schedule.  Which
+// tiles are computed whole and which are dealt out by k-blocks is chosen here, by simulating the candidates:
+// a pair's time is its k-blocks plus a fixed cost per partial tile it writes and helps to sum.
+struct GroupPlan {
+    int order[kMaxGroup];   // problems in the order of the tile list (ascending K: whole tiles first)
+    int dp_tiles, sk_first, sk_hi, sk_pairs;
+    int64_t sk_units;
+    double cost;
+};
+
+GroupPlan plan_group(const GemmArgs* g, int count, int npairs) {
+    constexpr double kPartialCost = 10.0;  // a partial tile (fp32 write, wait, share of the sum) in k-block periods
+    GroupPlan best;
+    memset(&best, 0, sizeof(best));
+    best.cost = 1e300;
+    int order[kMaxGroup];
+    for (int i = 0; i < count; ++i) order[i] = i;
+    std::stable_sort(order, order + count, [&](int a, int b) { return g[a].K < g[b].K; });
+    int T[kMaxGroup], G[kMaxGroup], base[kMaxGroup + 1];
+    base[0] = 0;
+    for (int i = 0; i < count; ++i) {
+        const GemmArgs& a = g[order[i]];
+        T[i] = (int)(((a.M + 2 * kBM - 1) / (2 * kBM)) * ((a.N + kStreamKTN - 1) / kStreamKTN));
+        G[i] = (int)(a.K / kBK);
+        base[i + 1] = base[i] + T[i];
+    }
+    const int total = base[count];
+    auto g_of_tile = [&](int t) { int q = 0; while (q + 1 < count && t >= base[q + 1]) ++q; return G[q]; };
+    // candidates for the number of whole tiles: the problem boundaries, and each rounded down to whole rounds
+    int cand[2 * kMaxGroup + 2], nc = 0;
+    for (int i = 0; i <= count; ++i) {
+        cand[nc++] = base[i];
+        cand[nc++] = base[i] / npairs * npairs;
+    }
+    std::vector<double> whole((size_t)npairs);
+    for (int ci = 0; ci < nc; ++ci) {
+        const int dp = cand[ci];
+        std::fill(whole.begin(), whole.end(), 0.0);
+        for (int t = 0; t < dp; ++t) whole[(size_t)(t % npairs)] += g_of_tile(t);
+        int64_t D = 0;
+        for (int t = dp; t < total; ++t) D += g_of_tile(t);
+        const int b = dp % npairs;
+        // units per pair of the first b pairs (which hold one whole tile more): balance the two classes
+        for (int pass = 0; pass < 2; ++pass) {
+            int H = 0;
+            if (pass == 1) {
+                if (b == 0 || D == 0) break;
+                const double extra = whole[0] - whole[(size_t)(npairs - 1)];
+                const double h = ((double)D - extra * (npairs - b)) / npairs;  // H with equal loads
+                H = (int)h;
+                if (H < 4) break;
+            }
+            const int64_t rest = D - (int64_t)b * H;
+            int sk_pairs = b == npairs ? 0 : npairs - b;
+            if (D > 0) {
+                if (sk_pairs == 0 || rest < 0) continue;
+                sk_pairs = (int)std::max<int64_t>(1, std::min<int64_t>(sk_pairs, rest / 2));
+                if (rest == 0) continue;
+            }
+            // simulate: dealt ranges and the partial tiles they cut
+            double worst = 0.0;
+            auto beg = [&](int q) -> int64_t {
+                if (q < b) return (int64_t)q * H;
+                if (q >= b + sk_pairs) return D;
+                return (int64_t)b * H + (int64_t)(q - b) * rest / sk_pairs;
+            };
+            // tile boundaries of the dealt units (prefix sums)
+            std::vector<int64_t> tb;
+            tb.push_back(0);
+            for (int t = dp; t < total; ++t) tb.push_back(tb.back() + g_of_tile(t));
+            for (int q = 0; q < npairs; ++q) {
+                double c = whole[(size_t)q];
+                if (D > 0) {
+                    const int64_t u0 = beg(q), u1 = beg(q + 1);
+                    if (u1 > u0) {
+                        c += (double)(u1 - u0);
+                        const bool cut0 = !std::binary_search(tb.begin(), tb.end(), u0);
+                        const bool cut1 = !std::binary_search(tb.begin(), tb.end(), u1);
+                        // first and last tile of the range: partial if the range cuts them
+                        const auto i0 = std::upper_bound(tb.begin(), tb.end(), u0) - tb.begin() - 1;
+                        const auto i1 = std::upper_bound(tb.begin(), tb.end(), u1 - 1) - tb.begin() - 1;
+                        int partial = 0;
+                        if (i0 == i1) partial = (cut0 || cut1) ? 1 : 0;
+                        else partial = (cut0 ? 1 : 0) + (cut1 ? 1 : 0);
+                        c += kPartialCost * partial;
+                    }
+                }
+                worst = std::max(worst, c);
+            }
+            if (worst < best.cost) {
+                best.cost = worst;
+                best.dp_tiles = dp;
+                best.sk_first = D > 0 ? b : 0;
+                best.sk_hi = H;
+                best.sk_pairs = D > 0 ? sk_pairs : 0;
+                best.sk_units = D;
+            }
+        }
+    }
+    for (int i = 0; i < count; ++i) best.order[i] = order[i];
+    return best;
+}
+
+template <int RES, int FMT>
+int launch_pair_group(const GemmArgs* g, int count, cudaStream_t stream) {
+    constexpr int TN = kStreamKTN, NG = 3, NP = kMaxGroup;
+    if (count < 1 || count > kMaxGroup) {
+        set_last_error("a group holds 1 to %d problems (got %d)", kMaxGroup, count);
+        return RESQ_ERR_SHAPE;
+    }
+    auto kern = gemm_pair_kernel<RES, TN, FMT, NG, NP>;
+    int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), kSmemBudget, "cudaFuncSetAttribute(gemm pair group)");
+    if (rc) return rc;
+    PairParams<NP> p;
+    memset(&p, 0, sizeof(p));
+    int64_t units = 0;
+    for (int i = 0; i < count; ++i)
+        units += ((g[i].M + 2 * kBM - 1) / (2 * kBM)) * ((g[i].N + TN - 1) / TN) * (g[i].K / kBK);
+    p.splits = 1;
+    p.acc_bufs = 2;
+    common_params(p, g[0], true);
+    int npairs = (int)std::min<int64_t>(std::min(device_sm_count() / 2, kStreamKMaxPairs), std::max<int64_t>(1, units / 2));
+    int smem_bytes = 0;
+    rc = pick_rings<RES, TN, FMT, NG>(p, (units + npairs - 1) / npairs, &smem_bytes);
+    if (rc) return rc;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    pair_launch_config<NG>(cfg, attr, npairs, smem_bytes, stream);
+    int max_clusters = 0;  // the pairs wait for one another at the end: all of them must be resident at once
+    rc = max_active_clusters(reinterpret_cast<const void*>(kern), &cfg, &max_clusters);
+    if (rc) return rc;
+    if (npairs > max_clusters) {
+        npairs = max_clusters;
+        cfg.gridDim = dim3((unsigned)(2 * npairs), 1, 1);
+    }
+    if (npairs < 1) {
+        set_last_error("gemm pair kernel: no cluster of two CTAs fits on this device");
+        return RESQ_ERR_CUDA;
+    }
+    const GroupPlan plan = plan_group(g, count, npairs);
+    PairMaps<NP> maps;
+    memset(&maps, 0, sizeof(maps));
+    p.nprob = count;
+    int tile_base = 0;
+    int64_t unit_base = 0;
+    for (int i = 0; i < count; ++i) {
+        const GemmArgs& a = g[plan.order[i]];
+        rc = make_problem_maps<RES, TN, FMT>(a, &maps.a[i], &maps.r[i], &maps.e[i], &maps.w[i]);
+        if (rc) return rc;
+        fill_problem<TN>(p.pr[i], a);
+        const int tiles = (int)((a.M + 2 * kBM - 1) / (2 * kBM)) * p.pr[i].ntiles_n;
+        p.pr[i].tile_base = tile_base;
+        p.pr[i].dealt_first = std::min(std::max(tile_base, plan.dp_tiles), tile_base + tiles);
+        p.pr[i].unit_base = unit_base;
+        unit_base += (int64_t)(tile_base + tiles - p.pr[i].dealt_first) * p.pr[i].G;
+        tile_base += tiles;
+    }
+    for (int i = count; i < NP; ++i) {  // unused entries: never matched by the lookups
+        maps.a[i] = maps.a[0];
+        maps.r[i] = maps.r[0];
+        maps.e[i] = maps.e[0];
+        maps.w[i] = maps.w[0];
+        p.pr[i] = p.pr[count - 1];
+        p.pr[i].tile_base = tile_base;
+        p.pr[i].dealt_first = tile_base;
+        p.pr[i].unit_base = unit_base;
+    }
+    p.num_tiles = tile_base;
+    p.dp_tiles = plan.dp_tiles;
+    p.sk_first = plan.sk_first;
+    p.sk_hi = plan.sk_hi;
+    p.sk_pairs = plan.sk_pairs;
+    p.sk_units = plan.sk_units;
+    if (unit_base != plan.sk_units) {
+        set_last_error("internal: group schedule is inconsistent (%lld dealt units planned, %lld laid out)", (long long)plan.sk_units,
+                       (long long)unit_base);
+        return RESQ_ERR_CUDA;
+    }
+    if ((size_t)(p.num_tiles - p.dp_tiles) * 2 * sizeof(unsigned int) > kWsFlags) {
+        set_last_error("internal: %d dealt tiles exceed the arrival counters of the K-streamed schedule", p.num_tiles - p.dp_tiles);
+        return RESQ_ERR_CUDA;
+    }
+    if (env_int("RESQ_GEMM_DEBUG", 0) & 1)
+        fprintf(stderr, "resq gemm group: %d problems, %d tiles, %d pairs: %d whole tiles, %lld dealt units (first %d pairs take %d each, %d pairs share the rest)\n",
+                count, p.num_tiles, npairs, p.dp_tiles, (long long)p.sk_units, p.sk_first, p.sk_hi, p.sk_pairs);
+    cudaError_t e;
+    {
+        LaunchScope scope(kKindGemm, stream);
+        e = cudaLaunchKernelEx(&cfg, kern, maps, p);
+    }
+    return e == cudaSuccess ? RESQ_OK : cuda_fail(e, "gemm_pair_kernel (group) launch");
 }
 
 template <int RES, int FMT>
@@ -987,6 +1298,14 @@ int streamk_fmt(const GemmArgs& g, cudaStream_t stream) {
     }
 }
 template <int FMT>
+int group_fmt(const GemmArgs* g, int count, cudaStream_t stream) {
+    switch (res_mode(g[0])) {
+        case kResSparse24: return launch_pair_group<kResSparse24, FMT>(g, count, stream);
+        case kResDense: return launch_pair_group<kResDense, FMT>(g, count, stream);
+        default: return launch_pair_group<kResNone, FMT>(g, count, stream);
+    }
+}
+template <int FMT>
 int pair_fmt(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {
     switch (res_mode(g)) {
         case kResSparse24: return dispatch_pair<kResSparse24, FMT>(g, tn, splits, stream);
@@ -1012,6 +1331,17 @@ int launch_gemm_pair_plainw(const GemmArgs& g, int tn, int splits, bool streamk,
 
 int launch_gemm_pair_streamk(const GemmArgs& g, cudaStream_t stream) {
     return g.fmt == kMXFP4 ? streamk_fmt<kMXFP4>(g, stream) : streamk_fmt<kHiF4>(g, stream);
+}
+
+// All problems share the weight format, the residual mode, the output type, the status word, the arrival counters and
+// the partial-tile slots of g[0].
+int launch_gemm_pair_group(const GemmArgs* g, int count, cudaStream_t stream) {
+    for (int i = 1; i < count; ++i)
+        if (g[i].fmt != g[0].fmt || res_mode(g[i]) != res_mode(g[0]) || g[i].out_dtype != g[0].out_dtype || g[i].w_bf16) {
+            set_last_error("internal: the problems of a group must share format, residual mode and output type");
+            return RESQ_ERR_CUDA;
+        }
+    return g[0].fmt == kMXFP4 ? group_fmt<kMXFP4>(g, count, stream) : group_fmt<kHiF4>(g, count, stream);
 }
 
 int launch_gemm_pair(const GemmArgs& g, int tn, int splits, cudaStream_t stream) {

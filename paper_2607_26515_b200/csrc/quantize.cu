@@ -213,19 +213,17 @@ __device__ __forceinline__ uint4 rht64_bf16x8(const uint4& raw, unsigned long lo
 // COMP (2:4 only): the residual image leaves in compressed form with its index metadata (a.r_comp, a.r_meta).
 // PROD = 3: the input is the randomized Hadamard transform of X (rht64_bf16x8).  PROD = 1: the input is x = bf16(SiLU(g) * u) of a.X (g) and a.X_up (u); PROD = 2: x = bf16((X * r[m]) * gamma[k])
 // with the row scales of rmsnorm_row_scale_kernel; computed on the fly, never stored.
+// Body of the chunk-per-lane kernel for the CTA (bx, by) of a grid of gx x gy CTAs over one problem.
 template <int FMT, bool RESIDUAL, bool IMG, bool COMP = false, int PROD = 0>
-__global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int rows_per_cta) {
-    pdl_wait();     // nothing below may touch global memory before the previous kernel of the stream is done
-    pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
-    if (a.clear_words && blockIdx.x == 0 && blockIdx.y == 0)
+__device__ __forceinline__ void quant_stream_body(const QuantArgs& a, int rows_per_cta, int bx, int by, int gx, int gy) {
+    if (a.clear_words && bx == 0 && by == 0)
         for (int i = threadIdx.x; i < a.n_clear_words; i += blockDim.x) a.clear_words[i] = 0u;
     if constexpr (COMP)
-        fill_meta_pad(a, ((int64_t)blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x,
-                      (int64_t)gridDim.x * gridDim.y * blockDim.x);
+        fill_meta_pad(a, ((int64_t)by * gx + bx) * blockDim.x + threadIdx.x, (int64_t)gx * gy * blockDim.x);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t k0 = ((int64_t)blockIdx.y * kWarpsPerCta + warp) * kColsPerWarp + lane * 8;
+    const int64_t k0 = ((int64_t)by * kWarpsPerCta + warp) * kColsPerWarp + lane * 8;
     const bool active = k0 < a.K;  // whole blocks are active or not (K is a multiple of the block size)
-    const int64_t m_begin = (int64_t)blockIdx.x * rows_per_cta;
+    const int64_t m_begin = (int64_t)bx * rows_per_cta;
     const int64_t m_end = min(a.M, m_begin + rows_per_cta);
     const int pattern = a.pattern;
     const unsigned grp = FMT == kHiF4 ? 0xFFu << (lane & 24) : 0xFu << (lane & 28);
@@ -410,6 +408,34 @@ __global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int
 #pragma unroll
         for (int i = 0; i < 8; ++i) atomicAdd(&a.scores[k0 + i], chan_acc[i]);
     }
+}
+
+template <int FMT, bool RESIDUAL, bool IMG, bool COMP = false, int PROD = 0>
+__global__ void __launch_bounds__(kThreads) quant_stream_kernel(QuantArgs a, int rows_per_cta) {
+    pdl_wait();     // nothing below may touch global memory before the previous kernel of the stream is done
+    pdl_trigger();  // the next kernel (the GEMM) may be scheduled and run its set-up
+    quant_stream_body<FMT, RESIDUAL, IMG, COMP, PROD>(a, rows_per_cta, (int)blockIdx.x, (int)blockIdx.y, (int)gridDim.x, (int)gridDim.y);
+}
+
+// The same pass over a group of independent activations in one launch (the quantizer side of *_resq_linear_group):
+// CTA b of the grid works on problem q with block_base[q] <= b < block_base[q + 1], as CTA (local % gx, local / gx) of
+// that problem's own grid.
+struct QuantGroup {
+    QuantArgs a[kMaxQuantGroup];
+    int rows_per_cta[kMaxQuantGroup], gx[kMaxQuantGroup], gy[kMaxQuantGroup];
+    int block_base[kMaxQuantGroup + 1];
+    int count;
+};
+
+template <int FMT, bool RESIDUAL, bool IMG, bool COMP>
+__global__ void __launch_bounds__(kThreads) quant_stream_group_kernel(const __grid_constant__ QuantGroup g) {
+    pdl_wait();
+    pdl_trigger();
+    int q = 0;
+#pragma unroll 1
+    while (q + 1 < g.count && (int)blockIdx.x >= g.block_base[q + 1]) ++q;
+    const int local = (int)blockIdx.x - g.block_base[q];
+    quant_stream_body<FMT, RESIDUAL, IMG, COMP, 0>(g.a[q], g.rows_per_cta[q], local % g.gx[q], local / g.gx[q], g.gx[q], g.gy[q]);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1965,6 +1991,45 @@ int launch_quantize(int fmt, const QuantArgs& a_in, cudaStream_t stream) {
     if (rc) return rc;
     if (global_sel) rc = launch_global_select(a, nscore, stream);
     return rc;
+}
+
+// One launch for a group of activations with a row-local selection (NONE, DENSE, n:4) that feed the GEMM (images).
+int launch_quantize_group(int fmt, const QuantArgs* a_in, int count, cudaStream_t stream) {
+    if (count < 1 || count > kMaxQuantGroup) {
+        set_last_error("a group holds 1 to %d problems (got %d)", kMaxQuantGroup, count);
+        return RESQ_ERR_SHAPE;
+    }
+    QuantGroup g;
+    memset(&g, 0, sizeof(g));
+    g.count = count;
+    const int pattern = a_in[0].pattern;
+    const bool residual = pattern != RESQ_S_NONE, comp = a_in[0].r_comp != nullptr;
+    int blocks = 0;
+    for (int i = 0; i < count; ++i) {
+        QuantArgs a = a_in[i];
+        if (a.keep_quarters < 1 || a.keep_quarters > 3) a.keep_quarters = 2;
+        if (a.pattern != pattern || (pattern != RESQ_S_NONE && pattern != RESQ_S_DENSE && pattern != RESQ_S_2_4) || !a.a_bf16 ||
+            (a.r_comp != nullptr) != comp || a.X_up || a.gamma || a.rht || (comp && a.keep_quarters != 2)) {
+            set_last_error("internal: a quantizer group takes one row-local pattern and the GEMM operand images");
+            return RESQ_ERR_CUDA;
+        }
+        g.a[i] = a;
+        g.rows_per_cta[i] = pick_rows_per_cta(a.M, a.K, pattern);
+        g.gx[i] = (int)((a.M + g.rows_per_cta[i] - 1) / g.rows_per_cta[i]);
+        g.gy[i] = (int)((a.K + (int64_t)kWarpsPerCta * kColsPerWarp - 1) / ((int64_t)kWarpsPerCta * kColsPerWarp));
+        g.block_base[i] = blocks;
+        blocks += g.gx[i] * g.gy[i];
+    }
+    for (int i = count; i <= kMaxQuantGroup; ++i) g.block_base[i] = blocks;
+    void (*kern)(QuantGroup);
+    if (fmt == kHiF4)
+        kern = residual ? (comp ? quant_stream_group_kernel<kHiF4, true, true, true> : quant_stream_group_kernel<kHiF4, true, true, false>)
+                        : quant_stream_group_kernel<kHiF4, false, true, false>;
+    else
+        kern = residual ? (comp ? quant_stream_group_kernel<kMXFP4, true, true, true> : quant_stream_group_kernel<kMXFP4, true, true, false>)
+                        : quant_stream_group_kernel<kMXFP4, false, true, false>;
+    LaunchScope scope(kKindQuant, stream);
+    return cuda_fail(launch_kernel(kern, dim3((unsigned)blocks), dim3(kThreads), 0, stream, g), "quant_stream_group_kernel launch");
 }
 
 int launch_dequantize(int fmt, const uint8_t* codes, const void* side, int64_t rows, int64_t K, float* out,

@@ -597,3 +597,59 @@ def test_bounded_wait_expires_and_the_context_stays_usable():
     m.debug_expire_next_wait(False)
     y = m.resq_linear(x, wc, ws, pattern, out_dtype=torch.float32, workspace=work)
     assert m.check(work) == 0
+
+
+GROUPS = {
+    # the four linears of a 3B block at decode size (gate_up narrowed for the oracle's sake): short and long K mixed
+    "block": ([(256, 2048, 2560), (256, 2048, 2048), (256, 2048, 4352), (256, 11008, 2048)], oracle.S_2_4, "hif4", torch.float32),
+    # different M, ragged N, fewer rows than one MMA tile
+    "ragged": ([(64, 1024, 512), (300, 512, 1000), (16, 2048, 264)], oracle.S_DENSE, "hif4", torch.bfloat16),
+    "single": ([(160, 704, 328)], oracle.S_NONE, "hif4", torch.float32),
+    "eight": ([(32 * (i + 1), 256 * (1 + i % 3), 136 * (i + 1)) for i in range(8)], oracle.S_2_4, "mxfp4", torch.float32),
+    # more whole tiles than CTA pairs, and a long-K problem whose k-blocks are dealt out
+    "many-tiles": ([(512, 512, 9728), (256, 512, 3000), (256, 8192, 512)], oracle.S_2_4, "hif4", torch.bfloat16),
+    "quarter": ([(128, 1024, 384), (256, 1024, 768)], oracle.keep_quarters(oracle.S_2_4, 1), "hif4", torch.float32),
+}
+
+
+@pytest.mark.parametrize("name", sorted(GROUPS))
+def test_linear_group_matches_the_oracle_problem_by_problem(name):
+    """*_resq_linear_group: one quantizer launch and one GEMM launch over the tiles of all problems; every problem is
+    checked element by element against the oracle, and a second run must reproduce the first bit for bit (the partial
+    tiles are summed in a fixed order)."""
+    m = rq()
+    shapes, pattern, fmt, out_dtype = GROUPS[name]
+    tensors, problems = [], []
+    for i, (M, K, N) in enumerate(shapes):
+        xb, wb = synth_xw(100 * len(name) + i, M, K, N, n_out=max(1, K // 512))
+        wc, ws = m.pack_weight(to_dev(wb), fmt)
+        tensors.append((xb, wb))
+        problems.append((to_dev(xb), wc, ws))
+    work = m.alloc_workspace(m.resq_group_workspace_bytes(problems, pattern, fmt, out_dtype))
+    launches0 = m.kernel_launches()
+    ys = m.resq_linear_group(problems, pattern, fmt, out_dtype=out_dtype, workspace=work)
+    assert m.kernel_launches() - launches0 == 2          # one quantizer kernel, one GEMM kernel
+    assert m.check(work) == 0, m.last_error()
+    first = [y.clone() for y in ys]
+    ys2 = m.resq_linear_group([p + (y,) for p, y in zip(problems, ys)], pattern, fmt, out_dtype=out_dtype, workspace=work)
+    assert m.check(work) == 0, m.last_error()
+    for (xb, wb), y, y1 in zip(tensors, ys2, first):
+        assert torch.equal(y, y1)
+        want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern, fmt)
+        check_close(y.float().cpu().numpy(), want["y"], want["abs_sum"], bf16_out=out_dtype == torch.bfloat16)
+
+
+def test_linear_group_argument_errors():
+    m = rq()
+    xb, wb = synth_xw(3, 64, 256, 128)
+    wc, ws = m.pack_weight(to_dev(wb))
+    x = to_dev(xb)
+    with pytest.raises(m.ResqError) as e:
+        m.resq_linear_group([(x, wc, ws)], oracle.S_CHAN50)     # tensor-wide selections run through the single call
+    assert e.value.status == 5
+    with pytest.raises(m.ResqError) as e:
+        m.resq_linear_group([(x, wc, ws)] * 9, oracle.S_2_4, workspace=m.alloc_workspace(1 << 20))
+    assert e.value.status == 2
+    with pytest.raises(m.ResqError) as e:
+        m.resq_linear_group([(x, wc, ws)], oracle.S_2_4, workspace=m.alloc_workspace(4096))
+    assert e.value.status == 4
