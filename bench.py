@@ -190,8 +190,9 @@ def time_oracle(cfg, pattern, fmt, rows, tensors):
 class Workload:
     """The tensors of one configuration on the device, and the step over its layers."""
 
-    def __init__(self, rq, torch, dev, cfg, pattern, fmt, out_dtype, host_copies=False):
+    def __init__(self, rq, torch, dev, cfg, pattern, fmt, out_dtype, host_copies=False, group=False):
         self.rq, self.torch, self.dev, self.cfg, self.pattern, self.fmt = rq, torch, dev, cfg, pattern, fmt
+        self.group = group
         self.layers = []
         w_bytes_total = 0
         for li, spec in enumerate(cfg.layers):
@@ -218,6 +219,11 @@ class Workload:
             if host_copies:
                 L["y_host"] = torch.empty((cfg.M, spec.N), dtype=out_dtype).pin_memory()
                 L["x_stage"] = torch.empty_like(L["x_sets"][0])
+        if group:  # the layers of a step as one *_resq_linear_group call (one quantizer launch, one GEMM launch)
+            self.group_problems = [[(L["x_sets"][k], L["w_sets"][k][0], L["w_sets"][k][1], L["y"]) for L in self.layers]
+                                   for k in range(n_sets)]
+            self.group_work = rq.alloc_workspace(rq.resq_group_workspace_bytes(self.group_problems[0], pattern, fmt, out_dtype), dev)
+        self.out_dtype = out_dtype
         self.l2_note = (f"rotating {n_sets} copies of weights and activations "
                         f"({n_sets * (w_bytes_total + act_bytes) / 1e6:.0f} MB > 126 MB L2)")
         self.w_bytes_total = w_bytes_total
@@ -227,11 +233,19 @@ class Workload:
 
     def step(self, i):
         k = i % self.n_sets
+        if self.group:
+            self.rq.resq_linear_group(self.group_problems[k], self.pattern, self.fmt, out_dtype=self.out_dtype,
+                                      workspace=self.group_work)
+            return
         for L in self.layers:
             wc, ws = L["w_sets"][k]
             self.rq.resq_linear(L["x_sets"][k], wc, ws, self.pattern, self.fmt, Y=L["y"], workspace=L["work"])
 
     def check(self):
+        if self.group:
+            if self.rq.check(self.group_work) != 0:
+                raise SystemExit("device status: " + self.rq.last_error())
+            return
         for L in self.layers:
             if self.rq.check(L["work"]) != 0:
                 raise SystemExit("device status: " + self.rq.last_error())
@@ -298,6 +312,8 @@ def main():
     ap.add_argument("--tokens", type=int, default=None, help="override M (profiling aid; not the benchmark workload)")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the end-to-end and per-kernel passes (profiling aid)")
     ap.add_argument("--headline-only", action="store_true", help="skip per_config / per_pattern / sweeps")
+    ap.add_argument("--group", action="store_true",
+                    help="run the step's layers as one *_resq_linear_group call (row-local selections only)")
     ap.add_argument("--quantizer-sweep", action="store_true",
                     help="only the bandwidth sweep of *_quantize_act over M x K (table on stderr and one JSON line)")
     ap.add_argument("--accuracy-contrast", action="store_true",
@@ -472,9 +488,9 @@ def main():
             return p * 4.0, src + " x 4 (nominal FP4 : bf16 ratio)"
         return p, src
 
-    def measure(cfg_, pattern_, fmt_, steps, sampler=None, e2e=False, verbose=False):
+    def measure(cfg_, pattern_, fmt_, steps, sampler=None, e2e=False, verbose=False, group=False):
         """Times `steps` steps of one workload (value), then the per-kernel pass; optionally the end-to-end pass."""
-        wl = Workload(rq, torch, dev, cfg_, pattern_, fmt_, out_dtype, host_copies=e2e)
+        wl = Workload(rq, torch, dev, cfg_, pattern_, fmt_, out_dtype, host_copies=e2e, group=group)
         for i in range(warmup):
             wl.step(i)
         wl.check()
@@ -505,7 +521,7 @@ def main():
             "gbs": world * wl.bytes_step / (ms_per_step * 1e-3) / 1e9,
             "clocks": clocks, "l2": wl.l2_note, "flops_step": wl.flops_step, "bytes_step": wl.bytes_step,
         }
-        if not args.skip_e2e:
+        if not args.skip_e2e and not group:
             per_layer = wl.profile(min(steps, 10))
             kinds = ("quantize", "select", "gemm", "splitk_reduce")
             tot = {k: sum(pl[k][0] for pl in per_layer) for k in kinds}
@@ -610,10 +626,13 @@ def main():
         time.sleep(0.25)
 
     # ---- headline workload
-    head = measure(cfg, pattern, fmt, args.steps, sampler=sampler, e2e=not args.skip_e2e, verbose=args.verbose)
+    head = measure(cfg, pattern, fmt, args.steps, sampler=sampler, e2e=not args.skip_e2e and not args.group, verbose=args.verbose,
+                   group=args.group)
+    if args.group:
+        config_desc["call"] = "one *_resq_linear_group call per step"
     config_desc["l2"] = head["l2"]
     config_desc["launch"] = "one CUDA graph replay per step" if use_graph else "eager launches"
-    if args.skip_e2e:
+    if args.skip_e2e or args.group:
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": head["tflops"], "unit": "TFLOP/s", "ms_per_step": head["ms_per_step"],
                               "config": config_desc, "note": "profiling aid run: no e2e / roofline passes"}))
@@ -643,7 +662,14 @@ def main():
             c = CONFIGS[ci]
             r = measure(c, c.patterns[0], "hif4", n_small, sampler=sampler)
             rf = gemm_roofline(r, "hif4")
+            grouped = None
+            if c.patterns[0] in (0, 1, 2) and c.M <= 1024:  # a row-local selection at decode size: also as one grouped call
+                rg = measure(c, c.patterns[0], "hif4", n_small, group=True)
+                grouped = {"ms_per_step": rg["ms_per_step"], "tflops": rg["tflops"], "launches_per_step": rg["launches_per_step"],
+                           "frac_of_bf16_burst": rg["tflops"] / peaks["bf16_tflops"],
+                           "call": "hif4_resq_linear_group over the step's layers (one quantizer launch, one GEMM launch)"}
             per_config.append({"config": ci, "name": c.name, "M": c.M, "pattern": PATTERN_NAMES[c.patterns[0]], "format": "hif4",
+                               "grouped": grouped,
                                "ms_per_step": r["ms_per_step"], "tflops": r["tflops"], "gb_per_s": r["gbs"],
                                "gemm_frac_of_peak": rf["frac"], "peak_source": rf["peak_source"],
                                "quantizer_share": rf["quantizer_share_of_kernel_time"], "select_share": rf["select_share_of_kernel_time"],
@@ -672,9 +698,13 @@ def main():
         for M in (16, 32, 64, 128, 256):
             cM = dataclasses.replace(c1, M=M, name=f"{c1.name} M={M}")
             r = measure(cM, PATTERN_IDS["2:4"], "hif4", n_small)
+            rg = measure(cM, PATTERN_IDS["2:4"], "hif4", n_small, group=True)
             sweep.append({"M": M, "us_per_step": r["ms_per_step"] * 1e3, "tflops": r["tflops"], "gb_per_s": r["gbs"],
-                          "frac_of_hbm": r["gbs"] / peaks["hbm_gbs"], "launches_per_step": r["launches_per_step"]})
-        extras["decode_sweep"] = {"workload": "config 1 layers, S_2:4, HiF4; algorithmic bytes = bf16 X + packed W + bf16 Y",
+                          "frac_of_hbm": r["gbs"] / peaks["hbm_gbs"], "launches_per_step": r["launches_per_step"],
+                          "grouped_us_per_step": rg["ms_per_step"] * 1e3, "grouped_tflops": rg["tflops"],
+                          "grouped_frac_of_hbm": rg["gbs"] / peaks["hbm_gbs"], "grouped_launches_per_step": rg["launches_per_step"]})
+        extras["decode_sweep"] = {"workload": "config 1 layers, S_2:4, HiF4; algorithmic bytes = bf16 X + packed W + bf16 Y; "
+                                              "per-layer calls, and the four layers as one grouped call",
                                   "hbm_peak_gbs": peaks["hbm_gbs"], "points": sweep}
         # ---- quantizer alone
         bpe, rows = quantizer_sweep("hif4", (256, 1024, 4096, 16384, 32768), args.verbose)

@@ -82,6 +82,7 @@ struct PairParams {
     int debug;
     unsigned int* timeline;  // device buffer for a per-role event log of pair 0 (or null)
     int timeline_first;      // first k-block iteration that is logged
+    int timeline_pair;       // the pair that logs
 #endif
     // K-streamed schedule (streamk != 0): the first dp_tiles tiles of the list are computed whole, tile t by pair
     // t mod npairs, and written out directly; the sk_units (tile, k-block) units of the remaining tiles are dealt
@@ -388,7 +389,7 @@ gemm_pair_kernel(const __grid_constant__ PairMaps<NP> maps, const __grid_constan
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 #ifdef RESQ_TIMELINE
     unsigned int* tlog = reinterpret_cast<unsigned int*>(tmem_slot + 4);  // [8 roles][32 iterations] (512 B)
-    const bool tl = p.timeline != nullptr && (blockIdx.x >> 1) == 0;
+    const bool tl = p.timeline != nullptr && (int)(blockIdx.x >> 1) == p.timeline_pair;
     const int kTl0 = p.timeline_first;  // first logged iteration
 #define EVT(k) do { if (tl) p.timeline[512 + (int)rank * 16 + (k)] = (unsigned int)(clock64() - t_kernel0); } while (0)
 #define TLOG(role, it) do { if (tl && (it) >= kTl0 && (it) < kTl0 + 32) tlog[(role) * 32 + ((it) - kTl0)] = (unsigned int)clock64(); } while (0)
@@ -831,7 +832,7 @@ gemm_pair_kernel(const __grid_constant__ PairMaps<NP> maps, const __grid_constan
         if (threadIdx.x == 0) { tr.end(13); EVT(7); }
     }
 #ifdef RESQ_TIMELINE
-    if (tl && threadIdx.x < 256) p.timeline[blockIdx.x * 256 + threadIdx.x] = tlog[threadIdx.x];
+    if (tl && threadIdx.x < 256) p.timeline[rank * 256 + threadIdx.x] = tlog[threadIdx.x];
 #endif
     ptx::cluster_sync();  // no CTA leaves while the peer may still signal its barriers or read its shared memory
 #ifdef RESQ_TIMELINE
@@ -979,6 +980,7 @@ void common_params(PairParams<NP>& p, const GemmArgs& g, bool streamk) {
         const char* tp = getenv("RESQ_GEMM_TIMELINE_PTR");
         p.timeline = tp && *tp ? reinterpret_cast<unsigned int*>(strtoull(tp, nullptr, 0)) : nullptr;
         p.timeline_first = env_int("RESQ_GEMM_TIMELINE_FIRST", 96);
+        p.timeline_pair = env_int("RESQ_GEMM_TIMELINE_PAIR", 0);
     }
 #endif
 }
@@ -1106,6 +1108,7 @@ GroupPlan plan_group(const GemmArgs* g, int count, int npairs) {
     std::vector<double> whole((size_t)npairs);
     for (int ci = 0; ci < nc; ++ci) {
         const int dp = cand[ci];
+        if ((size_t)(total - dp) * 2 * sizeof(unsigned int) > kWsFlags) continue;  // an arrival counter per dealt tile and rank
         std::fill(whole.begin(), whole.end(), 0.0);
         for (int t = 0; t < dp; ++t) whole[(size_t)(t % npairs)] += g_of_tile(t);
         int64_t D = 0;
@@ -1158,7 +1161,8 @@ GroupPlan plan_group(const GemmArgs* g, int count, int npairs) {
                 }
                 worst = std::max(worst, c);
             }
-            if (worst < best.cost) {
+            // (at equal cost the plan with more whole tiles wins: less partial-tile traffic)
+            if (worst < best.cost || (worst == best.cost && dp > best.dp_tiles)) {
                 best.cost = worst;
                 best.dp_tiles = dp;
                 best.sk_first = D > 0 ? b : 0;
@@ -1209,6 +1213,10 @@ int launch_pair_group(const GemmArgs* g, int count, cudaStream_t stream) {
         return RESQ_ERR_CUDA;
     }
     const GroupPlan plan = plan_group(g, count, npairs);
+    if (plan.cost >= 1e300) {
+        set_last_error("gemm pair group: no schedule fits the arrival counters (too many output tiles with long K)");
+        return RESQ_ERR_SHAPE;
+    }
     PairMaps<NP> maps;
     memset(&maps, 0, sizeof(maps));
     p.nprob = count;
