@@ -1176,9 +1176,9 @@ GroupPlan plan_group(const GemmArgs* g, int count, int npairs) {
     return best;
 }
 
-template <int RES, int FMT>
+template <int RES, int FMT, int NG>
 int launch_pair_group(const GemmArgs* g, int count, cudaStream_t stream) {
-    constexpr int TN = kStreamKTN, NG = 3, NP = kMaxGroup;
+    constexpr int TN = kStreamKTN, NP = kMaxGroup;
     if (count < 1 || count > kMaxGroup) {
         set_last_error("a group holds 1 to %d problems (got %d)", kMaxGroup, count);
         return RESQ_ERR_SHAPE;
@@ -1307,10 +1307,11 @@ int streamk_fmt(const GemmArgs& g, cudaStream_t stream) {
 }
 template <int FMT>
 int group_fmt(const GemmArgs* g, int count, cudaStream_t stream) {
+    const bool four = env_int("RESQ_GEMM_GROUPS", 3) == 4;  // debugging override: four expander groups
     switch (res_mode(g[0])) {
-        case kResSparse24: return launch_pair_group<kResSparse24, FMT>(g, count, stream);
-        case kResDense: return launch_pair_group<kResDense, FMT>(g, count, stream);
-        default: return launch_pair_group<kResNone, FMT>(g, count, stream);
+        case kResSparse24: return four ? launch_pair_group<kResSparse24, FMT, 4>(g, count, stream) : launch_pair_group<kResSparse24, FMT, 3>(g, count, stream);
+        case kResDense: return four ? launch_pair_group<kResDense, FMT, 4>(g, count, stream) : launch_pair_group<kResDense, FMT, 3>(g, count, stream);
+        default: return four ? launch_pair_group<kResNone, FMT, 4>(g, count, stream) : launch_pair_group<kResNone, FMT, 3>(g, count, stream);
     }
 }
 template <int FMT>
