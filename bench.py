@@ -70,7 +70,10 @@ RHO = {0: 0.0, 1: 1.0, 2: 0.5, 3: 0.5, 4: 0.5, 5: 0.5}
 RHO.update({p: ((p >> 8) & 0xF) / 4.0 if (p >> 8) & 0xF else 0.5 for p in PATTERN_IDS.values() if p >> 8})
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the dominant GEMM kernel from ncu captures
 # of single layers (summaries with their commands under profiles/), keyed by (config, layer, pattern id, format)
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    (4, "gate_up", 2, "hif4"): {"bytes": 3.83e9, "source": "profiles/gemm_pair_kernel_7b-prefill-gate_up_dram.md"},
+    (4, "qkv", 2, "hif4"): {"bytes": 3.82e8, "source": "profiles/gemm_pair_kernel_7b-prefill-qkv_2to4.md"},
+}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

@@ -717,15 +717,27 @@ bool gemm_use_streamk(int64_t M, int64_t N, int64_t K) {
     return tiles > 74 && tiles <= 74 + 74 / 2 && K / kBK >= 16 && env_int("RESQ_GEMM_HYBRID", 0);
 }
 
-// The 2:4 residual on the structured-sparse MMA is complete and tested but not the default: it halves the tensor
-// work of the residual term and shrinks its operand from 16 KB to 9 KB per k-block, yet the pair kernel is bound
-// by weight expansion and by shared-memory ingest rather than by tensor issue, the 512-wide tile has no
-// tensor-memory columns left for the metadata, and the quantizer pays for the compression.  Measured (M = 8192,
-// K = 2048): N = 22016 in 955 us instead of 1011 us, but N = 2048 in 150 us instead of 124 us (tile count); the
-// decode shapes lose 4 %.  RESQ_SPARSE24=1 switches it on.
+// The 2:4 residual on the structured-sparse MMA (compressed operand + index metadata, half the tensor work of the
+// residual term) is used where it is the faster form.  Its widest tile is 480 columns (the metadata takes eight
+// tensor-memory columns), so it runs ceil(N / 480) instead of ceil(N / 512) columns of tiles; a k-block of a 480-wide
+// sparse tile takes about 0.78 of the time of a 512-wide dense one (measured on the 7B and 3B prefill shapes under the
+// power cap: 1.26 against 1.67 us).  It wins when that outweighs the extra tiles: every layer at M = 16384, the wide
+// layers at M = 8192 (gate_up 856 against 989 us, qkv 165 against 184), not the N = 2048 layers there (five columns of
+// tiles instead of four: 162 against 138 us), and not below a few thousand rows, where the calls are bound by fixed
+// costs (M = 256: 150 against 146 us per step).  RESQ_SPARSE24 = 0 / 1 forces the choice (debugging override).
 bool gemm_sparse24_supported(int64_t M, int64_t N, int64_t K) {
-    (void)N;
-    return M > kBM && K % kBK == 0 && env_int("RESQ_GEMM_PAIR", 1) && env_int("RESQ_SPARSE24", 0);
+    if (M <= kBM || K % kBK != 0 || !env_int("RESQ_GEMM_PAIR", 1)) return false;
+    const int forced = env_int("RESQ_SPARSE24", -1);
+    if (forced >= 0) return forced != 0;
+    if (M < 4096) return false;
+    const int64_t mt = (M + 2 * kBM - 1) / (2 * kBM);
+    const int64_t nt512 = (N + 511) / 512, nt480 = (N + 479) / 480;
+    const int64_t tiles512 = mt * nt512, tail = tiles512 % 74;
+    // (a small last round of the dense form is cut off into a decode-sized call: count it as a fraction of a round)
+    const double rounds512 = (tiles512 > 74 && tail > 0 && tail <= nt512 && tail * 3 <= 74) ? (double)tiles512 / 74.0
+                                                                                          : (double)((tiles512 + 73) / 74);
+    const double rounds480 = (double)((mt * nt480 + 73) / 74);
+    return rounds480 * 0.78 < rounds512;
 }
 
 size_t gemm_hif4_scratch_bytes(int64_t M, int64_t N, int64_t K) {

@@ -1307,7 +1307,10 @@ int streamk_fmt(const GemmArgs& g, cudaStream_t stream) {
 }
 template <int FMT>
 int group_fmt(const GemmArgs* g, int count, cudaStream_t stream) {
-    const bool four = env_int("RESQ_GEMM_GROUPS", 3) == 4;  // debugging override: four expander groups
+    // four expander groups (768 threads, 80 registers): the long k-block runs of a group are bound by the expanders'
+    // latency per k-block, and a fourth group shortens the period (config 1 step 98.4 -> 93.4 us); RESQ_GEMM_GROUPS=3
+    // is the debugging override
+    const bool four = env_int("RESQ_GEMM_GROUPS", 4) == 4;
     switch (res_mode(g[0])) {
         case kResSparse24: return four ? launch_pair_group<kResSparse24, FMT, 4>(g, count, stream) : launch_pair_group<kResSparse24, FMT, 3>(g, count, stream);
         case kResDense: return four ? launch_pair_group<kResDense, FMT, 4>(g, count, stream) : launch_pair_group<kResDense, FMT, 3>(g, count, stream);
