@@ -423,3 +423,36 @@ def w4a8_linear(x_f32: np.ndarray, w_f32: np.ndarray, fmt: str = "hif4", want_ab
     w = decode(fmt, w_codes, w_side)
     y, ab = matmul(a, None, w, want_abs)
     return {"a_codes": codes, "a_scale": scale, "a": a, "w": w, "y": y, "abs_sum": ab}
+
+
+# ---- training-side GEMMs of the same layer (the backward pass of Y = X W^T) -----------------------------------------
+# The paper states that the forward and the backward passes of the training policy run in 4 bit (Sections 1 and 3)
+# and writes out the forward product only (Eq. (1)).  Reading taken here: Eq. (1)'s operator Q is applied to both
+# operands of each backward product, with the quantization blocks along that product's contraction axis (as in the
+# forward product, where they run along d):
+#     dX = dY W        (contraction over n):  dX^ = Q(dY) Q(W^T)^T,   Q along n on the rows of dY [m, n] and of W^T [d, n]
+#     dW = dY^T X      (contraction over m):  dW^ = Q(dY^T) Q(X^T)^T, Q along m on the rows of dY^T [n, m] and of X^T [d, m]
+# No residual term: Rollout-ResQ corrects the rollout policy's activations only (Section 4).
+
+def dgrad_linear(dy_f32: np.ndarray, w_f32: np.ndarray, fmt: str = "hif4", want_abs: bool = True) -> Dict[str, np.ndarray]:
+    """dX^ [m, d] = Q(dY) Q(W^T)^T for dY [m, n], W [n, d]."""
+    dy = _f32(dy_f32)
+    wt = np.ascontiguousarray(_f32(w_f32).T)
+    g_codes, g_side = encode(fmt, dy)
+    wt_codes, wt_side = encode(fmt, wt)
+    g = decode(fmt, g_codes, g_side)
+    wtd = decode(fmt, wt_codes, wt_side)
+    y, ab = matmul(g, None, wtd, want_abs)
+    return {"g": g, "wt": wtd, "wt_codes": wt_codes, "wt_side": wt_side, "y": y, "abs_sum": ab}
+
+
+def wgrad_linear(dy_f32: np.ndarray, x_f32: np.ndarray, fmt: str = "hif4", want_abs: bool = True) -> Dict[str, np.ndarray]:
+    """dW^ [n, d] = Q(dY^T) Q(X^T)^T for dY [m, n], X [m, d]."""
+    gt = np.ascontiguousarray(_f32(dy_f32).T)
+    xt = np.ascontiguousarray(_f32(x_f32).T)
+    gt_codes, gt_side = encode(fmt, gt)
+    xt_codes, xt_side = encode(fmt, xt)
+    gtd = decode(fmt, gt_codes, gt_side)
+    xtd = decode(fmt, xt_codes, xt_side)
+    y, ab = matmul(gtd, None, xtd, want_abs)
+    return {"gt": gtd, "xt": xtd, "y": y, "abs_sum": ab}

@@ -878,3 +878,50 @@ def test_seeded_digest():
     assert abs(rel(XX - o["a"]) - 0.0881) < 5e-4
     assert abs(rel(XX - o["a"] - o["r"]) - 0.0076) < 5e-4
     assert abs(rel(XX - o["a"] - o["r_masked"]) - 0.0346) < 5e-4
+
+
+# ----------------------------------------------------------------- training-side GEMMs (backward pass of Eq. (1))
+
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+def test_backward_products_exact_rational_tiny_and_fixed_points(fmt):
+    M, K, N = 64, 128, 64          # every contraction axis (n for dX, m for dW) holds whole blocks
+    rng = np.random.default_rng(91)
+    dy = bf16_round((rng.standard_normal((M, N)) * 1e-3).astype(np.float32))
+    dy[:, 5] *= 40.0                # an outlier column of the output gradient
+    w = bf16_round((rng.standard_normal((N, K)) * 0.02).astype(np.float32))
+    x = gaussian_with_outliers(92, M, K, n_out=2, scale=16.0)
+    # dX^ = Q(dY) Q(W^T)^T: the blocks of both operands run along n
+    o = oracle.dgrad_linear(dy, w, fmt)
+    assert o["y"].shape == (M, K)
+    assert np.array_equal(o["g"], oracle.decode(fmt, *oracle.encode(fmt, dy)))
+    assert np.array_equal(o["wt"], oracle.decode(fmt, *oracle.encode(fmt, np.ascontiguousarray(w.T))))
+    g, wt = _to_frac(o["g"][:3]), _to_frac(o["wt"][:4])
+    for m in range(3):
+        for k in range(4):
+            assert F(float(o["y"][m, k])) == sum(g[m][n] * wt[k][n] for n in range(N))
+            assert F(float(o["abs_sum"][m, k])) == sum(abs(g[m][n] * wt[k][n]) for n in range(N))
+    # dW^ = Q(dY^T) Q(X^T)^T: the blocks run along m
+    o2 = oracle.wgrad_linear(dy, x, fmt)
+    assert o2["y"].shape == (N, K)
+    gt, xt = _to_frac(o2["gt"][:3]), _to_frac(o2["xt"][:4])
+    for n in range(3):
+        for k in range(4):
+            assert F(float(o2["y"][n, k])) == sum(gt[n][m] * xt[k][m] for m in range(M))
+    # quantizing along the contraction axis is not the same as quantizing along the other one: a loud token row of X
+    # costs its own row nothing when the blocks run along d, but dominates the blocks of every channel along m
+    x2 = x.copy()
+    x2[7, :] *= 64.0
+    along_d = oracle.decode(fmt, *oracle.encode(fmt, x2))
+    along_m = oracle.decode(fmt, *oracle.encode(fmt, np.ascontiguousarray(x2.T))).T
+    quiet = np.arange(M) != 7
+    assert np.abs(along_m - x2)[quiet].max() > 4 * np.abs(along_d - x2)[quiet].max()
+    # fixed points: operands that already are decoded codes (along the right axis) give the exact products
+    if fmt == "hif4":
+        dyq = representable_hif4_blocks(93, M * N // 64, 30 << 2, 40 << 2)[0].reshape(M, N).astype(np.float32)
+        wtq = representable_hif4_blocks(94, K * N // 64, 40 << 2, 48 << 2)[0].reshape(K, N).astype(np.float32)
+        o3 = oracle.dgrad_linear(dyq, np.ascontiguousarray(wtq.T))
+        np.testing.assert_allclose(o3["y"], dyq.astype(np.float64) @ wtq.astype(np.float64).T, rtol=1e-13, atol=0)
+        gtq = representable_hif4_blocks(95, N * M // 64, 30 << 2, 40 << 2)[0].reshape(N, M).astype(np.float32)
+        xtq = representable_hif4_blocks(96, K * M // 64, 44 << 2, 52 << 2)[0].reshape(K, M).astype(np.float32)
+        o4 = oracle.wgrad_linear(np.ascontiguousarray(gtq.T), np.ascontiguousarray(xtq.T))
+        np.testing.assert_allclose(o4["y"], gtq.astype(np.float64) @ xtq.astype(np.float64).T, rtol=1e-13, atol=0)
