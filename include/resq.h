@@ -211,6 +211,36 @@ RESQ_API int hif4_resq_linear_group(const resq_problem* problems, int count, int
 RESQ_API int mxfp4_resq_linear_group(const resq_problem* problems, int count, int pattern, int out_dtype,
                             void* workspace, size_t ws_bytes, void* stream);
 
+/* ---- the backward products of the layer, in 4 bit (training side) ---------------------------------------------------
+ * The paper's training policy runs its forward and backward passes in 4 bit (Sections 1 and 3) and writes out the
+ * forward product only, Eq. (1).  This library's reading: Eq. (1)'s operator Q on both operands of each backward
+ * product, with the quantization blocks along that product's contraction axis, no residual term:
+ *     dX^ [M, K] = Q(dY) Q(W^T)^T        dY [M, N], blocks along N;  W^T [K, N] packed once by *_pack_weight_transposed
+ *     dW^ [N, K] = Q(dY^T) Q(X^T)^T      dY^T [N, M], X^T [K, M], blocks along M (M a multiple of 64 / 32)
+ * Each is the layer call (*_resq_linear with RESQ_S_NONE) on transposed operands; the transposes are bf16 copies in the
+ * workspace.  Argument rules, output types and error behaviour as *_resq_linear.
+ *   *_pack_weight_transposed: W_bf16 [N, K] (ldw) -> wt_codes [K, N/2], wt_meta [K, N/64] (wt_scale [K, N/32]);
+ *       N a multiple of the block size; workspace of resq_transposed_workspace_bytes(N, K) bytes.
+ *   *_dgrad_linear: dY_bf16 [M, N] (lddy), the transposed pack, dX [M, K] (lddx); workspace *_dgrad_workspace_bytes.
+ *   *_wgrad_linear: dY_bf16 [M, N] (lddy), X_bf16 [M, K] (ldx), dW [N, K] (lddw); workspace *_wgrad_workspace_bytes. */
+RESQ_API size_t resq_transposed_workspace_bytes(int64_t N, int64_t K);
+RESQ_API int hif4_pack_weight_transposed(const void* W_bf16, int64_t N, int64_t K, int64_t ldw, void* wt_codes, void* wt_meta,
+                                void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_pack_weight_transposed(const void* W_bf16, int64_t N, int64_t K, int64_t ldw, void* wt_codes, void* wt_scale,
+                                 void* workspace, size_t ws_bytes, void* stream);
+RESQ_API size_t hif4_dgrad_workspace_bytes(int64_t M, int64_t N, int64_t K);
+RESQ_API size_t mxfp4_dgrad_workspace_bytes(int64_t M, int64_t N, int64_t K);
+RESQ_API int hif4_dgrad_linear(const void* dY_bf16, int64_t M, int64_t N, int64_t lddy, const void* wt_codes, const void* wt_meta,
+                      int64_t K, void* dX, int out_dtype, int64_t lddx, void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_dgrad_linear(const void* dY_bf16, int64_t M, int64_t N, int64_t lddy, const void* wt_codes, const void* wt_scale,
+                       int64_t K, void* dX, int out_dtype, int64_t lddx, void* workspace, size_t ws_bytes, void* stream);
+RESQ_API size_t hif4_wgrad_workspace_bytes(int64_t M, int64_t N, int64_t K);
+RESQ_API size_t mxfp4_wgrad_workspace_bytes(int64_t M, int64_t N, int64_t K);
+RESQ_API int hif4_wgrad_linear(const void* dY_bf16, const void* X_bf16, int64_t M, int64_t N, int64_t K, int64_t lddy, int64_t ldx,
+                      void* dW, int out_dtype, int64_t lddw, void* workspace, size_t ws_bytes, void* stream);
+RESQ_API int mxfp4_wgrad_linear(const void* dY_bf16, const void* X_bf16, int64_t M, int64_t N, int64_t K, int64_t lddy, int64_t ldx,
+                       void* dW, int out_dtype, int64_t lddw, void* workspace, size_t ws_bytes, void* stream);
+
 /* Weight-only ablation of Table 1 ("W4A16"): Y = X deq(Q(W))^T, the bf16 activations are used as they are
  * (no activation quantizer, no residual term); weights as produced by *_pack_weight.  Same argument rules,
  * output types and error behaviour as *_resq_linear; workspace of resq_w4a16_workspace_bytes(M, N, K) bytes

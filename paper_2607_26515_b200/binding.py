@@ -48,6 +48,17 @@ SYMBOLS = {
     "mxfp4_resq_group_workspace_bytes": (_sz, [_vp, _ci, _ci]),
     "hif4_resq_linear_group": (_ci, [_vp, _ci, _ci, _ci, _vp, _sz, _vp]),
     "mxfp4_resq_linear_group": (_ci, [_vp, _ci, _ci, _ci, _vp, _sz, _vp]),
+    "resq_transposed_workspace_bytes": (_sz, [_i64, _i64]),
+    "hif4_pack_weight_transposed": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _sz, _vp]),
+    "mxfp4_pack_weight_transposed": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _sz, _vp]),
+    "hif4_dgrad_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "mxfp4_dgrad_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "hif4_dgrad_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "mxfp4_dgrad_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "hif4_wgrad_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "mxfp4_wgrad_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "hif4_wgrad_linear": (_ci, [_vp, _vp, _i64, _i64, _i64, _i64, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
+    "mxfp4_wgrad_linear": (_ci, [_vp, _vp, _i64, _i64, _i64, _i64, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
     "resq_w4a16_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "resq_w4a8_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "hif4_w4a8_linear": (_ci, [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp, _ci, _i64, _vp, _sz, _vp]),
@@ -329,6 +340,56 @@ def resq_linear_group(problems, pattern: int, fmt: str = "hif4", out_dtype: torc
         ctypes.cast(arr, _vp), len(problems), pattern, OUT_BF16 if out_dtype == torch.bfloat16 else OUT_F32,
         workspace.data_ptr(), workspace.numel(), _stream(stream)))
     return ys
+
+
+def _out(rows: int, cols: int, dtype: torch.dtype, device) -> torch.Tensor:
+    """An output matrix whose rows start on 16-byte boundaries."""
+    return torch.empty((rows, (cols + 7) // 8 * 8), dtype=dtype, device=device)[:, :cols]
+
+
+def pack_weight_transposed(W: torch.Tensor, fmt: str = "hif4", stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """*_pack_weight_transposed: W bf16 [N,K] -> Q(W^T) as (codes [K,N/2], meta [K,N/64] | scale [K,N/32]), for dgrad."""
+    _require_bf16_matrix(W, "W")
+    N, K = W.shape
+    codes = torch.empty((K, N // 2), dtype=torch.uint8, device=W.device)
+    side = _side(fmt, K, N, W.device)
+    work = alloc_workspace(int(lib().resq_transposed_workspace_bytes(N, K)), W.device)
+    _check(_fn(fmt, "hif4_pack_weight_transposed", "mxfp4_pack_weight_transposed")(
+        W.data_ptr(), N, K, W.stride(0), codes.data_ptr(), side.data_ptr(), work.data_ptr(), work.numel(), _stream(stream)))
+    return codes, side
+
+
+def dgrad_linear(dY: torch.Tensor, wt_codes: torch.Tensor, wt_side: torch.Tensor, fmt: str = "hif4",
+                 out_dtype: torch.dtype = torch.bfloat16, workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """*_dgrad_linear: dX^ [M,K] = Q(dY) Q(W^T)^T with the transposed pack of the weight."""
+    _require_bf16_matrix(dY, "dY")
+    M, N = dY.shape
+    K = wt_codes.shape[0]
+    dX = _out(M, K, out_dtype, dY.device)
+    if workspace is None:
+        workspace = alloc_workspace(int(_fn(fmt, "hif4_dgrad_workspace_bytes", "mxfp4_dgrad_workspace_bytes")(M, N, K)), dY.device)
+    _check(_fn(fmt, "hif4_dgrad_linear", "mxfp4_dgrad_linear")(
+        dY.data_ptr(), M, N, dY.stride(0), wt_codes.data_ptr(), wt_side.data_ptr(), K, dX.data_ptr(),
+        OUT_BF16 if out_dtype == torch.bfloat16 else OUT_F32, dX.stride(0), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return dX
+
+
+def wgrad_linear(dY: torch.Tensor, X: torch.Tensor, fmt: str = "hif4", out_dtype: torch.dtype = torch.bfloat16,
+                 workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """*_wgrad_linear: dW^ [N,K] = Q(dY^T) Q(X^T)^T."""
+    _require_bf16_matrix(dY, "dY")
+    _require_bf16_matrix(X, "X")
+    M, N = dY.shape
+    K = X.shape[1]
+    if X.shape[0] != M:
+        raise ValueError("dY and X must have the same number of token rows")
+    dW = _out(N, K, out_dtype, dY.device)
+    if workspace is None:
+        workspace = alloc_workspace(int(_fn(fmt, "hif4_wgrad_workspace_bytes", "mxfp4_wgrad_workspace_bytes")(M, N, K)), dY.device)
+    _check(_fn(fmt, "hif4_wgrad_linear", "mxfp4_wgrad_linear")(
+        dY.data_ptr(), X.data_ptr(), M, N, K, dY.stride(0), X.stride(0), dW.data_ptr(),
+        OUT_BF16 if out_dtype == torch.bfloat16 else OUT_F32, dW.stride(0), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return dW
 
 
 def w4a16_linear(X: torch.Tensor, w_codes: torch.Tensor, w_side: torch.Tensor, fmt: str = "hif4",

@@ -613,6 +613,81 @@ int linear_group(int fmt, const resq_problem* pr, int count, int pattern, int ou
     return launch_gemm_pair_group(ga, count, st);
 }
 
+// ---- backward products of the layer (training side) ---------------------------------------------------------------
+// Both are Eq. (1) on transposed operands: the quantization blocks run along the product's own contraction axis.
+size_t transposed_bytes(int64_t rows, int64_t cols) { return align_up((size_t)rows * (size_t)cols * 2, 256); }
+
+int pack_weight_transposed(int fmt, const void* W, int64_t N, int64_t K, int64_t ldw, void* wt_codes, void* wt_side, void* workspace,
+                           size_t ws_bytes, void* stream) {
+    // W [N, K] -> Q(W^T): K rows of N values, blocks along N
+    if (!W || !wt_codes || !wt_side) {
+        set_last_error("pack_weight_transposed: NULL pointer");
+        return RESQ_ERR_NULL;
+    }
+    if (N <= 0 || K <= 0 || N % block_of(fmt) != 0) {
+        set_last_error("pack_weight_transposed: N=%lld K=%lld (N must be a positive multiple of %d)", (long long)N, (long long)K,
+                       block_of(fmt));
+        return RESQ_ERR_SHAPE;
+    }
+    if (!aligned16(W) || ldw < K || ldw % 8 != 0 || N % 8 != 0) {
+        set_last_error("pack_weight_transposed: W needs a 16-byte aligned base, ldw >= K, ldw %% 8 == 0");
+        return RESQ_ERR_ALIGN;
+    }
+    int rc = check_packed_outputs(wt_codes, wt_side, nullptr, nullptr);
+    if (rc) return rc;
+    rc = check_workspace(workspace, ws_bytes, transposed_bytes(K, N));
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    __nv_bfloat16* wt = static_cast<__nv_bfloat16*>(workspace);
+    rc = launch_transpose_bf16(static_cast<const __nv_bfloat16*>(W), N, K, ldw, wt, N, st);
+    if (rc) return rc;
+    return quantize_only(fmt, wt, K, N, N, wt_codes, wt_side, stream, "W^T");
+}
+
+size_t wgrad_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K) {
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    const size_t side = fmt == kHiF4 ? (size_t)K * (size_t)(M / kHif4Block) * 4 : (size_t)K * (size_t)(M / kMxBlock);
+    return linear_workspace_bytes(fmt, N, K, M, RESQ_S_NONE) + transposed_bytes(N, M) + transposed_bytes(K, M) +
+           align_up((size_t)K * (size_t)M / 2, 256) + align_up(side, 256);
+}
+
+int wgrad_linear(int fmt, const void* dY, const void* X, int64_t M, int64_t N, int64_t K, int64_t lddy, int64_t ldx, void* dW,
+                 int out_dtype, int64_t lddw, void* workspace, size_t ws_bytes, void* stream) {
+    if (!dY || !X || !dW) {
+        set_last_error("wgrad_linear: NULL pointer");
+        return RESQ_ERR_NULL;
+    }
+    if (M <= 0 || N <= 0 || K <= 0 || M % block_of(fmt) != 0) {
+        set_last_error("wgrad_linear: M=%lld N=%lld K=%lld (the contraction runs over M: a positive multiple of %d)", (long long)M,
+                       (long long)N, (long long)K, block_of(fmt));
+        return RESQ_ERR_SHAPE;
+    }
+    if (!aligned16(dY) || !aligned16(X) || lddy < N || ldx < K || lddy % 8 != 0 || ldx % 8 != 0 || M % 8 != 0) {
+        set_last_error("wgrad_linear: dY / X need 16-byte aligned bases and row pitches that are multiples of 8 and cover the rows");
+        return RESQ_ERR_ALIGN;
+    }
+    int rc = check_workspace(workspace, ws_bytes, wgrad_workspace_bytes(fmt, M, N, K));
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    size_t used = linear_workspace_bytes(fmt, N, K, M, RESQ_S_NONE);
+    __nv_bfloat16* gt = reinterpret_cast<__nv_bfloat16*>(ws + used);   // dY^T [N, M]
+    used += transposed_bytes(N, M);
+    __nv_bfloat16* xt = reinterpret_cast<__nv_bfloat16*>(ws + used);   // X^T [K, M]
+    used += transposed_bytes(K, M);
+    uint8_t* xt_codes = ws + used;
+    used += align_up((size_t)K * (size_t)M / 2, 256);
+    void* xt_side = ws + used;
+    rc = launch_transpose_bf16(static_cast<const __nv_bfloat16*>(dY), M, N, lddy, gt, M, st);
+    if (rc) return rc;
+    rc = launch_transpose_bf16(static_cast<const __nv_bfloat16*>(X), M, K, ldx, xt, M, st);
+    if (rc) return rc;
+    rc = quantize_only(fmt, xt, K, M, M, xt_codes, xt_side, stream, "X^T");
+    if (rc) return rc;
+    // dW^ [N, K] = Q(dY^T) Q(X^T)^T: the layer call with dY^T as its activation and Q(X^T) as its packed operand
+    return linear(fmt, gt, N, M, M, xt_codes, xt_side, K, RESQ_S_NONE, dW, out_dtype, lddw, workspace, ws_bytes, stream);
+}
+
 // Weight-only variant (Table 1, "W4A16"): Y = X deq(Q(W))^T with the bf16 activations used as they are.
 // Workspace: [header | counters | fp32 partial tiles].
 size_t w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
@@ -899,6 +974,36 @@ int hif4_resq_linear_group(const resq_problem* problems, int count, int pattern,
 int mxfp4_resq_linear_group(const resq_problem* problems, int count, int pattern, int out_dtype, void* workspace, size_t ws_bytes,
                             void* stream) {
     return linear_group(kMXFP4, problems, count, pattern, out_dtype, workspace, ws_bytes, stream);
+}
+
+size_t resq_transposed_workspace_bytes(int64_t N, int64_t K) { return N > 0 && K > 0 ? transposed_bytes(K, N) : 0; }
+int hif4_pack_weight_transposed(const void* W, int64_t N, int64_t K, int64_t ldw, void* wt_codes, void* wt_meta, void* workspace,
+                                size_t ws_bytes, void* stream) {
+    return pack_weight_transposed(kHiF4, W, N, K, ldw, wt_codes, wt_meta, workspace, ws_bytes, stream);
+}
+int mxfp4_pack_weight_transposed(const void* W, int64_t N, int64_t K, int64_t ldw, void* wt_codes, void* wt_scale, void* workspace,
+                                 size_t ws_bytes, void* stream) {
+    return pack_weight_transposed(kMXFP4, W, N, K, ldw, wt_codes, wt_scale, workspace, ws_bytes, stream);
+}
+size_t hif4_dgrad_workspace_bytes(int64_t M, int64_t N, int64_t K) { return linear_workspace_bytes(kHiF4, M, K, N, RESQ_S_NONE); }
+size_t mxfp4_dgrad_workspace_bytes(int64_t M, int64_t N, int64_t K) { return linear_workspace_bytes(kMXFP4, M, K, N, RESQ_S_NONE); }
+int hif4_dgrad_linear(const void* dY, int64_t M, int64_t N, int64_t lddy, const void* wt_codes, const void* wt_meta, int64_t K, void* dX,
+                      int out_dtype, int64_t lddx, void* workspace, size_t ws_bytes, void* stream) {
+    return linear(kHiF4, dY, M, N, lddy, wt_codes, wt_meta, K, RESQ_S_NONE, dX, out_dtype, lddx, workspace, ws_bytes, stream);
+}
+int mxfp4_dgrad_linear(const void* dY, int64_t M, int64_t N, int64_t lddy, const void* wt_codes, const void* wt_scale, int64_t K, void* dX,
+                       int out_dtype, int64_t lddx, void* workspace, size_t ws_bytes, void* stream) {
+    return linear(kMXFP4, dY, M, N, lddy, wt_codes, wt_scale, K, RESQ_S_NONE, dX, out_dtype, lddx, workspace, ws_bytes, stream);
+}
+size_t hif4_wgrad_workspace_bytes(int64_t M, int64_t N, int64_t K) { return wgrad_workspace_bytes(kHiF4, M, N, K); }
+size_t mxfp4_wgrad_workspace_bytes(int64_t M, int64_t N, int64_t K) { return wgrad_workspace_bytes(kMXFP4, M, N, K); }
+int hif4_wgrad_linear(const void* dY, const void* X, int64_t M, int64_t N, int64_t K, int64_t lddy, int64_t ldx, void* dW, int out_dtype,
+                      int64_t lddw, void* workspace, size_t ws_bytes, void* stream) {
+    return wgrad_linear(kHiF4, dY, X, M, N, K, lddy, ldx, dW, out_dtype, lddw, workspace, ws_bytes, stream);
+}
+int mxfp4_wgrad_linear(const void* dY, const void* X, int64_t M, int64_t N, int64_t K, int64_t lddy, int64_t ldx, void* dW, int out_dtype,
+                       int64_t lddw, void* workspace, size_t ws_bytes, void* stream) {
+    return wgrad_linear(kMXFP4, dY, X, M, N, K, lddy, ldx, dW, out_dtype, lddw, workspace, ws_bytes, stream);
 }
 
 int resq_check(void* workspace, void* stream) {

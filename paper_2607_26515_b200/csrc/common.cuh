@@ -141,6 +141,9 @@ int launch_quantize_group(int fmt, const QuantArgs* a, int count, cudaStream_t s
 // "W4A8": the decoded bf16 image of MXFP8-E4M3 quantized activations (blocks of 32, E8M0 scale), for the GEMM
 int launch_quantize_mxfp8_image(const __nv_bfloat16* X, int64_t M, int64_t K, int64_t ldx, __nv_bfloat16* img, uint32_t* clear_words,
                                 int n_clear_words, cudaStream_t stream);
+// dst [cols, rows] (row pitch ld_dst) = transpose of src [rows, cols] (row pitch ld_src)
+int launch_transpose_bf16(const __nv_bfloat16* src, int64_t rows, int64_t cols, int64_t ld_src, __nv_bfloat16* dst, int64_t ld_dst,
+                          cudaStream_t stream);
 int launch_dequantize(int fmt, const uint8_t* codes, const void* side, int64_t rows, int64_t K, float* out,
                       cudaStream_t stream);
 size_t quant_scratch_bytes(int64_t M, int64_t K, int pattern);  // scores + keep flags [+ histogram] (without header)

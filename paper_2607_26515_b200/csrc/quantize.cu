@@ -1993,6 +1993,35 @@ int launch_quantize(int fmt, const QuantArgs& a_in, cudaStream_t stream) {
     return rc;
 }
 
+// bf16 matrix transpose (the backward products quantize along their own contraction axes): 64 x 64 tiles through
+// shared memory, coalesced on both sides.
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols, int64_t ld_src,
+                                                             uint16_t* __restrict__ dst, int64_t ld_dst) {
+    pdl_wait();
+    pdl_trigger();
+    __shared__ uint16_t tile[64][66];
+    const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
+    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;  // 64 x 4
+    for (int i = ty; i < 64; i += 4) {
+        const int64_t r = r0 + i, c = c0 + tx;
+        tile[i][tx] = (r < rows && c < cols) ? src[r * ld_src + c] : (uint16_t)0;
+    }
+    __syncthreads();
+    for (int i = ty; i < 64; i += 4) {
+        const int64_t c = c0 + i, r = r0 + tx;  // dst row = source column
+        if (c < cols && r < rows) dst[c * ld_dst + r] = tile[tx][i];
+    }
+}
+
+int launch_transpose_bf16(const __nv_bfloat16* src, int64_t rows, int64_t cols, int64_t ld_src, __nv_bfloat16* dst, int64_t ld_dst,
+                          cudaStream_t stream) {
+    LaunchScope scope(kKindQuant, stream);
+    dim3 grid((unsigned)((cols + 63) / 64), (unsigned)((rows + 63) / 64));
+    return cuda_fail(launch_kernel(transpose_bf16_kernel, grid, dim3(256), 0, stream, reinterpret_cast<const uint16_t*>(src), rows, cols,
+                                   ld_src, reinterpret_cast<uint16_t*>(dst), ld_dst),
+                     "transpose_bf16_kernel launch");
+}
+
 // One launch for a group of activations with a row-local selection (NONE, DENSE, n:4) that feed the GEMM (images).
 int launch_quantize_group(int fmt, const QuantArgs* a_in, int count, cudaStream_t stream) {
     if (count < 1 || count > kMaxQuantGroup) {

@@ -653,3 +653,44 @@ def test_linear_group_argument_errors():
     with pytest.raises(m.ResqError) as e:
         m.resq_linear_group([(x, wc, ws)], oracle.S_2_4, workspace=m.alloc_workspace(4096))
     assert e.value.status == 4
+
+
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("shape", [(256, 512, 384), (64, 128, 1000), (1024, 2048, 640)])
+def test_backward_products_match_the_oracle(shape, fmt):
+    """*_pack_weight_transposed, *_dgrad_linear, *_wgrad_linear: Eq. (1) on the transposed operands of the backward
+    pass (blocks along each product's contraction axis); packed W^T bit-exact, dX^ and dW^ element by element."""
+    m = rq()
+    M, N, K = shape
+    rng = np.random.default_rng(M + N + K)
+    dy = (rng.standard_normal((M, N)) * 1e-3).astype(np.float32)
+    dy[:, rng.choice(N, 2, replace=False)] *= 30.0
+    dyb = f32_to_bf16_bits(dy)
+    xb, wb = synth_xw(5 * M + K, M, K, N, n_out=2)
+    # dgrad
+    want = oracle.dgrad_linear(bf16_bits_to_f32(dyb), bf16_bits_to_f32(wb), fmt)
+    wtc, wts = m.pack_weight_transposed(to_dev(wb), fmt)
+    assert np.array_equal(wtc.cpu().numpy(), want["wt_codes"])
+    side = wts.cpu().numpy()
+    assert np.array_equal(side.view(np.uint32) if side.dtype == np.int32 else side, want["wt_side"])
+    dx = m.dgrad_linear(to_dev(dyb), wtc, wts, fmt, out_dtype=torch.float32)
+    check_close(dx.cpu().numpy(), want["y"], want["abs_sum"])
+    # wgrad
+    want2 = oracle.wgrad_linear(bf16_bits_to_f32(dyb), bf16_bits_to_f32(xb), fmt)
+    dw = m.wgrad_linear(to_dev(dyb), to_dev(xb), fmt, out_dtype=torch.float32)
+    check_close(dw.cpu().numpy(), want2["y"], want2["abs_sum"])
+    dwb = m.wgrad_linear(to_dev(dyb), to_dev(xb), fmt, out_dtype=torch.bfloat16)
+    check_close(dwb.float().cpu().numpy(), want2["y"], want2["abs_sum"], bf16_out=True)
+
+
+def test_backward_products_argument_errors():
+    m = rq()
+    dy = torch.zeros((96, 128), dtype=torch.bfloat16, device="cuda")    # M = 96 is not a multiple of 64
+    x = torch.zeros((96, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(m.ResqError) as e:
+        m.wgrad_linear(dy, x)
+    assert e.value.status == 2
+    w = torch.zeros((96, 256), dtype=torch.bfloat16, device="cuda")      # N = 96: the blocks of W^T run along N
+    with pytest.raises(m.ResqError) as e:
+        m.pack_weight_transposed(w)
+    assert e.value.status == 2
