@@ -1105,6 +1105,13 @@ GroupPlan plan_group(const GemmArgs* g, int count, int npairs) {
         cand[nc++] = base[i];
         cand[nc++] = base[i] / npairs * npairs;
     }
+    // debugging overrides (tests reach both classes of ranges with them): the number of whole tiles and the units of
+    // the pairs that hold one whole tile more
+    const int force_dp = env_int("RESQ_GEMM_GROUP_DP", -1), force_hi = env_int("RESQ_GEMM_GROUP_HI", -1);
+    if (force_dp >= 0 && force_dp <= total) {
+        cand[0] = force_dp;
+        nc = 1;
+    }
     std::vector<double> whole((size_t)npairs);
     for (int ci = 0; ci < nc; ++ci) {
         const int dp = cand[ci];
@@ -1121,7 +1128,7 @@ GroupPlan plan_group(const GemmArgs* g, int count, int npairs) {
                 if (b == 0 || D == 0) break;
                 const double extra = whole[0] - whole[(size_t)(npairs - 1)];
                 const double h = ((double)D - extra * (npairs - b)) / npairs;  // H with equal loads
-                H = (int)h;
+                H = force_hi >= 0 ? force_hi : (int)h;
                 if (H < 4) break;
             }
             const int64_t rest = D - (int64_t)b * H;
@@ -1161,6 +1168,7 @@ GroupPlan plan_group(const GemmArgs* g, int count, int npairs) {
                 }
                 worst = std::max(worst, c);
             }
+            if (force_hi >= 0 && pass == 1) worst = 0.0;  // (forced)
             // (at equal cost the plan with more whole tiles wins: less partial-tile traffic)
             if (worst < best.cost || (worst == best.cost && dp > best.dp_tiles)) {
                 best.cost = worst;

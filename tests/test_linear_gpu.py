@@ -609,11 +609,16 @@ GROUPS = {
     # more whole tiles than CTA pairs, and a long-K problem whose k-blocks are dealt out
     "many-tiles": ([(512, 512, 9728), (256, 512, 3000), (256, 8192, 512)], oracle.S_2_4, "hif4", torch.bfloat16),
     "quarter": ([(128, 1024, 384), (256, 1024, 768)], oracle.keep_quarters(oracle.S_2_4, 1), "hif4", torch.float32),
+    # 100 short whole tiles and four long dealt ones: 26 pairs hold two whole tiles and still take a share of the dealt
+    # k-blocks (both classes of the schedule's ranges in one launch)
+    "two-classes": ([(256, 512, 25600), (256, 25600, 1024)], oracle.S_2_4, "hif4", torch.bfloat16),
+    # prefill-sized problems: several rounds of whole tiles, rows beyond one M tile
+    "tall": ([(2048, 1024, 4096), (1024, 4096, 1024)], oracle.S_DENSE, "hif4", torch.bfloat16),
 }
 
 
 @pytest.mark.parametrize("name", sorted(GROUPS))
-def test_linear_group_matches_the_oracle_problem_by_problem(name):
+def test_linear_group_matches_the_oracle_problem_by_problem(name, monkeypatch, capfd):
     """*_resq_linear_group: one quantizer launch and one GEMM launch over the tiles of all problems; every problem is
     checked element by element against the oracle, and a second run must reproduce the first bit for bit (the partial
     tiles are summed in a fixed order)."""
@@ -626,9 +631,17 @@ def test_linear_group_matches_the_oracle_problem_by_problem(name):
         tensors.append((xb, wb))
         problems.append((to_dev(xb), wc, ws))
     work = m.alloc_workspace(m.resq_group_workspace_bytes(problems, pattern, fmt, out_dtype))
+    monkeypatch.setenv("RESQ_GEMM_DEBUG", "1")           # the launcher prints the schedule it planned
+    if name == "two-classes":                            # (the planner's own choice gives the first 26 pairs no dealt units)
+        monkeypatch.setenv("RESQ_GEMM_GROUP_DP", "100")
+        monkeypatch.setenv("RESQ_GEMM_GROUP_HI", "16")
     launches0 = m.kernel_launches()
     ys = m.resq_linear_group(problems, pattern, fmt, out_dtype=out_dtype, workspace=work)
     assert m.kernel_launches() - launches0 == 2          # one quantizer kernel, one GEMM kernel
+    plan = capfd.readouterr().err
+    monkeypatch.delenv("RESQ_GEMM_DEBUG")
+    if name == "two-classes":
+        assert "100 whole tiles" in plan and "first 26 pairs take 16 each" in plan, plan
     assert m.check(work) == 0, m.last_error()
     first = [y.clone() for y in ys]
     ys2 = m.resq_linear_group([p + (y,) for p, y in zip(problems, ys)], pattern, fmt, out_dtype=out_dtype, workspace=work)
