@@ -10,16 +10,23 @@ namespace resq {
 // FMA with (scale, scale/16) and (-128 scale, -8 scale) yields q*scale exactly for both nibbles of a
 // byte; the sign bits are then XOR-ed in.  Per pair of elements: one byte permute, one logic op, one
 // packed FMA, one logic op.
+// The scale words are linear in the metadata fields: with v = (s << 5) + (77 << 7) + ((e2 + e3) << 7) the bf16 bits of the
+// scale (s << 5 already is (E << 7) | (Mn << 5)), the word (scale, scale / 16) is v * 0x10001 - 0x02000000 =
+// s * 0x00200020 + (e2 + e3) * 0x00800080 + 0x24802680.  They are formed by integer multiply-adds (which run beside the
+// integer-ALU pipe that the element work below saturates) from three single-bit extractions.
+__device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t r;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+    return r;
+}
 __device__ __forceinline__ uint4 expand_hif4_chunk(uint32_t c, uint32_t meta, int chunk) {
-    // bf16 bits of (4+Mn) * 2^(E-52): exponent field E - 52 + 2 + 127, top mantissa bits Mn; s = E<<2|Mn
-    // so (s << 5) already is (E << 7) | (Mn << 5).
-    const uint32_t base = ((meta & 255u) << 5) + (77u << 7) + (((meta >> (8 + chunk)) & 1u) << 7);
-    const uint32_t sa = base + (((meta >> (16 + 2 * chunk)) & 1u) << 7);
-    const uint32_t sb = base + (((meta >> (17 + 2 * chunk)) & 1u) << 7);
-    const uint32_t scale_a = sa * 0x10001u - 0x02000000u;  // (scale, scale / 16)
-    const uint32_t scale_b = sb * 0x10001u - 0x02000000u;
-    const uint32_t add_a = scale_a + 0x83808380u;          // -(128 * scale) in both halves
-    const uint32_t add_b = scale_b + 0x83808380u;
+    const uint32_t e2 = (meta >> (8 + chunk)) & 1u;
+    const uint32_t e3 = (meta >> (16 + 2 * chunk)) & 3u;
+    const uint32_t base = mad_u32(e2, 0x00800080u, mad_u32(meta & 255u, 0x00200020u, 0x24802680u));
+    const uint32_t scale_a = mad_u32(e3 & 1u, 0x00800080u, base);  // (scale, scale / 16)
+    const uint32_t scale_b = mad_u32(e3 >> 1, 0x00800080u, base);
+    const uint32_t add_a = mad_u32(e3 & 1u, 0x00800080u, base + 0x83808380u);  // -(128 * scale) in both halves
+    const uint32_t add_b = mad_u32(e3 >> 1, 0x00800080u, base + 0x83808380u);
     const uint32_t c4 = c << 4;
     uint32_t out[4];
 #pragma unroll

@@ -631,6 +631,10 @@ gemm_pair_kernel(const __grid_constant__ PairMaps<NP> maps, const __grid_constan
         constexpr int rows_per_warp = my_rows / kGroupWarps;  // 8, 16 or 32
         const int r_begin = ew * rows_per_warp;
         const int sub_row = lane >> 3, chunk = lane & 7;
+        // Byte offsets of this lane's 16-byte stores into an expanded slot, for even and odd q (row r = r_begin + 4 q +
+        // sub_row, chunk column chunk ^ (r & 7)): rows four apart flip bit 2 of the swizzle, rows eight apart share it.
+        const uint32_t st_even = (uint32_t)((r_begin + sub_row) * 128 + ((chunk ^ ((r_begin + sub_row) & 7)) << 4));
+        const uint32_t st_odd = (uint32_t)((r_begin + sub_row + 4) * 128 + ((chunk ^ ((r_begin + sub_row + 4) & 7)) << 4));
         uint32_t it0 = 0;  // k-block counter at the start of the current tile
         bool ok = true;
         SegIter<TN, NP> si(p, pair, npairs);
@@ -690,10 +694,9 @@ gemm_pair_kernel(const __grid_constant__ PairMaps<NP> maps, const __grid_constan
                 if (lane == 0) ptx::mbar_arrive(&r_empty[sr]);
 #pragma unroll
                 for (int q = 0; q < kIters; ++q) {
-                    const int r = r_begin + q * 4 + sub_row;
                     const uint4 v = FMT == kHiF4 ? expand_hif4_chunk(cw[q], mw[q], chunk)
                                                  : expand_mxfp4_chunk(cw[q], (mw[q] >> (8 * (chunk >> 2))) & 255u);
-                    *reinterpret_cast<uint4*>(bexp + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
+                    *reinterpret_cast<uint4*>(bexp + ((q & 1) ? st_odd : st_even) + (q >> 1) * 1024) = v;
                 }
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
@@ -1307,6 +1310,17 @@ namespace {
 int res_mode(const GemmArgs& g) { return g.r_comp ? kResSparse24 : g.r_bf16 ? kResDense : kResNone; }
 template <int FMT>
 int streamk_fmt(const GemmArgs& g, cudaStream_t stream) {
+    // Four expander groups (768 threads, 80 registers) once a pair walks a dozen k-blocks or more: long runs are bound by
+    // the expanders' latency per k-block (M = 512, 7B shapes: step 494 -> 476 us; 3B down projection at M = 256: 49.3 ->
+    // 47.9 us), short ones lose a microsecond to the larger CTA (qkv at M = 256: 27.9 -> 29.0 us).
+    const int64_t units = ((g.M + 2 * kBM - 1) / (2 * kBM)) * ((g.N + kStreamKTN - 1) / kStreamKTN) * (g.K / kBK);
+    if (env_int("RESQ_GEMM_SK_GROUPS", units / kStreamKMaxPairs >= 12 ? 4 : 3) == 4) {
+        switch (res_mode(g)) {
+            case kResSparse24: return launch_pair_variant<kResSparse24, kStreamKTN, FMT, 4>(g, 1, stream, true);
+            case kResDense: return launch_pair_variant<kResDense, kStreamKTN, FMT, 4>(g, 1, stream, true);
+            default: return launch_pair_variant<kResNone, kStreamKTN, FMT, 4>(g, 1, stream, true);
+        }
+    }
     switch (res_mode(g)) {
         case kResSparse24: return launch_pair_variant<kResSparse24, kStreamKTN, FMT, 3>(g, 1, stream, true);
         case kResDense: return launch_pair_variant<kResDense, kStreamKTN, FMT, 3>(g, 1, stream, true);
