@@ -922,7 +922,9 @@ int pick_rings(PairParams<NP>& p, int64_t kb_per_pair, int* smem_bytes) {
     if (per_group == 1 && kb_per_pair >= 8 && env_int("RESQ_GEMM_DEEP_E", 1)) {
         // three activation slots cover the latency of their loads, one raw-code slot per group is enough, and
         // the rest goes to expanded-weight slots (any number: a k-block's barrier slot is k-block mod SE)
-        const int sa2 = env_int("RESQ_GEMM_MIN_SA", 3), sr2 = std::max(kExpGroups, std::min(env_int("RESQ_GEMM_MIN_SR", kExpGroups), kMaxRing));
+        // (the 512-wide tile with a dense residual operand fits a fourth expanded-weight slot only next to two activation
+        // slots: measured 2 % faster there, slower everywhere else)
+        const int sa2 = env_int("RESQ_GEMM_MIN_SA", (RES == kResDense && TN == 512) ? 2 : 3), sr2 = std::max(kExpGroups, std::min(env_int("RESQ_GEMM_MIN_SR", kExpGroups), kMaxRing));
         const int left = kSmemBudget - fixed - sa2 * kAStage - sr2 * raw_stage;
         const int se2 = std::min(std::min(left / exp_stage, 2 * kExpGroups), kMaxRing);
         if (se2 > kExpGroups) {
