@@ -554,26 +554,34 @@ def main():
         # public call and reads its output back.  The layers of a step are independent calls, so their copies run on
         # two copy streams beside the compute stream (input of the next layer and output of the previous one overlap
         # the current layer's kernels); the layer with the largest output goes first.  A step ends when every output
-        # is in host memory.
+        # is in host memory.  With a selection that is local to a token row, a large layer is called on row chunks (the
+        # public call on sub-matrices of X and Y), so that the read-back of a chunk's output overlaps the next chunk's
+        # kernels instead of starting after the whole layer: the step is bound by the outputs crossing PCIe.
         s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
         order = sorted(wl.layers, key=lambda L: -L["y"].numel())
+        row_local = (wl.pattern & 0xFF) in (0, 1, 2, 3)
+        chunk_rows = 4096 if row_local and wl.cfg.M >= 8192 else wl.cfg.M
+        chunks = [(r0, min(wl.cfg.M, r0 + chunk_rows)) for r0 in range(0, wl.cfg.M, chunk_rows)]
 
         def step_e2e(i, capturing=False):
             k = i % wl.n_sets
             main_s = torch.cuda.current_stream()
             s_in.wait_stream(main_s)    # earlier work on the staging buffers is done (previous steps were synchronized)
             for L in order:
-                with torch.cuda.stream(s_in):
-                    L["x_stage"].copy_(L["x_host"], non_blocking=True)       # host -> device, pinned
-                    L["ev_in"] = s_in.record_event()
+                L["ev_in"] = []
+                for (r0, r1) in chunks:
+                    with torch.cuda.stream(s_in):
+                        L["x_stage"][r0:r1].copy_(L["x_host"][r0:r1], non_blocking=True)   # host -> device, pinned
+                        L["ev_in"].append(s_in.record_event())
             for L in order:
                 wc, ws = L["w_sets"][k]
-                main_s.wait_event(L["ev_in"])
-                rq.resq_linear(L["x_stage"], wc, ws, wl.pattern, wl.fmt, Y=L["y"], workspace=L["work"])
-                ev = main_s.record_event()
-                with torch.cuda.stream(s_out):
-                    s_out.wait_event(ev)
-                    L["y_host"].copy_(L["y"], non_blocking=True)             # device -> host
+                for ci, (r0, r1) in enumerate(chunks):
+                    main_s.wait_event(L["ev_in"][ci])
+                    rq.resq_linear(L["x_stage"][r0:r1], wc, ws, wl.pattern, wl.fmt, Y=L["y"][r0:r1], workspace=L["work"])
+                    ev = main_s.record_event()
+                    with torch.cuda.stream(s_out):
+                        s_out.wait_event(ev)
+                        L["y_host"][r0:r1].copy_(L["y"][r0:r1], non_blocking=True)         # device -> host
             if capturing:
                 main_s.wait_stream(s_out)   # join the copy branches into the captured stream
             else:
@@ -599,7 +607,9 @@ def main():
         h2d = sum(L["x_host"].numel() * 2 for L in wl.layers)
         d2h = sum(L["y_host"].numel() * L["y_host"].element_size() for L in wl.layers)
         return {"value": world * wl.flops_step / (ms_e2e / steps * 1e-3) / 1e12, "unit": "TFLOP/s",
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / steps}
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / steps,
+                "calls_per_layer": len(chunks), "note": "bound by the outputs crossing PCIe: d2h bytes / time = "
+                f"{d2h / (ms_e2e / steps * 1e-3) / 1e9:.1f} GB/s"}
 
     def gemm_roofline(res, fmt_):
         """Roofline object of the dominant kernel (the GEMM) from a measure() result."""
