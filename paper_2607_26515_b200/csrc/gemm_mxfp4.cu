@@ -5,7 +5,12 @@
 // operands straight from shared memory and applies the scales, which it reads from tensor memory: nothing is
 // expanded.  Selected entries of the residual are kept by zeroing the dropped codes (the quantizer does that).
 //
-// One CTA per SM walks 128 x 256 output tiles.  A stage is 256 values of K: 128 x 128 B of activation codes
+// One CTA per SM walks 128 x 256 output tiles, or (PAIR, for more than 128 token rows) a cluster of two CTAs walks
+// 256 x 256 tiles with tcgen05.mma.cta_group::2: each CTA loads the codes of its own 128 token rows and of HALF of the
+// tile's 256 weight rows (the tensor cores read the other half from the peer's shared memory), which cuts the bytes an
+// SM pulls from L2 per unit of tensor work by a quarter to a third -- the bound of this kernel.  Every CTA still stages
+// the scales of all 256 weight rows (each SM scales its own partial products).  No TMA multicast.
+// A stage is 256 values of K: 128 x 128 B of activation codes
 // (and as much for the residual), 256 x 128 B of weight codes, and their scales re-arranged into the 512-byte
 // atoms tcgen05.cp copies to tensor memory (32 rows x 16 B: byte r1 * 4 + g of row r0 is the scale of row
 // r0 + 32 * r1 for the g-th group of 32 values).
@@ -72,69 +77,104 @@ __device__ __forceinline__ uint64_t smem_desc_sf(uint32_t addr) {
     d |= (uint64_t)1 << 46;
     return d;
 }
+template <bool PAIR>
 __device__ __forceinline__ void tmem_cp_sf(uint32_t taddr, uint64_t desc) {
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
+    if constexpr (PAIR) asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
+    else asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
 }
+template <bool PAIR>
 __device__ __forceinline__ void umma_mxf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t sfa,
                                           uint32_t sfb, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-        :
-        : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
-        : "memory");
+    if constexpr (PAIR)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+            :
+            : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+            :
+            : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
+            : "memory");
 }
 
-template <bool RES>
+constexpr int kMaxStagesNative = 6;
+
+template <bool RES, bool PAIR>
 struct StageLayout {
-    static constexpr int kStagesN = RES ? 3 : 4;
+    static constexpr int kBBytes = PAIR ? kBTile / 2 : kBTile;          // weight codes this CTA loads per stage
+    static constexpr int kStagesN = PAIR ? (RES ? 4 : 6) : (RES ? 3 : 4);
     static constexpr int kA = 0;
     static constexpr int kAr = kATile;                                  // only with RES
     static constexpr int kB = kATile * (RES ? 2 : 1);
-    static constexpr int kSfAOff = kB + kBTile;
+    static constexpr int kSfAOff = kB + kBBytes;
     static constexpr int kSfArOff = kSfAOff + kSfA;                      // only with RES
     static constexpr int kSfBOff = kSfAOff + kSfA * (RES ? 2 : 1);
     static constexpr int kBytes = kSfBOff + kSfB;
-    static constexpr uint32_t kTxBytes = (uint32_t)(kATile * (RES ? 2 : 1) + kBTile);
+    static constexpr uint32_t kTxBytes = (uint32_t)(kATile * (RES ? 2 : 1) + kBBytes);
 };
 
-template <bool RES>
+template <bool RES, bool PAIR>
 __global__ void __launch_bounds__(kThreadsNative, 1)
 gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_r,
                          const __grid_constant__ CUtensorMap tmap_w, const NativeParams p) {
-    using L = StageLayout<RES>;
+    using L = StageLayout<RES, PAIR>;
     constexpr int S = L::kStagesN;
+    constexpr int kTileM = PAIR ? 2 * kBM : kBM;  // token rows of a tile (of the pair's tile)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * L::kBytes);
-    uint64_t* full = bars;            // [S] codes landed (TMA bytes) and scale atoms written (two gather warps)
-    uint64_t* empty = bars + 4;       // [S] the MMAs that read the stage completed
-    uint64_t* acc_full = bars + 8;    // accumulator complete
-    uint64_t* acc_empty = bars + 9;   // accumulator drained by the four epilogue warps
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+    // PAIR: the leader's "full" barriers collect both CTAs' bytes and gather warps; "empty" and "acc_full" are released in
+    // both CTAs by one multicast commit; the leader's "acc_empty" collects both CTAs' epilogue warps.
+    uint64_t* full = bars;                                // [S] codes landed (TMA bytes) and scale atoms written
+    uint64_t* empty = bars + kMaxStagesNative;            // [S] the MMAs that read the stage completed
+    uint64_t* acc_full = bars + 2 * kMaxStagesNative;     // accumulator complete
+    uint64_t* acc_empty = acc_full + 1;                   // accumulator drained by the epilogue warps
+    // PAIR, second CTA: its gather warps arrive here, and its otherwise idle warp 1 forwards each completed phase to the
+    // leader's "full" barrier (a remote arrive with cluster-scope release stalls its thread for hundreds of cycles:
+    // kept off the gather warps, which handle every stage)
+    uint64_t* sf_ready = acc_empty + 1;                   // [S]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sf_ready + kMaxStagesNative);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = (int)(p.K / kBKe);
+    const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;  // 0 = leader
+    const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, nworkers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            ptx::mbar_init(&full[s], 3);
+            // leader: an arrive.expect_tx per CTA, its own two gather warps, and (PAIR) the peer's forwarding thread
+            ptx::mbar_init(&full[s], PAIR ? 5 : 3);
             ptx::mbar_init(&empty[s], 1);
+            ptx::mbar_init(&sf_ready[s], 2);
         }
         ptx::mbar_init(acc_full, 1);
-        ptx::mbar_init(acc_empty, 4);
+        ptx::mbar_init(acc_empty, PAIR ? 8 : 4);
         *abort_flag = 0;
         ptx::mbar_fence_init();
     }
-    if (warp == 1) ptx::tmem_alloc(tmem_slot, kTmemColsNative);
+    if (warp == 1) {
+        if constexpr (PAIR) ptx::tmem_alloc_pair(tmem_slot, kTmemColsNative);
+        else ptx::tmem_alloc(tmem_slot, kTmemColsNative);
+    }
     ptx::tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) ptx::cluster_sync();  // the peer's barriers exist before anything arrives on them
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     pdl_trigger();
     pdl_wait();  // codes and scales of the activations come from the quantizer kernel just before
+    // arrive on full[s] of the leader
+    auto arrive_full = [&](uint64_t* bar) {
+        if constexpr (PAIR) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar, 0));
+        else ptx::mbar_arrive(bar);
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -144,8 +184,8 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
             ptx::tma_prefetch_desc(&tmap_w);
             uint32_t s = 0, ph = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile / p.ntiles_n) * kBM, n0 = (tile % p.ntiles_n) * kBN;
+            for (int tile = worker; tile < p.num_tiles && ok; tile += nworkers) {
+                const int m0 = (tile / p.ntiles_n) * kTileM + (int)rank * kBM, n0 = (tile % p.ntiles_n) * kBN;
                 for (int kb = 0; kb < nkb; ++kb) {
                     if (!ptx::mbar_wait_spin(&empty[s], ph ^ 1u, abort_flag)) {
                         report_timeout_native(p.status, 1);
@@ -153,23 +193,47 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                         break;
                     }
                     uint8_t* st = smem + (size_t)s * L::kBytes;
-                    ptx::mbar_arrive_expect_tx(&full[s], L::kTxBytes);
-                    ptx::tma_load_2d(st + L::kA, &tmap_a, &full[s], kb * kRowBytes, m0);
-                    if (RES) ptx::tma_load_2d(st + L::kAr, &tmap_r, &full[s], kb * kRowBytes, m0);
-                    ptx::tma_load_2d(st + L::kB, &tmap_w, &full[s], kb * kRowBytes, n0);
+                    if constexpr (PAIR) {
+                        const uint32_t fb = ptx::map_to_cta(&full[s], 0);
+                        ptx::mbar_arrive_expect_tx_cluster_relaxed(fb, L::kTxBytes);  // publishes nothing itself
+                        ptx::tma_load_2d_pair(st + L::kA, &tmap_a, fb, kb * kRowBytes, m0);
+                        if (RES) ptx::tma_load_2d_pair(st + L::kAr, &tmap_r, fb, kb * kRowBytes, m0);
+                        ptx::tma_load_2d_pair(st + L::kB, &tmap_w, fb, kb * kRowBytes, n0 + (int)rank * (kBN / 2));
+                    } else {
+                        ptx::mbar_arrive_expect_tx(&full[s], L::kTxBytes);
+                        ptx::tma_load_2d(st + L::kA, &tmap_a, &full[s], kb * kRowBytes, m0);
+                        if (RES) ptx::tma_load_2d(st + L::kAr, &tmap_r, &full[s], kb * kRowBytes, m0);
+                        ptx::tma_load_2d(st + L::kB, &tmap_w, &full[s], kb * kRowBytes, n0);
+                    }
                     if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (PAIR && lane == 0 && rank == 1) {
+            // forward the peer's "scale atoms written" to the leader, stage by stage
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            for (int tile = worker; tile < p.num_tiles && ok; tile += nworkers) {
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!ptx::mbar_wait_spin(&sf_ready[s], ph, abort_flag)) {
+                        report_timeout_native(p.status, 7);
+                        ok = false;
+                        break;
+                    }
+                    ptx::mbar_arrive_cluster(ptx::map_to_cta(&full[s], 0));
+                    if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+        if (lane == 0 && rank == 0) {
             const uint64_t desc0 = ptx::smem_desc_sw128_kmajor(0);
             const uint32_t smem_base16 = (ptx::smem_u32(smem) & 0x3FFFFu) >> 4;
             uint32_t s = 0, ph = 0, it = 0;
             int local_tile = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local_tile) {
+            for (int tile = worker; tile < p.num_tiles && ok; tile += nworkers, ++local_tile) {
                 if (!ptx::mbar_wait_spin(acc_empty, (uint32_t)(local_tile & 1) ^ 1u, abort_flag)) {
                     report_timeout_native(p.status, 6);
                     break;
@@ -187,11 +251,11 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                     const uint32_t sf = tmem_base + (uint32_t)(kAccCols + (it & 1u) * kSfSetCols);
 #pragma unroll
                     for (int ka = 0; ka < 2; ++ka) {
-                        tmem_cp_sf(sf + ka * 4, smem_desc_sf(st + L::kSfAOff + ka * kSfAtom));
-                        if (RES) tmem_cp_sf(sf + 8 + ka * 4, smem_desc_sf(st + L::kSfArOff + ka * kSfAtom));
+                        tmem_cp_sf<PAIR>(sf + ka * 4, smem_desc_sf(st + L::kSfAOff + ka * kSfAtom));
+                        if (RES) tmem_cp_sf<PAIR>(sf + 8 + ka * 4, smem_desc_sf(st + L::kSfArOff + ka * kSfAtom));
 #pragma unroll
                         for (int nb = 0; nb < 2; ++nb)
-                            tmem_cp_sf(sf + 16 + ka * 8 + nb * 4, smem_desc_sf(st + L::kSfBOff + (ka * 2 + nb) * kSfAtom));
+                            tmem_cp_sf<PAIR>(sf + 16 + ka * 8 + nb * 4, smem_desc_sf(st + L::kSfBOff + (ka * 2 + nb) * kSfAtom));
                     }
                     const uint32_t st16 = smem_base16 + s * (uint32_t)(L::kBytes >> 4);
                     const uint64_t adesc = desc0 + (uint64_t)(st16 + (L::kA >> 4));
@@ -201,18 +265,22 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                     for (int k4 = 0; k4 < 4; ++k4) {  // 64 values (32 B) of K per MMA: two scale groups
                         const int ka = k4 >> 1;
                         const uint32_t sfid = (uint32_t)(k4 & 1) * 2u;
-                        const uint32_t idesc = idesc_mxf4(kBM, kBN, sfid, sfid);
+                        const uint32_t idesc = idesc_mxf4(kTileM, kBN, sfid, sfid);
                         const uint32_t sfa = sf + ka * 4 + (sfid << 30), sfb = sf + 16 + ka * 8 + (sfid << 30);
-                        umma_mxf4(tmem_base, adesc + (uint64_t)(2 * k4), bdesc + (uint64_t)(2 * k4), idesc, sfa, sfb,
-                                  (kb > 0 || k4 > 0) ? 1u : 0u);
+                        umma_mxf4<PAIR>(tmem_base, adesc + (uint64_t)(2 * k4), bdesc + (uint64_t)(2 * k4), idesc, sfa, sfb,
+                                        (kb > 0 || k4 > 0) ? 1u : 0u);
                         if (RES)
-                            umma_mxf4(tmem_base, rdesc + (uint64_t)(2 * k4), bdesc + (uint64_t)(2 * k4), idesc,
-                                      sf + 8 + ka * 4 + (sfid << 30), sfb, 1u);
+                            umma_mxf4<PAIR>(tmem_base, rdesc + (uint64_t)(2 * k4), bdesc + (uint64_t)(2 * k4), idesc,
+                                            sf + 8 + ka * 4 + (sfid << 30), sfb, 1u);
                     }
-                    ptx::umma_commit(&empty[s]);
+                    if constexpr (PAIR) ptx::umma_commit_pair(&empty[s], 3);  // frees the stage in both CTAs
+                    else ptx::umma_commit(&empty[s]);
                     if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
                 }
-                if (ok) ptx::umma_commit(acc_full);
+                if (ok) {
+                    if constexpr (PAIR) ptx::umma_commit_pair(acc_full, 3);
+                    else ptx::umma_commit(acc_full);
+                }
             }
         }
     } else if (warp < 4) {
@@ -226,7 +294,7 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         bool ok = true;
         uint2 va[2], vr[2], vw[4];
         auto load_scales = [&](int tile, int kb) {
-            const int64_t m0 = (int64_t)(tile / p.ntiles_n) * kBM, n0 = (int64_t)(tile % p.ntiles_n) * kBN;
+            const int64_t m0 = (int64_t)(tile / p.ntiles_n) * kTileM + rank * kBM, n0 = (int64_t)(tile % p.ntiles_n) * kBN;
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 const int64_t m = m0 + t + 64 * j;
@@ -243,7 +311,7 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                 if (n < p.N) vw[j] = *reinterpret_cast<const uint2*>(p.w_scale + n * spr + kb * 8);
             }
         };
-        int tile = blockIdx.x, kb = 0;
+        int tile = worker, kb = 0;
         if (tile < p.num_tiles) load_scales(tile, kb);
         while (tile < p.num_tiles && ok) {
             if (!ptx::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) {
@@ -274,11 +342,14 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
             }
             ptx::fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&full[s]);
+            if (lane == 0) {
+                if (PAIR && rank == 1) ptx::mbar_arrive(&sf_ready[s]);
+                else ptx::mbar_arrive(&full[s]);
+            }
             if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
             if (++kb == nkb) {
                 kb = 0;
-                tile += gridDim.x;
+                tile += nworkers;
             }
             if (tile < p.num_tiles) load_scales(tile, kb);  // in flight while the next slot is awaited
         }
@@ -286,8 +357,8 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         // ------------------------------------------------------------------ epilogue (warps 4..7)
         const int quad = warp & 3;
         int local_tile = 0;
-        for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++local_tile) {
-            const int64_t m0 = (int64_t)(tile / p.ntiles_n) * kBM, n0 = (int64_t)(tile % p.ntiles_n) * kBN;
+        for (int tile = worker; tile < p.num_tiles; tile += nworkers, ++local_tile) {
+            const int64_t m0 = (int64_t)(tile / p.ntiles_n) * kTileM + rank * kBM, n0 = (int64_t)(tile % p.ntiles_n) * kBN;
             if (!ptx::mbar_wait(acc_full, (uint32_t)(local_tile & 1), abort_flag)) {
                 report_timeout_native(p.status, 4);
                 break;
@@ -302,7 +373,7 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                 if (cc == kBN / 32 - 1) {
                     ptx::tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(acc_empty);
+                    if (lane == 0) arrive_full(acc_empty);
                 }
                 if (m >= p.M) continue;
                 const int64_t nb = n0 + cc * 32;
@@ -342,15 +413,18 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     }
     ptx::tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) ptx::cluster_sync();  // no CTA leaves while the peer may still signal its barriers or read its shared memory
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, kTmemColsNative);
+        if constexpr (PAIR) ptx::tmem_dealloc_pair(tmem_base, kTmemColsNative);
+        else ptx::tmem_dealloc(tmem_base, kTmemColsNative);
     }
 }
 
-template <bool RES>
+template <bool RES, bool PAIR>
 int launch_native_variant(const Mxfp4NativeArgs& g, cudaStream_t stream) {
-    using L = StageLayout<RES>;
+    using L = StageLayout<RES, PAIR>;
+    constexpr int kTileM = PAIR ? 2 * kBM : kBM;
     CUtensorMap ta, tr, tw;
     int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.a_codes, (uint64_t)g.K / 2, (uint64_t)g.M, (uint64_t)g.K / 2,
                           kRowBytes, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -359,7 +433,7 @@ int launch_native_variant(const Mxfp4NativeArgs& g, cudaStream_t stream) {
                       (uint64_t)g.K / 2, kRowBytes, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
     rc = make_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_UINT8, g.w_codes, (uint64_t)g.K / 2, (uint64_t)g.N, (uint64_t)g.K / 2,
-                      kRowBytes, kBN, CU_TENSOR_MAP_SWIZZLE_128B);
+                      kRowBytes, PAIR ? kBN / 2 : kBN, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
     NativeParams p;
     p.a_scale = g.a_scale;
@@ -369,21 +443,40 @@ int launch_native_variant(const Mxfp4NativeArgs& g, cudaStream_t stream) {
     p.N = g.N;
     p.K = g.K;
     p.ntiles_n = (int)((g.N + kBN - 1) / kBN);
-    p.num_tiles = (int)((g.M + kBM - 1) / kBM) * p.ntiles_n;
+    p.num_tiles = (int)((g.M + kTileM - 1) / kTileM) * p.ntiles_n;
     p.Y = g.Y;
     p.out_f32 = g.out_dtype == RESQ_OUT_F32;
     p.ldy = g.ldy;
     p.status = g.status;
     const int smem_bytes = 1024 + L::kStagesN * L::kBytes + 256;
     static_assert(1024 + L::kStagesN * L::kBytes + 256 <= kSmemBudgetNative, "stages do not fit");
-    auto kern = gemm_mxfp4_native_kernel<RES>;
+    auto kern = gemm_mxfp4_native_kernel<RES, PAIR>;
     rc = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem_bytes, "cudaFuncSetAttribute(gemm mxfp4)");
     if (rc) return rc;
     const int num_sms = device_sm_count();
-    const unsigned grid = (unsigned)std::min(p.num_tiles, num_sms);
     LaunchScope scope(kKindGemm, stream);
-    return cuda_fail(launch_kernel(kern, dim3(grid), dim3(kThreadsNative), (size_t)smem_bytes, stream, ta, tr, tw, p),
-                     "gemm_mxfp4_native_kernel launch");
+    if constexpr (!PAIR) {
+        const unsigned grid = (unsigned)std::min(p.num_tiles, num_sms);
+        return cuda_fail(launch_kernel(kern, dim3(grid), dim3(kThreadsNative), (size_t)smem_bytes, stream, ta, tr, tw, p),
+                         "gemm_mxfp4_native_kernel launch");
+    } else {
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3((unsigned)(2 * std::min(p.num_tiles, num_sms / 2)), 1, 1);
+        cfg.blockDim = dim3(kThreadsNative, 1, 1);
+        cfg.dynamicSmemBytes = (size_t)smem_bytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pdl_enabled() ? 2 : 1;
+        return cuda_fail(cudaLaunchKernelEx(&cfg, kern, ta, tr, tw, p), "gemm_mxfp4_native_kernel (pair) launch");
+    }
 }
 
 }  // namespace
@@ -408,7 +501,14 @@ int launch_gemm_mxfp4_native(const Mxfp4NativeArgs& g, cudaStream_t stream) {
         set_last_error("native MXFP4 GEMM: scale arrays must be 8-byte aligned");
         return RESQ_ERR_ALIGN;
     }
-    return g.r_codes ? launch_native_variant<true>(g, stream) : launch_native_variant<false>(g, stream);
+    // CTA pairs (256 x 256 tiles, a third less L2 -> SM traffic per unit of tensor work) are built and parity-tested but
+    // measured slower than one CTA per tile (7B prefill shapes, whole step: NONE 3.34 against 2.98 ms, DENSE 4.30 against
+    // 4.19 ms; decode shapes lose more, having half as many tiles to spread): opt-in by RESQ_MXFP4_PAIR=1 (debugging
+    // override).  What the pair costs -- the scale copies and MMAs of both SMs issued by one thread, the cross-CTA
+    // arrivals on the critical path of every 256-value stage -- outweighs the saved traffic.
+    const bool pair = env_int("RESQ_MXFP4_PAIR", 0) != 0 && g.M > kBM;
+    if (pair) return g.r_codes ? launch_native_variant<true, true>(g, stream) : launch_native_variant<false, true>(g, stream);
+    return g.r_codes ? launch_native_variant<true, false>(g, stream) : launch_native_variant<false, false>(g, stream);
 }
 
 }  // namespace resq

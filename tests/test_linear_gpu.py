@@ -707,3 +707,16 @@ def test_backward_products_argument_errors():
     with pytest.raises(m.ResqError) as e:
         m.pack_weight_transposed(w)
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_DENSE, oracle.S_2_4, oracle.S_ROW50])
+@pytest.mark.parametrize("shape", [(288, 1024, 1000), (1024, 2048, 1100), (200, 256, 256)])
+def test_mxfp4_fp4_route_on_cta_pairs(shape, pattern, monkeypatch):
+    """The block-scaled FP4 route with tcgen05.mma.cta_group::2 (256 x 256 tiles over two SMs; opt-in): several tiles per
+    pair, ragged M and N, rows beyond one M tile."""
+    M, K, N = shape
+    monkeypatch.setenv("RESQ_MXFP4_NATIVE", "1")
+    monkeypatch.setenv("RESQ_MXFP4_PAIR", "1")
+    xb, wb = synth_xw(3 * M + N + pattern, M, K, N, n_out=max(1, K // 256))
+    run_case(xb, wb, pattern, fmt="mxfp4")
+    run_case(xb, wb, pattern, fmt="mxfp4", out_dtype=torch.bfloat16)
