@@ -71,8 +71,8 @@ RHO.update({p: ((p >> 8) & 0xF) / 4.0 if (p >> 8) & 0xF else 0.5 for p in PATTER
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the dominant GEMM kernel from ncu captures
 # of single layers (summaries with their commands under profiles/), keyed by (config, layer, pattern id, format)
 NCU_TRAFFIC = {
-    (4, "gate_up", 2, "hif4"): {"bytes": 3.83e9, "source": "profiles/gemm_pair_kernel_7b-prefill-gate_up_dram.md"},
-    (4, "qkv", 2, "hif4"): {"bytes": 3.82e8, "source": "profiles/gemm_pair_kernel_7b-prefill-qkv_2to4.md"},
+    (4, "gate_up", 2, "hif4"): {"bytes": 3.53e9, "source": "profiles/gemm_pair_kernel_7b-prefill-gate_up_dram.md"},
+    (4, "qkv", 2, "hif4"): {"bytes": 3.21e8, "source": "profiles/gemm_pair_kernel_7b-prefill-qkv_2to4.md"},
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
