@@ -449,6 +449,9 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
         a.a_bf16 = reinterpret_cast<__nv_bfloat16*>(region_a);
         a.r_bf16 = reinterpret_cast<__nv_bfloat16*>(region_r);
     }
+    // block-wise selection on the CTA-pair kernel: the GEMM reads the keep flags, the image stays unmasked
+    const bool block_lists = !native && pattern == RESQ_S_BLOCK32x64_50 && a.r_bf16 && gemm_block_lists_supported(M, N, K);
+    a.skip_image_mask = block_lists ? 1 : 0;
     rc = launch_quantize(fmt, a, st);
     if (rc) return rc;
     if (native) {
@@ -478,6 +481,7 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
     g.r_meta = a.r_meta;
     g.meta_rows128 = a.meta_rows128;
     g.meta_ka = a.meta_ka;
+    g.blk_flags = block_lists ? a.keep_flags : nullptr;
     g.w_codes = static_cast<const uint8_t*>(w_codes);
     g.w_side = w_side;
     g.w_bf16 = static_cast<const __nv_bfloat16*>(w_bf16);

@@ -123,6 +123,8 @@ struct QuantArgs {
     __nv_bfloat16* r_comp;  // [M, K/2]
     uint8_t* r_meta;
     int64_t meta_rows128, meta_ka;
+    // BLOCK only: leave r_bf16 unmasked (the GEMM takes the keep flags and loads zero tiles for the dropped blocks)
+    int skip_image_mask;
     // scratch
     double* scores;         // CHAN50: [K]; BLOCK: [(M/32) * (K/64)]
     uint8_t* keep_flags;    // CHAN50: [K]; BLOCK: [(M/32) * (K/64)]
@@ -159,6 +161,10 @@ struct GemmArgs {
     const __nv_bfloat16* r_comp;   // [M, K/2] the two kept values of every four consecutive channels, in channel order
     const uint8_t* r_meta;         // index metadata, sparse24_meta_offset() layout: meta_rows128 x meta_ka blocks of 2 KB
     int64_t meta_rows128, meta_ka;
+    // block-wise selection, with r_bf16 (CTA-pair kernel only): r_bf16 is the unmasked image of deq Q(dX) and
+    // blk_flags [(M/32), K/64] says which blocks of 32 rows x 64 channels are kept (nonzero); the kernel loads a zero tile
+    // in place of a dropped block
+    const uint8_t* blk_flags;
     const uint8_t* w_codes;        // [N, K/2]
     const void* w_side;            // [N, K/64] u32 or [N, K/32] u8
     const __nv_bfloat16* w_bf16;   // instead of w_codes / w_side: plain bf16 weights [N, K], row pitch ldw ("W16A4")
@@ -182,6 +188,8 @@ int launch_gemm_pair_group(const GemmArgs* g, int count, cudaStream_t stream);
 size_t gemm_pair_streamk_scratch_bytes();
 // Test hook behind resq_debug_expire_next_wait (gemm_pair.cu).
 void debug_expire_next_wait(int on);
+// Whether launch_gemm_hif4 takes the keep flags of the block-wise selection for this shape (see GemmArgs::blk_flags).
+bool gemm_block_lists_supported(int64_t M, int64_t N, int64_t K);
 // Whether launch_gemm_hif4 takes the compressed 2:4 residual for this shape (the CTA-pair kernel runs it).
 bool gemm_sparse24_supported(int64_t M, int64_t N, int64_t K);
 // Layout of the 2:4 index metadata, fixed by the sparse MMA: blocks of 128 rows x 128 K positions (2 KB, row bands

@@ -740,6 +740,20 @@ bool gemm_sparse24_supported(int64_t M, int64_t N, int64_t K) {
     return rounds480 * 0.78 < rounds512;
 }
 
+// Block-wise selection: the CTA-pair kernel can take the keep flags and an unmasked residual image, which saves the
+// read-modify-write pass over the image and the loads of the dropped blocks.  Used from 2048 token rows on: there the
+// pass is what costs (7B prefill shapes at M = 16384: quantizer + selection + GEMM 11.27 against 11.86 ms per step; the
+// wide layer's GEMM itself gains 4 %, the narrow ones lose up to 5 % to the four small boxes per tile), at M = 512 the
+// saved pass (7 us per layer) and the slower K-streamed GEMM (4-15 us) cancel.  RESQ_BLOCK_LISTS = 0 / 1 forces the
+// choice (debugging override).
+bool gemm_block_lists_supported(int64_t M, int64_t N, int64_t K) {
+    (void)N;
+    if (M <= pair_min_m() || M % 32 != 0 || K % kBK != 0 || !env_int("RESQ_GEMM_PAIR", 1)) return false;
+    const int forced = env_int("RESQ_BLOCK_LISTS", -1);
+    if (forced >= 0) return forced != 0;
+    return M >= 2048;
+}
+
 size_t gemm_hif4_scratch_bytes(int64_t M, int64_t N, int64_t K) {
     size_t classic = 0;
     const int splits = gemm_hif4_pick_splits(M, N, K);
@@ -782,6 +796,10 @@ int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream) {
         const int splits = (c.splits > 1 && g.splitk_partials && c.splits <= g.splits) ? c.splits : 1;
         return launch_gemm_pair_plainw(g, c.pair_tn >= 384 ? 512 : 256, splits, false, stream);
     }
+    if (g.blk_flags && (g.M <= pair_min_m() || !env_int("RESQ_GEMM_PAIR", 1))) {  // (any call the pair kernel runs takes them)
+        set_last_error("internal: keep flags given for a shape the pair kernel does not run");
+        return RESQ_ERR_CUDA;
+    }
     if (streamk) return launch_gemm_pair_streamk(g, stream);
     TileChoice tc = choose_tile(g.M, g.N, g.K, res, g.r_comp != nullptr);
     if (tc.splits > 1 && (!g.splitk_partials || tc.splits > g.splits)) tc.splits = 1;
@@ -806,6 +824,7 @@ int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream) {
             const int64_t lda = g.lda ? g.lda : g.K;
             tail_part.a_bf16 = g.a_bf16 + m0 * lda;
             if (g.r_bf16) tail_part.r_bf16 = g.r_bf16 + m0 * lda;
+            if (g.blk_flags) tail_part.blk_flags = g.blk_flags + (m0 / 32) * (g.K / kBK);
             tail_part.lda = lda;
             if (g.w_bf16) {
                 tail_part.w_bf16 = g.w_bf16 + n0 * g.ldw;

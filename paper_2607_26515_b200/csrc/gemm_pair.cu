@@ -61,6 +61,7 @@ struct PairProblem {
     int dealt_first;         // K-streamed schedule: first tile of the problem whose k-blocks are dealt out (else whole)
     int64_t unit_base;       //   and the (tile, k-block) units of the dealt tiles of the problems before it
     int meta_ka;             // sparse residual: metadata blocks (128 K positions) per 128-row band
+    const uint8_t* blk_flags;  // dense residual from an unmasked image: keep flags [(M / 32), G] of the 32 x 64 blocks, or null
 };
 
 template <int NP>
@@ -443,7 +444,7 @@ gemm_pair_kernel(const __grid_constant__ PairMaps<NP> maps, const __grid_constan
             for (int q = 0; q < (NP > 1 ? p.nprob : 1); ++q) {
                 ptx::tma_prefetch_desc(&maps.a[q]);
                 if (RES != kResNone) ptx::tma_prefetch_desc(&maps.r[q]);
-                if (RES == kResSparse24) ptx::tma_prefetch_desc(&maps.e[q]);
+                if (RES == kResSparse24 || (RES == kResDense && p.pr[q].blk_flags)) ptx::tma_prefetch_desc(&maps.e[q]);
             }
             uint32_t it = 0;
             bool ok = true;
@@ -455,6 +456,21 @@ gemm_pair_kernel(const __grid_constant__ PairMaps<NP> maps, const __grid_constan
                 const CUtensorMap* tmap_r = &maps.r[tc.prob];
                 const CUtensorMap* tmap_e = &maps.e[tc.prob];
                 const int meta_ka = p.pr[tc.prob].meta_ka;
+                // Block-wise selection: the residual tile is loaded as four boxes of 32 rows, a dropped block from beyond the
+                // tensor's last row (TMA fills it with zeros and reads nothing).  The flags of a k-block are fetched while
+                // the previous one waits for its slot.
+                const uint8_t* blk_flags = RES == kResDense ? p.pr[tc.prob].blk_flags : nullptr;
+                const int blk_G = p.pr[tc.prob].G, blk_M = p.pr[tc.prob].M;
+                const int oob_row = (blk_M + 2 * kBM - 1) / (2 * kBM) * (2 * kBM);
+                uint32_t fl[4] = {0u, 0u, 0u, 0u};
+                auto fetch_flags = [&](int kb) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const int row = my_m + 32 * g;
+                        fl[g] = row < blk_M ? ptx::ld_nc_u8(blk_flags + (size_t)(row >> 5) * blk_G + kb) : 0u;
+                    }
+                };
+                if (blk_flags && tc.nkb > 0) fetch_flags(tc.kb_begin);
                 for (int i = 0; i < tc.nkb; ++i, ++it) {
                     // The activation ring may be shallower than the ring of expanded weights whose barriers it shares
                     // (barrier slot = k-block mod SE): slot it % SA is free once the MMAs of k-block it - SA, which
@@ -481,7 +497,16 @@ gemm_pair_kernel(const __grid_constant__ PairMaps<NP> maps, const __grid_constan
                         full, (uint32_t)(kAStage - (RES == kResSparse24 && !with_meta ? kSpMetaBytes : 0)));
                     const int kx = kb * kBK;
                     ptx::tma_load_2d_pair(st, tmap_a, full, kx, my_m);
-                    if (RES == kResDense) ptx::tma_load_2d_pair(st + kATileBytes, tmap_r, full, kx, my_m);
+                    if (RES == kResDense) {
+                        if (blk_flags) {
+#pragma unroll
+                            for (int g = 0; g < 4; ++g)
+                                ptx::tma_load_2d_pair(st + kATileBytes + g * 32 * 128, tmap_e, full, kx, fl[g] ? my_m + 32 * g : oob_row);
+                            if (i + 1 < tc.nkb) fetch_flags(kb + 1);
+                        } else {
+                            ptx::tma_load_2d_pair(st + kATileBytes, tmap_r, full, kx, my_m);
+                        }
+                    }
                     if (RES == kResSparse24) {
                         ptx::tma_load_2d_pair(st + kATileBytes, tmap_r, full, kx / 2, my_m);
                         if (with_meta)  // rows of 256 bytes, eight per 128 x 128 block
@@ -876,6 +901,9 @@ int make_problem_maps(const GemmArgs& g, CUtensorMap* ta, CUtensorMap* tr, CUten
         rc = make_tmap_2d(tr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, RES == kResDense ? g.r_bf16 : g.a_bf16, (uint64_t)g.K, (uint64_t)g.M,
                           (uint64_t)(g.lda ? g.lda : g.K) * 2, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
         *te = *ta;
+        if (RES == kResDense && g.blk_flags && !rc)  // the same image in boxes of 32 rows (one block of the selection)
+            rc = make_tmap_2d(te, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, g.r_bf16, (uint64_t)g.K, (uint64_t)g.M,
+                              (uint64_t)(g.lda ? g.lda : g.K) * 2, kBK, 32, CU_TENSOR_MAP_SWIZZLE_128B);
     }
     if (rc) return rc;
     if (FMT == kPlainW)
@@ -898,6 +926,7 @@ void fill_problem(PairProblem& pb, const GemmArgs& g) {
     pb.dealt_first = 0;
     pb.unit_base = 0;
     pb.meta_ka = (int)g.meta_ka;
+    pb.blk_flags = g.r_bf16 ? g.blk_flags : nullptr;
 }
 
 // Ring depths from the shared-memory budget.  Ring slots: a multiple of the number of expander groups (group g works
@@ -1373,7 +1402,7 @@ int launch_gemm_pair_streamk(const GemmArgs& g, cudaStream_t stream) {
 // the partial-tile slots of g[0].
 int launch_gemm_pair_group(const GemmArgs* g, int count, cudaStream_t stream) {
     for (int i = 1; i < count; ++i)
-        if (g[i].fmt != g[0].fmt || res_mode(g[i]) != res_mode(g[0]) || g[i].out_dtype != g[0].out_dtype || g[i].w_bf16) {
+        if (g[i].fmt != g[0].fmt || res_mode(g[i]) != res_mode(g[0]) || g[i].out_dtype != g[0].out_dtype || g[i].w_bf16 || g[i].blk_flags) {
             set_last_error("internal: the problems of a group must share format, residual mode and output type");
             return RESQ_ERR_CUDA;
         }

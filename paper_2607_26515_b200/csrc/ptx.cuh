@@ -100,6 +100,12 @@ __device__ __forceinline__ uint32_t ld_nc_u16(const uint16_t* p) {
     return (uint32_t)v;
 }
 
+__device__ __forceinline__ uint32_t ld_nc_u8(const uint8_t* p) {
+    uint32_t v;
+    asm volatile("ld.global.nc.u8 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
 // ---- fences ----------------------------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }

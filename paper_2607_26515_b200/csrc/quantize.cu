@@ -1804,11 +1804,13 @@ static int launch_global_select(const QuantArgs& a, int64_t nscore, cudaStream_t
                        "topk_select_kernel launch");
     }
     if (rc) return rc;
-    if (a.mask_bits || a.r_bf16 || (a.r_codes && a.mask_r_codes)) {
+    // (block-wise selection feeding the CTA-pair GEMM: the image stays unmasked, the GEMM reads the keep flags)
+    __nv_bfloat16* mask_img = (a.skip_image_mask && a.pattern == RESQ_S_BLOCK32x64_50) ? nullptr : a.r_bf16;
+    if (a.mask_bits || mask_img || (a.r_codes && a.mask_r_codes)) {
         const int64_t n = a.M * (a.K / 8);
         LaunchScope scope(kKindSelect, stream);
         rc = cuda_fail(launch_kernel(apply_global_mask_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, stream, a.pattern, a.M,
-                                     a.K, (const uint8_t*)a.keep_flags, a.mask_bits, a.r_bf16, a.mask_r_codes ? a.r_codes : (uint8_t*)nullptr),
+                                     a.K, (const uint8_t*)a.keep_flags, a.mask_bits, mask_img, a.mask_r_codes ? a.r_codes : (uint8_t*)nullptr),
                        "apply_global_mask_kernel launch");
     }
     return rc;

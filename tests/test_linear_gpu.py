@@ -720,3 +720,27 @@ def test_mxfp4_fp4_route_on_cta_pairs(shape, pattern, monkeypatch):
     xb, wb = synth_xw(3 * M + N + pattern, M, K, N, n_out=max(1, K // 256))
     run_case(xb, wb, pattern, fmt="mxfp4")
     run_case(xb, wb, pattern, fmt="mxfp4", out_dtype=torch.bfloat16)
+
+
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("case", [(288, 512, 600, False, {}), (160, 192, 80, False, {}), (1056, 1152, 1100, False, {"RESQ_GEMM_STREAMK": "0"}),
+                                  (2432, 1152, 2600, False, {}), (1024, 2048, 1100, True, {}), (300, 4160, 520, False, {"RESQ_GEMM_SPLITS": "2"})],
+                         ids=["streamed-k", "ragged", "whole-tiles", "many-tiles", "per-strip", "k-split"])
+def test_block_selection_through_keep_flags(case, fmt, monkeypatch):
+    """BLOCK with the residual image left unmasked: the GEMM reads the keep flags and loads a zero tile in place of every
+    dropped block of 32 rows x 64 channels (the default from 2048 rows on; forced here on small shapes, every schedule)."""
+    M, K, N, strips, env = case
+    if M % 32:
+        pytest.skip("the block pattern needs M % 32 == 0")
+    monkeypatch.setenv("RESQ_BLOCK_LISTS", "1")
+    monkeypatch.setenv("RESQ_MXFP4_NATIVE", "0")
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    pattern = oracle.per_strip(oracle.S_BLOCK) if strips else oracle.S_BLOCK
+    xb, wb = synth_xw(1311 + M, M, K, N, n_out=max(1, K // 256))
+    y = run_case(xb, wb, pattern, fmt=fmt)
+    monkeypatch.setenv("RESQ_BLOCK_LISTS", "0")
+    y_masked = run_case(xb, wb, pattern, fmt=fmt)
+    assert torch.equal(y, y_masked)  # same operands, same order of accumulation
+    monkeypatch.setenv("RESQ_BLOCK_LISTS", "1")
+    run_case(xb, wb, pattern, fmt=fmt, out_dtype=torch.bfloat16)
