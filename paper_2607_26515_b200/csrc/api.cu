@@ -469,6 +469,8 @@ int linear(int fmt, const void* X, int64_t M, int64_t K, int64_t ldx, const void
         n.Y = Y;
         n.out_dtype = out_dtype;
         n.ldy = ldy;
+        n.partial_bytes = gemm_hif4_scratch_bytes(M, N, K);
+        n.partials = n.partial_bytes ? reinterpret_cast<float*>(ws + used) : nullptr;
         n.status = a.status;
         return launch_gemm_mxfp4_native(n, st);
     }

@@ -215,6 +215,8 @@ struct Mxfp4NativeArgs {
     void* Y;
     int out_dtype;
     int64_t ldy;
+    float* partials;          // fp32 scratch for the partial tiles of a K split (decode-sized calls), or null
+    size_t partial_bytes;
     DeviceStatus* status;
 };
 bool gemm_mxfp4_native_supported(int64_t M, int64_t N, int64_t K, bool res);

@@ -49,6 +49,10 @@ struct NativeParams {
     const uint8_t* w_scale;   // [N, K/32]
     int64_t M, N, K;
     int ntiles_n, num_tiles;
+    // K split: work item = (tile, split), split sp covers the stages [sp * kb_per_split, ...); with more than one split
+    // the items write fp32 partial tiles into slabs [split][M][N] that the reduce kernel sums in a fixed order
+    int splits, kb_per_split;
+    float* partials;
     void* Y;
     int out_f32;
     int64_t ldy;
@@ -144,6 +148,13 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = (int)(p.K / kBKe);
+    const int nitems = p.num_tiles * p.splits;
+    auto item_of = [&](int item, int& tile, int& sp, int& kb0, int& kb1) {
+        tile = item / p.splits;
+        sp = item - tile * p.splits;
+        kb0 = sp * p.kb_per_split;
+        kb1 = min(nkb, kb0 + p.kb_per_split);
+    };
     const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;  // 0 = leader
     const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, nworkers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
@@ -184,9 +195,11 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
             ptx::tma_prefetch_desc(&tmap_w);
             uint32_t s = 0, ph = 0;
             bool ok = true;
-            for (int tile = worker; tile < p.num_tiles && ok; tile += nworkers) {
+            for (int item = worker; item < nitems && ok; item += nworkers) {
+                int tile, sp, kb0, kb1;
+                item_of(item, tile, sp, kb0, kb1);
                 const int m0 = (tile / p.ntiles_n) * kTileM + (int)rank * kBM, n0 = (tile % p.ntiles_n) * kBN;
-                for (int kb = 0; kb < nkb; ++kb) {
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!ptx::mbar_wait_spin(&empty[s], ph ^ 1u, abort_flag)) {
                         report_timeout_native(p.status, 1);
                         ok = false;
@@ -215,8 +228,10 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
             // forward the peer's "scale atoms written" to the leader, stage by stage
             uint32_t s = 0, ph = 0;
             bool ok = true;
-            for (int tile = worker; tile < p.num_tiles && ok; tile += nworkers) {
-                for (int kb = 0; kb < nkb; ++kb) {
+            for (int item = worker; item < nitems && ok; item += nworkers) {
+                int tile, sp, kb0, kb1;
+                item_of(item, tile, sp, kb0, kb1);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!ptx::mbar_wait_spin(&sf_ready[s], ph, abort_flag)) {
                         report_timeout_native(p.status, 7);
                         ok = false;
@@ -233,13 +248,15 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
             uint32_t s = 0, ph = 0, it = 0;
             int local_tile = 0;
             bool ok = true;
-            for (int tile = worker; tile < p.num_tiles && ok; tile += nworkers, ++local_tile) {
+            for (int item = worker; item < nitems && ok; item += nworkers, ++local_tile) {
+                int tile, sp, kb0, kb1;
+                item_of(item, tile, sp, kb0, kb1);
                 if (!ptx::mbar_wait_spin(acc_empty, (uint32_t)(local_tile & 1) ^ 1u, abort_flag)) {
                     report_timeout_native(p.status, 6);
                     break;
                 }
                 ptx::tc_fence_after();
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     if (!ptx::mbar_wait_spin(&full[s], ph, abort_flag)) {
                         report_timeout_native(p.status, 2);
                         ok = false;
@@ -268,7 +285,7 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                         const uint32_t idesc = idesc_mxf4(kTileM, kBN, sfid, sfid);
                         const uint32_t sfa = sf + ka * 4 + (sfid << 30), sfb = sf + 16 + ka * 8 + (sfid << 30);
                         umma_mxf4<PAIR>(tmem_base, adesc + (uint64_t)(2 * k4), bdesc + (uint64_t)(2 * k4), idesc, sfa, sfb,
-                                        (kb > 0 || k4 > 0) ? 1u : 0u);
+                                        (kb > kb0 || k4 > 0) ? 1u : 0u);
                         if (RES)
                             umma_mxf4<PAIR>(tmem_base, rdesc + (uint64_t)(2 * k4), bdesc + (uint64_t)(2 * k4), idesc,
                                             sf + 8 + ka * 4 + (sfid << 30), sfb, 1u);
@@ -311,9 +328,12 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                 if (n < p.N) vw[j] = *reinterpret_cast<const uint2*>(p.w_scale + n * spr + kb * 8);
             }
         };
-        int tile = worker, kb = 0;
-        if (tile < p.num_tiles) load_scales(tile, kb);
-        while (tile < p.num_tiles && ok) {
+        int item = worker, tile = 0, sp = 0, kb = 0, kb1 = 0;
+        if (item < nitems) {
+            item_of(item, tile, sp, kb, kb1);
+            load_scales(tile, kb);
+        }
+        while (item < nitems && ok) {
             if (!ptx::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) {
                 report_timeout_native(p.status, 3);
                 ok = false;
@@ -347,18 +367,25 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                 else ptx::mbar_arrive(&full[s]);
             }
             if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
-            if (++kb == nkb) {
-                kb = 0;
-                tile += nworkers;
+            if (++kb == kb1) {
+                item += nworkers;
+                if (item < nitems) item_of(item, tile, sp, kb, kb1);
             }
-            if (tile < p.num_tiles) load_scales(tile, kb);  // in flight while the next slot is awaited
+            if (item < nitems) load_scales(tile, kb);  // in flight while the next slot is awaited
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 4..7)
         const int quad = warp & 3;
         int local_tile = 0;
-        for (int tile = worker; tile < p.num_tiles; tile += nworkers, ++local_tile) {
+        for (int item = worker; item < nitems; item += nworkers, ++local_tile) {
+            int tile, sp, kb0, kb1;
+            item_of(item, tile, sp, kb0, kb1);
             const int64_t m0 = (int64_t)(tile / p.ntiles_n) * kTileM + rank * kBM, n0 = (int64_t)(tile % p.ntiles_n) * kBN;
+            // (a K split writes fp32 partial tiles into the slab of its split)
+            const bool part = p.splits > 1;
+            void* const out = part ? static_cast<void*>(p.partials + (size_t)sp * (size_t)p.M * (size_t)p.N) : p.Y;
+            const int64_t ldo = part ? p.N : p.ldy;
+            const bool f32 = part || p.out_f32;
             if (!ptx::mbar_wait(acc_full, (uint32_t)(local_tile & 1), abort_flag)) {
                 report_timeout_native(p.status, 4);
                 break;
@@ -379,8 +406,8 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                 const int64_t nb = n0 + cc * 32;
                 const int64_t left = p.N - nb;
                 if (left <= 0) continue;
-                if (p.out_f32) {
-                    float* dst = reinterpret_cast<float*>(p.Y) + m * p.ldy + nb;
+                if (f32) {
+                    float* dst = reinterpret_cast<float*>(out) + m * ldo + nb;
                     if (left >= 32) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
@@ -391,7 +418,7 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                             if (j < left) dst[j] = __uint_as_float(v[j]);
                     }
                 } else {
-                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.Y) + m * p.ldy + nb;
+                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(out) + m * ldo + nb;
                     if (left >= 32) {
                         uint32_t o[16];
 #pragma unroll
@@ -421,6 +448,22 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     }
 }
 
+// K split of a decode-sized call with a long K range: enough (tile, split) items to give every SM one, at least two stages
+// of 256 values per split, as many slabs as fit into the scratch (down projections at M = 256 / 512: 39.6 -> 29.0 us and
+// 88.8 -> 66.2 us with the reduce launch).  RESQ_MXFP4_SPLITS is the debugging override.
+int native_splits(int64_t M, int64_t N, int64_t K, size_t partial_bytes) {
+    const int nkb = (int)(K / kBKe);
+    const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
+    int64_t want = std::min<int64_t>(148 / std::max<int64_t>(1, tiles), nkb / 2);
+    want = std::min<int64_t>(want, (int64_t)(partial_bytes / ((size_t)M * (size_t)N * 4)));
+    want = std::min<int64_t>(want, 16);
+    if (nkb < 16) want = 1;  // short K ranges: the second launch costs what the split saves (qkv at M = 256: 18.9 -> 28.8 us)
+    want = env_int("RESQ_MXFP4_SPLITS", (int)want);
+    if (want < 2 || (N & 3) != 0 || (size_t)want * (size_t)M * (size_t)N * 4 > partial_bytes) return 1;
+    const int per = (nkb + (int)want - 1) / (int)want;
+    return (nkb + per - 1) / per;  // (no empty split)
+}
+
 template <bool RES, bool PAIR>
 int launch_native_variant(const Mxfp4NativeArgs& g, cudaStream_t stream) {
     using L = StageLayout<RES, PAIR>;
@@ -444,6 +487,9 @@ int launch_native_variant(const Mxfp4NativeArgs& g, cudaStream_t stream) {
     p.K = g.K;
     p.ntiles_n = (int)((g.N + kBN - 1) / kBN);
     p.num_tiles = (int)((g.M + kTileM - 1) / kTileM) * p.ntiles_n;
+    p.splits = (!PAIR && g.partials) ? native_splits(g.M, g.N, g.K, g.partial_bytes) : 1;
+    p.kb_per_split = ((int)(g.K / kBKe) + p.splits - 1) / p.splits;
+    p.partials = g.partials;
     p.Y = g.Y;
     p.out_f32 = g.out_dtype == RESQ_OUT_F32;
     p.ldy = g.ldy;
@@ -454,12 +500,25 @@ int launch_native_variant(const Mxfp4NativeArgs& g, cudaStream_t stream) {
     rc = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem_bytes, "cudaFuncSetAttribute(gemm mxfp4)");
     if (rc) return rc;
     const int num_sms = device_sm_count();
-    LaunchScope scope(kKindGemm, stream);
     if constexpr (!PAIR) {
-        const unsigned grid = (unsigned)std::min(p.num_tiles, num_sms);
-        return cuda_fail(launch_kernel(kern, dim3(grid), dim3(kThreadsNative), (size_t)smem_bytes, stream, ta, tr, tw, p),
-                         "gemm_mxfp4_native_kernel launch");
+        const unsigned grid = (unsigned)std::min(p.num_tiles * p.splits, num_sms);
+        {
+            LaunchScope scope(kKindGemm, stream);
+            rc = cuda_fail(launch_kernel(kern, dim3(grid), dim3(kThreadsNative), (size_t)smem_bytes, stream, ta, tr, tw, p),
+                           "gemm_mxfp4_native_kernel launch");
+        }
+        if (rc || p.splits == 1) return rc;
+        GemmArgs red;  // the fixed-order sum of the slabs (the reduce kernel of the bf16 route)
+        memset(&red, 0, sizeof(red));
+        red.splitk_partials = g.partials;
+        red.M = g.M;
+        red.N = g.N;
+        red.Y = g.Y;
+        red.out_dtype = g.out_dtype;
+        red.ldy = g.ldy;
+        return launch_splitk_reduce(red, p.splits, stream);
     } else {
+        LaunchScope scope(kKindGemm, stream);
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof(cfg));
         cfg.gridDim = dim3((unsigned)(2 * std::min(p.num_tiles, num_sms / 2)), 1, 1);
@@ -490,7 +549,11 @@ bool gemm_mxfp4_native_supported(int64_t M, int64_t N, int64_t K, bool res) {
     // route splits K for decode-sized calls; its time is about 15 us plus the executed flops at 1 PFLOP/s.
     // (Both fitted to the layer shapes of the 3B / 7B configurations at M = 256 ... 16384.)
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
-    const double t_native = 8.0 + (double)((tiles + 147) / 148) * (double)(K / kBKe) * 1.1;
+    const int splits = native_splits(M, N, K, gemm_hif4_scratch_bytes(M, N, K));
+    const int per = ((int)(K / kBKe) + splits - 1) / splits;
+    // (a K split adds the reduce launch and the traffic of its slabs)
+    const double t_native = 8.0 + (double)((tiles * splits + 147) / 148) * (double)per * 1.1 +
+                            (splits > 1 ? 4.0 + (double)splits * (double)M * (double)N * 4.0 / 3.0e6 : 0.0);
     const double t_bf16 = 15.0 + 2.0 * (double)M * (double)N * (double)K * (res ? 2.0 : 1.0) / 1.0e9;
     return t_native < t_bf16;
 }

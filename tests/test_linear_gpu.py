@@ -744,3 +744,19 @@ def test_block_selection_through_keep_flags(case, fmt, monkeypatch):
     assert torch.equal(y, y_masked)  # same operands, same order of accumulation
     monkeypatch.setenv("RESQ_BLOCK_LISTS", "1")
     run_case(xb, wb, pattern, fmt=fmt, out_dtype=torch.bfloat16)
+
+
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_2_4, oracle.S_ROW50])
+@pytest.mark.parametrize("case", [(288, 1024, 1000, "3"), (200, 2304, 520, "4"), (256, 2048, 2560, None), (64, 11008, 2048, None)],
+                         ids=["two-splits", "three-uneven-splits", "decode-auto", "long-k-auto"])
+def test_mxfp4_fp4_route_with_a_k_split(case, pattern, monkeypatch):
+    """Decode-sized calls of the block-scaled FP4 route: (tile, K split) work items, fp32 partial slabs, fixed-order sum."""
+    M, K, N, splits = case
+    monkeypatch.setenv("RESQ_MXFP4_NATIVE", "1")
+    if splits:
+        monkeypatch.setenv("RESQ_MXFP4_SPLITS", splits)
+    xb, wb = synth_xw(5 * M + N + pattern, M, K, N, n_out=max(1, K // 256))
+    y = run_case(xb, wb, pattern, fmt="mxfp4")
+    y2 = run_case(xb, wb, pattern, fmt="mxfp4")
+    assert torch.equal(y, y2)
+    run_case(xb, wb, pattern, fmt="mxfp4", out_dtype=torch.bfloat16)
