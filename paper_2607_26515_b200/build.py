@@ -8,7 +8,7 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libresq.so")
-SOURCES = ["api.cu", "quantize.cu", "gemm_hif4.cu", "gemm_pair.cu", "gemm_mxfp4.cu", "static_scratch.cu"]
+SOURCES = ["api.cu", "quantize.cu", "gemm_hif4.cu", "gemm_pair.cu", "gemm_mxfp4.cu", "gemm_decode.cu", "static_scratch.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",

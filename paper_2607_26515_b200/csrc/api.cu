@@ -616,6 +616,7 @@ int linear_group(int fmt, const resq_problem* pr, int count, int pattern, int ou
     }
     rc = launch_quantize_group(fmt, qa, count, st);
     if (rc) return rc;
+    if (gemm_decode_supported(ga, count)) return launch_gemm_decode(ga, count, st);
     return launch_gemm_pair_group(ga, count, st);
 }
 

@@ -186,6 +186,11 @@ int launch_gemm_hif4(const GemmArgs& g, cudaStream_t stream);
 // the K-streamed schedule; status word, arrival counters and partial-tile slots are those of g[0] (gemm_pair.cu).
 int launch_gemm_pair_group(const GemmArgs* g, int count, cudaStream_t stream);
 size_t gemm_pair_streamk_scratch_bytes();
+// Decode-sized calls (every M <= 64): one launch with the weights as the MMA's M dimension and the tokens as its N
+// (gemm_decode.cu).  The problems share format, residual mode (none or the dense image), output type, and the status word,
+// arrival counters (kWsFlags zeroed bytes) and partial-tile scratch of g[0].
+bool gemm_decode_supported(const GemmArgs* g, int count);
+int launch_gemm_decode(const GemmArgs* g, int count, cudaStream_t stream);
 // Test hook behind resq_debug_expire_next_wait (gemm_pair.cu).
 void debug_expire_next_wait(int on);
 // Whether launch_gemm_hif4 takes the keep flags of the block-wise selection for this shape (see GemmArgs::blk_flags).

@@ -614,6 +614,13 @@ GROUPS = {
     "two-classes": ([(256, 512, 25600), (256, 25600, 1024)], oracle.S_2_4, "hif4", torch.bfloat16),
     # prefill-sized problems: several rounds of whole tiles, rows beyond one M tile
     "tall": ([(2048, 1024, 4096), (1024, 4096, 1024)], oracle.S_DENSE, "hif4", torch.bfloat16),
+    # at most 64 token rows everywhere: the decode kernel (weights as the MMA's M dimension, tokens as its N); tiles whose K
+    # range is shared by several CTAs, ragged N, token counts that are not multiples of 16
+    "decode-block": ([(16, 2048, 2560), (16, 2048, 2048), (16, 2048, 4352), (16, 11008, 2048)], oracle.S_2_4, "hif4", torch.bfloat16),
+    "decode-ragged": ([(40, 1024, 520), (64, 512, 1000), (7, 2048, 264)], oracle.S_DENSE, "hif4", torch.float32),
+    "decode-plain": ([(33, 704, 328), (48, 4160, 96)], oracle.S_NONE, "hif4", torch.float32),
+    "decode-three-quarters": ([(24, 1024, 384), (64, 2048, 136)], oracle.keep_quarters(oracle.S_2_4, 3), "mxfp4", torch.float32),
+    "decode-one": ([(64, 2048, 2048)], oracle.S_2_4, "mxfp4", torch.bfloat16),
 }
 
 
@@ -760,3 +767,24 @@ def test_mxfp4_fp4_route_with_a_k_split(case, pattern, monkeypatch):
     y2 = run_case(xb, wb, pattern, fmt="mxfp4")
     assert torch.equal(y, y2)
     run_case(xb, wb, pattern, fmt="mxfp4", out_dtype=torch.bfloat16)
+
+
+@pytest.mark.parametrize("fmt", ["hif4", "mxfp4"])
+@pytest.mark.parametrize("pattern", [oracle.S_NONE, oracle.S_DENSE, oracle.S_2_4])
+@pytest.mark.parametrize("shape", [(16, 2048, 2048), (32, 64, 16), (7, 192, 80), (32, 4160, 96), (24, 704, 328), (1, 1024, 1000)])
+def test_decode_kernel_on_single_problems(shape, pattern, fmt):
+    """Groups of one problem with at most 32 token rows run on the decode kernel (128 weight rows per tile as the MMA's M
+    dimension, K ranges cut evenly over the CTAs, last arrival sums a tile): one k-block, ragged N, long K, a single row."""
+    m = rq()
+    M, K, N = shape
+    xb, wb = synth_xw(7 * M + N + pattern, M, K, N, n_out=max(1, K // 256))
+    want = oracle.resq_linear(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), pattern, fmt)
+    wc, ws = m.pack_weight(to_dev(wb), fmt)
+    problems = [(to_dev(xb), wc, ws)]
+    for out_dtype in (torch.float32, torch.bfloat16):
+        work = m.alloc_workspace(m.resq_group_workspace_bytes(problems, pattern, fmt, out_dtype))
+        (y,) = m.resq_linear_group(problems, pattern, fmt, out_dtype=out_dtype, workspace=work)
+        assert m.check(work) == 0, m.last_error()
+        (y2,) = m.resq_linear_group(problems, pattern, fmt, out_dtype=out_dtype, workspace=work)
+        assert torch.equal(y, y2)
+        check_close(y.float().cpu().numpy(), want["y"], want["abs_sum"], bf16_out=out_dtype == torch.bfloat16)
