@@ -5,8 +5,8 @@
 // of the MMA (tcgen05.mma.cta_group::1.kind::f16, M = 128), and the token rows (rounded up to 16) are its N dimension; the
 // rows of the residual operand follow those of the main image in shared memory, so one MMA over N = 2 x tokens accumulates
 // both terms side by side and the epilogue adds them.  The accumulator is 128 lanes x (2) M columns and a partial tile is
-// M x 128 floats.  What bounds it: an MMA costs about 190 cycles at these sizes whatever N is (the read of its 128 x 32-byte
-// weight operand), four per k-block, next to about 570 cycles in which the sixteen expander warps expand a k-block.
+// M x 128 floats.  What bounds it is the integer pipe (two cycles per warp instruction): about 30 instructions per 8 weights
+// of expansion, and whatever else the loops execute next to them.
 //
 // Pipeline: a stage is a "quad" of four consecutive k-blocks -- one wait, one proxy fence and one arrive per quad and warp,
 // one commit per quad.  (With one k-block per stage the loop runs at the latency of a warp's wait -> expand -> fence ->
@@ -180,7 +180,9 @@ gemm_decode_kernel(const __grid_constant__ DecMaps maps, const __grid_constant__
         // the raw quad is a 128-byte-swizzled tile [128 rows][4 k-blocks x 32 bytes]: this thread's 8 bytes of k-block s
         // are in the logical 16-byte chunk 2 s + ch0 / 4
         const uint32_t rd_row = (uint32_t)(row * 128 + (ch0 & 3) * 4);
-        uint32_t qi = 0;  // quad counter
+        // The integer pipe is what this loop runs on (two cycles per warp instruction): everything but the expansion itself
+        // is kept out of it -- ring indices and phases advance by additions, the metadata pointer by a constant.
+        uint32_t st = 0, st_ph = 0, sr = 0, sr_ph = 0;  // stage of the expanded / token rings and its phase; same for the raw ring
         bool ok = true;
         DecIter di(p, cta, nctas);
         DecSeg sg;
@@ -188,33 +190,35 @@ gemm_decode_kernel(const __grid_constant__ DecMaps maps, const __grid_constant__
             const DecProblem& pb = p.pr[sg.prob];
             const int64_t n = (int64_t)sg.n0 + row;
             const bool row_ok = n < pb.N;
-            const int64_t G = pb.G;
-            const void* w_side = pb.w_side;
-            auto load_side = [&](int kb) -> uint32_t {
-                if (!row_ok || kb >= (int)G) return 0u;
-                if (FMT == kHiF4) return ptx::ld_nc_u32(reinterpret_cast<const uint32_t*>(w_side) + n * G + kb);
-                return ptx::ld_nc_u16(reinterpret_cast<const uint16_t*>(w_side) + n * G + kb);
+            const int G = pb.G;
+            // metadata words of this thread's row, from the segment's first k-block on (rows past N read row 0 and are never stored)
+            const uint8_t* side = static_cast<const uint8_t*>(pb.w_side) + ((row_ok ? n : 0) * (int64_t)G + sg.kb0) * (FMT == kHiF4 ? 4 : 2);
+            const int kb_left = G - sg.kb0;  // k-blocks up to the end of the row
+            auto load_quad = [&](int first, uint32_t (&m)[kDecQuad]) {
+#pragma unroll
+                for (int s = 0; s < kDecQuad; ++s) {
+                    if (first + s < kb_left) {
+                        if (FMT == kHiF4) m[s] = ptx::ld_nc_u32(reinterpret_cast<const uint32_t*>(side) + first + s);
+                        else m[s] = ptx::ld_nc_u16(reinterpret_cast<const uint16_t*>(side) + first + s);
+                    } else {
+                        m[s] = 0u;
+                    }
+                }
             };
             const int nq = (sg.nkb + kDecQuad - 1) / kDecQuad;
             // the metadata words of a quad are fetched while the previous quad is expanded
             uint32_t mn[kDecQuad];
-#pragma unroll
-            for (int s = 0; s < kDecQuad; ++s) mn[s] = load_side(sg.kb0 + s);
-            for (int j = 0; j < nq; ++j, ++qi) {
+            load_quad(0, mn);
+            for (int j = 0; j < nq; ++j) {
                 uint32_t mw[kDecQuad];
 #pragma unroll
                 for (int s = 0; s < kDecQuad; ++s) mw[s] = mn[s];
-                if (j + 1 < nq) {
-#pragma unroll
-                    for (int s = 0; s < kDecQuad; ++s) mn[s] = load_side(sg.kb0 + (j + 1) * kDecQuad + s);
-                }
+                if (j + 1 < nq) load_quad((j + 1) * kDecQuad, mn);
                 const int valid = min(kDecQuad, sg.nkb - j * kDecQuad);
-                const uint32_t st = qi & 1u, sr = qi % (uint32_t)SR;
                 // one lane polls the two barriers for its warp
                 int got = 1;
                 if (lane == 0)
-                    got = (ptx::mbar_wait_spin(&q_empty[st], ((qi >> 1) & 1u) ^ 1u, abort_flag) &&
-                           ptx::mbar_wait_spin(&r_full[sr], (qi / (uint32_t)SR) & 1u, abort_flag)) ? 1 : 0;
+                    got = (ptx::mbar_wait_spin(&q_empty[st], st_ph ^ 1u, abort_flag) && ptx::mbar_wait_spin(&r_full[sr], sr_ph, abort_flag)) ? 1 : 0;
                 ok = __shfl_sync(0xFFFFFFFFu, got, 0) != 0;
                 if (!ok) {
                     dec_timeout(p.status, 3);
@@ -248,6 +252,12 @@ gemm_decode_kernel(const __grid_constant__ DecMaps maps, const __grid_constant__
                 if (lane == 0) {
                     ptx::mbar_arrive(&e_full[st]);
                     ptx::mbar_arrive(&r_empty[sr]);
+                }
+                st ^= 1u;
+                if (st == 0) st_ph ^= 1u;
+                if (++sr == (uint32_t)SR) {
+                    sr = 0;
+                    sr_ph ^= 1u;
                 }
             }
         }
@@ -312,6 +322,10 @@ gemm_decode_kernel(const __grid_constant__ DecMaps maps, const __grid_constant__
             // accumulates the two terms side by side, and the epilogue adds them -- half as many instructions, each of
             // which costs the read of its 128 x 32-byte weight operand whatever N is.
             const uint32_t idesc = ptx::idesc_bf16_f32(kDecRows, RES ? 2 * ntok : ntok);
+            const uint64_t desc0 = ptx::smem_desc_sw128_kmajor(0);  // everything but the start address
+            const uint32_t w16 = (ptx::smem_u32(ring_e) & 0x3FFFFu) >> 4, t16 = (ptx::smem_u32(ring_a) & 0x3FFFFu) >> 4;
+            const uint32_t a_quad16 = (uint32_t)(a_quad >> 4);
+            const uint64_t a_stage16 = (uint64_t)(p.a_stage >> 4);
             uint32_t qi = 0;
             int lt = 0;
             bool ok = true;
@@ -337,14 +351,26 @@ gemm_decode_kernel(const __grid_constant__ DecMaps maps, const __grid_constant__
                     }
                     ptx::tc_fence_after();
                     const int valid = min(kDecQuad, sg.nkb - j * kDecQuad);
-                    const uint32_t w_addr = ptx::smem_u32(ring_e + (size_t)st * kDecExpQuad);
-                    const uint32_t t_addr = ptx::smem_u32(ring_a + (size_t)st * a_quad);
-                    for (int s = 0; s < valid; ++s) {
+                    // This thread shares its scheduler with four expander warps: its instruction stream is kept short
+                    // (descriptors advance by additions; a full quad is sixteen MMAs without a branch in between).
+                    uint64_t wd = desc0 + (uint64_t)(w16 + st * (uint32_t)(kDecExpQuad >> 4));
+                    uint64_t td = desc0 + (uint64_t)(t16 + st * a_quad16);
+                    if (valid == kDecQuad) {
 #pragma unroll
-                        for (int k = 0; k < kBK / 16; ++k) {
-                            const uint64_t wdesc = ptx::smem_desc_sw128_kmajor(w_addr + s * kDecExpStage + k * 32);
-                            const uint32_t tk = t_addr + s * p.a_stage + k * 32;
-                            ptx::umma_bf16(d, wdesc, ptx::smem_desc_sw128_kmajor(tk), idesc, (j > 0 || s > 0 || k > 0) ? 1u : 0u);
+                        for (int s = 0; s < kDecQuad; ++s) {
+#pragma unroll
+                            for (int k = 0; k < kBK / 16; ++k)
+                                ptx::umma_bf16(d, wd + (uint64_t)((s * kDecExpStage + k * 32) >> 4), td + (uint64_t)(2 * k), idesc,
+                                               (j > 0 || s > 0 || k > 0) ? 1u : 0u);
+                            td += a_stage16;
+                        }
+                    } else {
+                        for (int s = 0; s < valid; ++s) {
+#pragma unroll
+                            for (int k = 0; k < kBK / 16; ++k)
+                                ptx::umma_bf16(d, wd + (uint64_t)(2 * k), td + (uint64_t)(2 * k), idesc, (j > 0 || s > 0 || k > 0) ? 1u : 0u);
+                            wd += (uint64_t)(kDecExpStage >> 4);
+                            td += a_stage16;
                         }
                     }
                     ptx::umma_commit(&q_empty[st]);  // frees the token quad and the expanded quad
