@@ -185,8 +185,11 @@ RESQ_API int mxfp4_resq_linear(const void* X_bf16, int64_t M, int64_t K, int64_t
  * another (the q/k/v, gate and up projections of a block, the experts of a mixture, the layers of several models)
  * runs as ONE quantizer launch and ONE GEMM launch whose CTA pairs walk the output tiles of all problems: whole tiles
  * first, the k-blocks of the remaining tiles dealt out evenly, partial tiles summed in a fixed order inside the kernel
- * (bit-identical results run to run).  Each problem is exactly *_resq_linear: same quantizer, residual and selection,
- * results within the same tolerance (the fp32 summation order over K differs from the single call's).
+ * (bit-identical results run to run).  A group whose problems all have at most 32 token rows takes a kernel of its own:
+ * 128 weight rows are the M dimension of the MMA and the tokens its N, the (tile, k-block) units of all problems are cut
+ * into equal ranges, one per CTA, and the last CTA to finish a tile adds its partial tiles in k order (no CTA waits for
+ * another there).  Each problem is exactly *_resq_linear: same quantizer, residual and selection, results within the same
+ * tolerance (the fp32 summation order over K differs from the single call's).
  *   - `problems` is a HOST array read during the call; its tensor pointers are device pointers with the alignment
  *     rules of *_resq_linear; M, N, K may differ from problem to problem; any M >= 1.
  *   - pattern: RESQ_S_NONE, RESQ_S_DENSE or RESQ_S_2_4 (with RESQ_KEEP_QUARTERS), one for the whole group; the
