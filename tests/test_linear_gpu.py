@@ -621,6 +621,8 @@ GROUPS = {
     "decode-plain": ([(33, 704, 328), (48, 4160, 96)], oracle.S_NONE, "hif4", torch.float32),
     "decode-three-quarters": ([(24, 1024, 384), (64, 2048, 136)], oracle.keep_quarters(oracle.S_2_4, 3), "mxfp4", torch.float32),
     "decode-one": ([(64, 2048, 2048)], oracle.S_2_4, "mxfp4", torch.bfloat16),
+    # the 7B block's layers (gate_up narrowed for the oracle's sake) at 24 tokens: long K ranges shared by many CTAs
+    "decode-7b": ([(24, 3584, 4608), (24, 3584, 3584), (24, 3584, 4736), (24, 18944, 3584)], oracle.S_2_4, "hif4", torch.bfloat16),
 }
 
 
