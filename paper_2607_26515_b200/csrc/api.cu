@@ -560,8 +560,8 @@ int linear_group(int fmt, const resq_problem* pr, int count, int pattern, int ou
     QuantArgs qa[kMaxQuantGroup];
     GemmArgs ga[kMaxQuantGroup];
     size_t used = kWsHeader + kWsFlags;
-    bool sparse24 = pattern == RESQ_S_2_4 && quarters == 2;
-    for (int i = 0; i < count && sparse24; ++i) sparse24 = gemm_sparse24_supported(256, pr[i].N, pr[i].K);
+    // (the residual operand of a group is the dense masked image: the compressed 2:4 form pays from a few thousand token
+    // rows on, which is not what groups are for)
     for (int i = 0; i < count; ++i) {
         QuantArgs& a = qa[i];
         memset(&a, 0, sizeof(a));
@@ -581,14 +581,7 @@ int linear_group(int fmt, const resq_problem* pr, int count, int pattern, int ou
         if (pattern != RESQ_S_NONE) {
             uint8_t* region_r = ws + used;
             used += residual_region_bytes(a.M, a.K, pattern);
-            if (sparse24) {
-                a.r_comp = reinterpret_cast<__nv_bfloat16*>(region_r);
-                a.r_meta = region_r + align_up((size_t)a.M * (size_t)a.K, 256);
-                a.meta_rows128 = sparse24_rows128(a.M);
-                a.meta_ka = sparse24_ka(a.K);
-            } else {
-                a.r_bf16 = reinterpret_cast<__nv_bfloat16*>(region_r);
-            }
+            a.r_bf16 = reinterpret_cast<__nv_bfloat16*>(region_r);
         }
     }
     for (int i = 0; i < count; ++i) {

@@ -1365,7 +1365,9 @@ int group_fmt(const GemmArgs* g, int count, cudaStream_t stream) {
     // is the debugging override
     const bool four = env_int("RESQ_GEMM_GROUPS", 4) == 4;
     switch (res_mode(g[0])) {
-        case kResSparse24: return four ? launch_pair_group<kResSparse24, FMT, 4>(g, count, stream) : launch_pair_group<kResSparse24, FMT, 3>(g, count, stream);
+        case kResSparse24:
+            set_last_error("internal: a group takes the dense residual image");
+            return RESQ_ERR_CUDA;
         case kResDense: return four ? launch_pair_group<kResDense, FMT, 4>(g, count, stream) : launch_pair_group<kResDense, FMT, 3>(g, count, stream);
         default: return four ? launch_pair_group<kResNone, FMT, 4>(g, count, stream) : launch_pair_group<kResNone, FMT, 3>(g, count, stream);
     }
