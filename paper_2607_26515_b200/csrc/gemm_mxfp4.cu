@@ -245,6 +245,7 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         if (lane == 0 && rank == 0) {
             const uint64_t desc0 = ptx::smem_desc_sw128_kmajor(0);
             const uint32_t smem_base16 = (ptx::smem_u32(smem) & 0x3FFFFu) >> 4;
+            const uint64_t sf_desc0 = smem_desc_sf(0);  // everything but the start address
             uint32_t s = 0, ph = 0, it = 0;
             int local_tile = 0;
             bool ok = true;
@@ -263,16 +264,17 @@ gemm_mxfp4_native_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                         break;
                     }
                     ptx::tc_fence_after();
-                    const uint32_t st = ptx::smem_u32(smem) + s * (uint32_t)L::kBytes;
+                    // (this thread's instruction stream sits between the MMAs of consecutive stages: descriptors by additions)
+                    const uint64_t sfd = sf_desc0 + (uint64_t)(smem_base16 + s * (uint32_t)(L::kBytes >> 4));
                     // scales of this stage -> tensor memory (two column sets alternate between stages)
                     const uint32_t sf = tmem_base + (uint32_t)(kAccCols + (it & 1u) * kSfSetCols);
 #pragma unroll
                     for (int ka = 0; ka < 2; ++ka) {
-                        tmem_cp_sf<PAIR>(sf + ka * 4, smem_desc_sf(st + L::kSfAOff + ka * kSfAtom));
-                        if (RES) tmem_cp_sf<PAIR>(sf + 8 + ka * 4, smem_desc_sf(st + L::kSfArOff + ka * kSfAtom));
+                        tmem_cp_sf<PAIR>(sf + ka * 4, sfd + (uint64_t)((L::kSfAOff + ka * kSfAtom) >> 4));
+                        if (RES) tmem_cp_sf<PAIR>(sf + 8 + ka * 4, sfd + (uint64_t)((L::kSfArOff + ka * kSfAtom) >> 4));
 #pragma unroll
                         for (int nb = 0; nb < 2; ++nb)
-                            tmem_cp_sf<PAIR>(sf + 16 + ka * 8 + nb * 4, smem_desc_sf(st + L::kSfBOff + (ka * 2 + nb) * kSfAtom));
+                            tmem_cp_sf<PAIR>(sf + 16 + ka * 8 + nb * 4, sfd + (uint64_t)((L::kSfBOff + (ka * 2 + nb) * kSfAtom) >> 4));
                     }
                     const uint32_t st16 = smem_base16 + s * (uint32_t)(L::kBytes >> 4);
                     const uint64_t adesc = desc0 + (uint64_t)(st16 + (L::kA >> 4));
