@@ -2034,13 +2034,13 @@ int launch_quantize_group(int fmt, const QuantArgs* a_in, int count, cudaStream_
     memset(&g, 0, sizeof(g));
     g.count = count;
     const int pattern = a_in[0].pattern;
-    const bool residual = pattern != RESQ_S_NONE, comp = a_in[0].r_comp != nullptr;
+    const bool residual = pattern != RESQ_S_NONE;
     int blocks = 0;
     for (int i = 0; i < count; ++i) {
         QuantArgs a = a_in[i];
         if (a.keep_quarters < 1 || a.keep_quarters > 3) a.keep_quarters = 2;
         if (a.pattern != pattern || (pattern != RESQ_S_NONE && pattern != RESQ_S_DENSE && pattern != RESQ_S_2_4) || !a.a_bf16 ||
-            (a.r_comp != nullptr) != comp || a.X_up || a.gamma || a.rht || (comp && a.keep_quarters != 2)) {
+            a.r_comp || a.X_up || a.gamma || a.rht) {
             set_last_error("internal: a quantizer group takes one row-local pattern and the GEMM operand images");
             return RESQ_ERR_CUDA;
         }
@@ -2053,12 +2053,8 @@ int launch_quantize_group(int fmt, const QuantArgs* a_in, int count, cudaStream_
     }
     for (int i = count; i <= kMaxQuantGroup; ++i) g.block_base[i] = blocks;
     void (*kern)(QuantGroup);
-    if (fmt == kHiF4)
-        kern = residual ? (comp ? quant_stream_group_kernel<kHiF4, true, true, true> : quant_stream_group_kernel<kHiF4, true, true, false>)
-                        : quant_stream_group_kernel<kHiF4, false, true, false>;
-    else
-        kern = residual ? (comp ? quant_stream_group_kernel<kMXFP4, true, true, true> : quant_stream_group_kernel<kMXFP4, true, true, false>)
-                        : quant_stream_group_kernel<kMXFP4, false, true, false>;
+    if (fmt == kHiF4) kern = residual ? quant_stream_group_kernel<kHiF4, true, true, false> : quant_stream_group_kernel<kHiF4, false, true, false>;
+    else kern = residual ? quant_stream_group_kernel<kMXFP4, true, true, false> : quant_stream_group_kernel<kMXFP4, false, true, false>;
     LaunchScope scope(kKindQuant, stream);
     return cuda_fail(launch_kernel(kern, dim3((unsigned)blocks), dim3(kThreads), 0, stream, g), "quant_stream_group_kernel launch");
 }
